@@ -1,0 +1,339 @@
+#!/usr/bin/env python
+"""Benchmark of the MDN chunkwise forward (one "step" = one mdn_chunk_fwd call = the whole hot
+path: chunk map, coefficient scan, intra-chunk solve, inter-chunk propagation, output).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 2] [--impl ours|reference]
+
+Prints ONE JSON line.  Metric: tokens/s of the forward on the 1.3B-layer-shaped workload
+(B=8, H=16, T=4096, dk=dv=128, bf16), inputs resident in HBM.  N > 1 (torchrun): every rank
+runs its own batch of the same shape (batches are independent: no data-path collective);
+value = all ranks' tokens / max-over-ranks time ("weak" scaling).
+
+`--impl reference` times the fp64 CPU oracle (the only CPU code in this repository) on a
+bounded sample of the same workload; it is a deliberately slow program, reported for context.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import mdn_workloads as wl  # noqa: E402
+
+METRIC = "MDN chunkwise fwd tokens/s"
+UNIT = "tokens/s"
+BYTES_PER_HEAD_TOKEN_BF16 = 1040      # q,k,v read + o written (bf16, d=128) + four fp32 gates
+L2_BYTES = 126e6
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return dict(hbm_gbs=float(d["hbm_gbs"]), bf16_tflops=float(d["bf16_tflops"]),
+                    bf16_tflops_sustained=float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+def workload_desc(w: wl.Workload) -> str:
+    kind = "packed varlen" if w.varlen else "fixed length"
+    return "%s: B=%d,H=%d,T=%d,dk=%d,dv=%d,%s,chunk=64,%s" % (w.name, w.B, w.H, w.T, w.dk, w.dv, w.dtype, kind)
+
+
+def algorithmic_bytes(w: wl.Workload, n_state: int, has_init: bool) -> float:
+    es = 2 if w.dtype == "bf16" else 4
+    per_ht = es * (2 * w.dk + 2 * w.dv) + 16
+    states = n_state * w.H * w.dk * w.dv * 4 * (2 + (2 if has_init else 0))
+    return float(w.B * w.T * w.H * per_ht + states)
+
+
+def algorithmic_flops(w: wl.Workload) -> float:
+    return float(w.B * w.T * w.H) * (12 * w.dk * w.dv + 4 * 64 * (w.dk + w.dv))
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples during the timed region (reading only)."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", "-i", str(index), "--query-gpu=" + self.Q,
+                                       "--format=csv,noheader,nounits", "-lms", "50"],
+                                      stdout=self.f, stderr=subprocess.DEVNULL)
+        except OSError:
+            pass
+
+    def stop(self):
+        out = dict(sm_mhz=None, sm_max_mhz=None, reasons=[], samples=0)
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.f.read().splitlines():
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        self.f.close()
+        os.unlink(self.f.name)
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def oracle_sample_tokens_per_s(w: wl.Workload, inp, target_s: float):
+    """Times the oracle as it stands on a subset of (sequence, head) chains of this workload.
+    Returns (tokens/s, threads, description, seconds)."""
+    import oracle
+    N = len(inp["seq_len"])
+    total = N * w.H
+    rng = np.random.default_rng(0)
+    order = rng.permutation(total)
+
+    def run(chains):
+        t0 = time.perf_counter()
+        oracle.stepwise(inp["q"], inp["k"], inp["v"], inp["beta"], inp["log_alpha"], inp["log_mu"], inp["eta"],
+                        scale=inp["scale"], S0=inp["S0"], M0=inp["M0"], seq_start=inp["seq_start"],
+                        seq_len=inp["seq_len"], chains=chains)
+        return time.perf_counter() - t0
+
+    def head_tokens(chains):
+        return float(sum(int(inp["seq_len"][c // w.H]) for c in chains))
+
+    threads = oracle.num_threads()
+    probe = order[:min(total, max(threads, 4))]
+    t_probe = run(probe)
+    per_ht = t_probe / head_tokens(probe)
+    want = int(min(total, max(len(probe), target_s / max(per_ht, 1e-12) / (head_tokens(order) / total))))
+    chains = order[:want]
+    secs = run(chains)
+    ht = head_tokens(chains)
+    # a token is all H heads: tokens/s = head-tokens/s / H
+    return ht / w.H / secs, threads, "%d of %d (sequence, head) chains, %d head-tokens" % (len(chains), total, int(ht)), secs
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    inp = wl.make_inputs(w)
+    N = len(inp["seq_len"])
+    total = N * w.H
+    threads = oracle.num_threads()
+    chains = np.random.default_rng(0).permutation(total)[:min(total, 2 * max(threads, 4))]
+    ht = float(sum(int(inp["seq_len"][c // w.H]) for c in chains))
+
+    def step():
+        oracle.stepwise(inp["q"], inp["k"], inp["v"], inp["beta"], inp["log_alpha"], inp["log_mu"], inp["eta"],
+                        scale=inp["scale"], S0=inp["S0"], M0=inp["M0"], seq_start=inp["seq_start"],
+                        seq_len=inp["seq_len"], chains=chains)
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = time.perf_counter() - t0
+    value = ht / w.H * args.steps / dt
+    sample = "each step: %d of %d (sequence, head) chains = %d head-tokens" % (len(chains), total, int(ht))
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": workload_desc(w), "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+def run_ours(args, w):
+    import torch
+    import paper_2605_05838_b200 as mdn
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    from helpers import to_torch
+
+    mdn.lib()   # fail loudly if the CUDA library is missing
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    import dataclasses
+    wr = dataclasses.replace(w, seed=w.seed + rank)      # every rank its own batch
+    inp = wl.make_inputs(wr)
+    t = to_torch(inp, device="cuda:%d" % local)
+    o_dtype = torch.bfloat16 if w.dtype == "bf16" else torch.float32
+    N = len(inp["seq_len"])
+    p = mdn.make_params(t["q"], t["v"], num_seqs=(N if w.varlen else 0), scale=inp["scale"], o_dtype=o_dtype,
+                        path=args.path)
+    ws = torch.empty(mdn.workspace_bytes(p), dtype=torch.uint8, device=t["q"].device)
+    o = torch.empty((w.B, w.T, w.H, w.dv), dtype=o_dtype, device=t["q"].device)
+
+    def step():
+        return mdn.chunk_fwd(t["q"], t["k"], t["v"], t["beta"], t["log_alpha"], t["log_mu"], t["eta"],
+                             initial_S=t["initial_S"], initial_M=t["initial_M"], cu_seqlens=t["cu_seqlens"],
+                             scale=inp["scale"], o_dtype=o_dtype, path=args.path, workspace=ws, out=o)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    launches_per_step = mdn.last_launch_count()
+    barrier()
+    sampler = ClockSampler(local) if rank == 0 else None
+    stage_ev = [[torch.cuda.Event(enable_timing=True) for _ in range(mdn.NUM_STAGE_EVENTS)] for _ in range(args.steps)]
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for i in range(args.steps):
+        mdn.set_stage_events(stage_ev[i])
+        step()
+    mdn.set_stage_events(None)
+    ev1.record()
+    barrier()
+    elapsed_ms = ev0.elapsed_time(ev1)
+    clocks = sampler.stop() if sampler else None
+    if dist is not None:
+        tt = torch.tensor([elapsed_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(tt.item())
+    tokens_per_step = w.B * w.T * world
+    value = tokens_per_step * args.steps / (elapsed_ms * 1e-3)
+
+    # dominant kernel (the chain kernel: inter-chunk propagation + output), timed live
+    names = mdn.STAGE_NAMES
+    stage_ms = {names[s]: statistics.mean(stage_ev[i][s].elapsed_time(stage_ev[i][s + 1]) for i in range(args.steps))
+                for s in range(len(names))}
+    dom = max(stage_ms, key=stage_ms.get)
+    peaks = load_peaks()
+    abytes = algorithmic_bytes(w, N, t["initial_S"] is not None)
+    aflops = algorithmic_flops(w)
+    dom_s = stage_ms[dom] * 1e-3
+    achieved = abytes / dom_s / 1e9
+    roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
+                "kernel_ms": stage_ms[dom], "stage_ms": stage_ms,
+                "algorithmic_bytes": abytes, "algorithmic_flops": aflops,
+                "tensor_achieved_tflops": aflops / dom_s / 1e12,
+                "tensor_frac_of_burst_peak": aflops / dom_s / 1e12 / peaks["bf16_tflops"],
+                "whole_step_frac_hbm": abytes / (elapsed_ms / args.steps * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+    traffic_path = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(traffic_path):
+        tr = json.load(open(traffic_path)).get(w.name, {}).get(dom)
+        if tr:
+            roofline["traffic"] = tr
+
+    # end to end through the host-buffer entry point (pinned host memory, copies inside the timed region)
+    e2e = None
+    if rank == 0 or world > 1:
+        th = to_torch(inp, host_pinned=True)
+        arena = torch.empty(mdn.host_arena_bytes(p), dtype=torch.uint8, device=t["q"].device)
+        nst = N
+        out = (torch.empty((w.B, w.T, w.H, w.dv), dtype=o_dtype).pin_memory(),
+               torch.empty((nst, w.H, w.dk, w.dv), dtype=torch.float32).pin_memory(),
+               torch.empty((nst, w.H, w.dk, w.dv), dtype=torch.float32).pin_memory())
+
+        def e2e_step():
+            mdn.chunk_fwd_host(th["q"], th["k"], th["v"], th["beta"], th["log_alpha"], th["log_mu"], th["eta"],
+                               initial_S=th["initial_S"], initial_M=th["initial_M"], cu_seqlens=th["cu_seqlens"],
+                               scale=inp["scale"], o_dtype=o_dtype, path=args.path, arena=arena, out=out)
+
+        e2e_steps = max(2, min(args.steps, 5))
+        e2e_step()
+        barrier()
+        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a0.record()
+        for _ in range(e2e_steps):
+            e2e_step()
+        a1.record()
+        barrier()
+        e2e_ms = a0.elapsed_time(a1)
+        if dist is not None:
+            tt = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            e2e_ms = float(tt.item())
+        h2d = sum(x.numel() * x.element_size() for x in th.values() if x is not None)
+        d2h = sum(x.numel() * x.element_size() for x in out)
+        e2e = {"value": tokens_per_step * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps}
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        v, threads, desc, secs = oracle_sample_tokens_per_s(w, inp, target_s=args.cpu_seconds)
+        cpu = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc, "seconds": secs}
+
+    ws_in = abytes
+    print(json.dumps({
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if w.dtype == "bf16" else "f32",
+        "data": "synthetic",
+        "config": {"workload": workload_desc(w), "path": mdn.resolved_path(p),
+                   "parallelism": "independent batch per GPU, no collective",
+                   "l2": "inputs+outputs %.0f MB per step %s the 126 MB L2; no flush between steps"
+                         % (ws_in / 1e6, "exceed" if ws_in > L2_BYTES else "FIT IN")},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
+        "roofline": roofline, "cpu_baseline": cpu}))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", type=int, default=2, help="index into the named workloads (2 = headline)")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--path", default="auto", choices=["auto", "simt", "tensor"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    args = ap.parse_args()
+    w = wl.CONFIGS[args.config]
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()

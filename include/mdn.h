@@ -1,0 +1,183 @@
+/*
+ * libmdn: chunkwise-parallel forward of the stepwise-momentum delta-rule
+ * linear-attention recurrence (MDN), hand-written CUDA for sm_100a.
+ *
+ * The result is the one the token-by-token recurrence of Section 3.1 defines
+ * (Eq. 5-6, with the correction value v~_t = v_t - alpha_t S_{t-1}^T k_t):
+ *
+ *     M_t = mu_t M_{t-1} - eta_t k_t v~_t^T
+ *     S_t = alpha_t S_{t-1} - beta_t M_t
+ *     o_t = scale * S_t^T q_t            alpha_t = exp(log_alpha_t), mu_t = exp(log_mu_t)
+ *
+ * computed chunk by chunk (chunk size C = 64) with the chunkwise algorithm of
+ * Section 3.1 / Appendix C-D: per-chunk coefficients (Eq. 10), the intra-chunk
+ * unit-lower-triangular solve (Eq. 15), the inter-chunk propagation of S and M,
+ * and the chunk output (Eq. 11-12).
+ *
+ * Conventions for every entry point
+ *  - All data pointers are DEVICE pointers unless a comment says "host".
+ *  - Dense row-major layouts, innermost index last:
+ *      q, k   [B, T, H, dk]      v, o   [B, T, H, dv]
+ *      beta, log_alpha, log_mu, eta  [B, T, H]  float32
+ *      states [N, H, dk, dv] float32, N = B (fixed length) or num_seqs (packed)
+ *  - Packed / variable-length input: B = 1, T = total tokens, cu_seqlens holds
+ *    num_seqs+1 increasing token offsets (cu[0] = 0, cu[num_seqs] = T).  State
+ *    restarts at every sequence; chunks never straddle sequences; the last chunk
+ *    of a sequence may be short.
+ *  - The caller owns every buffer, including the workspace.  The library
+ *    allocates no device memory, keeps no state between calls, and only
+ *    enqueues work on the given stream (it never synchronises).
+ *  - Errors are returned as mdn_status; nothing throws, aborts or traps.
+ *    Invalid arguments are rejected on the host before anything is launched.
+ */
+#ifndef MDN_H_
+#define MDN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  MDN_OK = 0,
+  MDN_ERR_INVALID_ARG = 1,    /* NULL / misaligned pointer, bad shape                       */
+  MDN_ERR_UNSUPPORTED = 2,    /* valid request this build has no kernel for                 */
+  MDN_ERR_WORKSPACE = 3,      /* workspace NULL or smaller than mdn_chunk_fwd_workspace_bytes */
+  MDN_ERR_CUDA = 4,           /* a CUDA runtime call (launch, attribute) failed             */
+  MDN_ERR_DEVICE_TIMEOUT = 5  /* a bounded device-side wait ran out (reported by mdn_read_status) */
+} mdn_status;
+
+typedef enum { MDN_F32 = 0, MDN_BF16 = 1 } mdn_dtype;
+
+/* Which kernels run the chain (inter-chunk propagation + output). */
+typedef enum {
+  MDN_PATH_AUTO = 0,    /* fp32 i/o -> SIMT fp32; bf16 i/o -> tensor-core path          */
+  MDN_PATH_SIMT = 1,    /* fp32 FMA everywhere (any i/o dtype)                          */
+  MDN_PATH_TENSOR = 2   /* tcgen05 bf16 MMAs with fp32 TMEM accumulators (bf16 i/o, d=128) */
+} mdn_path;
+
+typedef struct {
+  int32_t B, T, H, dk, dv; /* packed input: B = 1, T = total tokens                         */
+  int32_t chunk;           /* must be 64                                                     */
+  int32_t num_seqs;        /* number of sequences when cu_seqlens != NULL, else 0            */
+  int32_t io_dtype;        /* mdn_dtype of q, k, v                                           */
+  int32_t o_dtype;         /* mdn_dtype of o                                                 */
+  int32_t path;            /* mdn_path                                                       */
+  float scale;             /* multiplies q; dk^-0.5 is the appendix listing's default,       */
+                           /* 1.0 gives the bare o_t = S_t^T q_t                             */
+} mdn_params;
+
+/* Bytes of device workspace mdn_chunk_fwd needs for these parameters (0 on invalid
+ * parameters).  Holds the chunk map, the per-chunk coefficient vectors and the
+ * per-chunk T and W matrices; contents are scratch. */
+size_t mdn_chunk_fwd_workspace_bytes(const mdn_params* p);
+
+/*
+ * The whole hot path (Section 3.1 "Chunkwise Algorithm"; Appendix C):
+ *   a0  chunk map from cu_seqlens (packed input only)
+ *   a1  coefficient scan: abar, mubar, b and the last-row weights per chunk (Eq. 10)
+ *   a2  intra-chunk system: A = tril((P K^T) .* Gamma^-, -1), T = (I + A)^-1 (Eq. 15),
+ *       W = scale * (Q K^T) .* Gamma (Eq. 12)
+ *   a3  per (sequence, head), chunks in order:  V~ = T (V - Diag(abar) K S + Diag(alpha b^-) K M),
+ *       S, M updates (state equations below Eq. 12)
+ *   a4  O = scale (Diag(abar) Q S - Diag(b) Q M) + W V~   (Eq. 11-12)
+ *
+ * eta may be NULL (eta = 1).  initial_S / initial_M may be NULL (zeros).
+ * final_S / final_M may be NULL (not written).  cu_seqlens NULL = fixed length.
+ * q, k, v, o and the states must be 16-byte aligned; workspace 256-byte aligned.
+ * Asynchronous on `cuda_stream` (a cudaStream_t; NULL = default stream).
+ */
+mdn_status mdn_chunk_fwd(const mdn_params* p,
+                         const void* q, const void* k, const void* v,
+                         const float* beta, const float* log_alpha, const float* log_mu,
+                         const float* eta,
+                         const float* initial_S, const float* initial_M,
+                         const int32_t* cu_seqlens,
+                         void* o, float* final_S, float* final_M,
+                         void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * The same call for HOST buffers (end-to-end use): copies q, k, v, the gates, the
+ * initial states and cu_seqlens from host memory into `arena`, runs mdn_chunk_fwd there,
+ * and copies o and the final states back.  All data pointers except `arena` are HOST
+ * pointers (pinned memory makes the copies asynchronous); `arena` is a DEVICE buffer of at
+ * least mdn_chunk_fwd_host_arena_bytes(p) bytes, 256-byte aligned, owned by the caller.
+ * Everything is enqueued on `cuda_stream`; the caller synchronises before reading o.
+ */
+size_t mdn_chunk_fwd_host_arena_bytes(const mdn_params* p);
+
+mdn_status mdn_chunk_fwd_host(const mdn_params* p,
+                              const void* q, const void* k, const void* v,
+                              const float* beta, const float* log_alpha, const float* log_mu,
+                              const float* eta,
+                              const float* initial_S, const float* initial_M,
+                              const int32_t* cu_seqlens,
+                              void* o, float* final_S, float* final_M,
+                              void* arena /* device */, size_t arena_bytes, void* cuda_stream);
+
+/*
+ * Stage entry points (the same kernels mdn_chunk_fwd launches, exposed so that each
+ * stage can be checked on its own).  Both write into `workspace` using the layout
+ * mdn_workspace_layout describes; mdn_intra_chunk expects mdn_coeff_scan's output there.
+ *
+ * mdn_coeff_scan (a0 + a1, Eq. 10): for every chunk slot s and head h, ten float32
+ * vectors of length 64 at  coef + ((s*H + h)*MDN_NUM_COEF + i)*64 :
+ *   i=0 abar_r   1 b_r   2 alpha_r*b_{r-1}   3 gamma_{last,r}*eta_r   4 (mubar_last/mubar_r)*eta_r
+ *   5 alpha_r    6 beta_r   7 mu_r   8 eta_r   9 mubar_r
+ * Positions past the end of a short chunk hold exact no-ops (alpha = mu = 1, beta = eta = 0).
+ *
+ * mdn_intra_chunk (a2, Eq. 15 and the mask of Eq. 12): per (s, h) the 64x64 row-major
+ * matrices T and W, as float32 (SIMT path) or bfloat16 (tensor path).
+ */
+#define MDN_NUM_COEF 10
+
+typedef struct {
+  int32_t num_slots;        /* chunk slots: B*ceil(T/64), or an upper bound T/64 + num_seqs when packed */
+  int32_t mat_dtype;        /* mdn_dtype of the T and W matrices                                         */
+  uint64_t off_status;      /* int32[4]: [0] 0 = ok, else first device-side error code                   */
+  uint64_t off_chunk_off;   /* int32[num_seqs+1]: first chunk slot of each sequence (packed only)        */
+  uint64_t off_slot_map;    /* int32[num_slots][4]: seq, first token, valid tokens n, local chunk index  */
+  uint64_t off_coef;        /* float32[num_slots][H][MDN_NUM_COEF][64]                                   */
+  uint64_t off_T;           /* [num_slots][H][64][64]                                                    */
+  uint64_t off_W;           /* [num_slots][H][64][64]  (tensor path: bf16 hi part; lo part follows)      */
+  uint64_t total_bytes;
+} mdn_ws_layout;
+
+mdn_status mdn_workspace_layout(const mdn_params* p, mdn_ws_layout* out /* host */);
+
+mdn_status mdn_coeff_scan(const mdn_params* p,
+                          const float* beta, const float* log_alpha, const float* log_mu,
+                          const float* eta, const int32_t* cu_seqlens,
+                          void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+mdn_status mdn_intra_chunk(const mdn_params* p, const void* q, const void* k,
+                           const int32_t* cu_seqlens,
+                           void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Copies the workspace status word to the host (synchronises the stream).  Returns MDN_OK,
+ * MDN_ERR_INVALID_ARG (cu_seqlens rejected by the device-side check) or
+ * MDN_ERR_DEVICE_TIMEOUT. */
+mdn_status mdn_read_status(const mdn_params* p, const void* workspace, void* cuda_stream);
+
+/* Static string for a status code (host pointer, never NULL). */
+const char* mdn_status_string(mdn_status s);
+
+/*
+ * Optional timing hooks for the stages of mdn_chunk_fwd.  `events` is a HOST array of
+ * MDN_NUM_STAGE_EVENTS created cudaEvent_t handles (copied by this call).  While set, every
+ * mdn_chunk_fwd on this host thread records, on its stream: events[0] before its first kernel,
+ * [1] after the chunk map + coefficient scan, [2] after the intra-chunk stage, [3] after the
+ * chain kernel (inter-chunk propagation + output).  NULL clears the hooks.
+ */
+#define MDN_NUM_STAGE_EVENTS 4
+mdn_status mdn_set_stage_events(void* const* events /* host */, int32_t n);
+
+/* Number of kernels the last mdn_* call on this host thread enqueued. */
+int32_t mdn_last_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MDN_H_ */

@@ -9,7 +9,7 @@ training (the paper trains on 4k-token sequences with 400M / 1.3B models);
 that data is not available here, so the shapes, dtypes and value structure
 are reproduced instead:
 
-* q, k: N(0,1) draws, L2-normalised per (token, head) vector (the layer
+* q, k: float32 N(0,1) draws, L2-normalised per (token, head) vector (the layer
   applies L2Norm to q and k, Section 3.3), then rounded once to the storage
   dtype.  v: N(0,1) (no normalisation in the layer).
 * gates: raw logits z ~ N(0,1) pushed through the stability-aware gate
@@ -83,9 +83,10 @@ CONFIGS: List[Workload] = [
 def round_to_bf16(x: np.ndarray) -> np.ndarray:
     """Round float32 values to the nearest bfloat16 (ties to even); returns float32."""
     x = np.ascontiguousarray(x, dtype=np.float32)
-    u = x.view(np.uint32).astype(np.uint64)
-    rounded = ((u + 0x7FFF + ((u >> 16) & 1)) >> 16) << 16
-    return rounded.astype(np.uint32).view(np.float32).reshape(x.shape)
+    u = x.view(np.uint32)
+    with np.errstate(over="ignore"):
+        rounded = (u + (np.uint32(0x7FFF) + ((u >> np.uint32(16)) & np.uint32(1)))) & np.uint32(0xFFFF0000)
+    return rounded.view(np.float32).reshape(x.shape)
 
 
 def bf16_bits(x: np.ndarray) -> np.ndarray:
@@ -103,15 +104,15 @@ def _rng(seed: int, stream: int) -> np.random.Generator:
     return np.random.default_rng([seed, stream])
 
 
-def _store(x64: np.ndarray, dtype: str) -> np.ndarray:
-    """Round fp64 draws once to the storage dtype; returned as float32 (exact)."""
-    x32 = x64.astype(np.float32)
+def _store(x: np.ndarray, dtype: str) -> np.ndarray:
+    """Round draws once to the storage dtype; returned as float32 (exact)."""
+    x32 = np.asarray(x, dtype=np.float32)
     return round_to_bf16(x32) if dtype == "bf16" else x32
 
 
 def _unit_rows(rng: np.random.Generator, shape, dtype: str) -> np.ndarray:
-    x = rng.standard_normal(shape)
-    x /= np.sqrt((x * x).sum(axis=-1, keepdims=True))
+    x = rng.standard_normal(shape, dtype=np.float32)
+    x /= np.sqrt(np.einsum("...d,...d->...", x, x, dtype=np.float64))[..., None].astype(np.float32)
     return _store(x, dtype)
 
 
@@ -164,7 +165,7 @@ def make_inputs(w: Workload, lengths: Optional[np.ndarray] = None) -> Dict[str, 
     B, T, H, dk, dv = w.B, w.T, w.H, w.dk, w.dv
     q = _unit_rows(_rng(w.seed, 0), (B, T, H, dk), w.dtype)
     k = _unit_rows(_rng(w.seed, 1), (B, T, H, dk), w.dtype)
-    v = _store(_rng(w.seed, 2).standard_normal((B, T, H, dv)), w.dtype)
+    v = _store(_rng(w.seed, 2).standard_normal((B, T, H, dv), dtype=np.float32), w.dtype)
     beta, log_alpha, log_mu, eta = draw_gates((B, T, H), w.seed, w.preset, dk)
 
     if w.varlen:

@@ -1,0 +1,262 @@
+"""Thin Python binding of libmdn (argument marshalling only).
+
+Every step of the path runs in the CUDA kernels behind the C ABI declared in
+include/mdn.h; this module turns torch tensors into pointers and sizes.  There is
+no CPU fallback: if the library is missing or was not built, importing the symbols
+raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Tuple
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libmdn.so")
+
+MDN_F32, MDN_BF16 = 0, 1
+PATH_AUTO, PATH_SIMT, PATH_TENSOR = 0, 1, 2
+_PATHS = {"auto": PATH_AUTO, "simt": PATH_SIMT, "tensor": PATH_TENSOR}
+PATH_NAMES = {PATH_AUTO: "auto", PATH_SIMT: "simt", PATH_TENSOR: "tensor"}
+NUM_COEF = 10
+CHUNK = 64
+NUM_STAGE_EVENTS = 4
+STAGE_NAMES = ["coeff_scan", "intra_chunk", "chain"]
+
+
+class MdnParams(ctypes.Structure):
+    _fields_ = [("B", ctypes.c_int32), ("T", ctypes.c_int32), ("H", ctypes.c_int32),
+                ("dk", ctypes.c_int32), ("dv", ctypes.c_int32), ("chunk", ctypes.c_int32),
+                ("num_seqs", ctypes.c_int32), ("io_dtype", ctypes.c_int32), ("o_dtype", ctypes.c_int32),
+                ("path", ctypes.c_int32), ("scale", ctypes.c_float)]
+
+
+class MdnWsLayout(ctypes.Structure):
+    _fields_ = [("num_slots", ctypes.c_int32), ("mat_dtype", ctypes.c_int32),
+                ("off_status", ctypes.c_uint64), ("off_chunk_off", ctypes.c_uint64),
+                ("off_slot_map", ctypes.c_uint64), ("off_coef", ctypes.c_uint64),
+                ("off_T", ctypes.c_uint64), ("off_W", ctypes.c_uint64), ("total_bytes", ctypes.c_uint64)]
+
+
+class MdnError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__("%s: %s (status %d)" % (where, status_string(status), status))
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libmdn.so (built in-tree by paper_2605_05838_b200.build); raises if absent."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError("libmdn.so not found at %s: run `python -m paper_2605_05838_b200.build`" % LIB_PATH)
+        L = ctypes.CDLL(LIB_PATH)
+        vp, P = ctypes.c_void_p, ctypes.POINTER(MdnParams)
+        L.mdn_chunk_fwd_workspace_bytes.restype = ctypes.c_size_t
+        L.mdn_chunk_fwd_workspace_bytes.argtypes = [P]
+        L.mdn_chunk_fwd_host_arena_bytes.restype = ctypes.c_size_t
+        L.mdn_chunk_fwd_host_arena_bytes.argtypes = [P]
+        L.mdn_chunk_fwd.restype = ctypes.c_int
+        L.mdn_chunk_fwd.argtypes = [P] + [vp] * 13 + [vp, ctypes.c_size_t, vp]
+        L.mdn_chunk_fwd_host.restype = ctypes.c_int
+        L.mdn_chunk_fwd_host.argtypes = [P] + [vp] * 13 + [vp, ctypes.c_size_t, vp]
+        L.mdn_workspace_layout.restype = ctypes.c_int
+        L.mdn_workspace_layout.argtypes = [P, ctypes.POINTER(MdnWsLayout)]
+        L.mdn_coeff_scan.restype = ctypes.c_int
+        L.mdn_coeff_scan.argtypes = [P] + [vp] * 5 + [vp, ctypes.c_size_t, vp]
+        L.mdn_intra_chunk.restype = ctypes.c_int
+        L.mdn_intra_chunk.argtypes = [P] + [vp] * 3 + [vp, ctypes.c_size_t, vp]
+        L.mdn_read_status.restype = ctypes.c_int
+        L.mdn_read_status.argtypes = [P, vp, vp]
+        L.mdn_status_string.restype = ctypes.c_char_p
+        L.mdn_status_string.argtypes = [ctypes.c_int]
+        L.mdn_set_stage_events.restype = ctypes.c_int
+        L.mdn_set_stage_events.argtypes = [ctypes.POINTER(vp), ctypes.c_int32]
+        L.mdn_last_launch_count.restype = ctypes.c_int32
+        L.mdn_last_launch_count.argtypes = []
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().mdn_status_string(int(status)).decode()
+
+
+def last_launch_count() -> int:
+    return int(lib().mdn_last_launch_count())
+
+
+def set_stage_events(events) -> None:
+    """events: NUM_STAGE_EVENTS torch.cuda.Event(enable_timing=True), or None to clear the hooks."""
+    if events is None:
+        st = lib().mdn_set_stage_events(None, 0)
+    else:
+        for e in events:
+            if not e.cuda_event:      # torch creates the handle lazily, on the first record
+                e.record()
+        arr = (ctypes.c_void_p * len(events))(*[ctypes.c_void_p(e.cuda_event) for e in events])
+        st = lib().mdn_set_stage_events(arr, len(events))
+    if st != 0:
+        raise MdnError(st, "mdn_set_stage_events")
+
+
+def resolved_path(p: "MdnParams") -> str:
+    """Which chain kernels a call with these parameters runs ("simt" or "tensor")."""
+    lay = workspace_layout(p)
+    return "tensor" if lay.mat_dtype == MDN_BF16 else "simt"
+
+
+def _dtype_code(dt: torch.dtype) -> int:
+    if dt == torch.float32:
+        return MDN_F32
+    if dt == torch.bfloat16:
+        return MDN_BF16
+    raise TypeError("q, k, v, o must be float32 or bfloat16, got %s" % dt)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream() -> ctypes.c_void_p:
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def make_params(q: torch.Tensor, v: torch.Tensor, *, num_seqs: int = 0, scale: Optional[float] = None,
+                o_dtype: Optional[torch.dtype] = None, path: str = "auto") -> MdnParams:
+    B, T, H, dk = q.shape
+    dv = v.shape[-1]
+    return MdnParams(B, T, H, dk, dv, CHUNK, int(num_seqs), _dtype_code(q.dtype),
+                     _dtype_code(o_dtype or q.dtype), _PATHS[path],
+                     float(dk) ** -0.5 if scale is None else float(scale))
+
+
+def workspace_bytes(p: MdnParams) -> int:
+    return int(lib().mdn_chunk_fwd_workspace_bytes(ctypes.byref(p)))
+
+
+def host_arena_bytes(p: MdnParams) -> int:
+    return int(lib().mdn_chunk_fwd_host_arena_bytes(ctypes.byref(p)))
+
+
+def workspace_layout(p: MdnParams) -> MdnWsLayout:
+    lay = MdnWsLayout()
+    st = lib().mdn_workspace_layout(ctypes.byref(p), ctypes.byref(lay))
+    if st != 0:
+        raise MdnError(st, "mdn_workspace_layout")
+    return lay
+
+
+def _check_inputs(q, k, v, gates, device_type: str):
+    for name, t in (("q", q), ("k", k), ("v", v)):
+        if t.device.type != device_type or not t.is_contiguous() or t.dim() != 4:
+            raise ValueError("%s must be a contiguous 4-d %s tensor" % (name, device_type))
+    if q.shape != k.shape or q.shape[:3] != v.shape[:3] or q.dtype != k.dtype or q.dtype != v.dtype:
+        raise ValueError("q, k, v shapes/dtypes disagree")
+    for name, t in gates:
+        if t is None:
+            continue
+        if t.device.type != device_type or not t.is_contiguous() or t.dtype != torch.float32 \
+                or tuple(t.shape) != tuple(q.shape[:3]):
+            raise ValueError("%s must be a contiguous float32 [B,T,H] %s tensor" % (name, device_type))
+
+
+def _check_state(name, t, shape, device_type):
+    if t is None:
+        return
+    if t.device.type != device_type or not t.is_contiguous() or t.dtype != torch.float32 or tuple(t.shape) != shape:
+        raise ValueError("%s must be a contiguous float32 %s tensor of shape %s" % (name, device_type, shape))
+
+
+def chunk_fwd(q, k, v, beta, log_alpha, log_mu, eta=None, *, initial_S=None, initial_M=None,
+              cu_seqlens=None, scale: Optional[float] = None, o_dtype: Optional[torch.dtype] = None,
+              path: str = "auto", output_final_state: bool = True, workspace: Optional[torch.Tensor] = None,
+              out: Optional[torch.Tensor] = None
+              ) -> Tuple[torch.Tensor, Optional[torch.Tensor], Optional[torch.Tensor]]:
+    """mdn_chunk_fwd on CUDA tensors (current stream).  Returns (o, final_S, final_M)."""
+    _check_inputs(q, k, v, (("beta", beta), ("log_alpha", log_alpha), ("log_mu", log_mu), ("eta", eta)), "cuda")
+    B, T, H, dk = q.shape
+    dv = v.shape[-1]
+    N = 0
+    if cu_seqlens is not None:
+        if cu_seqlens.device.type != "cuda" or cu_seqlens.dtype != torch.int32 or not cu_seqlens.is_contiguous():
+            raise ValueError("cu_seqlens must be a contiguous int32 cuda tensor")
+        N = cu_seqlens.numel() - 1
+    p = make_params(q, v, num_seqs=N, scale=scale, o_dtype=o_dtype, path=path)
+    nst = N if N > 0 else B
+    _check_state("initial_S", initial_S, (nst, H, dk, dv), "cuda")
+    _check_state("initial_M", initial_M, (nst, H, dk, dv), "cuda")
+    need = workspace_bytes(p)
+    if need == 0:
+        raise MdnError(2, "mdn_chunk_fwd_workspace_bytes")
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
+    o = out if out is not None else torch.empty((B, T, H, dv), dtype=o_dtype or q.dtype, device=q.device)
+    Sf = Mf = None
+    if output_final_state:
+        Sf = torch.empty((nst, H, dk, dv), dtype=torch.float32, device=q.device)
+        Mf = torch.empty((nst, H, dk, dv), dtype=torch.float32, device=q.device)
+    st = lib().mdn_chunk_fwd(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(beta), _ptr(log_alpha), _ptr(log_mu),
+                             _ptr(eta), _ptr(initial_S), _ptr(initial_M), _ptr(cu_seqlens), _ptr(o), _ptr(Sf),
+                             _ptr(Mf), _ptr(workspace), workspace.numel(), _stream())
+    if st != 0:
+        raise MdnError(st, "mdn_chunk_fwd")
+    return o, Sf, Mf
+
+
+def chunk_fwd_host(q, k, v, beta, log_alpha, log_mu, eta=None, *, initial_S=None, initial_M=None,
+                   cu_seqlens=None, scale: Optional[float] = None, o_dtype: Optional[torch.dtype] = None,
+                   path: str = "auto", output_final_state: bool = True, arena: Optional[torch.Tensor] = None,
+                   out=None, device="cuda:0"):
+    """mdn_chunk_fwd_host: all tensors are HOST tensors (pinned for async copies); `arena` is a
+    CUDA uint8 buffer of host_arena_bytes(p).  Returns host (o, final_S, final_M); synchronises."""
+    _check_inputs(q, k, v, (("beta", beta), ("log_alpha", log_alpha), ("log_mu", log_mu), ("eta", eta)), "cpu")
+    B, T, H, dk = q.shape
+    dv = v.shape[-1]
+    N = 0 if cu_seqlens is None else cu_seqlens.numel() - 1
+    p = make_params(q, v, num_seqs=N, scale=scale, o_dtype=o_dtype, path=path)
+    nst = N if N > 0 else B
+    _check_state("initial_S", initial_S, (nst, H, dk, dv), "cpu")
+    _check_state("initial_M", initial_M, (nst, H, dk, dv), "cpu")
+    need = host_arena_bytes(p)
+    if need == 0:
+        raise MdnError(2, "mdn_chunk_fwd_host_arena_bytes")
+    if arena is None:
+        arena = torch.empty(need, dtype=torch.uint8, device=device)
+    if out is None:
+        o = torch.empty((B, T, H, dv), dtype=o_dtype or q.dtype).pin_memory()
+        Sf = torch.empty((nst, H, dk, dv), dtype=torch.float32).pin_memory() if output_final_state else None
+        Mf = torch.empty((nst, H, dk, dv), dtype=torch.float32).pin_memory() if output_final_state else None
+    else:
+        o, Sf, Mf = out
+    with torch.cuda.device(arena.device):
+        st = lib().mdn_chunk_fwd_host(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(beta), _ptr(log_alpha),
+                                      _ptr(log_mu), _ptr(eta), _ptr(initial_S), _ptr(initial_M), _ptr(cu_seqlens),
+                                      _ptr(o), _ptr(Sf), _ptr(Mf), _ptr(arena), arena.numel(), _stream())
+        if st != 0:
+            raise MdnError(st, "mdn_chunk_fwd_host")
+        torch.cuda.current_stream().synchronize()
+    return o, Sf, Mf
+
+
+def coeff_scan(p: MdnParams, beta, log_alpha, log_mu, eta, cu_seqlens, workspace) -> None:
+    st = lib().mdn_coeff_scan(ctypes.byref(p), _ptr(beta), _ptr(log_alpha), _ptr(log_mu), _ptr(eta),
+                              _ptr(cu_seqlens), _ptr(workspace), workspace.numel(), _stream())
+    if st != 0:
+        raise MdnError(st, "mdn_coeff_scan")
+
+
+def intra_chunk(p: MdnParams, q, k, cu_seqlens, workspace) -> None:
+    st = lib().mdn_intra_chunk(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(cu_seqlens), _ptr(workspace),
+                               workspace.numel(), _stream())
+    if st != 0:
+        raise MdnError(st, "mdn_intra_chunk")
+
+
+def read_status(p: MdnParams, workspace) -> int:
+    return int(lib().mdn_read_status(ctypes.byref(p), _ptr(workspace), _stream()))

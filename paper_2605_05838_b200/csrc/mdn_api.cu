@@ -1,0 +1,274 @@
+// C ABI of libmdn: argument validation, workspace layout, kernel sequencing.
+// Every computation runs in the kernels; this file only checks and launches.
+#include <cstring>
+
+#include "mdn_common.cuh"
+
+namespace mdn {
+
+static thread_local int t_last_launches = 0;
+static thread_local cudaEvent_t t_stage_events[MDN_NUM_STAGE_EVENTS] = {nullptr, nullptr, nullptr, nullptr};
+static thread_local bool t_stage_events_on = false;
+
+static inline bool mark_stage(int i, cudaStream_t s) {
+  return !t_stage_events_on || cudaEventRecord(t_stage_events[i], s) == cudaSuccess;
+}
+
+static inline uint64_t align_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
+static inline bool aligned(const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+static mdn_path resolve_path(const mdn_params& p) {
+  if (p.path == MDN_PATH_AUTO) return p.io_dtype == MDN_BF16 && tensor_path_supported(p) ? MDN_PATH_TENSOR : MDN_PATH_SIMT;
+  return static_cast<mdn_path>(p.path);
+}
+
+static mdn_status check_params(const mdn_params* p) {
+  if (!p) return MDN_ERR_INVALID_ARG;
+  if (p->B <= 0 || p->T <= 0 || p->H <= 0) return MDN_ERR_INVALID_ARG;
+  if (p->chunk != C) return MDN_ERR_UNSUPPORTED;
+  if (!(p->dk == 64 || p->dk == 128) || !(p->dv == 64 || p->dv == 128)) return MDN_ERR_UNSUPPORTED;
+  if (p->io_dtype != MDN_F32 && p->io_dtype != MDN_BF16) return MDN_ERR_INVALID_ARG;
+  if (p->o_dtype != MDN_F32 && p->o_dtype != MDN_BF16) return MDN_ERR_INVALID_ARG;
+  if (p->path < MDN_PATH_AUTO || p->path > MDN_PATH_TENSOR) return MDN_ERR_INVALID_ARG;
+  if (p->num_seqs < 0) return MDN_ERR_INVALID_ARG;
+  if (p->num_seqs > 0 && p->B != 1) return MDN_ERR_INVALID_ARG;
+  if ((int64_t)p->B * p->T >= (int64_t)1 << 31) return MDN_ERR_UNSUPPORTED;
+  if (p->H > 1024) return MDN_ERR_UNSUPPORTED;
+  if (p->path == MDN_PATH_TENSOR && !tensor_path_supported(*p)) return MDN_ERR_UNSUPPORTED;
+  if (!(p->scale == p->scale)) return MDN_ERR_INVALID_ARG;
+  return MDN_OK;
+}
+
+static mdn_status make_layout(const mdn_params& p, mdn_ws_layout* lay) {
+  std::memset(lay, 0, sizeof(*lay));
+  const bool packed = p.num_seqs > 0;
+  const int64_t slots = packed ? (int64_t)p.T / C + p.num_seqs : (int64_t)p.B * ((p.T + C - 1) / C);
+  if (slots >= (int64_t)1 << 30) return MDN_ERR_UNSUPPORTED;
+  lay->num_slots = (int32_t)slots;
+  const bool tensor = resolve_path(p) == MDN_PATH_TENSOR;
+  lay->mat_dtype = tensor ? MDN_BF16 : MDN_F32;
+  const uint64_t mats = (uint64_t)slots * p.H * C * C;
+  uint64_t off = 0;
+  lay->off_status = off; off = align_up(off + 4 * sizeof(int32_t), 256);
+  lay->off_chunk_off = off; off = align_up(off + (uint64_t)(p.num_seqs + 1) * sizeof(int32_t), 256);
+  lay->off_slot_map = off; off = align_up(off + (packed ? (uint64_t)slots * 4 * sizeof(int32_t) : 0), 256);
+  lay->off_coef = off; off = align_up(off + (uint64_t)slots * p.H * MDN_NUM_COEF * C * sizeof(float), 256);
+  lay->off_T = off; off = align_up(off + mats * (tensor ? 2 : 4), 256);
+  lay->off_W = off; off = align_up(off + mats * 4, 256);   // fp32, or bf16 hi + bf16 lo
+  lay->total_bytes = off;
+  return MDN_OK;
+}
+
+static mdn_status make_plan(const mdn_params* p, const int32_t* cu, void* ws, size_t ws_bytes, void* stream,
+                            Plan* pl) {
+  mdn_status st = check_params(p);
+  if (st != MDN_OK) return st;
+  if ((p->num_seqs > 0) != (cu != nullptr)) return MDN_ERR_INVALID_ARG;
+  pl->p = *p;
+  pl->p.path = resolve_path(*p);
+  st = make_layout(*p, &pl->lay);
+  if (st != MDN_OK) return st;
+  if (!ws || ws_bytes < pl->lay.total_bytes || !aligned(ws, 256)) return MDN_ERR_WORKSPACE;
+  pl->ws = static_cast<char*>(ws);
+  pl->stream = static_cast<cudaStream_t>(stream);
+  ChunkGeom& g = pl->geom;
+  g.B = p->B; g.T = p->T; g.H = p->H;
+  g.num_seqs = cu ? p->num_seqs : p->B;
+  g.chunks_per_seq = (p->T + C - 1) / C;
+  g.num_slots = pl->lay.num_slots;
+  g.cu = cu;
+  g.chunk_off = cu ? reinterpret_cast<const int32_t*>(pl->ws + pl->lay.off_chunk_off) : nullptr;
+  g.slot_map = cu ? reinterpret_cast<const int32_t*>(pl->ws + pl->lay.off_slot_map) : nullptr;
+  return MDN_OK;
+}
+
+static mdn_status run_prep_and_scan(const Plan& pl, const float* beta, const float* log_alpha, const float* log_mu,
+                                    const float* eta, int* launches) {
+  if (!beta || !log_alpha || !log_mu) return MDN_ERR_INVALID_ARG;
+  if (!aligned(beta, 4) || !aligned(log_alpha, 4) || !aligned(log_mu, 4) || (eta && !aligned(eta, 4)))
+    return MDN_ERR_INVALID_ARG;
+  if (cudaMemsetAsync(pl.ws + pl.lay.off_status, 0, 4 * sizeof(int32_t), pl.stream) != cudaSuccess)
+    return MDN_ERR_CUDA;
+  if (launch_chunk_map(pl, launches) != cudaSuccess) return MDN_ERR_CUDA;
+  if (launch_coeff_scan(pl, beta, log_alpha, log_mu, eta, launches) != cudaSuccess) return MDN_ERR_CUDA;
+  return MDN_OK;
+}
+
+static mdn_status run_intra(const Plan& pl, const void* q, const void* k, int* launches) {
+  if (!q || !k || !aligned(q, 16) || !aligned(k, 16)) return MDN_ERR_INVALID_ARG;
+  cudaError_t e = pl.p.path == MDN_PATH_TENSOR ? launch_intra_tensor(pl, q, k, launches)
+                                               : launch_intra_simt(pl, q, k, launches);
+  return e == cudaSuccess ? MDN_OK : MDN_ERR_CUDA;
+}
+
+}  // namespace mdn
+
+using namespace mdn;
+
+extern "C" {
+
+size_t mdn_chunk_fwd_workspace_bytes(const mdn_params* p) {
+  mdn_ws_layout lay;
+  if (check_params(p) != MDN_OK || make_layout(*p, &lay) != MDN_OK) return 0;
+  return (size_t)lay.total_bytes;
+}
+
+mdn_status mdn_workspace_layout(const mdn_params* p, mdn_ws_layout* out) {
+  if (!out) return MDN_ERR_INVALID_ARG;
+  mdn_status st = check_params(p);
+  if (st != MDN_OK) return st;
+  return make_layout(*p, out);
+}
+
+mdn_status mdn_coeff_scan(const mdn_params* p, const float* beta, const float* log_alpha, const float* log_mu,
+                          const float* eta, const int32_t* cu_seqlens, void* workspace, size_t workspace_bytes,
+                          void* cuda_stream) {
+  t_last_launches = 0;
+  Plan pl;
+  mdn_status st = make_plan(p, cu_seqlens, workspace, workspace_bytes, cuda_stream, &pl);
+  if (st != MDN_OK) return st;
+  return run_prep_and_scan(pl, beta, log_alpha, log_mu, eta, &t_last_launches);
+}
+
+mdn_status mdn_intra_chunk(const mdn_params* p, const void* q, const void* k, const int32_t* cu_seqlens,
+                           void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  t_last_launches = 0;
+  Plan pl;
+  mdn_status st = make_plan(p, cu_seqlens, workspace, workspace_bytes, cuda_stream, &pl);
+  if (st != MDN_OK) return st;
+  return run_intra(pl, q, k, &t_last_launches);
+}
+
+mdn_status mdn_chunk_fwd(const mdn_params* p, const void* q, const void* k, const void* v, const float* beta,
+                         const float* log_alpha, const float* log_mu, const float* eta, const float* initial_S,
+                         const float* initial_M, const int32_t* cu_seqlens, void* o, float* final_S,
+                         float* final_M, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  t_last_launches = 0;
+  Plan pl;
+  mdn_status st = make_plan(p, cu_seqlens, workspace, workspace_bytes, cuda_stream, &pl);
+  if (st != MDN_OK) return st;
+  if (!q || !k || !v || !o) return MDN_ERR_INVALID_ARG;
+  if (!aligned(q, 16) || !aligned(k, 16) || !aligned(v, 16) || !aligned(o, 16)) return MDN_ERR_INVALID_ARG;
+  if ((initial_S && !aligned(initial_S, 16)) || (initial_M && !aligned(initial_M, 16)) ||
+      (final_S && !aligned(final_S, 16)) || (final_M && !aligned(final_M, 16)))
+    return MDN_ERR_INVALID_ARG;
+  if (!mark_stage(0, pl.stream)) return MDN_ERR_CUDA;
+  st = run_prep_and_scan(pl, beta, log_alpha, log_mu, eta, &t_last_launches);
+  if (st != MDN_OK) return st;
+  if (!mark_stage(1, pl.stream)) return MDN_ERR_CUDA;
+  st = run_intra(pl, q, k, &t_last_launches);
+  if (st != MDN_OK) return st;
+  if (!mark_stage(2, pl.stream)) return MDN_ERR_CUDA;
+  cudaError_t e = pl.p.path == MDN_PATH_TENSOR
+                      ? launch_chain_tensor(pl, q, k, v, initial_S, initial_M, o, final_S, final_M, &t_last_launches)
+                      : launch_chain_simt(pl, q, k, v, initial_S, initial_M, o, final_S, final_M, &t_last_launches);
+  if (e != cudaSuccess) return MDN_ERR_CUDA;
+  if (!mark_stage(3, pl.stream)) return MDN_ERR_CUDA;
+  return MDN_OK;
+}
+
+mdn_status mdn_set_stage_events(void* const* events, int32_t n) {
+  if (events == nullptr) { t_stage_events_on = false; return MDN_OK; }
+  if (n < MDN_NUM_STAGE_EVENTS) return MDN_ERR_INVALID_ARG;
+  for (int i = 0; i < MDN_NUM_STAGE_EVENTS; ++i) {
+    if (events[i] == nullptr) return MDN_ERR_INVALID_ARG;
+    t_stage_events[i] = static_cast<cudaEvent_t>(events[i]);
+  }
+  t_stage_events_on = true;
+  return MDN_OK;
+}
+
+// ---- host-buffer variant: arena = [q | k | v | 4 gates | S0 | M0 | cu | o | Sf | Mf | workspace]
+struct HostArena {
+  uint64_t q, k, v, gates[4], S0, M0, cu, o, Sf, Mf, ws, total;
+  uint64_t qk_bytes, v_bytes, gate_bytes, state_bytes, cu_bytes, o_bytes;
+};
+
+static bool host_arena(const mdn_params* p, HostArena* a) {
+  mdn_ws_layout lay;
+  if (check_params(p) != MDN_OK || make_layout(*p, &lay) != MDN_OK) return false;
+  const uint64_t tokens = (uint64_t)p->B * p->T, es = p->io_dtype == MDN_BF16 ? 2 : 4, eo = p->o_dtype == MDN_BF16 ? 2 : 4;
+  const uint64_t nstate = (uint64_t)(p->num_seqs > 0 ? p->num_seqs : p->B) * p->H * p->dk * p->dv;
+  a->qk_bytes = tokens * p->H * p->dk * es; a->v_bytes = tokens * p->H * p->dv * es;
+  a->gate_bytes = tokens * p->H * 4; a->state_bytes = nstate * 4;
+  a->cu_bytes = p->num_seqs > 0 ? (uint64_t)(p->num_seqs + 1) * 4 : 0; a->o_bytes = tokens * p->H * p->dv * eo;
+  uint64_t off = 0;
+  auto take = [&](uint64_t bytes) { uint64_t at = off; off = align_up(off + bytes, 256); return at; };
+  a->q = take(a->qk_bytes); a->k = take(a->qk_bytes); a->v = take(a->v_bytes);
+  for (int i = 0; i < 4; ++i) a->gates[i] = take(a->gate_bytes);
+  a->S0 = take(a->state_bytes); a->M0 = take(a->state_bytes); a->cu = take(a->cu_bytes);
+  a->o = take(a->o_bytes); a->Sf = take(a->state_bytes); a->Mf = take(a->state_bytes);
+  a->ws = take(lay.total_bytes); a->total = off;
+  return true;
+}
+
+size_t mdn_chunk_fwd_host_arena_bytes(const mdn_params* p) {
+  HostArena a;
+  return host_arena(p, &a) ? (size_t)a.total : 0;
+}
+
+mdn_status mdn_chunk_fwd_host(const mdn_params* p, const void* q, const void* k, const void* v, const float* beta,
+                              const float* log_alpha, const float* log_mu, const float* eta,
+                              const float* initial_S, const float* initial_M, const int32_t* cu_seqlens, void* o,
+                              float* final_S, float* final_M, void* arena, size_t arena_bytes, void* cuda_stream) {
+  HostArena a;
+  if (!host_arena(p, &a)) return check_params(p) != MDN_OK ? check_params(p) : MDN_ERR_UNSUPPORTED;
+  if (!arena || arena_bytes < a.total || !aligned(arena, 256)) return MDN_ERR_WORKSPACE;
+  if (!q || !k || !v || !beta || !log_alpha || !log_mu || !o) return MDN_ERR_INVALID_ARG;
+  if ((p->num_seqs > 0) != (cu_seqlens != nullptr)) return MDN_ERR_INVALID_ARG;
+  char* d = static_cast<char*>(arena);
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  auto h2d = [&](uint64_t off, const void* src, uint64_t bytes) {
+    return src == nullptr || bytes == 0 || cudaMemcpyAsync(d + off, src, bytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
+  };
+  auto d2h = [&](void* dst, uint64_t off, uint64_t bytes) {
+    return dst == nullptr || cudaMemcpyAsync(dst, d + off, bytes, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+  };
+  if (!h2d(a.q, q, a.qk_bytes) || !h2d(a.k, k, a.qk_bytes) || !h2d(a.v, v, a.v_bytes) ||
+      !h2d(a.gates[0], beta, a.gate_bytes) || !h2d(a.gates[1], log_alpha, a.gate_bytes) ||
+      !h2d(a.gates[2], log_mu, a.gate_bytes) || !h2d(a.gates[3], eta, a.gate_bytes) ||
+      !h2d(a.S0, initial_S, a.state_bytes) || !h2d(a.M0, initial_M, a.state_bytes) ||
+      !h2d(a.cu, cu_seqlens, a.cu_bytes))
+    return MDN_ERR_CUDA;
+  auto fp = [&](uint64_t off, const void* given) { return given ? reinterpret_cast<float*>(d + off) : nullptr; };
+  mdn_ws_layout lay;
+  make_layout(*p, &lay);
+  mdn_status st = mdn_chunk_fwd(p, d + a.q, d + a.k, d + a.v, fp(a.gates[0], beta), fp(a.gates[1], log_alpha),
+                                fp(a.gates[2], log_mu), fp(a.gates[3], eta), fp(a.S0, initial_S),
+                                fp(a.M0, initial_M),
+                                cu_seqlens ? reinterpret_cast<const int32_t*>(d + a.cu) : nullptr, d + a.o,
+                                fp(a.Sf, final_S), fp(a.Mf, final_M), d + a.ws, lay.total_bytes, cuda_stream);
+  if (st != MDN_OK) return st;
+  if (!d2h(o, a.o, a.o_bytes) || !d2h(final_S, a.Sf, a.state_bytes) || !d2h(final_M, a.Mf, a.state_bytes))
+    return MDN_ERR_CUDA;
+  return MDN_OK;
+}
+
+mdn_status mdn_read_status(const mdn_params* p, const void* workspace, void* cuda_stream) {
+  mdn_ws_layout lay;
+  if (!workspace || check_params(p) != MDN_OK || make_layout(*p, &lay) != MDN_OK) return MDN_ERR_INVALID_ARG;
+  int32_t word[4] = {0, 0, 0, 0};
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemcpyAsync(word, static_cast<const char*>(workspace) + lay.off_status, sizeof(word),
+                      cudaMemcpyDeviceToHost, s) != cudaSuccess)
+    return MDN_ERR_CUDA;
+  if (cudaStreamSynchronize(s) != cudaSuccess) return MDN_ERR_CUDA;
+  if (word[0] == kDevOk) return MDN_OK;
+  return word[0] == kDevBadCuSeqlens ? MDN_ERR_INVALID_ARG : MDN_ERR_DEVICE_TIMEOUT;
+}
+
+const char* mdn_status_string(mdn_status s) {
+  switch (s) {
+    case MDN_OK: return "ok";
+    case MDN_ERR_INVALID_ARG: return "invalid argument";
+    case MDN_ERR_UNSUPPORTED: return "unsupported configuration";
+    case MDN_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case MDN_ERR_CUDA: return "CUDA runtime error";
+    case MDN_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+  }
+  return "unknown status";
+}
+
+int32_t mdn_last_launch_count(void) { return t_last_launches; }
+
+}  // extern "C"

@@ -1,0 +1,113 @@
+// Shared declarations of the MDN chunkwise-forward kernels (sm_100a).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "mdn.h"
+
+namespace mdn {
+
+constexpr int C = 64;  // chunk size (Section 3.1; the appendix listing's default)
+
+// Indices of the per-(chunk, head) coefficient vectors (Eq. 10 and the state equations).
+enum Coef : int {
+  kAbar = 0,    // abar_r  = prod_{j<=r} alpha_j
+  kB = 1,       // b_r     = abar_r c_r           (weight of -M_[t] in S_r)
+  kAlphaBPrev = 2,  // alpha_r * b_{r-1}          (weight of +K M_[t] in the right-hand side)
+  kGS = 3,      // gamma_{last,r} * eta_r         (weight of k_r v~_r^T in S_[t+1])
+  kGM = 4,      // (mubar_last/mubar_r) * eta_r   (weight of -k_r v~_r^T in M_[t+1])
+  kAlpha = 5,
+  kBeta = 6,
+  kMu = 7,
+  kEta = 8,
+  kMubar = 9
+};
+
+// Device-side error codes written to the workspace status word.
+enum DevErr : int { kDevOk = 0, kDevBadCuSeqlens = 1, kDevTimeout = 2 };
+
+// Everything a kernel needs to find a chunk: either arithmetic (fixed length) or
+// the slot map the prep kernel wrote (packed input).
+struct ChunkGeom {
+  int B, T, H;
+  int num_seqs;          // sequences (B when fixed length)
+  int chunks_per_seq;    // fixed length only
+  int num_slots;
+  const int32_t* cu;         // packed only
+  const int32_t* chunk_off;  // packed only: first slot of each sequence [num_seqs+1]
+  const int32_t* slot_map;   // packed only: [num_slots][4]
+};
+
+struct SlotInfo {
+  int seq;      // sequence id, -1 when the slot is unused
+  int tok0;     // first token (index into the flattened [B*T] token axis)
+  int n;        // valid tokens in this chunk, 1..64
+  int local;    // chunk index inside its sequence
+};
+
+__device__ __forceinline__ SlotInfo slot_info(const ChunkGeom& g, int slot) {
+  SlotInfo s;
+  if (g.cu == nullptr) {
+    s.seq = slot / g.chunks_per_seq;
+    s.local = slot - s.seq * g.chunks_per_seq;
+    s.tok0 = s.seq * g.T + s.local * C;
+    s.n = min(C, g.T - s.local * C);
+  } else {
+    const int4 m = reinterpret_cast<const int4*>(g.slot_map)[slot];
+    s.seq = m.x; s.tok0 = m.y; s.n = m.z; s.local = m.w;
+  }
+  return s;
+}
+
+// Range of chunk slots and tokens of one sequence (for the chain kernels).
+struct SeqInfo { int slot0, nchunks, tok0, len; };
+
+__device__ __forceinline__ SeqInfo seq_info(const ChunkGeom& g, int seq) {
+  SeqInfo s;
+  if (g.cu == nullptr) {
+    s.slot0 = seq * g.chunks_per_seq; s.nchunks = g.chunks_per_seq; s.tok0 = seq * g.T; s.len = g.T;
+  } else {
+    s.slot0 = g.chunk_off[seq]; s.nchunks = g.chunk_off[seq + 1] - s.slot0;
+    s.tok0 = g.cu[seq]; s.len = g.cu[seq + 1] - s.tok0;
+  }
+  return s;
+}
+
+template <typename T> __device__ __forceinline__ float to_f32(T x);
+template <> __device__ __forceinline__ float to_f32<float>(float x) { return x; }
+template <> __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 x) { return __bfloat162float(x); }
+
+template <typename T> __device__ __forceinline__ T from_f32(float x);
+template <> __device__ __forceinline__ float from_f32<float>(float x) { return x; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float x) { return __float2bfloat16_rn(x); }
+
+// Host-side view of one call, filled by the API layer.
+struct Plan {
+  mdn_params p;
+  mdn_ws_layout lay;
+  ChunkGeom geom;
+  char* ws;
+  cudaStream_t stream;
+};
+
+// Launchers (one per .cu file).  Each returns the CUDA error of its launches and adds
+// the number of kernels it enqueued to *launches.
+cudaError_t launch_chunk_map(const Plan& pl, int* launches);
+cudaError_t launch_coeff_scan(const Plan& pl, const float* beta, const float* log_alpha,
+                              const float* log_mu, const float* eta, int* launches);
+cudaError_t launch_intra_simt(const Plan& pl, const void* q, const void* k, int* launches);
+cudaError_t launch_chain_simt(const Plan& pl, const void* q, const void* k, const void* v,
+                              const float* S0, const float* M0, void* o, float* Sf, float* Mf,
+                              int* launches);
+
+
+// Tensor-core (tcgen05) path: bf16 q/k/v, dk = dv = 128.
+bool tensor_path_supported(const mdn_params& p);
+cudaError_t launch_intra_tensor(const Plan& pl, const void* q, const void* k, int* launches);
+cudaError_t launch_chain_tensor(const Plan& pl, const void* q, const void* k, const void* v,
+                                const float* S0, const float* M0, void* o, float* Sf, float* Mf,
+                                int* launches);
+
+}  // namespace mdn

@@ -1,0 +1,83 @@
+"""The C-ABI library loads, exports every symbol include/mdn.h declares, and rejects bad
+arguments on the host (no GPU needed: validation happens before any launch)."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def mdn():
+    from paper_2605_05838_b200 import build
+    build.build()
+    import paper_2605_05838_b200 as m
+    m.lib()
+    return m
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "mdn.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(mdn_[a-z_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(mdn):
+    names = declared_symbols()
+    assert "mdn_chunk_fwd" in names and "mdn_chunk_fwd_workspace_bytes" in names and "mdn_status_string" in names
+    for n in names:
+        assert hasattr(mdn.lib(), n), n
+
+
+def test_status_strings(mdn):
+    assert mdn.status_string(0) == "ok"
+    assert all(mdn.status_string(s) for s in range(0, 7))
+
+
+def params(mdn, **kw):
+    base = dict(B=2, T=130, H=3, dk=64, dv=128, chunk=64, num_seqs=0, io_dtype=0, o_dtype=0, path=0, scale=0.125)
+    base.update(kw)
+    return mdn.MdnParams(**base)
+
+
+def test_workspace_layout_and_bounds(mdn):
+    p = params(mdn)
+    lay = mdn.workspace_layout(p)
+    assert lay.num_slots == 2 * 3                      # ceil(130/64) = 3 chunks per row
+    assert mdn.workspace_bytes(p) == lay.total_bytes > 0
+    assert lay.off_coef % 256 == 0 and lay.off_T % 256 == 0 and lay.off_W % 256 == 0
+    assert lay.off_T - lay.off_coef >= lay.num_slots * 3 * mdn.NUM_COEF * 64 * 4
+    packed = params(mdn, B=1, T=1000, num_seqs=7)
+    assert mdn.workspace_layout(packed).num_slots == 1000 // 64 + 7     # upper bound on sum ceil(len/64)
+    assert mdn.host_arena_bytes(p) > mdn.workspace_bytes(p)
+
+
+@pytest.mark.parametrize("kw", [dict(chunk=32), dict(dk=96), dict(dv=32), dict(B=0), dict(T=0), dict(H=0),
+                                dict(io_dtype=5), dict(path=9), dict(num_seqs=3), dict(num_seqs=-1)])
+def test_bad_params_rejected(mdn, kw):
+    assert mdn.workspace_bytes(params(mdn, **kw)) == 0
+
+
+def test_null_and_workspace_errors_before_any_launch(mdn):
+    L = mdn.lib()
+    p = params(mdn)
+    null = ctypes.c_void_p(None)
+    fake = ctypes.c_void_p(256 * 4096)   # never dereferenced: rejected by host validation first
+    args = [null] * 13
+    st = L.mdn_chunk_fwd(ctypes.byref(p), *args, null, 0, null)
+    assert mdn.status_string(st).startswith("workspace")
+    st = L.mdn_chunk_fwd(ctypes.byref(p), *args, fake, 16, null)
+    assert mdn.status_string(st).startswith("workspace")
+    st = L.mdn_chunk_fwd(ctypes.byref(p), *args, ctypes.c_void_p(256 * 4096 + 8), 1 << 40, null)
+    assert mdn.status_string(st).startswith("workspace")          # misaligned
+    st = L.mdn_chunk_fwd(ctypes.byref(p), *args, fake, 1 << 40, null)
+    assert mdn.status_string(st) == "invalid argument"            # q is NULL
+    bad = params(mdn, chunk=16)
+    st = L.mdn_chunk_fwd(ctypes.byref(bad), *args, fake, 1 << 40, null)
+    assert mdn.status_string(st).startswith("unsupported")
+    # cu_seqlens given but num_seqs == 0
+    a2 = list(args); a2[9] = fake
+    st = L.mdn_chunk_fwd(ctypes.byref(p), *a2, fake, 1 << 40, null)
+    assert mdn.status_string(st) == "invalid argument"

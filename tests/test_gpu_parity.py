@@ -1,0 +1,297 @@
+"""Parity of the CUDA path (through the C ABI) with the fp64 CPU oracle, element by element on the
+same seeded inputs.
+
+Tolerances (max |x - ref| / RMS(ref), RMS over the reference entries compared):
+  fp32 i/o            o, S, M <= 1e-4
+  bf16 i/o, fp32 o    o, S, M <= 2e-2
+  bf16 i/o, bf16 o    |o - ref| <= 2e-2 RMS + 2^-8 |ref| per element: storing the *exact* result in bf16
+                      already costs up to 2^-8 |ref| (>= 2e-2 RMS at the tails of these outputs), so the
+                      stored output is allowed that one rounding on top of the 2e-2 budget; the literal
+                      metric and the oracle-only storage floor are printed beside it.
+"""
+import dataclasses
+
+import numpy as np
+import pytest
+
+import mdn_workloads as wl
+from helpers import bf16_floor, chain_mask_tokens, rel_err, run_gpu, run_oracle, to_torch
+
+pytestmark = pytest.mark.gpu
+
+TOL_F32 = 1e-4
+TOL_BF16 = 2e-2
+
+
+@pytest.fixture(scope="module")
+def mdn():
+    import paper_2605_05838_b200 as m
+    m.lib()          # raises if the CUDA library is missing: no fallback
+    return m
+
+
+def tensor_ok(mdn, w):
+    p = mdn.MdnParams(w.B, w.T, w.H, w.dk, w.dv, 64, 0, 1, 1, 2, 1.0)
+    return w.dtype == "bf16" and mdn.workspace_bytes(p) > 0
+
+
+def paths_for(mdn, w):
+    return ["simt", "tensor"] if tensor_ok(mdn, w) else ["simt"]
+
+
+def check_bf16_store(o_bf16, o_ref, label):
+    mask = ~np.isnan(o_ref)
+    rms = np.sqrt(np.mean(o_ref[mask] ** 2))
+    excess = np.abs(o_bf16[mask] - o_ref[mask]) - 2.0 ** -8 * np.abs(o_ref[mask])
+    literal = rel_err(o_bf16, o_ref)
+    print("%s: bf16-store literal %.3e, oracle bf16 floor %.3e, excess over one rounding %.3e"
+          % (label, literal, bf16_floor(o_ref), excess.max() / rms))
+    assert excess.max() <= TOL_BF16 * rms
+
+
+def compare(mdn, inp, path, chains=None, tol=None, label=""):
+    w = inp["workload"]
+    o_ref, S_ref, M_ref = run_oracle(inp, chains)
+    if w.dtype == "f32":
+        o, S, M = run_gpu(mdn, inp, path=path)
+        errs = rel_err(o, o_ref), rel_err(S, S_ref), rel_err(M, M_ref)
+        print("%s[%s] fp32: o %.3e S %.3e M %.3e" % (label, path, *errs))
+        assert max(errs) <= (tol or TOL_F32)
+        return
+    import torch
+    o, S, M = run_gpu(mdn, inp, path=path, o_dtype=torch.float32)
+    errs = rel_err(o, o_ref), rel_err(S, S_ref), rel_err(M, M_ref)
+    print("%s[%s] bf16 in / fp32 out: o %.3e S %.3e M %.3e" % (label, path, *errs))
+    assert max(errs) <= (tol or TOL_BF16)
+    ob, Sb, Mb = run_gpu(mdn, inp, path=path)
+    check_bf16_store(ob, o_ref, "%s[%s]" % (label, path))
+    assert np.array_equal(Sb, S) and np.array_equal(Mb, M)     # states do not depend on o's dtype
+
+
+# ------------------------------------------------------------------------------------------ stages
+def test_coefficient_scan_matches_eq10(mdn):
+    import torch
+    from oracle import chunkwise as cw
+    w = wl.Workload("coef", B=2, T=150, H=3, dk=64, dv=64, dtype="f32", seed=3)
+    inp = wl.make_inputs(w)
+    inp["log_mu"][0, 70:80, 1] = -np.inf          # mu = 0 tokens
+    inp["beta"][1, 5:9, 2] = 0.0                  # beta = 0 tokens
+    t = to_torch(inp)
+    p = mdn.make_params(t["q"], t["v"])
+    lay = mdn.workspace_layout(p)
+    ws = torch.zeros(lay.total_bytes, dtype=torch.uint8, device="cuda")
+    mdn.coeff_scan(p, t["beta"], t["log_alpha"], t["log_mu"], t["eta"], None, ws)
+    assert mdn.last_launch_count() == 1
+    torch.cuda.synchronize()
+    nfl = lay.num_slots * w.H * mdn.NUM_COEF * 64
+    coef = ws[lay.off_coef: lay.off_coef + 4 * nfl].view(torch.float32).cpu().numpy().reshape(
+        lay.num_slots, w.H, mdn.NUM_COEF, 64).astype(np.float64)
+    nchunks = 3
+    for b in range(w.B):
+        for h in range(w.H):
+            for c in range(nchunks):
+                n = min(64, w.T - 64 * c)
+                sl = slice(64 * c, 64 * c + n)
+                la = inp["log_alpha"][b, sl, h]; lm = inp["log_mu"][b, sl, h]
+                be = inp["beta"][b, sl, h]; et = inp["eta"][b, sl, h].astype(np.float64)
+                if np.isinf(lm).any():
+                    abar, mubar, bb, G, Mm = cw.coefficients_by_products(la, lm, be)
+                else:
+                    abar, mubar, _, bb, G = cw.coefficients(la, lm, be)
+                    Mm = np.tril(mubar[:, None] / mubar[None, :])
+                got = coef[b * nchunks + c, h]
+                tol = dict(rtol=2e-5, atol=1e-7)
+                assert np.allclose(got[0, :n], abar, **tol) and np.allclose(got[9, :n], mubar, **tol)
+                assert np.allclose(got[1, :n], bb, **tol)
+                b_prev = np.concatenate([[0.0], bb[:-1]])
+                assert np.allclose(got[2, :n], np.exp(la.astype(np.float64)) * b_prev, **tol)
+                assert np.allclose(got[3, :n], G[-1] * et, **tol)
+                assert np.allclose(got[4, :n], Mm[-1] * et, **tol)
+                # exact no-ops past the end of a short chunk; last entries equal the last valid ones
+                assert (got[3, n:] == 0).all() and (got[4, n:] == 0).all()
+                assert np.allclose(got[0, 63], abar[-1], **tol) and np.allclose(got[1, 63], bb[-1], **tol)
+                assert np.allclose(got[9, 63], mubar[-1], **tol)
+
+
+def test_intra_chunk_T_and_W_match_eq15(mdn):
+    import torch
+    from oracle import chunkwise as cw
+    w = wl.Workload("intra", B=1, T=200, H=2, dk=64, dv=64, dtype="f32", seed=4, preset="F")
+    inp = wl.make_inputs(w)
+    inp["k"] = wl.correlated_keys(w, 0.8)          # makes the triangular system far from the identity
+    t = to_torch(inp)
+    p = mdn.make_params(t["q"], t["v"], scale=inp["scale"])
+    lay = mdn.workspace_layout(p)
+    ws = torch.zeros(lay.total_bytes, dtype=torch.uint8, device="cuda")
+    mdn.coeff_scan(p, t["beta"], t["log_alpha"], t["log_mu"], t["eta"], None, ws)
+    mdn.intra_chunk(p, t["q"], t["k"], None, ws)
+    torch.cuda.synchronize()
+    nm = lay.num_slots * w.H * 64 * 64
+    Tm = ws[lay.off_T: lay.off_T + 4 * nm].view(torch.float32).cpu().numpy().reshape(lay.num_slots, w.H, 64, 64)
+    Wm = ws[lay.off_W: lay.off_W + 4 * nm].view(torch.float32).cpu().numpy().reshape(lay.num_slots, w.H, 64, 64)
+    for h in range(w.H):
+        _, _, _, stages = cw.chunk_forward(inp["q"][0, :, h], inp["k"][0, :, h], inp["v"][0, :, h],
+                                           inp["beta"][0, :, h], inp["log_alpha"][0, :, h], inp["log_mu"][0, :, h],
+                                           inp["eta"][0, :, h], scale=inp["scale"], return_stages=True)
+        for c, st in enumerate(stages):
+            n = st["n"]
+            assert np.abs(st["T"] - np.eye(64)).max() > 0.05       # the solve is exercised
+            assert np.allclose(Tm[c, h], st["T"], rtol=1e-4, atol=1e-5)
+            sl = slice(64 * c, 64 * c + n)
+            Q = np.zeros((64, 64)); K = np.zeros((64, 64)); et = np.zeros(64)
+            Q[:n] = inp["q"][0, sl, h]; K[:n] = inp["k"][0, sl, h]; et[:n] = inp["eta"][0, sl, h]
+            W_ref = inp["scale"] * (Q @ (et[:, None] * K).T) * st["Gamma"]
+            assert np.allclose(Wm[c, h], W_ref, rtol=1e-4, atol=1e-6)
+
+
+# ------------------------------------------------------------------------------------------ named configs
+def test_config0_tiny_fp32(mdn):
+    inp = wl.make_inputs(wl.CONFIGS[0])
+    compare(mdn, inp, "simt", label="cfg0")
+
+
+@pytest.mark.parametrize("cfg", [1, 2, 3, 4])
+def test_named_bf16_configs_full_size(mdn, cfg):
+    w = wl.CONFIGS[cfg]
+    inp = wl.make_inputs(w)
+    N = len(inp["seq_len"])
+    rng = np.random.default_rng(cfg)
+    all_chains = np.arange(N * w.H)
+    if cfg == 1:
+        chains = all_chains
+    elif cfg == 2:      # first, last and 14 random chains of 128
+        chains = np.unique(np.concatenate([[0, N * w.H - 1], rng.choice(all_chains, 14, replace=False)]))
+    elif cfg == 3:      # 4 of 16 heads, all 65536 tokens (1024 serial chunk steps)
+        chains = np.array([0, 5, 10, 15])
+    else:               # every sequence, two heads each
+        chains = np.array([n * w.H + h for n in range(N) for h in (n % w.H, (n + 7) % w.H)])
+    for path in paths_for(mdn, w):
+        compare(mdn, inp, path, chains=chains, label=w.name)
+
+
+# ------------------------------------------------------------------------------------------ edge cases
+def small(dtype="f32", **kw):
+    base = dict(name="small", B=2, T=150, H=2, dk=64, dv=64, dtype=dtype, seed=11)
+    base.update(kw)
+    return wl.Workload(**base)
+
+
+@pytest.mark.parametrize("T", [1, 2, 63, 64, 65, 127, 129, 200])
+def test_ragged_lengths_fp32(mdn, T):
+    compare(mdn, wl.make_inputs(small(T=T, init_state_std=0.5)), "simt", label="T=%d" % T)
+
+
+@pytest.mark.parametrize("dk,dv", [(64, 128), (128, 64), (128, 128)])
+def test_head_dims_fp32(mdn, dk, dv):
+    compare(mdn, wl.make_inputs(small(dk=dk, dv=dv, T=130, init_state_std=0.3)), "simt", label="dk%d dv%d" % (dk, dv))
+
+
+def test_fast_forgetting_preset_and_correlated_keys(mdn):
+    w = small(T=300, preset="F", init_state_std=0.2)
+    inp = wl.make_inputs(w)
+    inp["k"] = wl.correlated_keys(w, 0.8)
+    compare(mdn, inp, "simt", label="preset F, correlated keys")
+    wb = small(dtype="bf16", dk=128, dv=128, T=300, preset="F", init_state_std=0.2)
+    inpb = wl.make_inputs(wb)
+    inpb["k"] = wl.correlated_keys(wb, 0.8)
+    for path in paths_for(mdn, wb):
+        compare(mdn, inpb, path, label="preset F bf16, correlated keys")
+
+
+def test_degenerate_gates(mdn):
+    """beta = 0 and mu = 0 tokens (the paper's log-domain kernels NaN at mu = 0), eta = None, scale = 1."""
+    w = small(T=140)
+    inp = wl.make_inputs(w)
+    inp["beta"][:, 10:30] = 0.0
+    inp["log_mu"][:, 40:90] = -np.inf
+    compare(mdn, inp, "simt", label="beta=0 / mu=0 tokens")
+    inp2 = wl.make_inputs(w)
+    inp2["log_mu"][:] = -np.inf                     # whole call reduces to the gated delta rule
+    compare(mdn, inp2, "simt", label="mu=0 everywhere")
+    inp3 = wl.make_inputs(w)
+    inp3["beta"][:] = 0.0
+    inp3["S0"] = np.random.default_rng(0).standard_normal((2, 2, 64, 64)).astype(np.float32)
+    inp3["M0"] = None
+    o, S, M = run_gpu(mdn, inp3, path="simt")
+    abar = np.exp(np.cumsum(inp3["log_alpha"].astype(np.float64), axis=1))[:, -1]       # [B,H]
+    assert np.allclose(S, abar[:, :, None, None] * inp3["S0"], rtol=1e-4, atol=1e-7)    # purely decayed state
+    inp4 = wl.make_inputs(w)
+    inp4["eta"] = None
+    inp4["scale"] = 1.0
+    o_ref, S_ref, M_ref = run_oracle(inp4)
+    o, S, M = run_gpu(mdn, inp4, path="simt")
+    assert max(rel_err(o, o_ref), rel_err(S, S_ref), rel_err(M, M_ref)) <= TOL_F32
+
+
+def test_packed_varlen_edge_lengths(mdn):
+    lens = np.array([1, 63, 64, 65, 129, 2, 300, 128])
+    w = small(B=1, T=int(lens.sum()), varlen=True, init_state_std=0.4)
+    inp = wl.make_inputs(w, lengths=lens)
+    compare(mdn, inp, "simt", label="packed")
+    wb = dataclasses.replace(w, dtype="bf16", dk=128, dv=128)
+    inpb = wl.make_inputs(wb, lengths=lens)
+    for path in paths_for(mdn, wb):
+        compare(mdn, inpb, path, label="packed bf16")
+
+
+def test_packed_equals_separate_calls_bitwise(mdn):
+    """A packed call must give, for each sequence, exactly what a call on that sequence alone gives."""
+    import torch
+    lens = np.array([70, 5, 200])
+    w = small(B=1, T=int(lens.sum()), varlen=True)
+    inp = wl.make_inputs(w, lengths=lens)
+    o, S, M = run_gpu(mdn, inp, path="simt")
+    for n, (s, l) in enumerate(zip(inp["seq_start"], inp["seq_len"])):
+        sub = dict(inp)
+        for name in ("q", "k", "v", "beta", "log_alpha", "log_mu", "eta"):
+            sub[name] = inp[name][:, s:s + l]
+        sub["cu_seqlens"] = None
+        sub["workload"] = dataclasses.replace(w, T=int(l), varlen=False)
+        o1, S1, M1 = run_gpu(mdn, sub, path="simt")
+        assert np.array_equal(o[:, s:s + l], o1) and np.array_equal(S[n], S1[0]) and np.array_equal(M[n], M1[0])
+
+
+def test_state_handoff_and_determinism(mdn):
+    w = small(T=256, init_state_std=0.1)
+    inp = wl.make_inputs(w)
+    o, S, M = run_gpu(mdn, inp, path="simt")
+    o2, S2, M2 = run_gpu(mdn, inp, path="simt")
+    assert np.array_equal(o, o2) and np.array_equal(S, S2) and np.array_equal(M, M2)     # no atomics on the path
+    a = dict(inp); b = dict(inp)
+    for name in ("q", "k", "v", "beta", "log_alpha", "log_mu", "eta"):
+        a[name] = inp[name][:, :128]; b[name] = inp[name][:, 128:]
+    a["workload"] = b["workload"] = dataclasses.replace(w, T=128)
+    oa, Sa, Ma = run_gpu(mdn, a, path="simt")
+    b["S0"], b["M0"] = Sa.astype(np.float32), Ma.astype(np.float32)
+    ob, Sb, Mb = run_gpu(mdn, b, path="simt")
+    # the split falls on a chunk boundary, so the two calls do the same arithmetic
+    assert np.array_equal(o[:, :128], oa) and np.array_equal(o[:, 128:], ob)
+    assert np.array_equal(S, Sb) and np.array_equal(M, Mb)
+
+
+def test_bad_cu_seqlens_is_reported_not_faulted(mdn):
+    import torch
+    w = small(B=1, T=128, varlen=True)
+    inp = wl.make_inputs(w, lengths=np.array([100, 28]))
+    t = to_torch(inp)
+    bad = torch.tensor([0, 100, 90], dtype=torch.int32, device="cuda")      # decreasing, and cu[N] != T
+    p = mdn.make_params(t["q"], t["v"], num_seqs=2)
+    ws = torch.zeros(mdn.workspace_bytes(p), dtype=torch.uint8, device="cuda")
+    o, S, M = mdn.chunk_fwd(t["q"], t["k"], t["v"], t["beta"], t["log_alpha"], t["log_mu"], t["eta"],
+                            cu_seqlens=bad, workspace=ws)
+    torch.cuda.synchronize()
+    assert mdn.status_string(mdn.read_status(p, ws)) == "invalid argument"
+    good = t["cu_seqlens"]
+    mdn.chunk_fwd(t["q"], t["k"], t["v"], t["beta"], t["log_alpha"], t["log_mu"], t["eta"], cu_seqlens=good,
+                  workspace=ws)
+    assert mdn.read_status(p, ws) == 0
+
+
+def test_host_buffer_entry_point(mdn):
+    w = small(T=130, init_state_std=0.2)
+    inp = wl.make_inputs(w)
+    t = to_torch(inp, host_pinned=True)
+    o, S, M = mdn.chunk_fwd_host(t["q"], t["k"], t["v"], t["beta"], t["log_alpha"], t["log_mu"], t["eta"],
+                                 initial_S=t["initial_S"], initial_M=t["initial_M"], scale=inp["scale"], path="simt")
+    o_d, S_d, M_d = run_gpu(mdn, inp, path="simt")
+    assert np.array_equal(o.numpy(), o_d) and np.array_equal(S.numpy(), S_d) and np.array_equal(M.numpy(), M_d)
