@@ -174,6 +174,19 @@ const char* mdn_status_string(mdn_status s);
 #define MDN_NUM_STAGE_EVENTS 4
 mdn_status mdn_set_stage_events(void* const* events /* host */, int32_t n);
 
+/*
+ * Diagnostic: runs one small tcgen05 / TMA case on one CTA (the operand configurations the
+ * tensor-core chain kernel uses) so that each can be checked against a host matmul.
+ *   mode 0: TMA 128-byte-swizzled load of a [64 x 128] bf16 matrix `a`; out = the raw 16 KB of shared memory
+ *   mode 1: out[128 x 64]  = a[128 x 128] * b[64 x 128]^T     (A and B from shared memory, K-major)
+ *   mode 2: out[128 x 64]  = a[128 x 64]  * b[64 x 64]^T      (A from tensor memory)
+ *   mode 3: out[128 x 128] = 1 - a[128 x 64] * b[64 x 128]    (A from tensor memory, negated; B MN-major via TMA;
+ *                                                              accumulating onto a preloaded D)
+ * a, b: bf16 row-major device buffers; out: float32 device buffer; status: device int32 (0 = ok).
+ */
+mdn_status mdn_selftest_umma(int32_t mode, const void* a, const void* b, float* out, int32_t* status,
+                             void* cuda_stream);
+
 /* Number of kernels the last mdn_* call on this host thread enqueued. */
 int32_t mdn_last_launch_count(void);
 
