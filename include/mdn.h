@@ -125,7 +125,7 @@ mdn_status mdn_chunk_fwd_host(const mdn_params* p,
  * mdn_coeff_scan (a0 + a1, Eq. 10): for every chunk slot s and head h, ten float32
  * vectors of length 64 at  coef + ((s*H + h)*MDN_NUM_COEF + i)*64 :
  *   i=0 abar_r   1 b_r   2 alpha_r*b_{r-1}   3 gamma_{last,r}*eta_r   4 (mubar_last/mubar_r)*eta_r
- *   5 alpha_r    6 beta_r   7 mu_r   8 eta_r   9 mubar_r
+ *   5 mubar_r    6 alpha_r  7 beta_r   8 mu_r   9 eta_r
  * Positions past the end of a short chunk hold exact no-ops (alpha = mu = 1, beta = eta = 0).
  *
  * mdn_intra_chunk (a2, Eq. 15 and the mask of Eq. 12): per (s, h) the 64x64 row-major

@@ -52,7 +52,7 @@ __global__ void __launch_bounds__(kChainThreads) chain_simt_kernel(
   float* Vt = Rs + C * NV;        // [64][NV]
   float* Tm = Vt + C * NV;        // [64][65]
   float* Wm = Tm + C * LM;        // [64][65]
-  float* cv = Wm + C * LM;        // [5][64] abar, b, alpha*b_prev, gS, gM ; [320] = mubar_last
+  float* cv = Wm + C * LM;        // [6][64] abar, b, alpha*b_prev, gS, gM, mubar
 
   const int tid = threadIdx.x, j = tid % NV, rg = tid / NV;
   const int vb = blockIdx.x % NVB, h = (blockIdx.x / NVB) % g.H, seq = blockIdx.x / (NVB * g.H);
@@ -80,8 +80,7 @@ __global__ void __launch_bounds__(kChainThreads) chain_simt_kernel(
       Wm[(idx >> 6) * LM + (idx & 63)] = Wmat[mat + idx];
     }
     const float* cf = coef + ((size_t)slot * g.H + h) * MDN_NUM_COEF * C;
-    for (int idx = tid; idx < 5 * C; idx += kChainThreads) cv[idx] = cf[idx];   // vectors 0..4 are contiguous
-    if (tid == 0) cv[5 * C] = cf[kMubar * C + C - 1];
+    for (int idx = tid; idx < kChainCoefs * C; idx += kChainThreads) cv[idx] = cf[idx];   // vectors 0..5 are contiguous
     __syncthreads();
 
     // ---- phase 1: K S, K M, Q S, Q M for rows rg + 8 i, column j
@@ -152,7 +151,7 @@ __global__ void __launch_bounds__(kChainThreads) chain_simt_kernel(
     }
     // every thread finished reading the old state two barriers ago, and each (d, j) entry is
     // updated by the one thread that owns it: no barrier needed before the write
-    const float abar_l = cv[kAbar * C + C - 1], b_l = cv[kB * C + C - 1], mubar_l = cv[5 * C];
+    const float abar_l = cv[kAbar * C + C - 1], b_l = cv[kB * C + C - 1], mubar_l = cv[kMubar * C + C - 1];
 #pragma unroll
     for (int i = 0; i < DPT; ++i) {
       const int d = rg + 8 * i;
@@ -172,7 +171,7 @@ __global__ void __launch_bounds__(kChainThreads) chain_simt_kernel(
 template <typename TIn, typename TO, int DK, int DV>
 static cudaError_t launch_one(const Plan& pl, const void* q, const void* k, const void* v, const float* S0,
                               const float* M0, void* o, float* Sf, float* Mf) {
-  const size_t smem = (size_t)(2 * DK * kNV + 2 * C * (DK + 1) + 2 * C * kNV + 2 * C * (C + 1) + 5 * C + 4) * sizeof(float);
+  const size_t smem = (size_t)(2 * DK * kNV + 2 * C * (DK + 1) + 2 * C * kNV + 2 * C * (C + 1) + kChainCoefs * C) * sizeof(float);
   auto kern = chain_simt_kernel<TIn, TO, DK, DV>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;

@@ -18,12 +18,13 @@ enum Coef : int {
   kAlphaBPrev = 2,  // alpha_r * b_{r-1}          (weight of +K M_[t] in the right-hand side)
   kGS = 3,      // gamma_{last,r} * eta_r         (weight of k_r v~_r^T in S_[t+1])
   kGM = 4,      // (mubar_last/mubar_r) * eta_r   (weight of -k_r v~_r^T in M_[t+1])
-  kAlpha = 5,
-  kBeta = 6,
-  kMu = 7,
-  kEta = 8,
-  kMubar = 9
+  kMubar = 5,   // mubar_r = prod_{j<=r} mu_j   (vectors 0..5 are what the chain kernels read)
+  kAlpha = 6,
+  kBeta = 7,
+  kMu = 8,
+  kEta = 9
 };
+constexpr int kChainCoefs = 6;
 
 // Device-side error codes written to the workspace status word.
 enum DevErr : int { kDevOk = 0, kDevBadCuSeqlens = 1, kDevTimeout = 2 };

@@ -101,7 +101,7 @@ def test_coefficient_scan_matches_eq10(mdn):
                     Mm = np.tril(mubar[:, None] / mubar[None, :])
                 got = coef[b * nchunks + c, h]
                 tol = dict(rtol=2e-5, atol=1e-7)
-                assert np.allclose(got[0, :n], abar, **tol) and np.allclose(got[9, :n], mubar, **tol)
+                assert np.allclose(got[0, :n], abar, **tol) and np.allclose(got[5, :n], mubar, **tol)
                 assert np.allclose(got[1, :n], bb, **tol)
                 b_prev = np.concatenate([[0.0], bb[:-1]])
                 assert np.allclose(got[2, :n], np.exp(la.astype(np.float64)) * b_prev, **tol)
@@ -110,7 +110,7 @@ def test_coefficient_scan_matches_eq10(mdn):
                 # exact no-ops past the end of a short chunk; last entries equal the last valid ones
                 assert (got[3, n:] == 0).all() and (got[4, n:] == 0).all()
                 assert np.allclose(got[0, 63], abar[-1], **tol) and np.allclose(got[1, 63], bb[-1], **tol)
-                assert np.allclose(got[9, 63], mubar[-1], **tol)
+                assert np.allclose(got[5, 63], mubar[-1], **tol)
 
 
 def test_intra_chunk_T_and_W_match_eq15(mdn):
