@@ -259,7 +259,7 @@ def run_ours(args, w):
 
     # end to end through the host-buffer entry point (pinned host memory, copies inside the timed region)
     e2e = None
-    if rank == 0 or world > 1:
+    if not args.no_e2e:
         th = to_torch(inp, host_pinned=True)
         arena = torch.empty(mdn.host_arena_bytes(p), dtype=torch.uint8, device=t["q"].device)
         nst = N
@@ -326,6 +326,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--path", default="auto", choices=["auto", "simt", "tensor"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg (profiling runs)")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     args = ap.parse_args()
     w = wl.CONFIGS[args.config]
