@@ -449,7 +449,7 @@ bool tensor_path_supported(const mdn_params& p) {
 }
 
 cudaError_t launch_intra_tensor(const Plan& pl, const void* q, const void* k, int* launches) {
-  return launch_intra_simt(pl, q, k, launches);   // bf16 T, W_hi, W_lo (layout says mat_dtype = bf16)
+  return launch_intra_mma(pl, q, k, launches);
 }
 
 cudaError_t launch_chain_tensor(const Plan& pl, const void* q, const void* k, const void* v, const float* S0,

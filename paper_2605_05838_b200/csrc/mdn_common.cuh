@@ -107,6 +107,7 @@ cudaError_t launch_chain_simt(const Plan& pl, const void* q, const void* k, cons
 // Tensor-core (tcgen05) path: bf16 q/k/v, dk = dv = 128.
 bool tensor_path_supported(const mdn_params& p);
 cudaError_t launch_intra_tensor(const Plan& pl, const void* q, const void* k, int* launches);
+cudaError_t launch_intra_mma(const Plan& pl, const void* q, const void* k, int* launches);
 cudaError_t launch_chain_tensor(const Plan& pl, const void* q, const void* k, const void* v,
                                 const float* S0, const float* M0, void* o, float* Sf, float* Mf,
                                 int* launches);
