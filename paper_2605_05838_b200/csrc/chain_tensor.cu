@@ -26,6 +26,7 @@
 // 8 TMA producer (2-stage ring: K, Q, V, T, W_hi, W_lo, 6 coefficient vectors per chunk);
 // 9 MMA issuer (one elected lane) and tensor-memory owner.  All hand-offs are mbarriers with
 // bounded waits; tensor-memory column reuse is ordered by those same barriers.
+#include <cstdlib>
 #include <cstring>
 
 #include "mdn_common.cuh"
@@ -77,7 +78,13 @@ struct ChainArgs {
   int32_t* status;
   float scale;
   uint32_t w_lo_row_offset;   // rows between the hi and lo parts in the W tensor map
+  uint32_t drop_lo;           // debug: bit 0 R, 1 V~_S/V~_M, 2 V~ (output), 3 W: leave that operand's lo part out
+  long long* timeline;        // debug: CTA 0 writes clock64() at [chunk*32 + event] (NULL = off)
 };
+
+// Timeline events (debug).
+enum Ev : int { kEvMmaStart = 0, kEvM1Seen, kEvRArrive, kEvM2Seen, kEvVArrive, kEvM3Seen, kEvSbArrive, kEvMqSeen,
+                kEvZqArrive, kEvMoSeen, kEvZuArrive, kEvMmaIssued, kEvRSeen, kEvVSeen, kEvTmaIssued, kEvFullSeen, kEvStoresDone };
 
 __device__ __forceinline__ void split_bf16(float x, float& hi, float& lo) {
   hi = bf16_round(x);
@@ -141,6 +148,10 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
     break;                                         \
   }
 
+  long long* const tline = (blockIdx.x == 0) ? a.timeline : nullptr;
+#define MDN_MARK(c, ev)                                                      \
+  if (tline != nullptr && lane == 0 && (warp & 3) == ((warp < 8) ? 0 : (warp & 3))) tline[(c) * 32 + (ev)] = clock64();
+
   if (warp == kWarpTma) {
     // ================================================================== TMA producer
     if (lane == 0) {
@@ -162,6 +173,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
         tma_load_2d(st + kStQ + 8192, &map_q, h * kD + 64, tok0, fb);
         tma_load_2d(st + kStWh, &map_w, 0, mat * C, fb);
         tma_load_2d(st + kStWl, &map_w, 0, mat * C + (int)a.w_lo_row_offset, fb);
+        MDN_MARK(c, kEvTmaIssued);
         issued = c + 1;
       }
       if (!ok) {   // giving up: let the copies already in flight land before the CTA exits
@@ -184,6 +196,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
         MDN_WAIT(s ? b_full1 : b_full0, (c >> 1) & 1);
         MDN_WAIT(b_sb, ph);
         tc_fence_after_sync();
+        MDN_MARK(c, kEvMmaStart);
         // ---- MMA-1a: X = S_b K^T, Y = M_b K^T
 #pragma unroll
         for (int k = 0; k < 8; ++k)
@@ -209,22 +222,25 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
         // ---- MMA-2: Y = (R_hi + R_lo)^T T^T
         MDN_WAIT(b_r, ph);
         tc_fence_after_sync();
+        MDN_MARK(c, kEvRSeen);
 #pragma unroll
         for (int k = 0; k < 4; ++k)
           umma_ts(tmem + kColY, tmem + kColX + k * 8, smem_desc_sw128(sT + k * 32, 16, 1024), id64, k > 0);
+        if (!(a.drop_lo & 1u)) {
 #pragma unroll
-        for (int k = 0; k < 4; ++k)
-          umma_ts(tmem + kColY, tmem + kColX + 32 + k * 8, smem_desc_sw128(sT + k * 32, 16, 1024), id64, true);
+          for (int k = 0; k < 4; ++k)
+            umma_ts(tmem + kColY, tmem + kColX + 32 + k * 8, smem_desc_sw128(sT + k * 32, 16, 1024), id64, true);
+        }
         umma_commit(b_m2);
         // ---- MMA-3: S^T += V~_S^T K, M^T -= V~_M^T K   (K tile read MN-major: N = dk, K = tokens)
         MDN_WAIT(b_v, ph);
         tc_fence_after_sync();
-#pragma unroll
-        for (int k = 0; k < 8; ++k)
+        MDN_MARK(c, kEvVSeen);
+        const int n3 = (a.drop_lo & 2u) ? 4 : 8;
+        for (int k = 0; k < n3; ++k)
           umma_ts(tmem + kColS, tmem + kColX + (k >> 2) * 32 + (k & 3) * 8,
                   smem_desc_sw128(sK + (k & 3) * 2048, 8192, 1024), id128_mn, true);
-#pragma unroll
-        for (int k = 0; k < 8; ++k)
+        for (int k = 0; k < n3; ++k)
           umma_ts(tmem + kColM, tmem + kColY + (k >> 2) * 32 + (k & 3) * 8,
                   smem_desc_sw128(sK + (k & 3) * 2048, 8192, 1024), id128_mn_neg, true);
         umma_commit(b_m3);
@@ -232,13 +248,18 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
 #pragma unroll
         for (int k = 0; k < 4; ++k)
           umma_ts(tmem + kColU, tmem + kColZ + k * 8, smem_desc_sw128(sWh + k * 32, 16, 1024), id64, k > 0);
+        if (!(a.drop_lo & 4u)) {
 #pragma unroll
-        for (int k = 0; k < 4; ++k)
-          umma_ts(tmem + kColU, tmem + kColZ + 32 + k * 8, smem_desc_sw128(sWh + k * 32, 16, 1024), id64, true);
+          for (int k = 0; k < 4; ++k)
+            umma_ts(tmem + kColU, tmem + kColZ + 32 + k * 8, smem_desc_sw128(sWh + k * 32, 16, 1024), id64, true);
+        }
+        if (!(a.drop_lo & 8u)) {
 #pragma unroll
-        for (int k = 0; k < 4; ++k)
-          umma_ts(tmem + kColU, tmem + kColZ + k * 8, smem_desc_sw128(sWl + k * 32, 16, 1024), id64, true);
+          for (int k = 0; k < 4; ++k)
+            umma_ts(tmem + kColU, tmem + kColZ + k * 8, smem_desc_sw128(sWl + k * 32, 16, 1024), id64, true);
+        }
         umma_commit(b_mo);
+        MDN_MARK(c, kEvMmaIssued);
       }
     }
   } else if (warp < 4) {
@@ -250,11 +271,13 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
       float al = 0.f, bl = 0.f, ml = 0.f;
       if (c > 0) {
         MDN_WAIT(b_m3, (c - 1) & 1);
+        MDN_MARK(c - 1, kEvM3Seen);
       }
       if (c < nch) {
         MDN_WAIT((c & 1) ? b_full1 : b_full0, (c >> 1) & 1);
         const float* cf = reinterpret_cast<const float*>(smem + kOffStage + (c & 1) * kStageBytes + kStCoef);
         al = cf[kAbar * C + C - 1]; bl = cf[kB * C + C - 1]; ml = cf[kMubar * C + C - 1];
+        MDN_MARK(c, kEvFullSeen);
       }
       __syncwarp();
       tc_fence_after_sync();
@@ -311,6 +334,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
       fence_proxy_async_smem();
       tc_fence_before_sync();
       mbar_arrive(b_sb);
+      MDN_MARK(c, kEvSbArrive);
 
       const uint32_t ph = c & 1;
       const uint8_t* stg = smem + kOffStage + (c & 1) * kStageBytes;
@@ -320,6 +344,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
       MDN_WAIT(b_m1, ph);
       __syncwarp();
       tc_fence_after_sync();
+      MDN_MARK(c, kEvM1Seen);
       {
         uint32_t hi[32], lo[32];
 #pragma unroll
@@ -349,11 +374,13 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
       }
       tc_fence_before_sync();
       mbar_arrive(b_r);
+      MDN_MARK(c, kEvRArrive);
       // ---------------- EPI-2: V~ -> (gamma_C eta) V~, ((mubar_C/mubar) eta) V~, V~ as bf16 hi, lo
       MDN_WAIT(b_m2, ph);
       MDN_WAIT(b_zq, ph);
       __syncwarp();
       tc_fence_after_sync();
+      MDN_MARK(c, kEvM2Seen);
       {
         uint32_t vt[64];
         tmem_ld32(tl + kColY, *reinterpret_cast<uint32_t(*)[32]>(&vt[0]));
@@ -384,6 +411,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
       }
       tc_fence_before_sync();
       mbar_arrive(b_v);
+      MDN_MARK(c, kEvVArrive);
       mbar_arrive((c & 1) ? b_empty1 : b_empty0);
     }
   } else {
@@ -400,6 +428,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
       MDN_WAIT(b_mq, ph);
       __syncwarp();
       tc_fence_after_sync();
+      MDN_MARK(c, kEvMqSeen);
       float oi[64];
 #pragma unroll
       for (int hh = 0; hh < 2; ++hh) {
@@ -415,26 +444,37 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
       }
       tc_fence_before_sync();
       mbar_arrive(b_zq);
+      MDN_MARK(c, kEvZqArrive);
       MDN_WAIT(b_mo, ph);
       __syncwarp();
       tc_fence_after_sync();
-#pragma unroll
-      for (int hh = 0; hh < 2; ++hh) {
-        uint32_t u[32];
-        tmem_ld32(tl + kColU + hh * 32, u);
+      MDN_MARK(c, kEvMoSeen);
+      {
+        uint32_t u[64];
+        tmem_ld32(tl + kColU, *reinterpret_cast<uint32_t(*)[32]>(&u[0]));
+        tmem_ld32(tl + kColU + 32, *reinterpret_cast<uint32_t(*)[32]>(&u[32]));
         tmem_wait_ld();
+        // U and this stage's coefficients are in registers: hand both back before the global stores
+        tc_fence_before_sync();
+        mbar_arrive(b_zu);
+        mbar_arrive((c & 1) ? b_empty1 : b_empty0);
+        MDN_MARK(c, kEvZuArrive);
+        if (!(a.drop_lo & 16u)) {
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          const int r = hh * 32 + j;
-          if (r < n) store_o<TO>(o + (tok + (size_t)r * H) * kD + d, oi[r] + __uint_as_float(u[j]));
+          for (int r = 0; r < 64; ++r)
+            if (r < n) store_o<TO>(o + (tok + (size_t)r * H) * kD + d, oi[r] + __uint_as_float(u[r]));
+        } else {   // debug: one store per thread instead of 64
+          float acc = 0.f;
+#pragma unroll
+          for (int r = 0; r < 64; ++r) acc += oi[r] + __uint_as_float(u[r]);
+          store_o<TO>(o + tok * kD + d, acc);
         }
+        MDN_MARK(c, kEvStoresDone);
       }
-      tc_fence_before_sync();
-      mbar_arrive(b_zu);
-      mbar_arrive((c & 1) ? b_empty1 : b_empty0);
     }
   }
 #undef MDN_WAIT
+#undef MDN_MARK
 
   if (!ok && lane == 0) atomicCAS(a.status, kDevOk, kDevTimeout);
   tc_fence_before_sync();
@@ -472,6 +512,10 @@ cudaError_t launch_chain_tensor(const Plan& pl, const void* q, const void* k, co
   a.status = reinterpret_cast<int32_t*>(pl.ws + pl.lay.off_status);
   a.scale = p.scale;
   a.w_lo_row_offset = (uint32_t)(mats * C);
+  const char* drop = getenv("MDN_DEBUG_DROP_LO");
+  a.drop_lo = drop ? (uint32_t)atoi(drop) : 0u;
+  const char* tl = getenv("MDN_DEBUG_TIMELINE");   // device address of an int64 buffer, [chunks][32]
+  a.timeline = tl ? reinterpret_cast<long long*>(strtoull(tl, nullptr, 0)) : nullptr;
   const unsigned grid = (unsigned)pl.geom.num_seqs * p.H;
   cudaError_t e;
   if (p.o_dtype == MDN_BF16) {
