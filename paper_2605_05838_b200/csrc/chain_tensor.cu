@@ -38,8 +38,8 @@ namespace {
 using namespace tc;
 
 constexpr int kD = 128;
-constexpr int kThreads = 320;
-constexpr int kWarpTma = 8, kWarpMma = 9;
+constexpr int kThreads = 448;
+constexpr int kWarpEpiB = 8, kWarpTma = 12, kWarpMma = 13;
 
 // shared memory (offsets from a 1024-byte aligned base)
 constexpr uint32_t kOffSb = 0, kOffMb = 32768, kOffStage = 65536;
@@ -55,16 +55,19 @@ constexpr uint32_t kColS = 0, kColM = 128, kColX = 256, kColY = 320, kColZ = 384
 
 struct Bars {
   uint64_t full[2], empty[2];
-  uint64_t sb;   // P(c) done: S_b, M_b in smem, scaled masters in tensor memory     (128 arrivals)
+  uint64_t sb;   // P(c): S_b, M_b in smem                                            (256 arrivals)
   uint64_t m1;   // MMA-1a done                                                      (commit)
   uint64_t mq;   // MMA-1b done                                                      (commit)
-  uint64_t r;    // EPI-1 done: R^T hi/lo in X                                        (128)
+  uint64_t r;    // EPI-1 done: R^T hi/lo in X                                        (256)
   uint64_t m2;   // MMA-2 done                                                       (commit)
   uint64_t zq;   // output epilogue has read Z, U (Q S, Q M)                          (128)
-  uint64_t v;    // EPI-2 done: V~_S, V~_M, V~ operands in X, Y, Z                    (128)
+  uint64_t v1;   // EPI-2a done: V~_S, V~_M operands in X, Y; masters pre-scaled      (256)
+  uint64_t v2;   // EPI-2b done: V~ operand in Z                                      (256)
   uint64_t m3;   // MMA-3 done                                                       (commit)
   uint64_t mo;   // MMA-3' done                                                      (commit)
   uint64_t zu;   // output epilogue has read U (intra-chunk output)                   (128)
+  uint64_t ga;   // critical-path epilogue group sync                                 (256)
+  uint64_t gb;   // output epilogue group sync                                        (128)
 };
 
 struct ChainArgs {
@@ -84,16 +87,16 @@ struct ChainArgs {
 
 // Timeline events (debug).
 enum Ev : int { kEvMmaStart = 0, kEvM1Seen, kEvRArrive, kEvM2Seen, kEvVArrive, kEvM3Seen, kEvSbArrive, kEvMqSeen,
-                kEvZqArrive, kEvMoSeen, kEvZuArrive, kEvMmaIssued, kEvRSeen, kEvVSeen, kEvTmaIssued, kEvFullSeen, kEvStoresDone };
+                kEvZqArrive, kEvMoSeen, kEvZuArrive, kEvMmaIssued, kEvRSeen, kEvVSeen, kEvTmaIssued, kEvFullSeen,
+                kEvStoresDone, kEvV2Arrive, kEvPrescaled, kEvE1Loaded, kEvE1Math, kEvE1Sync, kEvE1Stored, kEvPLoaded, kEvPStored };
 
-__device__ __forceinline__ void split_bf16(float x, float& hi, float& lo) {
-  hi = bf16_round(x);
-  lo = x - hi;
+template <typename TO> __device__ __forceinline__ void stage_o(uint8_t* tile, int r, int d, float x);
+template <> __device__ __forceinline__ void stage_o<float>(uint8_t* tile, int r, int d, float x) {
+  reinterpret_cast<float*>(tile)[r * kD + d] = x;
 }
-
-template <typename TO> __device__ __forceinline__ void store_o(TO* p, float x);
-template <> __device__ __forceinline__ void store_o<float>(float* p, float x) { *p = x; }
-template <> __device__ __forceinline__ void store_o<__nv_bfloat16>(__nv_bfloat16* p, float x) { *p = __float2bfloat16_rn(x); }
+template <> __device__ __forceinline__ void stage_o<__nv_bfloat16>(uint8_t* tile, int r, int d, float x) {
+  reinterpret_cast<__nv_bfloat16*>(tile)[r * kD + d] = __float2bfloat16_rn(x);
+}
 
 template <typename TO>
 __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainArgs a,
@@ -101,7 +104,8 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
                                                                   const __grid_constant__ CUtensorMap map_k,
                                                                   const __grid_constant__ CUtensorMap map_v,
                                                                   const __grid_constant__ CUtensorMap map_t,
-                                                                  const __grid_constant__ CUtensorMap map_w) {
+                                                                  const __grid_constant__ CUtensorMap map_w,
+                                                                  const __grid_constant__ CUtensorMap map_o) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   __shared__ __align__(8) Bars bars;
@@ -120,21 +124,23 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
   const uint32_t b_empty0 = smem_u32(&bars.empty[0]), b_empty1 = smem_u32(&bars.empty[1]);
   const uint32_t b_sb = smem_u32(&bars.sb), b_m1 = smem_u32(&bars.m1), b_mq = smem_u32(&bars.mq);
   const uint32_t b_r = smem_u32(&bars.r), b_m2 = smem_u32(&bars.m2), b_zq = smem_u32(&bars.zq);
-  const uint32_t b_v = smem_u32(&bars.v), b_m3 = smem_u32(&bars.m3), b_mo = smem_u32(&bars.mo);
-  const uint32_t b_zu = smem_u32(&bars.zu);
+  const uint32_t b_v1 = smem_u32(&bars.v1), b_v2 = smem_u32(&bars.v2), b_m3 = smem_u32(&bars.m3);
+  const uint32_t b_mo = smem_u32(&bars.mo), b_zu = smem_u32(&bars.zu);
+  const uint32_t b_ga = smem_u32(&bars.ga), b_gb = smem_u32(&bars.gb);
 
   if (tid == 0) {
     abort_flag = 0;
     mbar_init(b_full0, 1); mbar_init(b_full1, 1);
-    mbar_init(b_empty0, 256); mbar_init(b_empty1, 256);
-    mbar_init(b_sb, 128); mbar_init(b_r, 128); mbar_init(b_zq, 128); mbar_init(b_v, 128); mbar_init(b_zu, 128);
+    mbar_init(b_empty0, 257); mbar_init(b_empty1, 257);
+    mbar_init(b_sb, 256); mbar_init(b_r, 256); mbar_init(b_v1, 256); mbar_init(b_v2, 256); mbar_init(b_ga, 256);
+    mbar_init(b_zq, 128); mbar_init(b_zu, 128); mbar_init(b_gb, 128);
     mbar_init(b_m1, 1); mbar_init(b_mq, 1); mbar_init(b_m2, 1); mbar_init(b_m3, 1); mbar_init(b_mo, 1);
     mbar_fence_init();
   }
   if (warp == kWarpMma) tmem_alloc(smem_u32(&tmem_slot), 512);
   if (warp == kWarpTma && lane == 0) {
     prefetch_tensormap(&map_q); prefetch_tensormap(&map_k); prefetch_tensormap(&map_v);
-    prefetch_tensormap(&map_t); prefetch_tensormap(&map_w);
+    prefetch_tensormap(&map_t); prefetch_tensormap(&map_w); prefetch_tensormap(&map_o);
   }
   tc_fence_before_sync();
   __syncthreads();
@@ -147,10 +153,10 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
     ok = false;                                    \
     break;                                         \
   }
-
   long long* const tline = (blockIdx.x == 0) ? a.timeline : nullptr;
-#define MDN_MARK(c, ev)                                                      \
-  if (tline != nullptr && lane == 0 && (warp & 3) == ((warp < 8) ? 0 : (warp & 3))) tline[(c) * 32 + (ev)] = clock64();
+#define MDN_MARK(c, ev) \
+  if (tline != nullptr && lane == 0 && (warp == 0 || warp >= kWarpEpiB) && (warp & 3) == (warp >= kWarpTma ? (warp & 3) : 0)) \
+    tline[(c) * 32 + (ev)] = clock64();
 
   if (warp == kWarpTma) {
     // ================================================================== TMA producer
@@ -187,12 +193,18 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
       const uint32_t id64 = idesc_bf16(128, 64, false, false, false);
       const uint32_t id128_mn = idesc_bf16(128, 128, false, true, false);
       const uint32_t id128_mn_neg = idesc_bf16(128, 128, false, true, true);
-      const uint32_t sSb = s_base + kOffSb, sMb = s_base + kOffMb;
+      // descriptors: bases are fixed; stepping K by 16 elements = +32 bytes = +2 in the address field
+      const uint64_t dSb0 = smem_desc_sw128(s_base + kOffSb, 16, 1024), dSb1 = smem_desc_sw128(s_base + kOffSb + 16384, 16, 1024);
+      const uint64_t dMb0 = smem_desc_sw128(s_base + kOffMb, 16, 1024), dMb1 = smem_desc_sw128(s_base + kOffMb + 16384, 16, 1024);
       for (int c = 0; c < nch; ++c) {
         const int s = c & 1;
         const uint32_t ph = c & 1;
         const uint32_t st = s_base + kOffStage + s * kStageBytes;
-        const uint32_t sK = st + kStK, sQ = st + kStQ, sT = st + kStT, sWh = st + kStWh, sWl = st + kStWl;
+        const uint64_t dK0 = smem_desc_sw128(st + kStK, 16, 1024), dK1 = smem_desc_sw128(st + kStK + 8192, 16, 1024);
+        const uint64_t dQ0 = smem_desc_sw128(st + kStQ, 16, 1024), dQ1 = smem_desc_sw128(st + kStQ + 8192, 16, 1024);
+        const uint64_t dT = smem_desc_sw128(st + kStT, 16, 1024);
+        const uint64_t dWh = smem_desc_sw128(st + kStWh, 16, 1024), dWl = smem_desc_sw128(st + kStWl, 16, 1024);
+        const uint64_t dKmn = smem_desc_sw128(st + kStK, 8192, 1024);   // K tile read MN-major; +2048 B per 16 tokens
         MDN_WAIT(s ? b_full1 : b_full0, (c >> 1) & 1);
         MDN_WAIT(b_sb, ph);
         tc_fence_after_sync();
@@ -200,74 +212,68 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
         // ---- MMA-1a: X = S_b K^T, Y = M_b K^T
 #pragma unroll
         for (int k = 0; k < 8; ++k)
-          umma_ss(tmem + kColX, smem_desc_sw128(sSb + (k >> 2) * 16384 + (k & 3) * 32, 16, 1024),
-                  smem_desc_sw128(sK + (k >> 2) * 8192 + (k & 3) * 32, 16, 1024), id64, k > 0);
+          umma_ss(tmem + kColX, ((k >> 2) ? dSb1 : dSb0) + 2 * (k & 3), ((k >> 2) ? dK1 : dK0) + 2 * (k & 3), id64, k > 0);
 #pragma unroll
         for (int k = 0; k < 8; ++k)
-          umma_ss(tmem + kColY, smem_desc_sw128(sMb + (k >> 2) * 16384 + (k & 3) * 32, 16, 1024),
-                  smem_desc_sw128(sK + (k >> 2) * 8192 + (k & 3) * 32, 16, 1024), id64, k > 0);
+          umma_ss(tmem + kColY, ((k >> 2) ? dMb1 : dMb0) + 2 * (k & 3), ((k >> 2) ? dK1 : dK0) + 2 * (k & 3), id64, k > 0);
         umma_commit(b_m1);
         // ---- MMA-1b: Z = S_b Q^T, U = M_b Q^T (Z, U must have been drained by the output epilogue)
         MDN_WAIT(b_zu, ph ^ 1);
         tc_fence_after_sync();
 #pragma unroll
         for (int k = 0; k < 8; ++k)
-          umma_ss(tmem + kColZ, smem_desc_sw128(sSb + (k >> 2) * 16384 + (k & 3) * 32, 16, 1024),
-                  smem_desc_sw128(sQ + (k >> 2) * 8192 + (k & 3) * 32, 16, 1024), id64, k > 0);
+          umma_ss(tmem + kColZ, ((k >> 2) ? dSb1 : dSb0) + 2 * (k & 3), ((k >> 2) ? dQ1 : dQ0) + 2 * (k & 3), id64, k > 0);
 #pragma unroll
         for (int k = 0; k < 8; ++k)
-          umma_ss(tmem + kColU, smem_desc_sw128(sMb + (k >> 2) * 16384 + (k & 3) * 32, 16, 1024),
-                  smem_desc_sw128(sQ + (k >> 2) * 8192 + (k & 3) * 32, 16, 1024), id64, k > 0);
+          umma_ss(tmem + kColU, ((k >> 2) ? dMb1 : dMb0) + 2 * (k & 3), ((k >> 2) ? dQ1 : dQ0) + 2 * (k & 3), id64, k > 0);
         umma_commit(b_mq);
         // ---- MMA-2: Y = (R_hi + R_lo)^T T^T
         MDN_WAIT(b_r, ph);
         tc_fence_after_sync();
         MDN_MARK(c, kEvRSeen);
 #pragma unroll
-        for (int k = 0; k < 4; ++k)
-          umma_ts(tmem + kColY, tmem + kColX + k * 8, smem_desc_sw128(sT + k * 32, 16, 1024), id64, k > 0);
+        for (int k = 0; k < 4; ++k) umma_ts(tmem + kColY, tmem + kColX + k * 8, dT + 2 * k, id64, k > 0);
         if (!(a.drop_lo & 1u)) {
 #pragma unroll
-          for (int k = 0; k < 4; ++k)
-            umma_ts(tmem + kColY, tmem + kColX + 32 + k * 8, smem_desc_sw128(sT + k * 32, 16, 1024), id64, true);
+          for (int k = 0; k < 4; ++k) umma_ts(tmem + kColY, tmem + kColX + 32 + k * 8, dT + 2 * k, id64, true);
         }
         umma_commit(b_m2);
         // ---- MMA-3: S^T += V~_S^T K, M^T -= V~_M^T K   (K tile read MN-major: N = dk, K = tokens)
-        MDN_WAIT(b_v, ph);
+        MDN_WAIT(b_v1, ph);
         tc_fence_after_sync();
         MDN_MARK(c, kEvVSeen);
         const int n3 = (a.drop_lo & 2u) ? 4 : 8;
         for (int k = 0; k < n3; ++k)
-          umma_ts(tmem + kColS, tmem + kColX + (k >> 2) * 32 + (k & 3) * 8,
-                  smem_desc_sw128(sK + (k & 3) * 2048, 8192, 1024), id128_mn, true);
+          umma_ts(tmem + kColS, tmem + kColX + (k >> 2) * 32 + (k & 3) * 8, dKmn + 128 * (k & 3), id128_mn, true);
         for (int k = 0; k < n3; ++k)
-          umma_ts(tmem + kColM, tmem + kColY + (k >> 2) * 32 + (k & 3) * 8,
-                  smem_desc_sw128(sK + (k & 3) * 2048, 8192, 1024), id128_mn_neg, true);
+          umma_ts(tmem + kColM, tmem + kColY + (k >> 2) * 32 + (k & 3) * 8, dKmn + 128 * (k & 3), id128_mn_neg, true);
         umma_commit(b_m3);
         // ---- MMA-3': U = V~^T W^T  with  V~ = hi + lo, W = hi + lo (lo*lo dropped)
+        MDN_WAIT(b_v2, ph);
+        tc_fence_after_sync();
 #pragma unroll
-        for (int k = 0; k < 4; ++k)
-          umma_ts(tmem + kColU, tmem + kColZ + k * 8, smem_desc_sw128(sWh + k * 32, 16, 1024), id64, k > 0);
+        for (int k = 0; k < 4; ++k) umma_ts(tmem + kColU, tmem + kColZ + k * 8, dWh + 2 * k, id64, k > 0);
         if (!(a.drop_lo & 4u)) {
 #pragma unroll
-          for (int k = 0; k < 4; ++k)
-            umma_ts(tmem + kColU, tmem + kColZ + 32 + k * 8, smem_desc_sw128(sWh + k * 32, 16, 1024), id64, true);
+          for (int k = 0; k < 4; ++k) umma_ts(tmem + kColU, tmem + kColZ + 32 + k * 8, dWh + 2 * k, id64, true);
         }
         if (!(a.drop_lo & 8u)) {
 #pragma unroll
-          for (int k = 0; k < 4; ++k)
-            umma_ts(tmem + kColU, tmem + kColZ + k * 8, smem_desc_sw128(sWl + k * 32, 16, 1024), id64, true);
+          for (int k = 0; k < 4; ++k) umma_ts(tmem + kColU, tmem + kColZ + k * 8, dWl + 2 * k, id64, true);
         }
         umma_commit(b_mo);
         MDN_MARK(c, kEvMmaIssued);
       }
     }
-  } else if (warp < 4) {
+  } else if (warp < kWarpEpiB) {
     // ================================================================== critical-path epilogue (P, EPI-1, EPI-2)
-    const int d = tid;                                              // value column = tensor-memory lane
-    const uint32_t tl = tmem + (static_cast<uint32_t>(warp * 32) << 16);
+    // 8 warps: lane quarter q = warp & 3 (value columns 32q .. 32q+31), token / dk half hf = warp >> 2.
+    const int q4 = warp & 3, hf = warp >> 2;
+    const int d = q4 * 32 + lane;                                    // value column = tensor-memory lane
+    const uint32_t tl = tmem + (static_cast<uint32_t>(q4 * 32) << 16);
+    uint32_t ga_phase = 0;
     for (int c = 0; c <= nch; ++c) {
-      // ---------------- P(c)
+      // ---------------- P(c), part 1: bf16 copies of S^T, M^T for MMA-1 (or the final states)
       float al = 0.f, bl = 0.f, ml = 0.f;
       if (c > 0) {
         MDN_WAIT(b_m3, (c - 1) & 1);
@@ -282,7 +288,8 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
       __syncwarp();
       tc_fence_after_sync();
 #pragma unroll 1
-      for (int cs = 0; cs < 4; ++cs) {
+      for (int i = 0; i < 2; ++i) {
+        const int cs = 2 * hf + i;   // 32-column slice of dk
         uint32_t sr[32], mr[32];
         if (c == 0) {
 #pragma unroll
@@ -313,14 +320,6 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
             *reinterpret_cast<uint4*>(sb + off) = ps;
             *reinterpret_cast<uint4*>(mb + off) = pm;
           }
-#pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const float sv = __uint_as_float(sr[j]), mv = __uint_as_float(mr[j]);
-            sr[j] = __float_as_uint(al * sv - bl * mv);
-            mr[j] = __float_as_uint(ml * mv);
-          }
-          tmem_st32(tl + kColS + cs * 32, sr);
-          tmem_st32(tl + kColM + cs * 32, mr);
         } else {
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
@@ -330,100 +329,161 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
         }
       }
       if (c == nch) break;
-      tmem_wait_st();
       fence_proxy_async_smem();
-      tc_fence_before_sync();
       mbar_arrive(b_sb);
       MDN_MARK(c, kEvSbArrive);
+      // ---------------- P(c), part 2 (off the critical path, under MMA-1a): masters scaled by this chunk's
+      // (abar_C, b_C, mubar_C) so that MMA-3 can accumulate straight into them
+#pragma unroll 1
+      for (int i = 0; i < 2; ++i) {
+        const int cs = 2 * hf + i;
+        uint32_t sr[32], mr[32];
+        if (c == 0) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            sr[j] = __float_as_uint(a.S0 ? __ldg(a.S0 + st_off + (size_t)(cs * 32 + j) * kD + d) : 0.f);
+            mr[j] = __float_as_uint(a.M0 ? __ldg(a.M0 + st_off + (size_t)(cs * 32 + j) * kD + d) : 0.f);
+          }
+        } else {
+          tmem_ld32(tl + kColS + cs * 32, sr);
+          tmem_ld32(tl + kColM + cs * 32, mr);
+          tmem_wait_ld();
+        }
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          const float sv = __uint_as_float(sr[j]), mv = __uint_as_float(mr[j]);
+          sr[j] = __float_as_uint(al * sv - bl * mv);
+          mr[j] = __float_as_uint(ml * mv);
+        }
+        tmem_st32(tl + kColS + cs * 32, sr);
+        tmem_st32(tl + kColM + cs * 32, mr);
+      }
+      MDN_MARK(c, kEvPrescaled);
 
       const uint32_t ph = c & 1;
       const uint8_t* stg = smem + kOffStage + (c & 1) * kStageBytes;
       const float* cf = reinterpret_cast<const float*>(stg + kStCoef);
       const __nv_bfloat16* sV = reinterpret_cast<const __nv_bfloat16*>(stg + kStV);
+      const int r0 = 32 * hf;   // this warp's tokens
       // ---------------- EPI-1: R^T = V^T - abar .* X + (alpha b^-) .* Y  -> bf16 hi, lo in X
       MDN_WAIT(b_m1, ph);
       __syncwarp();
       tc_fence_after_sync();
       MDN_MARK(c, kEvM1Seen);
       {
-        uint32_t hi[32], lo[32];
-#pragma unroll
-        for (int hh = 0; hh < 2; ++hh) {
+        uint32_t hi[16], lo[16];
+        {
           uint32_t x[32], y[32];
-          tmem_ld32(tl + kColX + hh * 32, x);
-          tmem_ld32(tl + kColY + hh * 32, y);
+          tmem_ld32(tl + kColX + r0, x);
+          tmem_ld32(tl + kColY + r0, y);
           tmem_wait_ld();
+          MDN_MARK(c, kEvE1Loaded);
 #pragma unroll
-          for (int j = 0; j < 32; j += 2) {
-            const int r = hh * 32 + j;
-            const float2 ab = *reinterpret_cast<const float2*>(cf + kAbar * C + r);
-            const float2 pb = *reinterpret_cast<const float2*>(cf + kAlphaBPrev * C + r);
-            const float v0 = __bfloat162float(sV[r * kD + d]), v1 = __bfloat162float(sV[(r + 1) * kD + d]);
-            const float r0 = v0 - ab.x * __uint_as_float(x[j]) + pb.x * __uint_as_float(y[j]);
-            const float r1 = v1 - ab.y * __uint_as_float(x[j + 1]) + pb.y * __uint_as_float(y[j + 1]);
-            float h0, l0, h1, l1;
-            split_bf16(r0, h0, l0);
-            split_bf16(r1, h1, l1);
-            hi[r >> 1] = pack_bf16(h0, h1);
-            lo[r >> 1] = pack_bf16(l0, l1);
+          for (int j = 0; j < 32; j += 4) {
+            const float4 ab = *reinterpret_cast<const float4*>(cf + kAbar * C + r0 + j);
+            const float4 pb = *reinterpret_cast<const float4*>(cf + kAlphaBPrev * C + r0 + j);
+            const float v0 = __bfloat162float(sV[(r0 + j + 0) * kD + d]), v1 = __bfloat162float(sV[(r0 + j + 1) * kD + d]);
+            const float v2 = __bfloat162float(sV[(r0 + j + 2) * kD + d]), v3 = __bfloat162float(sV[(r0 + j + 3) * kD + d]);
+            const float e0 = v0 - ab.x * __uint_as_float(x[j + 0]) + pb.x * __uint_as_float(y[j + 0]);
+            const float e1 = v1 - ab.y * __uint_as_float(x[j + 1]) + pb.y * __uint_as_float(y[j + 1]);
+            const float e2 = v2 - ab.z * __uint_as_float(x[j + 2]) + pb.z * __uint_as_float(y[j + 2]);
+            const float e3 = v3 - ab.w * __uint_as_float(x[j + 3]) + pb.w * __uint_as_float(y[j + 3]);
+            split_pack_bf16(e0, e1, hi[j >> 1], lo[j >> 1]);
+            split_pack_bf16(e2, e3, hi[(j >> 1) + 1], lo[(j >> 1) + 1]);
           }
         }
-        tmem_st32(tl + kColX, hi);
-        tmem_st32(tl + kColX + 32, lo);
+        // the other half's warps may still be reading X: group sync before overwriting it
+        MDN_MARK(c, kEvE1Math);
+        tc_fence_before_sync();
+        mbar_arrive(b_ga);
+        MDN_WAIT(b_ga, ga_phase);
+        ga_phase ^= 1;
+        __syncwarp();
+        tc_fence_after_sync();
+        MDN_MARK(c, kEvE1Sync);
+        tmem_st16(tl + kColX + 16 * hf, hi);
+        tmem_st16(tl + kColX + 32 + 16 * hf, lo);
         tmem_wait_st();
+        MDN_MARK(c, kEvE1Stored);
       }
       tc_fence_before_sync();
       mbar_arrive(b_r);
       MDN_MARK(c, kEvRArrive);
-      // ---------------- EPI-2: V~ -> (gamma_C eta) V~, ((mubar_C/mubar) eta) V~, V~ as bf16 hi, lo
+      // ---------------- EPI-2: V~ -> (gamma_C eta) V~, ((mubar_C/mubar) eta) V~ [part a], V~ [part b]; bf16 hi, lo
       MDN_WAIT(b_m2, ph);
-      MDN_WAIT(b_zq, ph);
       __syncwarp();
       tc_fence_after_sync();
       MDN_MARK(c, kEvM2Seen);
       {
-        uint32_t vt[64];
-        tmem_ld32(tl + kColY, *reinterpret_cast<uint32_t(*)[32]>(&vt[0]));
-        tmem_ld32(tl + kColY + 32, *reinterpret_cast<uint32_t(*)[32]>(&vt[32]));
+        uint32_t vt[32];
+        tmem_ld32(tl + kColY + r0, vt);
         tmem_wait_ld();
+        {
+          uint32_t sh[16], sl[16];
 #pragma unroll
-        for (int gq = 0; gq < 4; ++gq) {
-          uint32_t sh[8], sl[8], mh[8], mlo[8], vh[8], vl[8];
-#pragma unroll
-          for (int jj = 0; jj < 8; ++jj) {
-            const int r = gq * 16 + 2 * jj;
-            const float2 gs = *reinterpret_cast<const float2*>(cf + kGS * C + r);
-            const float2 gm = *reinterpret_cast<const float2*>(cf + kGM * C + r);
-            const float v0 = __uint_as_float(vt[r]), v1 = __uint_as_float(vt[r + 1]);
-            float h0, l0, h1, l1;
-            split_bf16(gs.x * v0, h0, l0); split_bf16(gs.y * v1, h1, l1);
-            sh[jj] = pack_bf16(h0, h1); sl[jj] = pack_bf16(l0, l1);
-            split_bf16(gm.x * v0, h0, l0); split_bf16(gm.y * v1, h1, l1);
-            mh[jj] = pack_bf16(h0, h1); mlo[jj] = pack_bf16(l0, l1);
-            split_bf16(v0, h0, l0); split_bf16(v1, h1, l1);
-            vh[jj] = pack_bf16(h0, h1); vl[jj] = pack_bf16(l0, l1);
+          for (int j = 0; j < 32; j += 4) {
+            const float4 gs = *reinterpret_cast<const float4*>(cf + kGS * C + r0 + j);
+            split_pack_bf16(gs.x * __uint_as_float(vt[j]), gs.y * __uint_as_float(vt[j + 1]), sh[j >> 1], sl[j >> 1]);
+            split_pack_bf16(gs.z * __uint_as_float(vt[j + 2]), gs.w * __uint_as_float(vt[j + 3]), sh[(j >> 1) + 1],
+                            sl[(j >> 1) + 1]);
           }
-          tmem_st8(tl + kColX + gq * 8, sh); tmem_st8(tl + kColX + 32 + gq * 8, sl);
-          tmem_st8(tl + kColY + gq * 8, mh); tmem_st8(tl + kColY + 32 + gq * 8, mlo);
-          tmem_st8(tl + kColZ + gq * 8, vh); tmem_st8(tl + kColZ + 32 + gq * 8, vl);
+          tmem_st16(tl + kColX + 16 * hf, sh);          // X is free: MMA-2 has consumed R
+          tmem_st16(tl + kColX + 32 + 16 * hf, sl);
         }
-        tmem_wait_st();
+        {
+          uint32_t mh[16], mlo[16];
+#pragma unroll
+          for (int j = 0; j < 32; j += 4) {
+            const float4 gm = *reinterpret_cast<const float4*>(cf + kGM * C + r0 + j);
+            split_pack_bf16(gm.x * __uint_as_float(vt[j]), gm.y * __uint_as_float(vt[j + 1]), mh[j >> 1], mlo[j >> 1]);
+            split_pack_bf16(gm.z * __uint_as_float(vt[j + 2]), gm.w * __uint_as_float(vt[j + 3]), mh[(j >> 1) + 1],
+                            mlo[(j >> 1) + 1]);
+          }
+          // Y still holds V~ for the other half's warps until they have loaded it
+          tc_fence_before_sync();
+          mbar_arrive(b_ga);
+          MDN_WAIT(b_ga, ga_phase);
+          ga_phase ^= 1;
+          __syncwarp();
+          tc_fence_after_sync();
+          tmem_st16(tl + kColY + 16 * hf, mh);
+          tmem_st16(tl + kColY + 32 + 16 * hf, mlo);
+        }
+        tmem_wait_st();          // also covers the pre-scaled masters stored in P part 2
+        tc_fence_before_sync();
+        mbar_arrive(b_v1);
+        MDN_MARK(c, kEvVArrive);
+        // part b (off the critical path): V~ itself for the intra-chunk output, into Z once Q S has been read
+        {
+          uint32_t vh[16], vl[16];
+#pragma unroll
+          for (int j = 0; j < 32; j += 2) split_pack_bf16(__uint_as_float(vt[j]), __uint_as_float(vt[j + 1]), vh[j >> 1], vl[j >> 1]);
+          MDN_WAIT(b_zq, ph);
+          __syncwarp();
+          tc_fence_after_sync();
+          tmem_st16(tl + kColZ + 16 * hf, vh);
+          tmem_st16(tl + kColZ + 32 + 16 * hf, vl);
+          tmem_wait_st();
+        }
+        tc_fence_before_sync();
+        mbar_arrive(b_v2);
+        MDN_MARK(c, kEvV2Arrive);
       }
-      tc_fence_before_sync();
-      mbar_arrive(b_v);
-      MDN_MARK(c, kEvVArrive);
       mbar_arrive((c & 1) ? b_empty1 : b_empty0);
     }
   } else {
-    // ================================================================== output epilogue
-    const int d = tid - 128;
-    const uint32_t tl = tmem + (static_cast<uint32_t>((warp - 4) * 32) << 16);
-    TO* o = static_cast<TO*>(a.o);
+    // ================================================================== output epilogue (warps 8..11)
+    const int q4 = warp & 3;
+    const int d = q4 * 32 + lane;
+    const int t128 = tid - kWarpEpiB * 32;
+    const uint32_t tl = tmem + (static_cast<uint32_t>(q4 * 32) << 16);
+    uint32_t gb_phase = 0;
     for (int c = 0; c < nch; ++c) {
       const uint32_t ph = c & 1;
       const int n = min(C, sq.len - c * C);
-      const size_t tok = (size_t)(sq.tok0 + c * C) * H + h;
-      const float* cf = reinterpret_cast<const float*>(smem + kOffStage + (c & 1) * kStageBytes + kStCoef);
+      const int tok0 = sq.tok0 + c * C;
+      uint8_t* stg = smem + kOffStage + (c & 1) * kStageBytes;
+      const float* cf = reinterpret_cast<const float*>(stg + kStCoef);
       MDN_WAIT((c & 1) ? b_full1 : b_full0, (c >> 1) & 1);
       MDN_WAIT(b_mq, ph);
       __syncwarp();
@@ -437,9 +497,13 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
         tmem_ld32(tl + kColU + hh * 32, u);
         tmem_wait_ld();
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          const int r = hh * 32 + j;
-          oi[r] = a.scale * (cf[kAbar * C + r] * __uint_as_float(z[j]) - cf[kB * C + r] * __uint_as_float(u[j]));
+        for (int j = 0; j < 32; j += 4) {
+          const float4 ab = *reinterpret_cast<const float4*>(cf + kAbar * C + hh * 32 + j);
+          const float4 bb = *reinterpret_cast<const float4*>(cf + kB * C + hh * 32 + j);
+          oi[hh * 32 + j + 0] = a.scale * (ab.x * __uint_as_float(z[j + 0]) - bb.x * __uint_as_float(u[j + 0]));
+          oi[hh * 32 + j + 1] = a.scale * (ab.y * __uint_as_float(z[j + 1]) - bb.y * __uint_as_float(u[j + 1]));
+          oi[hh * 32 + j + 2] = a.scale * (ab.z * __uint_as_float(z[j + 2]) - bb.z * __uint_as_float(u[j + 2]));
+          oi[hh * 32 + j + 3] = a.scale * (ab.w * __uint_as_float(z[j + 3]) - bb.w * __uint_as_float(u[j + 3]));
         }
       }
       tc_fence_before_sync();
@@ -449,29 +513,46 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
       __syncwarp();
       tc_fence_after_sync();
       MDN_MARK(c, kEvMoSeen);
-      {
-        uint32_t u[64];
-        tmem_ld32(tl + kColU, *reinterpret_cast<uint32_t(*)[32]>(&u[0]));
-        tmem_ld32(tl + kColU + 32, *reinterpret_cast<uint32_t(*)[32]>(&u[32]));
+      // every MMA of this chunk is done and both epilogues are past this stage's V and coefficients:
+      // the stage's K/Q area becomes the [64 x 128] output tile
+#pragma unroll
+      for (int hh = 0; hh < 2; ++hh) {
+        uint32_t u[32];
+        tmem_ld32(tl + kColU + hh * 32, u);
         tmem_wait_ld();
-        // U and this stage's coefficients are in registers: hand both back before the global stores
-        tc_fence_before_sync();
-        mbar_arrive(b_zu);
-        mbar_arrive((c & 1) ? b_empty1 : b_empty0);
-        MDN_MARK(c, kEvZuArrive);
-        if (!(a.drop_lo & 16u)) {
 #pragma unroll
-          for (int r = 0; r < 64; ++r)
-            if (r < n) store_o<TO>(o + (tok + (size_t)r * H) * kD + d, oi[r] + __uint_as_float(u[r]));
-        } else {   // debug: one store per thread instead of 64
-          float acc = 0.f;
-#pragma unroll
-          for (int r = 0; r < 64; ++r) acc += oi[r] + __uint_as_float(u[r]);
-          store_o<TO>(o + tok * kD + d, acc);
-        }
-        MDN_MARK(c, kEvStoresDone);
+        for (int j = 0; j < 32; ++j) stage_o<TO>(stg, hh * 32 + j, d, oi[hh * 32 + j] + __uint_as_float(u[j]));
       }
+      tc_fence_before_sync();
+      mbar_arrive(b_zu);
+      MDN_MARK(c, kEvZuArrive);
+      fence_proxy_async_smem();
+      mbar_arrive(b_gb);
+      MDN_WAIT(b_gb, gb_phase);
+      gb_phase ^= 1;
+      if (n == C) {
+        if (t128 == 0) {
+          tma_store_2d(&map_o, h * kD, tok0, smem_u32(stg));
+          tma_store_commit();
+          tma_store_wait_read();
+          mbar_arrive((c & 1) ? b_empty1 : b_empty0);
+        }
+      } else {   // short chunk: rows >= n belong to another sequence, copy the valid rows with plain stores
+        constexpr int kChunksPerRow = kD * (int)sizeof(TO) / 16;
+        uint8_t* obase = static_cast<uint8_t*>(a.o);
+        for (int idx = t128; idx < n * kChunksPerRow; idx += 128) {
+          const int r = idx / kChunksPerRow, c16 = idx % kChunksPerRow;
+          const uint4 val = *reinterpret_cast<const uint4*>(stg + (size_t)r * kD * sizeof(TO) + c16 * 16);
+          *reinterpret_cast<uint4*>(obase + (((size_t)(tok0 + r) * H + h) * kD) * sizeof(TO) + c16 * 16) = val;
+        }
+        mbar_arrive(b_gb);
+        MDN_WAIT(b_gb, gb_phase);
+        gb_phase ^= 1;
+        if (t128 == 0) mbar_arrive((c & 1) ? b_empty1 : b_empty0);
+      }
+      MDN_MARK(c, kEvStoresDone);
     }
+    if (t128 == 0) tma_store_wait_all();
   }
 #undef MDN_WAIT
 #undef MDN_MARK
@@ -497,13 +578,16 @@ cudaError_t launch_chain_tensor(const Plan& pl, const void* q, const void* k, co
   const mdn_params& p = pl.p;
   const uint64_t tokens = (uint64_t)p.B * p.T;
   const uint64_t mats = (uint64_t)pl.geom.num_slots * p.H;
-  CUtensorMap mq, mk, mv, mt, mw;
+  CUtensorMap mq, mk, mv, mt, mw, mo;
   const uint64_t row = (uint64_t)p.H * kD;
   if (!encode_tma_2d_bf16(&mq, TmaMap2D{q, row, tokens, row * 2, 64, 64, true}) ||
       !encode_tma_2d_bf16(&mk, TmaMap2D{k, row, tokens, row * 2, 64, 64, true}) ||
       !encode_tma_2d_bf16(&mv, TmaMap2D{v, row, tokens, row * 2, 128, 64, false}) ||
       !encode_tma_2d_bf16(&mt, TmaMap2D{pl.ws + pl.lay.off_T, 64, mats * C, 128, 64, 64, true}) ||
       !encode_tma_2d_bf16(&mw, TmaMap2D{pl.ws + pl.lay.off_W, 64, 2 * mats * C, 128, 64, 64, true}))
+    return cudaErrorInvalidValue;
+  const bool o_bf16 = p.o_dtype == MDN_BF16;
+  if (!encode_tma_2d(&mo, TmaMap2D{o, row, tokens, row * (o_bf16 ? 2u : 4u), 128, 64, false}, !o_bf16))
     return cudaErrorInvalidValue;
   ChainArgs a;
   a.g = pl.geom;
@@ -522,12 +606,12 @@ cudaError_t launch_chain_tensor(const Plan& pl, const void* q, const void* k, co
     auto kern = chain_tensor_kernel<__nv_bfloat16>;
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
     if (e != cudaSuccess) return e;
-    kern<<<grid, kThreads, kSmemBytes, pl.stream>>>(a, mq, mk, mv, mt, mw);
+    kern<<<grid, kThreads, kSmemBytes, pl.stream>>>(a, mq, mk, mv, mt, mw, mo);
   } else {
     auto kern = chain_tensor_kernel<float>;
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
     if (e != cudaSuccess) return e;
-    kern<<<grid, kThreads, kSmemBytes, pl.stream>>>(a, mq, mk, mv, mt, mw);
+    kern<<<grid, kThreads, kSmemBytes, pl.stream>>>(a, mq, mk, mv, mt, mw, mo);
   }
   e = cudaGetLastError();
   if (e == cudaSuccess) ++*launches;

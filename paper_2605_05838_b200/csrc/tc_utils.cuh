@@ -89,6 +89,18 @@ __device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void* src, ui
       : "memory");
 }
 
+// 2-D tiled store shared -> global (bulk async group).  Never started at a negative coordinate.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* m, int x, int y, uint32_t src_smem) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(reinterpret_cast<uint64_t>(m)), "r"(src_smem), "r"(x), "r"(y)
+               : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// Returns once the bulk stores committed so far have finished READING shared memory.
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+// Returns once the bulk stores committed so far are complete (writes performed).
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
 // ----------------------------------------------------------------------------- 128-byte swizzle
 // Byte offset of element (row, col) of a [rows x 64] bf16 block (128-byte rows, 8-row / 1024-byte
 // atoms) in the layout both TMA (SWIZZLE_128B) and tcgen05 (layout type 2) use: the 16-byte chunk
@@ -213,6 +225,14 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 }
 __device__ __forceinline__ float bf16_round(float x) { return __bfloat162float(__float2bfloat16_rn(x)); }
 
+// (x0, x1) -> packed bf16 pair `hi` (round to nearest) and packed bf16 pair `lo` of the residuals
+// x - float(hi): together ~16 mantissa bits through two bf16 tensor-core operands.
+__device__ __forceinline__ void split_pack_bf16(float x0, float x1, uint32_t& hi, uint32_t& lo) {
+  hi = pack_bf16(x0, x1);
+  const float h0 = __uint_as_float(hi << 16), h1 = __uint_as_float(hi & 0xFFFF0000u);
+  lo = pack_bf16(x0 - h0, x1 - h1);
+}
+
 }  // namespace tc
 
 // ----------------------------------------------------------------------------- host: tensor maps
@@ -220,6 +240,7 @@ __device__ __forceinline__ float bf16_round(float x) { return __bfloat162float(_
 struct TmaMap2D {
   const void* base; uint64_t inner, outer; uint64_t row_stride_bytes; uint32_t box_inner, box_outer; bool swizzle128;
 };
-bool encode_tma_2d_bf16(CUtensorMap* out, const TmaMap2D& d);
+bool encode_tma_2d(CUtensorMap* out, const TmaMap2D& d, bool f32);   // element type bf16, or float32 when f32
+inline bool encode_tma_2d_bf16(CUtensorMap* out, const TmaMap2D& d) { return encode_tma_2d(out, d, false); }
 
 }  // namespace mdn

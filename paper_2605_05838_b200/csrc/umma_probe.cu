@@ -9,7 +9,7 @@
 
 namespace mdn {
 
-bool encode_tma_2d_bf16(CUtensorMap* out, const TmaMap2D& d) {
+bool encode_tma_2d(CUtensorMap* out, const TmaMap2D& d, bool f32) {
   typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -26,7 +26,7 @@ bool encode_tma_2d_bf16(CUtensorMap* out, const TmaMap2D& d) {
   const cuuint64_t strides[1] = {d.row_stride_bytes};
   const cuuint32_t box[2] = {d.box_inner, d.box_outer};
   const cuuint32_t estr[2] = {1, 1};
-  return fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(d.base), dims, strides, box, estr,
+  return fn(out, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(d.base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, d.swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
             CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
