@@ -38,8 +38,9 @@ namespace {
 using namespace tc;
 
 constexpr int kD = 128;
-constexpr int kThreads = 448;
-constexpr int kWarpEpiB = 8, kWarpTma = 12, kWarpMma = 13;
+constexpr int kThreads = 320;
+constexpr int kEpiWarps = 8, kWarpTma = 8, kWarpMma = 9;
+constexpr int kEpiThreads = kEpiWarps * 32;
 
 // shared memory (offsets from a 1024-byte aligned base)
 constexpr uint32_t kOffSb = 0, kOffMb = 32768, kOffStage = 65536;
@@ -54,20 +55,20 @@ static_assert(kStCoef + kCoefBytes <= kStageBytes, "stage layout");
 constexpr uint32_t kColS = 0, kColM = 128, kColX = 256, kColY = 320, kColZ = 384, kColU = 448;
 
 struct Bars {
-  uint64_t full[2], empty[2];
-  uint64_t sb;   // P(c): S_b, M_b in smem                                            (256 arrivals)
-  uint64_t m1;   // MMA-1a done                                                      (commit)
-  uint64_t mq;   // MMA-1b done                                                      (commit)
-  uint64_t r;    // EPI-1 done: R^T hi/lo in X                                        (256)
-  uint64_t m2;   // MMA-2 done                                                       (commit)
-  uint64_t zq;   // output epilogue has read Z, U (Q S, Q M)                          (128)
-  uint64_t v1;   // EPI-2a done: V~_S, V~_M operands in X, Y; masters pre-scaled      (256)
-  uint64_t v2;   // EPI-2b done: V~ operand in Z                                      (256)
-  uint64_t m3;   // MMA-3 done                                                       (commit)
-  uint64_t mo;   // MMA-3' done                                                      (commit)
-  uint64_t zu;   // output epilogue has read U (intra-chunk output)                   (128)
-  uint64_t ga;   // critical-path epilogue group sync                                 (256)
-  uint64_t gb;   // output epilogue group sync                                        (128)
+  uint64_t full[2];   // TMA loads of a stage landed                                   (1 + tx bytes)
+  uint64_t go[2];     // a stage's output tile is staged and nobody reads the stage any more (256)
+  uint64_t sb;        // P part 1: S_b, M_b in smem                                    (256)
+  uint64_t m1;        // MMA-1a done                                                   (commit)
+  uint64_t mq;        // MMA-1b done                                                   (commit)
+  uint64_t r;         // EPI-1 done: R^T hi/lo in X                                     (256)
+  uint64_t m2;        // MMA-2 done                                                    (commit)
+  uint64_t zq;        // Z, U (Q S, Q M) have been read                                 (256)
+  uint64_t v1;        // EPI-2a done: V~_S, V~_M operands in X, Y; masters pre-scaled   (256)
+  uint64_t v2;        // EPI-2b done: V~ operand in Z                                   (256)
+  uint64_t m3;        // MMA-3 done                                                    (commit)
+  uint64_t mo;        // MMA-3' done                                                   (commit)
+  uint64_t zu;        // U (intra-chunk output) has been read                           (256)
+  uint64_t ga;        // epilogue group sync                                            (256)
 };
 
 struct ChainArgs {
@@ -88,7 +89,7 @@ struct ChainArgs {
 // Timeline events (debug).
 enum Ev : int { kEvMmaStart = 0, kEvM1Seen, kEvRArrive, kEvM2Seen, kEvVArrive, kEvM3Seen, kEvSbArrive, kEvMqSeen,
                 kEvZqArrive, kEvMoSeen, kEvZuArrive, kEvMmaIssued, kEvRSeen, kEvVSeen, kEvTmaIssued, kEvFullSeen,
-                kEvStoresDone, kEvV2Arrive, kEvPrescaled, kEvE1Loaded, kEvE1Math, kEvE1Sync, kEvE1Stored, kEvPLoaded, kEvPStored };
+                kEvStoresDone, kEvV2Arrive, kEvPrescaled };
 
 template <typename TO> __device__ __forceinline__ void stage_o(uint8_t* tile, int r, int d, float x);
 template <> __device__ __forceinline__ void stage_o<float>(uint8_t* tile, int r, int d, float x) {
@@ -121,19 +122,19 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
 
   const uint32_t s_base = smem_u32(smem);
   const uint32_t b_full0 = smem_u32(&bars.full[0]), b_full1 = smem_u32(&bars.full[1]);
-  const uint32_t b_empty0 = smem_u32(&bars.empty[0]), b_empty1 = smem_u32(&bars.empty[1]);
+  const uint32_t b_go0 = smem_u32(&bars.go[0]), b_go1 = smem_u32(&bars.go[1]);
   const uint32_t b_sb = smem_u32(&bars.sb), b_m1 = smem_u32(&bars.m1), b_mq = smem_u32(&bars.mq);
   const uint32_t b_r = smem_u32(&bars.r), b_m2 = smem_u32(&bars.m2), b_zq = smem_u32(&bars.zq);
   const uint32_t b_v1 = smem_u32(&bars.v1), b_v2 = smem_u32(&bars.v2), b_m3 = smem_u32(&bars.m3);
-  const uint32_t b_mo = smem_u32(&bars.mo), b_zu = smem_u32(&bars.zu);
-  const uint32_t b_ga = smem_u32(&bars.ga), b_gb = smem_u32(&bars.gb);
+  const uint32_t b_mo = smem_u32(&bars.mo), b_zu = smem_u32(&bars.zu), b_ga = smem_u32(&bars.ga);
 
   if (tid == 0) {
     abort_flag = 0;
     mbar_init(b_full0, 1); mbar_init(b_full1, 1);
-    mbar_init(b_empty0, 257); mbar_init(b_empty1, 257);
-    mbar_init(b_sb, 256); mbar_init(b_r, 256); mbar_init(b_v1, 256); mbar_init(b_v2, 256); mbar_init(b_ga, 256);
-    mbar_init(b_zq, 128); mbar_init(b_zu, 128); mbar_init(b_gb, 128);
+    mbar_init(b_go0, kEpiThreads); mbar_init(b_go1, kEpiThreads);
+    mbar_init(b_sb, kEpiThreads); mbar_init(b_r, kEpiThreads); mbar_init(b_v1, kEpiThreads);
+    mbar_init(b_v2, kEpiThreads); mbar_init(b_ga, kEpiThreads); mbar_init(b_zq, kEpiThreads);
+    mbar_init(b_zu, kEpiThreads);
     mbar_init(b_m1, 1); mbar_init(b_mq, 1); mbar_init(b_m2, 1); mbar_init(b_m3, 1); mbar_init(b_mo, 1);
     mbar_fence_init();
   }
@@ -155,37 +156,55 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
   }
   long long* const tline = (blockIdx.x == 0) ? a.timeline : nullptr;
 #define MDN_MARK(c, ev) \
-  if (tline != nullptr && lane == 0 && (warp == 0 || warp >= kWarpEpiB) && (warp & 3) == (warp >= kWarpTma ? (warp & 3) : 0)) \
-    tline[(c) * 32 + (ev)] = clock64();
+  if (tline != nullptr && lane == 0 && (warp == 0 || warp >= kEpiWarps)) tline[(c) * 32 + (ev)] = clock64();
 
   if (warp == kWarpTma) {
-    // ================================================================== TMA producer
+    // ================================================================== TMA producer + output stores
+    // Stage s = c & 1 serves chunk c, then (as the staged output tile) is written out and refilled for chunk c + 2.
     if (lane == 0) {
       int issued = 0;
-      for (int c = 0; c < nch; ++c) {
+      for (int c = 0; c < nch + 2; ++c) {
         const int s = c & 1;
-        MDN_WAIT(s ? b_empty1 : b_empty0, ((c >> 1) & 1) ^ 1);
-        const uint32_t fb = s ? b_full1 : b_full0;
         const uint32_t st = s_base + kOffStage + s * kStageBytes;
-        const int tok0 = sq.tok0 + c * C;
-        const int mat = (sq.slot0 + c) * H + h;
-        mbar_arrive_expect_tx(fb, kTxBytes);
-        tma_load_2d(st + kStK, &map_k, h * kD, tok0, fb);
-        tma_load_2d(st + kStK + 8192, &map_k, h * kD + 64, tok0, fb);
-        bulk_load(st + kStCoef, a.coef + (size_t)mat * MDN_NUM_COEF * C, kCoefBytes, fb);
-        tma_load_2d(st + kStV, &map_v, h * kD, tok0, fb);
-        tma_load_2d(st + kStT, &map_t, 0, mat * C, fb);
-        tma_load_2d(st + kStQ, &map_q, h * kD, tok0, fb);
-        tma_load_2d(st + kStQ + 8192, &map_q, h * kD + 64, tok0, fb);
-        tma_load_2d(st + kStWh, &map_w, 0, mat * C, fb);
-        tma_load_2d(st + kStWl, &map_w, 0, mat * C + (int)a.w_lo_row_offset, fb);
-        MDN_MARK(c, kEvTmaIssued);
-        issued = c + 1;
+        if (c >= 2) {
+          const int co = c - 2;
+          MDN_WAIT(s ? b_go1 : b_go0, (co >> 1) & 1);
+          const int n = min(C, sq.len - co * C);
+          const int tok0 = sq.tok0 + co * C;
+          if (n == C) {
+            tma_store_2d(&map_o, h * kD, tok0, st);
+          } else {   // short chunk: rows >= n belong to another sequence; one bulk copy per valid row
+            for (int r = 0; r < n; ++r)
+              bulk_store(static_cast<uint8_t*>(a.o) + (((size_t)(tok0 + r) * H + h) * kD) * sizeof(TO),
+                         st + r * kD * (uint32_t)sizeof(TO), kD * (uint32_t)sizeof(TO));
+          }
+          tma_store_commit();
+          tma_store_wait_read();
+          MDN_MARK(co, kEvStoresDone);
+        }
+        if (c < nch) {
+          const uint32_t fb = s ? b_full1 : b_full0;
+          const int tok0 = sq.tok0 + c * C;
+          const int mat = (sq.slot0 + c) * H + h;
+          mbar_arrive_expect_tx(fb, kTxBytes);
+          tma_load_2d(st + kStK, &map_k, h * kD, tok0, fb);
+          tma_load_2d(st + kStK + 8192, &map_k, h * kD + 64, tok0, fb);
+          bulk_load(st + kStCoef, a.coef + (size_t)mat * MDN_NUM_COEF * C, kCoefBytes, fb);
+          tma_load_2d(st + kStV, &map_v, h * kD, tok0, fb);
+          tma_load_2d(st + kStT, &map_t, 0, mat * C, fb);
+          tma_load_2d(st + kStQ, &map_q, h * kD, tok0, fb);
+          tma_load_2d(st + kStQ + 8192, &map_q, h * kD + 64, tok0, fb);
+          tma_load_2d(st + kStWh, &map_w, 0, mat * C, fb);
+          tma_load_2d(st + kStWl, &map_w, 0, mat * C + (int)a.w_lo_row_offset, fb);
+          MDN_MARK(c, kEvTmaIssued);
+          issued = c + 1;
+        }
       }
       if (!ok) {   // giving up: let the copies already in flight land before the CTA exits
         for (int c = max(0, issued - 2); c < issued; ++c)
           for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait((c & 1) ? b_full1 : b_full0, (c >> 1) & 1); ++it) {}
       }
+      tma_store_wait_all();
     }
   } else if (warp == kWarpMma) {
     // ================================================================== MMA issuer
@@ -217,7 +236,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
         for (int k = 0; k < 8; ++k)
           umma_ss(tmem + kColY, ((k >> 2) ? dMb1 : dMb0) + 2 * (k & 3), ((k >> 2) ? dK1 : dK0) + 2 * (k & 3), id64, k > 0);
         umma_commit(b_m1);
-        // ---- MMA-1b: Z = S_b Q^T, U = M_b Q^T (Z, U must have been drained by the output epilogue)
+        // ---- MMA-1b: Z = S_b Q^T, U = M_b Q^T (U of the previous chunk must have been read)
         MDN_WAIT(b_zu, ph ^ 1);
         tc_fence_after_sync();
 #pragma unroll
@@ -265,15 +284,20 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
         MDN_MARK(c, kEvMmaIssued);
       }
     }
-  } else if (warp < kWarpEpiB) {
-    // ================================================================== critical-path epilogue (P, EPI-1, EPI-2)
-    // 8 warps: lane quarter q = warp & 3 (value columns 32q .. 32q+31), token / dk half hf = warp >> 2.
+  } else {
+    // ================================================================== epilogue warps 0..7
+    // lane quarter q4 = warp & 3 (value columns 32 q4 .. +31 = this warp's tensor-memory lanes),
+    // half hf = warp >> 2 (tokens 32 hf .. +31 in the per-token steps, dk columns 64 hf .. +63 in P).
     const int q4 = warp & 3, hf = warp >> 2;
-    const int d = q4 * 32 + lane;                                    // value column = tensor-memory lane
+    const int d = q4 * 32 + lane;
+    const int r0 = 32 * hf;
     const uint32_t tl = tmem + (static_cast<uint32_t>(q4 * 32) << 16);
     uint32_t ga_phase = 0;
+    float oi[32];   // scale (abar .* Q S - b .* Q M) for this thread's tokens, carried to the output step
+#pragma unroll
+    for (int j = 0; j < 32; ++j) oi[j] = 0.f;
     for (int c = 0; c <= nch; ++c) {
-      // ---------------- P(c), part 1: bf16 copies of S^T, M^T for MMA-1 (or the final states)
+      // ---------------- P(c): bf16 copies of S^T, M^T for MMA-1 (after the last chunk: final states)
       float al = 0.f, bl = 0.f, ml = 0.f;
       if (c > 0) {
         MDN_WAIT(b_m3, (c - 1) & 1);
@@ -320,6 +344,16 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
             *reinterpret_cast<uint4*>(sb + off) = ps;
             *reinterpret_cast<uint4*>(mb + off) = pm;
           }
+          // masters scaled by this chunk's (abar_C, b_C, mubar_C) so that MMA-3 can accumulate straight into
+          // them; the stores are asynchronous and only waited for before V~_S, V~_M are handed over
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            const float sv = __uint_as_float(sr[j]), mv = __uint_as_float(mr[j]);
+            sr[j] = __float_as_uint(al * sv - bl * mv);
+            mr[j] = __float_as_uint(ml * mv);
+          }
+          tmem_st32(tl + kColS + cs * 32, sr);
+          tmem_st32(tl + kColM + cs * 32, mr);
         } else {
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
@@ -328,87 +362,105 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
           }
         }
       }
-      if (c == nch) break;
-      fence_proxy_async_smem();
-      mbar_arrive(b_sb);
-      MDN_MARK(c, kEvSbArrive);
-      // ---------------- P(c), part 2 (off the critical path, under MMA-1a): masters scaled by this chunk's
-      // (abar_C, b_C, mubar_C) so that MMA-3 can accumulate straight into them
-#pragma unroll 1
-      for (int i = 0; i < 2; ++i) {
-        const int cs = 2 * hf + i;
-        uint32_t sr[32], mr[32];
-        if (c == 0) {
-#pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            sr[j] = __float_as_uint(a.S0 ? __ldg(a.S0 + st_off + (size_t)(cs * 32 + j) * kD + d) : 0.f);
-            mr[j] = __float_as_uint(a.M0 ? __ldg(a.M0 + st_off + (size_t)(cs * 32 + j) * kD + d) : 0.f);
-          }
-        } else {
-          tmem_ld32(tl + kColS + cs * 32, sr);
-          tmem_ld32(tl + kColM + cs * 32, mr);
-          tmem_wait_ld();
-        }
-#pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          const float sv = __uint_as_float(sr[j]), mv = __uint_as_float(mr[j]);
-          sr[j] = __float_as_uint(al * sv - bl * mv);
-          mr[j] = __float_as_uint(ml * mv);
-        }
-        tmem_st32(tl + kColS + cs * 32, sr);
-        tmem_st32(tl + kColM + cs * 32, mr);
+      if (c < nch) {
+        fence_proxy_async_smem();
+        mbar_arrive(b_sb);
+        MDN_MARK(c, kEvSbArrive);
       }
+      // ---------------- output of the previous chunk (under MMA-1a): o^T = oi + U, staged as a [64 x 128] tile in
+      // the previous chunk's stage (all its MMAs are done and nobody reads its tiles any more)
+      if (c > 0) {
+        const int cp = c - 1;
+        uint8_t* stp = smem + kOffStage + (cp & 1) * kStageBytes;
+        MDN_WAIT(b_mo, cp & 1);
+        __syncwarp();
+        tc_fence_after_sync();
+        MDN_MARK(cp, kEvMoSeen);
+        {
+          uint32_t u[32];
+          tmem_ld32(tl + kColU + r0, u);
+          tmem_wait_ld();
+          tc_fence_before_sync();
+          mbar_arrive(b_zu);
+          MDN_MARK(cp, kEvZuArrive);
+#pragma unroll
+          for (int j = 0; j < 32; ++j) stage_o<TO>(stp, r0 + j, d, oi[j] + __uint_as_float(u[j]));
+        }
+        fence_proxy_async_smem();
+        mbar_arrive((cp & 1) ? b_go1 : b_go0);
+      }
+      if (c == nch) break;
       MDN_MARK(c, kEvPrescaled);
 
       const uint32_t ph = c & 1;
       const uint8_t* stg = smem + kOffStage + (c & 1) * kStageBytes;
       const float* cf = reinterpret_cast<const float*>(stg + kStCoef);
       const __nv_bfloat16* sV = reinterpret_cast<const __nv_bfloat16*>(stg + kStV);
-      const int r0 = 32 * hf;   // this warp's tokens
       // ---------------- EPI-1: R^T = V^T - abar .* X + (alpha b^-) .* Y  -> bf16 hi, lo in X
-      MDN_WAIT(b_m1, ph);
-      __syncwarp();
-      tc_fence_after_sync();
-      MDN_MARK(c, kEvM1Seen);
       {
+        // V and the coefficients do not depend on the MMA: fetch them while MMA-1a runs
+        float vv[32];
+#pragma unroll
+        for (int j = 0; j < 32; ++j) vv[j] = __bfloat162float(sV[(r0 + j) * kD + d]);
+        MDN_WAIT(b_m1, ph);
+        __syncwarp();
+        tc_fence_after_sync();
+        MDN_MARK(c, kEvM1Seen);
         uint32_t hi[16], lo[16];
         {
           uint32_t x[32], y[32];
           tmem_ld32(tl + kColX + r0, x);
           tmem_ld32(tl + kColY + r0, y);
           tmem_wait_ld();
-          MDN_MARK(c, kEvE1Loaded);
 #pragma unroll
           for (int j = 0; j < 32; j += 4) {
             const float4 ab = *reinterpret_cast<const float4*>(cf + kAbar * C + r0 + j);
             const float4 pb = *reinterpret_cast<const float4*>(cf + kAlphaBPrev * C + r0 + j);
-            const float v0 = __bfloat162float(sV[(r0 + j + 0) * kD + d]), v1 = __bfloat162float(sV[(r0 + j + 1) * kD + d]);
-            const float v2 = __bfloat162float(sV[(r0 + j + 2) * kD + d]), v3 = __bfloat162float(sV[(r0 + j + 3) * kD + d]);
-            const float e0 = v0 - ab.x * __uint_as_float(x[j + 0]) + pb.x * __uint_as_float(y[j + 0]);
-            const float e1 = v1 - ab.y * __uint_as_float(x[j + 1]) + pb.y * __uint_as_float(y[j + 1]);
-            const float e2 = v2 - ab.z * __uint_as_float(x[j + 2]) + pb.z * __uint_as_float(y[j + 2]);
-            const float e3 = v3 - ab.w * __uint_as_float(x[j + 3]) + pb.w * __uint_as_float(y[j + 3]);
+            const float e0 = vv[j + 0] - ab.x * __uint_as_float(x[j + 0]) + pb.x * __uint_as_float(y[j + 0]);
+            const float e1 = vv[j + 1] - ab.y * __uint_as_float(x[j + 1]) + pb.y * __uint_as_float(y[j + 1]);
+            const float e2 = vv[j + 2] - ab.z * __uint_as_float(x[j + 2]) + pb.z * __uint_as_float(y[j + 2]);
+            const float e3 = vv[j + 3] - ab.w * __uint_as_float(x[j + 3]) + pb.w * __uint_as_float(y[j + 3]);
             split_pack_bf16(e0, e1, hi[j >> 1], lo[j >> 1]);
             split_pack_bf16(e2, e3, hi[(j >> 1) + 1], lo[(j >> 1) + 1]);
           }
         }
         // the other half's warps may still be reading X: group sync before overwriting it
-        MDN_MARK(c, kEvE1Math);
         tc_fence_before_sync();
         mbar_arrive(b_ga);
         MDN_WAIT(b_ga, ga_phase);
         ga_phase ^= 1;
         __syncwarp();
         tc_fence_after_sync();
-        MDN_MARK(c, kEvE1Sync);
         tmem_st16(tl + kColX + 16 * hf, hi);
         tmem_st16(tl + kColX + 32 + 16 * hf, lo);
         tmem_wait_st();
-        MDN_MARK(c, kEvE1Stored);
       }
       tc_fence_before_sync();
       mbar_arrive(b_r);
       MDN_MARK(c, kEvRArrive);
+      // ---------------- inter-chunk output terms (under MMA-2): oi = scale (abar .* Q S - b .* Q M)
+      {
+        MDN_WAIT(b_mq, ph);
+        __syncwarp();
+        tc_fence_after_sync();
+        MDN_MARK(c, kEvMqSeen);
+        uint32_t z[32], u[32];
+        tmem_ld32(tl + kColZ + r0, z);
+        tmem_ld32(tl + kColU + r0, u);
+        tmem_wait_ld();
+        tc_fence_before_sync();
+        mbar_arrive(b_zq);
+        MDN_MARK(c, kEvZqArrive);
+#pragma unroll
+        for (int j = 0; j < 32; j += 4) {
+          const float4 ab = *reinterpret_cast<const float4*>(cf + kAbar * C + r0 + j);
+          const float4 bb = *reinterpret_cast<const float4*>(cf + kB * C + r0 + j);
+          oi[j + 0] = a.scale * (ab.x * __uint_as_float(z[j + 0]) - bb.x * __uint_as_float(u[j + 0]));
+          oi[j + 1] = a.scale * (ab.y * __uint_as_float(z[j + 1]) - bb.y * __uint_as_float(u[j + 1]));
+          oi[j + 2] = a.scale * (ab.z * __uint_as_float(z[j + 2]) - bb.z * __uint_as_float(u[j + 2]));
+          oi[j + 3] = a.scale * (ab.w * __uint_as_float(z[j + 3]) - bb.w * __uint_as_float(u[j + 3]));
+        }
+      }
       // ---------------- EPI-2: V~ -> (gamma_C eta) V~, ((mubar_C/mubar) eta) V~ [part a], V~ [part b]; bf16 hi, lo
       MDN_WAIT(b_m2, ph);
       __syncwarp();
@@ -453,7 +505,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
         tc_fence_before_sync();
         mbar_arrive(b_v1);
         MDN_MARK(c, kEvVArrive);
-        // part b (off the critical path): V~ itself for the intra-chunk output, into Z once Q S has been read
+        // part b (under MMA-3): V~ itself for the intra-chunk output, into Z once every warp has read Q S
         {
           uint32_t vh[16], vl[16];
 #pragma unroll
@@ -469,90 +521,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
         mbar_arrive(b_v2);
         MDN_MARK(c, kEvV2Arrive);
       }
-      mbar_arrive((c & 1) ? b_empty1 : b_empty0);
     }
-  } else {
-    // ================================================================== output epilogue (warps 8..11)
-    const int q4 = warp & 3;
-    const int d = q4 * 32 + lane;
-    const int t128 = tid - kWarpEpiB * 32;
-    const uint32_t tl = tmem + (static_cast<uint32_t>(q4 * 32) << 16);
-    uint32_t gb_phase = 0;
-    for (int c = 0; c < nch; ++c) {
-      const uint32_t ph = c & 1;
-      const int n = min(C, sq.len - c * C);
-      const int tok0 = sq.tok0 + c * C;
-      uint8_t* stg = smem + kOffStage + (c & 1) * kStageBytes;
-      const float* cf = reinterpret_cast<const float*>(stg + kStCoef);
-      MDN_WAIT((c & 1) ? b_full1 : b_full0, (c >> 1) & 1);
-      MDN_WAIT(b_mq, ph);
-      __syncwarp();
-      tc_fence_after_sync();
-      MDN_MARK(c, kEvMqSeen);
-      float oi[64];
-#pragma unroll
-      for (int hh = 0; hh < 2; ++hh) {
-        uint32_t z[32], u[32];
-        tmem_ld32(tl + kColZ + hh * 32, z);
-        tmem_ld32(tl + kColU + hh * 32, u);
-        tmem_wait_ld();
-#pragma unroll
-        for (int j = 0; j < 32; j += 4) {
-          const float4 ab = *reinterpret_cast<const float4*>(cf + kAbar * C + hh * 32 + j);
-          const float4 bb = *reinterpret_cast<const float4*>(cf + kB * C + hh * 32 + j);
-          oi[hh * 32 + j + 0] = a.scale * (ab.x * __uint_as_float(z[j + 0]) - bb.x * __uint_as_float(u[j + 0]));
-          oi[hh * 32 + j + 1] = a.scale * (ab.y * __uint_as_float(z[j + 1]) - bb.y * __uint_as_float(u[j + 1]));
-          oi[hh * 32 + j + 2] = a.scale * (ab.z * __uint_as_float(z[j + 2]) - bb.z * __uint_as_float(u[j + 2]));
-          oi[hh * 32 + j + 3] = a.scale * (ab.w * __uint_as_float(z[j + 3]) - bb.w * __uint_as_float(u[j + 3]));
-        }
-      }
-      tc_fence_before_sync();
-      mbar_arrive(b_zq);
-      MDN_MARK(c, kEvZqArrive);
-      MDN_WAIT(b_mo, ph);
-      __syncwarp();
-      tc_fence_after_sync();
-      MDN_MARK(c, kEvMoSeen);
-      // every MMA of this chunk is done and both epilogues are past this stage's V and coefficients:
-      // the stage's K/Q area becomes the [64 x 128] output tile
-#pragma unroll
-      for (int hh = 0; hh < 2; ++hh) {
-        uint32_t u[32];
-        tmem_ld32(tl + kColU + hh * 32, u);
-        tmem_wait_ld();
-#pragma unroll
-        for (int j = 0; j < 32; ++j) stage_o<TO>(stg, hh * 32 + j, d, oi[hh * 32 + j] + __uint_as_float(u[j]));
-      }
-      tc_fence_before_sync();
-      mbar_arrive(b_zu);
-      MDN_MARK(c, kEvZuArrive);
-      fence_proxy_async_smem();
-      mbar_arrive(b_gb);
-      MDN_WAIT(b_gb, gb_phase);
-      gb_phase ^= 1;
-      if (n == C) {
-        if (t128 == 0) {
-          tma_store_2d(&map_o, h * kD, tok0, smem_u32(stg));
-          tma_store_commit();
-          tma_store_wait_read();
-          mbar_arrive((c & 1) ? b_empty1 : b_empty0);
-        }
-      } else {   // short chunk: rows >= n belong to another sequence, copy the valid rows with plain stores
-        constexpr int kChunksPerRow = kD * (int)sizeof(TO) / 16;
-        uint8_t* obase = static_cast<uint8_t*>(a.o);
-        for (int idx = t128; idx < n * kChunksPerRow; idx += 128) {
-          const int r = idx / kChunksPerRow, c16 = idx % kChunksPerRow;
-          const uint4 val = *reinterpret_cast<const uint4*>(stg + (size_t)r * kD * sizeof(TO) + c16 * 16);
-          *reinterpret_cast<uint4*>(obase + (((size_t)(tok0 + r) * H + h) * kD) * sizeof(TO) + c16 * 16) = val;
-        }
-        mbar_arrive(b_gb);
-        MDN_WAIT(b_gb, gb_phase);
-        gb_phase ^= 1;
-        if (t128 == 0) mbar_arrive((c & 1) ? b_empty1 : b_empty0);
-      }
-      MDN_MARK(c, kEvStoresDone);
-    }
-    if (t128 == 0) tma_store_wait_all();
   }
 #undef MDN_WAIT
 #undef MDN_MARK
