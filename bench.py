@@ -61,6 +61,28 @@ def algorithmic_flops(w: wl.Workload) -> float:
     return float(w.B * w.T * w.H) * (12 * w.dk * w.dv + 4 * 64 * (w.dk + w.dv))
 
 
+def rank_workload(w: wl.Workload, rank: int) -> wl.Workload:
+    """Every rank runs its own batch of the same shape (seed offset by rank): batches are independent
+    problems, so there is no data-path collective."""
+    import dataclasses
+    return dataclasses.replace(w, seed=w.seed + rank)
+
+
+def max_over_ranks(value: float, dist, device) -> float:
+    """Max of a per-rank scalar over all ranks (the job's time is its slowest rank's)."""
+    if dist is None:
+        return float(value)
+    import torch
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_tokens_per_s(w: wl.Workload, world: int, steps: int, elapsed_ms: float) -> float:
+    """Whole-job throughput: all ranks' tokens over the max-over-ranks time."""
+    return w.B * w.T * world * steps / (elapsed_ms * 1e-3)
+
+
 class ClockSampler:
     """nvidia-smi clock / throttle-reason samples during the timed region (reading only)."""
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
@@ -72,7 +94,7 @@ class ClockSampler:
         self.p = None
         try:
             self.p = subprocess.Popen(["nvidia-smi", "-i", str(index), "--query-gpu=" + self.Q,
-                                       "--format=csv,noheader,nounits", "-lms", "50"],
+                                       "--format=csv,noheader,nounits", "-lms", "20"],
                                       stdout=self.f, stderr=subprocess.DEVNULL)
         except OSError:
             pass
@@ -190,8 +212,7 @@ def run_ours(args, w):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
-    import dataclasses
-    wr = dataclasses.replace(w, seed=w.seed + rank)      # every rank its own batch
+    wr = rank_workload(w, rank)
     inp = wl.make_inputs(wr)
     t = to_torch(inp, device="cuda:%d" % local)
     o_dtype = torch.bfloat16 if w.dtype == "bf16" else torch.float32
@@ -227,12 +248,9 @@ def run_ours(args, w):
     barrier()
     elapsed_ms = ev0.elapsed_time(ev1)
     clocks = sampler.stop() if sampler else None
-    if dist is not None:
-        tt = torch.tensor([elapsed_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(tt.item())
+    elapsed_ms = max_over_ranks(elapsed_ms, dist, "cuda")
     tokens_per_step = w.B * w.T * world
-    value = tokens_per_step * args.steps / (elapsed_ms * 1e-3)
+    value = job_tokens_per_s(w, world, args.steps, elapsed_ms)
 
     # dominant kernel (the chain kernel: inter-chunk propagation + output), timed live
     names = mdn.STAGE_NAMES
@@ -282,10 +300,7 @@ def run_ours(args, w):
         a1.record()
         barrier()
         e2e_ms = a0.elapsed_time(a1)
-        if dist is not None:
-            tt = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            e2e_ms = float(tt.item())
+        e2e_ms = max_over_ranks(e2e_ms, dist, "cuda")
         h2d = sum(x.numel() * x.element_size() for x in th.values() if x is not None)
         d2h = sum(x.numel() * x.element_size() for x in out)
         e2e = {"value": tokens_per_step * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT,
@@ -320,8 +335,8 @@ def run_ours(args, w):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--config", type=int, default=2, help="index into the named workloads (2 = headline)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--path", default="auto", choices=["auto", "simt", "tensor"])
