@@ -46,7 +46,9 @@ typedef enum {
   MDN_ERR_UNSUPPORTED = 2,    /* valid request this build has no kernel for                 */
   MDN_ERR_WORKSPACE = 3,      /* workspace NULL or smaller than mdn_chunk_fwd_workspace_bytes */
   MDN_ERR_CUDA = 4,           /* a CUDA runtime call (launch, attribute) failed             */
-  MDN_ERR_DEVICE_TIMEOUT = 5  /* a bounded device-side wait ran out (reported by mdn_read_status) */
+  MDN_ERR_DEVICE_TIMEOUT = 5, /* a bounded device-side wait ran out (reported by mdn_read_status) */
+  MDN_ERR_STATIC_SCRATCH = 6  /* mdn_chunk_fwd_static_scratch: the problem needs more scratch than  */
+                              /* MDN_STATIC_SCRATCH_BYTES                                            */
 } mdn_status;
 
 typedef enum { MDN_F32 = 0, MDN_BF16 = 1 } mdn_dtype;
@@ -116,6 +118,42 @@ mdn_status mdn_chunk_fwd_host(const mdn_params* p,
                               const int32_t* cu_seqlens,
                               void* o, float* final_S, float* final_M,
                               void* arena /* device */, size_t arena_bytes, void* cuda_stream);
+
+/*
+ * The forward for callers that cannot allocate device memory (the paper has no counterpart: this
+ * is a packaging variant of mdn_chunk_fwd, same kernels, same result).
+ *
+ * Who needs it: code that has no way to obtain a workspace at the time of the call - a server
+ * that gave all device memory to its own arena at start-up, a plugin whose host forbids allocator
+ * calls, a loop that cannot tolerate the device-wide synchronisation an allocation or free
+ * causes.  Instead of a caller-supplied workspace, the scratch lives in a fixed array of
+ * MDN_STATIC_SCRATCH_BYTES that is part of the library image; the call allocates nothing
+ * (no cudaMalloc, no cudaFree, no allocating library routine).  The caller still passes every
+ * input and output buffer, exactly as for mdn_chunk_fwd.
+ *
+ * Limits and rules:
+ *  - mdn_chunk_fwd_workspace_bytes(p) must not exceed MDN_STATIC_SCRATCH_BYTES (32 MiB: about
+ *    1200 chunk-head pairs, e.g. 4800 tokens x 16 heads); larger problems return
+ *    MDN_ERR_STATIC_SCRATCH and launch nothing.
+ *  - Every GPU that loads the library holds the array until the process exits.
+ *  - The first call on each device looks up the array's device address (a one-time set-up on the
+ *    host, made with that device current); make that first call before any stream capture.
+ *  - All calls share the one array, and it keeps the previous call's contents (the call clears the
+ *    part that must start at zero itself).  Calls whose kernels can overlap on the GPU - different
+ *    streams, or several host threads - race on it: serialise them, or use mdn_chunk_fwd.
+ *  - The device-side cu_seqlens check still turns a bad cu_seqlens into a no-op, but its status
+ *    word is inside the array and cannot be read back with mdn_read_status.
+ */
+#define MDN_STATIC_SCRATCH_BYTES (32u << 20)
+
+mdn_status mdn_chunk_fwd_static_scratch(const mdn_params* p,
+                                        const void* q, const void* k, const void* v,
+                                        const float* beta, const float* log_alpha, const float* log_mu,
+                                        const float* eta,
+                                        const float* initial_S, const float* initial_M,
+                                        const int32_t* cu_seqlens,
+                                        void* o, float* final_S, float* final_M,
+                                        void* cuda_stream);
 
 /*
  * Stage entry points (the same kernels mdn_chunk_fwd launches, exposed so that each

@@ -65,6 +65,8 @@ def lib() -> ctypes.CDLL:
         L.mdn_chunk_fwd.argtypes = [P] + [vp] * 13 + [vp, ctypes.c_size_t, vp]
         L.mdn_chunk_fwd_host.restype = ctypes.c_int
         L.mdn_chunk_fwd_host.argtypes = [P] + [vp] * 13 + [vp, ctypes.c_size_t, vp]
+        L.mdn_chunk_fwd_static_scratch.restype = ctypes.c_int
+        L.mdn_chunk_fwd_static_scratch.argtypes = [P] + [vp] * 13 + [vp]
         L.mdn_workspace_layout.restype = ctypes.c_int
         L.mdn_workspace_layout.argtypes = [P, ctypes.POINTER(MdnWsLayout)]
         L.mdn_coeff_scan.restype = ctypes.c_int
@@ -209,6 +211,34 @@ def chunk_fwd(q, k, v, beta, log_alpha, log_mu, eta=None, *, initial_S=None, ini
     if st != 0:
         raise MdnError(st, "mdn_chunk_fwd")
     return o, Sf, Mf
+
+
+STATIC_SCRATCH_BYTES = 32 << 20
+
+
+def chunk_fwd_static_scratch(q, k, v, beta, log_alpha, log_mu, eta=None, *, out, final_S=None, final_M=None,
+                             initial_S=None, initial_M=None, cu_seqlens=None, scale: Optional[float] = None,
+                             path: str = "auto") -> None:
+    """mdn_chunk_fwd_static_scratch: the forward without a workspace argument, for callers that
+    cannot allocate device memory.  This wrapper allocates nothing either: `out` (and the optional
+    `final_S`, `final_M`) are tensors the caller already owns and are written in place.  Raises
+    MdnError (status 6) when the problem needs more than STATIC_SCRATCH_BYTES of scratch.  Calls share
+    one built-in scratch array: do not let two of them overlap on the GPU."""
+    _check_inputs(q, k, v, (("beta", beta), ("log_alpha", log_alpha), ("log_mu", log_mu), ("eta", eta)), "cuda")
+    B, T, H, dk = q.shape
+    dv = v.shape[-1]
+    N = 0 if cu_seqlens is None else cu_seqlens.numel() - 1
+    p = make_params(q, v, num_seqs=N, scale=scale, o_dtype=out.dtype, path=path)
+    nst = N if N > 0 else B
+    for name, t in (("initial_S", initial_S), ("initial_M", initial_M), ("final_S", final_S), ("final_M", final_M)):
+        _check_state(name, t, (nst, H, dk, dv), "cuda")
+    if tuple(out.shape) != (B, T, H, dv) or not out.is_contiguous() or out.device.type != "cuda":
+        raise ValueError("out must be a contiguous cuda tensor of shape [B,T,H,dv]")
+    st = lib().mdn_chunk_fwd_static_scratch(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(beta), _ptr(log_alpha),
+                                            _ptr(log_mu), _ptr(eta), _ptr(initial_S), _ptr(initial_M),
+                                            _ptr(cu_seqlens), _ptr(out), _ptr(final_S), _ptr(final_M), _stream())
+    if st != 0:
+        raise MdnError(st, "mdn_chunk_fwd_static_scratch")
 
 
 def chunk_fwd_host(q, k, v, beta, log_alpha, log_mu, eta=None, *, initial_S=None, initial_M=None,

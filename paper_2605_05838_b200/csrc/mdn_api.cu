@@ -265,6 +265,7 @@ const char* mdn_status_string(mdn_status s) {
     case MDN_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
     case MDN_ERR_CUDA: return "CUDA runtime error";
     case MDN_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+    case MDN_ERR_STATIC_SCRATCH: return "problem needs more scratch than the built-in static buffer holds";
   }
   return "unknown status";
 }
