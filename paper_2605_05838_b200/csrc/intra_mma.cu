@@ -1,30 +1,37 @@
 // a2 for the tensor-core path: per (chunk, head)
-//   kk = K K^T, qk = Q K^T            warp-level bf16 tensor-core MMAs (fp32 accumulate), lower triangle only
+//   kk = K K^T, qk = Q K^T            warp-level bf16 tensor-core MMAs (fp32 accumulate), lower triangle only;
+//                                      K, Q tiles arrive by TMA (128-byte swizzle), fragments by swizzled ldmatrix
 //   Gamma (Eq. 10)                     column recurrences  gamma_{r,i} = alpha_r gamma_{r-1,i} + beta_r m_{r,i}
 //   A = tril(alpha_r gamma_{r-1,i} eta_i kk, -1)          = (P K^T) .* Gamma^-   (Gamma^- = Gamma shifted one row down)
-//   W = scale gamma_{r,i} eta_i qk                          written as bf16 hi + lo
-//   T = (I + A)^{-1}                   fp32, blocked: invert the four 16x16 diagonal blocks by forward
-//                                      substitution, then  T_21 = -T_22 A_21 T_11  at block sizes 16 and 32
-//                                      (Eq. 15; the paper substitutes row by row over all 64 rows)
-// One 128-thread CTA per (chunk, head); ~53 KB of shared memory, so four CTAs share an SM.
-// The K.K^T / Q.K^T products here are 12 % of the path's FLOPs and the kernel is bound by reading
-// q, k once and writing T, W: warp-level mma.sync is enough, the big contractions are in the chain kernel.
+//   W = scale gamma_{r,i} eta_i qk                          written from the fragments as bf16 hi + lo
+//   T = (I + A)^{-1}                   blocked: the four 16x16 diagonal blocks by fp32 forward substitution, then
+//                                      T_21 = -T_22 A_21 T_11 at block sizes 16 and 32 with tf32 tensor-core MMAs
+//                                      (Eq. 15; the paper substitutes row by row over all 64 rows).  T leaves as bf16,
+//                                      so tf32 (10-bit mantissa) block products cost nothing visible.
+// One 128-thread CTA per (chunk, head); ~51 KB of shared memory, four CTAs per SM.
+// The K K^T / Q K^T products are 12 % of the path's FLOPs and this kernel is bound by reading q, k
+// once and writing T, W: warp-level mma.sync is enough here, the big contractions are in the chain kernel.
+#include <cstring>
+
 #include "mdn_common.cuh"
+#include "tc_utils.cuh"
 
 namespace mdn {
 namespace {
 
+using namespace tc;
+
 constexpr int kThreads = 128;
 constexpr int kD = 128;
-constexpr int LDK = kD + 8;   // bf16 elements per smem row (272 B: 16-byte aligned, conflict-free for ldmatrix)
-constexpr int LM = C + 1;     // fp32 elements per row of the 64x64 matrices
+constexpr int LM = C + 4;     // fp32 elements per row of the 64x64 matrices (16-byte aligned rows)
 
-constexpr uint32_t kOffK = 0;
-constexpr uint32_t kOffQ = C * LDK * 2;              // 17408
-constexpr uint32_t kOffG = 2 * C * LDK * 2;          // 34816
-constexpr uint32_t kOffCv = kOffG + C * LM * 4;      // 51456
-constexpr uint32_t kSmem = kOffCv + 4 * C * 4;       // 52480
-static_assert(C * LM * 4 <= C * LDK * 2, "fp32 64x64 matrices alias the bf16 tiles");
+constexpr uint32_t kOffK = 0, kOffQ = 16384;                 // bf16 tiles, two [64 x 128 B] swizzled blocks each
+constexpr uint32_t kOffG = 32768;                            // Gamma [64][68] fp32; later T
+constexpr uint32_t kOffCv = kOffG + C * LM * 4;              // alpha, beta, mu, eta
+constexpr uint32_t kOffA = 0;                                // A [64][68] fp32 (aliases the tiles once the MMAs are done)
+constexpr uint32_t kOffP = C * LM * 4;                       // product scratch [32][68] fp32 (aliases the tiles too)
+constexpr uint32_t kSmem = kOffCv + 4 * C * 4 + 1024;        // + slack for the 1024-byte alignment
+static_assert(kOffP + 32 * LM * 4 <= kOffG, "A and the product scratch fit in the tile area");
 
 __device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
@@ -39,52 +46,104 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
+__device__ __forceinline__ uint32_t to_tf32(float x) {
+  uint32_t r;
+  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
+  return r;
+}
+__device__ __forceinline__ void mma_tf32(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+      "{%0, %1, %2, %3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
 
-__device__ __forceinline__ void load_tile(__nv_bfloat16* dst, const __nv_bfloat16* src, int row_stride, int n, int tid) {
-  for (int idx = tid; idx < C * (kD / 8); idx += kThreads) {
-    const int r = idx >> 4, c8 = idx & 15;
-    uint4 val = make_uint4(0, 0, 0, 0);
-    if (r < n) val = __ldg(reinterpret_cast<const uint4*>(src + (size_t)r * row_stride) + c8);
-    *reinterpret_cast<uint4*>(dst + r * LDK + c8 * 8) = val;
+// Byte offset of the 16-byte chunk `c16` (0..15 over the 128 columns) of row `row` in a swizzled tile.
+__device__ __forceinline__ uint32_t tile_chunk(uint32_t row, uint32_t c16) {
+  return (c16 >> 3) * 8192 + row * 128 + (((c16 & 7) ^ (row & 7)) << 4);
+}
+
+// C[16 x 8*NT] (+)= A[16 x 8*KS] * B[8*KS x 8*NT], fp32 matrices in shared memory (row stride LM), tf32 MMAs.
+// a: &A[row0][k0], b: &B[k0][col0].  Fragment coordinates: g = lane / 4, t = lane % 4.
+template <int KS, int NT>
+__device__ __forceinline__ void block_mma_tf32(float (&acc)[NT][4], const float* a, const float* b, int g, int t) {
+#pragma unroll
+  for (int ks = 0; ks < KS; ++ks) {
+    uint32_t af[4];
+    af[0] = to_tf32(a[g * LM + ks * 8 + t]);
+    af[1] = to_tf32(a[(g + 8) * LM + ks * 8 + t]);
+    af[2] = to_tf32(a[g * LM + ks * 8 + t + 4]);
+    af[3] = to_tf32(a[(g + 8) * LM + ks * 8 + t + 4]);
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      const uint32_t b0 = to_tf32(b[(ks * 8 + t) * LM + nt * 8 + g]);
+      const uint32_t b1 = to_tf32(b[(ks * 8 + t + 4) * LM + nt * 8 + g]);
+      mma_tf32(acc[nt], af, b0, b1);
+    }
   }
 }
 
-__global__ void __launch_bounds__(kThreads) intra_mma_kernel(ChunkGeom g, const __nv_bfloat16* __restrict__ q,
-                                                            const __nv_bfloat16* __restrict__ k,
+__global__ void __launch_bounds__(kThreads) intra_mma_kernel(ChunkGeom g, const __grid_constant__ CUtensorMap map_q,
+                                                            const __grid_constant__ CUtensorMap map_k,
                                                             const float* __restrict__ coef, float scale,
                                                             __nv_bfloat16* __restrict__ Tout,
-                                                            __nv_bfloat16* __restrict__ Wout, size_t w_lo_offset) {
-  extern __shared__ __align__(16) uint8_t smem[];
+                                                            __nv_bfloat16* __restrict__ Wout, size_t w_lo_offset,
+                                                            int32_t* __restrict__ status) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  __shared__ __align__(8) uint64_t bar_tiles;
+  __shared__ int abort_flag;
   const int slot = blockIdx.x / g.H, h = blockIdx.x % g.H;
   const SlotInfo si = slot_info(g, slot);
   if (si.seq < 0) return;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  __nv_bfloat16* Ks = reinterpret_cast<__nv_bfloat16*>(smem + kOffK);
-  __nv_bfloat16* Qs = reinterpret_cast<__nv_bfloat16*>(smem + kOffQ);
+  const int fg = lane >> 2, ft = lane & 3;   // MMA fragment coordinates
   float* Gs = reinterpret_cast<float*>(smem + kOffG);     // Gamma; later T
-  float* cv = reinterpret_cast<float*>(smem + kOffCv);    // alpha, beta, mu, eta
-  float* Af = reinterpret_cast<float*>(smem + kOffK);     // A    (aliases the K tile once the MMAs are done)
-  float* Wf = reinterpret_cast<float*>(smem + kOffQ);     // W    (aliases the Q tile); later product scratch
+  float* cv = reinterpret_cast<float*>(smem + kOffCv);
+  float* Af = reinterpret_cast<float*>(smem + kOffA);
+  float* Pf = reinterpret_cast<float*>(smem + kOffP);
   float* Tf = Gs;
+  const uint32_t bar = smem_u32(&bar_tiles);
+  const uint32_t s_base = smem_u32(smem);
 
-  const size_t tok = (size_t)si.tok0 * g.H + h;
-  load_tile(Ks, k + tok * kD, g.H * kD, si.n, tid);
-  load_tile(Qs, q + tok * kD, g.H * kD, si.n, tid);
+  if (tid == 0) {
+    abort_flag = 0;
+    mbar_init(bar, 1);
+    mbar_fence_init();
+    mbar_arrive_expect_tx(bar, 32768);
+    tma_load_2d(s_base + kOffK, &map_k, h * kD, si.tok0, bar);
+    tma_load_2d(s_base + kOffK + 8192, &map_k, h * kD + 64, si.tok0, bar);
+    tma_load_2d(s_base + kOffQ, &map_q, h * kD, si.tok0, bar);
+    tma_load_2d(s_base + kOffQ + 8192, &map_q, h * kD + 64, si.tok0, bar);
+  }
   const float* cf = coef + ((size_t)slot * g.H + h) * MDN_NUM_COEF * C;
   for (int idx = tid; idx < 4 * C; idx += kThreads) cv[idx] = cf[kAlpha * C + idx];
-  __syncthreads();
+  __syncthreads();   // coefficients in smem; barrier initialised before anyone waits on it
 
-  // ---- Gamma columns (threads 0..63) ahead of the light MMA share of warps 0 and 1
+  // ---- Gamma columns (threads 0..63) while the tiles are in flight
   if (tid < C) {
     const int i = tid;
     float m = 1.f, gam = 0.f;
-    for (int r = i; r < C; ++r) {
-      const float al = cv[0 * C + r], be = cv[1 * C + r], mu = cv[2 * C + r];
-      if (r > i) m *= mu;
-      gam = fmaf(be, m, al * gam);
-      Gs[r * LM + i] = gam;
+    for (int r4 = i & ~3; r4 < C; r4 += 4) {
+      const float4 al = *reinterpret_cast<const float4*>(cv + 0 * C + r4);
+      const float4 be = *reinterpret_cast<const float4*>(cv + 1 * C + r4);
+      const float4 mu = *reinterpret_cast<const float4*>(cv + 2 * C + r4);
+      const float alv[4] = {al.x, al.y, al.z, al.w}, bev[4] = {be.x, be.y, be.z, be.w}, muv[4] = {mu.x, mu.y, mu.z, mu.w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int r = r4 + e;
+        if (r >= i) {
+          if (r > i) m *= muv[e];
+          gam = fmaf(bev[e], m, alv[e] * gam);
+          Gs[r * LM + i] = gam;
+        }
+      }
     }
   }
+
+  bool ok = mbar_wait(bar, 0, &abort_flag);
+  __syncwarp();
 
   // ---- kk, qk for rows 16*warp .. +15, columns 0 .. 16*warp+15 (n-tiles of 8)
   float kk[8][4], qk[8][4];
@@ -92,22 +151,20 @@ __global__ void __launch_bounds__(kThreads) intra_mma_kernel(ChunkGeom g, const 
   for (int t = 0; t < 8; ++t)
 #pragma unroll
     for (int e = 0; e < 4; ++e) kk[t][e] = qk[t][e] = 0.f;
-  {
-    const int r0 = warp * 16;
-    const uint32_t a_row = r0 + (lane & 7) + ((lane >> 3) & 1) * 8, a_col = (lane >> 4) * 8;
-    const uint32_t b_row = (lane & 7) + (lane >> 4) * 8, b_col = ((lane >> 3) & 1) * 8;
-    const uint32_t ks_base = static_cast<uint32_t>(__cvta_generic_to_shared(Ks));
-    const uint32_t qs_base = static_cast<uint32_t>(__cvta_generic_to_shared(Qs));
+  if (ok) {
+    const uint32_t a_row = warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8, a_c = lane >> 4;
+    const uint32_t b_row = (lane & 7) + (lane >> 4) * 8, b_c = (lane >> 3) & 1;
+    const uint32_t ks_base = s_base + kOffK, qs_base = s_base + kOffQ;
 #pragma unroll 2
     for (int ks = 0; ks < kD / 16; ++ks) {
       uint32_t ka0, ka1, ka2, ka3, qa0, qa1, qa2, qa3;
-      ldmatrix_x4(ks_base + (a_row * LDK + ks * 16 + a_col) * 2, ka0, ka1, ka2, ka3);
-      ldmatrix_x4(qs_base + (a_row * LDK + ks * 16 + a_col) * 2, qa0, qa1, qa2, qa3);
+      ldmatrix_x4(ks_base + tile_chunk(a_row, ks * 2 + a_c), ka0, ka1, ka2, ka3);
+      ldmatrix_x4(qs_base + tile_chunk(a_row, ks * 2 + a_c), qa0, qa1, qa2, qa3);
 #pragma unroll
       for (int tp = 0; tp < 4; ++tp) {
         if (tp <= warp) {   // n-tiles 2tp, 2tp+1 cover columns 16tp .. 16tp+15
           uint32_t b0, b1, b2, b3;
-          ldmatrix_x4(ks_base + ((tp * 16 + b_row) * LDK + ks * 16 + b_col) * 2, b0, b1, b2, b3);
+          ldmatrix_x4(ks_base + tile_chunk(tp * 16 + b_row, ks * 2 + b_c), b0, b1, b2, b3);
           mma_bf16(kk[2 * tp], ka0, ka1, ka2, ka3, b0, b1);
           mma_bf16(kk[2 * tp + 1], ka0, ka1, ka2, ka3, b2, b3);
           mma_bf16(qk[2 * tp], qa0, qa1, qa2, qa3, b0, b1);
@@ -118,53 +175,58 @@ __global__ void __launch_bounds__(kThreads) intra_mma_kernel(ChunkGeom g, const 
   }
   __syncthreads();   // Gamma complete; every warp is done reading the K and Q tiles
 
-  // ---- A and W from the accumulator fragments (rows lane/4 and lane/4+8, column pairs)
+  // ---- A (to smem, fp32) and W (to global, bf16 hi + lo) from the accumulator fragments.
+  // Tokens past the end of a short chunk (rows >= n hold another sequence's data) are masked here.
+  const size_t mat = ((size_t)slot * g.H + h) * C * C;
   {
-    const int rbase = warp * 16 + (lane >> 2), cbase = (lane & 3) * 2;
+    const int rbase = warp * 16 + fg, cbase = ft * 2;
 #pragma unroll
     for (int t = 0; t < 8; ++t) {
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const int r = rbase + (e >> 1) * 8, i = t * 8 + cbase + (e & 1);
-        float av = 0.f, wv = 0.f;
-        if (i <= r) {
-          const float et = cv[3 * C + i];
-          wv = scale * Gs[r * LM + i] * et * qk[t][e];
-          if (i < r) av = cv[0 * C + r] * Gs[(r - 1) * LM + i] * et * kk[t][e];
+      for (int half = 0; half < 2; ++half) {
+        const int r = rbase + half * 8, i0 = t * 8 + cbase;
+        float av[2] = {0.f, 0.f}, wv[2] = {0.f, 0.f};
+        if (r < si.n) {
+          const float alr = cv[0 * C + r];
+#pragma unroll
+          for (int e = 0; e < 2; ++e) {
+            const int i = i0 + e;
+            if (i <= r) {
+              const float et = cv[3 * C + i];
+              wv[e] = scale * Gs[r * LM + i] * et * qk[t][half * 2 + e];
+              if (i < r) av[e] = alr * Gs[(r - 1) * LM + i] * et * kk[t][half * 2 + e];
+            }
+          }
         }
-        Af[r * LM + i] = av;
-        Wf[r * LM + i] = wv;
+        *reinterpret_cast<float2*>(Af + r * LM + i0) = make_float2(av[0], av[1]);
+        uint32_t hi, lo;
+        split_pack_bf16(wv[0], wv[1], hi, lo);
+        *reinterpret_cast<uint32_t*>(Wout + mat + r * C + i0) = hi;
+        *reinterpret_cast<uint32_t*>(Wout + w_lo_offset + mat + r * C + i0) = lo;
       }
     }
   }
-  __syncthreads();   // A, W complete; Gamma no longer needed (T takes its place)
+  __syncthreads();   // A complete; Gamma no longer needed (T takes its place)
+  for (int idx = tid; idx < C * LM / 4; idx += kThreads) reinterpret_cast<float4*>(Tf)[idx] = make_float4(0.f, 0.f, 0.f, 0.f);
+  __syncthreads();
 
-  const size_t mat = ((size_t)slot * g.H + h) * C * C;
-  // ---- W out as bf16 hi + lo (16-byte stores), and step 1 of the inverse on threads 0..63
-  for (int idx = tid; idx < C * 8; idx += kThreads) {
-    const int r = idx >> 3, c0 = (idx & 7) * 8;
-    __align__(16) __nv_bfloat16 hi[8], lo[8];
-#pragma unroll
-    for (int x = 0; x < 8; ++x) {
-      const float w = Wf[r * LM + c0 + x];
-      hi[x] = __float2bfloat16_rn(w);
-      lo[x] = __float2bfloat16_rn(w - __bfloat162float(hi[x]));
-    }
-    *reinterpret_cast<uint4*>(Wout + mat + r * C + c0) = *reinterpret_cast<const uint4*>(hi);
-    *reinterpret_cast<uint4*>(Wout + w_lo_offset + mat + r * C + c0) = *reinterpret_cast<const uint4*>(lo);
-  }
-  for (int idx = tid; idx < C * LM; idx += kThreads) Tf[idx] = 0.f;
-  __syncthreads();   // W is out (its buffer becomes scratch); T zeroed
-
-  // step 1: D_b = (I + A_bb)^{-1} for the four 16x16 diagonal blocks; thread = (block, column)
+  // step 1: D_b = (I + A_bb)^{-1} for the four 16x16 diagonal blocks; thread = (block, column), fp32
   if (tid < C) {
     const int b0 = (tid >> 4) * 16, j = tid & 15;
     float x[16];
 #pragma unroll
     for (int r = 0; r < 16; ++r) {
+      float arow[16];
+#pragma unroll
+      for (int m4 = 0; m4 < 16; m4 += 4) {
+        if (m4 < r) {
+          const float4 v4 = *reinterpret_cast<const float4*>(Af + (b0 + r) * LM + b0 + m4);
+          arow[m4] = v4.x; arow[m4 + 1] = v4.y; arow[m4 + 2] = v4.z; arow[m4 + 3] = v4.w;
+        }
+      }
       float acc = (r == j) ? 1.f : 0.f;
 #pragma unroll
-      for (int m = 0; m < r; ++m) acc = fmaf(-Af[(b0 + r) * LM + b0 + m], x[m], acc);
+      for (int m = 0; m < r; ++m) acc = fmaf(-arow[m], x[m], acc);
       x[r] = acc;
     }
 #pragma unroll
@@ -172,68 +234,58 @@ __global__ void __launch_bounds__(kThreads) intra_mma_kernel(ChunkGeom g, const 
   }
   __syncthreads();
 
-  float* Pf = Wf;   // product scratch, row stride LM
-  // step 2: inside each 32x32 diagonal block s: T_lo = -D_hi (A_lo D_lo), 16x16 blocks
-  {
-    const int s = tid >> 6, rr = (tid & 63) >> 2, c0 = (tid & 3) * 4;
-    const int R0 = 32 * s + 16, C0 = 32 * s;
-    float acc[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll 4
-    for (int m = 0; m < 16; ++m) {
-      const float av = Af[(R0 + rr) * LM + C0 + m];
+  // step 2: inside each 32x32 diagonal block s: T_lo = -D_hi (A_lo D_lo); 16x16 blocks, warp s does block s
+  if (warp < 2) {
+    const int R0 = 32 * warp + 16, C0 = 32 * warp;
+    float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+    block_mma_tf32<2, 2>(acc, Af + R0 * LM + C0, Tf + C0 * LM + C0, fg, ft);
+    float* P = Pf + warp * 16 * LM;
 #pragma unroll
-      for (int x = 0; x < 4; ++x) acc[x] = fmaf(av, Tf[(C0 + m) * LM + C0 + c0 + x], acc[x]);
+    for (int nt = 0; nt < 2; ++nt) {
+      *reinterpret_cast<float2*>(P + fg * LM + nt * 8 + 2 * ft) = make_float2(acc[nt][0], acc[nt][1]);
+      *reinterpret_cast<float2*>(P + (fg + 8) * LM + nt * 8 + 2 * ft) = make_float2(acc[nt][2], acc[nt][3]);
     }
+    __syncwarp();
+    float acc2[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+    block_mma_tf32<2, 2>(acc2, Tf + R0 * LM + R0, P, fg, ft);
 #pragma unroll
-    for (int x = 0; x < 4; ++x) Pf[(R0 + rr) * LM + c0 + x] = acc[x];
-    __syncthreads();
-#pragma unroll
-    for (int x = 0; x < 4; ++x) acc[x] = 0.f;
-#pragma unroll 4
-    for (int m = 0; m < 16; ++m) {
-      const float tv = Tf[(R0 + rr) * LM + R0 + m];
-#pragma unroll
-      for (int x = 0; x < 4; ++x) acc[x] = fmaf(tv, Pf[(R0 + m) * LM + c0 + x], acc[x]);
+    for (int nt = 0; nt < 2; ++nt) {
+      *reinterpret_cast<float2*>(Tf + (R0 + fg) * LM + C0 + nt * 8 + 2 * ft) = make_float2(-acc2[nt][0], -acc2[nt][1]);
+      *reinterpret_cast<float2*>(Tf + (R0 + fg + 8) * LM + C0 + nt * 8 + 2 * ft) = make_float2(-acc2[nt][2], -acc2[nt][3]);
     }
-#pragma unroll
-    for (int x = 0; x < 4; ++x) Tf[(R0 + rr) * LM + C0 + c0 + x] = -acc[x];
   }
   __syncthreads();
-  // step 3: T[32:64, 0:32] = -T[32:64, 32:64] (A[32:64, 0:32] T[0:32, 0:32])
+  // step 3: T[32:64, 0:32] = -T[32:64, 32:64] (A[32:64, 0:32] T[0:32, 0:32]); warp = (row tile, column half)
   {
-    const int rr = tid >> 2, c0 = (tid & 3) * 8;
-    float acc[8];
+    const int mt = warp & 1, n0 = (warp >> 1) * 16;
+    float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+    block_mma_tf32<4, 2>(acc, Af + (32 + 16 * mt) * LM, Tf + n0, fg, ft);
 #pragma unroll
-    for (int x = 0; x < 8; ++x) acc[x] = 0.f;
-#pragma unroll 4
-    for (int m = 0; m < 32; ++m) {
-      const float av = Af[(32 + rr) * LM + m];
-#pragma unroll
-      for (int x = 0; x < 8; ++x) acc[x] = fmaf(av, Tf[m * LM + c0 + x], acc[x]);
+    for (int nt = 0; nt < 2; ++nt) {
+      *reinterpret_cast<float2*>(Pf + (16 * mt + fg) * LM + n0 + nt * 8 + 2 * ft) = make_float2(acc[nt][0], acc[nt][1]);
+      *reinterpret_cast<float2*>(Pf + (16 * mt + fg + 8) * LM + n0 + nt * 8 + 2 * ft) = make_float2(acc[nt][2], acc[nt][3]);
     }
-#pragma unroll
-    for (int x = 0; x < 8; ++x) Pf[rr * LM + c0 + x] = acc[x];
     __syncthreads();
+    float acc2[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+    block_mma_tf32<4, 2>(acc2, Tf + (32 + 16 * mt) * LM + 32, Pf + n0, fg, ft);
 #pragma unroll
-    for (int x = 0; x < 8; ++x) acc[x] = 0.f;
-#pragma unroll 4
-    for (int m = 0; m < 32; ++m) {
-      const float tv = Tf[(32 + rr) * LM + 32 + m];
-#pragma unroll
-      for (int x = 0; x < 8; ++x) acc[x] = fmaf(tv, Pf[m * LM + c0 + x], acc[x]);
+    for (int nt = 0; nt < 2; ++nt) {
+      *reinterpret_cast<float2*>(Tf + (32 + 16 * mt + fg) * LM + n0 + nt * 8 + 2 * ft) = make_float2(-acc2[nt][0], -acc2[nt][1]);
+      *reinterpret_cast<float2*>(Tf + (32 + 16 * mt + fg + 8) * LM + n0 + nt * 8 + 2 * ft) = make_float2(-acc2[nt][2], -acc2[nt][3]);
     }
-#pragma unroll
-    for (int x = 0; x < 8; ++x) Tf[(32 + rr) * LM + c0 + x] = -acc[x];
   }
   __syncthreads();
 
   for (int idx = tid; idx < C * 8; idx += kThreads) {
     const int r = idx >> 3, c0 = (idx & 7) * 8;
-    __align__(16) __nv_bfloat16 tv[8];
-#pragma unroll
-    for (int x = 0; x < 8; ++x) tv[x] = __float2bfloat16_rn(Tf[r * LM + c0 + x]);
-    *reinterpret_cast<uint4*>(Tout + mat + r * C + c0) = *reinterpret_cast<const uint4*>(tv);
+    const float4 t0 = *reinterpret_cast<const float4*>(Tf + r * LM + c0);
+    const float4 t1 = *reinterpret_cast<const float4*>(Tf + r * LM + c0 + 4);
+    uint4 packed;
+    packed.x = pack_bf16(t0.x, t0.y); packed.y = pack_bf16(t0.z, t0.w);
+    packed.z = pack_bf16(t1.x, t1.y); packed.w = pack_bf16(t1.z, t1.w);
+    *reinterpret_cast<uint4*>(Tout + mat + r * C + c0) = packed;
   }
+  if (!ok && tid == 0) atomicCAS(status, kDevOk, kDevTimeout);
 }
 
 }  // namespace
@@ -242,11 +294,15 @@ cudaError_t launch_intra_mma(const Plan& pl, const void* q, const void* k, int* 
   cudaError_t e = cudaFuncSetAttribute(intra_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmem);
   if (e != cudaSuccess) return e;
   const size_t n_mats = (size_t)pl.geom.num_slots * pl.p.H;
+  const uint64_t tokens = (uint64_t)pl.p.B * pl.p.T, row = (uint64_t)pl.p.H * kD;
+  CUtensorMap mq, mk;
+  if (!encode_tma_2d_bf16(&mq, TmaMap2D{q, row, tokens, row * 2, 64, 64, true}) ||
+      !encode_tma_2d_bf16(&mk, TmaMap2D{k, row, tokens, row * 2, 64, 64, true}))
+    return cudaErrorInvalidValue;
   intra_mma_kernel<<<(unsigned)n_mats, kThreads, kSmem, pl.stream>>>(
-      pl.geom, static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(k),
-      reinterpret_cast<const float*>(pl.ws + pl.lay.off_coef), pl.p.scale,
+      pl.geom, mq, mk, reinterpret_cast<const float*>(pl.ws + pl.lay.off_coef), pl.p.scale,
       reinterpret_cast<__nv_bfloat16*>(pl.ws + pl.lay.off_T), reinterpret_cast<__nv_bfloat16*>(pl.ws + pl.lay.off_W),
-      n_mats * C * C);
+      n_mats * C * C, reinterpret_cast<int32_t*>(pl.ws + pl.lay.off_status));
   e = cudaGetLastError();
   if (e == cudaSuccess) ++*launches;
   return e;

@@ -144,6 +144,45 @@ def test_intra_chunk_T_and_W_match_eq15(mdn):
             assert np.allclose(Wm[c, h], W_ref, rtol=1e-4, atol=1e-6)
 
 
+def test_intra_chunk_tensor_path_T_and_W(mdn):
+    """bf16 T and W_hi + W_lo of the tensor-path kernel (tf32 block products inside the inverse)."""
+    import torch
+    from oracle import chunkwise as cw
+    w = wl.Workload("intra_t", B=1, T=250, H=2, dk=128, dv=128, dtype="bf16", seed=6, preset="F")
+    if not tensor_ok(mdn, w):
+        pytest.skip("tensor path not built")
+    inp = wl.make_inputs(w)
+    inp["k"] = wl.correlated_keys(w, 0.8)
+    t = to_torch(inp)
+    p = mdn.make_params(t["q"], t["v"], scale=inp["scale"], path="tensor")
+    lay = mdn.workspace_layout(p)
+    assert lay.mat_dtype == 1
+    ws = torch.zeros(lay.total_bytes, dtype=torch.uint8, device="cuda")
+    mdn.coeff_scan(p, t["beta"], t["log_alpha"], t["log_mu"], t["eta"], None, ws)
+    mdn.intra_chunk(p, t["q"], t["k"], None, ws)
+    torch.cuda.synchronize()
+    assert mdn.read_status(p, ws) == 0
+    nm = lay.num_slots * w.H * 64 * 64
+    def mats(off):
+        return ws[off: off + 2 * nm].view(torch.bfloat16).float().cpu().numpy().reshape(lay.num_slots, w.H, 64, 64)
+    Tm, Wh, Wl = mats(lay.off_T), mats(lay.off_W), mats(lay.off_W + 2 * nm)
+    for h in range(w.H):
+        _, _, _, stages = cw.chunk_forward(inp["q"][0, :, h], inp["k"][0, :, h], inp["v"][0, :, h],
+                                           inp["beta"][0, :, h], inp["log_alpha"][0, :, h], inp["log_mu"][0, :, h],
+                                           inp["eta"][0, :, h], scale=inp["scale"], return_stages=True)
+        for c, st in enumerate(stages):
+            n = st["n"]
+            assert np.abs(st["T"] - np.eye(64)).max() > 0.05
+            # bf16 storage of T: one rounding (2^-8 relative) plus the tf32 block products
+            assert np.abs(Tm[c, h] - st["T"]).max() <= 2.0 ** -8 * np.abs(st["T"]).max() + 2e-3
+            assert (np.triu(Tm[c, h], 1) == 0).all() and (np.diag(Tm[c, h]) == 1).all()
+            sl = slice(64 * c, 64 * c + n)
+            Q = np.zeros((64, 128)); K = np.zeros((64, 128)); et = np.zeros(64)
+            Q[:n] = inp["q"][0, sl, h]; K[:n] = inp["k"][0, sl, h]; et[:n] = inp["eta"][0, sl, h]
+            W_ref = inp["scale"] * (Q @ (et[:, None] * K).T) * st["Gamma"]
+            assert np.allclose(Wh[c, h] + Wl[c, h], W_ref, rtol=1e-4, atol=1e-6)     # hi + lo ~ 16 mantissa bits
+
+
 # ------------------------------------------------------------------------------------------ named configs
 def test_config0_tiny_fp32(mdn):
     inp = wl.make_inputs(wl.CONFIGS[0])
