@@ -225,6 +225,10 @@ mdn_status mdn_set_stage_events(void* const* events /* host */, int32_t n);
 mdn_status mdn_selftest_umma(int32_t mode, const void* a, const void* b, float* out, int32_t* status,
                              void* cuda_stream);
 
+/* Text of the CUDA runtime error behind the last MDN_ERR_CUDA returned on this host thread by the
+ * intra-chunk or chain launches (static string, host pointer). */
+const char* mdn_last_cuda_error_string(void);
+
 /* Number of kernels the last mdn_* call on this host thread enqueued. */
 int32_t mdn_last_launch_count(void);
 

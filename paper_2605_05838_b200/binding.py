@@ -43,7 +43,10 @@ class MdnWsLayout(ctypes.Structure):
 class MdnError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
-        super().__init__("%s: %s (status %d)" % (where, status_string(status), status))
+        detail = ""
+        if status == 4:
+            detail = ": " + lib().mdn_last_cuda_error_string().decode()
+        super().__init__("%s: %s (status %d)%s" % (where, status_string(status), status, detail))
 
 
 _lib = None
@@ -81,6 +84,8 @@ def lib() -> ctypes.CDLL:
         L.mdn_set_stage_events.argtypes = [ctypes.POINTER(vp), ctypes.c_int32]
         L.mdn_selftest_umma.restype = ctypes.c_int
         L.mdn_selftest_umma.argtypes = [ctypes.c_int32, vp, vp, vp, vp, vp]
+        L.mdn_last_cuda_error_string.restype = ctypes.c_char_p
+        L.mdn_last_cuda_error_string.argtypes = []
         L.mdn_last_launch_count.restype = ctypes.c_int32
         L.mdn_last_launch_count.argtypes = []
         _lib = L

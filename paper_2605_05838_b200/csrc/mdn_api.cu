@@ -7,6 +7,7 @@
 namespace mdn {
 
 static thread_local int t_last_launches = 0;
+static thread_local int t_last_cuda_error = 0;
 static thread_local cudaEvent_t t_stage_events[MDN_NUM_STAGE_EVENTS] = {nullptr, nullptr, nullptr, nullptr};
 static thread_local bool t_stage_events_on = false;
 
@@ -98,6 +99,7 @@ static mdn_status run_intra(const Plan& pl, const void* q, const void* k, int* l
   if (!q || !k || !aligned(q, 16) || !aligned(k, 16)) return MDN_ERR_INVALID_ARG;
   cudaError_t e = pl.p.path == MDN_PATH_TENSOR ? launch_intra_tensor(pl, q, k, launches)
                                                : launch_intra_simt(pl, q, k, launches);
+  if (e != cudaSuccess) t_last_cuda_error = (int)e;
   return e == cudaSuccess ? MDN_OK : MDN_ERR_CUDA;
 }
 
@@ -162,7 +164,7 @@ mdn_status mdn_chunk_fwd(const mdn_params* p, const void* q, const void* k, cons
   cudaError_t e = pl.p.path == MDN_PATH_TENSOR
                       ? launch_chain_tensor(pl, q, k, v, initial_S, initial_M, o, final_S, final_M, &t_last_launches)
                       : launch_chain_simt(pl, q, k, v, initial_S, initial_M, o, final_S, final_M, &t_last_launches);
-  if (e != cudaSuccess) return MDN_ERR_CUDA;
+  if (e != cudaSuccess) { t_last_cuda_error = (int)e; return MDN_ERR_CUDA; }
   if (!mark_stage(3, pl.stream)) return MDN_ERR_CUDA;
   return MDN_OK;
 }
@@ -271,5 +273,9 @@ const char* mdn_status_string(mdn_status s) {
 }
 
 int32_t mdn_last_launch_count(void) { return t_last_launches; }
+
+const char* mdn_last_cuda_error_string(void) {
+  return t_last_cuda_error == 0 ? "no CUDA error recorded" : cudaGetErrorString((cudaError_t)t_last_cuda_error);
+}
 
 }  // extern "C"

@@ -262,6 +262,60 @@ def test_degenerate_gates(mdn):
     assert max(rel_err(o, o_ref), rel_err(S, S_ref), rel_err(M, M_ref)) <= TOL_F32
 
 
+@pytest.mark.parametrize("T", [1, 2, 63, 64, 65, 127, 129, 300])
+def test_ragged_lengths_tensor_path(mdn, T):
+    w = wl.Workload("ragged_bf16", B=2, T=T, H=2, dk=128, dv=128, dtype="bf16", init_state_std=0.3, seed=31)
+    if not tensor_ok(mdn, w):
+        pytest.skip("tensor path not built")
+    compare(mdn, wl.make_inputs(w), "tensor", label="tensor T=%d" % T)
+
+
+def test_degenerate_gates_tensor_path(mdn):
+    """beta = 0 tokens, mu = 0 tokens, mu = 0 everywhere (gated delta rule), eta = None, scale = 1 on tcgen05."""
+    w = wl.Workload("degenerate_bf16", B=2, T=200, H=2, dk=128, dv=128, dtype="bf16", seed=32)
+    if not tensor_ok(mdn, w):
+        pytest.skip("tensor path not built")
+    inp = wl.make_inputs(w)
+    inp["beta"][:, 10:30] = 0.0
+    inp["log_mu"][:, 40:150] = -np.inf
+    compare(mdn, inp, "tensor", label="tensor beta=0 / mu=0 tokens")
+    inp2 = wl.make_inputs(w)
+    inp2["log_mu"][:] = -np.inf
+    compare(mdn, inp2, "tensor", label="tensor mu=0 everywhere")
+    inp3 = wl.make_inputs(w)
+    inp3["eta"] = None
+    inp3["scale"] = 1.0
+    compare(mdn, inp3, "tensor", label="tensor eta=None scale=1")
+    inp4 = wl.make_inputs(w)
+    inp4["beta"][:] = 0.0
+    inp4["S0"] = np.random.default_rng(0).standard_normal((2, 2, 128, 128)).astype(np.float32)
+    import torch
+    o, S, M = run_gpu(mdn, inp4, path="tensor", o_dtype=torch.float32)
+    abar = np.exp(np.cumsum(inp4["log_alpha"].astype(np.float64), axis=1))[:, -1]
+    assert np.allclose(S, abar[:, :, None, None] * inp4["S0"], rtol=1e-4, atol=1e-7)    # purely decayed state, exact path
+
+
+def test_state_handoff_and_determinism_tensor_path(mdn):
+    import torch
+    w = wl.Workload("handoff_bf16", B=1, T=512, H=3, dk=128, dv=128, dtype="bf16", init_state_std=0.1, seed=33)
+    if not tensor_ok(mdn, w):
+        pytest.skip("tensor path not built")
+    inp = wl.make_inputs(w)
+    o, S, M = run_gpu(mdn, inp, path="tensor")
+    o2, S2, M2 = run_gpu(mdn, inp, path="tensor")
+    assert np.array_equal(o, o2) and np.array_equal(S, S2) and np.array_equal(M, M2)
+    a = dict(inp); b = dict(inp)
+    for name in ("q", "k", "v", "beta", "log_alpha", "log_mu", "eta"):
+        a[name] = inp[name][:, :256]; b[name] = inp[name][:, 256:]
+    a["workload"] = b["workload"] = dataclasses.replace(w, T=256)
+    oa, Sa, Ma = run_gpu(mdn, a, path="tensor")
+    b["S0"], b["M0"] = Sa.astype(np.float32), Ma.astype(np.float32)
+    ob, Sb, Mb = run_gpu(mdn, b, path="tensor")
+    # the split falls on a chunk boundary and the state is handed over in fp32: same arithmetic
+    assert np.array_equal(o[:, :256], oa) and np.array_equal(o[:, 256:], ob)
+    assert np.array_equal(S, Sb) and np.array_equal(M, Mb)
+
+
 def test_packed_varlen_edge_lengths(mdn):
     lens = np.array([1, 63, 64, 65, 129, 2, 300, 128])
     w = small(B=1, T=int(lens.sum()), varlen=True, init_state_std=0.4)
