@@ -116,6 +116,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int H = a.g.H;
   const int seq = blockIdx.x / H, h = blockIdx.x % H;
+  grid_dependency_wait();   // chunk map, coefficients, T and W come from the previous kernels
   const SeqInfo sq = seq_info(a.g, seq);
   const int nch = sq.nchunks;
   const size_t st_off = ((size_t)seq * H + h) * kD * kD;
@@ -575,14 +576,14 @@ cudaError_t launch_chain_tensor(const Plan& pl, const void* q, const void* k, co
     auto kern = chain_tensor_kernel<__nv_bfloat16>;
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
     if (e != cudaSuccess) return e;
-    kern<<<grid, kThreads, kSmemBytes, pl.stream>>>(a, mq, mk, mv, mt, mw, mo);
+    e = launch_pdl(kern, dim3(grid), dim3(kThreads), kSmemBytes, pl.stream, a, mq, mk, mv, mt, mw, mo);
   } else {
     auto kern = chain_tensor_kernel<float>;
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
     if (e != cudaSuccess) return e;
-    kern<<<grid, kThreads, kSmemBytes, pl.stream>>>(a, mq, mk, mv, mt, mw, mo);
+    e = launch_pdl(kern, dim3(grid), dim3(kThreads), kSmemBytes, pl.stream, a, mq, mk, mv, mt, mw, mo);
   }
-  e = cudaGetLastError();
+  if (e == cudaSuccess) e = cudaGetLastError();
   if (e == cudaSuccess) ++*launches;
   return e;
 }

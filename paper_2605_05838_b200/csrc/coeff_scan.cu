@@ -127,6 +127,7 @@ __global__ void __launch_bounds__(kScanWarps * 32) coeff_scan_kernel(ChunkGeom g
                                                                     float* __restrict__ coef) {
   extern __shared__ float sm[];   // [4][64*H]: log_alpha, log_mu, beta, eta
   const int slot = blockIdx.x;
+  grid_dependency_wait();   // the chunk map (packed input) comes from the previous kernel
   const SlotInfo si = slot_info(g, slot);
   if (si.seq < 0) return;
   const int H = g.H, tid = threadIdx.x;
@@ -205,6 +206,7 @@ __global__ void __launch_bounds__(kScanWarps * 32) coeff_scan_kernel(ChunkGeom g
     put(kEta, et[0], et[1]);
     put(kMubar, mbar0, mbar1);
   }
+  grid_launch_dependents();
 }
 
 cudaError_t launch_coeff_scan(const Plan& pl, const float* beta, const float* log_alpha, const float* log_mu,

@@ -95,6 +95,7 @@ __global__ void __launch_bounds__(kThreads) intra_mma_kernel(ChunkGeom g, const 
   __shared__ __align__(8) uint64_t bar_tiles;
   __shared__ int abort_flag;
   const int slot = blockIdx.x / g.H, h = blockIdx.x % g.H;
+  grid_dependency_wait();   // chunk map and coefficients come from the previous kernels
   const SlotInfo si = slot_info(g, slot);
   if (si.seq < 0) return;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -286,6 +287,7 @@ __global__ void __launch_bounds__(kThreads) intra_mma_kernel(ChunkGeom g, const 
     *reinterpret_cast<uint4*>(Tout + mat + r * C + c0) = packed;
   }
   if (!ok && tid == 0) atomicCAS(status, kDevOk, kDevTimeout);
+  grid_launch_dependents();
 }
 
 }  // namespace
@@ -299,11 +301,12 @@ cudaError_t launch_intra_mma(const Plan& pl, const void* q, const void* k, int* 
   if (!encode_tma_2d_bf16(&mq, TmaMap2D{q, row, tokens, row * 2, 64, 64, true}) ||
       !encode_tma_2d_bf16(&mk, TmaMap2D{k, row, tokens, row * 2, 64, 64, true}))
     return cudaErrorInvalidValue;
-  intra_mma_kernel<<<(unsigned)n_mats, kThreads, kSmem, pl.stream>>>(
-      pl.geom, mq, mk, reinterpret_cast<const float*>(pl.ws + pl.lay.off_coef), pl.p.scale,
-      reinterpret_cast<__nv_bfloat16*>(pl.ws + pl.lay.off_T), reinterpret_cast<__nv_bfloat16*>(pl.ws + pl.lay.off_W),
-      n_mats * C * C, reinterpret_cast<int32_t*>(pl.ws + pl.lay.off_status));
-  e = cudaGetLastError();
+  e = launch_pdl(intra_mma_kernel, dim3((unsigned)n_mats), dim3(kThreads), kSmem, pl.stream, pl.geom, mq, mk,
+                 reinterpret_cast<const float*>(pl.ws + pl.lay.off_coef), pl.p.scale,
+                 reinterpret_cast<__nv_bfloat16*>(pl.ws + pl.lay.off_T),
+                 reinterpret_cast<__nv_bfloat16*>(pl.ws + pl.lay.off_W), n_mats * C * C,
+                 reinterpret_cast<int32_t*>(pl.ws + pl.lay.off_status));
+  if (e == cudaSuccess) e = cudaGetLastError();
   if (e == cudaSuccess) ++*launches;
   return e;
 }
