@@ -28,10 +28,15 @@ constexpr int LM = C + 4;     // fp32 elements per row of the 64x64 matrices (16
 constexpr uint32_t kOffK = 0, kOffQ = 16384;                 // bf16 tiles, two [64 x 128 B] swizzled blocks each
 constexpr uint32_t kOffG = 32768;                            // Gamma [64][68] fp32; later T
 constexpr uint32_t kOffCv = kOffG + C * LM * 4;              // alpha, beta, mu, eta
-constexpr uint32_t kOffA = 0;                                // A [64][68] fp32 (aliases the tiles once the MMAs are done)
-constexpr uint32_t kOffP = C * LM * 4;                       // product scratch [32][68] fp32 (aliases the tiles too)
+// the tile area is reused once the MMAs are done: first as the bf16 staging of W_hi / W_lo, then for A and scratch
+constexpr int LW = C + 8;                                    // bf16 elements per staged W row (144 B: conflict-free)
+constexpr uint32_t kOffWh = 0, kOffWl = C * LW * 2;          // W_hi, W_lo staging [64][72] bf16
+constexpr uint32_t kOffA = 0;                                // A [64][68] fp32
+constexpr int LD16 = 16 * 16 + 4;                            // floats per compact 16x16 diagonal block (+4: bank shift)
+constexpr uint32_t kOffAd = C * LM * 4;                      // the four diagonal blocks of A, compact
+constexpr uint32_t kOffP = kOffAd + 4 * LD16 * 4;            // product scratch [32][68] fp32
 constexpr uint32_t kSmem = kOffCv + 4 * C * 4 + 1024;        // + slack for the 1024-byte alignment
-static_assert(kOffP + 32 * LM * 4 <= kOffG, "A and the product scratch fit in the tile area");
+static_assert(kOffP + 32 * LM * 4 <= kOffG && kOffWl + C * LW * 2 <= kOffG, "reuse of the tile area");
 
 __device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
@@ -103,7 +108,10 @@ __global__ void __launch_bounds__(kThreads) intra_mma_kernel(ChunkGeom g, const 
   float* Gs = reinterpret_cast<float*>(smem + kOffG);     // Gamma; later T
   float* cv = reinterpret_cast<float*>(smem + kOffCv);
   float* Af = reinterpret_cast<float*>(smem + kOffA);
+  float* Ad = reinterpret_cast<float*>(smem + kOffAd);
   float* Pf = reinterpret_cast<float*>(smem + kOffP);
+  __nv_bfloat16* Wsh = reinterpret_cast<__nv_bfloat16*>(smem + kOffWh);
+  __nv_bfloat16* Wsl = reinterpret_cast<__nv_bfloat16*>(smem + kOffWl);
   float* Tf = Gs;
   const uint32_t bar = smem_u32(&bar_tiles);
   const uint32_t s_base = smem_u32(smem);
@@ -176,35 +184,53 @@ __global__ void __launch_bounds__(kThreads) intra_mma_kernel(ChunkGeom g, const 
   }
   __syncthreads();   // Gamma complete; every warp is done reading the K and Q tiles
 
-  // ---- A (to smem, fp32) and W (to global, bf16 hi + lo) from the accumulator fragments.
+  // ---- W, then A, from the accumulator fragments (rows fg and fg + 8 of the warp's 16, column pairs).
   // Tokens past the end of a short chunk (rows >= n hold another sequence's data) are masked here.
   const size_t mat = ((size_t)slot * g.H + h) * C * C;
-  {
-    const int rbase = warp * 16 + fg, cbase = ft * 2;
+  const int rbase = warp * 16 + fg, cbase = ft * 2;
 #pragma unroll
-    for (int t = 0; t < 8; ++t) {
+  for (int t = 0; t < 8; ++t) {
 #pragma unroll
-      for (int half = 0; half < 2; ++half) {
-        const int r = rbase + half * 8, i0 = t * 8 + cbase;
-        float av[2] = {0.f, 0.f}, wv[2] = {0.f, 0.f};
-        if (r < si.n) {
-          const float alr = cv[0 * C + r];
+    for (int half = 0; half < 2; ++half) {
+      const int r = rbase + half * 8, i0 = t * 8 + cbase;
+      float wv[2] = {0.f, 0.f};
+      if (r < si.n) {
 #pragma unroll
-          for (int e = 0; e < 2; ++e) {
-            const int i = i0 + e;
-            if (i <= r) {
-              const float et = cv[3 * C + i];
-              wv[e] = scale * Gs[r * LM + i] * et * qk[t][half * 2 + e];
-              if (i < r) av[e] = alr * Gs[(r - 1) * LM + i] * et * kk[t][half * 2 + e];
-            }
-          }
+        for (int e = 0; e < 2; ++e) {
+          const int i = i0 + e;
+          if (i <= r) wv[e] = scale * Gs[r * LM + i] * cv[3 * C + i] * qk[t][half * 2 + e];
         }
-        *reinterpret_cast<float2*>(Af + r * LM + i0) = make_float2(av[0], av[1]);
-        uint32_t hi, lo;
-        split_pack_bf16(wv[0], wv[1], hi, lo);
-        *reinterpret_cast<uint32_t*>(Wout + mat + r * C + i0) = hi;
-        *reinterpret_cast<uint32_t*>(Wout + w_lo_offset + mat + r * C + i0) = lo;
       }
+      uint32_t hi, lo;
+      split_pack_bf16(wv[0], wv[1], hi, lo);
+      *reinterpret_cast<uint32_t*>(Wsh + r * LW + i0) = hi;
+      *reinterpret_cast<uint32_t*>(Wsl + r * LW + i0) = lo;
+    }
+  }
+  __syncthreads();
+  for (int idx = tid; idx < C * 8; idx += kThreads) {   // coalesced 16-byte stores of W_hi, W_lo
+    const int r = idx >> 3, c0 = (idx & 7) * 8;
+    *reinterpret_cast<uint4*>(Wout + mat + r * C + c0) = *reinterpret_cast<const uint4*>(Wsh + r * LW + c0);
+    *reinterpret_cast<uint4*>(Wout + w_lo_offset + mat + r * C + c0) = *reinterpret_cast<const uint4*>(Wsl + r * LW + c0);
+  }
+  __syncthreads();   // staging read out; the area now takes A
+#pragma unroll
+  for (int t = 0; t < 8; ++t) {
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+      const int r = rbase + half * 8, i0 = t * 8 + cbase;
+      float av[2] = {0.f, 0.f};
+      if (r < si.n) {
+        const float alr = cv[0 * C + r];
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const int i = i0 + e;
+          if (i < r) av[e] = alr * Gs[(r - 1) * LM + i] * cv[3 * C + i] * kk[t][half * 2 + e];
+        }
+      }
+      *reinterpret_cast<float2*>(Af + r * LM + i0) = make_float2(av[0], av[1]);
+      if ((t >> 1) == warp)   // the warp's diagonal 16x16 block, kept compact for the forward substitution
+        *reinterpret_cast<float2*>(Ad + warp * LD16 + (r - warp * 16) * 16 + (i0 - warp * 16)) = make_float2(av[0], av[1]);
     }
   }
   __syncthreads();   // A complete; Gamma no longer needed (T takes its place)
@@ -221,7 +247,7 @@ __global__ void __launch_bounds__(kThreads) intra_mma_kernel(ChunkGeom g, const 
 #pragma unroll
       for (int m4 = 0; m4 < 16; m4 += 4) {
         if (m4 < r) {
-          const float4 v4 = *reinterpret_cast<const float4*>(Af + (b0 + r) * LM + b0 + m4);
+          const float4 v4 = *reinterpret_cast<const float4*>(Ad + (tid >> 4) * LD16 + r * 16 + m4);
           arow[m4] = v4.x; arow[m4 + 1] = v4.y; arow[m4 + 2] = v4.z; arow[m4 + 3] = v4.w;
         }
       }
