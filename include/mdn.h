@@ -120,6 +120,21 @@ mdn_status mdn_chunk_fwd_host(const mdn_params* p,
                               void* arena /* device */, size_t arena_bytes, void* cuda_stream);
 
 /*
+ * Recurrent decode step (Section 3.3: the recurrent form, Eq. 5-6, is what autoregressive decoding
+ * uses): one new token per sequence, carried state updated IN PLACE.
+ *     v~ = v - alpha S^T k;   M <- mu M - eta k v~^T;   S <- alpha S - beta M;   o = scale S^T q
+ * p->T must be 1 and p->num_seqs 0 (one token per batch row); q, k: [B,1,H,dk]; v, o: [B,1,H,dv];
+ * beta, log_alpha, log_mu, eta (NULL = 1): [B,1,H] float32; S, M: [B,H,dk,dv] float32, read and
+ * written.  No workspace.  Feeding the final states of mdn_chunk_fwd (prefill) into this call
+ * continues the same recurrence.  Asynchronous on `cuda_stream`.
+ */
+mdn_status mdn_decode_step(const mdn_params* p,
+                           const void* q, const void* k, const void* v,
+                           const float* beta, const float* log_alpha, const float* log_mu,
+                           const float* eta,
+                           float* S, float* M, void* o, void* cuda_stream);
+
+/*
  * The forward for callers that cannot allocate device memory (the paper has no counterpart: this
  * is a packaging variant of mdn_chunk_fwd, same kernels, same result).
  *

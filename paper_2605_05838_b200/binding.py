@@ -70,6 +70,8 @@ def lib() -> ctypes.CDLL:
         L.mdn_chunk_fwd_host.argtypes = [P] + [vp] * 13 + [vp, ctypes.c_size_t, vp]
         L.mdn_chunk_fwd_static_scratch.restype = ctypes.c_int
         L.mdn_chunk_fwd_static_scratch.argtypes = [P] + [vp] * 13 + [vp]
+        L.mdn_decode_step.restype = ctypes.c_int
+        L.mdn_decode_step.argtypes = [P] + [vp] * 10 + [vp]
         L.mdn_workspace_layout.restype = ctypes.c_int
         L.mdn_workspace_layout.argtypes = [P, ctypes.POINTER(MdnWsLayout)]
         L.mdn_coeff_scan.restype = ctypes.c_int
@@ -216,6 +218,26 @@ def chunk_fwd(q, k, v, beta, log_alpha, log_mu, eta=None, *, initial_S=None, ini
     if st != 0:
         raise MdnError(st, "mdn_chunk_fwd")
     return o, Sf, Mf
+
+
+def decode_step(q, k, v, beta, log_alpha, log_mu, eta, S, M, *, scale: Optional[float] = None,
+                o_dtype: Optional[torch.dtype] = None, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """mdn_decode_step: one token per sequence (q, k: [B,1,H,dk]; v: [B,1,H,dv]; gates [B,1,H]); the fp32
+    states S, M [B,H,dk,dv] are updated in place.  Returns o [B,1,H,dv]."""
+    _check_inputs(q, k, v, (("beta", beta), ("log_alpha", log_alpha), ("log_mu", log_mu), ("eta", eta)), "cuda")
+    B, T, H, dk = q.shape
+    dv = v.shape[-1]
+    if T != 1:
+        raise ValueError("decode_step takes exactly one token per sequence")
+    _check_state("S", S, (B, H, dk, dv), "cuda")
+    _check_state("M", M, (B, H, dk, dv), "cuda")
+    p = make_params(q, v, scale=scale, o_dtype=o_dtype, path="auto")
+    o = out if out is not None else torch.empty((B, 1, H, dv), dtype=o_dtype or q.dtype, device=q.device)
+    st = lib().mdn_decode_step(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(beta), _ptr(log_alpha), _ptr(log_mu),
+                               _ptr(eta), _ptr(S), _ptr(M), _ptr(o), _stream())
+    if st != 0:
+        raise MdnError(st, "mdn_decode_step")
+    return o
 
 
 STATIC_SCRATCH_BYTES = 32 << 20

@@ -169,6 +169,23 @@ mdn_status mdn_chunk_fwd(const mdn_params* p, const void* q, const void* k, cons
   return MDN_OK;
 }
 
+mdn_status mdn_decode_step(const mdn_params* p, const void* q, const void* k, const void* v, const float* beta,
+                           const float* log_alpha, const float* log_mu, const float* eta, float* S, float* M,
+                           void* o, void* cuda_stream) {
+  t_last_launches = 0;
+  mdn_status st = check_params(p);
+  if (st != MDN_OK) return st;
+  if (p->T != 1 || p->num_seqs != 0) return MDN_ERR_INVALID_ARG;
+  if (!q || !k || !v || !beta || !log_alpha || !log_mu || !S || !M || !o) return MDN_ERR_INVALID_ARG;
+  if (!aligned(q, 16) || !aligned(k, 16) || !aligned(v, 16) || !aligned(o, 16) || !aligned(S, 16) || !aligned(M, 16))
+    return MDN_ERR_INVALID_ARG;
+  const cudaError_t e = launch_decode_step(*p, q, k, v, beta, log_alpha, log_mu, eta, S, M, o,
+                                           static_cast<cudaStream_t>(cuda_stream));
+  if (e != cudaSuccess) { t_last_cuda_error = (int)e; return MDN_ERR_CUDA; }
+  t_last_launches = 1;
+  return MDN_OK;
+}
+
 mdn_status mdn_set_stage_events(void* const* events, int32_t n) {
   if (events == nullptr) { t_stage_events_on = false; return MDN_OK; }
   if (n < MDN_NUM_STAGE_EVENTS) return MDN_ERR_INVALID_ARG;

@@ -131,4 +131,10 @@ cudaError_t launch_chain_tensor(const Plan& pl, const void* q, const void* k, co
                                 const float* S0, const float* M0, void* o, float* Sf, float* Mf,
                                 int* launches);
 
+
+// Recurrent decode step (one token per sequence, state updated in place).
+cudaError_t launch_decode_step(const mdn_params& p, const void* q, const void* k, const void* v, const float* beta,
+                               const float* log_alpha, const float* log_mu, const float* eta, float* S, float* M,
+                               void* o, cudaStream_t st);
+
 }  // namespace mdn
