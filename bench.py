@@ -342,6 +342,55 @@ def run_ours(args, w):
         dist.destroy_process_group()
 
 
+def run_decode(args):
+    """Secondary benchmark (not the headline): mdn_decode_step, one token for each of `--decode-batch`
+    sequences, H=16, dk=dv=128, bf16 tokens, fp32 states updated in place.  HBM-bound: every step reads
+    and writes both dk x dv fp32 state matrices of every (sequence, head)."""
+    import torch
+    import paper_2605_05838_b200 as mdn
+    mdn.lib()
+    torch.cuda.set_device(0)
+    B, H, d = args.decode_batch, 16, 128
+    g = torch.Generator(device="cuda").manual_seed(0)
+    mk = lambda *shape: torch.randn(*shape, device="cuda", generator=g)
+    q = torch.nn.functional.normalize(mk(B, 1, H, d), dim=-1).to(torch.bfloat16)
+    k = torch.nn.functional.normalize(mk(B, 1, H, d), dim=-1).to(torch.bfloat16)
+    v = mk(B, 1, H, d).to(torch.bfloat16)
+    beta = torch.full((B, 1, H), 0.03, device="cuda"); la = torch.full((B, 1, H), -0.08, device="cuda")
+    lm = torch.full((B, 1, H), -0.03, device="cuda"); eta = torch.ones((B, 1, H), device="cuda")
+    # several state sets so that consecutive steps do not find their state in the 126 MB L2
+    n_sets = max(2, int(2 * L2_BYTES // (2 * B * H * d * d * 4)) + 1)
+    states = [(0.02 * mk(B, H, d, d), 0.02 * mk(B, H, d, d)) for _ in range(n_sets)]
+    o = torch.empty((B, 1, H, d), dtype=torch.bfloat16, device="cuda")
+
+    def step(i):
+        S, M = states[i % n_sets]
+        mdn.decode_step(q, k, v, beta, la, lm, eta, S, M, out=o)
+
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(args.steps):
+        step(i)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / args.steps
+    peaks = load_peaks()
+    abytes = float(B * H * (4 * d * d * 4 + 3 * d * 2 + d * 2 + 16))
+    print(json.dumps({
+        "metric": "MDN decode step tokens/s", "value": B / (ms * 1e-3), "unit": "tokens/s", "n_gpus": 1,
+        "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": "decode: B=%d,H=16,dk=dv=128, one token per sequence, fp32 states in place" % B,
+                   "l2": "%d rotating state sets (%.0f MB) exceed the 126 MB L2" % (n_sets, n_sets * 2 * B * H * d * d * 4 / 1e6)},
+        "gpu_launches": args.steps,
+        "roofline": {"bound": "hbm", "kernel": "decode_step", "achieved": abytes / (ms * 1e-3) / 1e9,
+                     "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": abytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                     "traffic": None, "peak_source": peaks["source"], "algorithmic_bytes": abytes}}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -353,7 +402,12 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg (profiling runs)")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    ap.add_argument("--decode", action="store_true", help="secondary benchmark: the recurrent decode step")
+    ap.add_argument("--decode-batch", type=int, default=128)
     args = ap.parse_args()
+    if args.decode:
+        run_decode(args)
+        return
     w = wl.CONFIGS[args.config]
     if args.impl == "reference":
         run_reference(args, w)

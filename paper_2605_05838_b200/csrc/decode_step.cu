@@ -39,9 +39,11 @@ __global__ void __launch_bounds__(kThreads) decode_step_kernel(int H, const TIn*
   const float be = beta[chain], et = eta ? eta[chain] : 1.f;
   float* Sp = S + (size_t)chain * DK * DV + (size_t)(dg * RPT) * DV + j;
   float* Mp = M + (size_t)chain * DK * DV + (size_t)(dg * RPT) * DV + j;
-  float sreg[RPT];
-#pragma unroll
+  float sreg[RPT], mreg[RPT];   // both loads are issued up front: the prediction needs S only, but M's
+#pragma unroll                  // latency then hides behind it
   for (int i = 0; i < RPT; ++i) sreg[i] = Sp[(size_t)i * DV];
+#pragma unroll
+  for (int i = 0; i < RPT; ++i) mreg[i] = Mp[(size_t)i * DV];
   __syncthreads();
   float part = 0.f;
 #pragma unroll
@@ -55,7 +57,7 @@ __global__ void __launch_bounds__(kThreads) decode_step_kernel(int H, const TIn*
   float opart = 0.f;
 #pragma unroll
   for (int i = 0; i < RPT; ++i) {
-    const float m_new = mu * Mp[(size_t)i * DV] - et * ks[dg * RPT + i] * vt;
+    const float m_new = mu * mreg[i] - et * ks[dg * RPT + i] * vt;
     const float s_new = alpha * sreg[i] - be * m_new;
     Mp[(size_t)i * DV] = m_new;
     Sp[(size_t)i * DV] = s_new;
