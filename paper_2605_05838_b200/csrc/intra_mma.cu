@@ -134,7 +134,8 @@ __global__ void __launch_bounds__(kThreads) intra_mma_kernel(ChunkGeom g, const 
   if (tid < C) {
     const int i = tid;
     float m = 1.f, gam = 0.f;
-    for (int r4 = i & ~3; r4 < C; r4 += 4) {
+    int r4 = i & ~3;
+    {   // first group of four: rows below i are skipped
       const float4 al = *reinterpret_cast<const float4*>(cv + 0 * C + r4);
       const float4 be = *reinterpret_cast<const float4*>(cv + 1 * C + r4);
       const float4 mu = *reinterpret_cast<const float4*>(cv + 2 * C + r4);
@@ -148,6 +149,16 @@ __global__ void __launch_bounds__(kThreads) intra_mma_kernel(ChunkGeom g, const 
           Gs[r * LM + i] = gam;
         }
       }
+    }
+    for (r4 += 4; r4 < C; r4 += 4) {
+      const float4 al = *reinterpret_cast<const float4*>(cv + 0 * C + r4);
+      const float4 be = *reinterpret_cast<const float4*>(cv + 1 * C + r4);
+      const float4 mu = *reinterpret_cast<const float4*>(cv + 2 * C + r4);
+      float* grow = Gs + r4 * LM + i;
+      m *= mu.x; gam = fmaf(be.x, m, al.x * gam); grow[0] = gam;
+      m *= mu.y; gam = fmaf(be.y, m, al.y * gam); grow[LM] = gam;
+      m *= mu.z; gam = fmaf(be.z, m, al.z * gam); grow[2 * LM] = gam;
+      m *= mu.w; gam = fmaf(be.w, m, al.w * gam); grow[3 * LM] = gam;
     }
   }
 
@@ -184,8 +195,10 @@ __global__ void __launch_bounds__(kThreads) intra_mma_kernel(ChunkGeom g, const 
   }
   __syncthreads();   // Gamma complete; every warp is done reading the K and Q tiles
 
-  // ---- W, then A, from the accumulator fragments (rows fg and fg + 8 of the warp's 16, column pairs).
-  // Tokens past the end of a short chunk (rows >= n hold another sequence's data) are masked here.
+  // ---- W and A from the accumulator fragments (rows fg and fg + 8 of the warp's 16, column pairs), one pass:
+  // W goes to the bf16 staging, A stays in the kk registers until the staging has been written out.
+  // Tiles left of the warp's diagonal block need no mask, tiles right of it are zero; tokens past the end of a
+  // short chunk (rows >= n hold another sequence's data) are masked.
   const size_t mat = ((size_t)slot * g.H + h) * C * C;
   const int rbase = warp * 16 + fg, cbase = ft * 2;
 #pragma unroll
@@ -193,16 +206,28 @@ __global__ void __launch_bounds__(kThreads) intra_mma_kernel(ChunkGeom g, const 
 #pragma unroll
     for (int half = 0; half < 2; ++half) {
       const int r = rbase + half * 8, i0 = t * 8 + cbase;
-      float wv[2] = {0.f, 0.f};
-      if (r < si.n) {
-#pragma unroll
-        for (int e = 0; e < 2; ++e) {
-          const int i = i0 + e;
-          if (i <= r) wv[e] = scale * Gs[r * LM + i] * cv[3 * C + i] * qk[t][half * 2 + e];
+      float wv0 = 0.f, wv1 = 0.f, av0 = 0.f, av1 = 0.f;
+      if ((t >> 1) <= warp && r < si.n) {
+        const float2 gw = *reinterpret_cast<const float2*>(Gs + r * LM + i0);
+        const float2 et = *reinterpret_cast<const float2*>(cv + 3 * C + i0);
+        const float alr = cv[0 * C + r];
+        float2 ga = make_float2(0.f, 0.f);
+        if (r > 0) ga = *reinterpret_cast<const float2*>(Gs + (r - 1) * LM + i0);
+        wv0 = scale * gw.x * et.x * qk[t][half * 2];
+        wv1 = scale * gw.y * et.y * qk[t][half * 2 + 1];
+        av0 = alr * ga.x * et.x * kk[t][half * 2];
+        av1 = alr * ga.y * et.y * kk[t][half * 2 + 1];
+        if ((t >> 1) == warp) {   // diagonal block: W keeps i <= r, A keeps i < r
+          if (i0 > r) { wv0 = 0.f; }
+          if (i0 + 1 > r) { wv1 = 0.f; }
+          if (i0 >= r) { av0 = 0.f; }
+          if (i0 + 1 >= r) { av1 = 0.f; }
         }
       }
+      kk[t][half * 2] = av0;
+      kk[t][half * 2 + 1] = av1;
       uint32_t hi, lo;
-      split_pack_bf16(wv[0], wv[1], hi, lo);
+      split_pack_bf16(wv0, wv1, hi, lo);
       *reinterpret_cast<uint32_t*>(Wsh + r * LW + i0) = hi;
       *reinterpret_cast<uint32_t*>(Wsl + r * LW + i0) = lo;
     }
@@ -219,18 +244,10 @@ __global__ void __launch_bounds__(kThreads) intra_mma_kernel(ChunkGeom g, const 
 #pragma unroll
     for (int half = 0; half < 2; ++half) {
       const int r = rbase + half * 8, i0 = t * 8 + cbase;
-      float av[2] = {0.f, 0.f};
-      if (r < si.n) {
-        const float alr = cv[0 * C + r];
-#pragma unroll
-        for (int e = 0; e < 2; ++e) {
-          const int i = i0 + e;
-          if (i < r) av[e] = alr * Gs[(r - 1) * LM + i] * cv[3 * C + i] * kk[t][half * 2 + e];
-        }
-      }
-      *reinterpret_cast<float2*>(Af + r * LM + i0) = make_float2(av[0], av[1]);
+      const float2 av = make_float2(kk[t][half * 2], kk[t][half * 2 + 1]);
+      *reinterpret_cast<float2*>(Af + r * LM + i0) = av;
       if ((t >> 1) == warp)   // the warp's diagonal 16x16 block, kept compact for the forward substitution
-        *reinterpret_cast<float2*>(Ad + warp * LD16 + (r - warp * 16) * 16 + (i0 - warp * 16)) = make_float2(av[0], av[1]);
+        *reinterpret_cast<float2*>(Ad + warp * LD16 + (r - warp * 16) * 16 + (i0 - warp * 16)) = av;
     }
   }
   __syncthreads();   // A complete; Gamma no longer needed (T takes its place)
