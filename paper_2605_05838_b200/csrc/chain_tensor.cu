@@ -539,8 +539,8 @@ bool tensor_path_supported(const mdn_params& p) {
   return p.io_dtype == MDN_BF16 && p.dk == kD && p.dv == kD && p.chunk == C;
 }
 
-cudaError_t launch_intra_tensor(const Plan& pl, const void* q, const void* k, int* launches) {
-  return launch_intra_mma(pl, q, k, launches);
+cudaError_t launch_intra_tensor(const Plan& pl, const void* q, const void* k, const GateArgs& gates, int* launches) {
+  return launch_intra_mma(pl, q, k, gates, launches);
 }
 
 cudaError_t launch_chain_tensor(const Plan& pl, const void* q, const void* k, const void* v, const float* S0,

@@ -12,6 +12,7 @@
 // No logarithm of beta, no division: beta = 0 and mu = 0 give exact zeros.
 // Each recurrence is an affine scan evaluated with warp shuffles: one warp per
 // (chunk, head), two consecutive positions per lane.
+#include "coeff_scan.cuh"
 #include "mdn_common.cuh"
 
 namespace mdn {
@@ -86,35 +87,6 @@ cudaError_t launch_chunk_map(const Plan& pl, int* launches) {
 }
 
 // ------------------------------------------------------------------------------------ a1
-// Affine map x -> a*x + c; compose(f_later, f_earlier).
-struct Affine { float a, c; };
-__device__ __forceinline__ Affine compose(Affine later, Affine earlier) {
-  return Affine{later.a * earlier.a, fmaf(later.a, earlier.c, later.c)};
-}
-
-// Inclusive scan over lanes in increasing order: result(l) = f_l o ... o f_0.
-__device__ __forceinline__ Affine warp_scan_up(Affine f, int lane) {
-#pragma unroll
-  for (int off = 1; off < 32; off <<= 1) {
-    Affine o;
-    o.a = __shfl_up_sync(0xffffffffu, f.a, off);
-    o.c = __shfl_up_sync(0xffffffffu, f.c, off);
-    if (lane >= off) f = compose(f, o);
-  }
-  return f;
-}
-// Inclusive scan in decreasing order: result(l) = f_l o f_{l+1} o ... o f_31.
-__device__ __forceinline__ Affine warp_scan_down(Affine f, int lane) {
-#pragma unroll
-  for (int off = 1; off < 32; off <<= 1) {
-    Affine o;
-    o.a = __shfl_down_sync(0xffffffffu, f.a, off);
-    o.c = __shfl_down_sync(0xffffffffu, f.c, off);
-    if (lane + off < 32) f = compose(f, o);
-  }
-  return f;
-}
-
 constexpr int kScanWarps = 8;
 
 // grid = chunk slots; block = 8 warps.  The [n x H] block of each gate is one contiguous
@@ -149,7 +121,7 @@ __global__ void __launch_bounds__(kScanWarps * 32) coeff_scan_kernel(ChunkGeom g
   __syncthreads();
 
   const int warp = tid >> 5, lane = tid & 31;
-  const int r0 = 2 * lane, r1 = r0 + 1;
+  const int r0 = 2 * lane;
   for (int h = warp; h < H; h += kScanWarps) {
     // exact no-ops past the end of a short chunk: alpha = mu = 1, beta = eta = 0
     float al[2], mu[2], be[2], et[2];
@@ -162,49 +134,21 @@ __global__ void __launch_bounds__(kScanWarps * 32) coeff_scan_kernel(ChunkGeom g
       be[e] = ok ? sm[2 * C * H + r * H + h] : 0.0f;
       et[e] = ok ? sm[3 * C * H + r * H + h] : 0.0f;
     }
-    // forward products abar, mubar
-    Affine pa = warp_scan_up(Affine{al[0] * al[1], 0.f}, lane);
-    Affine pm = warp_scan_up(Affine{mu[0] * mu[1], 0.f}, lane);
-    float ea = __shfl_up_sync(0xffffffffu, pa.a, 1), em = __shfl_up_sync(0xffffffffu, pm.a, 1);
-    if (lane == 0) { ea = 1.f; em = 1.f; }
-    const float abar0 = ea * al[0], abar1 = abar0 * al[1];
-    const float mbar0 = em * mu[0], mbar1 = mbar0 * mu[1];
-    // b_r = alpha_r b_{r-1} + beta_r mubar_r
-    const Affine f0{al[0], be[0] * mbar0}, f1{al[1], be[1] * mbar1};
-    Affine fb = warp_scan_up(compose(f1, f0), lane);
-    float bprev = __shfl_up_sync(0xffffffffu, fb.c, 1);
-    if (lane == 0) bprev = 0.f;
-    const float b0 = fmaf(al[0], bprev, f0.c), b1 = fmaf(al[1], b0, f1.c);
-    // backward: A_i = prod_{l>i} alpha_l, m_i = prod_{l>i} mu_l
-    Affine sa = warp_scan_down(Affine{al[0] * al[1], 0.f}, lane);
-    Affine smu = warp_scan_down(Affine{mu[0] * mu[1], 0.f}, lane);
-    float xa = __shfl_down_sync(0xffffffffu, sa.a, 1), xm = __shfl_down_sync(0xffffffffu, smu.a, 1);
-    if (lane == 31) { xa = 1.f; xm = 1.f; }
-    const float A1 = xa, A0 = xa * al[1];
-    const float m1 = xm, m0 = xm * mu[1];
-    // g_i = A_i beta_i + mu_{i+1} g_{i+1}
-    float mu_next = __shfl_down_sync(0xffffffffu, mu[0], 1);
-    if (lane == 31) mu_next = 0.f;
-    const Affine h1{mu_next, A1 * be[1]}, h0{mu[1], A0 * be[0]};
-    Affine fg = warp_scan_down(compose(h0, h1), lane);
-    float gnext = __shfl_down_sync(0xffffffffu, fg.c, 1);
-    if (lane == 31) gnext = 0.f;
-    const float g1 = fmaf(mu_next, gnext, h1.c), g0 = fmaf(mu[1], g1, h0.c);
-
+    const HeadCoefs hc = scan_head(al, mu, be, et, lane);
     float* out = coef + ((size_t)slot * H + h) * MDN_NUM_COEF * C;
     auto put = [&](int which, float x0, float x1) {
       reinterpret_cast<float2*>(out + which * C)[lane] = make_float2(x0, x1);
     };
-    put(kAbar, abar0, abar1);
-    put(kB, b0, b1);
-    put(kAlphaBPrev, al[0] * bprev, al[1] * b0);
-    put(kGS, g0 * et[0], g1 * et[1]);
-    put(kGM, m0 * et[0], m1 * et[1]);
+    put(kAbar, hc.abar[0], hc.abar[1]);
+    put(kB, hc.b[0], hc.b[1]);
+    put(kAlphaBPrev, hc.ab_prev[0], hc.ab_prev[1]);
+    put(kGS, hc.gs[0], hc.gs[1]);
+    put(kGM, hc.gm[0], hc.gm[1]);
     put(kAlpha, al[0], al[1]);
     put(kBeta, be[0], be[1]);
     put(kMu, mu[0], mu[1]);
     put(kEta, et[0], et[1]);
-    put(kMubar, mbar0, mbar1);
+    put(kMubar, hc.mubar[0], hc.mubar[1]);
   }
   grid_launch_dependents();
 }

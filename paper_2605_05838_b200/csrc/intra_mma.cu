@@ -13,6 +13,7 @@
 // once and writing T, W: warp-level mma.sync is enough here, the big contractions are in the chain kernel.
 #include <cstring>
 
+#include "coeff_scan.cuh"
 #include "mdn_common.cuh"
 #include "tc_utils.cuh"
 
@@ -91,7 +92,7 @@ __device__ __forceinline__ void block_mma_tf32(float (&acc)[NT][4], const float*
 
 __global__ void __launch_bounds__(kThreads) intra_mma_kernel(ChunkGeom g, const __grid_constant__ CUtensorMap map_q,
                                                             const __grid_constant__ CUtensorMap map_k,
-                                                            const float* __restrict__ coef, float scale,
+                                                            float* __restrict__ coef, GateArgs gates, float scale,
                                                             __nv_bfloat16* __restrict__ Tout,
                                                             __nv_bfloat16* __restrict__ Wout, size_t w_lo_offset,
                                                             int32_t* __restrict__ status) {
@@ -126,9 +127,36 @@ __global__ void __launch_bounds__(kThreads) intra_mma_kernel(ChunkGeom g, const 
     tma_load_2d(s_base + kOffQ, &map_q, h * kD, si.tok0, bar);
     tma_load_2d(s_base + kOffQ + 8192, &map_q, h * kD + 64, si.tok0, bar);
   }
-  const float* cf = coef + ((size_t)slot * g.H + h) * MDN_NUM_COEF * C;
-  for (int idx = tid; idx < 4 * C; idx += kThreads) cv[idx] = cf[kAlpha * C + idx];
-  __syncthreads();   // coefficients in smem; barrier initialised before anyone waits on it
+  float* cf = coef + ((size_t)slot * g.H + h) * MDN_NUM_COEF * C;
+  if (gates.log_alpha == nullptr) {
+    for (int idx = tid; idx < 4 * C; idx += kThreads) cv[idx] = cf[kAlpha * C + idx];
+    __syncthreads();   // coefficients in smem; barrier initialised before anyone waits on it
+  } else {
+    // fused coefficient scan (Eq. 10): this head's gates (stride H floats), then one warp runs the scans,
+    // keeps alpha, beta, mu, eta in smem for the Gamma recurrence and writes the chain kernel's six vectors
+    if (tid < C) {
+      const bool valid = tid < si.n;
+      const size_t gi = ((size_t)si.tok0 + tid) * g.H + h;
+      cv[0 * C + tid] = valid ? expf(__ldg(gates.log_alpha + gi)) : 1.f;
+      cv[1 * C + tid] = valid ? __ldg(gates.beta + gi) : 0.f;
+      cv[2 * C + tid] = valid ? expf(__ldg(gates.log_mu + gi)) : 1.f;
+      cv[3 * C + tid] = valid ? (gates.eta ? __ldg(gates.eta + gi) : 1.f) : 0.f;
+    }
+    __syncthreads();   // gates in smem; barrier initialised before anyone waits on it
+    if (warp == 3) {   // an otherwise idle warp, concurrently with the Gamma recurrence of warps 0 and 1
+      const float2 a2 = reinterpret_cast<const float2*>(cv + 0 * C)[lane], b2 = reinterpret_cast<const float2*>(cv + 1 * C)[lane];
+      const float2 m2 = reinterpret_cast<const float2*>(cv + 2 * C)[lane], e2 = reinterpret_cast<const float2*>(cv + 3 * C)[lane];
+      const float al[2] = {a2.x, a2.y}, be[2] = {b2.x, b2.y}, mu[2] = {m2.x, m2.y}, et[2] = {e2.x, e2.y};
+      const HeadCoefs hc = scan_head(al, mu, be, et, lane);
+      auto put = [&](int which, float x0, float x1) { reinterpret_cast<float2*>(cf + which * C)[lane] = make_float2(x0, x1); };
+      put(kAbar, hc.abar[0], hc.abar[1]);
+      put(kB, hc.b[0], hc.b[1]);
+      put(kAlphaBPrev, hc.ab_prev[0], hc.ab_prev[1]);
+      put(kGS, hc.gs[0], hc.gs[1]);
+      put(kGM, hc.gm[0], hc.gm[1]);
+      put(kMubar, hc.mubar[0], hc.mubar[1]);
+    }
+  }
 
   // ---- Gamma columns (threads 0..63) while the tiles are in flight
   if (tid < C) {
@@ -335,7 +363,7 @@ __global__ void __launch_bounds__(kThreads) intra_mma_kernel(ChunkGeom g, const 
 
 }  // namespace
 
-cudaError_t launch_intra_mma(const Plan& pl, const void* q, const void* k, int* launches) {
+cudaError_t launch_intra_mma(const Plan& pl, const void* q, const void* k, const GateArgs& gates, int* launches) {
   cudaError_t e = cudaFuncSetAttribute(intra_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmem);
   if (e != cudaSuccess) return e;
   const size_t n_mats = (size_t)pl.geom.num_slots * pl.p.H;
@@ -345,7 +373,7 @@ cudaError_t launch_intra_mma(const Plan& pl, const void* q, const void* k, int* 
       !encode_tma_2d_bf16(&mk, TmaMap2D{k, row, tokens, row * 2, 64, 64, true}))
     return cudaErrorInvalidValue;
   e = launch_pdl(intra_mma_kernel, dim3((unsigned)n_mats), dim3(kThreads), kSmem, pl.stream, pl.geom, mq, mk,
-                 reinterpret_cast<const float*>(pl.ws + pl.lay.off_coef), pl.p.scale,
+                 reinterpret_cast<float*>(pl.ws + pl.lay.off_coef), gates, pl.p.scale,
                  reinterpret_cast<__nv_bfloat16*>(pl.ws + pl.lay.off_T),
                  reinterpret_cast<__nv_bfloat16*>(pl.ws + pl.lay.off_W), n_mats * C * C,
                  reinterpret_cast<int32_t*>(pl.ws + pl.lay.off_status));

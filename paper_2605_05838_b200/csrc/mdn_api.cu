@@ -83,21 +83,24 @@ static mdn_status make_plan(const mdn_params* p, const int32_t* cu, void* ws, si
   return MDN_OK;
 }
 
+// with_scan = false: only the status word and the chunk map (the tensor path runs the scan inside its
+// intra-chunk kernel).
 static mdn_status run_prep_and_scan(const Plan& pl, const float* beta, const float* log_alpha, const float* log_mu,
-                                    const float* eta, int* launches) {
+                                    const float* eta, int* launches, bool with_scan = true) {
   if (!beta || !log_alpha || !log_mu) return MDN_ERR_INVALID_ARG;
   if (!aligned(beta, 4) || !aligned(log_alpha, 4) || !aligned(log_mu, 4) || (eta && !aligned(eta, 4)))
     return MDN_ERR_INVALID_ARG;
   if (cudaMemsetAsync(pl.ws + pl.lay.off_status, 0, 4 * sizeof(int32_t), pl.stream) != cudaSuccess)
     return MDN_ERR_CUDA;
   if (launch_chunk_map(pl, launches) != cudaSuccess) return MDN_ERR_CUDA;
-  if (launch_coeff_scan(pl, beta, log_alpha, log_mu, eta, launches) != cudaSuccess) return MDN_ERR_CUDA;
+  if (with_scan && launch_coeff_scan(pl, beta, log_alpha, log_mu, eta, launches) != cudaSuccess) return MDN_ERR_CUDA;
   return MDN_OK;
 }
 
-static mdn_status run_intra(const Plan& pl, const void* q, const void* k, int* launches) {
+static mdn_status run_intra(const Plan& pl, const void* q, const void* k, int* launches,
+                            const GateArgs& gates = GateArgs{nullptr, nullptr, nullptr, nullptr}) {
   if (!q || !k || !aligned(q, 16) || !aligned(k, 16)) return MDN_ERR_INVALID_ARG;
-  cudaError_t e = pl.p.path == MDN_PATH_TENSOR ? launch_intra_tensor(pl, q, k, launches)
+  cudaError_t e = pl.p.path == MDN_PATH_TENSOR ? launch_intra_tensor(pl, q, k, gates, launches)
                                                : launch_intra_simt(pl, q, k, launches);
   if (e != cudaSuccess) t_last_cuda_error = (int)e;
   return e == cudaSuccess ? MDN_OK : MDN_ERR_CUDA;
@@ -155,10 +158,14 @@ mdn_status mdn_chunk_fwd(const mdn_params* p, const void* q, const void* k, cons
       (final_S && !aligned(final_S, 16)) || (final_M && !aligned(final_M, 16)))
     return MDN_ERR_INVALID_ARG;
   if (!mark_stage(0, pl.stream)) return MDN_ERR_CUDA;
-  st = run_prep_and_scan(pl, beta, log_alpha, log_mu, eta, &t_last_launches);
+  // tensor path: the intra-chunk kernel runs the coefficient scan itself (one kernel and one round trip of
+  // the coefficient vectors less); SIMT path: stand-alone scan kernel
+  const bool fused_scan = pl.p.path == MDN_PATH_TENSOR;
+  st = run_prep_and_scan(pl, beta, log_alpha, log_mu, eta, &t_last_launches, !fused_scan);
   if (st != MDN_OK) return st;
   if (!mark_stage(1, pl.stream)) return MDN_ERR_CUDA;
-  st = run_intra(pl, q, k, &t_last_launches);
+  st = fused_scan ? run_intra(pl, q, k, &t_last_launches, GateArgs{beta, log_alpha, log_mu, eta})
+                  : run_intra(pl, q, k, &t_last_launches);
   if (st != MDN_OK) return st;
   if (!mark_stage(2, pl.stream)) return MDN_ERR_CUDA;
   cudaError_t e = pl.p.path == MDN_PATH_TENSOR

@@ -103,6 +103,10 @@ template <typename T> __device__ __forceinline__ T from_f32(float x);
 template <> __device__ __forceinline__ float from_f32<float>(float x) { return x; }
 template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float x) { return __float2bfloat16_rn(x); }
 
+// Raw gate pointers ([B,T,H] fp32) for kernels that run the coefficient scan themselves; all NULL = the
+// coefficients are already in the workspace.
+struct GateArgs { const float* beta; const float* log_alpha; const float* log_mu; const float* eta; };
+
 // Host-side view of one call, filled by the API layer.
 struct Plan {
   mdn_params p;
@@ -125,8 +129,8 @@ cudaError_t launch_chain_simt(const Plan& pl, const void* q, const void* k, cons
 
 // Tensor-core (tcgen05) path: bf16 q/k/v, dk = dv = 128.
 bool tensor_path_supported(const mdn_params& p);
-cudaError_t launch_intra_tensor(const Plan& pl, const void* q, const void* k, int* launches);
-cudaError_t launch_intra_mma(const Plan& pl, const void* q, const void* k, int* launches);
+cudaError_t launch_intra_tensor(const Plan& pl, const void* q, const void* k, const GateArgs& gates, int* launches);
+cudaError_t launch_intra_mma(const Plan& pl, const void* q, const void* k, const GateArgs& gates, int* launches);
 cudaError_t launch_chain_tensor(const Plan& pl, const void* q, const void* k, const void* v,
                                 const float* S0, const float* M0, void* o, float* Sf, float* Mf,
                                 int* launches);
