@@ -69,7 +69,24 @@ typedef struct {
   int32_t path;            /* mdn_path                                                       */
   float scale;             /* multiplies q; dk^-0.5 is the appendix listing's default,       */
                            /* 1.0 gives the bare o_t = S_t^T q_t                             */
+  int32_t segments;        /* tensor path, fixed-length input: split every sequence into this */
+                           /* many segments whose chunk chains run in PARALLEL (see below);   */
+                           /* 0 = choose automatically, 1 = off, 3..32 = forced               */
 } mdn_params;
+
+/*
+ * Parallel inter-chunk scan for long sequences with few (sequence, head) chains (Section 3.2 views the
+ * recurrence as a linear dynamical system on the stacked state [S; M]).  With V = 0 a run of chunks
+ * maps [S; M] linearly, so for a segment g of a sequence
+ *     [S; M]_end = Phi_g [S; M]_start + Psi_g ,
+ * where Psi_g is the segment run from a zero state and the two halves of Phi_g (2dk x 2dk) are the
+ * segment run with V = 0 from the states (I, 0) and (0, I).  mdn_chunk_fwd then runs
+ *   1. in parallel: segment 0 as usual, and for every middle segment the three runs giving Psi, Phi;
+ *   2. a short serial combine over segments (fp32) giving every segment's true start state;
+ *   3. in parallel: segments 1.. as usual from those start states (outputs and final state).
+ * The result is the same recurrence; only rounding differs.  Chosen automatically when the call has
+ * too few chains to fill the GPU and the sequences are long (e.g. B=1, H=16, T=65536).
+ */
 
 /* Bytes of device workspace mdn_chunk_fwd needs for these parameters (0 on invalid
  * parameters).  Holds the chunk map, the per-chunk coefficient vectors and the
@@ -196,6 +213,9 @@ typedef struct {
   uint64_t off_T;           /* [num_slots][H][64][64]                                                    */
   uint64_t off_W;           /* [num_slots][H][64][64]  (tensor path: bf16 hi part; lo part follows)      */
   uint64_t total_bytes;
+  uint64_t off_seg;         /* segment states, Psi and Phi matrices of the parallel scan (fp32)          */
+  int32_t segments;         /* segments per sequence the call will use (1 = plain serial chain)          */
+  int32_t reserved;
 } mdn_ws_layout;
 
 mdn_status mdn_workspace_layout(const mdn_params* p, mdn_ws_layout* out /* host */);

@@ -30,14 +30,15 @@ class MdnParams(ctypes.Structure):
     _fields_ = [("B", ctypes.c_int32), ("T", ctypes.c_int32), ("H", ctypes.c_int32),
                 ("dk", ctypes.c_int32), ("dv", ctypes.c_int32), ("chunk", ctypes.c_int32),
                 ("num_seqs", ctypes.c_int32), ("io_dtype", ctypes.c_int32), ("o_dtype", ctypes.c_int32),
-                ("path", ctypes.c_int32), ("scale", ctypes.c_float)]
+                ("path", ctypes.c_int32), ("scale", ctypes.c_float), ("segments", ctypes.c_int32)]
 
 
 class MdnWsLayout(ctypes.Structure):
     _fields_ = [("num_slots", ctypes.c_int32), ("mat_dtype", ctypes.c_int32),
                 ("off_status", ctypes.c_uint64), ("off_chunk_off", ctypes.c_uint64),
                 ("off_slot_map", ctypes.c_uint64), ("off_coef", ctypes.c_uint64),
-                ("off_T", ctypes.c_uint64), ("off_W", ctypes.c_uint64), ("total_bytes", ctypes.c_uint64)]
+                ("off_T", ctypes.c_uint64), ("off_W", ctypes.c_uint64), ("total_bytes", ctypes.c_uint64),
+                ("off_seg", ctypes.c_uint64), ("segments", ctypes.c_int32), ("reserved", ctypes.c_int32)]
 
 
 class MdnError(RuntimeError):
@@ -139,12 +140,12 @@ def _stream() -> ctypes.c_void_p:
 
 
 def make_params(q: torch.Tensor, v: torch.Tensor, *, num_seqs: int = 0, scale: Optional[float] = None,
-                o_dtype: Optional[torch.dtype] = None, path: str = "auto") -> MdnParams:
+                o_dtype: Optional[torch.dtype] = None, path: str = "auto", segments: int = 0) -> MdnParams:
     B, T, H, dk = q.shape
     dv = v.shape[-1]
     return MdnParams(B, T, H, dk, dv, CHUNK, int(num_seqs), _dtype_code(q.dtype),
                      _dtype_code(o_dtype or q.dtype), _PATHS[path],
-                     float(dk) ** -0.5 if scale is None else float(scale))
+                     float(dk) ** -0.5 if scale is None else float(scale), int(segments))
 
 
 def workspace_bytes(p: MdnParams) -> int:
@@ -187,9 +188,10 @@ def _check_state(name, t, shape, device_type):
 def chunk_fwd(q, k, v, beta, log_alpha, log_mu, eta=None, *, initial_S=None, initial_M=None,
               cu_seqlens=None, scale: Optional[float] = None, o_dtype: Optional[torch.dtype] = None,
               path: str = "auto", output_final_state: bool = True, workspace: Optional[torch.Tensor] = None,
-              out: Optional[torch.Tensor] = None
+              out: Optional[torch.Tensor] = None, segments: int = 0
               ) -> Tuple[torch.Tensor, Optional[torch.Tensor], Optional[torch.Tensor]]:
-    """mdn_chunk_fwd on CUDA tensors (current stream).  Returns (o, final_S, final_M)."""
+    """mdn_chunk_fwd on CUDA tensors (current stream).  Returns (o, final_S, final_M).
+    segments: 0 = automatic, 1 = plain serial chain, >= 3 = force the parallel inter-chunk scan."""
     _check_inputs(q, k, v, (("beta", beta), ("log_alpha", log_alpha), ("log_mu", log_mu), ("eta", eta)), "cuda")
     B, T, H, dk = q.shape
     dv = v.shape[-1]
@@ -198,7 +200,7 @@ def chunk_fwd(q, k, v, beta, log_alpha, log_mu, eta=None, *, initial_S=None, ini
         if cu_seqlens.device.type != "cuda" or cu_seqlens.dtype != torch.int32 or not cu_seqlens.is_contiguous():
             raise ValueError("cu_seqlens must be a contiguous int32 cuda tensor")
         N = cu_seqlens.numel() - 1
-    p = make_params(q, v, num_seqs=N, scale=scale, o_dtype=o_dtype, path=path)
+    p = make_params(q, v, num_seqs=N, scale=scale, o_dtype=o_dtype, path=path, segments=segments)
     nst = N if N > 0 else B
     _check_state("initial_S", initial_S, (nst, H, dk, dv), "cuda")
     _check_state("initial_M", initial_M, (nst, H, dk, dv), "cuda")

@@ -48,6 +48,7 @@ constexpr uint32_t kStK = 0, kStQ = 16384, kStV = 32768, kStT = 49152, kStWh = 5
 constexpr uint32_t kCoefBytes = kChainCoefs * C * sizeof(float);
 constexpr uint32_t kStageBytes = 75776;
 constexpr uint32_t kTxBytes = 3 * 16384 + 3 * 8192 + kCoefBytes;
+constexpr uint32_t kTxQW = 16384 + 2 * 8192, kTxV = 16384;   // bytes of the Q + W_hi + W_lo tiles, of the V tile
 constexpr uint32_t kSmemBytes = kOffStage + 2 * kStageBytes + 1024;
 static_assert(kStCoef + kCoefBytes <= kStageBytes, "stage layout");
 
@@ -82,6 +83,13 @@ struct ChainArgs {
   int32_t* status;
   float scale;
   uint32_t w_lo_row_offset;   // rows between the hi and lo parts in the W tensor map
+  // parallel inter-chunk scan (seg_G = 0: off, one CTA walks all chunks of its chain)
+  int seg_G;                  // segments per sequence
+  int seg_phase;              // 1: segment 0 + the Psi / Phi runs of the middle segments; 3: segments 1.. from E
+  float* seg_E;               // [chains][G-1][2][dk*dv]  state at the END of segment g (start of g+1)
+  float* seg_Psi;             // [chains][G-2][2][dk*dv]  segment run from a zero state
+  float* seg_PhiS;            // [chains][G-2][2][dk*dv]  segment run with V = 0 from (S, M) = (I, 0)
+  float* seg_PhiM;            // [chains][G-2][2][dk*dv]  ... from (0, I)
   uint32_t drop_lo;           // debug: bit 0 R, 1 V~_S/V~_M, 2 V~ (output), 3 W: leave that operand's lo part out
   long long* timeline;        // debug: CTA 0 writes clock64() at [chunk*32 + event] (NULL = off)
 };
@@ -115,11 +123,56 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int H = a.g.H;
-  const int seq = blockIdx.x / H, h = blockIdx.x % H;
-  grid_dependency_wait();   // chunk map, coefficients, T and W come from the previous kernels
-  const SeqInfo sq = seq_info(a.g, seq);
+  // ---- work item: which chain, which segment of it, which kind of run
+  int chain = blockIdx.x, seg = 0, run = 0;   // run 0: the real thing; 1: Psi; 2: Phi from (I, 0); 3: Phi from (0, I)
+  if (a.seg_G > 0) {
+    if (a.seg_phase == 1) {
+      const int items = 1 + 3 * (a.seg_G - 2);
+      chain = blockIdx.x / items;
+      const int w = blockIdx.x % items;
+      if (w > 0) { seg = 1 + (w - 1) / 3; run = 1 + (w - 1) % 3; }
+    } else {
+      chain = blockIdx.x / (a.seg_G - 1);
+      seg = 1 + blockIdx.x % (a.seg_G - 1);
+    }
+  }
+  const int seq = chain / H, h = chain % H;
+  grid_dependency_wait();   // chunk map, coefficients, T and W (and segment states) come from the previous kernels
+  SeqInfo sq = seq_info(a.g, seq);
+  if (a.seg_G > 0) {        // restrict the view to this segment's chunks
+    const int per = (sq.nchunks + a.seg_G - 1) / a.seg_G;
+    const int cb = min(sq.nchunks, seg * per), ce = min(sq.nchunks, (seg + 1) * per);
+    sq.slot0 += cb;
+    sq.tok0 += cb * C;
+    sq.len = (ce > cb) ? min(sq.len - cb * C, (ce - cb) * C) : 0;
+    sq.nchunks = ce - cb;
+  }
   const int nch = sq.nchunks;
-  const size_t st_off = ((size_t)seq * H + h) * kD * kD;
+  const size_t st_off = (size_t)chain * kD * kD;
+  // ---- where the start state comes from, where the end state goes, whether V counts, whether o is written
+  const float* S0p = a.S0 ? a.S0 + st_off : nullptr;
+  const float* M0p = a.M0 ? a.M0 + st_off : nullptr;
+  float* Sfp = a.Sf ? a.Sf + st_off : nullptr;
+  float* Mfp = a.Mf ? a.Mf + st_off : nullptr;
+  bool id_s = false, id_m = false, v_zero = false, write_o = true;
+  if (a.seg_G > 0) {
+    constexpr size_t kMat = (size_t)kD * kD;
+    auto e_ptr = [&](int gi, int which) { return a.seg_E + (((size_t)chain * (a.seg_G - 1) + gi) * 2 + which) * kMat; };
+    if (run == 0) {
+      if (seg > 0) { S0p = e_ptr(seg - 1, 0); M0p = e_ptr(seg - 1, 1); }
+      if (seg < a.seg_G - 1) {
+        Sfp = (seg == 0) ? e_ptr(0, 0) : nullptr;
+        Mfp = (seg == 0) ? e_ptr(0, 1) : nullptr;
+      }
+    } else {
+      write_o = false;
+      S0p = M0p = nullptr;
+      id_s = run == 2; id_m = run == 3; v_zero = run >= 2;
+      float* base = (run == 1 ? a.seg_Psi : run == 2 ? a.seg_PhiS : a.seg_PhiM) +
+                    (((size_t)chain * (a.seg_G - 2) + (seg - 1)) * 2) * kMat;
+      Sfp = base; Mfp = base + kMat;
+    }
+  }
 
   const uint32_t s_base = smem_u32(smem);
   const uint32_t b_full0 = smem_u32(&bars.full[0]), b_full1 = smem_u32(&bars.full[1]);
@@ -172,7 +225,9 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
           MDN_WAIT(s ? b_go1 : b_go0, (co >> 1) & 1);
           const int n = min(C, sq.len - co * C);
           const int tok0 = sq.tok0 + co * C;
-          if (n == C) {
+          if (!write_o) {
+            // Psi / Phi runs of the parallel scan produce states only
+          } else if (n == C) {
             tma_store_2d(&map_o, h * kD, tok0, st);
           } else {   // short chunk: rows >= n belong to another sequence; one bulk copy per valid row
             for (int r = 0; r < n; ++r)
@@ -187,16 +242,19 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
           const uint32_t fb = s ? b_full1 : b_full0;
           const int tok0 = sq.tok0 + c * C;
           const int mat = (sq.slot0 + c) * H + h;
-          mbar_arrive_expect_tx(fb, kTxBytes);
+          // state-only runs need neither Q nor W, and the V = 0 runs no V either
+          mbar_arrive_expect_tx(fb, kTxBytes - (write_o ? 0u : kTxQW) - (v_zero ? kTxV : 0u));
           tma_load_2d(st + kStK, &map_k, h * kD, tok0, fb);
           tma_load_2d(st + kStK + 8192, &map_k, h * kD + 64, tok0, fb);
           bulk_load(st + kStCoef, a.coef + (size_t)mat * MDN_NUM_COEF * C, kCoefBytes, fb);
-          tma_load_2d(st + kStV, &map_v, h * kD, tok0, fb);
+          if (!v_zero) tma_load_2d(st + kStV, &map_v, h * kD, tok0, fb);
           tma_load_2d(st + kStT, &map_t, 0, mat * C, fb);
-          tma_load_2d(st + kStQ, &map_q, h * kD, tok0, fb);
-          tma_load_2d(st + kStQ + 8192, &map_q, h * kD + 64, tok0, fb);
-          tma_load_2d(st + kStWh, &map_w, 0, mat * C, fb);
-          tma_load_2d(st + kStWl, &map_w, 0, mat * C + (int)a.w_lo_row_offset, fb);
+          if (write_o) {
+            tma_load_2d(st + kStQ, &map_q, h * kD, tok0, fb);
+            tma_load_2d(st + kStQ + 8192, &map_q, h * kD + 64, tok0, fb);
+            tma_load_2d(st + kStWh, &map_w, 0, mat * C, fb);
+            tma_load_2d(st + kStWl, &map_w, 0, mat * C + (int)a.w_lo_row_offset, fb);
+          }
           MDN_MARK(c, kEvTmaIssued);
           issued = c + 1;
         }
@@ -238,15 +296,17 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
           umma_ss(tmem + kColY, ((k >> 2) ? dMb1 : dMb0) + 2 * (k & 3), ((k >> 2) ? dK1 : dK0) + 2 * (k & 3), id64, k > 0);
         umma_commit(b_m1);
         // ---- MMA-1b: Z = S_b Q^T, U = M_b Q^T (U of the previous chunk must have been read)
-        MDN_WAIT(b_zu, ph ^ 1);
-        tc_fence_after_sync();
+        if (write_o) {
+          MDN_WAIT(b_zu, ph ^ 1);
+          tc_fence_after_sync();
 #pragma unroll
-        for (int k = 0; k < 8; ++k)
-          umma_ss(tmem + kColZ, ((k >> 2) ? dSb1 : dSb0) + 2 * (k & 3), ((k >> 2) ? dQ1 : dQ0) + 2 * (k & 3), id64, k > 0);
+          for (int k = 0; k < 8; ++k)
+            umma_ss(tmem + kColZ, ((k >> 2) ? dSb1 : dSb0) + 2 * (k & 3), ((k >> 2) ? dQ1 : dQ0) + 2 * (k & 3), id64, k > 0);
 #pragma unroll
-        for (int k = 0; k < 8; ++k)
-          umma_ss(tmem + kColU, ((k >> 2) ? dMb1 : dMb0) + 2 * (k & 3), ((k >> 2) ? dQ1 : dQ0) + 2 * (k & 3), id64, k > 0);
-        umma_commit(b_mq);
+          for (int k = 0; k < 8; ++k)
+            umma_ss(tmem + kColU, ((k >> 2) ? dMb1 : dMb0) + 2 * (k & 3), ((k >> 2) ? dQ1 : dQ0) + 2 * (k & 3), id64, k > 0);
+          umma_commit(b_mq);
+        }
         // ---- MMA-2: Y = (R_hi + R_lo)^T T^T
         MDN_WAIT(b_r, ph);
         tc_fence_after_sync();
@@ -268,6 +328,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
         for (int k = 0; k < n3; ++k)
           umma_ts(tmem + kColM, tmem + kColY + (k >> 2) * 32 + (k & 3) * 8, dKmn + 128 * (k & 3), id128_mn_neg, true);
         umma_commit(b_m3);
+        if (!write_o) continue;   // state-only run: no output terms
         // ---- MMA-3': U = V~^T W^T  with  V~ = hi + lo, W = hi + lo (lo*lo dropped)
         MDN_WAIT(b_v2, ph);
         tc_fence_after_sync();
@@ -319,8 +380,9 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
         if (c == 0) {
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
-            sr[j] = __float_as_uint(a.S0 ? __ldg(a.S0 + st_off + (size_t)(cs * 32 + j) * kD + d) : 0.f);
-            mr[j] = __float_as_uint(a.M0 ? __ldg(a.M0 + st_off + (size_t)(cs * 32 + j) * kD + d) : 0.f);
+            const float unit = (cs * 32 + j == d) ? 1.f : 0.f;
+            sr[j] = __float_as_uint(S0p ? __ldg(S0p + (size_t)(cs * 32 + j) * kD + d) : (id_s ? unit : 0.f));
+            mr[j] = __float_as_uint(M0p ? __ldg(M0p + (size_t)(cs * 32 + j) * kD + d) : (id_m ? unit : 0.f));
           }
         } else {
           tmem_ld32(tl + kColS + cs * 32, sr);
@@ -358,8 +420,8 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
         } else {
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
-            if (a.Sf) a.Sf[st_off + (size_t)(cs * 32 + j) * kD + d] = __uint_as_float(sr[j]);
-            if (a.Mf) a.Mf[st_off + (size_t)(cs * 32 + j) * kD + d] = __uint_as_float(mr[j]);
+            if (Sfp) Sfp[(size_t)(cs * 32 + j) * kD + d] = __uint_as_float(sr[j]);
+            if (Mfp) Mfp[(size_t)(cs * 32 + j) * kD + d] = __uint_as_float(mr[j]);
           }
         }
       }
@@ -370,7 +432,10 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
       }
       // ---------------- output of the previous chunk (under MMA-1a): o^T = oi + U, staged as a [64 x 128] tile in
       // the previous chunk's stage (all its MMAs are done and nobody reads its tiles any more)
-      if (c > 0) {
+      if (c > 0 && !write_o) {
+        // state-only run: MMA-3 of the previous chunk (waited for above) was the last reader of its stage
+        mbar_arrive(((c - 1) & 1) ? b_go1 : b_go0);
+      } else if (c > 0) {
         const int cp = c - 1;
         uint8_t* stp = smem + kOffStage + (cp & 1) * kStageBytes;
         MDN_WAIT(b_mo, cp & 1);
@@ -402,7 +467,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
         // V and the coefficients do not depend on the MMA: fetch them while MMA-1a runs
         float vv[32];
 #pragma unroll
-        for (int j = 0; j < 32; ++j) vv[j] = __bfloat162float(sV[(r0 + j) * kD + d]);
+        for (int j = 0; j < 32; ++j) vv[j] = v_zero ? 0.f : __bfloat162float(sV[(r0 + j) * kD + d]);
         MDN_WAIT(b_m1, ph);
         __syncwarp();
         tc_fence_after_sync();
@@ -440,7 +505,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
       mbar_arrive(b_r);
       MDN_MARK(c, kEvRArrive);
       // ---------------- inter-chunk output terms (under MMA-2): oi = scale (abar .* Q S - b .* Q M)
-      {
+      if (write_o) {
         MDN_WAIT(b_mq, ph);
         __syncwarp();
         tc_fence_after_sync();
@@ -507,7 +572,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
         mbar_arrive(b_v1);
         MDN_MARK(c, kEvVArrive);
         // part b (under MMA-3): V~ itself for the intra-chunk output, into Z once every warp has read Q S
-        {
+        if (write_o) {
           uint32_t vh[16], vl[16];
 #pragma unroll
           for (int j = 0; j < 32; j += 2) split_pack_bf16(__uint_as_float(vt[j]), __uint_as_float(vt[j + 1]), vh[j >> 1], vl[j >> 1]);
@@ -517,9 +582,9 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
           tmem_st16(tl + kColZ + 16 * hf, vh);
           tmem_st16(tl + kColZ + 32 + 16 * hf, vl);
           tmem_wait_st();
+          tc_fence_before_sync();
+          mbar_arrive(b_v2);
         }
-        tc_fence_before_sync();
-        mbar_arrive(b_v2);
         MDN_MARK(c, kEvV2Arrive);
       }
     }
@@ -570,22 +635,73 @@ cudaError_t launch_chain_tensor(const Plan& pl, const void* q, const void* k, co
   a.drop_lo = drop ? (uint32_t)atoi(drop) : 0u;
   const char* tl = getenv("MDN_DEBUG_TIMELINE");   // device address of an int64 buffer, [chunks][32]
   a.timeline = tl ? reinterpret_cast<long long*>(strtoull(tl, nullptr, 0)) : nullptr;
-  const unsigned grid = (unsigned)pl.geom.num_seqs * p.H;
-  cudaError_t e;
-  if (p.o_dtype == MDN_BF16) {
-    auto kern = chain_tensor_kernel<__nv_bfloat16>;
-    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
-    if (e != cudaSuccess) return e;
-    e = launch_pdl(kern, dim3(grid), dim3(kThreads), kSmemBytes, pl.stream, a, mq, mk, mv, mt, mw, mo);
-  } else {
-    auto kern = chain_tensor_kernel<float>;
-    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
-    if (e != cudaSuccess) return e;
-    e = launch_pdl(kern, dim3(grid), dim3(kThreads), kSmemBytes, pl.stream, a, mq, mk, mv, mt, mw, mo);
+  a.seg_G = 0; a.seg_phase = 0;
+  a.seg_E = a.seg_Psi = a.seg_PhiS = a.seg_PhiM = nullptr;
+  const unsigned chains = (unsigned)pl.geom.num_seqs * p.H;
+  auto launch = [&](unsigned grid) -> cudaError_t {
+    cudaError_t e;
+    if (p.o_dtype == MDN_BF16) {
+      auto kern = chain_tensor_kernel<__nv_bfloat16>;
+      e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+      if (e != cudaSuccess) return e;
+      e = launch_pdl(kern, dim3(grid), dim3(kThreads), kSmemBytes, pl.stream, a, mq, mk, mv, mt, mw, mo);
+    } else {
+      auto kern = chain_tensor_kernel<float>;
+      e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+      if (e != cudaSuccess) return e;
+      e = launch_pdl(kern, dim3(grid), dim3(kThreads), kSmemBytes, pl.stream, a, mq, mk, mv, mt, mw, mo);
+    }
+    if (e == cudaSuccess) e = cudaGetLastError();
+    if (e == cudaSuccess) ++*launches;
+    return e;
+  };
+  const int G = pl.lay.segments;
+  if (G <= 1) return launch(chains);
+
+  // ---- parallel inter-chunk scan: Psi / Phi of the middle segments, serial combine, then all segments for real
+  constexpr size_t kMat = (size_t)kD * kD;
+  float* seg = reinterpret_cast<float*>(pl.ws + pl.lay.off_seg);
+  a.seg_G = G;
+  a.seg_E = seg;
+  a.seg_Psi = a.seg_E + (size_t)chains * (G - 1) * 2 * kMat;
+  a.seg_PhiS = a.seg_Psi + (size_t)chains * (G - 2) * 2 * kMat;
+  a.seg_PhiM = a.seg_PhiS + (size_t)chains * (G - 2) * 2 * kMat;
+  a.seg_phase = 1;
+  cudaError_t e = launch(chains * (1 + 3 * (G - 2)));
+  if (e != cudaSuccess) return e;
+  e = launch_seg_combine(pl, G, a.seg_E, a.seg_Psi, a.seg_PhiS, a.seg_PhiM, launches);
+  if (e != cudaSuccess) return e;
+  a.seg_phase = 3;
+  return launch(chains * (G - 1));
+}
+
+size_t seg_scratch_bytes(const mdn_params& p, int segments) {
+  if (segments <= 1) return 0;
+  const size_t chains = (size_t)p.B * p.H, mat = (size_t)p.dk * p.dv * sizeof(float);
+  return chains * ((size_t)(segments - 1) * 2 + (size_t)(segments - 2) * 6) * mat;
+}
+
+// Segments per sequence for the parallel scan, from a wave-count model of the two chain launches (one CTA per
+// SM, every CTA walks ceil(nch / G) chunks; a middle segment costs three extra runs) plus about four chunk-times
+// per step of the serial combine.  The scan is used only where the model predicts at most 0.7 of the serial
+// chain's time and every segment keeps at least 8 chunks; otherwise 1 (off).
+int choose_segments(const mdn_params& p) {
+  if (!tensor_path_supported(p) || p.num_seqs > 0) return 1;
+  if (p.segments == 1) return 1;
+  if (p.segments >= 3) return p.segments;
+  constexpr long kSMs = 148;
+  const long nch = (p.T + C - 1) / C, chains = (long)p.B * p.H;
+  auto waves = [&](long ctas) { return (ctas + kSMs - 1) / kSMs; };
+  const long serial = waves(chains) * nch;
+  long best_cost = serial;
+  int best = 1;
+  for (int g = 3; g <= 32 && nch / g >= 8; ++g) {
+    const long per = (nch + g - 1) / g;
+    // (a state-only run takes about 0.9 of a full one: it skips the output terms, which mostly hide anyway)
+    const long cost = (waves(chains * (1 + 3 * (g - 2))) * 9 * per) / 10 + waves(chains * (g - 1)) * per + 4 * (g - 2);
+    if (cost * 10 <= serial * 7 && cost < best_cost) { best_cost = cost; best = g; }
   }
-  if (e == cudaSuccess) e = cudaGetLastError();
-  if (e == cudaSuccess) ++*launches;
-  return e;
+  return best;
 }
 
 }  // namespace mdn

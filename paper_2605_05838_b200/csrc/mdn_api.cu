@@ -37,6 +37,7 @@ static mdn_status check_params(const mdn_params* p) {
   if (p->H > 1024) return MDN_ERR_UNSUPPORTED;
   if (p->path == MDN_PATH_TENSOR && !tensor_path_supported(*p)) return MDN_ERR_UNSUPPORTED;
   if (!(p->scale == p->scale)) return MDN_ERR_INVALID_ARG;
+  if (p->segments < 0 || p->segments == 2 || p->segments > 32) return MDN_ERR_INVALID_ARG;
   return MDN_OK;
 }
 
@@ -56,6 +57,8 @@ static mdn_status make_layout(const mdn_params& p, mdn_ws_layout* lay) {
   lay->off_coef = off; off = align_up(off + (uint64_t)slots * p.H * MDN_NUM_COEF * C * sizeof(float), 256);
   lay->off_T = off; off = align_up(off + mats * (tensor ? 2 : 4), 256);
   lay->off_W = off; off = align_up(off + mats * 4, 256);   // fp32, or bf16 hi + bf16 lo
+  lay->segments = (tensor && !packed) ? choose_segments(p) : 1;
+  lay->off_seg = off; off = align_up(off + (lay->segments > 1 ? seg_scratch_bytes(p, lay->segments) : 0), 256);
   lay->total_bytes = off;
   return MDN_OK;
 }

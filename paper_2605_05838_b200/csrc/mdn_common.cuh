@@ -134,6 +134,12 @@ cudaError_t launch_intra_mma(const Plan& pl, const void* q, const void* k, const
 cudaError_t launch_chain_tensor(const Plan& pl, const void* q, const void* k, const void* v,
                                 const float* S0, const float* M0, void* o, float* Sf, float* Mf,
                                 int* launches);
+// Segment bookkeeping of the parallel inter-chunk scan: per chain (G-1) states E, (G-2) Psi and 2 (G-2) Phi
+// halves, each a pair of [dk x dv] fp32 matrices.
+size_t seg_scratch_bytes(const mdn_params& p, int segments);
+int choose_segments(const mdn_params& p);
+cudaError_t launch_seg_combine(const Plan& pl, int G, float* E, const float* Psi, const float* PhiS,
+                               const float* PhiM, int* launches);
 
 
 // Recurrent decode step (one token per sequence, state updated in place).

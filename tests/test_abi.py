@@ -37,7 +37,8 @@ def test_status_strings(mdn):
 
 
 def params(mdn, **kw):
-    base = dict(B=2, T=130, H=3, dk=64, dv=128, chunk=64, num_seqs=0, io_dtype=0, o_dtype=0, path=0, scale=0.125)
+    base = dict(B=2, T=130, H=3, dk=64, dv=128, chunk=64, num_seqs=0, io_dtype=0, o_dtype=0, path=0, scale=0.125,
+                segments=0)
     base.update(kw)
     return mdn.MdnParams(**base)
 
@@ -54,8 +55,27 @@ def test_workspace_layout_and_bounds(mdn):
     assert mdn.host_arena_bytes(p) > mdn.workspace_bytes(p)
 
 
+def test_segment_choice_for_the_parallel_inter_chunk_scan(mdn):
+    """Host-side rule only: few long chains are split, anything that already fills the GPU is not."""
+    bf = dict(dk=128, dv=128, io_dtype=1, o_dtype=1)
+    seg = lambda **kw: mdn.workspace_layout(params(mdn, **{**bf, **kw})).segments
+    assert seg(B=1, H=16, T=65536) >= 4              # 16 chains, 1024 chunks each
+    assert seg(B=8, H=16, T=4096) == 1               # 128 chains
+    assert seg(B=4, H=8, T=2048) == 1                # short
+    assert seg(B=1, H=16, T=65536, segments=1) == 1 and seg(B=1, H=16, T=65536, segments=5) == 5
+    assert seg(B=1, H=16, T=65536, path=1) == 1      # SIMT path: no scan
+    assert seg(B=1, H=16, T=65536, num_seqs=3) == 1  # packed input: no scan
+    assert seg(B=1, H=16, T=65536, io_dtype=0, o_dtype=0) == 1
+    with_scan = mdn.workspace_layout(params(mdn, **bf, B=1, H=16, T=65536))
+    without = mdn.workspace_layout(params(mdn, **bf, B=1, H=16, T=65536, segments=1))
+    G = with_scan.segments
+    assert with_scan.total_bytes - without.total_bytes >= 16 * ((G - 1) * 2 + (G - 2) * 6) * 128 * 128 * 4
+    assert with_scan.off_seg % 256 == 0
+
+
 @pytest.mark.parametrize("kw", [dict(chunk=32), dict(dk=96), dict(dv=32), dict(B=0), dict(T=0), dict(H=0),
-                                dict(io_dtype=5), dict(path=9), dict(num_seqs=3), dict(num_seqs=-1)])
+                                dict(io_dtype=5), dict(path=9), dict(num_seqs=3), dict(num_seqs=-1), dict(segments=2),
+                                dict(segments=33), dict(segments=-1)])
 def test_bad_params_rejected(mdn, kw):
     assert mdn.workspace_bytes(params(mdn, **kw)) == 0
 

@@ -31,7 +31,7 @@ def mdn():
 
 
 def tensor_ok(mdn, w):
-    p = mdn.MdnParams(w.B, w.T, w.H, w.dk, w.dv, 64, 0, 1, 1, 2, 1.0)
+    p = mdn.MdnParams(w.B, w.T, w.H, w.dk, w.dv, 64, 0, 1, 1, 2, 1.0, 0)
     return w.dtype == "bf16" and mdn.workspace_bytes(p) > 0
 
 
@@ -293,6 +293,41 @@ def test_degenerate_gates_tensor_path(mdn):
     o, S, M = run_gpu(mdn, inp4, path="tensor", o_dtype=torch.float32)
     abar = np.exp(np.cumsum(inp4["log_alpha"].astype(np.float64), axis=1))[:, -1]
     assert np.allclose(S, abar[:, :, None, None] * inp4["S0"], rtol=1e-4, atol=1e-7)    # purely decayed state, exact path
+
+
+@pytest.mark.parametrize("segments,T", [(3, 64 * 9), (4, 64 * 13 + 17), (8, 64 * 40 + 1), (5, 64 * 3 + 5), (16, 64 * 33)])
+def test_parallel_inter_chunk_scan_forced(mdn, segments, T):
+    """The segmented scan (zero-state runs, V = 0 basis runs, serial combine, real runs) against the stepwise
+    oracle, and against the plain serial chain; includes a ragged tail and more segments than chunks."""
+    import torch
+    w = wl.Workload("segscan", B=2, T=T, H=3, dk=128, dv=128, dtype="bf16", init_state_std=0.3, seed=40 + segments)
+    if not tensor_ok(mdn, w):
+        pytest.skip("tensor path not built")
+    inp = wl.make_inputs(w)
+    o_ref, S_ref, M_ref = run_oracle(inp)
+    o1, S1, M1 = run_gpu(mdn, inp, path="tensor", o_dtype=torch.float32, segments=1)
+    og, Sg, Mg = run_gpu(mdn, inp, path="tensor", o_dtype=torch.float32, segments=segments)
+    e1 = rel_err(o1, o_ref), rel_err(S1, S_ref), rel_err(M1, M_ref)
+    eg = rel_err(og, o_ref), rel_err(Sg, S_ref), rel_err(Mg, M_ref)
+    print("serial   o %.3e S %.3e M %.3e" % e1)
+    print("G = %-3d  o %.3e S %.3e M %.3e" % ((segments,) + eg))
+    assert max(eg) <= TOL_BF16
+    nch = (T + 63) // 64
+    per = (nch + segments - 1) // segments * 64        # tokens of segment 0: computed by the same real run
+    assert np.array_equal(og[:, :per], o1[:, :per])
+    og2, Sg2, Mg2 = run_gpu(mdn, inp, path="tensor", o_dtype=torch.float32, segments=segments)
+    assert np.array_equal(og, og2) and np.array_equal(Sg, Sg2) and np.array_equal(Mg, Mg2)
+
+
+def test_parallel_scan_is_chosen_for_few_long_chains(mdn):
+    w3, w2 = wl.CONFIGS[3], wl.CONFIGS[2]
+    if not tensor_ok(mdn, w3):
+        pytest.skip("tensor path not built")
+    lay3 = mdn.workspace_layout(mdn.MdnParams(w3.B, w3.T, w3.H, w3.dk, w3.dv, 64, 0, 1, 1, 0, 1.0, 0))
+    lay2 = mdn.workspace_layout(mdn.MdnParams(w2.B, w2.T, w2.H, w2.dk, w2.dv, 64, 0, 1, 1, 0, 1.0, 0))
+    assert lay3.segments >= 4 and lay2.segments == 1
+    off = mdn.workspace_layout(mdn.MdnParams(w3.B, w3.T, w3.H, w3.dk, w3.dv, 64, 0, 1, 1, 0, 1.0, 1))
+    assert off.segments == 1 and off.total_bytes < lay3.total_bytes
 
 
 def test_state_handoff_and_determinism_tensor_path(mdn):
