@@ -15,6 +15,7 @@ bounded sample of the same workload; it is a deliberately slow program, reported
 from __future__ import annotations
 
 import argparse
+import ctypes
 import json
 import os
 import statistics
@@ -391,6 +392,55 @@ def run_decode(args):
                      "traffic": None, "peak_source": peaks["source"], "algorithmic_bytes": abytes}}))
 
 
+def run_layer_ops(args, w):
+    """Secondary benchmark (not the headline): the forward with the layer's element-wise operations (gate
+    parameterisation, q/k pre-processing, output norm + gate), once absorbed by the kernels and once as passes of
+    their own around the unchanged forward.  Same workload, inputs resident in HBM, CUDA events."""
+    import torch
+    import paper_2605_05838_b200 as mdn
+    mdn.lib()
+    torch.cuda.set_device(0)
+    inp = wl.make_layer_inputs(w)
+    dt = torch.bfloat16 if w.dtype == "bf16" else torch.float32
+    dev = lambda x, d=torch.float32: torch.from_numpy(np.ascontiguousarray(x)).to("cuda").to(d)
+    q, k, v, g = dev(inp["q"], dt), dev(inp["k"], dt), dev(inp["v"], dt), dev(inp["g"], dt)
+    gates = [dev(inp[n]) for n in ("x_beta", "x_alpha", "x_mu", "x_eta")]
+    gp = dict(a_alpha=dev(inp["a_alpha"]), b_alpha=dev(inp["b_alpha"]), a_mu=dev(inp["a_mu"]), b_mu=dev(inp["b_mu"]),
+              s=inp["s"], tau=inp["tau"], log_mu_min=inp["log_mu_min"])
+    dvec, wn = dev(inp["d"]), dev(inp["w_norm"])
+    out = torch.empty_like(v)
+    res = {}
+    for mode in ("fused", "separate"):
+        ops = mdn.make_layer_ops(q, v, gate_param=gp, qk_norm=dict(d=dvec, eps=inp["qk_eps"]),
+                                 out_norm_gate=dict(g=g, w=wn, eps=inp["rms_eps"]), separate_passes=mode == "separate")
+        need = int(mdn.lib().mdn_chunk_fwd_fused_workspace_bytes(
+            ctypes.byref(mdn.make_params(q, v, scale=inp["scale"], path=args.path)), ctypes.byref(ops)))
+        ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+
+        def step():
+            mdn.chunk_fwd(q, k, v, *gates, scale=inp["scale"], path=args.path, layer_ops=ops, workspace=ws, out=out)
+
+        for _ in range(max(args.warmup, 3)):
+            step()
+        launches = mdn.last_launch_count()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.steps):
+            step()
+        e1.record()
+        torch.cuda.synchronize()
+        res[mode] = {"ms_per_step": e0.elapsed_time(e1) / args.steps, "launches_per_step": launches}
+    tokens = w.B * w.T
+    print(json.dumps({
+        "metric": "MDN chunkwise fwd with layer ops tokens/s", "value": tokens / (res["fused"]["ms_per_step"] * 1e-3),
+        "unit": "tokens/s", "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "ms_per_step": res["fused"]["ms_per_step"], "higher_is_better": True, "dtype": w.dtype, "data": "synthetic",
+        "config": {"workload": workload_desc(w), "ops": "gate parameterisation + q/k L2Norm(q - d k) + RMSNorm*sigmoid gate"},
+        "gpu_launches": res["fused"]["launches_per_step"] * args.steps,
+        "separate_passes": res["separate"], "fused": res["fused"]}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -404,11 +454,16 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--decode", action="store_true", help="secondary benchmark: the recurrent decode step")
     ap.add_argument("--decode-batch", type=int, default=128)
+    ap.add_argument("--layer-ops", action="store_true",
+                    help="secondary benchmark: forward with the layer's element-wise operations, fused vs separate passes")
     args = ap.parse_args()
     if args.decode:
         run_decode(args)
         return
     w = wl.CONFIGS[args.config]
+    if args.layer_ops:
+        run_layer_ops(args, w)
+        return
     if args.impl == "reference":
         run_reference(args, w)
     else:

@@ -188,20 +188,77 @@ mdn_status mdn_chunk_fwd_static_scratch(const mdn_params* p,
                                         void* cuda_stream);
 
 /*
+ * The forward with the layer's element-wise operations fused in (Section 3.3, "Model Architecture" and
+ * "Stability Aware Gating Parameterization"): none of them needs weights beyond per-head scalars, and each
+ * would otherwise be a pass of its own over q, k, o or the gates.
+ *
+ *  raw_gates != 0: the beta / log_alpha / log_mu / eta arguments of the call hold the RAW per-head projections
+ *    x_beta, x_alpha, x_mu, x_eta ([B,T,H] float32, all four required) and the gates are
+ *        eta       = tanh(x_eta / tau) + 1                  theta = arctan(eta * s)
+ *        log_alpha = f_alpha(x_alpha) + log cos^2(theta)    beta  = sigmoid(x_beta) * sin^2(theta)
+ *        log_mu    = max(f_mu(x_mu), log_mu_min)            f(x)  = -a_h * softplus(x + b_h)
+ *    with per-head a_h, b_h (decay_a_alpha .. decay_b_mu: device float32[H], all four required).
+ *  qk_norm != 0:  q <- L2Norm(q - d_h k),  k <- L2Norm(k),  L2Norm(x) = x / sqrt(sum x^2 + qk_eps), qk_eps > 0;
+ *    d: device float32[H] or NULL (= 0).  Both use the un-normalised k (the correction comes before the norm).
+ *  out_norm_gate != 0: the output written to `o` is  sigmoid(g) * RMSNorm(o) * w  per head, RMSNorm(o) =
+ *    o / sqrt(mean_j o_j^2 + rms_eps);  g: device [B,T,H,dv] in the i/o dtype; w: device float32[dv] or NULL (= 1).
+ *  separate_passes != 0: run q/k pre-processing, the gate parameterisation and the output step as kernels of
+ *    their own before / after the unchanged forward (needs the larger workspace below).  It is what the fused
+ *    form is measured against, and the way the fp32 SIMT path always runs qk_norm and out_norm_gate.
+ *
+ * Fused form (tensor path): the gate formulas run inside the coefficient scan; the norms of k and q - d k come
+ * from the diagonals of the K K^T and Q K^T tiles the intra-chunk kernel computes anyway and are applied to
+ * fp32 accumulators (q and k are never rewritten or re-rounded); the output step runs in the chain kernel's
+ * output epilogue.  All pointers are device pointers; the struct itself is host memory, read during the call.
+ */
+typedef struct {
+  int32_t raw_gates;
+  const float* decay_a_alpha;
+  const float* decay_b_alpha;
+  const float* decay_a_mu;
+  const float* decay_b_mu;
+  float s, tau, log_mu_min;
+  int32_t qk_norm;
+  const float* d;
+  float qk_eps;
+  int32_t out_norm_gate;
+  const void* g;
+  const float* w;
+  float rms_eps;
+  int32_t separate_passes;
+} mdn_layer_ops;
+
+/* Workspace bytes of mdn_chunk_fwd_fused for these parameters and operations (0 on invalid ones);
+ * never less than mdn_chunk_fwd_workspace_bytes(p). */
+size_t mdn_chunk_fwd_fused_workspace_bytes(const mdn_params* p, const mdn_layer_ops* ops /* host */);
+
+/* mdn_chunk_fwd with `ops` applied; ops == NULL or all switches 0 is mdn_chunk_fwd itself.  Same
+ * argument rules, ownership and error behaviour. */
+mdn_status mdn_chunk_fwd_fused(const mdn_params* p, const mdn_layer_ops* ops /* host */,
+                               const void* q, const void* k, const void* v,
+                               const float* beta, const float* log_alpha, const float* log_mu,
+                               const float* eta,
+                               const float* initial_S, const float* initial_M,
+                               const int32_t* cu_seqlens,
+                               void* o, float* final_S, float* final_M,
+                               void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * Stage entry points (the same kernels mdn_chunk_fwd launches, exposed so that each
  * stage can be checked on its own).  Both write into `workspace` using the layout
  * mdn_workspace_layout describes; mdn_intra_chunk expects mdn_coeff_scan's output there.
  *
- * mdn_coeff_scan (a0 + a1, Eq. 10): for every chunk slot s and head h, ten float32
+ * mdn_coeff_scan (a0 + a1, Eq. 10): for every chunk slot s and head h, twelve float32
  * vectors of length 64 at  coef + ((s*H + h)*MDN_NUM_COEF + i)*64 :
  *   i=0 abar_r   1 b_r   2 alpha_r*b_{r-1}   3 gamma_{last,r}*eta_r   4 (mubar_last/mubar_r)*eta_r
- *   5 mubar_r    6 alpha_r  7 beta_r   8 mu_r   9 eta_r
+ *   5 mubar_r    6 1/|k_r|   7 1/|q_r - d k_r|   (both 1 unless the fused q/k norm is on; then 3 and 4
+ *   also carry the factor 1/|k_r|)   8 alpha_r  9 beta_r   10 mu_r   11 eta_r
  * Positions past the end of a short chunk hold exact no-ops (alpha = mu = 1, beta = eta = 0).
  *
  * mdn_intra_chunk (a2, Eq. 15 and the mask of Eq. 12): per (s, h) the 64x64 row-major
  * matrices T and W, as float32 (SIMT path) or bfloat16 (tensor path).
  */
-#define MDN_NUM_COEF 10
+#define MDN_NUM_COEF 12
 
 typedef struct {
   int32_t num_slots;        /* chunk slots: B*ceil(T/64), or an upper bound T/64 + num_seqs when packed */

@@ -194,6 +194,40 @@ def make_inputs(w: Workload, lengths: Optional[np.ndarray] = None) -> Dict[str, 
                 scale=w.scale, workload=w)
 
 
+def make_layer_inputs(w: Workload, s: float = 0.25, d_in: int = 2048) -> Dict[str, object]:
+    """Inputs of the forward WITH the layer's element-wise operations (Section 3.3): un-normalised q, k (stand-ins
+    for the activations after ShortConv + SiLU), the raw per-head gate projections, the per-head parameters and
+    the output gate.  Draws only: none of the operations is evaluated here.
+
+    Adds to make_inputs(w): q, k replaced by N(0, sigma_h^2) rows (sigma_h in [0.5, 2] per head);
+      x_beta, x_alpha, x_mu, x_eta [B,T,H] float32;  a_alpha, b_alpha, a_mu, b_mu, d [H] float32;
+      s, tau = sqrt(d_in / H), log_mu_min = -1;  g [B,T,H,dv] (stored in w.dtype), w_norm [dv] float32;
+      qk_eps = 1e-6, rms_eps = 1e-5.
+    """
+    inp = make_inputs(w)
+    B, T, H, dk, dv = w.B, w.T, w.H, w.dk, w.dv
+    sig = _rng(w.seed, 20).uniform(0.5, 2.0, (1, 1, H, 1)).astype(np.float32)
+    inp["q"] = _store(_rng(w.seed, 21).standard_normal((B, T, H, dk), dtype=np.float32) * sig, w.dtype)
+    inp["k"] = _store(_rng(w.seed, 22).standard_normal((B, T, H, dk), dtype=np.float32) * sig, w.dtype)
+    f32 = np.float32
+    inp["x_beta"] = _rng(w.seed, 23).standard_normal((B, T, H), dtype=f32)
+    inp["x_alpha"] = _rng(w.seed, 24).standard_normal((B, T, H), dtype=f32)
+    inp["x_mu"] = _rng(w.seed, 25).standard_normal((B, T, H), dtype=f32)
+    inp["x_eta"] = (8.0 * _rng(w.seed, 26).standard_normal((B, T, H), dtype=f32)).astype(f32)
+    inp["a_alpha"] = _rng(w.seed, 27).uniform(0.5, 8.0, H).astype(f32)
+    inp["b_alpha"] = (-4.0 + 0.5 * _rng(w.seed, 28).standard_normal(H)).astype(f32)
+    inp["a_mu"] = _rng(w.seed, 29).uniform(0.5, 8.0, H).astype(f32)
+    inp["b_mu"] = (-3.0 + 0.5 * _rng(w.seed, 30).standard_normal(H)).astype(f32)
+    inp["d"] = _rng(w.seed, 31).uniform(-0.2, 0.5, H).astype(f32)
+    inp["s"], inp["tau"], inp["log_mu_min"] = float(s), float(math.sqrt(d_in / H)), -1.0
+    inp["g"] = _store(1.5 * _rng(w.seed, 32).standard_normal((B, T, H, dv), dtype=f32), w.dtype)
+    inp["w_norm"] = _rng(w.seed, 33).uniform(0.5, 1.5, dv).astype(f32)
+    inp["qk_eps"], inp["rms_eps"] = 1e-6, 1e-5
+    for name in ("beta", "log_alpha", "log_mu", "eta"):
+        del inp[name]
+    return inp
+
+
 def correlated_keys(w: Workload, rho: float = 0.8) -> np.ndarray:
     """Unit keys sharing a common direction per head (pairwise cosine ~ rho): with
     i.i.d. keys the intra-chunk triangular system is nearly the identity, so this

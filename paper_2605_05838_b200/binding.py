@@ -20,7 +20,7 @@ MDN_F32, MDN_BF16 = 0, 1
 PATH_AUTO, PATH_SIMT, PATH_TENSOR = 0, 1, 2
 _PATHS = {"auto": PATH_AUTO, "simt": PATH_SIMT, "tensor": PATH_TENSOR}
 PATH_NAMES = {PATH_AUTO: "auto", PATH_SIMT: "simt", PATH_TENSOR: "tensor"}
-NUM_COEF = 10
+NUM_COEF = 12
 CHUNK = 64
 NUM_STAGE_EVENTS = 4
 STAGE_NAMES = ["coeff_scan", "intra_chunk", "chain"]
@@ -39,6 +39,17 @@ class MdnWsLayout(ctypes.Structure):
                 ("off_slot_map", ctypes.c_uint64), ("off_coef", ctypes.c_uint64),
                 ("off_T", ctypes.c_uint64), ("off_W", ctypes.c_uint64), ("total_bytes", ctypes.c_uint64),
                 ("off_seg", ctypes.c_uint64), ("segments", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+
+
+class MdnLayerOps(ctypes.Structure):
+    """mdn_layer_ops of include/mdn.h (Section 3.3 element-wise operations absorbed by the forward)."""
+    _fields_ = [("raw_gates", ctypes.c_int32),
+                ("decay_a_alpha", ctypes.c_void_p), ("decay_b_alpha", ctypes.c_void_p),
+                ("decay_a_mu", ctypes.c_void_p), ("decay_b_mu", ctypes.c_void_p),
+                ("s", ctypes.c_float), ("tau", ctypes.c_float), ("log_mu_min", ctypes.c_float),
+                ("qk_norm", ctypes.c_int32), ("d", ctypes.c_void_p), ("qk_eps", ctypes.c_float),
+                ("out_norm_gate", ctypes.c_int32), ("g", ctypes.c_void_p), ("w", ctypes.c_void_p),
+                ("rms_eps", ctypes.c_float), ("separate_passes", ctypes.c_int32)]
 
 
 class MdnError(RuntimeError):
@@ -67,6 +78,10 @@ def lib() -> ctypes.CDLL:
         L.mdn_chunk_fwd_host_arena_bytes.argtypes = [P]
         L.mdn_chunk_fwd.restype = ctypes.c_int
         L.mdn_chunk_fwd.argtypes = [P] + [vp] * 13 + [vp, ctypes.c_size_t, vp]
+        L.mdn_chunk_fwd_fused.restype = ctypes.c_int
+        L.mdn_chunk_fwd_fused.argtypes = [P, ctypes.POINTER(MdnLayerOps)] + [vp] * 13 + [vp, ctypes.c_size_t, vp]
+        L.mdn_chunk_fwd_fused_workspace_bytes.restype = ctypes.c_size_t
+        L.mdn_chunk_fwd_fused_workspace_bytes.argtypes = [P, ctypes.POINTER(MdnLayerOps)]
         L.mdn_chunk_fwd_host.restype = ctypes.c_int
         L.mdn_chunk_fwd_host.argtypes = [P] + [vp] * 13 + [vp, ctypes.c_size_t, vp]
         L.mdn_chunk_fwd_static_scratch.restype = ctypes.c_int
@@ -164,6 +179,46 @@ def workspace_layout(p: MdnParams) -> MdnWsLayout:
     return lay
 
 
+def _f32_vec(name, t, n):
+    if t is None:
+        return None
+    if t.device.type != "cuda" or t.dtype != torch.float32 or not t.is_contiguous() or t.numel() != n:
+        raise ValueError("%s must be a contiguous float32 cuda tensor of %d elements" % (name, n))
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def make_layer_ops(q, v, *, gate_param=None, qk_norm=None, out_norm_gate=None, separate_passes=False):
+    """Builds mdn_layer_ops from tensors (marshalling only; keep the tensors alive until the call returns).
+      gate_param    = dict(a_alpha, b_alpha, a_mu, b_mu: float32 [H]; s, tau: float; log_mu_min=-1.0): the gate
+                      arguments of the call are then the raw projections x_beta, x_alpha, x_mu, x_eta
+      qk_norm       = dict(d: float32 [H] or None, eps: float)
+      out_norm_gate = dict(g: [B,T,H,dv] in q's dtype, w: float32 [dv] or None, eps: float)"""
+    H, dv = q.shape[2], v.shape[-1]
+    ops = MdnLayerOps()
+    if gate_param is not None:
+        ops.raw_gates = 1
+        ops.decay_a_alpha = _f32_vec("a_alpha", gate_param["a_alpha"], H)
+        ops.decay_b_alpha = _f32_vec("b_alpha", gate_param["b_alpha"], H)
+        ops.decay_a_mu = _f32_vec("a_mu", gate_param["a_mu"], H)
+        ops.decay_b_mu = _f32_vec("b_mu", gate_param["b_mu"], H)
+        ops.s, ops.tau = float(gate_param["s"]), float(gate_param["tau"])
+        ops.log_mu_min = float(gate_param.get("log_mu_min", -1.0))
+    if qk_norm is not None:
+        ops.qk_norm = 1
+        ops.d = _f32_vec("d", qk_norm.get("d"), H)
+        ops.qk_eps = float(qk_norm["eps"])
+    if out_norm_gate is not None:
+        g = out_norm_gate["g"]
+        if g.device.type != "cuda" or g.dtype != q.dtype or not g.is_contiguous() or tuple(g.shape) != tuple(v.shape):
+            raise ValueError("g must be a contiguous cuda tensor with v's shape and dtype")
+        ops.out_norm_gate = 1
+        ops.g = ctypes.c_void_p(g.data_ptr())
+        ops.w = _f32_vec("w", out_norm_gate.get("w"), dv)
+        ops.rms_eps = float(out_norm_gate["eps"])
+    ops.separate_passes = 1 if separate_passes else 0
+    return ops
+
+
 def _check_inputs(q, k, v, gates, device_type: str):
     for name, t in (("q", q), ("k", k), ("v", v)):
         if t.device.type != device_type or not t.is_contiguous() or t.dim() != 4:
@@ -188,10 +243,13 @@ def _check_state(name, t, shape, device_type):
 def chunk_fwd(q, k, v, beta, log_alpha, log_mu, eta=None, *, initial_S=None, initial_M=None,
               cu_seqlens=None, scale: Optional[float] = None, o_dtype: Optional[torch.dtype] = None,
               path: str = "auto", output_final_state: bool = True, workspace: Optional[torch.Tensor] = None,
-              out: Optional[torch.Tensor] = None, segments: int = 0
+              out: Optional[torch.Tensor] = None, segments: int = 0, layer_ops: Optional[MdnLayerOps] = None
               ) -> Tuple[torch.Tensor, Optional[torch.Tensor], Optional[torch.Tensor]]:
-    """mdn_chunk_fwd on CUDA tensors (current stream).  Returns (o, final_S, final_M).
-    segments: 0 = automatic, 1 = plain serial chain, >= 3 = force the parallel inter-chunk scan."""
+    """mdn_chunk_fwd (mdn_chunk_fwd_fused when layer_ops is given) on CUDA tensors, current stream.
+    Returns (o, final_S, final_M).
+    segments: 0 = automatic, 1 = plain serial chain, >= 3 = force the parallel inter-chunk scan.
+    layer_ops: from make_layer_ops; with its gate_param set, beta / log_alpha / log_mu / eta are the raw
+    projections x_beta / x_alpha / x_mu / x_eta."""
     _check_inputs(q, k, v, (("beta", beta), ("log_alpha", log_alpha), ("log_mu", log_mu), ("eta", eta)), "cuda")
     B, T, H, dk = q.shape
     dv = v.shape[-1]
@@ -204,7 +262,10 @@ def chunk_fwd(q, k, v, beta, log_alpha, log_mu, eta=None, *, initial_S=None, ini
     nst = N if N > 0 else B
     _check_state("initial_S", initial_S, (nst, H, dk, dv), "cuda")
     _check_state("initial_M", initial_M, (nst, H, dk, dv), "cuda")
-    need = workspace_bytes(p)
+    if layer_ops is None:
+        need = workspace_bytes(p)
+    else:
+        need = int(lib().mdn_chunk_fwd_fused_workspace_bytes(ctypes.byref(p), ctypes.byref(layer_ops)))
     if need == 0:
         raise MdnError(2, "mdn_chunk_fwd_workspace_bytes")
     if workspace is None:
@@ -214,11 +275,15 @@ def chunk_fwd(q, k, v, beta, log_alpha, log_mu, eta=None, *, initial_S=None, ini
     if output_final_state:
         Sf = torch.empty((nst, H, dk, dv), dtype=torch.float32, device=q.device)
         Mf = torch.empty((nst, H, dk, dv), dtype=torch.float32, device=q.device)
-    st = lib().mdn_chunk_fwd(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(beta), _ptr(log_alpha), _ptr(log_mu),
-                             _ptr(eta), _ptr(initial_S), _ptr(initial_M), _ptr(cu_seqlens), _ptr(o), _ptr(Sf),
-                             _ptr(Mf), _ptr(workspace), workspace.numel(), _stream())
+    tail = (_ptr(q), _ptr(k), _ptr(v), _ptr(beta), _ptr(log_alpha), _ptr(log_mu), _ptr(eta), _ptr(initial_S),
+            _ptr(initial_M), _ptr(cu_seqlens), _ptr(o), _ptr(Sf), _ptr(Mf), _ptr(workspace), workspace.numel(),
+            _stream())
+    if layer_ops is None:
+        st = lib().mdn_chunk_fwd(ctypes.byref(p), *tail)
+    else:
+        st = lib().mdn_chunk_fwd_fused(ctypes.byref(p), ctypes.byref(layer_ops), *tail)
     if st != 0:
-        raise MdnError(st, "mdn_chunk_fwd")
+        raise MdnError(st, "mdn_chunk_fwd_fused" if layer_ops is not None else "mdn_chunk_fwd")
     return o, Sf, Mf
 
 

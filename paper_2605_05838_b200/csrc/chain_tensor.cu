@@ -70,6 +70,8 @@ struct Bars {
   uint64_t mo;        // MMA-3' done                                                   (commit)
   uint64_t zu;        // U (intra-chunk output) has been read                           (256)
   uint64_t ga;        // epilogue group sync                                            (256)
+  uint64_t gfull[2];  // output-gate tile of a stage's chunk landed (fused output step)   (1 + tx bytes)
+  uint64_t pn[2];     // fused output step: partial sums of a token half are in shared memory (128 each)
 };
 
 struct ChainArgs {
@@ -90,6 +92,12 @@ struct ChainArgs {
   float* seg_Psi;             // [chains][G-2][2][dk*dv]  segment run from a zero state
   float* seg_PhiS;            // [chains][G-2][2][dk*dv]  segment run with V = 0 from (S, M) = (I, 0)
   float* seg_PhiM;            // [chains][G-2][2][dk*dv]  ... from (0, I)
+  // layer operations absorbed by this kernel (Section 3.3)
+  int qk_on;                  // q <- L2Norm(q - d k), k <- L2Norm(k): coefficient vectors 6, 7 hold 1/|k|, 1/|q - d k|
+  const float* qk_d;          // [H] or NULL
+  int post_on;                // o <- sigmoid(g) * RMSNorm(o) * w; the g tile of a chunk takes its V tile's place
+  const float* post_w;        // [dv] or NULL
+  float post_eps;
   uint32_t drop_lo;           // debug: bit 0 R, 1 V~_S/V~_M, 2 V~ (output), 3 W: leave that operand's lo part out
   long long* timeline;        // debug: CTA 0 writes clock64() at [chunk*32 + event] (NULL = off)
 };
@@ -107,19 +115,21 @@ template <> __device__ __forceinline__ void stage_o<__nv_bfloat16>(uint8_t* tile
   reinterpret_cast<__nv_bfloat16*>(tile)[r * kD + d] = __float2bfloat16_rn(x);
 }
 
-template <typename TO>
+template <typename TO, bool kLayer>
 __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainArgs a,
                                                                   const __grid_constant__ CUtensorMap map_q,
                                                                   const __grid_constant__ CUtensorMap map_k,
                                                                   const __grid_constant__ CUtensorMap map_v,
                                                                   const __grid_constant__ CUtensorMap map_t,
                                                                   const __grid_constant__ CUtensorMap map_w,
-                                                                  const __grid_constant__ CUtensorMap map_o) {
+                                                                  const __grid_constant__ CUtensorMap map_o,
+                                                                  const __grid_constant__ CUtensorMap map_g) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   __shared__ __align__(8) Bars bars;
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
+  __shared__ float ssq_part[2][4][32];   // fused RMSNorm: per token half, per lane quarter, per token
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int H = a.g.H;
@@ -181,6 +191,11 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
   const uint32_t b_r = smem_u32(&bars.r), b_m2 = smem_u32(&bars.m2), b_zq = smem_u32(&bars.zq);
   const uint32_t b_v1 = smem_u32(&bars.v1), b_v2 = smem_u32(&bars.v2), b_m3 = smem_u32(&bars.m3);
   const uint32_t b_mo = smem_u32(&bars.mo), b_zu = smem_u32(&bars.zu), b_ga = smem_u32(&bars.ga);
+  const uint32_t b_gf0 = smem_u32(&bars.gfull[0]), b_gf1 = smem_u32(&bars.gfull[1]);
+  // kLayer = false compiles the layer operations out: the plain forward keeps its instruction count
+  const bool qk_on = kLayer && a.qk_on;
+  const bool post = kLayer && a.post_on && write_o;
+  const float dh = (qk_on && a.qk_d) ? __ldg(a.qk_d + h) : 0.f;
 
   if (tid == 0) {
     abort_flag = 0;
@@ -190,12 +205,15 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
     mbar_init(b_v2, kEpiThreads); mbar_init(b_ga, kEpiThreads); mbar_init(b_zq, kEpiThreads);
     mbar_init(b_zu, kEpiThreads);
     mbar_init(b_m1, 1); mbar_init(b_mq, 1); mbar_init(b_m2, 1); mbar_init(b_m3, 1); mbar_init(b_mo, 1);
+    mbar_init(b_gf0, 1); mbar_init(b_gf1, 1);
+    mbar_init(smem_u32(&bars.pn[0]), 128); mbar_init(smem_u32(&bars.pn[1]), 128);
     mbar_fence_init();
   }
   if (warp == kWarpMma) tmem_alloc(smem_u32(&tmem_slot), 512);
   if (warp == kWarpTma && lane == 0) {
     prefetch_tensormap(&map_q); prefetch_tensormap(&map_k); prefetch_tensormap(&map_v);
     prefetch_tensormap(&map_t); prefetch_tensormap(&map_w); prefetch_tensormap(&map_o);
+    if (post) prefetch_tensormap(&map_g);
   }
   tc_fence_before_sync();
   __syncthreads();
@@ -216,7 +234,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
     // ================================================================== TMA producer + output stores
     // Stage s = c & 1 serves chunk c, then (as the staged output tile) is written out and refilled for chunk c + 2.
     if (lane == 0) {
-      int issued = 0;
+      int issued = 0, g_issued = 0;
       for (int c = 0; c < nch + 2; ++c) {
         const int s = c & 1;
         const uint32_t st = s_base + kOffStage + s * kStageBytes;
@@ -258,10 +276,22 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
           MDN_MARK(c, kEvTmaIssued);
           issued = c + 1;
         }
+        if (post && c >= 1 && c - 1 < nch) {
+          // fused output step: once every epilogue thread has read V of chunk c - 1 (EPI-1 done), its place in the
+          // stage takes that chunk's output-gate tile, well ahead of the chunk's output epilogue
+          const int cg = c - 1;
+          MDN_WAIT(b_r, cg & 1);
+          const uint32_t gb = (cg & 1) ? b_gf1 : b_gf0;
+          mbar_arrive_expect_tx(gb, kTxV);
+          tma_load_2d(s_base + kOffStage + (cg & 1) * kStageBytes + kStV, &map_g, h * kD, sq.tok0 + cg * C, gb);
+          g_issued = cg + 1;
+        }
       }
       if (!ok) {   // giving up: let the copies already in flight land before the CTA exits
         for (int c = max(0, issued - 2); c < issued; ++c)
           for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait((c & 1) ? b_full1 : b_full0, (c >> 1) & 1); ++it) {}
+        for (int c = max(0, g_issued - 2); c < g_issued; ++c)
+          for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait((c & 1) ? b_gf1 : b_gf0, (c >> 1) & 1); ++it) {}
       }
       tma_store_wait_all();
     }
@@ -354,7 +384,8 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
     const int d = q4 * 32 + lane;
     const int r0 = 32 * hf;
     const uint32_t tl = tmem + (static_cast<uint32_t>(q4 * 32) << 16);
-    uint32_t ga_phase = 0;
+    uint32_t ga_phase = 0, pn_phase = 0;
+    const uint32_t b_pn = smem_u32(&bars.pn[hf]);
     float oi[32];   // scale (abar .* Q S - b .* Q M) for this thread's tokens, carried to the output step
 #pragma unroll
     for (int j = 0; j < 32; ++j) oi[j] = 0.f;
@@ -449,8 +480,46 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
           tc_fence_before_sync();
           mbar_arrive(b_zu);
           MDN_MARK(cp, kEvZuArrive);
+          if (!post) {
 #pragma unroll
-          for (int j = 0; j < 32; ++j) stage_o<TO>(stp, r0 + j, d, oi[j] + __uint_as_float(u[j]));
+            for (int j = 0; j < 32; ++j) stage_o<TO>(stp, r0 + j, d, oi[j] + __uint_as_float(u[j]));
+          } else {
+            // fused output step: y = sigmoid(g) * o / sqrt(mean_d o^2 + eps) * w_d.  The sum over the value
+            // dimension runs over the 32 lanes (transposing butterfly: lane l ends with token l's partial sum)
+            // and then over the four warps of this token half through shared memory.
+            float val[32], sqv[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              val[j] = oi[j] + __uint_as_float(u[j]);
+              sqv[j] = val[j] * val[j];
+            }
+#pragma unroll
+            for (int off = 16; off >= 1; off >>= 1) {
+              const bool up = (lane & off) != 0;
+#pragma unroll
+              for (int i = 0; i < off; ++i) {
+                const float keep = up ? sqv[i + off] : sqv[i];
+                const float send = up ? sqv[i] : sqv[i + off];
+                sqv[i] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+              }
+            }
+            ssq_part[hf][q4][lane] = sqv[0];
+            mbar_arrive(b_pn);
+            MDN_WAIT(b_pn, pn_phase);
+            pn_phase ^= 1;
+            __syncwarp();
+            const float tot = ssq_part[hf][0][lane] + ssq_part[hf][1][lane] + ssq_part[hf][2][lane] + ssq_part[hf][3][lane];
+            const float rstd = 1.f / sqrtf(tot * (1.f / kD) + a.post_eps);
+            const float wd = a.post_w ? __ldg(a.post_w + d) : 1.f;
+            MDN_WAIT((cp & 1) ? b_gf1 : b_gf0, (cp >> 1) & 1);
+            const __nv_bfloat16* sG = reinterpret_cast<const __nv_bfloat16*>(stp + kStV);
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              const float gj = __bfloat162float(sG[(r0 + j) * kD + d]);
+              const float gate = __fdividef(1.f, 1.f + __expf(-gj));
+              stage_o<TO>(stp, r0 + j, d, val[j] * __shfl_sync(0xffffffffu, rstd, j) * wd * gate);
+            }
+          }
         }
         fence_proxy_async_smem();
         mbar_arrive((cp & 1) ? b_go1 : b_go0);
@@ -482,10 +551,30 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
           for (int j = 0; j < 32; j += 4) {
             const float4 ab = *reinterpret_cast<const float4*>(cf + kAbar * C + r0 + j);
             const float4 pb = *reinterpret_cast<const float4*>(cf + kAlphaBPrev * C + r0 + j);
-            const float e0 = vv[j + 0] - ab.x * __uint_as_float(x[j + 0]) + pb.x * __uint_as_float(y[j + 0]);
-            const float e1 = vv[j + 1] - ab.y * __uint_as_float(x[j + 1]) + pb.y * __uint_as_float(y[j + 1]);
-            const float e2 = vv[j + 2] - ab.z * __uint_as_float(x[j + 2]) + pb.z * __uint_as_float(y[j + 2]);
-            const float e3 = vv[j + 3] - ab.w * __uint_as_float(x[j + 3]) + pb.w * __uint_as_float(y[j + 3]);
+            float e0, e1, e2, e3;
+            if (qk_on) {
+              // k' = k / |k|: X, Y are products with the raw k tile, so the norm scales the accumulators; the
+              // output correction q - d k turns Q S - d K S, Q M - d K M: its K terms are taken from X, Y here
+              const float4 rk = *reinterpret_cast<const float4*>(cf + kRk * C + r0 + j);
+              const float4 bb = *reinterpret_cast<const float4*>(cf + kB * C + r0 + j);
+              const float x0 = __uint_as_float(x[j + 0]), x1 = __uint_as_float(x[j + 1]);
+              const float x2 = __uint_as_float(x[j + 2]), x3 = __uint_as_float(x[j + 3]);
+              const float y0 = __uint_as_float(y[j + 0]), y1 = __uint_as_float(y[j + 1]);
+              const float y2 = __uint_as_float(y[j + 2]), y3 = __uint_as_float(y[j + 3]);
+              e0 = vv[j + 0] - rk.x * (ab.x * x0 - pb.x * y0);
+              e1 = vv[j + 1] - rk.y * (ab.y * x1 - pb.y * y1);
+              e2 = vv[j + 2] - rk.z * (ab.z * x2 - pb.z * y2);
+              e3 = vv[j + 3] - rk.w * (ab.w * x3 - pb.w * y3);
+              oi[j + 0] = -dh * (ab.x * x0 - bb.x * y0);
+              oi[j + 1] = -dh * (ab.y * x1 - bb.y * y1);
+              oi[j + 2] = -dh * (ab.z * x2 - bb.z * y2);
+              oi[j + 3] = -dh * (ab.w * x3 - bb.w * y3);
+            } else {
+              e0 = vv[j + 0] - ab.x * __uint_as_float(x[j + 0]) + pb.x * __uint_as_float(y[j + 0]);
+              e1 = vv[j + 1] - ab.y * __uint_as_float(x[j + 1]) + pb.y * __uint_as_float(y[j + 1]);
+              e2 = vv[j + 2] - ab.z * __uint_as_float(x[j + 2]) + pb.z * __uint_as_float(y[j + 2]);
+              e3 = vv[j + 3] - ab.w * __uint_as_float(x[j + 3]) + pb.w * __uint_as_float(y[j + 3]);
+            }
             split_pack_bf16(e0, e1, hi[j >> 1], lo[j >> 1]);
             split_pack_bf16(e2, e3, hi[(j >> 1) + 1], lo[(j >> 1) + 1]);
           }
@@ -521,10 +610,18 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
         for (int j = 0; j < 32; j += 4) {
           const float4 ab = *reinterpret_cast<const float4*>(cf + kAbar * C + r0 + j);
           const float4 bb = *reinterpret_cast<const float4*>(cf + kB * C + r0 + j);
-          oi[j + 0] = a.scale * (ab.x * __uint_as_float(z[j + 0]) - bb.x * __uint_as_float(u[j + 0]));
-          oi[j + 1] = a.scale * (ab.y * __uint_as_float(z[j + 1]) - bb.y * __uint_as_float(u[j + 1]));
-          oi[j + 2] = a.scale * (ab.z * __uint_as_float(z[j + 2]) - bb.z * __uint_as_float(u[j + 2]));
-          oi[j + 3] = a.scale * (ab.w * __uint_as_float(z[j + 3]) - bb.w * __uint_as_float(u[j + 3]));
+          if (qk_on) {   // q' = (q - d k) / |q - d k|: the K terms are already in oi
+            const float4 rq = *reinterpret_cast<const float4*>(cf + kRq * C + r0 + j);
+            oi[j + 0] = a.scale * rq.x * (oi[j + 0] + ab.x * __uint_as_float(z[j + 0]) - bb.x * __uint_as_float(u[j + 0]));
+            oi[j + 1] = a.scale * rq.y * (oi[j + 1] + ab.y * __uint_as_float(z[j + 1]) - bb.y * __uint_as_float(u[j + 1]));
+            oi[j + 2] = a.scale * rq.z * (oi[j + 2] + ab.z * __uint_as_float(z[j + 2]) - bb.z * __uint_as_float(u[j + 2]));
+            oi[j + 3] = a.scale * rq.w * (oi[j + 3] + ab.w * __uint_as_float(z[j + 3]) - bb.w * __uint_as_float(u[j + 3]));
+          } else {
+            oi[j + 0] = a.scale * (ab.x * __uint_as_float(z[j + 0]) - bb.x * __uint_as_float(u[j + 0]));
+            oi[j + 1] = a.scale * (ab.y * __uint_as_float(z[j + 1]) - bb.y * __uint_as_float(u[j + 1]));
+            oi[j + 2] = a.scale * (ab.z * __uint_as_float(z[j + 2]) - bb.z * __uint_as_float(u[j + 2]));
+            oi[j + 3] = a.scale * (ab.w * __uint_as_float(z[j + 3]) - bb.w * __uint_as_float(u[j + 3]));
+          }
         }
       }
       // ---------------- EPI-2: V~ -> (gamma_C eta) V~, ((mubar_C/mubar) eta) V~ [part a], V~ [part b]; bf16 hi, lo
@@ -613,7 +710,7 @@ cudaError_t launch_chain_tensor(const Plan& pl, const void* q, const void* k, co
   const mdn_params& p = pl.p;
   const uint64_t tokens = (uint64_t)p.B * p.T;
   const uint64_t mats = (uint64_t)pl.geom.num_slots * p.H;
-  CUtensorMap mq, mk, mv, mt, mw, mo;
+  CUtensorMap mq, mk, mv, mt, mw, mo, mg;
   const uint64_t row = (uint64_t)p.H * kD;
   if (!encode_tma_2d_bf16(&mq, TmaMap2D{q, row, tokens, row * 2, 64, 64, true}) ||
       !encode_tma_2d_bf16(&mk, TmaMap2D{k, row, tokens, row * 2, 64, 64, true}) ||
@@ -624,7 +721,12 @@ cudaError_t launch_chain_tensor(const Plan& pl, const void* q, const void* k, co
   const bool o_bf16 = p.o_dtype == MDN_BF16;
   if (!encode_tma_2d(&mo, TmaMap2D{o, row, tokens, row * (o_bf16 ? 2u : 4u), 128, 64, false}, !o_bf16))
     return cudaErrorInvalidValue;
+  // the output-gate tensor has V's shape and dtype; without the fused output step the map is never used
+  if (!encode_tma_2d_bf16(&mg, TmaMap2D{pl.post.on ? pl.post.g : v, row, tokens, row * 2, 128, 64, false}))
+    return cudaErrorInvalidValue;
   ChainArgs a;
+  a.qk_on = pl.qk.on; a.qk_d = pl.qk.d;
+  a.post_on = pl.post.on; a.post_w = pl.post.w; a.post_eps = pl.post.eps;
   a.g = pl.geom;
   a.coef = reinterpret_cast<const float*>(pl.ws + pl.lay.off_coef);
   a.S0 = S0; a.M0 = M0; a.o = o; a.Sf = Sf; a.Mf = Mf;
@@ -638,22 +740,20 @@ cudaError_t launch_chain_tensor(const Plan& pl, const void* q, const void* k, co
   a.seg_G = 0; a.seg_phase = 0;
   a.seg_E = a.seg_Psi = a.seg_PhiS = a.seg_PhiM = nullptr;
   const unsigned chains = (unsigned)pl.geom.num_seqs * p.H;
-  auto launch = [&](unsigned grid) -> cudaError_t {
-    cudaError_t e;
-    if (p.o_dtype == MDN_BF16) {
-      auto kern = chain_tensor_kernel<__nv_bfloat16>;
-      e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
-      if (e != cudaSuccess) return e;
-      e = launch_pdl(kern, dim3(grid), dim3(kThreads), kSmemBytes, pl.stream, a, mq, mk, mv, mt, mw, mo);
-    } else {
-      auto kern = chain_tensor_kernel<float>;
-      e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
-      if (e != cudaSuccess) return e;
-      e = launch_pdl(kern, dim3(grid), dim3(kThreads), kSmemBytes, pl.stream, a, mq, mk, mv, mt, mw, mo);
-    }
+  const bool layer = a.qk_on || a.post_on;
+  auto launch_as = [&](auto kern, unsigned grid) -> cudaError_t {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    if (e != cudaSuccess) return e;
+    e = launch_pdl(kern, dim3(grid), dim3(kThreads), kSmemBytes, pl.stream, a, mq, mk, mv, mt, mw, mo, mg);
     if (e == cudaSuccess) e = cudaGetLastError();
     if (e == cudaSuccess) ++*launches;
     return e;
+  };
+  auto launch = [&](unsigned grid) -> cudaError_t {
+    if (p.o_dtype == MDN_BF16)
+      return layer ? launch_as(chain_tensor_kernel<__nv_bfloat16, true>, grid)
+                   : launch_as(chain_tensor_kernel<__nv_bfloat16, false>, grid);
+    return layer ? launch_as(chain_tensor_kernel<float, true>, grid) : launch_as(chain_tensor_kernel<float, false>, grid);
   };
   const int G = pl.lay.segments;
   if (G <= 1) return launch(chains);

@@ -95,7 +95,7 @@ constexpr int kScanWarps = 8;
 __global__ void __launch_bounds__(kScanWarps * 32) coeff_scan_kernel(ChunkGeom g, const float* __restrict__ beta,
                                                                     const float* __restrict__ log_alpha,
                                                                     const float* __restrict__ log_mu,
-                                                                    const float* __restrict__ eta,
+                                                                    const float* __restrict__ eta, GateParam gp,
                                                                     float* __restrict__ coef) {
   extern __shared__ float sm[];   // [4][64*H]: log_alpha, log_mu, beta, eta
   const int slot = blockIdx.x;
@@ -128,11 +128,13 @@ __global__ void __launch_bounds__(kScanWarps * 32) coeff_scan_kernel(ChunkGeom g
 #pragma unroll
     for (int e = 0; e < 2; ++e) {
       const int r = r0 + e;
-      const bool ok = r < si.n;
-      al[e] = ok ? expf(sm[0 * C * H + r * H + h]) : 1.0f;
-      mu[e] = ok ? expf(sm[1 * C * H + r * H + h]) : 1.0f;
-      be[e] = ok ? sm[2 * C * H + r * H + h] : 0.0f;
-      et[e] = ok ? sm[3 * C * H + r * H + h] : 0.0f;
+      al[e] = mu[e] = 1.0f;
+      be[e] = et[e] = 0.0f;
+      if (r < si.n) {
+        const TokenGates tg = load_token_gates(gp, h, sm[0 * C * H + r * H + h], sm[1 * C * H + r * H + h],
+                                               sm[2 * C * H + r * H + h], sm[3 * C * H + r * H + h]);
+        al[e] = tg.alpha; mu[e] = tg.mu; be[e] = tg.beta; et[e] = tg.eta;
+      }
     }
     const HeadCoefs hc = scan_head(al, mu, be, et, lane);
     float* out = coef + ((size_t)slot * H + h) * MDN_NUM_COEF * C;
@@ -149,6 +151,8 @@ __global__ void __launch_bounds__(kScanWarps * 32) coeff_scan_kernel(ChunkGeom g
     put(kMu, mu[0], mu[1]);
     put(kEta, et[0], et[1]);
     put(kMubar, hc.mubar[0], hc.mubar[1]);
+    put(kRk, 1.0f, 1.0f);
+    put(kRq, 1.0f, 1.0f);
   }
   grid_launch_dependents();
 }
@@ -161,7 +165,7 @@ cudaError_t launch_coeff_scan(const Plan& pl, const float* beta, const float* lo
     if (e != cudaSuccess) return e;
   }
   coeff_scan_kernel<<<pl.geom.num_slots, kScanWarps * 32, smem, pl.stream>>>(
-      pl.geom, beta, log_alpha, log_mu, eta, reinterpret_cast<float*>(pl.ws + pl.lay.off_coef));
+      pl.geom, beta, log_alpha, log_mu, eta, pl.gp, reinterpret_cast<float*>(pl.ws + pl.lay.off_coef));
   ++*launches;
   return cudaGetLastError();
 }

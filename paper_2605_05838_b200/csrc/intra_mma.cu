@@ -28,7 +28,8 @@ constexpr int LM = C + 4;     // fp32 elements per row of the 64x64 matrices (16
 
 constexpr uint32_t kOffK = 0, kOffQ = 16384;                 // bf16 tiles, two [64 x 128 B] swizzled blocks each
 constexpr uint32_t kOffG = 32768;                            // Gamma [64][68] fp32; later T
-constexpr uint32_t kOffCv = kOffG + C * LM * 4;              // alpha, beta, mu, eta
+constexpr uint32_t kOffCv = kOffG + C * LM * 4;              // alpha, beta, mu, eta, then the q/k-norm vectors
+constexpr int kCvVecs = 11;                                  // + gamma_C eta, (mubar_C/mubar) eta, 1/|k|, 1/|q - dk|, |q|^2, q.k, |k|^2
 // the tile area is reused once the MMAs are done: first as the bf16 staging of W_hi / W_lo, then for A and scratch
 constexpr int LW = C + 8;                                    // bf16 elements per staged W row (144 B: conflict-free)
 constexpr uint32_t kOffWh = 0, kOffWl = C * LW * 2;          // W_hi, W_lo staging [64][72] bf16
@@ -36,7 +37,7 @@ constexpr uint32_t kOffA = 0;                                // A [64][68] fp32
 constexpr int LD16 = 16 * 16 + 4;                            // floats per compact 16x16 diagonal block (+4: bank shift)
 constexpr uint32_t kOffAd = C * LM * 4;                      // the four diagonal blocks of A, compact
 constexpr uint32_t kOffP = kOffAd + 4 * LD16 * 4;            // product scratch [32][68] fp32
-constexpr uint32_t kSmem = kOffCv + 4 * C * 4 + 1024;        // + slack for the 1024-byte alignment
+constexpr uint32_t kSmem = kOffCv + kCvVecs * C * 4 + 1024;        // + slack for the 1024-byte alignment
 static_assert(kOffP + 32 * LM * 4 <= kOffG && kOffWl + C * LW * 2 <= kOffG, "reuse of the tile area");
 
 __device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
@@ -92,7 +93,8 @@ __device__ __forceinline__ void block_mma_tf32(float (&acc)[NT][4], const float*
 
 __global__ void __launch_bounds__(kThreads) intra_mma_kernel(ChunkGeom g, const __grid_constant__ CUtensorMap map_q,
                                                             const __grid_constant__ CUtensorMap map_k,
-                                                            float* __restrict__ coef, GateArgs gates, float scale,
+                                                            float* __restrict__ coef, GateArgs gates, GateParam gp,
+                                                            QkNorm qkn, float scale,
                                                             __nv_bfloat16* __restrict__ Tout,
                                                             __nv_bfloat16* __restrict__ Wout, size_t w_lo_offset,
                                                             int32_t* __restrict__ status) {
@@ -130,6 +132,8 @@ __global__ void __launch_bounds__(kThreads) intra_mma_kernel(ChunkGeom g, const 
   float* cf = coef + ((size_t)slot * g.H + h) * MDN_NUM_COEF * C;
   if (gates.log_alpha == nullptr) {
     for (int idx = tid; idx < 4 * C; idx += kThreads) cv[idx] = cf[kAlpha * C + idx];
+    if (qkn.on)
+      for (int idx = tid; idx < 2 * C; idx += kThreads) cv[4 * C + idx] = cf[kGS * C + idx];   // gamma_C eta, (mubar_C/mubar) eta
     __syncthreads();   // coefficients in smem; barrier initialised before anyone waits on it
   } else {
     // fused coefficient scan (Eq. 10): this head's gates (stride H floats), then one warp runs the scans,
@@ -137,10 +141,14 @@ __global__ void __launch_bounds__(kThreads) intra_mma_kernel(ChunkGeom g, const 
     if (tid < C) {
       const bool valid = tid < si.n;
       const size_t gi = ((size_t)si.tok0 + tid) * g.H + h;
-      cv[0 * C + tid] = valid ? expf(__ldg(gates.log_alpha + gi)) : 1.f;
-      cv[1 * C + tid] = valid ? __ldg(gates.beta + gi) : 0.f;
-      cv[2 * C + tid] = valid ? expf(__ldg(gates.log_mu + gi)) : 1.f;
-      cv[3 * C + tid] = valid ? (gates.eta ? __ldg(gates.eta + gi) : 1.f) : 0.f;
+      TokenGates tg{1.f, 1.f, 0.f, 0.f};
+      if (valid)
+        tg = load_token_gates(gp, h, __ldg(gates.log_alpha + gi), __ldg(gates.log_mu + gi), __ldg(gates.beta + gi),
+                              gates.eta ? __ldg(gates.eta + gi) : 1.f);
+      cv[0 * C + tid] = tg.alpha;
+      cv[1 * C + tid] = tg.beta;
+      cv[2 * C + tid] = tg.mu;
+      cv[3 * C + tid] = tg.eta;
     }
     __syncthreads();   // gates in smem; barrier initialised before anyone waits on it
     if (warp == 3) {   // an otherwise idle warp, concurrently with the Gamma recurrence of warps 0 and 1
@@ -155,6 +163,13 @@ __global__ void __launch_bounds__(kThreads) intra_mma_kernel(ChunkGeom g, const 
       put(kGS, hc.gs[0], hc.gs[1]);
       put(kGM, hc.gm[0], hc.gm[1]);
       put(kMubar, hc.mubar[0], hc.mubar[1]);
+      if (qkn.on) {   // the last-row weights get their 1/|k| factor once the norms are known
+        reinterpret_cast<float2*>(cv + 4 * C)[lane] = make_float2(hc.gs[0], hc.gs[1]);
+        reinterpret_cast<float2*>(cv + 5 * C)[lane] = make_float2(hc.gm[0], hc.gm[1]);
+      } else {
+        put(kRk, 1.f, 1.f);
+        put(kRq, 1.f, 1.f);
+      }
     }
   }
 
@@ -221,6 +236,49 @@ __global__ void __launch_bounds__(kThreads) intra_mma_kernel(ChunkGeom g, const 
       }
     }
   }
+  if (qkn.on) {
+    // fused q/k norm: |k_r|^2 and q_r . k_r are the diagonals of the two products; |q_r|^2 is summed from the
+    // Q tile (two threads per row); then  |q - d k|^2 = |q|^2 - 2 d q.k + d^2 |k|^2
+    if (ok) {
+      const int row = tid >> 1, hb = tid & 1;
+      float ssq = 0.f;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const uint4 u = *reinterpret_cast<const uint4*>(smem + kOffQ + tile_chunk(row, hb * 8 + j));
+        const uint32_t w4[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float lo = __uint_as_float(w4[e] << 16), hi = __uint_as_float(w4[e] & 0xffff0000u);
+          ssq = fmaf(lo, lo, fmaf(hi, hi, ssq));
+        }
+      }
+      ssq += __shfl_xor_sync(0xffffffffu, ssq, 1);
+      if (hb == 0) cv[8 * C + row] = ssq;
+    }
+#pragma unroll
+    for (int t = 0; t < 8; ++t) {
+      if ((t >> 1) == warp) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int r = warp * 16 + fg + (e >> 1) * 8, i = t * 8 + ft * 2 + (e & 1);
+          if (r == i) { cv[9 * C + r] = qk[t][e]; cv[10 * C + r] = kk[t][e]; }
+        }
+      }
+    }
+    __syncthreads();
+    if (tid < C) {
+      const float dh = qkn.d ? __ldg(qkn.d + h) : 0.f;
+      const float nk2 = cv[10 * C + tid], nq2 = cv[8 * C + tid], qkd = cv[9 * C + tid];
+      const float rk = 1.f / sqrtf(nk2 + qkn.eps);
+      const float rq = 1.f / sqrtf(fmaxf(nq2 - 2.f * dh * qkd + dh * dh * nk2, 0.f) + qkn.eps);
+      cv[6 * C + tid] = rk;
+      cv[7 * C + tid] = rq;
+      cf[kGS * C + tid] = cv[4 * C + tid] * rk;
+      cf[kGM * C + tid] = cv[5 * C + tid] * rk;
+      cf[kRk * C + tid] = rk;
+      cf[kRq * C + tid] = rq;
+    }
+  }
   __syncthreads();   // Gamma complete; every warp is done reading the K and Q tiles
 
   // ---- W and A from the accumulator fragments (rows fg and fg + 8 of the warp's 16, column pairs), one pass:
@@ -241,10 +299,18 @@ __global__ void __launch_bounds__(kThreads) intra_mma_kernel(ChunkGeom g, const 
         const float alr = cv[0 * C + r];
         float2 ga = make_float2(0.f, 0.f);
         if (r > 0) ga = *reinterpret_cast<const float2*>(Gs + (r - 1) * LM + i0);
-        wv0 = scale * gw.x * et.x * qk[t][half * 2];
-        wv1 = scale * gw.y * et.y * qk[t][half * 2 + 1];
-        av0 = alr * ga.x * et.x * kk[t][half * 2];
-        av1 = alr * ga.y * et.y * kk[t][half * 2 + 1];
+        float q0 = qk[t][half * 2], q1 = qk[t][half * 2 + 1], k0 = kk[t][half * 2], k1 = kk[t][half * 2 + 1];
+        if (qkn.on) {   // (q_r - d k_r) . k_i / (|q_r - d k_r| |k_i|)  and  k_r . k_i / (|k_r| |k_i|)
+          const float dh = qkn.d ? __ldg(qkn.d + h) : 0.f;
+          const float2 rki = *reinterpret_cast<const float2*>(cv + 6 * C + i0);
+          const float rkr = cv[6 * C + r], rqr = cv[7 * C + r];
+          q0 = (q0 - dh * k0) * rqr * rki.x; q1 = (q1 - dh * k1) * rqr * rki.y;
+          k0 *= rkr * rki.x; k1 *= rkr * rki.y;
+        }
+        wv0 = scale * gw.x * et.x * q0;
+        wv1 = scale * gw.y * et.y * q1;
+        av0 = alr * ga.x * et.x * k0;
+        av1 = alr * ga.y * et.y * k1;
         if ((t >> 1) == warp) {   // diagonal block: W keeps i <= r, A keeps i < r
           if (i0 > r) { wv0 = 0.f; }
           if (i0 + 1 > r) { wv1 = 0.f; }
@@ -373,7 +439,7 @@ cudaError_t launch_intra_mma(const Plan& pl, const void* q, const void* k, const
       !encode_tma_2d_bf16(&mk, TmaMap2D{k, row, tokens, row * 2, 64, 64, true}))
     return cudaErrorInvalidValue;
   e = launch_pdl(intra_mma_kernel, dim3((unsigned)n_mats), dim3(kThreads), kSmem, pl.stream, pl.geom, mq, mk,
-                 reinterpret_cast<float*>(pl.ws + pl.lay.off_coef), gates, pl.p.scale,
+                 reinterpret_cast<float*>(pl.ws + pl.lay.off_coef), gates, pl.gp, pl.qk, pl.p.scale,
                  reinterpret_cast<__nv_bfloat16*>(pl.ws + pl.lay.off_T),
                  reinterpret_cast<__nv_bfloat16*>(pl.ws + pl.lay.off_W), n_mats * C * C,
                  reinterpret_cast<int32_t*>(pl.ws + pl.lay.off_status));

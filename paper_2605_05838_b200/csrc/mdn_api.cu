@@ -75,6 +75,9 @@ static mdn_status make_plan(const mdn_params* p, const int32_t* cu, void* ws, si
   if (!ws || ws_bytes < pl->lay.total_bytes || !aligned(ws, 256)) return MDN_ERR_WORKSPACE;
   pl->ws = static_cast<char*>(ws);
   pl->stream = static_cast<cudaStream_t>(stream);
+  pl->gp = GateParam{};
+  pl->qk = QkNorm{};
+  pl->post = OutPost{};
   ChunkGeom& g = pl->geom;
   g.B = p->B; g.T = p->T; g.H = p->H;
   g.num_seqs = cu ? p->num_seqs : p->B;
@@ -147,14 +150,11 @@ mdn_status mdn_intra_chunk(const mdn_params* p, const void* q, const void* k, co
   return run_intra(pl, q, k, &t_last_launches);
 }
 
-mdn_status mdn_chunk_fwd(const mdn_params* p, const void* q, const void* k, const void* v, const float* beta,
-                         const float* log_alpha, const float* log_mu, const float* eta, const float* initial_S,
-                         const float* initial_M, const int32_t* cu_seqlens, void* o, float* final_S,
-                         float* final_M, void* workspace, size_t workspace_bytes, void* cuda_stream) {
-  t_last_launches = 0;
-  Plan pl;
-  mdn_status st = make_plan(p, cu_seqlens, workspace, workspace_bytes, cuda_stream, &pl);
-  if (st != MDN_OK) return st;
+// The forward proper on a finished plan (chunk map, scan, intra-chunk stage, chain); pl.gp / pl.qk / pl.post say
+// which layer operations the kernels absorb.
+static mdn_status run_forward(const Plan& pl, const void* q, const void* k, const void* v, const float* beta,
+                              const float* log_alpha, const float* log_mu, const float* eta, const float* initial_S,
+                              const float* initial_M, void* o, float* final_S, float* final_M) {
   if (!q || !k || !v || !o) return MDN_ERR_INVALID_ARG;
   if (!aligned(q, 16) || !aligned(k, 16) || !aligned(v, 16) || !aligned(o, 16)) return MDN_ERR_INVALID_ARG;
   if ((initial_S && !aligned(initial_S, 16)) || (initial_M && !aligned(initial_M, 16)) ||
@@ -164,7 +164,7 @@ mdn_status mdn_chunk_fwd(const mdn_params* p, const void* q, const void* k, cons
   // tensor path: the intra-chunk kernel runs the coefficient scan itself (one kernel and one round trip of
   // the coefficient vectors less); SIMT path: stand-alone scan kernel
   const bool fused_scan = pl.p.path == MDN_PATH_TENSOR;
-  st = run_prep_and_scan(pl, beta, log_alpha, log_mu, eta, &t_last_launches, !fused_scan);
+  mdn_status st = run_prep_and_scan(pl, beta, log_alpha, log_mu, eta, &t_last_launches, !fused_scan);
   if (st != MDN_OK) return st;
   if (!mark_stage(1, pl.stream)) return MDN_ERR_CUDA;
   st = fused_scan ? run_intra(pl, q, k, &t_last_launches, GateArgs{beta, log_alpha, log_mu, eta})
@@ -176,6 +176,109 @@ mdn_status mdn_chunk_fwd(const mdn_params* p, const void* q, const void* k, cons
                       : launch_chain_simt(pl, q, k, v, initial_S, initial_M, o, final_S, final_M, &t_last_launches);
   if (e != cudaSuccess) { t_last_cuda_error = (int)e; return MDN_ERR_CUDA; }
   if (!mark_stage(3, pl.stream)) return MDN_ERR_CUDA;
+  return MDN_OK;
+}
+
+mdn_status mdn_chunk_fwd(const mdn_params* p, const void* q, const void* k, const void* v, const float* beta,
+                         const float* log_alpha, const float* log_mu, const float* eta, const float* initial_S,
+                         const float* initial_M, const int32_t* cu_seqlens, void* o, float* final_S,
+                         float* final_M, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  t_last_launches = 0;
+  Plan pl;
+  mdn_status st = make_plan(p, cu_seqlens, workspace, workspace_bytes, cuda_stream, &pl);
+  if (st != MDN_OK) return st;
+  return run_forward(pl, q, k, v, beta, log_alpha, log_mu, eta, initial_S, initial_M, o, final_S, final_M);
+}
+
+// ---- the forward with layer operations
+static bool ops_active(const mdn_layer_ops* ops) {
+  return ops && (ops->raw_gates || ops->qk_norm || ops->out_norm_gate);
+}
+
+static mdn_status check_ops(const mdn_layer_ops& f) {
+  if (f.raw_gates) {
+    if (!f.decay_a_alpha || !f.decay_b_alpha || !f.decay_a_mu || !f.decay_b_mu) return MDN_ERR_INVALID_ARG;
+    if (!(f.tau > 0.f) || !(f.s == f.s) || !(f.log_mu_min == f.log_mu_min)) return MDN_ERR_INVALID_ARG;
+  }
+  if (f.qk_norm && !(f.qk_eps > 0.f)) return MDN_ERR_INVALID_ARG;
+  if (f.out_norm_gate && (!f.g || !aligned(f.g, 16) || !(f.rms_eps >= 0.f))) return MDN_ERR_INVALID_ARG;
+  return MDN_OK;
+}
+
+// Scratch of the separate passes, appended to the plain workspace: q', k' (i/o dtype) and the four gate arrays.
+struct SepLayout { uint64_t q, k, gates[4], total; bool qk_sep, out_sep, gate_sep; };
+
+static mdn_status sep_layout(const mdn_params& p, const mdn_layer_ops& f, const mdn_ws_layout& lay, SepLayout* sl) {
+  const bool simt = resolve_path(p) != MDN_PATH_TENSOR;
+  sl->qk_sep = f.qk_norm && (f.separate_passes || simt);
+  sl->out_sep = f.out_norm_gate && (f.separate_passes || simt);
+  sl->gate_sep = f.raw_gates && f.separate_passes;
+  const uint64_t tokens = (uint64_t)p.B * p.T, es = p.io_dtype == MDN_BF16 ? 2 : 4;
+  uint64_t off = lay.total_bytes;
+  auto take = [&](uint64_t bytes) { uint64_t at = off; off = align_up(off + bytes, 256); return at; };
+  sl->q = take(sl->qk_sep ? tokens * p.H * p.dk * es : 0);
+  sl->k = take(sl->qk_sep ? tokens * p.H * p.dk * es : 0);
+  for (int i = 0; i < 4; ++i) sl->gates[i] = take(sl->gate_sep ? tokens * p.H * 4 : 0);
+  sl->total = off;
+  return MDN_OK;
+}
+
+size_t mdn_chunk_fwd_fused_workspace_bytes(const mdn_params* p, const mdn_layer_ops* ops) {
+  mdn_ws_layout lay;
+  if (check_params(p) != MDN_OK || make_layout(*p, &lay) != MDN_OK) return 0;
+  if (!ops_active(ops)) return (size_t)lay.total_bytes;
+  if (check_ops(*ops) != MDN_OK) return 0;
+  SepLayout sl;
+  sep_layout(*p, *ops, lay, &sl);
+  return (size_t)sl.total;
+}
+
+mdn_status mdn_chunk_fwd_fused(const mdn_params* p, const mdn_layer_ops* ops, const void* q, const void* k,
+                               const void* v, const float* beta, const float* log_alpha, const float* log_mu,
+                               const float* eta, const float* initial_S, const float* initial_M,
+                               const int32_t* cu_seqlens, void* o, float* final_S, float* final_M, void* workspace,
+                               size_t workspace_bytes, void* cuda_stream) {
+  if (!ops_active(ops))
+    return mdn_chunk_fwd(p, q, k, v, beta, log_alpha, log_mu, eta, initial_S, initial_M, cu_seqlens, o, final_S,
+                         final_M, workspace, workspace_bytes, cuda_stream);
+  t_last_launches = 0;
+  mdn_status st = check_params(p);
+  if (st != MDN_OK) return st;
+  st = check_ops(*ops);
+  if (st != MDN_OK) return st;
+  Plan pl;
+  st = make_plan(p, cu_seqlens, workspace, workspace_bytes, cuda_stream, &pl);
+  if (st != MDN_OK) return st;
+  SepLayout sl;
+  sep_layout(*p, *ops, pl.lay, &sl);
+  if (workspace_bytes < sl.total) return MDN_ERR_WORKSPACE;
+  if (!q || !k || !aligned(q, 16) || !aligned(k, 16) || !o || !aligned(o, 16)) return MDN_ERR_INVALID_ARG;
+  if (ops->raw_gates) {
+    if (!beta || !log_alpha || !log_mu || !eta) return MDN_ERR_INVALID_ARG;
+    pl.gp = GateParam{1, ops->decay_a_alpha, ops->decay_b_alpha, ops->decay_a_mu, ops->decay_b_mu, ops->s,
+                      1.0f / ops->tau, ops->log_mu_min};
+  }
+  const QkNorm qk{ops->qk_norm ? 1 : 0, ops->d, ops->qk_eps};
+  const OutPost post{ops->out_norm_gate ? 1 : 0, ops->g, ops->w, ops->rms_eps};
+  char* ws = pl.ws;
+  if (sl.gate_sep) {
+    float* g4[4];
+    for (int i = 0; i < 4; ++i) g4[i] = reinterpret_cast<float*>(ws + sl.gates[i]);
+    if (launch_gate_param(pl, beta, log_alpha, log_mu, eta, g4[0], g4[1], g4[2], g4[3], &t_last_launches) != cudaSuccess)
+      return MDN_ERR_CUDA;
+    beta = g4[0]; log_alpha = g4[1]; log_mu = g4[2]; eta = g4[3];
+    pl.gp = GateParam{};
+  }
+  if (sl.qk_sep) {
+    if (launch_qk_prep(pl, qk, q, k, ws + sl.q, ws + sl.k, &t_last_launches) != cudaSuccess) return MDN_ERR_CUDA;
+    q = ws + sl.q; k = ws + sl.k;
+  } else {
+    pl.qk = qk;
+  }
+  if (!sl.out_sep) pl.post = post;
+  st = run_forward(pl, q, k, v, beta, log_alpha, log_mu, eta, initial_S, initial_M, o, final_S, final_M);
+  if (st != MDN_OK) return st;
+  if (sl.out_sep && launch_out_norm_gate(pl, post, o, &t_last_launches) != cudaSuccess) return MDN_ERR_CUDA;
   return MDN_OK;
 }
 

@@ -5,6 +5,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "layer_ops.cuh"
 #include "mdn.h"
 
 namespace mdn {
@@ -18,13 +19,16 @@ enum Coef : int {
   kAlphaBPrev = 2,  // alpha_r * b_{r-1}          (weight of +K M_[t] in the right-hand side)
   kGS = 3,      // gamma_{last,r} * eta_r         (weight of k_r v~_r^T in S_[t+1])
   kGM = 4,      // (mubar_last/mubar_r) * eta_r   (weight of -k_r v~_r^T in M_[t+1])
-  kMubar = 5,   // mubar_r = prod_{j<=r} mu_j   (vectors 0..5 are what the chain kernels read)
-  kAlpha = 6,
-  kBeta = 7,
-  kMu = 8,
-  kEta = 9
+  kMubar = 5,   // mubar_r = prod_{j<=r} mu_j
+  kRk = 6,      // 1 / |k_r|         (fused q/k norm; 1 otherwise)
+  kRq = 7,      // 1 / |q_r - d k_r| (vectors 0..7 are what the chain kernels read)
+  kAlpha = 8,
+  kBeta = 9,
+  kMu = 10,
+  kEta = 11
 };
-constexpr int kChainCoefs = 6;
+constexpr int kChainCoefs = 8;
+static_assert(kEta + 1 == MDN_NUM_COEF, "coefficient vector count");
 
 // Device-side error codes written to the workspace status word.
 enum DevErr : int { kDevOk = 0, kDevBadCuSeqlens = 1, kDevTimeout = 2 };
@@ -107,6 +111,17 @@ template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(flo
 // coefficients are already in the workspace.
 struct GateArgs { const float* beta; const float* log_alpha; const float* log_mu; const float* eta; };
 
+// One (token, head)'s alpha, mu, beta, eta from the gate arrays (raw projections when gp.raw).
+struct TokenGates { float alpha, mu, beta, eta; };
+__device__ __forceinline__ TokenGates load_token_gates(const GateParam& gp, int h, float v_log_alpha, float v_log_mu,
+                                                       float v_beta, float v_eta) {
+  if (gp.raw) {
+    const GateValues gv = gate_transform(gp, h, v_log_alpha, v_log_mu, v_beta, v_eta);
+    return TokenGates{expf(gv.log_alpha), expf(gv.log_mu), gv.beta, gv.eta};
+  }
+  return TokenGates{expf(v_log_alpha), expf(v_log_mu), v_beta, v_eta};
+}
+
 // Host-side view of one call, filled by the API layer.
 struct Plan {
   mdn_params p;
@@ -114,6 +129,9 @@ struct Plan {
   ChunkGeom geom;
   char* ws;
   cudaStream_t stream;
+  GateParam gp;    // layer operations the kernels absorb (all off for the plain forward)
+  QkNorm qk;
+  OutPost post;
 };
 
 // Launchers (one per .cu file).  Each returns the CUDA error of its launches and adds
@@ -121,6 +139,13 @@ struct Plan {
 cudaError_t launch_chunk_map(const Plan& pl, int* launches);
 cudaError_t launch_coeff_scan(const Plan& pl, const float* beta, const float* log_alpha,
                               const float* log_mu, const float* eta, int* launches);
+// The layer operations as passes of their own (layer_ops.cu).
+cudaError_t launch_gate_param(const Plan& pl, const float* x_beta, const float* x_alpha, const float* x_mu,
+                              const float* x_eta, float* beta, float* log_alpha, float* log_mu, float* eta,
+                              int* launches);
+cudaError_t launch_qk_prep(const Plan& pl, const QkNorm& qk, const void* q, const void* k, void* q_out, void* k_out,
+                           int* launches);
+cudaError_t launch_out_norm_gate(const Plan& pl, const OutPost& post, void* o, int* launches);
 cudaError_t launch_intra_simt(const Plan& pl, const void* q, const void* k, int* launches);
 cudaError_t launch_chain_simt(const Plan& pl, const void* q, const void* k, const void* v,
                               const float* S0, const float* M0, void* o, float* Sf, float* Mf,
