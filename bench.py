@@ -412,7 +412,7 @@ def run_layer_ops(args, w):
     res = {}
     for mode in ("fused", "separate"):
         ops = mdn.make_layer_ops(q, v, gate_param=gp, qk_norm=dict(d=dvec, eps=inp["qk_eps"]),
-                                 out_norm_gate=dict(g=g, w=wn, eps=inp["rms_eps"]), separate_passes=mode == "separate")
+                                 out_norm_gate=dict(g=g, w=wn, eps=inp["rms_eps"]), placement=mode)
         need = int(mdn.lib().mdn_chunk_fwd_fused_workspace_bytes(
             ctypes.byref(mdn.make_params(q, v, scale=inp["scale"], path=args.path)), ctypes.byref(ops)))
         ws = torch.empty(need, dtype=torch.uint8, device="cuda")
@@ -438,7 +438,7 @@ def run_layer_ops(args, w):
         "ms_per_step": res["fused"]["ms_per_step"], "higher_is_better": True, "dtype": w.dtype, "data": "synthetic",
         "config": {"workload": workload_desc(w), "ops": "gate parameterisation + q/k L2Norm(q - d k) + RMSNorm*sigmoid gate"},
         "gpu_launches": res["fused"]["launches_per_step"] * args.steps,
-        "separate_passes": res["separate"], "fused": res["fused"]}))
+        "placement": {"inside the kernels": res["fused"], "separate passes": res["separate"]}}))
 
 
 def main():

@@ -202,11 +202,12 @@ mdn_status mdn_chunk_fwd_static_scratch(const mdn_params* p,
  *    d: device float32[H] or NULL (= 0).  Both use the un-normalised k (the correction comes before the norm).
  *  out_norm_gate != 0: the output written to `o` is  sigmoid(g) * RMSNorm(o) * w  per head, RMSNorm(o) =
  *    o / sqrt(mean_j o_j^2 + rms_eps);  g: device [B,T,H,dv] in the i/o dtype; w: device float32[dv] or NULL (= 1).
- *  separate_passes != 0: run q/k pre-processing, the gate parameterisation and the output step as kernels of
- *    their own before / after the unchanged forward (needs the larger workspace below).  It is what the fused
- *    form is measured against, and the way the fp32 SIMT path always runs qk_norm and out_norm_gate.
+ *  placement: 0 = inside the forward's kernels (below); 1 = all three as kernels of their own before / after the
+ *    unchanged forward (needs the larger workspace below; the normalised q, k are then stored in the i/o dtype).
+ *    1 is what 0 is measured against; the fp32 SIMT path always runs qk_norm and out_norm_gate as passes of
+ *    their own, whatever the value.
  *
- * Fused form (tensor path): the gate formulas run inside the coefficient scan; the norms of k and q - d k come
+ * Inside the kernels (tensor path): the gate formulas run inside the coefficient scan; the norms of k and q - d k come
  * from the diagonals of the K K^T and Q K^T tiles the intra-chunk kernel computes anyway and are applied to
  * fp32 accumulators (q and k are never rewritten or re-rounded); the output step runs in the chain kernel's
  * output epilogue.  All pointers are device pointers; the struct itself is host memory, read during the call.
@@ -225,7 +226,7 @@ typedef struct {
   const void* g;
   const float* w;
   float rms_eps;
-  int32_t separate_passes;
+  int32_t placement;
 } mdn_layer_ops;
 
 /* Workspace bytes of mdn_chunk_fwd_fused for these parameters and operations (0 on invalid ones);
@@ -251,7 +252,7 @@ mdn_status mdn_chunk_fwd_fused(const mdn_params* p, const mdn_layer_ops* ops /* 
  * mdn_coeff_scan (a0 + a1, Eq. 10): for every chunk slot s and head h, twelve float32
  * vectors of length 64 at  coef + ((s*H + h)*MDN_NUM_COEF + i)*64 :
  *   i=0 abar_r   1 b_r   2 alpha_r*b_{r-1}   3 gamma_{last,r}*eta_r   4 (mubar_last/mubar_r)*eta_r
- *   5 mubar_r    6 1/|k_r|   7 1/|q_r - d k_r|   (both 1 unless the fused q/k norm is on; then 3 and 4
+ *   5 mubar_r    6 1/|k_r|   7 1/|q_r - d k_r|   (both 1 unless the fused q/k norm is on; then 2, 3 and 4
  *   also carry the factor 1/|k_r|)   8 alpha_r  9 beta_r   10 mu_r   11 eta_r
  * Positions past the end of a short chunk hold exact no-ops (alpha = mu = 1, beta = eta = 0).
  *

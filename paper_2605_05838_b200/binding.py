@@ -49,7 +49,7 @@ class MdnLayerOps(ctypes.Structure):
                 ("s", ctypes.c_float), ("tau", ctypes.c_float), ("log_mu_min", ctypes.c_float),
                 ("qk_norm", ctypes.c_int32), ("d", ctypes.c_void_p), ("qk_eps", ctypes.c_float),
                 ("out_norm_gate", ctypes.c_int32), ("g", ctypes.c_void_p), ("w", ctypes.c_void_p),
-                ("rms_eps", ctypes.c_float), ("separate_passes", ctypes.c_int32)]
+                ("rms_eps", ctypes.c_float), ("placement", ctypes.c_int32)]
 
 
 class MdnError(RuntimeError):
@@ -187,12 +187,13 @@ def _f32_vec(name, t, n):
     return ctypes.c_void_p(t.data_ptr())
 
 
-def make_layer_ops(q, v, *, gate_param=None, qk_norm=None, out_norm_gate=None, separate_passes=False):
+def make_layer_ops(q, v, *, gate_param=None, qk_norm=None, out_norm_gate=None, placement="fused"):
     """Builds mdn_layer_ops from tensors (marshalling only; keep the tensors alive until the call returns).
       gate_param    = dict(a_alpha, b_alpha, a_mu, b_mu: float32 [H]; s, tau: float; log_mu_min=-1.0): the gate
                       arguments of the call are then the raw projections x_beta, x_alpha, x_mu, x_eta
       qk_norm       = dict(d: float32 [H] or None, eps: float)
-      out_norm_gate = dict(g: [B,T,H,dv] in q's dtype, w: float32 [dv] or None, eps: float)"""
+      out_norm_gate = dict(g: [B,T,H,dv] in q's dtype, w: float32 [dv] or None, eps: float)
+      placement     = "fused" (inside the forward's kernels) or "separate" (kernels of their own)"""
     H, dv = q.shape[2], v.shape[-1]
     ops = MdnLayerOps()
     if gate_param is not None:
@@ -215,7 +216,7 @@ def make_layer_ops(q, v, *, gate_param=None, qk_norm=None, out_norm_gate=None, s
         ops.g = ctypes.c_void_p(g.data_ptr())
         ops.w = _f32_vec("w", out_norm_gate.get("w"), dv)
         ops.rms_eps = float(out_norm_gate["eps"])
-    ops.separate_passes = 1 if separate_passes else 0
+    ops.placement = {"fused": 0, "separate": 1}[placement]
     return ops
 
 

@@ -22,6 +22,11 @@
 // rounding to plain bf16 would dominate the error budget); raw q/k tiles are never rescaled before
 // an MMA - every row/column scaling is applied to fp32 accumulators.
 //
+// Layer operations (template flag kLayer; Section 3.3): with the fused q/k step the accumulators X, Y are scaled by
+// 1 / |k| (folded into the coefficient vectors), EPI-1 leaves -d K S, -d K M in Z, U and MMA-1b runs after MMA-2,
+// accumulating onto them; with the fused output step the staged fp32 tile is re-read row-wise for RMSNorm, weight
+// and sigmoid gate before the TMA store.  kLayer = false is the plain forward, compiled without any of it.
+//
 // Warp roles: 0-3 critical-path epilogue (P, EPI-1, EPI-2); 4-7 output epilogue (EPI-o);
 // 8 TMA producer (2-stage ring: K, Q, V, T, W_hi, W_lo, 6 coefficient vectors per chunk);
 // 9 MMA issuer (one elected lane) and tensor-memory owner.  All hand-offs are mbarriers with
@@ -70,7 +75,6 @@ struct Bars {
   uint64_t mo;        // MMA-3' done                                                   (commit)
   uint64_t zu;        // U (intra-chunk output) has been read                           (256)
   uint64_t ga;        // epilogue group sync                                            (256)
-  uint64_t gfull[2];  // output-gate tile of a stage's chunk landed (fused output step)   (1 + tx bytes)
   uint64_t pn[2];     // fused output step: partial sums of a token half are in shared memory (128 each)
 };
 
@@ -95,8 +99,9 @@ struct ChainArgs {
   // layer operations absorbed by this kernel (Section 3.3)
   int qk_on;                  // q <- L2Norm(q - d k), k <- L2Norm(k): coefficient vectors 6, 7 hold 1/|k|, 1/|q - d k|
   const float* qk_d;          // [H] or NULL
-  int post_on;                // o <- sigmoid(g) * RMSNorm(o) * w; the g tile of a chunk takes its V tile's place
+  int post_on;                // o <- sigmoid(g) * RMSNorm(o) * w in the output epilogue
   const float* post_w;        // [dv] or NULL
+  const void* post_g;         // [B,T,H,dv] bf16
   float post_eps;
   uint32_t drop_lo;           // debug: bit 0 R, 1 V~_S/V~_M, 2 V~ (output), 3 W: leave that operand's lo part out
   long long* timeline;        // debug: CTA 0 writes clock64() at [chunk*32 + event] (NULL = off)
@@ -106,6 +111,13 @@ struct ChainArgs {
 enum Ev : int { kEvMmaStart = 0, kEvM1Seen, kEvRArrive, kEvM2Seen, kEvVArrive, kEvM3Seen, kEvSbArrive, kEvMqSeen,
                 kEvZqArrive, kEvMoSeen, kEvZuArrive, kEvMmaIssued, kEvRSeen, kEvVSeen, kEvTmaIssued, kEvFullSeen,
                 kEvStoresDone, kEvV2Arrive, kEvPrescaled };
+
+// sigmoid(x) = (1 + tanh(x / 2)) / 2 with the one-instruction tanh approximation (relative error ~2^-11)
+__device__ __forceinline__ float sigmoid_fast(float x) {
+  float t;
+  asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(0.5f * x));
+  return fmaf(0.5f, t, 0.5f);
+}
 
 template <typename TO> __device__ __forceinline__ void stage_o(uint8_t* tile, int r, int d, float x);
 template <> __device__ __forceinline__ void stage_o<float>(uint8_t* tile, int r, int d, float x) {
@@ -122,14 +134,13 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
                                                                   const __grid_constant__ CUtensorMap map_v,
                                                                   const __grid_constant__ CUtensorMap map_t,
                                                                   const __grid_constant__ CUtensorMap map_w,
-                                                                  const __grid_constant__ CUtensorMap map_o,
-                                                                  const __grid_constant__ CUtensorMap map_g) {
+                                                                  const __grid_constant__ CUtensorMap map_o) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   __shared__ __align__(8) Bars bars;
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
-  __shared__ float ssq_part[2][4][32];   // fused RMSNorm: per token half, per lane quarter, per token
+  __shared__ __align__(16) float w_sm[kLayer ? kD : 4];   // RMSNorm weight of the fused output step
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int H = a.g.H;
@@ -191,7 +202,6 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
   const uint32_t b_r = smem_u32(&bars.r), b_m2 = smem_u32(&bars.m2), b_zq = smem_u32(&bars.zq);
   const uint32_t b_v1 = smem_u32(&bars.v1), b_v2 = smem_u32(&bars.v2), b_m3 = smem_u32(&bars.m3);
   const uint32_t b_mo = smem_u32(&bars.mo), b_zu = smem_u32(&bars.zu), b_ga = smem_u32(&bars.ga);
-  const uint32_t b_gf0 = smem_u32(&bars.gfull[0]), b_gf1 = smem_u32(&bars.gfull[1]);
   // kLayer = false compiles the layer operations out: the plain forward keeps its instruction count
   const bool qk_on = kLayer && a.qk_on;
   const bool post = kLayer && a.post_on && write_o;
@@ -205,15 +215,14 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
     mbar_init(b_v2, kEpiThreads); mbar_init(b_ga, kEpiThreads); mbar_init(b_zq, kEpiThreads);
     mbar_init(b_zu, kEpiThreads);
     mbar_init(b_m1, 1); mbar_init(b_mq, 1); mbar_init(b_m2, 1); mbar_init(b_m3, 1); mbar_init(b_mo, 1);
-    mbar_init(b_gf0, 1); mbar_init(b_gf1, 1);
     mbar_init(smem_u32(&bars.pn[0]), 128); mbar_init(smem_u32(&bars.pn[1]), 128);
     mbar_fence_init();
   }
+  if (kLayer && tid < kD) w_sm[tid] = (a.post_on && a.post_w) ? __ldg(a.post_w + tid) : 1.f;
   if (warp == kWarpMma) tmem_alloc(smem_u32(&tmem_slot), 512);
   if (warp == kWarpTma && lane == 0) {
     prefetch_tensormap(&map_q); prefetch_tensormap(&map_k); prefetch_tensormap(&map_v);
     prefetch_tensormap(&map_t); prefetch_tensormap(&map_w); prefetch_tensormap(&map_o);
-    if (post) prefetch_tensormap(&map_g);
   }
   tc_fence_before_sync();
   __syncthreads();
@@ -234,7 +243,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
     // ================================================================== TMA producer + output stores
     // Stage s = c & 1 serves chunk c, then (as the staged output tile) is written out and refilled for chunk c + 2.
     if (lane == 0) {
-      int issued = 0, g_issued = 0;
+      int issued = 0;
       for (int c = 0; c < nch + 2; ++c) {
         const int s = c & 1;
         const uint32_t st = s_base + kOffStage + s * kStageBytes;
@@ -243,14 +252,16 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
           MDN_WAIT(s ? b_go1 : b_go0, (co >> 1) & 1);
           const int n = min(C, sq.len - co * C);
           const int tok0 = sq.tok0 + co * C;
+          // the finished tile: at the start of the stage, except the bf16 tile of the fused output step (T / W area)
+          const uint32_t src = st + ((post && sizeof(TO) == 2) ? kStT : 0u);
           if (!write_o) {
             // Psi / Phi runs of the parallel scan produce states only
           } else if (n == C) {
-            tma_store_2d(&map_o, h * kD, tok0, st);
+            tma_store_2d(&map_o, h * kD, tok0, src);
           } else {   // short chunk: rows >= n belong to another sequence; one bulk copy per valid row
             for (int r = 0; r < n; ++r)
               bulk_store(static_cast<uint8_t*>(a.o) + (((size_t)(tok0 + r) * H + h) * kD) * sizeof(TO),
-                         st + r * kD * (uint32_t)sizeof(TO), kD * (uint32_t)sizeof(TO));
+                         src + r * kD * (uint32_t)sizeof(TO), kD * (uint32_t)sizeof(TO));
           }
           tma_store_commit();
           tma_store_wait_read();
@@ -276,22 +287,10 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
           MDN_MARK(c, kEvTmaIssued);
           issued = c + 1;
         }
-        if (post && c >= 1 && c - 1 < nch) {
-          // fused output step: once every epilogue thread has read V of chunk c - 1 (EPI-1 done), its place in the
-          // stage takes that chunk's output-gate tile, well ahead of the chunk's output epilogue
-          const int cg = c - 1;
-          MDN_WAIT(b_r, cg & 1);
-          const uint32_t gb = (cg & 1) ? b_gf1 : b_gf0;
-          mbar_arrive_expect_tx(gb, kTxV);
-          tma_load_2d(s_base + kOffStage + (cg & 1) * kStageBytes + kStV, &map_g, h * kD, sq.tok0 + cg * C, gb);
-          g_issued = cg + 1;
-        }
       }
       if (!ok) {   // giving up: let the copies already in flight land before the CTA exits
         for (int c = max(0, issued - 2); c < issued; ++c)
           for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait((c & 1) ? b_full1 : b_full0, (c >> 1) & 1); ++it) {}
-        for (int c = max(0, g_issued - 2); c < g_issued; ++c)
-          for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait((c & 1) ? b_gf1 : b_gf0, (c >> 1) & 1); ++it) {}
       }
       tma_store_wait_all();
     }
@@ -325,17 +324,32 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
         for (int k = 0; k < 8; ++k)
           umma_ss(tmem + kColY, ((k >> 2) ? dMb1 : dMb0) + 2 * (k & 3), ((k >> 2) ? dK1 : dK0) + 2 * (k & 3), id64, k > 0);
         umma_commit(b_m1);
-        // ---- MMA-1b: Z = S_b Q^T, U = M_b Q^T (U of the previous chunk must have been read)
-        if (write_o) {
-          MDN_WAIT(b_zu, ph ^ 1);
-          tc_fence_after_sync();
+        // ---- MMA-1b: Z = S_b Q^T, U = M_b Q^T (U of the previous chunk must have been read).  With the fused q/k
+        // step it runs after MMA-2 instead and ACCUMULATES onto -d K S, -d K M, which EPI-1 has put into Z, U.
+#define MDN_MMA_1B(onto)                                                                                                  \
+  {                                                                                                                        \
+    MDN_WAIT(b_zu, ph ^ 1);                                                                                                \
+    tc_fence_after_sync();                                                                                                 \
+    _Pragma("unroll") for (int k = 0; k < 8; ++k)                                                                          \
+        umma_ss(tmem + kColZ, ((k >> 2) ? dSb1 : dSb0) + 2 * (k & 3), ((k >> 2) ? dQ1 : dQ0) + 2 * (k & 3), id64, (onto) || k > 0); \
+    _Pragma("unroll") for (int k = 0; k < 8; ++k)                                                                          \
+        umma_ss(tmem + kColU, ((k >> 2) ? dMb1 : dMb0) + 2 * (k & 3), ((k >> 2) ? dQ1 : dQ0) + 2 * (k & 3), id64, (onto) || k > 0); \
+    umma_commit(b_mq);                                                                                                     \
+  }
+        if constexpr (!kLayer) {
+          if (write_o) {
+            MDN_WAIT(b_zu, ph ^ 1);
+            tc_fence_after_sync();
 #pragma unroll
-          for (int k = 0; k < 8; ++k)
-            umma_ss(tmem + kColZ, ((k >> 2) ? dSb1 : dSb0) + 2 * (k & 3), ((k >> 2) ? dQ1 : dQ0) + 2 * (k & 3), id64, k > 0);
+            for (int k = 0; k < 8; ++k)
+              umma_ss(tmem + kColZ, ((k >> 2) ? dSb1 : dSb0) + 2 * (k & 3), ((k >> 2) ? dQ1 : dQ0) + 2 * (k & 3), id64, k > 0);
 #pragma unroll
-          for (int k = 0; k < 8; ++k)
-            umma_ss(tmem + kColU, ((k >> 2) ? dMb1 : dMb0) + 2 * (k & 3), ((k >> 2) ? dQ1 : dQ0) + 2 * (k & 3), id64, k > 0);
-          umma_commit(b_mq);
+            for (int k = 0; k < 8; ++k)
+              umma_ss(tmem + kColU, ((k >> 2) ? dMb1 : dMb0) + 2 * (k & 3), ((k >> 2) ? dQ1 : dQ0) + 2 * (k & 3), id64, k > 0);
+            umma_commit(b_mq);
+          }
+        } else {
+          if (write_o && !qk_on) MDN_MMA_1B(false);
         }
         // ---- MMA-2: Y = (R_hi + R_lo)^T T^T
         MDN_WAIT(b_r, ph);
@@ -348,6 +362,9 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
           for (int k = 0; k < 4; ++k) umma_ts(tmem + kColY, tmem + kColX + 32 + k * 8, dT + 2 * k, id64, true);
         }
         umma_commit(b_m2);
+        if constexpr (kLayer) {
+          if (write_o && qk_on) MDN_MMA_1B(true);
+        }
         // ---- MMA-3: S^T += V~_S^T K, M^T -= V~_M^T K   (K tile read MN-major: N = dk, K = tokens)
         MDN_WAIT(b_v1, ph);
         tc_fence_after_sync();
@@ -387,6 +404,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
     uint32_t ga_phase = 0, pn_phase = 0;
     const uint32_t b_pn = smem_u32(&bars.pn[hf]);
     float oi[32];   // scale (abar .* Q S - b .* Q M) for this thread's tokens, carried to the output step
+
 #pragma unroll
     for (int j = 0; j < 32; ++j) oi[j] = 0.f;
     for (int c = 0; c <= nch; ++c) {
@@ -469,6 +487,14 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
       } else if (c > 0) {
         const int cp = c - 1;
         uint8_t* stp = smem + kOffStage + (cp & 1) * kStageBytes;
+        // fused output step: this thread's share of the chunk's output-gate rows is four threads per token, 8-byte
+        // pieces (each warp-load covers eight full 32-byte sectors); the rows are pulled towards L2 here and read
+        // once the tile is staged, when registers are free again
+        const int t128 = q4 * 32 + lane, prow = r0 + (t128 >> 2), part = t128 & 3;
+        const bool g_live = post && cp * C + prow < sq.len;
+        const uint2* gp = reinterpret_cast<const uint2*>(static_cast<const __nv_bfloat16*>(a.post_g) +
+                                                         ((size_t)(sq.tok0 + cp * C + prow) * H + h) * kD) + part;
+        if (g_live && part < 2) asm volatile("prefetch.global.L2 [%0];" ::"l"(gp + 15 * part));   // bytes 0 and 128 of the row
         MDN_WAIT(b_mo, cp & 1);
         __syncwarp();
         tc_fence_after_sync();
@@ -484,40 +510,46 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
 #pragma unroll
             for (int j = 0; j < 32; ++j) stage_o<TO>(stp, r0 + j, d, oi[j] + __uint_as_float(u[j]));
           } else {
-            // fused output step: y = sigmoid(g) * o / sqrt(mean_d o^2 + eps) * w_d.  The sum over the value
-            // dimension runs over the 32 lanes (transposing butterfly: lane l ends with token l's partial sum)
-            // and then over the four warps of this token half through shared memory.
-            float val[32], sqv[32];
+            // fused output step: y = sigmoid(g) * o / sqrt(mean_d o^2 + eps) * w_d.  The fp32 tile is staged first
+            // (value columns across lanes), then re-read row-wise: four threads per token sum its 128 squares,
+            // rescale, gate and write the final tile (in place for fp32 output, into the T / W area for bf16).
+            float* tile = reinterpret_cast<float*>(stp);
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-              val[j] = oi[j] + __uint_as_float(u[j]);
-              sqv[j] = val[j] * val[j];
-            }
+            for (int j = 0; j < 32; ++j) tile[(r0 + j) * kD + d] = oi[j] + __uint_as_float(u[j]);
+            uint2 graw[8];
 #pragma unroll
-            for (int off = 16; off >= 1; off >>= 1) {
-              const bool up = (lane & off) != 0;
-#pragma unroll
-              for (int i = 0; i < off; ++i) {
-                const float keep = up ? sqv[i + off] : sqv[i];
-                const float send = up ? sqv[i] : sqv[i + off];
-                sqv[i] = keep + __shfl_xor_sync(0xffffffffu, send, off);
-              }
-            }
-            ssq_part[hf][q4][lane] = sqv[0];
+            for (int i = 0; i < 8; ++i) graw[i] = g_live ? __ldg(gp + 4 * i) : make_uint2(0u, 0u);
             mbar_arrive(b_pn);
             MDN_WAIT(b_pn, pn_phase);
             pn_phase ^= 1;
             __syncwarp();
-            const float tot = ssq_part[hf][0][lane] + ssq_part[hf][1][lane] + ssq_part[hf][2][lane] + ssq_part[hf][3][lane];
-            const float rstd = 1.f / sqrtf(tot * (1.f / kD) + a.post_eps);
-            const float wd = a.post_w ? __ldg(a.post_w + d) : 1.f;
-            MDN_WAIT((cp & 1) ? b_gf1 : b_gf0, (cp >> 1) & 1);
-            const __nv_bfloat16* sG = reinterpret_cast<const __nv_bfloat16*>(stp + kStV);
+            const int row = prow;
+            float4 ov[8];
+            float ss = 0.f;
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-              const float gj = __bfloat162float(sG[(r0 + j) * kD + d]);
-              const float gate = __fdividef(1.f, 1.f + __expf(-gj));
-              stage_o<TO>(stp, r0 + j, d, val[j] * __shfl_sync(0xffffffffu, rstd, j) * wd * gate);
+            for (int i = 0; i < 8; ++i) {   // interleaved 16-byte pieces: the four threads of a row cover 64 B at a time
+              ov[i] = *reinterpret_cast<const float4*>(tile + row * kD + (part + 4 * i) * 4);
+              ss = fmaf(ov[i].x, ov[i].x, fmaf(ov[i].y, ov[i].y, fmaf(ov[i].z, ov[i].z, fmaf(ov[i].w, ov[i].w, ss))));
+            }
+            ss += __shfl_xor_sync(0xffffffffu, ss, 1);
+            ss += __shfl_xor_sync(0xffffffffu, ss, 2);
+            const float rstd = rsqrtf(ss * (1.f / kD) + a.post_eps);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const int col = (part + 4 * i) * 4;
+              const float4 wv = *reinterpret_cast<const float4*>(w_sm + col);
+              const uint2 gr = graw[i];
+              const float g0 = __uint_as_float(gr.x << 16), g1 = __uint_as_float(gr.x & 0xffff0000u);
+              const float g2 = __uint_as_float(gr.y << 16), g3 = __uint_as_float(gr.y & 0xffff0000u);
+              const float y0 = ov[i].x * rstd * wv.x * sigmoid_fast(g0), y1 = ov[i].y * rstd * wv.y * sigmoid_fast(g1);
+              const float y2 = ov[i].z * rstd * wv.z * sigmoid_fast(g2), y3 = ov[i].w * rstd * wv.w * sigmoid_fast(g3);
+              if (sizeof(TO) == 4) {
+                *reinterpret_cast<float4*>(tile + row * kD + col) = make_float4(y0, y1, y2, y3);
+              } else {
+                uint2 pk;
+                pk.x = pack_bf16(y0, y1); pk.y = pack_bf16(y2, y3);
+                *reinterpret_cast<uint2*>(stp + kStT + (row * kD + col) * 2) = pk;
+              }
             }
           }
         }
@@ -553,22 +585,23 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
             const float4 pb = *reinterpret_cast<const float4*>(cf + kAlphaBPrev * C + r0 + j);
             float e0, e1, e2, e3;
             if (qk_on) {
-              // k' = k / |k|: X, Y are products with the raw k tile, so the norm scales the accumulators; the
-              // output correction q - d k turns Q S - d K S, Q M - d K M: its K terms are taken from X, Y here
+              // k' = k / |k|: X, Y are products with the raw k tile, so the norm scales the accumulators (vector 2
+              // already carries the factor); the output correction q - d k turns Q S into Q S - d K S (same for M):
+              // its K terms are X, Y themselves, handed to the tensor core as the start value of Z, U
               const float4 rk = *reinterpret_cast<const float4*>(cf + kRk * C + r0 + j);
-              const float4 bb = *reinterpret_cast<const float4*>(cf + kB * C + r0 + j);
               const float x0 = __uint_as_float(x[j + 0]), x1 = __uint_as_float(x[j + 1]);
               const float x2 = __uint_as_float(x[j + 2]), x3 = __uint_as_float(x[j + 3]);
               const float y0 = __uint_as_float(y[j + 0]), y1 = __uint_as_float(y[j + 1]);
               const float y2 = __uint_as_float(y[j + 2]), y3 = __uint_as_float(y[j + 3]);
-              e0 = vv[j + 0] - rk.x * (ab.x * x0 - pb.x * y0);
-              e1 = vv[j + 1] - rk.y * (ab.y * x1 - pb.y * y1);
-              e2 = vv[j + 2] - rk.z * (ab.z * x2 - pb.z * y2);
-              e3 = vv[j + 3] - rk.w * (ab.w * x3 - pb.w * y3);
-              oi[j + 0] = -dh * (ab.x * x0 - bb.x * y0);
-              oi[j + 1] = -dh * (ab.y * x1 - bb.y * y1);
-              oi[j + 2] = -dh * (ab.z * x2 - bb.z * y2);
-              oi[j + 3] = -dh * (ab.w * x3 - bb.w * y3);
+              e0 = vv[j + 0] - (rk.x * ab.x) * x0 + pb.x * y0;
+              e1 = vv[j + 1] - (rk.y * ab.y) * x1 + pb.y * y1;
+              e2 = vv[j + 2] - (rk.z * ab.z) * x2 + pb.z * y2;
+              e3 = vv[j + 3] - (rk.w * ab.w) * x3 + pb.w * y3;
+              // -d K S, -d K M: MMA-1b will accumulate Q S, Q M onto them
+              x[j + 0] = __float_as_uint(-dh * x0); x[j + 1] = __float_as_uint(-dh * x1);
+              x[j + 2] = __float_as_uint(-dh * x2); x[j + 3] = __float_as_uint(-dh * x3);
+              y[j + 0] = __float_as_uint(-dh * y0); y[j + 1] = __float_as_uint(-dh * y1);
+              y[j + 2] = __float_as_uint(-dh * y2); y[j + 3] = __float_as_uint(-dh * y3);
             } else {
               e0 = vv[j + 0] - ab.x * __uint_as_float(x[j + 0]) + pb.x * __uint_as_float(y[j + 0]);
               e1 = vv[j + 1] - ab.y * __uint_as_float(x[j + 1]) + pb.y * __uint_as_float(y[j + 1]);
@@ -577,6 +610,10 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
             }
             split_pack_bf16(e0, e1, hi[j >> 1], lo[j >> 1]);
             split_pack_bf16(e2, e3, hi[(j >> 1) + 1], lo[(j >> 1) + 1]);
+          }
+          if (qk_on && write_o) {   // own lanes only; MMA-3' of the previous chunk and this thread's read of U are done
+            tmem_st32(tl + kColZ + r0, x);
+            tmem_st32(tl + kColU + r0, y);
           }
         }
         // the other half's warps may still be reading X: group sync before overwriting it
@@ -593,36 +630,61 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
       tc_fence_before_sync();
       mbar_arrive(b_r);
       MDN_MARK(c, kEvRArrive);
-      // ---------------- inter-chunk output terms (under MMA-2): oi = scale (abar .* Q S - b .* Q M)
-      if (write_o) {
-        MDN_WAIT(b_mq, ph);
-        __syncwarp();
-        tc_fence_after_sync();
-        MDN_MARK(c, kEvMqSeen);
-        uint32_t z[32], u[32];
-        tmem_ld32(tl + kColZ + r0, z);
-        tmem_ld32(tl + kColU + r0, u);
-        tmem_wait_ld();
-        tc_fence_before_sync();
-        mbar_arrive(b_zq);
-        MDN_MARK(c, kEvZqArrive);
+      // ---------------- inter-chunk output terms: oi = scale (abar .* Q S - b .* Q M), under MMA-2; with the fused
+      // q/k step Z, U arrive later (MMA-1b follows MMA-2) and already hold Q S - d K S, Q M - d K M: then this
+      // step runs under MMA-3 instead
+#define MDN_INTER_CHUNK_TERMS()                                                                              \
+  {                                                                                                          \
+    MDN_WAIT(b_mq, ph);                                                                                      \
+    __syncwarp();                                                                                            \
+    tc_fence_after_sync();                                                                                   \
+    MDN_MARK(c, kEvMqSeen);                                                                                  \
+    uint32_t z[32], u[32];                                                                                   \
+    tmem_ld32(tl + kColZ + r0, z);                                                                           \
+    tmem_ld32(tl + kColU + r0, u);                                                                           \
+    tmem_wait_ld();                                                                                          \
+    tc_fence_before_sync();                                                                                  \
+    mbar_arrive(b_zq);                                                                                       \
+    MDN_MARK(c, kEvZqArrive);                                                                                \
+    _Pragma("unroll") for (int j = 0; j < 32; j += 4) {                                                      \
+      const float4 ab = *reinterpret_cast<const float4*>(cf + kAbar * C + r0 + j);                           \
+      const float4 bb = *reinterpret_cast<const float4*>(cf + kB * C + r0 + j);                              \
+      float4 sc = make_float4(a.scale, a.scale, a.scale, a.scale);                                           \
+      if (qk_on) { /* q' = (q - d k) / |q - d k| */                                                          \
+        const float4 rq = *reinterpret_cast<const float4*>(cf + kRq * C + r0 + j);                           \
+        sc.x *= rq.x; sc.y *= rq.y; sc.z *= rq.z; sc.w *= rq.w;                                              \
+      }                                                                                                      \
+      oi[j + 0] = sc.x * (ab.x * __uint_as_float(z[j + 0]) - bb.x * __uint_as_float(u[j + 0]));              \
+      oi[j + 1] = sc.y * (ab.y * __uint_as_float(z[j + 1]) - bb.y * __uint_as_float(u[j + 1]));              \
+      oi[j + 2] = sc.z * (ab.z * __uint_as_float(z[j + 2]) - bb.z * __uint_as_float(u[j + 2]));              \
+      oi[j + 3] = sc.w * (ab.w * __uint_as_float(z[j + 3]) - bb.w * __uint_as_float(u[j + 3]));              \
+    }                                                                                                        \
+  }
+      if constexpr (!kLayer) {
+        if (write_o) {
+          MDN_WAIT(b_mq, ph);
+          __syncwarp();
+          tc_fence_after_sync();
+          MDN_MARK(c, kEvMqSeen);
+          uint32_t z[32], u[32];
+          tmem_ld32(tl + kColZ + r0, z);
+          tmem_ld32(tl + kColU + r0, u);
+          tmem_wait_ld();
+          tc_fence_before_sync();
+          mbar_arrive(b_zq);
+          MDN_MARK(c, kEvZqArrive);
 #pragma unroll
-        for (int j = 0; j < 32; j += 4) {
-          const float4 ab = *reinterpret_cast<const float4*>(cf + kAbar * C + r0 + j);
-          const float4 bb = *reinterpret_cast<const float4*>(cf + kB * C + r0 + j);
-          if (qk_on) {   // q' = (q - d k) / |q - d k|: the K terms are already in oi
-            const float4 rq = *reinterpret_cast<const float4*>(cf + kRq * C + r0 + j);
-            oi[j + 0] = a.scale * rq.x * (oi[j + 0] + ab.x * __uint_as_float(z[j + 0]) - bb.x * __uint_as_float(u[j + 0]));
-            oi[j + 1] = a.scale * rq.y * (oi[j + 1] + ab.y * __uint_as_float(z[j + 1]) - bb.y * __uint_as_float(u[j + 1]));
-            oi[j + 2] = a.scale * rq.z * (oi[j + 2] + ab.z * __uint_as_float(z[j + 2]) - bb.z * __uint_as_float(u[j + 2]));
-            oi[j + 3] = a.scale * rq.w * (oi[j + 3] + ab.w * __uint_as_float(z[j + 3]) - bb.w * __uint_as_float(u[j + 3]));
-          } else {
+          for (int j = 0; j < 32; j += 4) {
+            const float4 ab = *reinterpret_cast<const float4*>(cf + kAbar * C + r0 + j);
+            const float4 bb = *reinterpret_cast<const float4*>(cf + kB * C + r0 + j);
             oi[j + 0] = a.scale * (ab.x * __uint_as_float(z[j + 0]) - bb.x * __uint_as_float(u[j + 0]));
             oi[j + 1] = a.scale * (ab.y * __uint_as_float(z[j + 1]) - bb.y * __uint_as_float(u[j + 1]));
             oi[j + 2] = a.scale * (ab.z * __uint_as_float(z[j + 2]) - bb.z * __uint_as_float(u[j + 2]));
             oi[j + 3] = a.scale * (ab.w * __uint_as_float(z[j + 3]) - bb.w * __uint_as_float(u[j + 3]));
           }
         }
+      } else {
+        if (write_o && !qk_on) MDN_INTER_CHUNK_TERMS();
       }
       // ---------------- EPI-2: V~ -> (gamma_C eta) V~, ((mubar_C/mubar) eta) V~ [part a], V~ [part b]; bf16 hi, lo
       MDN_WAIT(b_m2, ph);
@@ -668,6 +730,9 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
         tc_fence_before_sync();
         mbar_arrive(b_v1);
         MDN_MARK(c, kEvVArrive);
+        if constexpr (kLayer) {
+          if (write_o && qk_on) MDN_INTER_CHUNK_TERMS();
+        }
         // part b (under MMA-3): V~ itself for the intra-chunk output, into Z once every warp has read Q S
         if (write_o) {
           uint32_t vh[16], vl[16];
@@ -686,6 +751,8 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
       }
     }
   }
+#undef MDN_INTER_CHUNK_TERMS
+#undef MDN_MMA_1B
 #undef MDN_WAIT
 #undef MDN_MARK
 
@@ -710,7 +777,7 @@ cudaError_t launch_chain_tensor(const Plan& pl, const void* q, const void* k, co
   const mdn_params& p = pl.p;
   const uint64_t tokens = (uint64_t)p.B * p.T;
   const uint64_t mats = (uint64_t)pl.geom.num_slots * p.H;
-  CUtensorMap mq, mk, mv, mt, mw, mo, mg;
+  CUtensorMap mq, mk, mv, mt, mw, mo;
   const uint64_t row = (uint64_t)p.H * kD;
   if (!encode_tma_2d_bf16(&mq, TmaMap2D{q, row, tokens, row * 2, 64, 64, true}) ||
       !encode_tma_2d_bf16(&mk, TmaMap2D{k, row, tokens, row * 2, 64, 64, true}) ||
@@ -721,12 +788,9 @@ cudaError_t launch_chain_tensor(const Plan& pl, const void* q, const void* k, co
   const bool o_bf16 = p.o_dtype == MDN_BF16;
   if (!encode_tma_2d(&mo, TmaMap2D{o, row, tokens, row * (o_bf16 ? 2u : 4u), 128, 64, false}, !o_bf16))
     return cudaErrorInvalidValue;
-  // the output-gate tensor has V's shape and dtype; without the fused output step the map is never used
-  if (!encode_tma_2d_bf16(&mg, TmaMap2D{pl.post.on ? pl.post.g : v, row, tokens, row * 2, 128, 64, false}))
-    return cudaErrorInvalidValue;
   ChainArgs a;
   a.qk_on = pl.qk.on; a.qk_d = pl.qk.d;
-  a.post_on = pl.post.on; a.post_w = pl.post.w; a.post_eps = pl.post.eps;
+  a.post_on = pl.post.on; a.post_w = pl.post.w; a.post_g = pl.post.g; a.post_eps = pl.post.eps;
   a.g = pl.geom;
   a.coef = reinterpret_cast<const float*>(pl.ws + pl.lay.off_coef);
   a.S0 = S0; a.M0 = M0; a.o = o; a.Sf = Sf; a.Mf = Mf;
@@ -744,7 +808,7 @@ cudaError_t launch_chain_tensor(const Plan& pl, const void* q, const void* k, co
   auto launch_as = [&](auto kern, unsigned grid) -> cudaError_t {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
     if (e != cudaSuccess) return e;
-    e = launch_pdl(kern, dim3(grid), dim3(kThreads), kSmemBytes, pl.stream, a, mq, mk, mv, mt, mw, mo, mg);
+    e = launch_pdl(kern, dim3(grid), dim3(kThreads), kSmemBytes, pl.stream, a, mq, mk, mv, mt, mw, mo);
     if (e == cudaSuccess) e = cudaGetLastError();
     if (e == cudaSuccess) ++*launches;
     return e;

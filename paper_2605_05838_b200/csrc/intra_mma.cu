@@ -29,7 +29,7 @@ constexpr int LM = C + 4;     // fp32 elements per row of the 64x64 matrices (16
 constexpr uint32_t kOffK = 0, kOffQ = 16384;                 // bf16 tiles, two [64 x 128 B] swizzled blocks each
 constexpr uint32_t kOffG = 32768;                            // Gamma [64][68] fp32; later T
 constexpr uint32_t kOffCv = kOffG + C * LM * 4;              // alpha, beta, mu, eta, then the q/k-norm vectors
-constexpr int kCvVecs = 11;                                  // + gamma_C eta, (mubar_C/mubar) eta, 1/|k|, 1/|q - dk|, |q|^2, q.k, |k|^2
+constexpr int kCvVecs = 12;                                  // + gamma_C eta, (mubar_C/mubar) eta, 1/|k|, 1/|q - dk|, |q|^2, q.k, |k|^2
 // the tile area is reused once the MMAs are done: first as the bf16 staging of W_hi / W_lo, then for A and scratch
 constexpr int LW = C + 8;                                    // bf16 elements per staged W row (144 B: conflict-free)
 constexpr uint32_t kOffWh = 0, kOffWl = C * LW * 2;          // W_hi, W_lo staging [64][72] bf16
@@ -133,7 +133,10 @@ __global__ void __launch_bounds__(kThreads) intra_mma_kernel(ChunkGeom g, const 
   if (gates.log_alpha == nullptr) {
     for (int idx = tid; idx < 4 * C; idx += kThreads) cv[idx] = cf[kAlpha * C + idx];
     if (qkn.on)
-      for (int idx = tid; idx < 2 * C; idx += kThreads) cv[4 * C + idx] = cf[kGS * C + idx];   // gamma_C eta, (mubar_C/mubar) eta
+      for (int idx = tid; idx < 2 * C; idx += kThreads) {   // gamma_C eta, (mubar_C/mubar) eta; alpha b^-
+        cv[4 * C + idx] = cf[kGS * C + idx];
+        if (idx < C) cv[11 * C + idx] = cf[kAlphaBPrev * C + idx];
+      }
     __syncthreads();   // coefficients in smem; barrier initialised before anyone waits on it
   } else {
     // fused coefficient scan (Eq. 10): this head's gates (stride H floats), then one warp runs the scans,
@@ -166,6 +169,7 @@ __global__ void __launch_bounds__(kThreads) intra_mma_kernel(ChunkGeom g, const 
       if (qkn.on) {   // the last-row weights get their 1/|k| factor once the norms are known
         reinterpret_cast<float2*>(cv + 4 * C)[lane] = make_float2(hc.gs[0], hc.gs[1]);
         reinterpret_cast<float2*>(cv + 5 * C)[lane] = make_float2(hc.gm[0], hc.gm[1]);
+        reinterpret_cast<float2*>(cv + 11 * C)[lane] = make_float2(hc.ab_prev[0], hc.ab_prev[1]);
       } else {
         put(kRk, 1.f, 1.f);
         put(kRq, 1.f, 1.f);
@@ -275,6 +279,7 @@ __global__ void __launch_bounds__(kThreads) intra_mma_kernel(ChunkGeom g, const 
       cv[7 * C + tid] = rq;
       cf[kGS * C + tid] = cv[4 * C + tid] * rk;
       cf[kGM * C + tid] = cv[5 * C + tid] * rk;
+      cf[kAlphaBPrev * C + tid] = cv[11 * C + tid] * rk;
       cf[kRk * C + tid] = rk;
       cf[kRq * C + tid] = rq;
     }

@@ -202,6 +202,7 @@ static mdn_status check_ops(const mdn_layer_ops& f) {
   }
   if (f.qk_norm && !(f.qk_eps > 0.f)) return MDN_ERR_INVALID_ARG;
   if (f.out_norm_gate && (!f.g || !aligned(f.g, 16) || !(f.rms_eps >= 0.f))) return MDN_ERR_INVALID_ARG;
+  if (f.placement < 0 || f.placement > 1) return MDN_ERR_INVALID_ARG;
   return MDN_OK;
 }
 
@@ -210,9 +211,11 @@ struct SepLayout { uint64_t q, k, gates[4], total; bool qk_sep, out_sep, gate_se
 
 static mdn_status sep_layout(const mdn_params& p, const mdn_layer_ops& f, const mdn_ws_layout& lay, SepLayout* sl) {
   const bool simt = resolve_path(p) != MDN_PATH_TENSOR;
-  sl->qk_sep = f.qk_norm && (f.separate_passes || simt);
-  sl->out_sep = f.out_norm_gate && (f.separate_passes || simt);
-  sl->gate_sep = f.raw_gates && f.separate_passes;
+  // placement 0: inside the kernels wherever the path can (tensor path: all three; SIMT path: the gate formulas);
+  // 1: all as passes of their own
+  sl->qk_sep = f.qk_norm && (f.placement == 1 || simt);
+  sl->out_sep = f.out_norm_gate && (f.placement == 1 || simt);
+  sl->gate_sep = f.raw_gates && f.placement == 1;
   const uint64_t tokens = (uint64_t)p.B * p.T, es = p.io_dtype == MDN_BF16 ? 2 : 4;
   uint64_t off = lay.total_bytes;
   auto take = [&](uint64_t bytes) { uint64_t at = off; off = align_up(off + bytes, 256); return at; };

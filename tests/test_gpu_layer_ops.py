@@ -61,7 +61,7 @@ def oracle_layer(inp, which, chains=None, round_qk=False):
     return o, S, M
 
 
-def run_fused(mdn, inp, which, *, path="auto", separate=False, o_dtype=None, segments=0):
+def run_fused(mdn, inp, which, *, path="auto", placement="fused", o_dtype=None, segments=0):
     import torch
     w = inp["workload"]
     dt = torch.bfloat16 if w.dtype == "bf16" else torch.float32
@@ -76,7 +76,7 @@ def run_fused(mdn, inp, which, *, path="auto", separate=False, o_dtype=None, seg
         gp = None
     qk = dict(d=dev(inp["d"]), eps=inp["qk_eps"]) if "qk" in which else None
     out = dict(g=dev(inp["g"], dt), w=dev(inp["w_norm"]), eps=inp["rms_eps"]) if "out" in which else None
-    ops = mdn.make_layer_ops(q, v, gate_param=gp, qk_norm=qk, out_norm_gate=out, separate_passes=separate)
+    ops = mdn.make_layer_ops(q, v, gate_param=gp, qk_norm=qk, out_norm_gate=out, placement=placement)
     cu = None if inp["cu_seqlens"] is None else torch.from_numpy(inp["cu_seqlens"]).to("cuda")
     o, S, M = mdn.chunk_fwd(q, k, v, *gates, initial_S=dev(inp["S0"]), initial_M=dev(inp["M0"]), cu_seqlens=cu,
                             scale=inp["scale"], path=path, o_dtype=o_dtype, layer_ops=ops, segments=segments)
@@ -128,17 +128,17 @@ def tensor_ok(mdn, w):
 
 
 @pytest.mark.parametrize("which", [("gates",), ("qk",), ("out",), ALL])
-@pytest.mark.parametrize("separate", [False, True])
-def test_tensor_path_each_operation_and_all(mdn, which, separate):
+@pytest.mark.parametrize("placement", ["fused", "separate"])
+def test_tensor_path_each_operation_and_all(mdn, which, placement):
     import torch
     w = wl.Workload("layer_bf16", B=2, T=300, H=3, dk=128, dv=128, dtype="bf16", init_state_std=0.05, seed=52)
     if not tensor_ok(mdn, w):
         pytest.skip("tensor path not built")
     inp = compose(w, which)
-    ref = oracle_layer(inp, which, round_qk=separate)
-    got = run_fused(mdn, inp, which, path="tensor", separate=separate, o_dtype=torch.float32)
+    ref = oracle_layer(inp, which, round_qk=placement == "separate")
+    got = run_fused(mdn, inp, which, path="tensor", placement=placement, o_dtype=torch.float32)
     errs = errs3(got, ref)
-    print("bf16 %s %s: o %.3e S %.3e M %.3e" % ("+".join(which), "separate" if separate else "fused", *errs))
+    print("bf16 %s %s: o %.3e S %.3e M %.3e" % ("+".join(which), placement, *errs))
     assert max(errs) <= TOL_BF16
 
 
