@@ -245,6 +245,32 @@ mdn_status mdn_chunk_fwd_fused(const mdn_params* p, const mdn_layer_ops* ops /* 
                                void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * Backward of mdn_chunk_fwd (Section 3.1: the training pass differentiates the same recurrence; like the paper's
+ * kernels this keeps no per-token states and rebuilds them from per-chunk checkpoints):
+ * given d_o = dL/do ([B,T,H,dv], o_dtype) and optionally dL/d(final_S), dL/d(final_M) ([N,H,dk,dv] float32, NULL =
+ * zero), writes the float32 gradients
+ *     dq, dk [B,T,H,dk];  dv [B,T,H,dv];  dbeta, dlog_alpha, dlog_mu, deta [B,T,H] (deta may be NULL);
+ *     d_initial_S, d_initial_M [N,H,dk,dv] (either may be NULL).
+ * q, k, v, the gates, the initial states, cu_seqlens, p: exactly the forward call's.  The pass recomputes the
+ * forward itself, token by token in float32 (any dk, dv in {64, 128}; p->path and p->segments are ignored), so it
+ * does not need the forward's outputs.  Workspace: mdn_chunk_bwd_workspace_bytes(p) bytes, 256-byte aligned,
+ * scratch.  Same ownership, stream and error rules as mdn_chunk_fwd; the partial sums over value-column blocks are
+ * added in a fixed order, so results are reproducible run to run.
+ */
+size_t mdn_chunk_bwd_workspace_bytes(const mdn_params* p);
+
+mdn_status mdn_chunk_bwd(const mdn_params* p,
+                         const void* q, const void* k, const void* v,
+                         const float* beta, const float* log_alpha, const float* log_mu, const float* eta,
+                         const float* initial_S, const float* initial_M,
+                         const int32_t* cu_seqlens,
+                         const void* d_o, const float* d_final_S, const float* d_final_M,
+                         float* dq, float* dk, float* dv,
+                         float* dbeta, float* dlog_alpha, float* dlog_mu, float* deta,
+                         float* d_initial_S, float* d_initial_M,
+                         void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * Stage entry points (the same kernels mdn_chunk_fwd launches, exposed so that each
  * stage can be checked on its own).  Both write into `workspace` using the layout
  * mdn_workspace_layout describes; mdn_intra_chunk expects mdn_coeff_scan's output there.

@@ -82,6 +82,10 @@ def lib() -> ctypes.CDLL:
         L.mdn_chunk_fwd_fused.argtypes = [P, ctypes.POINTER(MdnLayerOps)] + [vp] * 13 + [vp, ctypes.c_size_t, vp]
         L.mdn_chunk_fwd_fused_workspace_bytes.restype = ctypes.c_size_t
         L.mdn_chunk_fwd_fused_workspace_bytes.argtypes = [P, ctypes.POINTER(MdnLayerOps)]
+        L.mdn_chunk_bwd.restype = ctypes.c_int
+        L.mdn_chunk_bwd.argtypes = [P] + [vp] * 22 + [vp, ctypes.c_size_t, vp]
+        L.mdn_chunk_bwd_workspace_bytes.restype = ctypes.c_size_t
+        L.mdn_chunk_bwd_workspace_bytes.argtypes = [P]
         L.mdn_chunk_fwd_host.restype = ctypes.c_int
         L.mdn_chunk_fwd_host.argtypes = [P] + [vp] * 13 + [vp, ctypes.c_size_t, vp]
         L.mdn_chunk_fwd_static_scratch.restype = ctypes.c_int
@@ -286,6 +290,46 @@ def chunk_fwd(q, k, v, beta, log_alpha, log_mu, eta=None, *, initial_S=None, ini
     if st != 0:
         raise MdnError(st, "mdn_chunk_fwd_fused" if layer_ops is not None else "mdn_chunk_fwd")
     return o, Sf, Mf
+
+
+def chunk_bwd(q, k, v, beta, log_alpha, log_mu, eta, d_o, *, initial_S=None, initial_M=None, cu_seqlens=None,
+              d_final_S=None, d_final_M=None, scale: Optional[float] = None, workspace: Optional[torch.Tensor] = None):
+    """mdn_chunk_bwd on CUDA tensors (current stream): gradients of mdn_chunk_fwd's outputs' loss.
+    d_o: [B,T,H,dv] (its dtype is taken as the forward's o_dtype).  Returns a dict of float32 tensors
+    dq, dk, dv, dbeta, dlog_alpha, dlog_mu, deta (None when eta is None), d_initial_S, d_initial_M."""
+    _check_inputs(q, k, v, (("beta", beta), ("log_alpha", log_alpha), ("log_mu", log_mu), ("eta", eta)), "cuda")
+    B, T, H, dk = q.shape
+    dv = v.shape[-1]
+    if d_o.device.type != "cuda" or not d_o.is_contiguous() or tuple(d_o.shape) != (B, T, H, dv):
+        raise ValueError("d_o must be a contiguous cuda tensor of o's shape")
+    N = 0
+    if cu_seqlens is not None:
+        if cu_seqlens.device.type != "cuda" or cu_seqlens.dtype != torch.int32 or not cu_seqlens.is_contiguous():
+            raise ValueError("cu_seqlens must be a contiguous int32 cuda tensor")
+        N = cu_seqlens.numel() - 1
+    p = make_params(q, v, num_seqs=N, scale=scale, o_dtype=d_o.dtype)
+    nst = N if N > 0 else B
+    for name, t in (("initial_S", initial_S), ("initial_M", initial_M), ("d_final_S", d_final_S), ("d_final_M", d_final_M)):
+        _check_state(name, t, (nst, H, dk, dv), "cuda")
+    need = int(lib().mdn_chunk_bwd_workspace_bytes(ctypes.byref(p)))
+    if need == 0:
+        raise MdnError(2, "mdn_chunk_bwd_workspace_bytes")
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
+    f32 = dict(dtype=torch.float32, device=q.device)
+    g = dict(dq=torch.empty((B, T, H, dk), **f32), dk=torch.empty((B, T, H, dk), **f32),
+             dv=torch.empty((B, T, H, dv), **f32), dbeta=torch.empty((B, T, H), **f32),
+             dlog_alpha=torch.empty((B, T, H), **f32), dlog_mu=torch.empty((B, T, H), **f32),
+             deta=torch.empty((B, T, H), **f32) if eta is not None else None,
+             d_initial_S=torch.empty((nst, H, dk, dv), **f32), d_initial_M=torch.empty((nst, H, dk, dv), **f32))
+    st = lib().mdn_chunk_bwd(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(beta), _ptr(log_alpha), _ptr(log_mu),
+                             _ptr(eta), _ptr(initial_S), _ptr(initial_M), _ptr(cu_seqlens), _ptr(d_o), _ptr(d_final_S),
+                             _ptr(d_final_M), _ptr(g["dq"]), _ptr(g["dk"]), _ptr(g["dv"]), _ptr(g["dbeta"]),
+                             _ptr(g["dlog_alpha"]), _ptr(g["dlog_mu"]), _ptr(g["deta"]), _ptr(g["d_initial_S"]),
+                             _ptr(g["d_initial_M"]), _ptr(workspace), workspace.numel(), _stream())
+    if st != 0:
+        raise MdnError(st, "mdn_chunk_bwd")
+    return g
 
 
 def decode_step(q, k, v, beta, log_alpha, log_mu, eta, S, M, *, scale: Optional[float] = None,

@@ -285,6 +285,61 @@ mdn_status mdn_chunk_fwd_fused(const mdn_params* p, const mdn_layer_ops* ops, co
   return MDN_OK;
 }
 
+// ---- backward
+static uint64_t bwd_scratch_base(const mdn_ws_layout& lay) { return align_up(lay.off_coef, 256); }
+
+size_t mdn_chunk_bwd_workspace_bytes(const mdn_params* p) {
+  mdn_ws_layout lay;
+  if (check_params(p) != MDN_OK || make_layout(*p, &lay) != MDN_OK) return 0;
+  BwdScratch bs;
+  bwd_scratch_layout(*p, lay.num_slots, &bs);
+  return (size_t)(bwd_scratch_base(lay) + bs.total);   // status word and chunk map, then the backward's scratch
+}
+
+mdn_status mdn_chunk_bwd(const mdn_params* p, const void* q, const void* k, const void* v, const float* beta,
+                         const float* log_alpha, const float* log_mu, const float* eta, const float* initial_S,
+                         const float* initial_M, const int32_t* cu_seqlens, const void* d_o, const float* d_final_S,
+                         const float* d_final_M, float* dq, float* dk, float* dv, float* dbeta, float* dlog_alpha,
+                         float* dlog_mu, float* deta, float* d_initial_S, float* d_initial_M, void* workspace,
+                         size_t workspace_bytes, void* cuda_stream) {
+  t_last_launches = 0;
+  mdn_status st = check_params(p);
+  if (st != MDN_OK) return st;
+  if ((p->num_seqs > 0) != (cu_seqlens != nullptr)) return MDN_ERR_INVALID_ARG;
+  const size_t need = mdn_chunk_bwd_workspace_bytes(p);
+  if (!workspace || workspace_bytes < need || !aligned(workspace, 256)) return MDN_ERR_WORKSPACE;
+  if (!q || !k || !v || !beta || !log_alpha || !log_mu || !d_o || !dq || !dk || !dv || !dbeta || !dlog_alpha || !dlog_mu)
+    return MDN_ERR_INVALID_ARG;
+  if (!aligned(q, 16) || !aligned(k, 16) || !aligned(v, 16) || !aligned(d_o, 16) || !aligned(dq, 16) ||
+      !aligned(dk, 16) || !aligned(dv, 16))
+    return MDN_ERR_INVALID_ARG;
+  Plan pl;
+  pl.p = *p;
+  pl.p.path = MDN_PATH_SIMT;
+  st = make_layout(*p, &pl.lay);
+  if (st != MDN_OK) return st;
+  pl.ws = static_cast<char*>(workspace);
+  pl.stream = static_cast<cudaStream_t>(cuda_stream);
+  pl.gp = GateParam{}; pl.qk = QkNorm{}; pl.post = OutPost{};
+  ChunkGeom& g = pl.geom;
+  g.B = p->B; g.T = p->T; g.H = p->H;
+  g.num_seqs = cu_seqlens ? p->num_seqs : p->B;
+  g.chunks_per_seq = (p->T + C - 1) / C;
+  g.num_slots = pl.lay.num_slots;
+  g.cu = cu_seqlens;
+  g.chunk_off = cu_seqlens ? reinterpret_cast<const int32_t*>(pl.ws + pl.lay.off_chunk_off) : nullptr;
+  g.slot_map = cu_seqlens ? reinterpret_cast<const int32_t*>(pl.ws + pl.lay.off_slot_map) : nullptr;
+  if (cudaMemsetAsync(pl.ws + pl.lay.off_status, 0, 4 * sizeof(int32_t), pl.stream) != cudaSuccess) return MDN_ERR_CUDA;
+  if (launch_chunk_map(pl, &t_last_launches) != cudaSuccess) return MDN_ERR_CUDA;
+  BwdScratch bs;
+  bwd_scratch_layout(*p, pl.lay.num_slots, &bs);
+  const BwdIo io{q, k, v, beta, log_alpha, log_mu, eta, initial_S, initial_M, d_o, d_final_S, d_final_M,
+                 dq, dk, dv, dbeta, dlog_alpha, dlog_mu, deta, d_initial_S, d_initial_M};
+  const cudaError_t e = launch_bwd_stepwise(pl, io, pl.ws + bwd_scratch_base(pl.lay), bs, &t_last_launches);
+  if (e != cudaSuccess) { t_last_cuda_error = (int)e; return MDN_ERR_CUDA; }
+  return MDN_OK;
+}
+
 mdn_status mdn_decode_step(const mdn_params* p, const void* q, const void* k, const void* v, const float* beta,
                            const float* log_alpha, const float* log_mu, const float* eta, float* S, float* M,
                            void* o, void* cuda_stream) {

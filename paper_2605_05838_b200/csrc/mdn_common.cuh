@@ -167,6 +167,20 @@ cudaError_t launch_seg_combine(const Plan& pl, int G, float* E, const float* Psi
                                const float* PhiM, int* launches);
 
 
+// Backward (bwd_stepwise.cu).  Scratch offsets are relative to the scratch base the API layer places after the
+// forward's workspace regions.
+struct BwdScratch { uint64_t part_q, part_k, part_g, ck, prev, total; };
+struct BwdIo {
+  const void* q; const void* k; const void* v;
+  const float* beta; const float* log_alpha; const float* log_mu; const float* eta;
+  const float* S0; const float* M0;
+  const void* d_o; const float* dSf; const float* dMf;
+  float* dq; float* dk; float* dv; float* dbeta; float* dlog_alpha; float* dlog_mu; float* deta;
+  float* dS0; float* dM0;
+};
+void bwd_scratch_layout(const mdn_params& p, int num_slots, BwdScratch* s);
+cudaError_t launch_bwd_stepwise(const Plan& pl, const BwdIo& io, char* scratch, const BwdScratch& sl, int* launches);
+
 // Recurrent decode step (one token per sequence, state updated in place).
 cudaError_t launch_decode_step(const mdn_params& p, const void* q, const void* k, const void* v, const float* beta,
                                const float* log_alpha, const float* log_mu, const float* eta, float* S, float* M,
