@@ -441,6 +441,54 @@ def run_layer_ops(args, w):
         "placement": {"inside the kernels": res["fused"], "separate passes": res["separate"]}}))
 
 
+def run_backward(args, w):
+    """Secondary benchmark (not the headline): mdn_chunk_bwd (all gradients) on the same workload, inputs and the
+    upstream gradient resident in HBM, CUDA events."""
+    import torch
+    import paper_2605_05838_b200 as mdn
+    mdn.lib()
+    torch.cuda.set_device(0)
+    inp = wl.make_inputs(w)
+    dt = torch.bfloat16 if w.dtype == "bf16" else torch.float32
+    dev = lambda x, d=torch.float32: None if x is None else torch.from_numpy(np.ascontiguousarray(x)).to("cuda").to(d)
+    q, k, v = dev(inp["q"], dt), dev(inp["k"], dt), dev(inp["v"], dt)
+    gates = [dev(inp[n]) for n in ("beta", "log_alpha", "log_mu", "eta")]
+    cu = None if inp["cu_seqlens"] is None else torch.from_numpy(inp["cu_seqlens"]).to("cuda")
+    d_o = torch.randn(v.shape, device="cuda", generator=torch.Generator(device="cuda").manual_seed(1)).to(dt)
+    need = int(mdn.lib().mdn_chunk_bwd_workspace_bytes(ctypes.byref(mdn.make_params(q, v, num_seqs=0 if cu is None else cu.numel() - 1))))
+    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+
+    def step():
+        return mdn.chunk_bwd(q, k, v, *gates, d_o, initial_S=dev(inp["S0"]), initial_M=dev(inp["M0"]), cu_seqlens=cu,
+                             scale=inp["scale"], workspace=ws)
+
+    warm = max(args.warmup, 3)
+    for _ in range(warm):
+        step()
+    launches = mdn.last_launch_count()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / args.steps
+    peaks = load_peaks()
+    tokens, es = w.B * w.T, (2 if w.dtype == "bf16" else 4)
+    # reads q, k, v, dO and four gates; writes dq, dk, dv (fp32) and four gate gradients
+    abytes = float(tokens * w.H * ((2 * w.dk + 2 * w.dv) * es + 16 + (2 * w.dk + w.dv) * 4 + 16))
+    print(json.dumps({
+        "metric": "MDN chunkwise bwd tokens/s", "value": tokens / (ms * 1e-3), "unit": "tokens/s", "n_gpus": 1,
+        "steps": args.steps, "warmup": warm, "ms_per_step": ms, "higher_is_better": True, "dtype": "f32",
+        "data": "synthetic", "config": {"workload": workload_desc(w), "form": "token-level adjoint recurrence, "
+                                        "per-chunk checkpoints and recomputation (fp32)"},
+        "gpu_launches": launches * args.steps, "workspace_bytes": need,
+        "roofline": {"bound": "hbm", "kernel": "bwd_stepwise", "achieved": abytes / (ms * 1e-3) / 1e9,
+                     "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": abytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                     "traffic": None, "peak_source": peaks["source"], "algorithmic_bytes": abytes}}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -454,6 +502,7 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--decode", action="store_true", help="secondary benchmark: the recurrent decode step")
     ap.add_argument("--decode-batch", type=int, default=128)
+    ap.add_argument("--backward", action="store_true", help="secondary benchmark: mdn_chunk_bwd (all gradients)")
     ap.add_argument("--layer-ops", action="store_true",
                     help="secondary benchmark: forward with the layer's element-wise operations, fused vs separate passes")
     args = ap.parse_args()
@@ -463,6 +512,9 @@ def main():
     w = wl.CONFIGS[args.config]
     if args.layer_ops:
         run_layer_ops(args, w)
+        return
+    if args.backward:
+        run_backward(args, w)
         return
     if args.impl == "reference":
         run_reference(args, w)

@@ -15,7 +15,7 @@
 //     dv~ = -eta GM^T k = dv;  dalpha = <GS, S_{t-1}> - dv~.(S_{t-1}^T k);  dmu = <GM, M_{t-1}>;
 //     dk = -eta a - alpha S_{t-1} dv~;  GS <- alpha (GS - k dv~^T);  GM <- mu GM.
 // Sums over rows (per column) go through an 8 x 32 shared array; sums over the 32 columns (per row) through
-// [dk][33] shared tiles read back by two threads per row; three block barriers per token.
+// [dk][33] shared tiles read back by two threads per row; two block barriers per adjoint step.
 #include "mdn_common.cuh"
 
 namespace mdn {
@@ -177,28 +177,34 @@ __global__ void __launch_bounds__(kBT, DK == 128 && sizeof(TIn) == 4 ? 1 : 2) bw
       if (dg == 0) { vts[t * kNV + lane] = vt; preds[t * kNV + lane] = pred; }
     }
     __syncthreads();
-    // adjoint steps
+    // adjoint steps; S_{t-1}, M_{t-1} of the next token to be processed are fetched one token ahead
+    float Sp[RPT], Mp[RPT];
+    if (n > 0) {
+      const float* pp = prevp + (size_t)(n - 1) * 2 * DK * kNV;
+#pragma unroll
+      for (int r = 0; r < RPT; ++r) {
+        Sp[r] = pp[(size_t)(dg * RPT + r) * kNV + lane];
+        Mp[r] = pp[(size_t)(DK + dg * RPT + r) * kNV + lane];
+      }
+    }
     for (int t = n - 1; t >= 0; --t) {
-      const float* pp = prevp + (size_t)t * 2 * DK * kNV;
       const float al = gts[0 * C + t], mu = gts[1 * C + t], be = gts[2 * C + t], et = gts[3 * C + t];
       const float doj = dos[t * kNV + lane], vtj = vts[t * kNV + lane];
       const size_t grow = (tok0 + t) * H + h;
-      float Sp[RPT], kr[RPT];
+      float kr[RPT];
       float nb = 0.f, na = 0.f, nm = 0.f, w = 0.f;
 #pragma unroll
       for (int r = 0; r < RPT; ++r) {
         const int row = dg * RPT + r;
-        Sp[r] = pp[(size_t)row * kNV + lane];
-        const float Mp = pp[(size_t)(DK + row) * kNV + lane];
         kr[r] = to_f32<TIn>(ks[t * DK + row]);
         const float qr = to_f32<TIn>(__ldg(qg + grow * DK + row));
-        const float m_t = mu * Mp - et * kr[r] * vtj;
+        const float m_t = mu * Mp[r] - et * kr[r] * vtj;
         const float s_t = al * Sp[r] - be * m_t;
         GS[r] = fmaf(a.scale * qr, doj, GS[r]);
         nb = fmaf(GS[r], m_t, nb);
         na = fmaf(GS[r], Sp[r], na);
         GM[r] = fmaf(-be, GS[r], GM[r]);
-        nm = fmaf(GM[r], Mp, nm);
+        nm = fmaf(GM[r], Mp[r], nm);
         tileA[row * kLT + lane] = s_t * doj;
         tileB[row * kLT + lane] = GM[r] * vtj;
         w = fmaf(GM[r], kr[r], w);
@@ -225,6 +231,20 @@ __global__ void __launch_bounds__(kBT, DK == 128 && sizeof(TIn) == 4 ? 1 : 2) bw
       sb += __shfl_xor_sync(0xffffffffu, sb, 1);
 #pragma unroll
       for (int r = 0; r < RPT; ++r) tileC[(dg * RPT + r) * kLT + lane] = Sp[r] * dvt;
+      if (t > 0) {   // the previous state of token t - 1: in flight while this token is finished
+        const float* pp = prevp + (size_t)(t - 1) * 2 * DK * kNV;
+#pragma unroll
+        for (int r = 0; r < RPT; ++r) {
+          Sp[r] = pp[(size_t)(dg * RPT + r) * kNV + lane];
+          Mp[r] = pp[(size_t)(DK + dg * RPT + r) * kNV + lane];
+        }
+      }
+      if (tid == 0 && t < n - 1) {   // deta of the token processed before this one (its k . a partials are complete)
+        float te = 0.f;
+#pragma unroll
+        for (int g8 = 0; g8 < kGroups; ++g8) te += scal[g8 * 4 + 3];
+        a.part_g[(((size_t)cb * a.g.B * a.g.T + (tok0 + t + 1)) * H + h) * 4 + 3] = -te;
+      }
       if (dg == 0) {
         a.dv_out[grow * DV + j] = dvt;
         const float dp = warp_sum(dvt * preds[t * kNV + lane]);
@@ -261,13 +281,13 @@ __global__ void __launch_bounds__(kBT, DK == 128 && sizeof(TIn) == 4 ? 1 : 2) bw
         GS[r] = al * (GS[r] - kr[r] * dvt);
         GM[r] *= mu;
       }
-      __syncthreads();   // (3) scal[.][3] complete; tiles free for the next token
-      if (tid == 0) {
-        float te = 0.f;
+    }
+    __syncthreads();   // k . a partials of the chunk's first token; tiles free for the next chunk
+    if (tid == 0 && n > 0) {
+      float te = 0.f;
 #pragma unroll
-        for (int g8 = 0; g8 < kGroups; ++g8) te += scal[g8 * 4 + 3];
-        a.part_g[(((size_t)cb * a.g.B * a.g.T + (tok0 + t)) * H + h) * 4 + 3] = -te;   // deta
-      }
+      for (int g8 = 0; g8 < kGroups; ++g8) te += scal[g8 * 4 + 3];
+      a.part_g[(((size_t)cb * a.g.B * a.g.T + tok0) * H + h) * 4 + 3] = -te;
     }
   }
 #pragma unroll
