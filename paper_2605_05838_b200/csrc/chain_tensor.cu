@@ -27,10 +27,10 @@
 // accumulating onto them; with the fused output step the staged fp32 tile is re-read row-wise for RMSNorm, weight
 // and sigmoid gate before the TMA store.  kLayer = false is the plain forward, compiled without any of it.
 //
-// Warp roles: 0-3 critical-path epilogue (P, EPI-1, EPI-2); 4-7 output epilogue (EPI-o);
-// 8 TMA producer (2-stage ring: K, Q, V, T, W_hi, W_lo, 6 coefficient vectors per chunk);
-// 9 MMA issuer (one elected lane) and tensor-memory owner.  All hand-offs are mbarriers with
-// bounded waits; tensor-memory column reuse is ordered by those same barriers.
+// Warp roles: 8 (plain forward) or 16 (with layer operations) epilogue warps, lane quarter x token group, every one
+// running P, EPI-o, EPI-1, EPI-2 on its share; then the TMA producer (2-stage ring: K, Q, V, T, W_hi, W_lo, 8 coefficient vectors per chunk; it also
+// issues the output stores) and the MMA issuer (one elected lane, tensor-memory owner).  All hand-offs are
+// mbarriers with bounded waits; tensor-memory column reuse is ordered by those same barriers.
 #include <cstdlib>
 #include <cstring>
 
@@ -43,9 +43,20 @@ namespace {
 using namespace tc;
 
 constexpr int kD = 128;
-constexpr int kThreads = 320;
-constexpr int kEpiWarps = 8, kWarpTma = 8, kWarpMma = 9;
-constexpr int kEpiThreads = kEpiWarps * 32;
+// Epilogue warps: 4 lane quarters (value rows 32 q .. +31 = the tensor-memory lanes a warp may touch) x TG token
+// groups of 64 / TG tokens, followed by the TMA producer warp and the MMA issuer warp.  The epilogue steps are bound
+// by fixed latencies (tensor-memory round trips, group barriers), not by instruction issue: the plain forward is
+// as fast with 8 epilogue warps (TG = 2, 168 registers per thread) as with 16; the variant with the layer
+// operations, whose output step is instruction-heavy, gains 3 % from 16 (TG = 4, 96 registers).
+template <int TG> struct Roles {
+  static_assert(TG == 2 || TG == 4, "token groups");
+  static constexpr int kTG = TG;
+  static constexpr int kTok = C / TG;          // tokens per epilogue warp in the per-token steps
+  static constexpr int kPk = kTok / 2;         // 32-bit words of packed bf16 pairs for those tokens
+  static constexpr int kEpiWarps = 4 * TG;
+  static constexpr int kThreads = (kEpiWarps + 2) * 32;
+};
+constexpr int token_groups(bool layer) { return layer ? 4 : 2; }
 
 // shared memory (offsets from a 1024-byte aligned base)
 constexpr uint32_t kOffSb = 0, kOffMb = 32768, kOffStage = 65536;
@@ -75,7 +86,7 @@ struct Bars {
   uint64_t mo;        // MMA-3' done                                                   (commit)
   uint64_t zu;        // U (intra-chunk output) has been read                           (256)
   uint64_t ga;        // epilogue group sync                                            (256)
-  uint64_t pn[2];     // fused output step: partial sums of a token half are in shared memory (128 each)
+  uint64_t pn[4];     // fused output step: the staged rows of a token group are in shared memory (128 each)
 };
 
 struct ChainArgs {
@@ -128,7 +139,7 @@ template <> __device__ __forceinline__ void stage_o<__nv_bfloat16>(uint8_t* tile
 }
 
 template <typename TO, bool kLayer>
-__global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainArgs a,
+__global__ void __launch_bounds__(Roles<token_groups(kLayer)>::kThreads, 1) chain_tensor_kernel(const ChainArgs a,
                                                                   const __grid_constant__ CUtensorMap map_q,
                                                                   const __grid_constant__ CUtensorMap map_k,
                                                                   const __grid_constant__ CUtensorMap map_v,
@@ -142,6 +153,9 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
   __shared__ int abort_flag;
   __shared__ __align__(16) float w_sm[kLayer ? kD : 4];   // RMSNorm weight of the fused output step
 
+  using R = Roles<token_groups(kLayer)>;
+  constexpr int kTG = R::kTG, kTok = R::kTok, kPk = R::kPk, kEpiWarps = R::kEpiWarps;
+  constexpr int kWarpTma = kEpiWarps, kWarpMma = kEpiWarps + 1, kEpiThreads = kEpiWarps * 32;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int H = a.g.H;
   // ---- work item: which chain, which segment of it, which kind of run
@@ -215,7 +229,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
     mbar_init(b_v2, kEpiThreads); mbar_init(b_ga, kEpiThreads); mbar_init(b_zq, kEpiThreads);
     mbar_init(b_zu, kEpiThreads);
     mbar_init(b_m1, 1); mbar_init(b_mq, 1); mbar_init(b_m2, 1); mbar_init(b_m3, 1); mbar_init(b_mo, 1);
-    mbar_init(smem_u32(&bars.pn[0]), 128); mbar_init(smem_u32(&bars.pn[1]), 128);
+    for (int i = 0; i < kTG; ++i) mbar_init(smem_u32(&bars.pn[i]), 128);
     mbar_fence_init();
   }
   if (kLayer && tid < kD) w_sm[tid] = (a.post_on && a.post_w) ? __ldg(a.post_w + tid) : 1.f;
@@ -394,19 +408,19 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
       }
     }
   } else {
-    // ================================================================== epilogue warps 0..7
+    // ================================================================== epilogue warps
     // lane quarter q4 = warp & 3 (value columns 32 q4 .. +31 = this warp's tensor-memory lanes),
-    // half hf = warp >> 2 (tokens 32 hf .. +31 in the per-token steps, dk columns 64 hf .. +63 in P).
-    const int q4 = warp & 3, hf = warp >> 2;
+    // token group hf = warp >> 2 (tokens kTok hf .. +kTok-1 in the per-token steps, a share of the dk columns in P).
+    const int q4 = warp & 3, hf = warp >> 2;   // hf: token group
     const int d = q4 * 32 + lane;
-    const int r0 = 32 * hf;
+    const int r0 = kTok * hf;
     const uint32_t tl = tmem + (static_cast<uint32_t>(q4 * 32) << 16);
     uint32_t ga_phase = 0, pn_phase = 0;
     const uint32_t b_pn = smem_u32(&bars.pn[hf]);
-    float oi[32];   // scale (abar .* Q S - b .* Q M) for this thread's tokens, carried to the output step
+    float oi[kTok];   // scale (abar .* Q S - b .* Q M) for this thread's tokens, carried to the output step
 
 #pragma unroll
-    for (int j = 0; j < 32; ++j) oi[j] = 0.f;
+    for (int j = 0; j < kTok; ++j) oi[j] = 0.f;
     for (int c = 0; c <= nch; ++c) {
       // ---------------- P(c): bf16 copies of S^T, M^T for MMA-1 (after the last chunk: final states)
       float al = 0.f, bl = 0.f, ml = 0.f;
@@ -422,55 +436,111 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
       }
       __syncwarp();
       tc_fence_after_sync();
+      if constexpr (kTG == 2) {   // two passes of 32 dk columns (kept textually apart: the plain forward's schedule is fragile)
 #pragma unroll 1
-      for (int i = 0; i < 2; ++i) {
-        const int cs = 2 * hf + i;   // 32-column slice of dk
-        uint32_t sr[32], mr[32];
-        if (c == 0) {
+        for (int i = 0; i < 2; ++i) {
+          const int cs = 2 * hf + i;   // 32-column slice of dk
+          uint32_t sr[32], mr[32];
+          if (c == 0) {
 #pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const float unit = (cs * 32 + j == d) ? 1.f : 0.f;
-            sr[j] = __float_as_uint(S0p ? __ldg(S0p + (size_t)(cs * 32 + j) * kD + d) : (id_s ? unit : 0.f));
-            mr[j] = __float_as_uint(M0p ? __ldg(M0p + (size_t)(cs * 32 + j) * kD + d) : (id_m ? unit : 0.f));
+            for (int j = 0; j < 32; ++j) {
+              const float unit = (cs * 32 + j == d) ? 1.f : 0.f;
+              sr[j] = __float_as_uint(S0p ? __ldg(S0p + (size_t)(cs * 32 + j) * kD + d) : (id_s ? unit : 0.f));
+              mr[j] = __float_as_uint(M0p ? __ldg(M0p + (size_t)(cs * 32 + j) * kD + d) : (id_m ? unit : 0.f));
+            }
+          } else {
+            tmem_ld32(tl + kColS + cs * 32, sr);
+            tmem_ld32(tl + kColM + cs * 32, mr);
+            tmem_wait_ld();
           }
-        } else {
-          tmem_ld32(tl + kColS + cs * 32, sr);
-          tmem_ld32(tl + kColM + cs * 32, mr);
-          tmem_wait_ld();
+          if (c < nch) {
+            uint8_t* sb = smem + kOffSb + (cs >> 1) * 16384;
+            uint8_t* mb = smem + kOffMb + (cs >> 1) * 16384;
+#pragma unroll
+            for (int j8 = 0; j8 < 4; ++j8) {
+              uint4 ps, pm;
+              ps.x = pack_bf16(__uint_as_float(sr[j8 * 8 + 0]), __uint_as_float(sr[j8 * 8 + 1]));
+              ps.y = pack_bf16(__uint_as_float(sr[j8 * 8 + 2]), __uint_as_float(sr[j8 * 8 + 3]));
+              ps.z = pack_bf16(__uint_as_float(sr[j8 * 8 + 4]), __uint_as_float(sr[j8 * 8 + 5]));
+              ps.w = pack_bf16(__uint_as_float(sr[j8 * 8 + 6]), __uint_as_float(sr[j8 * 8 + 7]));
+              pm.x = pack_bf16(__uint_as_float(mr[j8 * 8 + 0]), __uint_as_float(mr[j8 * 8 + 1]));
+              pm.y = pack_bf16(__uint_as_float(mr[j8 * 8 + 2]), __uint_as_float(mr[j8 * 8 + 3]));
+              pm.z = pack_bf16(__uint_as_float(mr[j8 * 8 + 4]), __uint_as_float(mr[j8 * 8 + 5]));
+              pm.w = pack_bf16(__uint_as_float(mr[j8 * 8 + 6]), __uint_as_float(mr[j8 * 8 + 7]));
+              const uint32_t off = sw128_offset(d, (cs & 1) * 32 + j8 * 8);
+              *reinterpret_cast<uint4*>(sb + off) = ps;
+              *reinterpret_cast<uint4*>(mb + off) = pm;
+            }
+            // masters scaled by this chunk's (abar_C, b_C, mubar_C) so that MMA-3 can accumulate straight into
+            // them; the stores are asynchronous and only waited for before V~_S, V~_M are handed over
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              const float sv = __uint_as_float(sr[j]), mv = __uint_as_float(mr[j]);
+              sr[j] = __float_as_uint(al * sv - bl * mv);
+              mr[j] = __float_as_uint(ml * mv);
+            }
+            tmem_st32(tl + kColS + cs * 32, sr);
+            tmem_st32(tl + kColM + cs * 32, mr);
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              if (Sfp) Sfp[(size_t)(cs * 32 + j) * kD + d] = __uint_as_float(sr[j]);
+              if (Mfp) Mfp[(size_t)(cs * 32 + j) * kD + d] = __uint_as_float(mr[j]);
+            }
+          }
         }
-        if (c < nch) {
-          uint8_t* sb = smem + kOffSb + (cs >> 1) * 16384;
-          uint8_t* mb = smem + kOffMb + (cs >> 1) * 16384;
+      } else {
+        constexpr int kPw = (kTG == 4) ? 16 : 32;   // dk columns per pass (a warp owns 128 / kTG of them)
+#pragma unroll 1
+        for (int i = 0; i < 128 / kTG / kPw; ++i) {
+          const int col0 = hf * (128 / kTG) + i * kPw;
+          uint32_t sr[kPw], mr[kPw];
+          if (c == 0) {
 #pragma unroll
-          for (int j8 = 0; j8 < 4; ++j8) {
-            uint4 ps, pm;
-            ps.x = pack_bf16(__uint_as_float(sr[j8 * 8 + 0]), __uint_as_float(sr[j8 * 8 + 1]));
-            ps.y = pack_bf16(__uint_as_float(sr[j8 * 8 + 2]), __uint_as_float(sr[j8 * 8 + 3]));
-            ps.z = pack_bf16(__uint_as_float(sr[j8 * 8 + 4]), __uint_as_float(sr[j8 * 8 + 5]));
-            ps.w = pack_bf16(__uint_as_float(sr[j8 * 8 + 6]), __uint_as_float(sr[j8 * 8 + 7]));
-            pm.x = pack_bf16(__uint_as_float(mr[j8 * 8 + 0]), __uint_as_float(mr[j8 * 8 + 1]));
-            pm.y = pack_bf16(__uint_as_float(mr[j8 * 8 + 2]), __uint_as_float(mr[j8 * 8 + 3]));
-            pm.z = pack_bf16(__uint_as_float(mr[j8 * 8 + 4]), __uint_as_float(mr[j8 * 8 + 5]));
-            pm.w = pack_bf16(__uint_as_float(mr[j8 * 8 + 6]), __uint_as_float(mr[j8 * 8 + 7]));
-            const uint32_t off = sw128_offset(d, (cs & 1) * 32 + j8 * 8);
-            *reinterpret_cast<uint4*>(sb + off) = ps;
-            *reinterpret_cast<uint4*>(mb + off) = pm;
+            for (int j = 0; j < kPw; ++j) {
+              const float unit = (col0 + j == d) ? 1.f : 0.f;
+              sr[j] = __float_as_uint(S0p ? __ldg(S0p + (size_t)(col0 + j) * kD + d) : (id_s ? unit : 0.f));
+              mr[j] = __float_as_uint(M0p ? __ldg(M0p + (size_t)(col0 + j) * kD + d) : (id_m ? unit : 0.f));
+            }
+          } else {
+            tmem_ld_n<kPw>(tl + kColS + col0, sr);
+            tmem_ld_n<kPw>(tl + kColM + col0, mr);
+            tmem_wait_ld();
           }
-          // masters scaled by this chunk's (abar_C, b_C, mubar_C) so that MMA-3 can accumulate straight into
-          // them; the stores are asynchronous and only waited for before V~_S, V~_M are handed over
+          if (c < nch) {
+            uint8_t* sb = smem + kOffSb + (col0 >> 6) * 16384;
+            uint8_t* mb = smem + kOffMb + (col0 >> 6) * 16384;
 #pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const float sv = __uint_as_float(sr[j]), mv = __uint_as_float(mr[j]);
-            sr[j] = __float_as_uint(al * sv - bl * mv);
-            mr[j] = __float_as_uint(ml * mv);
-          }
-          tmem_st32(tl + kColS + cs * 32, sr);
-          tmem_st32(tl + kColM + cs * 32, mr);
-        } else {
+            for (int j8 = 0; j8 < kPw / 8; ++j8) {
+              uint4 ps, pm;
+              ps.x = pack_bf16(__uint_as_float(sr[j8 * 8 + 0]), __uint_as_float(sr[j8 * 8 + 1]));
+              ps.y = pack_bf16(__uint_as_float(sr[j8 * 8 + 2]), __uint_as_float(sr[j8 * 8 + 3]));
+              ps.z = pack_bf16(__uint_as_float(sr[j8 * 8 + 4]), __uint_as_float(sr[j8 * 8 + 5]));
+              ps.w = pack_bf16(__uint_as_float(sr[j8 * 8 + 6]), __uint_as_float(sr[j8 * 8 + 7]));
+              pm.x = pack_bf16(__uint_as_float(mr[j8 * 8 + 0]), __uint_as_float(mr[j8 * 8 + 1]));
+              pm.y = pack_bf16(__uint_as_float(mr[j8 * 8 + 2]), __uint_as_float(mr[j8 * 8 + 3]));
+              pm.z = pack_bf16(__uint_as_float(mr[j8 * 8 + 4]), __uint_as_float(mr[j8 * 8 + 5]));
+              pm.w = pack_bf16(__uint_as_float(mr[j8 * 8 + 6]), __uint_as_float(mr[j8 * 8 + 7]));
+              const uint32_t off = sw128_offset(d, (col0 & 63) + j8 * 8);
+              *reinterpret_cast<uint4*>(sb + off) = ps;
+              *reinterpret_cast<uint4*>(mb + off) = pm;
+            }
+            // masters scaled by this chunk's (abar_C, b_C, mubar_C) so that MMA-3 can accumulate straight into
+            // them; the stores are asynchronous and only waited for before V~_S, V~_M are handed over
 #pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            if (Sfp) Sfp[(size_t)(cs * 32 + j) * kD + d] = __uint_as_float(sr[j]);
-            if (Mfp) Mfp[(size_t)(cs * 32 + j) * kD + d] = __uint_as_float(mr[j]);
+            for (int j = 0; j < kPw; ++j) {
+              const float sv = __uint_as_float(sr[j]), mv = __uint_as_float(mr[j]);
+              sr[j] = __float_as_uint(al * sv - bl * mv);
+              mr[j] = __float_as_uint(ml * mv);
+            }
+            tmem_st_n<kPw>(tl + kColS + col0, sr);
+            tmem_st_n<kPw>(tl + kColM + col0, mr);
+          } else {
+#pragma unroll
+            for (int j = 0; j < kPw; ++j) {
+              if (Sfp) Sfp[(size_t)(col0 + j) * kD + d] = __uint_as_float(sr[j]);
+              if (Mfp) Mfp[(size_t)(col0 + j) * kD + d] = __uint_as_float(mr[j]);
+            }
           }
         }
       }
@@ -490,53 +560,54 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
         // fused output step: this thread's share of the chunk's output-gate rows is four threads per token, 8-byte
         // pieces (each warp-load covers eight full 32-byte sectors); the rows are pulled towards L2 here and read
         // once the tile is staged, when registers are free again
-        const int t128 = q4 * 32 + lane, prow = r0 + (t128 >> 2), part = t128 & 3;
+        constexpr int kTpr = 128 / kTok, kPieces = 32 / kTpr;   // threads per row, 16-byte pieces per thread
+        const int t128 = q4 * 32 + lane, prow = r0 + t128 / kTpr, part = t128 % kTpr;
         const bool g_live = post && cp * C + prow < sq.len;
         const uint2* gp = reinterpret_cast<const uint2*>(static_cast<const __nv_bfloat16*>(a.post_g) +
                                                          ((size_t)(sq.tok0 + cp * C + prow) * H + h) * kD) + part;
-        if (g_live && part < 2) asm volatile("prefetch.global.L2 [%0];" ::"l"(gp + 15 * part));   // bytes 0 and 128 of the row
+        if (g_live && part < 2) asm volatile("prefetch.global.L2 [%0];" ::"l"(gp + 15 * part));   // bytes 0 and 128 of the row (parts 0, 1)
         MDN_WAIT(b_mo, cp & 1);
         __syncwarp();
         tc_fence_after_sync();
         MDN_MARK(cp, kEvMoSeen);
         {
-          uint32_t u[32];
-          tmem_ld32(tl + kColU + r0, u);
+          uint32_t u[kTok];
+          tmem_ld_n<kTok>(tl + kColU + r0, u);
           tmem_wait_ld();
           tc_fence_before_sync();
           mbar_arrive(b_zu);
           MDN_MARK(cp, kEvZuArrive);
           if (!post) {
 #pragma unroll
-            for (int j = 0; j < 32; ++j) stage_o<TO>(stp, r0 + j, d, oi[j] + __uint_as_float(u[j]));
+            for (int j = 0; j < kTok; ++j) stage_o<TO>(stp, r0 + j, d, oi[j] + __uint_as_float(u[j]));
           } else {
             // fused output step: y = sigmoid(g) * o / sqrt(mean_d o^2 + eps) * w_d.  The fp32 tile is staged first
             // (value columns across lanes), then re-read row-wise: four threads per token sum its 128 squares,
             // rescale, gate and write the final tile (in place for fp32 output, into the T / W area for bf16).
             float* tile = reinterpret_cast<float*>(stp);
 #pragma unroll
-            for (int j = 0; j < 32; ++j) tile[(r0 + j) * kD + d] = oi[j] + __uint_as_float(u[j]);
-            uint2 graw[8];
+            for (int j = 0; j < kTok; ++j) tile[(r0 + j) * kD + d] = oi[j] + __uint_as_float(u[j]);
+            uint2 graw[kPieces];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) graw[i] = g_live ? __ldg(gp + 4 * i) : make_uint2(0u, 0u);
+            for (int i = 0; i < kPieces; ++i) graw[i] = g_live ? __ldg(gp + kTpr * i) : make_uint2(0u, 0u);
             mbar_arrive(b_pn);
             MDN_WAIT(b_pn, pn_phase);
             pn_phase ^= 1;
             __syncwarp();
             const int row = prow;
-            float4 ov[8];
+            float4 ov[kPieces];
             float ss = 0.f;
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {   // interleaved 16-byte pieces: the four threads of a row cover 64 B at a time
-              ov[i] = *reinterpret_cast<const float4*>(tile + row * kD + (part + 4 * i) * 4);
+            for (int i = 0; i < kPieces; ++i) {   // interleaved 16-byte pieces: a row's threads cover contiguous bytes
+              ov[i] = *reinterpret_cast<const float4*>(tile + row * kD + (part + kTpr * i) * 4);
               ss = fmaf(ov[i].x, ov[i].x, fmaf(ov[i].y, ov[i].y, fmaf(ov[i].z, ov[i].z, fmaf(ov[i].w, ov[i].w, ss))));
             }
-            ss += __shfl_xor_sync(0xffffffffu, ss, 1);
-            ss += __shfl_xor_sync(0xffffffffu, ss, 2);
+#pragma unroll
+            for (int off = 1; off < kTpr; off <<= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
             const float rstd = rsqrtf(ss * (1.f / kD) + a.post_eps);
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-              const int col = (part + 4 * i) * 4;
+            for (int i = 0; i < kPieces; ++i) {
+              const int col = (part + kTpr * i) * 4;
               const float4 wv = *reinterpret_cast<const float4*>(w_sm + col);
               const uint2 gr = graw[i];
               const float g0 = __uint_as_float(gr.x << 16), g1 = __uint_as_float(gr.x & 0xffff0000u);
@@ -566,21 +637,21 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
       // ---------------- EPI-1: R^T = V^T - abar .* X + (alpha b^-) .* Y  -> bf16 hi, lo in X
       {
         // V and the coefficients do not depend on the MMA: fetch them while MMA-1a runs
-        float vv[32];
+        float vv[kTok];
 #pragma unroll
-        for (int j = 0; j < 32; ++j) vv[j] = v_zero ? 0.f : __bfloat162float(sV[(r0 + j) * kD + d]);
+        for (int j = 0; j < kTok; ++j) vv[j] = v_zero ? 0.f : __bfloat162float(sV[(r0 + j) * kD + d]);
         MDN_WAIT(b_m1, ph);
         __syncwarp();
         tc_fence_after_sync();
         MDN_MARK(c, kEvM1Seen);
-        uint32_t hi[16], lo[16];
+        uint32_t hi[kPk], lo[kPk];
         {
-          uint32_t x[32], y[32];
-          tmem_ld32(tl + kColX + r0, x);
-          tmem_ld32(tl + kColY + r0, y);
+          uint32_t x[kTok], y[kTok];
+          tmem_ld_n<kTok>(tl + kColX + r0, x);
+          tmem_ld_n<kTok>(tl + kColY + r0, y);
           tmem_wait_ld();
 #pragma unroll
-          for (int j = 0; j < 32; j += 4) {
+          for (int j = 0; j < kTok; j += 4) {
             const float4 ab = *reinterpret_cast<const float4*>(cf + kAbar * C + r0 + j);
             const float4 pb = *reinterpret_cast<const float4*>(cf + kAlphaBPrev * C + r0 + j);
             float e0, e1, e2, e3;
@@ -612,8 +683,8 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
             split_pack_bf16(e2, e3, hi[(j >> 1) + 1], lo[(j >> 1) + 1]);
           }
           if (qk_on && write_o) {   // own lanes only; MMA-3' of the previous chunk and this thread's read of U are done
-            tmem_st32(tl + kColZ + r0, x);
-            tmem_st32(tl + kColU + r0, y);
+            tmem_st_n<kTok>(tl + kColZ + r0, x);
+            tmem_st_n<kTok>(tl + kColU + r0, y);
           }
         }
         // the other half's warps may still be reading X: group sync before overwriting it
@@ -623,8 +694,8 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
         ga_phase ^= 1;
         __syncwarp();
         tc_fence_after_sync();
-        tmem_st16(tl + kColX + 16 * hf, hi);
-        tmem_st16(tl + kColX + 32 + 16 * hf, lo);
+        tmem_st_n<kPk>(tl + kColX + kPk * hf, hi);
+        tmem_st_n<kPk>(tl + kColX + 32 + kPk * hf, lo);
         tmem_wait_st();
       }
       tc_fence_before_sync();
@@ -639,14 +710,14 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
     __syncwarp();                                                                                            \
     tc_fence_after_sync();                                                                                   \
     MDN_MARK(c, kEvMqSeen);                                                                                  \
-    uint32_t z[32], u[32];                                                                                   \
-    tmem_ld32(tl + kColZ + r0, z);                                                                           \
-    tmem_ld32(tl + kColU + r0, u);                                                                           \
+    uint32_t z[kTok], u[kTok];                                                                               \
+    tmem_ld_n<kTok>(tl + kColZ + r0, z);                                                                     \
+    tmem_ld_n<kTok>(tl + kColU + r0, u);                                                                     \
     tmem_wait_ld();                                                                                          \
     tc_fence_before_sync();                                                                                  \
     mbar_arrive(b_zq);                                                                                       \
     MDN_MARK(c, kEvZqArrive);                                                                                \
-    _Pragma("unroll") for (int j = 0; j < 32; j += 4) {                                                      \
+    _Pragma("unroll") for (int j = 0; j < kTok; j += 4) {                                                    \
       const float4 ab = *reinterpret_cast<const float4*>(cf + kAbar * C + r0 + j);                           \
       const float4 bb = *reinterpret_cast<const float4*>(cf + kB * C + r0 + j);                              \
       float4 sc = make_float4(a.scale, a.scale, a.scale, a.scale);                                           \
@@ -666,15 +737,15 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
           __syncwarp();
           tc_fence_after_sync();
           MDN_MARK(c, kEvMqSeen);
-          uint32_t z[32], u[32];
-          tmem_ld32(tl + kColZ + r0, z);
-          tmem_ld32(tl + kColU + r0, u);
+          uint32_t z[kTok], u[kTok];
+          tmem_ld_n<kTok>(tl + kColZ + r0, z);
+          tmem_ld_n<kTok>(tl + kColU + r0, u);
           tmem_wait_ld();
           tc_fence_before_sync();
           mbar_arrive(b_zq);
           MDN_MARK(c, kEvZqArrive);
 #pragma unroll
-          for (int j = 0; j < 32; j += 4) {
+          for (int j = 0; j < kTok; j += 4) {
             const float4 ab = *reinterpret_cast<const float4*>(cf + kAbar * C + r0 + j);
             const float4 bb = *reinterpret_cast<const float4*>(cf + kB * C + r0 + j);
             oi[j + 0] = a.scale * (ab.x * __uint_as_float(z[j + 0]) - bb.x * __uint_as_float(u[j + 0]));
@@ -692,25 +763,25 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
       tc_fence_after_sync();
       MDN_MARK(c, kEvM2Seen);
       {
-        uint32_t vt[32];
-        tmem_ld32(tl + kColY + r0, vt);
+        uint32_t vt[kTok];
+        tmem_ld_n<kTok>(tl + kColY + r0, vt);
         tmem_wait_ld();
         {
-          uint32_t sh[16], sl[16];
+          uint32_t sh[kPk], sl[kPk];
 #pragma unroll
-          for (int j = 0; j < 32; j += 4) {
+          for (int j = 0; j < kTok; j += 4) {
             const float4 gs = *reinterpret_cast<const float4*>(cf + kGS * C + r0 + j);
             split_pack_bf16(gs.x * __uint_as_float(vt[j]), gs.y * __uint_as_float(vt[j + 1]), sh[j >> 1], sl[j >> 1]);
             split_pack_bf16(gs.z * __uint_as_float(vt[j + 2]), gs.w * __uint_as_float(vt[j + 3]), sh[(j >> 1) + 1],
                             sl[(j >> 1) + 1]);
           }
-          tmem_st16(tl + kColX + 16 * hf, sh);          // X is free: MMA-2 has consumed R
-          tmem_st16(tl + kColX + 32 + 16 * hf, sl);
+          tmem_st_n<kPk>(tl + kColX + kPk * hf, sh);          // X is free: MMA-2 has consumed R
+          tmem_st_n<kPk>(tl + kColX + 32 + kPk * hf, sl);
         }
         {
-          uint32_t mh[16], mlo[16];
+          uint32_t mh[kPk], mlo[kPk];
 #pragma unroll
-          for (int j = 0; j < 32; j += 4) {
+          for (int j = 0; j < kTok; j += 4) {
             const float4 gm = *reinterpret_cast<const float4*>(cf + kGM * C + r0 + j);
             split_pack_bf16(gm.x * __uint_as_float(vt[j]), gm.y * __uint_as_float(vt[j + 1]), mh[j >> 1], mlo[j >> 1]);
             split_pack_bf16(gm.z * __uint_as_float(vt[j + 2]), gm.w * __uint_as_float(vt[j + 3]), mh[(j >> 1) + 1],
@@ -723,8 +794,8 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
           ga_phase ^= 1;
           __syncwarp();
           tc_fence_after_sync();
-          tmem_st16(tl + kColY + 16 * hf, mh);
-          tmem_st16(tl + kColY + 32 + 16 * hf, mlo);
+          tmem_st_n<kPk>(tl + kColY + kPk * hf, mh);
+          tmem_st_n<kPk>(tl + kColY + 32 + kPk * hf, mlo);
         }
         tmem_wait_st();          // also covers the pre-scaled masters stored in P part 2
         tc_fence_before_sync();
@@ -735,14 +806,14 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tensor_kernel(const ChainAr
         }
         // part b (under MMA-3): V~ itself for the intra-chunk output, into Z once every warp has read Q S
         if (write_o) {
-          uint32_t vh[16], vl[16];
+          uint32_t vh[kPk], vl[kPk];
 #pragma unroll
-          for (int j = 0; j < 32; j += 2) split_pack_bf16(__uint_as_float(vt[j]), __uint_as_float(vt[j + 1]), vh[j >> 1], vl[j >> 1]);
+          for (int j = 0; j < kTok; j += 2) split_pack_bf16(__uint_as_float(vt[j]), __uint_as_float(vt[j + 1]), vh[j >> 1], vl[j >> 1]);
           MDN_WAIT(b_zq, ph);
           __syncwarp();
           tc_fence_after_sync();
-          tmem_st16(tl + kColZ + 16 * hf, vh);
-          tmem_st16(tl + kColZ + 32 + 16 * hf, vl);
+          tmem_st_n<kPk>(tl + kColZ + kPk * hf, vh);
+          tmem_st_n<kPk>(tl + kColZ + 32 + kPk * hf, vl);
           tmem_wait_st();
           tc_fence_before_sync();
           mbar_arrive(b_v2);
@@ -808,7 +879,8 @@ cudaError_t launch_chain_tensor(const Plan& pl, const void* q, const void* k, co
   auto launch_as = [&](auto kern, unsigned grid) -> cudaError_t {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
     if (e != cudaSuccess) return e;
-    e = launch_pdl(kern, dim3(grid), dim3(kThreads), kSmemBytes, pl.stream, a, mq, mk, mv, mt, mw, mo);
+    const unsigned threads = layer ? Roles<token_groups(true)>::kThreads : Roles<token_groups(false)>::kThreads;
+    e = launch_pdl(kern, dim3(grid), dim3(threads), kSmemBytes, pl.stream, a, mq, mk, mv, mt, mw, mo);
     if (e == cudaSuccess) e = cudaGetLastError();
     if (e == cudaSuccess) ++*launches;
     return e;
