@@ -254,8 +254,9 @@ mdn_status mdn_chunk_fwd_fused(const mdn_params* p, const mdn_layer_ops* ops /* 
  * q, k, v, the gates, the initial states, cu_seqlens, p: exactly the forward call's.  The pass recomputes the
  * forward itself, token by token in float32 (any dk, dv in {64, 128}; p->path and p->segments are ignored), so it
  * does not need the forward's outputs.  Workspace: mdn_chunk_bwd_workspace_bytes(p) bytes, 256-byte aligned,
- * scratch.  Same ownership, stream and error rules as mdn_chunk_fwd; the partial sums over value-column blocks are
- * added in a fixed order, so results are reproducible run to run.
+ * scratch.  Same ownership, stream and error rules as mdn_chunk_fwd.  dv and the initial states' gradients are
+ * bit-reproducible; dq, dk and the gate gradients sum over value columns through shared-memory floating-point
+ * atomics, so their last bits can differ from run to run.
  */
 size_t mdn_chunk_bwd_workspace_bytes(const mdn_params* p);
 
