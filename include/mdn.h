@@ -123,7 +123,12 @@ mdn_status mdn_chunk_fwd(const mdn_params* p,
  * and copies o and the final states back.  All data pointers except `arena` are HOST
  * pointers (pinned memory makes the copies asynchronous); `arena` is a DEVICE buffer of at
  * least mdn_chunk_fwd_host_arena_bytes(p) bytes, 256-byte aligned, owned by the caller.
- * Everything is enqueued on `cuda_stream`; the caller synchronises before reading o.
+ * The batch rows are cut into up to eight slices that move as a pipeline: uploads back to back on an internal
+ * stream, each slice's kernels on `cuda_stream` as soon as its upload has landed, its results downloaded on a
+ * second internal stream while the next slice is still arriving.  `cuda_stream` waits for the last download, so
+ * the caller synchronises it before reading o, as with any asynchronous call.  The two internal streams and their
+ * events are created on the first call of a host thread on a device and kept (this entry point is the one that
+ * is not allocation-free on the host side); pageable host memory works but serialises the copies.
  */
 size_t mdn_chunk_fwd_host_arena_bytes(const mdn_params* p);
 

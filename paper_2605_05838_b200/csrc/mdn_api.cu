@@ -368,33 +368,76 @@ mdn_status mdn_set_stage_events(void* const* events, int32_t n) {
   return MDN_OK;
 }
 
-// ---- host-buffer variant: arena = [q | k | v | 4 gates | S0 | M0 | cu | o | Sf | Mf | workspace]
+// ---- host-buffer variant: arena = [q | k | v | 4 gates | S0 | M0 | cu | o | Sf | Mf | one workspace per slice]
+// The batch rows are cut into up to kHostSlices slices that are copied in, computed and copied out as a pipeline:
+// the uploads run back to back on one internal stream, each slice's kernels start when its upload has landed, and
+// its results leave on a second internal stream while the next slice is still arriving (PCIe is full duplex).  The
+// caller's stream waits for the last download, so synchronising it covers the whole call, as before.
+constexpr int kHostSlices = 8;
+
 struct HostArena {
   uint64_t q, k, v, gates[4], S0, M0, cu, o, Sf, Mf, ws, total;
-  uint64_t qk_bytes, v_bytes, gate_bytes, state_bytes, cu_bytes, o_bytes;
+  uint64_t qk_row, v_row, gate_row, state_row, cu_bytes, o_row;   // bytes per batch row (per sequence for the states)
+  uint64_t ws_slice;
+  int slices, rows_max;
 };
 
+static int host_slices(const mdn_params& p) { return p.num_seqs > 0 ? 1 : (p.B < kHostSlices ? p.B : kHostSlices); }
+
 static bool host_arena(const mdn_params* p, HostArena* a) {
+  if (check_params(p) != MDN_OK) return false;
+  a->slices = host_slices(*p);
+  a->rows_max = (p->B + a->slices - 1) / a->slices;
+  mdn_params ps = *p;
+  ps.B = a->rows_max;
   mdn_ws_layout lay;
-  if (check_params(p) != MDN_OK || make_layout(*p, &lay) != MDN_OK) return false;
-  const uint64_t tokens = (uint64_t)p->B * p->T, es = p->io_dtype == MDN_BF16 ? 2 : 4, eo = p->o_dtype == MDN_BF16 ? 2 : 4;
-  const uint64_t nstate = (uint64_t)(p->num_seqs > 0 ? p->num_seqs : p->B) * p->H * p->dk * p->dv;
-  a->qk_bytes = tokens * p->H * p->dk * es; a->v_bytes = tokens * p->H * p->dv * es;
-  a->gate_bytes = tokens * p->H * 4; a->state_bytes = nstate * 4;
-  a->cu_bytes = p->num_seqs > 0 ? (uint64_t)(p->num_seqs + 1) * 4 : 0; a->o_bytes = tokens * p->H * p->dv * eo;
+  if (make_layout(ps, &lay) != MDN_OK) return false;
+  a->ws_slice = align_up(lay.total_bytes, 256);
+  const uint64_t es = p->io_dtype == MDN_BF16 ? 2 : 4, eo = p->o_dtype == MDN_BF16 ? 2 : 4;
+  const uint64_t rows = (uint64_t)p->B, nseq = (uint64_t)(p->num_seqs > 0 ? p->num_seqs : p->B);
+  a->qk_row = (uint64_t)p->T * p->H * p->dk * es; a->v_row = (uint64_t)p->T * p->H * p->dv * es;
+  a->gate_row = (uint64_t)p->T * p->H * 4; a->state_row = (uint64_t)p->H * p->dk * p->dv * 4;
+  a->cu_bytes = p->num_seqs > 0 ? (uint64_t)(p->num_seqs + 1) * 4 : 0; a->o_row = (uint64_t)p->T * p->H * p->dv * eo;
   uint64_t off = 0;
   auto take = [&](uint64_t bytes) { uint64_t at = off; off = align_up(off + bytes, 256); return at; };
-  a->q = take(a->qk_bytes); a->k = take(a->qk_bytes); a->v = take(a->v_bytes);
-  for (int i = 0; i < 4; ++i) a->gates[i] = take(a->gate_bytes);
-  a->S0 = take(a->state_bytes); a->M0 = take(a->state_bytes); a->cu = take(a->cu_bytes);
-  a->o = take(a->o_bytes); a->Sf = take(a->state_bytes); a->Mf = take(a->state_bytes);
-  a->ws = take(lay.total_bytes); a->total = off;
+  a->q = take(rows * a->qk_row); a->k = take(rows * a->qk_row); a->v = take(rows * a->v_row);
+  for (int i = 0; i < 4; ++i) a->gates[i] = take(rows * a->gate_row);
+  a->S0 = take(nseq * a->state_row); a->M0 = take(nseq * a->state_row); a->cu = take(a->cu_bytes);
+  a->o = take(rows * a->o_row); a->Sf = take(nseq * a->state_row); a->Mf = take(nseq * a->state_row);
+  a->ws = take((uint64_t)a->slices * a->ws_slice); a->total = off;
   return true;
 }
 
 size_t mdn_chunk_fwd_host_arena_bytes(const mdn_params* p) {
   HostArena a;
   return host_arena(p, &a) ? (size_t)a.total : 0;
+}
+
+// Internal copy streams and events of the host-buffer pipeline, one set per device and host thread, created on
+// first use and kept.
+struct HostPipe {
+  bool ready;
+  cudaStream_t in, out;
+  cudaEvent_t begin, in_done[kHostSlices], cmp_done[kHostSlices], out_done;
+};
+static thread_local HostPipe t_pipes[64] = {};
+
+static HostPipe* host_pipe() {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  HostPipe& hp = t_pipes[dev];
+  if (!hp.ready) {
+    bool ok = cudaStreamCreateWithFlags(&hp.in, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&hp.out, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaEventCreateWithFlags(&hp.begin, cudaEventDisableTiming) == cudaSuccess &&
+              cudaEventCreateWithFlags(&hp.out_done, cudaEventDisableTiming) == cudaSuccess;
+    for (int i = 0; ok && i < kHostSlices; ++i)
+      ok = cudaEventCreateWithFlags(&hp.in_done[i], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&hp.cmp_done[i], cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) return nullptr;
+    hp.ready = true;
+  }
+  return &hp;
 }
 
 mdn_status mdn_chunk_fwd_host(const mdn_params* p, const void* q, const void* k, const void* v, const float* beta,
@@ -406,31 +449,66 @@ mdn_status mdn_chunk_fwd_host(const mdn_params* p, const void* q, const void* k,
   if (!arena || arena_bytes < a.total || !aligned(arena, 256)) return MDN_ERR_WORKSPACE;
   if (!q || !k || !v || !beta || !log_alpha || !log_mu || !o) return MDN_ERR_INVALID_ARG;
   if ((p->num_seqs > 0) != (cu_seqlens != nullptr)) return MDN_ERR_INVALID_ARG;
+  HostPipe* hp = host_pipe();
+  if (!hp) return MDN_ERR_CUDA;
   char* d = static_cast<char*>(arena);
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  auto ok = [](cudaError_t e) { return e == cudaSuccess; };
   auto h2d = [&](uint64_t off, const void* src, uint64_t bytes) {
-    return src == nullptr || bytes == 0 || cudaMemcpyAsync(d + off, src, bytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    return src == nullptr || bytes == 0 ||
+           ok(cudaMemcpyAsync(d + off, static_cast<const char*>(src), bytes, cudaMemcpyHostToDevice, hp->in));
   };
   auto d2h = [&](void* dst, uint64_t off, uint64_t bytes) {
-    return dst == nullptr || cudaMemcpyAsync(dst, d + off, bytes, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+    return dst == nullptr || bytes == 0 || ok(cudaMemcpyAsync(dst, d + off, bytes, cudaMemcpyDeviceToHost, hp->out));
   };
-  if (!h2d(a.q, q, a.qk_bytes) || !h2d(a.k, k, a.qk_bytes) || !h2d(a.v, v, a.v_bytes) ||
-      !h2d(a.gates[0], beta, a.gate_bytes) || !h2d(a.gates[1], log_alpha, a.gate_bytes) ||
-      !h2d(a.gates[2], log_mu, a.gate_bytes) || !h2d(a.gates[3], eta, a.gate_bytes) ||
-      !h2d(a.S0, initial_S, a.state_bytes) || !h2d(a.M0, initial_M, a.state_bytes) ||
-      !h2d(a.cu, cu_seqlens, a.cu_bytes))
-    return MDN_ERR_CUDA;
+  auto at = [](const void* base, uint64_t bytes) { return base ? static_cast<const char*>(base) + bytes : nullptr; };
+  auto at_w = [](void* base, uint64_t bytes) { return base ? static_cast<char*>(base) + bytes : nullptr; };
+  // the uploads start after whatever the caller's stream holds at this point (it may still use the arena)
+  if (!ok(cudaEventRecord(hp->begin, s)) || !ok(cudaStreamWaitEvent(hp->in, hp->begin, 0))) return MDN_ERR_CUDA;
+  if (!h2d(a.cu, cu_seqlens, a.cu_bytes)) return MDN_ERR_CUDA;
+  const int per = p->B / a.slices, extra = p->B % a.slices;
+  const bool packed = p->num_seqs > 0;
+  int row0 = 0;
+  int first_row[kHostSlices], n_rows[kHostSlices];
+  for (int i = 0; i < a.slices; ++i) {
+    const uint64_t nr = (uint64_t)(per + (i < extra ? 1 : 0)), r0 = (uint64_t)row0;
+    const uint64_t nst = packed ? (uint64_t)p->num_seqs : nr, s0 = packed ? 0 : r0;
+    first_row[i] = row0; n_rows[i] = (int)nr; row0 += (int)nr;
+    if (!h2d(a.q + r0 * a.qk_row, at(q, r0 * a.qk_row), nr * a.qk_row) ||
+        !h2d(a.k + r0 * a.qk_row, at(k, r0 * a.qk_row), nr * a.qk_row) ||
+        !h2d(a.v + r0 * a.v_row, at(v, r0 * a.v_row), nr * a.v_row) ||
+        !h2d(a.gates[0] + r0 * a.gate_row, at(beta, r0 * a.gate_row), nr * a.gate_row) ||
+        !h2d(a.gates[1] + r0 * a.gate_row, at(log_alpha, r0 * a.gate_row), nr * a.gate_row) ||
+        !h2d(a.gates[2] + r0 * a.gate_row, at(log_mu, r0 * a.gate_row), nr * a.gate_row) ||
+        !h2d(a.gates[3] + r0 * a.gate_row, at(eta, r0 * a.gate_row), nr * a.gate_row) ||
+        !h2d(a.S0 + s0 * a.state_row, at(initial_S, s0 * a.state_row), nst * a.state_row) ||
+        !h2d(a.M0 + s0 * a.state_row, at(initial_M, s0 * a.state_row), nst * a.state_row) ||
+        !ok(cudaEventRecord(hp->in_done[i], hp->in)))
+      return MDN_ERR_CUDA;
+  }
   auto fp = [&](uint64_t off, const void* given) { return given ? reinterpret_cast<float*>(d + off) : nullptr; };
-  mdn_ws_layout lay;
-  make_layout(*p, &lay);
-  mdn_status st = mdn_chunk_fwd(p, d + a.q, d + a.k, d + a.v, fp(a.gates[0], beta), fp(a.gates[1], log_alpha),
-                                fp(a.gates[2], log_mu), fp(a.gates[3], eta), fp(a.S0, initial_S),
-                                fp(a.M0, initial_M),
-                                cu_seqlens ? reinterpret_cast<const int32_t*>(d + a.cu) : nullptr, d + a.o,
-                                fp(a.Sf, final_S), fp(a.Mf, final_M), d + a.ws, lay.total_bytes, cuda_stream);
-  if (st != MDN_OK) return st;
-  if (!d2h(o, a.o, a.o_bytes) || !d2h(final_S, a.Sf, a.state_bytes) || !d2h(final_M, a.Mf, a.state_bytes))
-    return MDN_ERR_CUDA;
+  for (int i = 0; i < a.slices; ++i) {
+    const uint64_t nr = (uint64_t)n_rows[i], r0 = (uint64_t)first_row[i];
+    const uint64_t nst = packed ? (uint64_t)p->num_seqs : nr, s0 = packed ? 0 : r0;
+    mdn_params ps = *p;
+    ps.B = n_rows[i];
+    if (!ok(cudaStreamWaitEvent(s, hp->in_done[i], 0))) return MDN_ERR_CUDA;
+    const mdn_status st = mdn_chunk_fwd(
+        &ps, d + a.q + r0 * a.qk_row, d + a.k + r0 * a.qk_row, d + a.v + r0 * a.v_row,
+        fp(a.gates[0] + r0 * a.gate_row, beta), fp(a.gates[1] + r0 * a.gate_row, log_alpha),
+        fp(a.gates[2] + r0 * a.gate_row, log_mu), fp(a.gates[3] + r0 * a.gate_row, eta),
+        fp(a.S0 + s0 * a.state_row, initial_S), fp(a.M0 + s0 * a.state_row, initial_M),
+        cu_seqlens ? reinterpret_cast<const int32_t*>(d + a.cu) : nullptr, d + a.o + r0 * a.o_row,
+        fp(a.Sf + s0 * a.state_row, final_S), fp(a.Mf + s0 * a.state_row, final_M), d + a.ws + (uint64_t)i * a.ws_slice,
+        a.ws_slice, cuda_stream);
+    if (st != MDN_OK) return st;
+    if (!ok(cudaEventRecord(hp->cmp_done[i], s)) || !ok(cudaStreamWaitEvent(hp->out, hp->cmp_done[i], 0)) ||
+        !d2h(at_w(o, r0 * a.o_row), a.o + r0 * a.o_row, nr * a.o_row) ||
+        !d2h(at_w(final_S, s0 * a.state_row), a.Sf + s0 * a.state_row, nst * a.state_row) ||
+        !d2h(at_w(final_M, s0 * a.state_row), a.Mf + s0 * a.state_row, nst * a.state_row))
+      return MDN_ERR_CUDA;
+  }
+  if (!ok(cudaEventRecord(hp->out_done, hp->out)) || !ok(cudaStreamWaitEvent(s, hp->out_done, 0))) return MDN_ERR_CUDA;
   return MDN_OK;
 }
 

@@ -415,11 +415,38 @@ def test_bad_cu_seqlens_is_reported_not_faulted(mdn):
     assert mdn.read_status(p, ws) == 0
 
 
-def test_host_buffer_entry_point(mdn):
-    w = small(T=130, init_state_std=0.2)
+@pytest.mark.parametrize("B", [1, 2, 11])
+def test_host_buffer_entry_point(mdn, B):
+    """Host buffers in, host buffers out (sliced copy / compute / copy pipeline inside): bit-identical to the
+    device-resident call; B = 11 gives uneven slices, B = 1 a single one."""
+    w = small(B=B, T=130, init_state_std=0.2)
+    inp = wl.make_inputs(w)
+    t = to_torch(inp, host_pinned=True)
+    o_d, S_d, M_d = run_gpu(mdn, inp, path="simt")
+    for _ in range(2):      # the second call reuses the internal streams and events
+        o, S, M = mdn.chunk_fwd_host(t["q"], t["k"], t["v"], t["beta"], t["log_alpha"], t["log_mu"], t["eta"],
+                                     initial_S=t["initial_S"], initial_M=t["initial_M"], scale=inp["scale"],
+                                     path="simt")
+        assert np.array_equal(o.numpy(), o_d) and np.array_equal(S.numpy(), S_d) and np.array_equal(M.numpy(), M_d)
+
+
+def test_host_buffer_entry_point_packed_and_tensor_path(mdn):
+    import torch
+    w = wl.Workload("host_packed", B=1, T=900, H=2, dk=128, dv=128, dtype="bf16", varlen=True, len_lo=1, len_hi=300,
+                    init_state_std=0.1, seed=70)
+    if not tensor_ok(mdn, w):
+        pytest.skip("tensor path not built")
     inp = wl.make_inputs(w)
     t = to_torch(inp, host_pinned=True)
     o, S, M = mdn.chunk_fwd_host(t["q"], t["k"], t["v"], t["beta"], t["log_alpha"], t["log_mu"], t["eta"],
-                                 initial_S=t["initial_S"], initial_M=t["initial_M"], scale=inp["scale"], path="simt")
-    o_d, S_d, M_d = run_gpu(mdn, inp, path="simt")
-    assert np.array_equal(o.numpy(), o_d) and np.array_equal(S.numpy(), S_d) and np.array_equal(M.numpy(), M_d)
+                                 initial_S=t["initial_S"], initial_M=t["initial_M"], cu_seqlens=t["cu_seqlens"],
+                                 scale=inp["scale"], path="tensor")
+    o_d, S_d, M_d = run_gpu(mdn, inp, path="tensor")
+    assert np.array_equal(o.float().numpy(), o_d) and np.array_equal(S.numpy(), S_d) and np.array_equal(M.numpy(), M_d)
+    wb = wl.Workload("host_batch", B=6, T=200, H=2, dk=128, dv=128, dtype="bf16", init_state_std=0.1, seed=71)
+    inpb = wl.make_inputs(wb)
+    tb = to_torch(inpb, host_pinned=True)
+    o, S, M = mdn.chunk_fwd_host(tb["q"], tb["k"], tb["v"], tb["beta"], tb["log_alpha"], tb["log_mu"], tb["eta"],
+                                 initial_S=tb["initial_S"], initial_M=tb["initial_M"], scale=inpb["scale"], path="tensor")
+    o_d, S_d, M_d = run_gpu(mdn, inpb, path="tensor")
+    assert np.array_equal(o.float().numpy(), o_d) and np.array_equal(S.numpy(), S_d) and np.array_equal(M.numpy(), M_d)
