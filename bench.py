@@ -364,9 +364,17 @@ def run_decode(args):
     states = [(0.02 * mk(B, H, d, d), 0.02 * mk(B, H, d, d)) for _ in range(n_sets)]
     o = torch.empty((B, 1, H, d), dtype=torch.bfloat16, device="cuda")
 
+    ops = None
+    if args.layer_ops:      # the same step with the layer's element-wise operations inside the kernel
+        hv = lambda lo, hi: torch.rand(H, device="cuda", generator=g) * (hi - lo) + lo
+        ops = mdn.make_layer_ops(q, v, gate_param=dict(a_alpha=hv(0.5, 8.0), b_alpha=hv(-4.5, -3.5), a_mu=hv(0.5, 8.0),
+                                                       b_mu=hv(-3.5, -2.5), s=0.25, tau=11.3),
+                                 qk_norm=dict(d=hv(-0.2, 0.5), eps=1e-6),
+                                 out_norm_gate=dict(g=mk(B, 1, H, d).to(torch.bfloat16), w=None, eps=1e-5))
+
     def step(i):
         S, M = states[i % n_sets]
-        mdn.decode_step(q, k, v, beta, la, lm, eta, S, M, out=o)
+        mdn.decode_step(q, k, v, beta, la, lm, eta, S, M, out=o, layer_ops=ops)
 
     for i in range(max(args.warmup, 3)):
         step(i)
@@ -384,7 +392,8 @@ def run_decode(args):
         "metric": "MDN decode step tokens/s", "value": B / (ms * 1e-3), "unit": "tokens/s", "n_gpus": 1,
         "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True,
         "dtype": "f32", "data": "synthetic",
-        "config": {"workload": "decode: B=%d,H=16,dk=dv=128, one token per sequence, fp32 states in place" % B,
+        "config": {"workload": "decode: B=%d,H=16,dk=dv=128, one token per sequence, fp32 states in place%s"
+                               % (B, ", layer operations inside the kernel" if ops is not None else ""),
                    "l2": "%d rotating state sets (%.0f MB) exceed the 126 MB L2" % (n_sets, n_sets * 2 * B * H * d * d * 4 / 1e6)},
         "gpu_launches": args.steps,
         "roofline": {"bound": "hbm", "kernel": "decode_step", "achieved": abytes / (ms * 1e-3) / 1e9,
@@ -510,7 +519,7 @@ def main():
         run_decode(args)
         return
     w = wl.CONFIGS[args.config]
-    if args.layer_ops:
+    if args.layer_ops and not args.decode:
         run_layer_ops(args, w)
         return
     if args.backward:

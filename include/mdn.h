@@ -156,6 +156,17 @@ mdn_status mdn_decode_step(const mdn_params* p,
                            const float* eta,
                            float* S, float* M, void* o, void* cuda_stream);
 
+/* mdn_decode_step with the layer's element-wise operations (mdn_layer_ops, below) applied to the one token:
+ * gate formulas, q <- L2Norm(q - d k), k <- L2Norm(k), o <- sigmoid(g) * RMSNorm(o) * w; g: [B,1,H,dv].
+ * `placement` is ignored: gates and q / k run inside the step's kernel, the output norm and gate as a second small
+ * kernel over the step's o (measured faster than reducing across the head's CTAs).  ops == NULL is mdn_decode_step. */
+struct mdn_layer_ops_s;
+mdn_status mdn_decode_step_fused(const mdn_params* p, const struct mdn_layer_ops_s* ops,
+                                 const void* q, const void* k, const void* v,
+                                 const float* beta, const float* log_alpha, const float* log_mu,
+                                 const float* eta,
+                                 float* S, float* M, void* o, void* cuda_stream);
+
 /*
  * The forward for callers that cannot allocate device memory (the paper has no counterpart: this
  * is a packaging variant of mdn_chunk_fwd, same kernels, same result).
@@ -217,7 +228,7 @@ mdn_status mdn_chunk_fwd_static_scratch(const mdn_params* p,
  * fp32 accumulators (q and k are never rewritten or re-rounded); the output step runs in the chain kernel's
  * output epilogue.  All pointers are device pointers; the struct itself is host memory, read during the call.
  */
-typedef struct {
+typedef struct mdn_layer_ops_s {
   int32_t raw_gates;
   const float* decay_a_alpha;
   const float* decay_b_alpha;

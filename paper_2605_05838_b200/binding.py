@@ -92,6 +92,8 @@ def lib() -> ctypes.CDLL:
         L.mdn_chunk_fwd_static_scratch.argtypes = [P] + [vp] * 13 + [vp]
         L.mdn_decode_step.restype = ctypes.c_int
         L.mdn_decode_step.argtypes = [P] + [vp] * 10 + [vp]
+        L.mdn_decode_step_fused.restype = ctypes.c_int
+        L.mdn_decode_step_fused.argtypes = [P, ctypes.POINTER(MdnLayerOps)] + [vp] * 10 + [vp]
         L.mdn_workspace_layout.restype = ctypes.c_int
         L.mdn_workspace_layout.argtypes = [P, ctypes.POINTER(MdnWsLayout)]
         L.mdn_coeff_scan.restype = ctypes.c_int
@@ -333,9 +335,10 @@ def chunk_bwd(q, k, v, beta, log_alpha, log_mu, eta, d_o, *, initial_S=None, ini
 
 
 def decode_step(q, k, v, beta, log_alpha, log_mu, eta, S, M, *, scale: Optional[float] = None,
-                o_dtype: Optional[torch.dtype] = None, out: Optional[torch.Tensor] = None) -> torch.Tensor:
-    """mdn_decode_step: one token per sequence (q, k: [B,1,H,dk]; v: [B,1,H,dv]; gates [B,1,H]); the fp32
-    states S, M [B,H,dk,dv] are updated in place.  Returns o [B,1,H,dv]."""
+                o_dtype: Optional[torch.dtype] = None, out: Optional[torch.Tensor] = None,
+                layer_ops: Optional[MdnLayerOps] = None) -> torch.Tensor:
+    """mdn_decode_step (mdn_decode_step_fused when layer_ops is given): one token per sequence (q, k: [B,1,H,dk];
+    v: [B,1,H,dv]; gates [B,1,H]); the fp32 states S, M [B,H,dk,dv] are updated in place.  Returns o [B,1,H,dv]."""
     _check_inputs(q, k, v, (("beta", beta), ("log_alpha", log_alpha), ("log_mu", log_mu), ("eta", eta)), "cuda")
     B, T, H, dk = q.shape
     dv = v.shape[-1]
@@ -345,8 +348,12 @@ def decode_step(q, k, v, beta, log_alpha, log_mu, eta, S, M, *, scale: Optional[
     _check_state("M", M, (B, H, dk, dv), "cuda")
     p = make_params(q, v, scale=scale, o_dtype=o_dtype, path="auto")
     o = out if out is not None else torch.empty((B, 1, H, dv), dtype=o_dtype or q.dtype, device=q.device)
-    st = lib().mdn_decode_step(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(beta), _ptr(log_alpha), _ptr(log_mu),
-                               _ptr(eta), _ptr(S), _ptr(M), _ptr(o), _stream())
+    tail = (_ptr(q), _ptr(k), _ptr(v), _ptr(beta), _ptr(log_alpha), _ptr(log_mu), _ptr(eta), _ptr(S), _ptr(M), _ptr(o),
+            _stream())
+    if layer_ops is None:
+        st = lib().mdn_decode_step(ctypes.byref(p), *tail)
+    else:
+        st = lib().mdn_decode_step_fused(ctypes.byref(p), ctypes.byref(layer_ops), *tail)
     if st != 0:
         raise MdnError(st, "mdn_decode_step")
     return o

@@ -118,6 +118,9 @@ using namespace mdn;
 
 extern "C" {
 
+static bool ops_active(const mdn_layer_ops* ops);
+static mdn_status check_ops(const mdn_layer_ops& f);
+
 size_t mdn_chunk_fwd_workspace_bytes(const mdn_params* p) {
   mdn_ws_layout lay;
   if (check_params(p) != MDN_OK || make_layout(*p, &lay) != MDN_OK) return 0;
@@ -340,9 +343,9 @@ mdn_status mdn_chunk_bwd(const mdn_params* p, const void* q, const void* k, cons
   return MDN_OK;
 }
 
-mdn_status mdn_decode_step(const mdn_params* p, const void* q, const void* k, const void* v, const float* beta,
-                           const float* log_alpha, const float* log_mu, const float* eta, float* S, float* M,
-                           void* o, void* cuda_stream) {
+static mdn_status decode_common(const mdn_params* p, const mdn_layer_ops* ops, const void* q, const void* k,
+                                const void* v, const float* beta, const float* log_alpha, const float* log_mu,
+                                const float* eta, float* S, float* M, void* o, void* cuda_stream) {
   t_last_launches = 0;
   mdn_status st = check_params(p);
   if (st != MDN_OK) return st;
@@ -350,11 +353,44 @@ mdn_status mdn_decode_step(const mdn_params* p, const void* q, const void* k, co
   if (!q || !k || !v || !beta || !log_alpha || !log_mu || !S || !M || !o) return MDN_ERR_INVALID_ARG;
   if (!aligned(q, 16) || !aligned(k, 16) || !aligned(v, 16) || !aligned(o, 16) || !aligned(S, 16) || !aligned(M, 16))
     return MDN_ERR_INVALID_ARG;
-  const cudaError_t e = launch_decode_step(*p, q, k, v, beta, log_alpha, log_mu, eta, S, M, o,
-                                           static_cast<cudaStream_t>(cuda_stream));
+  GateParam gp{};
+  QkNorm qk{};
+  OutPost post{};
+  if (ops_active(ops)) {
+    st = check_ops(*ops);
+    if (st != MDN_OK) return st;
+    if (ops->raw_gates) {
+      if (!eta) return MDN_ERR_INVALID_ARG;
+      gp = GateParam{1, ops->decay_a_alpha, ops->decay_b_alpha, ops->decay_a_mu, ops->decay_b_mu, ops->s,
+                     1.0f / ops->tau, ops->log_mu_min};
+    }
+    qk = QkNorm{ops->qk_norm ? 1 : 0, ops->d, ops->qk_eps};
+    post = OutPost{ops->out_norm_gate ? 1 : 0, ops->g, ops->w, ops->rms_eps};
+  }
+  cudaError_t e = launch_decode_step(*p, q, k, v, beta, log_alpha, log_mu, eta, S, M, o, gp, qk,
+                                     static_cast<cudaStream_t>(cuda_stream));
   if (e != cudaSuccess) { t_last_cuda_error = (int)e; return MDN_ERR_CUDA; }
   t_last_launches = 1;
+  if (post.on) {   // the output norm and gate over the step's o (one head row per warp; o is L2-resident)
+    Plan pl;
+    pl.p = *p;
+    pl.stream = static_cast<cudaStream_t>(cuda_stream);
+    e = launch_out_norm_gate(pl, post, o, &t_last_launches);
+    if (e != cudaSuccess) { t_last_cuda_error = (int)e; return MDN_ERR_CUDA; }
+  }
   return MDN_OK;
+}
+
+mdn_status mdn_decode_step(const mdn_params* p, const void* q, const void* k, const void* v, const float* beta,
+                           const float* log_alpha, const float* log_mu, const float* eta, float* S, float* M,
+                           void* o, void* cuda_stream) {
+  return decode_common(p, nullptr, q, k, v, beta, log_alpha, log_mu, eta, S, M, o, cuda_stream);
+}
+
+mdn_status mdn_decode_step_fused(const mdn_params* p, const mdn_layer_ops* ops, const void* q, const void* k,
+                                 const void* v, const float* beta, const float* log_alpha, const float* log_mu,
+                                 const float* eta, float* S, float* M, void* o, void* cuda_stream) {
+  return decode_common(p, ops, q, k, v, beta, log_alpha, log_mu, eta, S, M, o, cuda_stream);
 }
 
 mdn_status mdn_set_stage_events(void* const* events, int32_t n) {

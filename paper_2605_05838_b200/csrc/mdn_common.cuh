@@ -184,6 +184,6 @@ cudaError_t launch_bwd_stepwise(const Plan& pl, const BwdIo& io, char* scratch, 
 // Recurrent decode step (one token per sequence, state updated in place).
 cudaError_t launch_decode_step(const mdn_params& p, const void* q, const void* k, const void* v, const float* beta,
                                const float* log_alpha, const float* log_mu, const float* eta, float* S, float* M,
-                               void* o, cudaStream_t st);
+                               void* o, const GateParam& gp, const QkNorm& qk, cudaStream_t st);
 
 }  // namespace mdn

@@ -208,6 +208,38 @@ def test_config1_full_size_fused(mdn):
     assert max(errs) <= TOL_BF16
 
 
+@pytest.mark.parametrize("dtype,dk,dv", [("f32", 64, 64), ("f32", 128, 128), ("bf16", 128, 128), ("bf16", 64, 128)])
+def test_decode_step_with_layer_operations(mdn, dtype, dk, dv):
+    """mdn_decode_step_fused token by token (serving path) against the oracle pipeline on the whole sequence."""
+    import torch
+    w = wl.Workload("layer_decode", B=3, T=24, H=2, dk=dk, dv=dv, dtype=dtype, init_state_std=0.2, seed=57)
+    inp = wl.make_layer_inputs(w, s=1.0)
+    ref = oracle_layer(inp, ALL)
+    dt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    dev = lambda x, d=torch.float32: torch.from_numpy(np.ascontiguousarray(x)).to("cuda").to(d)
+    q, k, v, g = dev(inp["q"], dt), dev(inp["k"], dt), dev(inp["v"], dt), dev(inp["g"], dt)
+    xb, xa, xm, xe = (dev(inp[n]) for n in ("x_beta", "x_alpha", "x_mu", "x_eta"))
+    gp = dict(a_alpha=dev(inp["a_alpha"]), b_alpha=dev(inp["b_alpha"]), a_mu=dev(inp["a_mu"]), b_mu=dev(inp["b_mu"]),
+              s=inp["s"], tau=inp["tau"], log_mu_min=inp["log_mu_min"])
+    dvec, wn = dev(inp["d"]), dev(inp["w_norm"])
+    S, M = dev(inp["S0"]), dev(inp["M0"])
+    outs = []
+    for t in range(w.T):
+        sl = slice(t, t + 1)
+        c = lambda x: x[:, sl].contiguous()
+        gt = c(g)
+        ops = mdn.make_layer_ops(c(q), c(v), gate_param=gp, qk_norm=dict(d=dvec, eps=inp["qk_eps"]),
+                                 out_norm_gate=dict(g=gt, w=wn, eps=inp["rms_eps"]))
+        outs.append(mdn.decode_step(c(q), c(k), c(v), c(xb), c(xa), c(xm), c(xe), S, M, scale=inp["scale"],
+                                    o_dtype=torch.float32, layer_ops=ops))
+    torch.cuda.synchronize()
+    f = lambda x: x.float().cpu().numpy().astype(np.float64)
+    got = (f(torch.cat(outs, dim=1)), f(S), f(M))
+    errs = errs3(got, ref)
+    print("decode + layer ops %s dk%d dv%d: o %.3e S %.3e M %.3e" % (dtype, dk, dv, *errs))
+    assert max(errs) <= 1e-4          # the decode kernel computes in fp32 whatever the i/o dtype
+
+
 def test_fused_argument_validation(mdn):
     import torch
     w = wl.Workload("layer_args", B=1, T=64, H=2, dk=64, dv=64, dtype="f32", seed=56)
