@@ -79,13 +79,11 @@ struct Bars {
   uint64_t mq;        // MMA-1b done                                                   (commit)
   uint64_t r;         // EPI-1 done: R^T hi/lo in X                                     (256)
   uint64_t m2;        // MMA-2 done                                                    (commit)
-  uint64_t zq;        // Z, U (Q S, Q M) have been read                                 (256)
   uint64_t v1;        // EPI-2a done: V~_S, V~_M operands in X, Y; masters pre-scaled   (256)
   uint64_t v2;        // EPI-2b done: V~ operand in Z                                   (256)
   uint64_t m3;        // MMA-3 done                                                    (commit)
   uint64_t mo;        // MMA-3' done                                                   (commit)
   uint64_t zu;        // U (intra-chunk output) has been read                           (256)
-  uint64_t ga;        // epilogue group sync                                            (256)
   uint64_t pn[4];     // fused output step: the staged rows of a token group are in shared memory (128 each)
 };
 
@@ -213,9 +211,9 @@ __global__ void __launch_bounds__(Roles<token_groups(kLayer)>::kThreads, 1) chai
   const uint32_t b_full0 = smem_u32(&bars.full[0]), b_full1 = smem_u32(&bars.full[1]);
   const uint32_t b_go0 = smem_u32(&bars.go[0]), b_go1 = smem_u32(&bars.go[1]);
   const uint32_t b_sb = smem_u32(&bars.sb), b_m1 = smem_u32(&bars.m1), b_mq = smem_u32(&bars.mq);
-  const uint32_t b_r = smem_u32(&bars.r), b_m2 = smem_u32(&bars.m2), b_zq = smem_u32(&bars.zq);
+  const uint32_t b_r = smem_u32(&bars.r), b_m2 = smem_u32(&bars.m2);
   const uint32_t b_v1 = smem_u32(&bars.v1), b_v2 = smem_u32(&bars.v2), b_m3 = smem_u32(&bars.m3);
-  const uint32_t b_mo = smem_u32(&bars.mo), b_zu = smem_u32(&bars.zu), b_ga = smem_u32(&bars.ga);
+  const uint32_t b_mo = smem_u32(&bars.mo), b_zu = smem_u32(&bars.zu);
   // kLayer = false compiles the layer operations out: the plain forward keeps its instruction count
   const bool qk_on = kLayer && a.qk_on;
   const bool post = kLayer && a.post_on && write_o;
@@ -226,7 +224,7 @@ __global__ void __launch_bounds__(Roles<token_groups(kLayer)>::kThreads, 1) chai
     mbar_init(b_full0, 1); mbar_init(b_full1, 1);
     mbar_init(b_go0, kEpiThreads); mbar_init(b_go1, kEpiThreads);
     mbar_init(b_sb, kEpiThreads); mbar_init(b_r, kEpiThreads); mbar_init(b_v1, kEpiThreads);
-    mbar_init(b_v2, kEpiThreads); mbar_init(b_ga, kEpiThreads); mbar_init(b_zq, kEpiThreads);
+    mbar_init(b_v2, kEpiThreads);
     mbar_init(b_zu, kEpiThreads);
     mbar_init(b_m1, 1); mbar_init(b_mq, 1); mbar_init(b_m2, 1); mbar_init(b_m3, 1); mbar_init(b_mo, 1);
     for (int i = 0; i < kTG; ++i) mbar_init(smem_u32(&bars.pn[i]), 128);
@@ -311,6 +309,11 @@ __global__ void __launch_bounds__(Roles<token_groups(kLayer)>::kThreads, 1) chai
   } else if (warp == kWarpMma) {
     // ================================================================== MMA issuer
     if (lane == 0) {
+      // Column of the bf16 A operands the epilogue leaves in X, Y, Z: K-step k covers tokens 16k .. 16k + 15; the
+      // epilogue warp that owns those tokens keeps hi (part 0) and lo (part 1) inside its own kTok columns
+      auto a_col = [](int part, int k) {
+        return static_cast<uint32_t>(kTok * ((16 * k) / kTok) + kPk * part + ((16 * k) % kTok) / 2);
+      };
       const uint32_t id64 = idesc_bf16(128, 64, false, false, false);
       const uint32_t id128_mn = idesc_bf16(128, 128, false, true, false);
       const uint32_t id128_mn_neg = idesc_bf16(128, 128, false, true, true);
@@ -370,10 +373,10 @@ __global__ void __launch_bounds__(Roles<token_groups(kLayer)>::kThreads, 1) chai
         tc_fence_after_sync();
         MDN_MARK(c, kEvRSeen);
 #pragma unroll
-        for (int k = 0; k < 4; ++k) umma_ts(tmem + kColY, tmem + kColX + k * 8, dT + 2 * k, id64, k > 0);
+        for (int k = 0; k < 4; ++k) umma_ts(tmem + kColY, tmem + kColX + a_col(0, k), dT + 2 * k, id64, k > 0);
         if (!(a.drop_lo & 1u)) {
 #pragma unroll
-          for (int k = 0; k < 4; ++k) umma_ts(tmem + kColY, tmem + kColX + 32 + k * 8, dT + 2 * k, id64, true);
+          for (int k = 0; k < 4; ++k) umma_ts(tmem + kColY, tmem + kColX + a_col(1, k), dT + 2 * k, id64, true);
         }
         umma_commit(b_m2);
         if constexpr (kLayer) {
@@ -385,23 +388,23 @@ __global__ void __launch_bounds__(Roles<token_groups(kLayer)>::kThreads, 1) chai
         MDN_MARK(c, kEvVSeen);
         const int n3 = (a.drop_lo & 2u) ? 4 : 8;
         for (int k = 0; k < n3; ++k)
-          umma_ts(tmem + kColS, tmem + kColX + (k >> 2) * 32 + (k & 3) * 8, dKmn + 128 * (k & 3), id128_mn, true);
+          umma_ts(tmem + kColS, tmem + kColX + a_col(k >> 2, k & 3), dKmn + 128 * (k & 3), id128_mn, true);
         for (int k = 0; k < n3; ++k)
-          umma_ts(tmem + kColM, tmem + kColY + (k >> 2) * 32 + (k & 3) * 8, dKmn + 128 * (k & 3), id128_mn_neg, true);
+          umma_ts(tmem + kColM, tmem + kColY + a_col(k >> 2, k & 3), dKmn + 128 * (k & 3), id128_mn_neg, true);
         umma_commit(b_m3);
         if (!write_o) continue;   // state-only run: no output terms
         // ---- MMA-3': U = V~^T W^T  with  V~ = hi + lo, W = hi + lo (lo*lo dropped)
         MDN_WAIT(b_v2, ph);
         tc_fence_after_sync();
 #pragma unroll
-        for (int k = 0; k < 4; ++k) umma_ts(tmem + kColU, tmem + kColZ + k * 8, dWh + 2 * k, id64, k > 0);
+        for (int k = 0; k < 4; ++k) umma_ts(tmem + kColU, tmem + kColZ + a_col(0, k), dWh + 2 * k, id64, k > 0);
         if (!(a.drop_lo & 4u)) {
 #pragma unroll
-          for (int k = 0; k < 4; ++k) umma_ts(tmem + kColU, tmem + kColZ + 32 + k * 8, dWh + 2 * k, id64, true);
+          for (int k = 0; k < 4; ++k) umma_ts(tmem + kColU, tmem + kColZ + a_col(1, k), dWh + 2 * k, id64, true);
         }
         if (!(a.drop_lo & 8u)) {
 #pragma unroll
-          for (int k = 0; k < 4; ++k) umma_ts(tmem + kColU, tmem + kColZ + k * 8, dWl + 2 * k, id64, true);
+          for (int k = 0; k < 4; ++k) umma_ts(tmem + kColU, tmem + kColZ + a_col(0, k), dWl + 2 * k, id64, true);
         }
         umma_commit(b_mo);
         MDN_MARK(c, kEvMmaIssued);
@@ -415,7 +418,7 @@ __global__ void __launch_bounds__(Roles<token_groups(kLayer)>::kThreads, 1) chai
     const int d = q4 * 32 + lane;
     const int r0 = kTok * hf;
     const uint32_t tl = tmem + (static_cast<uint32_t>(q4 * 32) << 16);
-    uint32_t ga_phase = 0, pn_phase = 0;
+    uint32_t pn_phase = 0;
     const uint32_t b_pn = smem_u32(&bars.pn[hf]);
     float oi[kTok];   // scale (abar .* Q S - b .* Q M) for this thread's tokens, carried to the output step
 
@@ -687,15 +690,10 @@ __global__ void __launch_bounds__(Roles<token_groups(kLayer)>::kThreads, 1) chai
             tmem_st_n<kTok>(tl + kColU + r0, y);
           }
         }
-        // the other half's warps may still be reading X: group sync before overwriting it
-        tc_fence_before_sync();
-        mbar_arrive(b_ga);
-        MDN_WAIT(b_ga, ga_phase);
-        ga_phase ^= 1;
-        __syncwarp();
-        tc_fence_after_sync();
-        tmem_st_n<kPk>(tl + kColX + kPk * hf, hi);
-        tmem_st_n<kPk>(tl + kColX + 32 + kPk * hf, lo);
+        // hi and lo both go into the columns this warp has just read (its own kTok columns of X): no other warp
+        // touches them, so no group barrier is needed before overwriting
+        tmem_st_n<kPk>(tl + kColX + r0, hi);
+        tmem_st_n<kPk>(tl + kColX + r0 + kPk, lo);
         tmem_wait_st();
       }
       tc_fence_before_sync();
@@ -715,7 +713,6 @@ __global__ void __launch_bounds__(Roles<token_groups(kLayer)>::kThreads, 1) chai
     tmem_ld_n<kTok>(tl + kColU + r0, u);                                                                     \
     tmem_wait_ld();                                                                                          \
     tc_fence_before_sync();                                                                                  \
-    mbar_arrive(b_zq);                                                                                       \
     MDN_MARK(c, kEvZqArrive);                                                                                \
     _Pragma("unroll") for (int j = 0; j < kTok; j += 4) {                                                    \
       const float4 ab = *reinterpret_cast<const float4*>(cf + kAbar * C + r0 + j);                           \
@@ -742,7 +739,6 @@ __global__ void __launch_bounds__(Roles<token_groups(kLayer)>::kThreads, 1) chai
           tmem_ld_n<kTok>(tl + kColU + r0, u);
           tmem_wait_ld();
           tc_fence_before_sync();
-          mbar_arrive(b_zq);
           MDN_MARK(c, kEvZqArrive);
 #pragma unroll
           for (int j = 0; j < kTok; j += 4) {
@@ -775,8 +771,8 @@ __global__ void __launch_bounds__(Roles<token_groups(kLayer)>::kThreads, 1) chai
             split_pack_bf16(gs.z * __uint_as_float(vt[j + 2]), gs.w * __uint_as_float(vt[j + 3]), sh[(j >> 1) + 1],
                             sl[(j >> 1) + 1]);
           }
-          tmem_st_n<kPk>(tl + kColX + kPk * hf, sh);          // X is free: MMA-2 has consumed R
-          tmem_st_n<kPk>(tl + kColX + 32 + kPk * hf, sl);
+          tmem_st_n<kPk>(tl + kColX + r0, sh);          // X is free: MMA-2 has consumed R
+          tmem_st_n<kPk>(tl + kColX + r0 + kPk, sl);
         }
         {
           uint32_t mh[kPk], mlo[kPk];
@@ -787,15 +783,9 @@ __global__ void __launch_bounds__(Roles<token_groups(kLayer)>::kThreads, 1) chai
             split_pack_bf16(gm.z * __uint_as_float(vt[j + 2]), gm.w * __uint_as_float(vt[j + 3]), mh[(j >> 1) + 1],
                             mlo[(j >> 1) + 1]);
           }
-          // Y still holds V~ for the other half's warps until they have loaded it
-          tc_fence_before_sync();
-          mbar_arrive(b_ga);
-          MDN_WAIT(b_ga, ga_phase);
-          ga_phase ^= 1;
-          __syncwarp();
-          tc_fence_after_sync();
-          tmem_st_n<kPk>(tl + kColY + kPk * hf, mh);
-          tmem_st_n<kPk>(tl + kColY + 32 + kPk * hf, mlo);
+          // over this warp's own columns of Y (the V~ it has loaded above)
+          tmem_st_n<kPk>(tl + kColY + r0, mh);
+          tmem_st_n<kPk>(tl + kColY + r0 + kPk, mlo);
         }
         tmem_wait_st();          // also covers the pre-scaled masters stored in P part 2
         tc_fence_before_sync();
@@ -804,16 +794,13 @@ __global__ void __launch_bounds__(Roles<token_groups(kLayer)>::kThreads, 1) chai
         if constexpr (kLayer) {
           if (write_o && qk_on) MDN_INTER_CHUNK_TERMS();
         }
-        // part b (under MMA-3): V~ itself for the intra-chunk output, into Z once every warp has read Q S
+        // part b (under MMA-3): V~ itself for the intra-chunk output, into Z
         if (write_o) {
           uint32_t vh[kPk], vl[kPk];
 #pragma unroll
           for (int j = 0; j < kTok; j += 2) split_pack_bf16(__uint_as_float(vt[j]), __uint_as_float(vt[j + 1]), vh[j >> 1], vl[j >> 1]);
-          MDN_WAIT(b_zq, ph);
-          __syncwarp();
-          tc_fence_after_sync();
-          tmem_st_n<kPk>(tl + kColZ + kPk * hf, vh);
-          tmem_st_n<kPk>(tl + kColZ + 32 + kPk * hf, vl);
+          tmem_st_n<kPk>(tl + kColZ + r0, vh);          // own columns of Z: this thread has read its Q S entries
+          tmem_st_n<kPk>(tl + kColZ + r0 + kPk, vl);
           tmem_wait_st();
           tc_fence_before_sync();
           mbar_arrive(b_v2);
