@@ -353,17 +353,14 @@ __global__ void __launch_bounds__(Roles<token_groups(kLayer)>::kThreads, 1) chai
         umma_ss(tmem + kColU, ((k >> 2) ? dMb1 : dMb0) + 2 * (k & 3), ((k >> 2) ? dQ1 : dQ0) + 2 * (k & 3), id64, (onto) || k > 0); \
     umma_commit(b_mq);                                                                                                     \
   }
+        // ---- MMA-1b (output terms, off the critical path).  The tensor pipe runs its MMAs in issue order, so a group
+        // issued here delays MMA-2 by whatever of it is still running when EPI-1 is done: only Z = S_b Q^T is issued
+        // here (it fits under EPI-1) ...
         if constexpr (!kLayer) {
           if (write_o) {
-            MDN_WAIT(b_zu, ph ^ 1);
-            tc_fence_after_sync();
 #pragma unroll
             for (int k = 0; k < 8; ++k)
               umma_ss(tmem + kColZ, ((k >> 2) ? dSb1 : dSb0) + 2 * (k & 3), ((k >> 2) ? dQ1 : dQ0) + 2 * (k & 3), id64, k > 0);
-#pragma unroll
-            for (int k = 0; k < 8; ++k)
-              umma_ss(tmem + kColU, ((k >> 2) ? dMb1 : dMb0) + 2 * (k & 3), ((k >> 2) ? dQ1 : dQ0) + 2 * (k & 3), id64, k > 0);
-            umma_commit(b_mq);
           }
         } else {
           if (write_o && !qk_on) MDN_MMA_1B(false);
@@ -379,7 +376,17 @@ __global__ void __launch_bounds__(Roles<token_groups(kLayer)>::kThreads, 1) chai
           for (int k = 0; k < 4; ++k) umma_ts(tmem + kColY, tmem + kColX + a_col(1, k), dT + 2 * k, id64, true);
         }
         umma_commit(b_m2);
-        if constexpr (kLayer) {
+        // ... and U = M_b Q^T here: it fits under EPI-2 and is done before MMA-3 can start
+        if constexpr (!kLayer) {
+          if (write_o) {
+            MDN_WAIT(b_zu, ph ^ 1);
+            tc_fence_after_sync();
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+              umma_ss(tmem + kColU, ((k >> 2) ? dMb1 : dMb0) + 2 * (k & 3), ((k >> 2) ? dQ1 : dQ0) + 2 * (k & 3), id64, k > 0);
+            umma_commit(b_mq);
+          }
+        } else {
           if (write_o && qk_on) MDN_MMA_1B(true);
         }
         // ---- MMA-3: S^T += V~_S^T K, M^T -= V~_M^T K   (K tile read MN-major: N = dk, K = tokens)
@@ -728,29 +735,7 @@ __global__ void __launch_bounds__(Roles<token_groups(kLayer)>::kThreads, 1) chai
       oi[j + 3] = sc.w * (ab.w * __uint_as_float(z[j + 3]) - bb.w * __uint_as_float(u[j + 3]));              \
     }                                                                                                        \
   }
-      if constexpr (!kLayer) {
-        if (write_o) {
-          MDN_WAIT(b_mq, ph);
-          __syncwarp();
-          tc_fence_after_sync();
-          MDN_MARK(c, kEvMqSeen);
-          uint32_t z[kTok], u[kTok];
-          tmem_ld_n<kTok>(tl + kColZ + r0, z);
-          tmem_ld_n<kTok>(tl + kColU + r0, u);
-          tmem_wait_ld();
-          tc_fence_before_sync();
-          MDN_MARK(c, kEvZqArrive);
-#pragma unroll
-          for (int j = 0; j < kTok; j += 4) {
-            const float4 ab = *reinterpret_cast<const float4*>(cf + kAbar * C + r0 + j);
-            const float4 bb = *reinterpret_cast<const float4*>(cf + kB * C + r0 + j);
-            oi[j + 0] = a.scale * (ab.x * __uint_as_float(z[j + 0]) - bb.x * __uint_as_float(u[j + 0]));
-            oi[j + 1] = a.scale * (ab.y * __uint_as_float(z[j + 1]) - bb.y * __uint_as_float(u[j + 1]));
-            oi[j + 2] = a.scale * (ab.z * __uint_as_float(z[j + 2]) - bb.z * __uint_as_float(u[j + 2]));
-            oi[j + 3] = a.scale * (ab.w * __uint_as_float(z[j + 3]) - bb.w * __uint_as_float(u[j + 3]));
-          }
-        }
-      } else {
+      if constexpr (kLayer) {
         if (write_o && !qk_on) MDN_INTER_CHUNK_TERMS();
       }
       // ---------------- EPI-2: V~ -> (gamma_C eta) V~, ((mubar_C/mubar) eta) V~ [part a], V~ [part b]; bf16 hi, lo
@@ -791,7 +776,29 @@ __global__ void __launch_bounds__(Roles<token_groups(kLayer)>::kThreads, 1) chai
         tc_fence_before_sync();
         mbar_arrive(b_v1);
         MDN_MARK(c, kEvVArrive);
-        if constexpr (kLayer) {
+        if constexpr (!kLayer) {
+          if (write_o) {
+            MDN_WAIT(b_mq, ph);
+            __syncwarp();
+            tc_fence_after_sync();
+            MDN_MARK(c, kEvMqSeen);
+            uint32_t z[kTok], u[kTok];
+            tmem_ld_n<kTok>(tl + kColZ + r0, z);
+            tmem_ld_n<kTok>(tl + kColU + r0, u);
+            tmem_wait_ld();
+            tc_fence_before_sync();
+            MDN_MARK(c, kEvZqArrive);
+#pragma unroll
+            for (int j = 0; j < kTok; j += 4) {
+              const float4 ab = *reinterpret_cast<const float4*>(cf + kAbar * C + r0 + j);
+              const float4 bb = *reinterpret_cast<const float4*>(cf + kB * C + r0 + j);
+              oi[j + 0] = a.scale * (ab.x * __uint_as_float(z[j + 0]) - bb.x * __uint_as_float(u[j + 0]));
+              oi[j + 1] = a.scale * (ab.y * __uint_as_float(z[j + 1]) - bb.y * __uint_as_float(u[j + 1]));
+              oi[j + 2] = a.scale * (ab.z * __uint_as_float(z[j + 2]) - bb.z * __uint_as_float(u[j + 2]));
+              oi[j + 3] = a.scale * (ab.w * __uint_as_float(z[j + 3]) - bb.w * __uint_as_float(u[j + 3]));
+            }
+          }
+        } else {
           if (write_o && qk_on) MDN_INTER_CHUNK_TERMS();
         }
         // part b (under MMA-3): V~ itself for the intra-chunk output, into Z
