@@ -22,8 +22,8 @@ __global__ void __launch_bounds__(256) gate_param_kernel(GateParam gp, int H, si
   }
 }
 
-// E consecutive elements moved as one 4-, 8- or 16-byte access.
-template <typename T, int E> struct alignas(sizeof(T) * E) Pack { T v[E]; };
+// E consecutive elements moved as one access of up to 16 bytes (two when TG is wider than TO).
+template <typename T, int E> struct alignas(sizeof(T) * E <= 16 ? sizeof(T) * E : 16) Pack { T v[E]; };
 
 __device__ __forceinline__ float warp_sum(float x) {
 #pragma unroll
@@ -31,92 +31,108 @@ __device__ __forceinline__ float warp_sum(float x) {
   return x;
 }
 
-// rows = B*T*H head rows of D elements; lane l owns elements l*E .. l*E+E-1 (E = D / 32, contiguous).  A warp takes
-// kRowsPerIter consecutive rows per iteration and issues all their loads before the first reduction, so that enough
-// bytes are in flight per SM to reach HBM bandwidth.
+// rows = B*T*H head rows of D elements.  Every lane moves 16 bytes per access (E = 16 / sizeof(T) consecutive
+// elements), so a row takes LPR = D / E lanes and a warp covers 32 / LPR rows per access; kRowsPerIter such accesses
+// are issued before the first reduction, so that enough bytes are in flight per SM to approach HBM bandwidth.
 constexpr int kRowsPerIter = 4;
+
+template <int LPR> __device__ __forceinline__ float row_sum(float x) {
+#pragma unroll
+  for (int off = LPR / 2; off > 0; off >>= 1) x += __shfl_xor_sync(0xffffffffu, x, off);
+  return x;
+}
 
 template <typename T, int D>
 __global__ void __launch_bounds__(256) qk_prep_kernel(size_t rows, int H, QkNorm qk, const T* __restrict__ q,
                                                      const T* __restrict__ k, T* __restrict__ q_out,
                                                      T* __restrict__ k_out) {
-  constexpr int E = D / 32, R = kRowsPerIter;
-  const int lane = threadIdx.x & 31;
+  constexpr int E = 16 / sizeof(T), LPR = D / E, RPW = 32 / LPR, R = kRowsPerIter;
+  const int lane = threadIdx.x & 31, sub = lane / LPR, l = lane % LPR;
   const size_t warps = (size_t)gridDim.x * (blockDim.x >> 5);
-  for (size_t row0 = ((size_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) * R; row0 < rows; row0 += warps * R) {
+  const size_t warp_id = (size_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  for (size_t row0 = warp_id * (RPW * R); row0 < rows; row0 += warps * (RPW * R)) {
     Pack<T, E> kp[R], qp[R];
 #pragma unroll
     for (int r = 0; r < R; ++r) {
-      if (row0 + r < rows) {
-        kp[r] = *reinterpret_cast<const Pack<T, E>*>(k + (row0 + r) * D + lane * E);
-        qp[r] = *reinterpret_cast<const Pack<T, E>*>(q + (row0 + r) * D + lane * E);
+      const size_t row = row0 + (size_t)r * RPW + sub;
+      if (row < rows) {
+        kp[r] = *reinterpret_cast<const Pack<T, E>*>(k + row * D + l * E);
+        qp[r] = *reinterpret_cast<const Pack<T, E>*>(q + row * D + l * E);
       }
     }
 #pragma unroll
     for (int r = 0; r < R; ++r) {
-      if (row0 + r >= rows) break;
-      const size_t row = row0 + r;
-      const float d = qk.d ? __ldg(qk.d + (int)(row % H)) : 0.f;
+      const size_t row = row0 + (size_t)r * RPW + sub;
+      const bool live = row < rows;     // (all lanes take part in the shuffles)
+      const float d = (live && qk.d) ? __ldg(qk.d + (int)(row % H)) : 0.f;
       float qv[E], kv[E];
       float sq = 0.f, sk = 0.f;
 #pragma unroll
       for (int e = 0; e < E; ++e) {
-        kv[e] = to_f32<T>(kp[r].v[e]);
-        qv[e] = to_f32<T>(qp[r].v[e]) - d * kv[e];
+        kv[e] = live ? to_f32<T>(kp[r].v[e]) : 0.f;
+        qv[e] = live ? to_f32<T>(qp[r].v[e]) - d * kv[e] : 0.f;
         sq = fmaf(qv[e], qv[e], sq);
         sk = fmaf(kv[e], kv[e], sk);
       }
-      const float rq = 1.f / sqrtf(warp_sum(sq) + qk.eps), rk = 1.f / sqrtf(warp_sum(sk) + qk.eps);
-      Pack<T, E> qo, ko;
+      const float rq = rsqrtf(row_sum<LPR>(sq) + qk.eps), rk = rsqrtf(row_sum<LPR>(sk) + qk.eps);
+      if (live) {
+        Pack<T, E> qo, ko;
 #pragma unroll
-      for (int e = 0; e < E; ++e) {
-        qo.v[e] = from_f32<T>(qv[e] * rq);
-        ko.v[e] = from_f32<T>(kv[e] * rk);
+        for (int e = 0; e < E; ++e) {
+          qo.v[e] = from_f32<T>(qv[e] * rq);
+          ko.v[e] = from_f32<T>(kv[e] * rk);
+        }
+        *reinterpret_cast<Pack<T, E>*>(q_out + row * D + l * E) = qo;
+        *reinterpret_cast<Pack<T, E>*>(k_out + row * D + l * E) = ko;
       }
-      *reinterpret_cast<Pack<T, E>*>(q_out + row * D + lane * E) = qo;
-      *reinterpret_cast<Pack<T, E>*>(k_out + row * D + lane * E) = ko;
     }
   }
 }
 
+// TO and TG may differ in size: the lane's E = 16 / sizeof(TO) elements are one 16-byte access of o and one 16- or
+// 8-byte (or two 16-byte) access of g.
 template <typename TO, typename TG, int D>
 __global__ void __launch_bounds__(256) out_norm_gate_kernel(size_t rows, OutPost post, TO* __restrict__ o) {
-  constexpr int E = D / 32, R = kRowsPerIter;
-  const int lane = threadIdx.x & 31;
+  constexpr int E = 16 / sizeof(TO), LPR = D / E, RPW = 32 / LPR, R = kRowsPerIter;
+  const int lane = threadIdx.x & 31, sub = lane / LPR, l = lane % LPR;
   const TG* __restrict__ g = static_cast<const TG*>(post.g);
   float wv[E];
 #pragma unroll
-  for (int e = 0; e < E; ++e) wv[e] = post.w ? __ldg(post.w + lane * E + e) : 1.f;
+  for (int e = 0; e < E; ++e) wv[e] = post.w ? __ldg(post.w + l * E + e) : 1.f;
   const size_t warps = (size_t)gridDim.x * (blockDim.x >> 5);
-  for (size_t row0 = ((size_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) * R; row0 < rows; row0 += warps * R) {
+  const size_t warp_id = (size_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  for (size_t row0 = warp_id * (RPW * R); row0 < rows; row0 += warps * (RPW * R)) {
     Pack<TO, E> op[R];
     Pack<TG, E> gp[R];
 #pragma unroll
     for (int r = 0; r < R; ++r) {
-      if (row0 + r < rows) {
-        op[r] = *reinterpret_cast<const Pack<TO, E>*>(o + (row0 + r) * D + lane * E);
-        gp[r] = *reinterpret_cast<const Pack<TG, E>*>(g + (row0 + r) * D + lane * E);
+      const size_t row = row0 + (size_t)r * RPW + sub;
+      if (row < rows) {
+        op[r] = *reinterpret_cast<const Pack<TO, E>*>(o + row * D + l * E);
+        gp[r] = *reinterpret_cast<const Pack<TG, E>*>(g + row * D + l * E);
       }
     }
 #pragma unroll
     for (int r = 0; r < R; ++r) {
-      if (row0 + r >= rows) break;
-      const size_t row = row0 + r;
+      const size_t row = row0 + (size_t)r * RPW + sub;
+      const bool live = row < rows;
       float ov[E];
       float ss = 0.f;
 #pragma unroll
       for (int e = 0; e < E; ++e) {
-        ov[e] = to_f32<TO>(op[r].v[e]);
+        ov[e] = live ? to_f32<TO>(op[r].v[e]) : 0.f;
         ss = fmaf(ov[e], ov[e], ss);
       }
-      const float rstd = 1.f / sqrtf(warp_sum(ss) * (1.f / D) + post.eps);
-      Pack<TO, E> yo;
+      const float rstd = rsqrtf(row_sum<LPR>(ss) * (1.f / D) + post.eps);
+      if (live) {
+        Pack<TO, E> yo;
 #pragma unroll
-      for (int e = 0; e < E; ++e) {
-        const float gate = 1.f / (1.f + expf(-to_f32<TG>(gp[r].v[e])));
-        yo.v[e] = from_f32<TO>(gate * ov[e] * rstd * wv[e]);
+        for (int e = 0; e < E; ++e) {
+          const float gate = __fdividef(1.f, 1.f + __expf(-to_f32<TG>(gp[r].v[e])));   // 2 special-function ops
+          yo.v[e] = from_f32<TO>(gate * ov[e] * rstd * wv[e]);
+        }
+        *reinterpret_cast<Pack<TO, E>*>(o + row * D + l * E) = yo;
       }
-      *reinterpret_cast<Pack<TO, E>*>(o + row * D + lane * E) = yo;
     }
   }
 }
@@ -141,7 +157,7 @@ cudaError_t launch_gate_param(const Plan& pl, const float* x_beta, const float* 
 cudaError_t launch_qk_prep(const Plan& pl, const QkNorm& qk, const void* q, const void* k, void* q_out, void* k_out,
                            int* launches) {
   const size_t rows = (size_t)pl.p.B * pl.p.T * pl.p.H;
-  const unsigned grid = blocks_for(rows, 8 * kRowsPerIter);
+  const unsigned grid = blocks_for(rows, 16 * kRowsPerIter);
   const bool bf = pl.p.io_dtype == MDN_BF16;
 #define MDN_QK_CASE(T, D)                                                                                   \
   qk_prep_kernel<T, D><<<grid, 256, 0, pl.stream>>>(rows, pl.p.H, qk, static_cast<const T*>(q),             \
@@ -159,7 +175,7 @@ cudaError_t launch_qk_prep(const Plan& pl, const QkNorm& qk, const void* q, cons
 
 cudaError_t launch_out_norm_gate(const Plan& pl, const OutPost& post, void* o, int* launches) {
   const size_t rows = (size_t)pl.p.B * pl.p.T * pl.p.H;
-  const unsigned grid = blocks_for(rows, 8 * kRowsPerIter);
+  const unsigned grid = blocks_for(rows, 16 * kRowsPerIter);
   const bool obf = pl.p.o_dtype == MDN_BF16, gbf = pl.p.io_dtype == MDN_BF16;
 #define MDN_OUT_CASE(TO, TG, D) out_norm_gate_kernel<TO, TG, D><<<grid, 256, 0, pl.stream>>>(rows, post, static_cast<TO*>(o))
 #define MDN_OUT_D(D)                                                   \
