@@ -224,12 +224,22 @@ def run_ours(args, w):
     p = mdn.make_params(t["q"], t["v"], num_seqs=(N if w.varlen else 0), scale=inp["scale"], o_dtype=o_dtype,
                         path=args.path)
     ws = torch.empty(mdn.workspace_bytes(p), dtype=torch.uint8, device=t["q"].device)
-    o = torch.empty((w.B, w.T, w.H, w.dv), dtype=o_dtype, device=t["q"].device)
+    # a workload whose inputs + outputs fit in the 126 MB L2 would be timed out of cache: rotate enough copies of
+    # every input and of the output that one round exceeds twice the L2
+    io_bytes = algorithmic_bytes(w, N, t["initial_S"] is not None)
+    n_copies = 1 if io_bytes > L2_BYTES else int(2 * L2_BYTES // io_bytes) + 1
+    clone = lambda d: {k_: (v_.clone() if torch.is_tensor(v_) else v_) for k_, v_ in d.items()}
+    sets = [t] + [clone(t) for _ in range(n_copies - 1)]
+    outs = [torch.empty((w.B, w.T, w.H, w.dv), dtype=o_dtype, device=t["q"].device) for _ in range(n_copies)]
+    calls = [0]
 
     def step():
-        return mdn.chunk_fwd(t["q"], t["k"], t["v"], t["beta"], t["log_alpha"], t["log_mu"], t["eta"],
-                             initial_S=t["initial_S"], initial_M=t["initial_M"], cu_seqlens=t["cu_seqlens"],
-                             scale=inp["scale"], o_dtype=o_dtype, path=args.path, workspace=ws, out=o)
+        i = calls[0] % n_copies
+        calls[0] += 1
+        ti = sets[i]
+        return mdn.chunk_fwd(ti["q"], ti["k"], ti["v"], ti["beta"], ti["log_alpha"], ti["log_mu"], ti["eta"],
+                             initial_S=ti["initial_S"], initial_M=ti["initial_M"], cu_seqlens=ti["cu_seqlens"],
+                             scale=inp["scale"], o_dtype=o_dtype, path=args.path, workspace=ws, out=outs[i])
 
     def barrier():
         if dist is not None:
@@ -283,6 +293,8 @@ def run_ours(args, w):
                 "algorithmic_bytes": abytes, "algorithmic_flops": aflops,
                 "tensor_achieved_tflops": aflops / dom_s / 1e12,
                 "tensor_frac_of_burst_peak": aflops / dom_s / 1e12 / peaks["bf16_tflops"],
+                "frac_of_nominal_hbm_8tbs": achieved / 8000.0,
+                "tensor_frac_of_nominal_2250tf": aflops / dom_s / 1e12 / 2250.0,
                 "whole_step_frac_hbm": abytes / (elapsed_ms / args.steps * 1e-3) / 1e9 / peaks["hbm_gbs"]}
     roofline["traffic"] = NCU_TRAFFIC_BYTES.get((w.name, dom))
 
@@ -335,8 +347,10 @@ def run_ours(args, w):
         "data": "synthetic",
         "config": {"workload": workload_desc(w), "path": mdn.resolved_path(p),
                    "parallelism": "independent batch per GPU, no collective",
-                   "l2": "inputs+outputs %.0f MB per step %s the 126 MB L2; no flush between steps"
-                         % (ws_in / 1e6, "exceed" if ws_in > L2_BYTES else "FIT IN")},
+                   "l2": ("inputs+outputs %.0f MB per step exceed the 126 MB L2; no flush between steps" % (ws_in / 1e6))
+                         if n_copies == 1 else
+                         ("inputs+outputs %.0f MB per step fit in the 126 MB L2: %d copies rotated (%.0f MB per round)"
+                          % (ws_in / 1e6, n_copies, n_copies * ws_in / 1e6))},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
         "roofline": roofline, "cpu_baseline": cpu}))
     if dist is not None:
