@@ -100,6 +100,15 @@ def test_fast_forgetting_preset_and_degenerate_gates(mdn):
     check(*run_both(mdn, inp, *upstream(w, inp, 3)), "preset F, beta=0, mu=0 tokens")
 
 
+def test_config2_full_size_two_chains(mdn):
+    """The launch configuration bench.py --backward times (B=8, H=16, T=4096, dk=dv=128, bf16), two sampled chains."""
+    w = wl.CONFIGS[2]
+    inp = wl.make_inputs(w)
+    d_o, dS, dM = upstream(w, inp, 5)
+    got, ref = run_both(mdn, inp, d_o, dS, dM, chains=np.array([3, 126]))
+    check(got, ref, "config 2 (2 of 128 chains)")
+
+
 def test_config1_sampled_chains_and_repeatability(mdn):
     import torch
     w = wl.CONFIGS[1]
