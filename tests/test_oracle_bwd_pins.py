@@ -122,3 +122,23 @@ def test_chain_subset_matches_full():
         assert np.array_equal(sub[name][0, :, 1], full[name][0, :, 1])
         assert np.array_equal(sub[name][1, :, 2], full[name][1, :, 2])
         assert np.isnan(sub[name][0, :, 0]).all()
+
+
+@pytest.mark.parametrize("T,chunk", [(64, 64), (150, 64), (37, 16)])
+def test_chunk_form_backward_equals_stepwise_backward(T, chunk):
+    """oracle/chunkwise_bwd.py differentiates the chunkwise algorithm matrix by matrix (adjoint state recurrence,
+    dA = -tril(dR V~^T, -1) through the inverse, coefficient adjoints, scans in reverse); it must give the gradients of
+    the token-by-token backward, which finite differences pin above.  Several chunks, a ragged last chunk."""
+    from oracle import chunkwise_bwd as cb
+    p = problem(11, T=T, H=2, dk=6, dv=5)
+    ref = grads(p)
+    for h in range(2):
+        g = cb.chain_backward(p["q"][0, :, h], p["k"][0, :, h], p["v"][0, :, h], p["beta"][0, :, h],
+                              p["log_alpha"][0, :, h], p["log_mu"][0, :, h], p["eta"][0, :, h], p["w_o"][0, :, h],
+                              scale=p["scale"], S0=p["S0"][0, h], M0=p["M0"][0, h], dS_final=p["w_S"][0, h],
+                              dM_final=p["w_M"][0, h], chunk=chunk)
+        for name in ("dq", "dk", "dv", "dbeta", "dlog_alpha", "dlog_mu", "deta"):
+            r = ref[name][0, :, h]
+            assert np.allclose(g[name], r, rtol=1e-9, atol=1e-11 * max(1.0, np.abs(r).max())), (name, h)
+        assert np.allclose(g["dS0"], ref["dS0"][0, h], rtol=1e-9, atol=1e-12)
+        assert np.allclose(g["dM0"], ref["dM0"][0, h], rtol=1e-9, atol=1e-12)
