@@ -153,7 +153,9 @@ __global__ void __launch_bounds__(Roles<token_groups(kLayer)>::kThreads, 1) chai
 
   using R = Roles<token_groups(kLayer)>;
   constexpr int kTG = R::kTG, kTok = R::kTok, kPk = R::kPk, kEpiWarps = R::kEpiWarps;
-  constexpr int kWarpTma = kEpiWarps, kWarpMma = kEpiWarps + 1, kEpiThreads = kEpiWarps * 32;
+  constexpr int kWarpTma = kEpiWarps, kWarpMma = kEpiWarps + 1;
+  constexpr bool kWarpArrive = kLayer;   // epilogue hand-overs: one mbarrier arrival per warp, or one per thread
+  constexpr int kArrivals = kWarpArrive ? kEpiWarps : kEpiWarps * 32;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int H = a.g.H;
   // ---- work item: which chain, which segment of it, which kind of run
@@ -222,10 +224,10 @@ __global__ void __launch_bounds__(Roles<token_groups(kLayer)>::kThreads, 1) chai
   if (tid == 0) {
     abort_flag = 0;
     mbar_init(b_full0, 1); mbar_init(b_full1, 1);
-    mbar_init(b_go0, kEpiThreads); mbar_init(b_go1, kEpiThreads);
-    mbar_init(b_sb, kEpiThreads); mbar_init(b_r, kEpiThreads); mbar_init(b_v1, kEpiThreads);
-    mbar_init(b_v2, kEpiThreads);
-    mbar_init(b_zu, kEpiThreads);
+    mbar_init(b_go0, kArrivals); mbar_init(b_go1, kArrivals);
+    mbar_init(b_sb, kArrivals); mbar_init(b_r, kArrivals); mbar_init(b_v1, kArrivals);
+    mbar_init(b_v2, kArrivals);
+    mbar_init(b_zu, kArrivals);
     mbar_init(b_m1, 1); mbar_init(b_mq, 1); mbar_init(b_m2, 1); mbar_init(b_m3, 1); mbar_init(b_mo, 1);
     for (int i = 0; i < kTG; ++i) mbar_init(smem_u32(&bars.pn[i]), 128);
     mbar_fence_init();
@@ -248,6 +250,18 @@ __global__ void __launch_bounds__(Roles<token_groups(kLayer)>::kThreads, 1) chai
     break;                                         \
   }
   long long* const tline = (blockIdx.x == 0) ? a.timeline : nullptr;
+  // Hand-over arrivals of the epilogue.  With 16 epilogue warps (layer variant) one arrival per warp, after the warp
+  // has converged (every lane's stores and fences precede it): 32 x fewer shared-memory atomics in front of every
+  // hand-over, 2 % of the step.  The 8-warp plain forward measured 1 % slower that way and keeps one per thread.
+#define MDN_WARP_ARRIVE(bar)             \
+  {                                      \
+    if constexpr (kWarpArrive) {         \
+      __syncwarp();                      \
+      if (lane == 0) mbar_arrive(bar);   \
+    } else {                             \
+      mbar_arrive(bar);                  \
+    }                                    \
+  }
 #define MDN_MARK(c, ev) \
   if (tline != nullptr && lane == 0 && (warp == 0 || warp >= kEpiWarps)) tline[(c) * 32 + (ev)] = clock64();
 
@@ -556,14 +570,14 @@ __global__ void __launch_bounds__(Roles<token_groups(kLayer)>::kThreads, 1) chai
       }
       if (c < nch) {
         fence_proxy_async_smem();
-        mbar_arrive(b_sb);
+        MDN_WARP_ARRIVE(b_sb);
         MDN_MARK(c, kEvSbArrive);
       }
       // ---------------- output of the previous chunk (under MMA-1a): o^T = oi + U, staged as a [64 x 128] tile in
       // the previous chunk's stage (all its MMAs are done and nobody reads its tiles any more)
       if (c > 0 && !write_o) {
         // state-only run: MMA-3 of the previous chunk (waited for above) was the last reader of its stage
-        mbar_arrive(((c - 1) & 1) ? b_go1 : b_go0);
+        MDN_WARP_ARRIVE(((c - 1) & 1) ? b_go1 : b_go0);
       } else if (c > 0) {
         const int cp = c - 1;
         uint8_t* stp = smem + kOffStage + (cp & 1) * kStageBytes;
@@ -585,7 +599,7 @@ __global__ void __launch_bounds__(Roles<token_groups(kLayer)>::kThreads, 1) chai
           tmem_ld_n<kTok>(tl + kColU + r0, u);
           tmem_wait_ld();
           tc_fence_before_sync();
-          mbar_arrive(b_zu);
+          MDN_WARP_ARRIVE(b_zu);
           MDN_MARK(cp, kEvZuArrive);
           if (!post) {
 #pragma unroll
@@ -635,7 +649,7 @@ __global__ void __launch_bounds__(Roles<token_groups(kLayer)>::kThreads, 1) chai
           }
         }
         fence_proxy_async_smem();
-        mbar_arrive((cp & 1) ? b_go1 : b_go0);
+        MDN_WARP_ARRIVE((cp & 1) ? b_go1 : b_go0);
       }
       if (c == nch) break;
       MDN_MARK(c, kEvPrescaled);
@@ -704,7 +718,7 @@ __global__ void __launch_bounds__(Roles<token_groups(kLayer)>::kThreads, 1) chai
         tmem_wait_st();
       }
       tc_fence_before_sync();
-      mbar_arrive(b_r);
+      MDN_WARP_ARRIVE(b_r);
       MDN_MARK(c, kEvRArrive);
       // ---------------- inter-chunk output terms: oi = scale (abar .* Q S - b .* Q M), under MMA-2; with the fused
       // q/k step Z, U arrive later (MMA-1b follows MMA-2) and already hold Q S - d K S, Q M - d K M: then this
@@ -774,7 +788,7 @@ __global__ void __launch_bounds__(Roles<token_groups(kLayer)>::kThreads, 1) chai
         }
         tmem_wait_st();          // also covers the pre-scaled masters stored in P part 2
         tc_fence_before_sync();
-        mbar_arrive(b_v1);
+        MDN_WARP_ARRIVE(b_v1);
         MDN_MARK(c, kEvVArrive);
         if constexpr (!kLayer) {
           if (write_o) {
@@ -810,7 +824,7 @@ __global__ void __launch_bounds__(Roles<token_groups(kLayer)>::kThreads, 1) chai
           tmem_st_n<kPk>(tl + kColZ + r0 + kPk, vl);
           tmem_wait_st();
           tc_fence_before_sync();
-          mbar_arrive(b_v2);
+          MDN_WARP_ARRIVE(b_v2);
         }
         MDN_MARK(c, kEvV2Arrive);
       }
@@ -818,6 +832,7 @@ __global__ void __launch_bounds__(Roles<token_groups(kLayer)>::kThreads, 1) chai
   }
 #undef MDN_INTER_CHUNK_TERMS
 #undef MDN_MMA_1B
+#undef MDN_WARP_ARRIVE
 #undef MDN_WAIT
 #undef MDN_MARK
 
