@@ -412,7 +412,9 @@ def run_decode(args):
         "gpu_launches": args.steps,
         "roofline": {"bound": "hbm", "kernel": "decode_step", "achieved": abytes / (ms * 1e-3) / 1e9,
                      "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": abytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
-                     "traffic": None, "peak_source": peaks["source"], "algorithmic_bytes": abytes}}))
+                     # ncu dram bytes per launch at B=128 without the layer operations (profiles/decode_step_b128.md)
+                     "traffic": 484.3e6 if (B == 128 and ops is None) else None,
+                     "peak_source": peaks["source"], "algorithmic_bytes": abytes}}))
 
 
 def run_layer_ops(args, w):
