@@ -20,6 +20,7 @@
 // T; 52 KB with the fused q/k norm) and 64 (128) columns of tensor memory.  Tensor memory is released before the CTA signals its dependents, so the chain kernel
 // (which takes all 512 columns of an SM) can never be resident beside a CTA of this kernel that still has to allocate.
 #include <cstring>
+#include <type_traits>
 
 #include "coeff_scan.cuh"
 #include "mdn_common.cuh"
@@ -265,26 +266,37 @@ __global__ void __launch_bounds__(kThreads, kQk ? 4 : kCtasPerSm) intra_mma_kern
   {
     float G = 0.f, a = 1.f, mu_next = 0.f;
     const uint32_t cv_s = s_base + kOffCv;
-    float4 al = lds_f4(cv_s + (C - 4) * 4), be = lds_f4(cv_s + (C + C - 4) * 4), mu = lds_f4(cv_s + (2 * C + C - 4) * 4),
-           et = lds_f4(cv_s + (3 * C + C - 4) * 4);
+    auto walk = [&](auto from_tag, auto to_tag) {   // columns from + 3 down to `to`, in groups of four
+      constexpr int kFrom = decltype(from_tag)::value, kTo = decltype(to_tag)::value;
+      float4 al = lds_f4(cv_s + kFrom * 4), be = lds_f4(cv_s + (C + kFrom) * 4), mu = lds_f4(cv_s + (2 * C + kFrom) * 4),
+             et = lds_f4(cv_s + (3 * C + kFrom) * 4);
 #pragma unroll
-    for (int i4 = C - 4; i4 >= 0; i4 -= 4) {
-      const float alv[4] = {al.x, al.y, al.z, al.w}, bev[4] = {be.x, be.y, be.z, be.w}, muv[4] = {mu.x, mu.y, mu.z, mu.w},
-                  etv[4] = {et.x, et.y, et.z, et.w};
-      if (i4 >= 4) {   // the next group's gate values, fetched ahead of the dependent chain
-        al = lds_f4(cv_s + (i4 - 4) * 4); be = lds_f4(cv_s + (C + i4 - 4) * 4); mu = lds_f4(cv_s + (2 * C + i4 - 4) * 4);
-        et = lds_f4(cv_s + (3 * C + i4 - 4) * 4);
-      }
+      for (int i4 = kFrom; i4 >= kTo; i4 -= 4) {
+        const float alv[4] = {al.x, al.y, al.z, al.w}, bev[4] = {be.x, be.y, be.z, be.w}, muv[4] = {mu.x, mu.y, mu.z, mu.w},
+                    etv[4] = {et.x, et.y, et.z, et.w};
+        if (i4 >= kTo + 4) {   // the next group's gate values, fetched ahead of the dependent chain
+          al = lds_f4(cv_s + (i4 - 4) * 4); be = lds_f4(cv_s + (C + i4 - 4) * 4); mu = lds_f4(cv_s + (2 * C + i4 - 4) * 4);
+          et = lds_f4(cv_s + (3 * C + i4 - 4) * 4);
+        }
 #pragma unroll
-      for (int e = 3; e >= 0; --e) {
-        const int i = i4 + e;
-        const bool p = i <= rp;
-        G = fmaf(mu_next, G, (p ? bev[e] : 0.f) * a);
-        a *= p ? alv[e] : 1.f;
-        f[i] = G * etv[e];
-        mu_next = muv[e];
+        for (int e = 3; e >= 0; --e) {
+          const int i = i4 + e;
+          const bool p = i <= rp;
+          G = fmaf(mu_next, G, (p ? bev[e] : 0.f) * a);
+          a *= p ? alv[e] : 1.f;
+          f[i] = G * etv[e];
+          mu_next = muv[e];
+        }
       }
+    };
+    if (warp & 1) {   // rows 32..63; the rows 0..31 of the other warps are empty right of column 31
+      walk(std::integral_constant<int, C - 4>{}, std::integral_constant<int, C / 2>{});
+    } else {
+#pragma unroll
+      for (int i = C / 2; i < C; ++i) f[i] = 0.f;
+      mu_next = 0.f;
     }
+    walk(std::integral_constant<int, C / 2 - 4>{}, std::integral_constant<int, 0>{});
   }
 
   bool ok = true;
