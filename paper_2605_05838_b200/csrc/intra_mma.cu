@@ -264,7 +264,7 @@ __global__ void __launch_bounds__(kThreads, kQk ? 4 : kCtasPerSm) intra_mma_kern
   const int rp = (r < si.n) ? (w_thread ? r : r - 1) : -1;
   float f[C];
   {
-    float G = 0.f, a = 1.f, mu_next = 0.f;
+    float G = 0.f, a = 0.f, mu_next = 0.f;
     const uint32_t cv_s = s_base + kOffCv;
     auto walk = [&](auto from_tag, auto to_tag) {   // columns from + 3 down to `to`, in groups of four
       constexpr int kFrom = decltype(from_tag)::value, kTo = decltype(to_tag)::value;
@@ -281,9 +281,9 @@ __global__ void __launch_bounds__(kThreads, kQk ? 4 : kCtasPerSm) intra_mma_kern
 #pragma unroll
         for (int e = 3; e >= 0; --e) {
           const int i = i4 + e;
-          const bool p = i <= rp;
-          G = fmaf(mu_next, G, (p ? bev[e] : 0.f) * a);
-          a *= p ? alv[e] : 1.f;
+          a = (i == rp) ? 1.f : a;   // a (and with it G) stays 0 until the walk reaches the row's last column
+          G = fmaf(mu_next, G, bev[e] * a);
+          a *= alv[e];
           f[i] = G * etv[e];
           mu_next = muv[e];
         }
