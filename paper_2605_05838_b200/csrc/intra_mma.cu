@@ -255,7 +255,7 @@ __global__ void __launch_bounds__(kThreads, kQk ? 4 : kCtasPerSm) intra_mma_kern
   }
 
 
-  // ---- the thread's row of Gamma, times eta, in registers: f[i] = gamma_{rp,i} eta_i for i <= rp, else 0, where
+  // ---- the thread's row of Gamma, times eta (and scale or alpha_r), in registers: f[i] ~ gamma_{rp,i} eta_i for i <= rp, else 0, where
   // rp = r for a W row (mask i <= r) and r - 1 for an A row (Gamma shifted one row down, mask i < r).  Tokens past
   // the end of a short chunk (they hold another sequence's data) get empty rows.  Walking i from 63 down,
   //   G <- mu_{i+1} G + beta_i a,   a <- a alpha_i      (a = prod_{i<l<=rp} alpha_l; both idle while i > rp)
@@ -265,6 +265,8 @@ __global__ void __launch_bounds__(kThreads, kQk ? 4 : kCtasPerSm) intra_mma_kern
   float f[C];
   {
     float G = 0.f, a = 0.f, mu_next = 0.f;
+    // the row's constant factor rides on the seed of a (G is linear in it): scale for a W row, alpha_r for an A row
+    const float seed = w_thread ? scale : cv[0 * C + r];
     const uint32_t cv_s = s_base + kOffCv;
     auto walk = [&](auto from_tag, auto to_tag) {   // columns from + 3 down to `to`, in groups of four
       constexpr int kFrom = decltype(from_tag)::value, kTo = decltype(to_tag)::value;
@@ -281,7 +283,7 @@ __global__ void __launch_bounds__(kThreads, kQk ? 4 : kCtasPerSm) intra_mma_kern
 #pragma unroll
         for (int e = 3; e >= 0; --e) {
           const int i = i4 + e;
-          a = (i == rp) ? 1.f : a;   // a (and with it G) stays 0 until the walk reaches the row's last column
+          a = (i == rp) ? seed : a;   // a (and with it G) stays 0 until the walk reaches the row's last column
           G = fmaf(mu_next, G, bev[e] * a);
           a *= alv[e];
           f[i] = G * etv[e];
@@ -357,7 +359,6 @@ __global__ void __launch_bounds__(kThreads, kQk ? 4 : kCtasPerSm) intra_mma_kern
   const size_t mat = ((size_t)slot * g.H + h) * C * C;
   if (!w_thread) {
     const int rbk = r >> 4, rl = r & 15;
-    const float alr = cv[0 * C + r] * rn_r;
 #pragma unroll
     for (int cb = 0; cb < 4; ++cb) {
       if (cb < reach) {
@@ -369,17 +370,19 @@ __global__ void __launch_bounds__(kThreads, kQk ? 4 : kCtasPerSm) intra_mma_kern
 #pragma unroll
           for (int j4 = 0; j4 < 16; j4 += 4) {
             const int i = cb * 16 + j4;
-            float4 rki = make_float4(1.f, 1.f, 1.f, 1.f);
-            if constexpr (kQk) rki = *reinterpret_cast<const float4*>(cv + 6 * C + i);
-            *reinterpret_cast<float4*>(dst + j4) =
-                make_float4(alr * f[i] * rki.x * x[j4], alr * f[i + 1] * rki.y * x[j4 + 1], alr * f[i + 2] * rki.z * x[j4 + 2],
-                            alr * f[i + 3] * rki.w * x[j4 + 3]);
+            if constexpr (kQk) {
+              const float4 rki = *reinterpret_cast<const float4*>(cv + 6 * C + i);
+              *reinterpret_cast<float4*>(dst + j4) =
+                  make_float4(rn_r * f[i] * rki.x * x[j4], rn_r * f[i + 1] * rki.y * x[j4 + 1], rn_r * f[i + 2] * rki.z * x[j4 + 2],
+                              rn_r * f[i + 3] * rki.w * x[j4 + 3]);
+            } else {
+              *reinterpret_cast<float4*>(dst + j4) = make_float4(f[i] * x[j4], f[i + 1] * x[j4 + 1], f[i + 2] * x[j4 + 2], f[i + 3] * x[j4 + 3]);
+            }
           }
         }
       }
     }
   } else {
-    const float sr = scale * rn_r;
     uint8_t* w_hi = smem + kOffWh + r * 128;
     uint8_t* w_lo = smem + kOffWl + r * 128;
 #pragma unroll
@@ -402,7 +405,7 @@ __global__ void __launch_bounds__(kThreads, kQk ? 4 : kCtasPerSm) intra_mma_kern
         }
         float w[16];
 #pragma unroll
-        for (int j = 0; j < 16; ++j) w[j] = sr * f[cb * 16 + j] * x[j];
+        for (int j = 0; j < 16; ++j) w[j] = kQk ? rn_r * f[cb * 16 + j] * x[j] : f[cb * 16 + j] * x[j];
 #pragma unroll
         for (int hf = 0; hf < 2; ++hf) {
           split_pack_bf16(w[hf * 8 + 0], w[hf * 8 + 1], hi4[hf].x, lo4[hf].x);
