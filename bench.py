@@ -457,7 +457,15 @@ def run_layer_ops(args, w):
         torch.cuda.synchronize()
         res[mode] = {"ms_per_step": e0.elapsed_time(e1) / args.steps, "launches_per_step": launches}
     tokens = w.B * w.T
+    peaks = load_peaks()
+    es = 2 if w.dtype == "bf16" else 4
+    # algorithmic bytes of the whole step: q, k, v, g read and o written once, four fp32 raw gates, final states
+    abytes = float(tokens * w.H * ((2 * w.dk + 3 * w.dv) * es + 16) + 2 * w.B * w.H * w.dk * w.dv * 4)
+    ach = abytes / (res["fused"]["ms_per_step"] * 1e-3) / 1e9
     print(json.dumps({
+        "roofline": {"bound": "hbm", "kernel": "whole step (two kernels)", "achieved": ach, "peak": peaks["hbm_gbs"],
+                     "unit": "GB/s", "frac": ach / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
+                     "algorithmic_bytes": abytes},
         "metric": "MDN chunkwise fwd with layer ops tokens/s", "value": tokens / (res["fused"]["ms_per_step"] * 1e-3),
         "unit": "tokens/s", "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3),
         "ms_per_step": res["fused"]["ms_per_step"], "higher_is_better": True, "dtype": w.dtype, "data": "synthetic",
