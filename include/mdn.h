@@ -261,6 +261,30 @@ mdn_status mdn_chunk_fwd_fused(const mdn_params* p, const mdn_layer_ops* ops /* 
                                void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * Forward that also keeps the state at the START of every chunk (Section 3.2: the chunkwise form carries the pair
+ * (S, M) from chunk to chunk; a chunk-parallel backward starts from those states).  Arguments as mdn_chunk_fwd,
+ * plus `chunk_states`: a DEVICE buffer of mdn_chunk_states_bytes(p) bytes, 1024-byte aligned, owned by the caller.
+ * For every (chunk slot, head), in the workspace's slot order, it receives 65536 bytes: the bf16 copy of S^T
+ * (value index x key index, 128 x 128) and then that of M^T, each as two blocks (key index 0..63, 64..127) of 128
+ * rows x 128 bytes whose 16-byte pieces are XOR-swizzled with (row mod 8) - the image a K-major tcgen05 operand
+ * has in shared memory, so a later kernel can fetch a block with one untiled bulk copy.  These are the copies the
+ * forward's own tensor-core products read (the fp32 masters stay on chip).
+ * Tensor path only (bf16 input, dk = dv = 128): MDN_ERR_UNSUPPORTED otherwise.  The serial chain is used
+ * (p->segments is ignored).  Workspace as for mdn_chunk_fwd.
+ */
+size_t mdn_chunk_states_bytes(const mdn_params* p);
+
+mdn_status mdn_chunk_fwd_keep_states(const mdn_params* p,
+                                     const void* q, const void* k, const void* v,
+                                     const float* beta, const float* log_alpha, const float* log_mu,
+                                     const float* eta,
+                                     const float* initial_S, const float* initial_M,
+                                     const int32_t* cu_seqlens,
+                                     void* o, float* final_S, float* final_M,
+                                     void* chunk_states,
+                                     void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * Backward of mdn_chunk_fwd (Section 3.1: the training pass differentiates the same recurrence; like the paper's
  * kernels this keeps no per-token states and rebuilds them from per-chunk checkpoints):
  * given d_o = dL/do ([B,T,H,dv], o_dtype) and optionally dL/d(final_S), dL/d(final_M) ([N,H,dk,dv] float32, NULL =

@@ -82,6 +82,10 @@ def lib() -> ctypes.CDLL:
         L.mdn_chunk_fwd_fused.argtypes = [P, ctypes.POINTER(MdnLayerOps)] + [vp] * 13 + [vp, ctypes.c_size_t, vp]
         L.mdn_chunk_fwd_fused_workspace_bytes.restype = ctypes.c_size_t
         L.mdn_chunk_fwd_fused_workspace_bytes.argtypes = [P, ctypes.POINTER(MdnLayerOps)]
+        L.mdn_chunk_states_bytes.restype = ctypes.c_size_t
+        L.mdn_chunk_states_bytes.argtypes = [P]
+        L.mdn_chunk_fwd_keep_states.restype = ctypes.c_int
+        L.mdn_chunk_fwd_keep_states.argtypes = [P] + [vp] * 14 + [vp, ctypes.c_size_t, vp]
         L.mdn_chunk_bwd.restype = ctypes.c_int
         L.mdn_chunk_bwd.argtypes = [P] + [vp] * 22 + [vp, ctypes.c_size_t, vp]
         L.mdn_chunk_bwd_workspace_bytes.restype = ctypes.c_size_t
@@ -250,13 +254,15 @@ def _check_state(name, t, shape, device_type):
 def chunk_fwd(q, k, v, beta, log_alpha, log_mu, eta=None, *, initial_S=None, initial_M=None,
               cu_seqlens=None, scale: Optional[float] = None, o_dtype: Optional[torch.dtype] = None,
               path: str = "auto", output_final_state: bool = True, workspace: Optional[torch.Tensor] = None,
-              out: Optional[torch.Tensor] = None, segments: int = 0, layer_ops: Optional[MdnLayerOps] = None
-              ) -> Tuple[torch.Tensor, Optional[torch.Tensor], Optional[torch.Tensor]]:
+              out: Optional[torch.Tensor] = None, segments: int = 0, layer_ops: Optional[MdnLayerOps] = None,
+              keep_chunk_states: bool = False):
     """mdn_chunk_fwd (mdn_chunk_fwd_fused when layer_ops is given) on CUDA tensors, current stream.
     Returns (o, final_S, final_M).
     segments: 0 = automatic, 1 = plain serial chain, >= 3 = force the parallel inter-chunk scan.
     layer_ops: from make_layer_ops; with its gate_param set, beta / log_alpha / log_mu / eta are the raw
-    projections x_beta / x_alpha / x_mu / x_eta."""
+    projections x_beta / x_alpha / x_mu / x_eta.
+    keep_chunk_states: mdn_chunk_fwd_keep_states; returns (o, final_S, final_M, chunk_states, workspace) where
+    chunk_states is the raw uint8 buffer (unpack_chunk_states turns it into float tensors)."""
     _check_inputs(q, k, v, (("beta", beta), ("log_alpha", log_alpha), ("log_mu", log_mu), ("eta", eta)), "cuda")
     B, T, H, dk = q.shape
     dv = v.shape[-1]
@@ -285,6 +291,17 @@ def chunk_fwd(q, k, v, beta, log_alpha, log_mu, eta=None, *, initial_S=None, ini
     tail = (_ptr(q), _ptr(k), _ptr(v), _ptr(beta), _ptr(log_alpha), _ptr(log_mu), _ptr(eta), _ptr(initial_S),
             _ptr(initial_M), _ptr(cu_seqlens), _ptr(o), _ptr(Sf), _ptr(Mf), _ptr(workspace), workspace.numel(),
             _stream())
+    if keep_chunk_states:
+        if layer_ops is not None:
+            raise ValueError("keep_chunk_states and layer_ops exclude each other")
+        nbytes = int(lib().mdn_chunk_states_bytes(ctypes.byref(p)))
+        if nbytes == 0:
+            raise MdnError(2, "mdn_chunk_states_bytes")
+        states = torch.empty(nbytes, dtype=torch.uint8, device=q.device)
+        st = lib().mdn_chunk_fwd_keep_states(ctypes.byref(p), *tail[:13], _ptr(states), *tail[13:])
+        if st != 0:
+            raise MdnError(st, "mdn_chunk_fwd_keep_states")
+        return o, Sf, Mf, states, workspace
     if layer_ops is None:
         st = lib().mdn_chunk_fwd(ctypes.byref(p), *tail)
     else:
@@ -292,6 +309,20 @@ def chunk_fwd(q, k, v, beta, log_alpha, log_mu, eta=None, *, initial_S=None, ini
     if st != 0:
         raise MdnError(st, "mdn_chunk_fwd_fused" if layer_ops is not None else "mdn_chunk_fwd")
     return o, Sf, Mf
+
+
+def unpack_chunk_states(states: torch.Tensor, H: int):
+    """The buffer of mdn_chunk_fwd_keep_states as float32 tensors (S, M) of shape [slots, H, dk, dv] (dk = dv = 128):
+    undoes the transposition and the 128-byte swizzle of the shared-memory image."""
+    raw = states.view(torch.bfloat16).view(-1, H, 2, 2, 128, 8, 8)          # slot, head, S|M, key half, row, piece, elem
+    rows = torch.arange(128, device=states.device)
+    piece = torch.arange(8, device=states.device)
+    src = (piece[None, :] ^ (rows[:, None] & 7))                            # where logical piece c of row r lies
+    idx = src[None, None, None, None, :, :, None].expand(raw.shape[0], H, 2, 2, 128, 8, 8)
+    logical = torch.gather(raw, 5, idx).reshape(-1, H, 2, 2, 128, 64)       # [.., row = value index, 64 key indices]
+    full = torch.cat([logical[:, :, :, 0], logical[:, :, :, 1]], dim=-1)    # [slot, H, 2, value, key]
+    full = full.transpose(-1, -2).float()                                   # [slot, H, 2, key, value]
+    return full[:, :, 0].contiguous(), full[:, :, 1].contiguous()
 
 
 def chunk_bwd(q, k, v, beta, log_alpha, log_mu, eta, d_o, *, initial_S=None, initial_M=None, cu_seqlens=None,

@@ -84,6 +84,7 @@ struct Bars {
   uint64_t m3;        // MMA-3 done                                                    (commit)
   uint64_t mo;        // MMA-3' done                                                   (commit)
   uint64_t zu;        // U (intra-chunk output) has been read                           (256)
+  uint64_t dump;      // the producer has copied S_b, M_b of a chunk out (chunk-state dump only)   (1)
   uint64_t pn[4];     // fused output step: the staged rows of a token group are in shared memory (128 each)
 };
 
@@ -112,6 +113,12 @@ struct ChainArgs {
   const float* post_w;        // [dv] or NULL
   const void* post_g;         // [B,T,H,dv] bf16
   float post_eps;
+  // training / backward support
+  uint8_t* dump;              // NULL, or [slot][H][65536]: the bf16 copies S_b^T | M_b^T of the state at the START of
+                              // every chunk, as they lie in shared memory (two [128 x 128 B] swizzled blocks each)
+  int state_only;             // no output terms (no Q, W loads, no output MMAs): states (and the dump) only
+  int end_scalars_in_rk;      // (abar_C, b_C, mubar_C) of a chunk are entries 0..2 of coefficient vector 6, not the
+                              // last entries of vectors 0, 1, 5 (the adjoint chain decouples them)
   uint32_t drop_lo;           // debug: bit 0 R, 1 V~_S/V~_M, 2 V~ (output), 3 W: leave that operand's lo part out
   long long* timeline;        // debug: CTA 0 writes clock64() at [chunk*32 + event] (NULL = off)
 };
@@ -136,7 +143,9 @@ template <> __device__ __forceinline__ void stage_o<__nv_bfloat16>(uint8_t* tile
   reinterpret_cast<__nv_bfloat16*>(tile)[r * kD + d] = __float2bfloat16_rn(x);
 }
 
-template <typename TO, bool kLayer>
+// kTrain compiles in the chunk-state dump, the state-only switch and the decoupled end-of-chunk scalars (the plain
+// forward's instantiation stays as it is: its schedule is fragile, a runtime test of these options cost it 2 %)
+template <typename TO, bool kLayer, bool kTrain = false>
 __global__ void __launch_bounds__(Roles<token_groups(kLayer)>::kThreads, 1) chain_tensor_kernel(const ChainArgs a,
                                                                   const __grid_constant__ CUtensorMap map_q,
                                                                   const __grid_constant__ CUtensorMap map_k,
@@ -208,6 +217,9 @@ __global__ void __launch_bounds__(Roles<token_groups(kLayer)>::kThreads, 1) chai
       Sfp = base; Mfp = base + kMat;
     }
   }
+  if constexpr (kTrain) {
+    if (a.state_only) write_o = false;
+  }
 
   const uint32_t s_base = smem_u32(smem);
   const uint32_t b_full0 = smem_u32(&bars.full[0]), b_full1 = smem_u32(&bars.full[1]);
@@ -215,7 +227,7 @@ __global__ void __launch_bounds__(Roles<token_groups(kLayer)>::kThreads, 1) chai
   const uint32_t b_sb = smem_u32(&bars.sb), b_m1 = smem_u32(&bars.m1), b_mq = smem_u32(&bars.mq);
   const uint32_t b_r = smem_u32(&bars.r), b_m2 = smem_u32(&bars.m2);
   const uint32_t b_v1 = smem_u32(&bars.v1), b_v2 = smem_u32(&bars.v2), b_m3 = smem_u32(&bars.m3);
-  const uint32_t b_mo = smem_u32(&bars.mo), b_zu = smem_u32(&bars.zu);
+  const uint32_t b_mo = smem_u32(&bars.mo), b_zu = smem_u32(&bars.zu), b_dump = smem_u32(&bars.dump);
   // kLayer = false compiles the layer operations out: the plain forward keeps its instruction count
   const bool qk_on = kLayer && a.qk_on;
   const bool post = kLayer && a.post_on && write_o;
@@ -228,6 +240,7 @@ __global__ void __launch_bounds__(Roles<token_groups(kLayer)>::kThreads, 1) chai
     mbar_init(b_sb, kArrivals); mbar_init(b_r, kArrivals); mbar_init(b_v1, kArrivals);
     mbar_init(b_v2, kArrivals);
     mbar_init(b_zu, kArrivals);
+    mbar_init(b_dump, 1);
     mbar_init(b_m1, 1); mbar_init(b_mq, 1); mbar_init(b_m2, 1); mbar_init(b_m3, 1); mbar_init(b_mo, 1);
     for (int i = 0; i < kTG; ++i) mbar_init(smem_u32(&bars.pn[i]), 128);
     mbar_fence_init();
@@ -312,6 +325,14 @@ __global__ void __launch_bounds__(Roles<token_groups(kLayer)>::kThreads, 1) chai
           }
           MDN_MARK(c, kEvTmaIssued);
           issued = c + 1;
+        }
+        if (kTrain && a.dump != nullptr && c >= 1 && c <= nch) {   // the state copies of chunk c - 1 (handed over long ago)
+          MDN_WAIT(b_sb, (c - 1) & 1);
+          uint8_t* dst = a.dump + ((size_t)(sq.slot0 + c - 1) * H + h) * 65536;
+          for (int b = 0; b < 4; ++b) bulk_store(dst + b * 16384, s_base + kOffSb + b * 16384, 16384);
+          tma_store_commit();
+          tma_store_wait_read();
+          mbar_arrive(b_dump);
         }
       }
       if (!ok) {   // giving up: let the copies already in flight land before the CTA exits
@@ -455,7 +476,12 @@ __global__ void __launch_bounds__(Roles<token_groups(kLayer)>::kThreads, 1) chai
       if (c < nch) {
         MDN_WAIT((c & 1) ? b_full1 : b_full0, (c >> 1) & 1);
         const float* cf = reinterpret_cast<const float*>(smem + kOffStage + (c & 1) * kStageBytes + kStCoef);
-        al = cf[kAbar * C + C - 1]; bl = cf[kB * C + C - 1]; ml = cf[kMubar * C + C - 1];
+        if (kTrain && a.end_scalars_in_rk) {
+          al = cf[kRk * C + 0]; bl = cf[kRk * C + 1]; ml = cf[kRk * C + 2];
+        } else {
+          al = cf[kAbar * C + C - 1]; bl = cf[kB * C + C - 1]; ml = cf[kMubar * C + C - 1];
+        }
+        if (kTrain && a.dump != nullptr && c > 0) MDN_WAIT(b_dump, (c - 1) & 1);
         MDN_MARK(c, kEvFullSeen);
       }
       __syncwarp();
@@ -881,6 +907,7 @@ cudaError_t launch_chain_tensor(const Plan& pl, const void* q, const void* k, co
   a.drop_lo = drop ? (uint32_t)atoi(drop) : 0u;
   const char* tl = getenv("MDN_DEBUG_TIMELINE");   // device address of an int64 buffer, [chunks][32]
   a.timeline = tl ? reinterpret_cast<long long*>(strtoull(tl, nullptr, 0)) : nullptr;
+  a.dump = pl.chain_dump; a.state_only = pl.chain_state_only; a.end_scalars_in_rk = pl.chain_end_scalars_in_rk;
   a.seg_G = 0; a.seg_phase = 0;
   a.seg_E = a.seg_Psi = a.seg_PhiS = a.seg_PhiM = nullptr;
   const unsigned chains = (unsigned)pl.geom.num_seqs * p.H;
@@ -895,6 +922,12 @@ cudaError_t launch_chain_tensor(const Plan& pl, const void* q, const void* k, co
     return e;
   };
   auto launch = [&](unsigned grid) -> cudaError_t {
+    const bool train = a.dump != nullptr || a.state_only || a.end_scalars_in_rk;
+    if (train) {   // plain forward with the training options (no layer operations there)
+      if (layer) return cudaErrorInvalidValue;
+      return p.o_dtype == MDN_BF16 ? launch_as(chain_tensor_kernel<__nv_bfloat16, false, true>, grid)
+                                   : launch_as(chain_tensor_kernel<float, false, true>, grid);
+    }
     if (p.o_dtype == MDN_BF16)
       return layer ? launch_as(chain_tensor_kernel<__nv_bfloat16, true>, grid)
                    : launch_as(chain_tensor_kernel<__nv_bfloat16, false>, grid);

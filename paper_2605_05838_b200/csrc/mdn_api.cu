@@ -193,6 +193,33 @@ mdn_status mdn_chunk_fwd(const mdn_params* p, const void* q, const void* k, cons
   return run_forward(pl, q, k, v, beta, log_alpha, log_mu, eta, initial_S, initial_M, o, final_S, final_M);
 }
 
+// ---- the forward that keeps the chunk-start states (tensor path, serial chain)
+size_t mdn_chunk_states_bytes(const mdn_params* p) {
+  mdn_ws_layout lay;
+  if (check_params(p) != MDN_OK || make_layout(*p, &lay) != MDN_OK) return 0;
+  if (resolve_path(*p) != MDN_PATH_TENSOR) return 0;
+  return (size_t)lay.num_slots * p->H * 65536;
+}
+
+mdn_status mdn_chunk_fwd_keep_states(const mdn_params* p, const void* q, const void* k, const void* v,
+                                     const float* beta, const float* log_alpha, const float* log_mu,
+                                     const float* eta, const float* initial_S, const float* initial_M,
+                                     const int32_t* cu_seqlens, void* o, float* final_S, float* final_M,
+                                     void* chunk_states, void* workspace, size_t workspace_bytes,
+                                     void* cuda_stream) {
+  t_last_launches = 0;
+  if (check_params(p) != MDN_OK) return check_params(p);
+  if (resolve_path(*p) != MDN_PATH_TENSOR) return MDN_ERR_UNSUPPORTED;
+  if (!chunk_states || !aligned(chunk_states, 1024)) return MDN_ERR_INVALID_ARG;
+  mdn_params ps = *p;
+  ps.segments = 1;
+  Plan pl;
+  mdn_status st = make_plan(&ps, cu_seqlens, workspace, workspace_bytes, cuda_stream, &pl);
+  if (st != MDN_OK) return st;
+  pl.chain_dump = static_cast<uint8_t*>(chunk_states);
+  return run_forward(pl, q, k, v, beta, log_alpha, log_mu, eta, initial_S, initial_M, o, final_S, final_M);
+}
+
 // ---- the forward with layer operations
 static bool ops_active(const mdn_layer_ops* ops) {
   return ops && (ops->raw_gates || ops->qk_norm || ops->out_norm_gate);

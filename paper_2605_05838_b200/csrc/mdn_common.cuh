@@ -132,6 +132,10 @@ struct Plan {
   GateParam gp;    // layer operations the kernels absorb (all off for the plain forward)
   QkNorm qk;
   OutPost post;
+  // chain kernel options of the training / backward entry points (all off for the forward)
+  uint8_t* chain_dump = nullptr;
+  int chain_state_only = 0;
+  int chain_end_scalars_in_rk = 0;
 };
 
 // Launchers (one per .cu file).  Each returns the CUDA error of its launches and adds
