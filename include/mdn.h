@@ -285,6 +285,39 @@ mdn_status mdn_chunk_fwd_keep_states(const mdn_params* p,
                                      void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * Chunk-parallel backward, stage 1 (Section 3.2 differentiated chunk by chunk): the adjoint of the inter-chunk
+ * state recurrence.  With dS', dM' the adjoints of the carried pair at the END of a chunk,
+ *     dV~ = W^T dO + g_S . (K dS') - g_M . (K dM'),   dR = T^T dV~,
+ *     dS  = abar_C dS' - K^T (abar . dR) + scale Q^T (abar . dO),
+ *     dM  = -b_C dS' + mubar_C dM' + K^T (p . dR) - scale Q^T (b . dO)
+ * walk the chunks of every sequence from the last to the first.  This has the shape of the forward's own chunk step
+ * with the roles of S and M exchanged, so it is run by the forward's chain kernel on an extended problem (per
+ * chunk a real step and a step that adds the two Q terms) built from the forward's workspace.
+ *   p, q, k: the forward call's (tensor path, fixed-length input, o_dtype bf16); d_o = dL/do, [B,T,H,dv] bf16;
+ *   d_final_S, d_final_M: dL/d(final states), [B,H,dk,dv] float32 or NULL (zero);
+ *   fwd_workspace: the workspace of an mdn_chunk_fwd_keep_states call with the same p and inputs, untouched since
+ *     (T, W and the coefficient vectors are read from it);
+ *   adjoint_states: DEVICE buffer of mdn_bwd_adjoint_states_bytes(p) bytes, 1024-byte aligned.  Per sequence and
+ *     head it receives 2 x nchunks entries of 65536 bytes in the layout of mdn_chunk_fwd_keep_states with dM^T in
+ *     the first half and dS^T in the second: entry 2 (nchunks - 1 - c) is the adjoint pair at the END of chunk c,
+ *     entry 2 (nchunks - 1 - c) + 1 the pair after chunk c's K terms and before its Q terms;
+ *   d_initial_S, d_initial_M: dL/d(initial states), [B,H,dk,dv] float32, or NULL;
+ *   workspace: mdn_bwd_state_chain_workspace_bytes(p) bytes, 1024-byte aligned, scratch.
+ * The gradients of q, k, v and the gates follow from these adjoint states and the kept forward states chunk by chunk,
+ * in parallel; that stage is not part of this entry point (mdn_chunk_bwd is the complete backward).
+ */
+size_t mdn_bwd_state_chain_workspace_bytes(const mdn_params* p);
+size_t mdn_bwd_adjoint_states_bytes(const mdn_params* p);
+
+mdn_status mdn_bwd_state_chain(const mdn_params* p,
+                               const void* q, const void* k, const void* d_o,
+                               const float* d_final_S, const float* d_final_M,
+                               void* fwd_workspace, size_t fwd_workspace_bytes,
+                               void* adjoint_states,
+                               float* d_initial_S, float* d_initial_M,
+                               void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * Backward of mdn_chunk_fwd (Section 3.1: the training pass differentiates the same recurrence; like the paper's
  * kernels this keeps no per-token states and rebuilds them from per-chunk checkpoints):
  * given d_o = dL/do ([B,T,H,dv], o_dtype) and optionally dL/d(final_S), dL/d(final_M) ([N,H,dk,dv] float32, NULL =

@@ -154,11 +154,14 @@ def chain_backward(q, k, v, beta, log_alpha, log_mu, eta, d_o, scale=1.0, S0=Non
     dM = np.zeros((dk, dv)) if dM_final is None else np.asarray(dM_final, dtype=f8)
     out = dict(dq=np.zeros((T_, dk)), dk=np.zeros((T_, dk)), dv=np.zeros((T_, dv)), dbeta=np.zeros(T_),
                dlog_alpha=np.zeros(T_), dlog_mu=np.zeros(T_), deta=np.zeros(T_))
+    adj_end = []                # (dS', dM') at the END of every chunk, last chunk first
     for sl, S_c, M_c, co, fw in reversed(saved):
+        adj_end.append((dS, dM))
         g = chunk_backward(q[sl], k[sl], S_c, M_c, co, fw, d_o[sl], dS, dM, alpha[sl], mu[sl], beta[sl], eta[sl], scale)
         out["dq"][sl], out["dk"][sl], out["dv"][sl] = g["dQ"], g["dK"], g["dV"]
         for name in ("dbeta", "dlog_alpha", "dlog_mu", "deta"):
             out[name][sl] = g[name]
         dS, dM = g["dS"], g["dM"]
     out["dS0"], out["dM0"] = dS, dM
+    out["adj_end"] = adj_end[::-1]      # indexed by chunk
     return out

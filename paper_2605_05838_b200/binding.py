@@ -86,6 +86,12 @@ def lib() -> ctypes.CDLL:
         L.mdn_chunk_states_bytes.argtypes = [P]
         L.mdn_chunk_fwd_keep_states.restype = ctypes.c_int
         L.mdn_chunk_fwd_keep_states.argtypes = [P] + [vp] * 14 + [vp, ctypes.c_size_t, vp]
+        L.mdn_bwd_state_chain_workspace_bytes.restype = ctypes.c_size_t
+        L.mdn_bwd_state_chain_workspace_bytes.argtypes = [P]
+        L.mdn_bwd_adjoint_states_bytes.restype = ctypes.c_size_t
+        L.mdn_bwd_adjoint_states_bytes.argtypes = [P]
+        L.mdn_bwd_state_chain.restype = ctypes.c_int
+        L.mdn_bwd_state_chain.argtypes = [P] + [vp] * 6 + [ctypes.c_size_t] + [vp] * 4 + [ctypes.c_size_t, vp]
         L.mdn_chunk_bwd.restype = ctypes.c_int
         L.mdn_chunk_bwd.argtypes = [P] + [vp] * 22 + [vp, ctypes.c_size_t, vp]
         L.mdn_chunk_bwd_workspace_bytes.restype = ctypes.c_size_t
@@ -323,6 +329,29 @@ def unpack_chunk_states(states: torch.Tensor, H: int):
     full = torch.cat([logical[:, :, :, 0], logical[:, :, :, 1]], dim=-1)    # [slot, H, 2, value, key]
     full = full.transpose(-1, -2).float()                                   # [slot, H, 2, key, value]
     return full[:, :, 0].contiguous(), full[:, :, 1].contiguous()
+
+
+def bwd_state_chain(q, k, d_o, fwd_workspace, *, v_dim: int, d_final_S=None, d_final_M=None,
+                    scale: Optional[float] = None, want_initial: bool = True):
+    """mdn_bwd_state_chain after a chunk_fwd(..., keep_chunk_states=True) call whose workspace is `fwd_workspace`.
+    Returns (adjoint_states, d_initial_S, d_initial_M): the raw adjoint-state buffer (2 entries per chunk, see
+    include/mdn.h; unpack_chunk_states gives (dM, dS) per entry) and the initial states' gradients."""
+    B, T, H, dk = q.shape
+    p = make_params(q, d_o, scale=scale, o_dtype=torch.bfloat16, path="tensor")
+    nbytes = int(lib().mdn_bwd_adjoint_states_bytes(ctypes.byref(p)))
+    need = int(lib().mdn_bwd_state_chain_workspace_bytes(ctypes.byref(p)))
+    if nbytes == 0 or need == 0:
+        raise MdnError(2, "mdn_bwd_state_chain_workspace_bytes")
+    adj = torch.empty(nbytes, dtype=torch.uint8, device=q.device)
+    ws = torch.empty(need, dtype=torch.uint8, device=q.device)
+    dS0 = torch.empty((B, H, dk, v_dim), dtype=torch.float32, device=q.device) if want_initial else None
+    dM0 = torch.empty((B, H, dk, v_dim), dtype=torch.float32, device=q.device) if want_initial else None
+    st = lib().mdn_bwd_state_chain(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(d_o), _ptr(d_final_S), _ptr(d_final_M),
+                                   _ptr(fwd_workspace), fwd_workspace.numel(), _ptr(adj), _ptr(dS0), _ptr(dM0),
+                                   _ptr(ws), ws.numel(), _stream())
+    if st != 0:
+        raise MdnError(st, "mdn_bwd_state_chain")
+    return adj, dS0, dM0
 
 
 def chunk_bwd(q, k, v, beta, log_alpha, log_mu, eta, d_o, *, initial_S=None, initial_M=None, cu_seqlens=None,

@@ -1,0 +1,160 @@
+// Chunk-parallel backward, first stage: the adjoint of the inter-chunk state recurrence (Section 3.2, the chunk
+// form  S' = abar_C S - b_C M + K^T (g_S . V~),  M' = mubar_C M - K^T (g_M . V~),  V~ = T (V - abar . K S + p . K M),
+// O = scale (abar . Q S - b . Q M) + W V~, differentiated with respect to the carried pair).
+//
+// With dS', dM' the adjoints at the END of a chunk,
+//     dV~ = W^T dO + g_S . (K dS') - g_M . (K dM'),      dR = T^T dV~,
+//     dS  = abar_C dS' - K^T (abar . dR) + scale Q^T (abar . dO),
+//     dM  = -b_C dS' + mubar_C dM' + K^T (p . dR) - scale Q^T (b . dO).
+// This has the shape of the forward's own chunk step with the roles exchanged (dM for S, dS for M):
+//     X = K dM', Y = K dS',  "R" = V' - g_M . X + g_S . Y  with V' = W^T dO,  "V~" = T^T "R" = dR,
+//     dM = mubar_C dM' - b_C dS' + K^T (p . dR),   dS = abar_C dS' - K^T (abar . dR),
+// followed by a second, state-only step that adds the two Q terms (K := Q, V := dO, T := I, no decay).
+// So the adjoint chain is run by the forward's chain kernel itself (chain_tensor.cu, training instantiation) on an
+// "extended" problem built here: per chunk, in REVERSE chunk order, a real step and an injection step.  This file
+// holds the kernel that builds that problem from the forward's workspace (T, W, coefficient vectors) and q, k, dO.
+#include "mdn_common.cuh"
+#include "tc_utils.cuh"
+
+namespace mdn {
+namespace {
+
+using namespace tc;
+
+constexpr int kD = 128;
+constexpr int kPrepThreads = 256;
+constexpr int LWT = C + 4;   // floats per row of W^T in shared memory
+
+struct PrepArgs {
+  ChunkGeom g;                      // the forward's geometry (fixed length)
+  const __nv_bfloat16* q; const __nv_bfloat16* k; const __nv_bfloat16* d_o;
+  const float* coef;                // forward: [slot][H][MDN_NUM_COEF][64]
+  const __nv_bfloat16* T;           // forward: [slot][H][64][64]
+  const __nv_bfloat16* W;           // forward: hi part, lo part w_lo_offset elements later
+  size_t w_lo_offset;
+  float scale;
+  // the extended problem: 2 chunks per forward chunk, sequence s = rows [s * 2 nch * 64, ..) of k_ext, v_ext
+  __nv_bfloat16* k_ext; __nv_bfloat16* v_ext;   // [B][2 nch 64][H][128]
+  float* coef_ext;                  // [2 slots][H][MDN_NUM_COEF][64]
+  __nv_bfloat16* T_ext;             // [2 slots][H][64][64]
+};
+
+__global__ void __launch_bounds__(kPrepThreads) bwd_prep_kernel(PrepArgs a) {
+  extern __shared__ __align__(16) uint8_t smem_raw[];
+  float* Wt = reinterpret_cast<float*>(smem_raw);                          // [64][LWT]: W^T, fp32 (hi + lo)
+  __nv_bfloat16* Tt = reinterpret_cast<__nv_bfloat16*>(Wt + C * LWT);      // [64][64 + 8]: T
+  const int slot = blockIdx.x / a.g.H, h = blockIdx.x % a.g.H, H = a.g.H;
+  const SlotInfo si = slot_info(a.g, slot);
+  if (si.seq < 0) return;
+  const int tid = threadIdx.x;
+  const int nch = a.g.chunks_per_seq;
+  // extended chunk indices of this forward chunk: the real step, then the injection step
+  const int e_real = si.seq * 2 * nch + 2 * (nch - 1 - si.local), e_inj = e_real + 1;
+  const size_t mat = ((size_t)slot * H + h) * C * C;
+
+  // ---- W^T (fp32) and T into shared memory
+  for (int idx = tid; idx < C * C; idx += kPrepThreads) {
+    const int r = idx >> 6, i = idx & 63;
+    Wt[i * LWT + r] = __bfloat162float(a.W[mat + idx]) + __bfloat162float(a.W[a.w_lo_offset + mat + idx]);
+    Tt[r * (C + 8) + i] = a.T[mat + idx];
+  }
+  __syncthreads();
+
+  // ---- V' = W^T dO for the real step, dO itself for the injection step; thread = (value column j, half of the rows i)
+  {
+    const int j = tid & (kD - 1), half = tid >> 7;
+    float docol[C];
+#pragma unroll
+    for (int r = 0; r < C; ++r)
+      docol[r] = r < si.n ? __bfloat162float(a.d_o[((size_t)(si.tok0 + r) * H + h) * kD + j]) : 0.f;
+    for (int i = half * 32; i < half * 32 + 32; ++i) {
+      float acc = 0.f;
+#pragma unroll
+      for (int r4 = 0; r4 < C; r4 += 4) {
+        const float4 w4 = *reinterpret_cast<const float4*>(Wt + i * LWT + r4);
+        acc = fmaf(w4.x, docol[r4], acc); acc = fmaf(w4.y, docol[r4 + 1], acc);
+        acc = fmaf(w4.z, docol[r4 + 2], acc); acc = fmaf(w4.w, docol[r4 + 3], acc);
+      }
+      a.v_ext[((size_t)(e_real * C + i) * H + h) * kD + j] = __float2bfloat16_rn(i < si.n ? acc : 0.f);
+    }
+#pragma unroll
+    for (int r = 0; r < C; ++r)
+      if ((r >> 5) == half) a.v_ext[((size_t)(e_inj * C + r) * H + h) * kD + j] = __float2bfloat16_rn(docol[r]);
+  }
+
+  // ---- keys of the two steps: k (real), q (injection); rows past the end of a short chunk are zero
+  for (int idx = tid; idx < C * (kD / 8); idx += kPrepThreads) {
+    const int r = idx >> 4, c8 = (idx & 15) * 8;
+    uint4 kv = make_uint4(0u, 0u, 0u, 0u), qv = kv;
+    if (r < si.n) {
+      kv = *reinterpret_cast<const uint4*>(a.k + ((size_t)(si.tok0 + r) * H + h) * kD + c8);
+      qv = *reinterpret_cast<const uint4*>(a.q + ((size_t)(si.tok0 + r) * H + h) * kD + c8);
+    }
+    *reinterpret_cast<uint4*>(a.k_ext + ((size_t)(e_real * C + r) * H + h) * kD + c8) = kv;
+    *reinterpret_cast<uint4*>(a.k_ext + ((size_t)(e_inj * C + r) * H + h) * kD + c8) = qv;
+  }
+
+  // ---- T^T (real), I (injection)
+  const size_t mat_r = ((size_t)e_real * H + h) * C * C, mat_i = ((size_t)e_inj * H + h) * C * C;
+  for (int idx = tid; idx < C * C; idx += kPrepThreads) {
+    const int r = idx >> 6, i = idx & 63;
+    a.T_ext[mat_r + idx] = Tt[i * (C + 8) + r];
+    a.T_ext[mat_i + idx] = __float2bfloat16_rn(r == i ? 1.f : 0.f);
+  }
+
+  // ---- coefficient vectors.  Real step: abar' = g_M, p' = g_S, g_S' = p, g_M' = abar, end-of-chunk scalars
+  // (mubar_C, b_C, abar_C) in vector 6.  Injection step: no decay, g_S' = -scale b, g_M' = -scale abar.
+  const float* cf = a.coef + ((size_t)slot * H + h) * MDN_NUM_COEF * C;
+  float* cr = a.coef_ext + ((size_t)e_real * H + h) * MDN_NUM_COEF * C;
+  float* ci = a.coef_ext + ((size_t)e_inj * H + h) * MDN_NUM_COEF * C;
+  for (int idx = tid; idx < MDN_NUM_COEF * C; idx += kPrepThreads) {
+    const int vec = idx >> 6, r = idx & 63;
+    const bool live = r < si.n;
+    float xr = 0.f, xi = 0.f;
+    switch (vec) {
+      case kAbar: xr = live ? cf[kGM * C + r] : 0.f; break;
+      case kAlphaBPrev: xr = live ? cf[kGS * C + r] : 0.f; break;
+      case kGS: xr = live ? cf[kAlphaBPrev * C + r] : 0.f; xi = live ? -a.scale * cf[kB * C + r] : 0.f; break;
+      case kGM: xr = live ? cf[kAbar * C + r] : 0.f; xi = live ? -a.scale * cf[kAbar * C + r] : 0.f; break;
+      case kRk:
+        xr = r == 0 ? cf[kMubar * C + C - 1] : r == 1 ? cf[kB * C + C - 1] : r == 2 ? cf[kAbar * C + C - 1] : 1.f;
+        xi = r == 1 ? 0.f : 1.f;
+        break;
+      case kRq: xr = 1.f; xi = 1.f; break;
+      default: break;   // b, mubar and the per-token gates are not read by a state-only run
+    }
+    cr[idx] = xr;
+    ci[idx] = xi;
+  }
+}
+
+}  // namespace
+
+size_t bwd_prep_smem_bytes() { return (size_t)C * LWT * 4 + (size_t)C * (C + 8) * 2; }
+
+cudaError_t launch_bwd_prep(const Plan& fwd, const void* q, const void* k, const void* d_o, void* k_ext, void* v_ext,
+                            float* coef_ext, void* T_ext, int* launches) {
+  PrepArgs a;
+  a.g = fwd.geom;
+  a.q = static_cast<const __nv_bfloat16*>(q);
+  a.k = static_cast<const __nv_bfloat16*>(k);
+  a.d_o = static_cast<const __nv_bfloat16*>(d_o);
+  a.coef = reinterpret_cast<const float*>(fwd.ws + fwd.lay.off_coef);
+  a.T = reinterpret_cast<const __nv_bfloat16*>(fwd.ws + fwd.lay.off_T);
+  a.W = reinterpret_cast<const __nv_bfloat16*>(fwd.ws + fwd.lay.off_W);
+  a.w_lo_offset = (size_t)fwd.geom.num_slots * fwd.p.H * C * C;
+  a.scale = fwd.p.scale;
+  a.k_ext = static_cast<__nv_bfloat16*>(k_ext);
+  a.v_ext = static_cast<__nv_bfloat16*>(v_ext);
+  a.coef_ext = coef_ext;
+  a.T_ext = static_cast<__nv_bfloat16*>(T_ext);
+  const size_t smem = bwd_prep_smem_bytes();
+  cudaError_t e = cudaFuncSetAttribute(bwd_prep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  bwd_prep_kernel<<<dim3((unsigned)fwd.geom.num_slots * fwd.p.H), dim3(kPrepThreads), smem, fwd.stream>>>(a);
+  e = cudaGetLastError();
+  if (e == cudaSuccess) ++*launches;
+  return e;
+}
+
+}  // namespace mdn

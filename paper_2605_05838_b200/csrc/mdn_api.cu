@@ -220,6 +220,73 @@ mdn_status mdn_chunk_fwd_keep_states(const mdn_params* p, const void* q, const v
   return run_forward(pl, q, k, v, beta, log_alpha, log_mu, eta, initial_S, initial_M, o, final_S, final_M);
 }
 
+// ---- chunk-parallel backward, stage 1: the adjoint of the inter-chunk state recurrence
+struct AdjLayout { mdn_params pe; mdn_ws_layout le; uint64_t k_ext, v_ext, ws_ext, total; };
+
+static mdn_status adj_layout(const mdn_params* p, AdjLayout* a) {
+  mdn_status st = check_params(p);
+  if (st != MDN_OK) return st;
+  if (resolve_path(*p) != MDN_PATH_TENSOR || p->num_seqs > 0) return MDN_ERR_UNSUPPORTED;
+  a->pe = *p;
+  a->pe.T = 2 * ((p->T + p->chunk - 1) / p->chunk) * p->chunk;   // a real and an injection step per chunk
+  a->pe.segments = 1;
+  a->pe.path = MDN_PATH_TENSOR;
+  st = make_layout(a->pe, &a->le);
+  if (st != MDN_OK) return st;
+  const uint64_t rows = (uint64_t)p->B * a->pe.T * p->H * p->dk * 2;
+  uint64_t off = 0;
+  auto take = [&](uint64_t bytes) { uint64_t at = off; off = align_up(off + bytes, 1024); return at; };
+  a->k_ext = take(rows); a->v_ext = take(rows); a->ws_ext = take(a->le.total_bytes); a->total = off;
+  return MDN_OK;
+}
+
+size_t mdn_bwd_state_chain_workspace_bytes(const mdn_params* p) {
+  AdjLayout a;
+  return adj_layout(p, &a) == MDN_OK ? (size_t)a.total : 0;
+}
+
+size_t mdn_bwd_adjoint_states_bytes(const mdn_params* p) {
+  AdjLayout a;
+  return adj_layout(p, &a) == MDN_OK ? (size_t)a.le.num_slots * p->H * 65536 : 0;
+}
+
+mdn_status mdn_bwd_state_chain(const mdn_params* p, const void* q, const void* k, const void* d_o,
+                               const float* d_final_S, const float* d_final_M, void* fwd_workspace,
+                               size_t fwd_workspace_bytes, void* adjoint_states, float* d_initial_S,
+                               float* d_initial_M, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  t_last_launches = 0;
+  AdjLayout al;
+  mdn_status st = adj_layout(p, &al);
+  if (st != MDN_OK) return st;
+  if (!q || !k || !d_o || !adjoint_states || !aligned(adjoint_states, 1024)) return MDN_ERR_INVALID_ARG;
+  if (!aligned(q, 16) || !aligned(k, 16) || !aligned(d_o, 16)) return MDN_ERR_INVALID_ARG;
+  if (p->o_dtype != MDN_BF16) return MDN_ERR_UNSUPPORTED;   // d_o is read as bf16
+  if (!workspace || workspace_bytes < al.total || !aligned(workspace, 1024)) return MDN_ERR_WORKSPACE;
+  mdn_params pf = *p;
+  pf.segments = 1;
+  Plan fwd;
+  st = make_plan(&pf, nullptr, fwd_workspace, fwd_workspace_bytes, cuda_stream, &fwd);
+  if (st != MDN_OK) return st;
+  char* w = static_cast<char*>(workspace);
+  Plan ext;
+  st = make_plan(&al.pe, nullptr, w + al.ws_ext, al.le.total_bytes, cuda_stream, &ext);
+  if (st != MDN_OK) return st;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemsetAsync(ext.ws + ext.lay.off_status, 0, 16, s) != cudaSuccess) return MDN_ERR_CUDA;
+  cudaError_t e = launch_bwd_prep(fwd, q, k, d_o, w + al.k_ext, w + al.v_ext,
+                                  reinterpret_cast<float*>(ext.ws + ext.lay.off_coef), ext.ws + ext.lay.off_T,
+                                  &t_last_launches);
+  if (e != cudaSuccess) { t_last_cuda_error = (int)e; return MDN_ERR_CUDA; }
+  // the forward's chain kernel on the extended problem, roles exchanged: its "S" is dM, its "M" is dS
+  ext.chain_dump = static_cast<uint8_t*>(adjoint_states);
+  ext.chain_state_only = 1;
+  ext.chain_end_scalars_in_rk = 1;
+  e = launch_chain_tensor(ext, w + al.k_ext, w + al.k_ext, w + al.v_ext, d_final_M, d_final_S, w + al.v_ext,
+                          d_initial_M, d_initial_S, &t_last_launches);
+  if (e != cudaSuccess) { t_last_cuda_error = (int)e; return MDN_ERR_CUDA; }
+  return MDN_OK;
+}
+
 // ---- the forward with layer operations
 static bool ops_active(const mdn_layer_ops* ops) {
   return ops && (ops->raw_gates || ops->qk_norm || ops->out_norm_gate);

@@ -141,6 +141,9 @@ struct Plan {
 // Launchers (one per .cu file).  Each returns the CUDA error of its launches and adds
 // the number of kernels it enqueued to *launches.
 cudaError_t launch_chunk_map(const Plan& pl, int* launches);
+// bwd_chunk.cu: builds the extended problem of the adjoint state chain from the forward's workspace
+cudaError_t launch_bwd_prep(const Plan& fwd, const void* q, const void* k, const void* d_o, void* k_ext, void* v_ext,
+                            float* coef_ext, void* T_ext, int* launches);
 cudaError_t launch_coeff_scan(const Plan& pl, const float* beta, const float* log_alpha,
                               const float* log_mu, const float* eta, int* launches);
 // The layer operations as passes of their own (layer_ops.cu).

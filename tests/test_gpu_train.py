@@ -64,3 +64,49 @@ def test_keep_chunk_states(mdn, name, kw):
     fs, fm = bf16_floor(S_ref), bf16_floor(M_ref)
     print("chunk-start states (%s, %d slots): S %.3e (bf16 floor %.3e) M %.3e (floor %.3e)" % (name, n, es, fs, em, fm))
     assert es <= fs + TOL_OVER_FLOOR and em <= fm + TOL_OVER_FLOOR
+
+
+@pytest.mark.parametrize("T, with_final", [(64 * 4 + 20, True), (64 * 3, False)])
+def test_bwd_state_chain(mdn, T, with_final):
+    """Adjoint of the inter-chunk state recurrence (stage 1 of the chunk-parallel backward) against the fp64 chunk-form
+    backward oracle: the adjoint pair at the end of every chunk and the gradients of the initial states."""
+    import torch
+    from oracle import chunkwise_bwd as ob
+    w = wl.Workload("adj_chain", B=2, T=T, H=2, dk=128, dv=128, dtype="bf16", init_state_std=0.1, seed=83)
+    inp = wl.make_inputs(w)
+    t = to_torch(inp)
+    rng = np.random.default_rng(5)
+    d_o = wl.round_to_bf16(rng.standard_normal((w.B, w.T, w.H, w.dv)).astype(np.float32))
+    dSf = (0.1 * rng.standard_normal((w.B, w.H, w.dk, w.dv))).astype(np.float32) if with_final else None
+    dMf = (0.1 * rng.standard_normal((w.B, w.H, w.dk, w.dv))).astype(np.float32) if with_final else None
+    dev = lambda x, dt=torch.float32: None if x is None else torch.from_numpy(x).to("cuda").to(dt)
+    _, _, _, _, ws = mdn.chunk_fwd(t["q"], t["k"], t["v"], t["beta"], t["log_alpha"], t["log_mu"], t["eta"],
+                                   initial_S=t["initial_S"], initial_M=t["initial_M"], scale=inp["scale"], path="tensor",
+                                   keep_chunk_states=True)
+    adj, dS0, dM0 = mdn.bwd_state_chain(t["q"], t["k"], dev(d_o, torch.bfloat16), ws, v_dim=w.dv, d_final_S=dev(dSf),
+                                        d_final_M=dev(dMf), scale=inp["scale"])
+    torch.cuda.synchronize()
+    dM_e, dS_e = mdn.unpack_chunk_states(adj, w.H)       # entries: first half = dM, second half = dS
+    dM_e, dS_e = dM_e.cpu().numpy(), dS_e.cpu().numpy()
+    nch = (T + 63) // 64
+    ref_S, ref_M, got_S, got_M = [], [], [], []
+    ref_S0, ref_M0 = np.zeros((w.B, w.H, w.dk, w.dv)), np.zeros((w.B, w.H, w.dk, w.dv))
+    for b in range(w.B):
+        for h in range(w.H):
+            g = ob.chain_backward(inp["q"][b, :, h], inp["k"][b, :, h], inp["v"][b, :, h], inp["beta"][b, :, h],
+                                  inp["log_alpha"][b, :, h], inp["log_mu"][b, :, h], inp["eta"][b, :, h], d_o[b, :, h],
+                                  scale=inp["scale"], S0=inp["S0"][b, h], M0=inp["M0"][b, h],
+                                  dS_final=None if dSf is None else dSf[b, h], dM_final=None if dMf is None else dMf[b, h])
+            ref_S0[b, h], ref_M0[b, h] = g["dS0"], g["dM0"]
+            for c in range(nch):
+                e = b * 2 * nch + 2 * (nch - 1 - c)
+                ref_S.append(g["adj_end"][c][0]); ref_M.append(g["adj_end"][c][1])
+                got_S.append(dS_e[e, h]); got_M.append(dM_e[e, h])
+    ref_S, ref_M, got_S, got_M = map(np.stack, (ref_S, ref_M, got_S, got_M))
+    es, em = rel_err(got_S, ref_S), rel_err(got_M, ref_M)
+    e0s, e0m = rel_err(dS0.cpu().numpy(), ref_S0), rel_err(dM0.cpu().numpy(), ref_M0)
+    fs, fm = bf16_floor(ref_S), bf16_floor(ref_M)
+    print("adjoint states at chunk ends: dS %.3e (bf16 floor %.3e) dM %.3e (floor %.3e); d_initial: dS0 %.3e dM0 %.3e"
+          % (es, fs, em, fm, e0s, e0m))
+    assert es <= fs + 1e-2 and em <= fm + 1e-2
+    assert max(e0s, e0m) <= 2e-2
