@@ -318,6 +318,31 @@ mdn_status mdn_bwd_state_chain(const mdn_params* p,
                                void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * The chunk-parallel backward (Section 3.2 differentiated chunk by chunk, on the tensor cores): the same gradients
+ * as mdn_chunk_bwd, computed as
+ *   1. the forward's state recurrence again, keeping (S, M) at the start of every chunk (mdn_chunk_fwd_keep_states
+ *      without the output terms),
+ *   2. the adjoint state recurrence (mdn_bwd_state_chain),
+ *   3. per (chunk, head), in parallel: dV = dR, dQ, dK, the adjoints of the coefficient vectors and of the two
+ *      masks, and from those the gate gradients by the recurrences of Eq. 10 in reverse.
+ * Arguments as mdn_chunk_bwd (no cu_seqlens: fixed-length input only).  Tensor path only: bf16 q, k, v, bf16 d_o,
+ * dk = dv = 128; MDN_ERR_UNSUPPORTED otherwise.  Operands are bf16 / tf32 with fp32 accumulation, so the gradients
+ * carry the forward's bf16-level error (see the tests), not mdn_chunk_bwd's fp32 exactness.  deta,
+ * d_initial_S, d_initial_M may be NULL.  Workspace: mdn_chunk_bwd_chunked_workspace_bytes(p), 1024-byte aligned.
+ */
+size_t mdn_chunk_bwd_chunked_workspace_bytes(const mdn_params* p);
+
+mdn_status mdn_chunk_bwd_chunked(const mdn_params* p,
+                                 const void* q, const void* k, const void* v,
+                                 const float* beta, const float* log_alpha, const float* log_mu, const float* eta,
+                                 const float* initial_S, const float* initial_M,
+                                 const void* d_o, const float* d_final_S, const float* d_final_M,
+                                 float* dq, float* dk, float* dv,
+                                 float* dbeta, float* dlog_alpha, float* dlog_mu, float* deta,
+                                 float* d_initial_S, float* d_initial_M,
+                                 void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * Backward of mdn_chunk_fwd (Section 3.1: the training pass differentiates the same recurrence; like the paper's
  * kernels this keeps no per-token states and rebuilds them from per-chunk checkpoints):
  * given d_o = dL/do ([B,T,H,dv], o_dtype) and optionally dL/d(final_S), dL/d(final_M) ([N,H,dk,dv] float32, NULL =

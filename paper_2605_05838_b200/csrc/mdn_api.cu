@@ -287,6 +287,71 @@ mdn_status mdn_bwd_state_chain(const mdn_params* p, const void* q, const void* k
   return MDN_OK;
 }
 
+// ---- the chunk-parallel backward: state-only forward keeping the chunk states, adjoint chain, per-chunk stage
+struct ChunkedBwdLayout { AdjLayout al; mdn_ws_layout lf; uint64_t ws_fwd, fwd_states, adj_states, stage, total; };
+
+static mdn_status chunked_bwd_layout(const mdn_params* p, ChunkedBwdLayout* c) {
+  mdn_status st = adj_layout(p, &c->al);
+  if (st != MDN_OK) return st;
+  mdn_params pf = *p;
+  pf.segments = 1;
+  st = make_layout(pf, &c->lf);
+  if (st != MDN_OK) return st;
+  uint64_t off = 0;
+  auto take = [&](uint64_t bytes) { uint64_t at = off; off = align_up(off + bytes, 1024); return at; };
+  c->ws_fwd = take(c->lf.total_bytes);
+  c->fwd_states = take((uint64_t)c->lf.num_slots * p->H * 65536);
+  c->adj_states = take((uint64_t)c->al.le.num_slots * p->H * 65536);
+  c->stage = take(c->al.total);
+  c->total = off;
+  return MDN_OK;
+}
+
+size_t mdn_chunk_bwd_chunked_workspace_bytes(const mdn_params* p) {
+  ChunkedBwdLayout c;
+  return chunked_bwd_layout(p, &c) == MDN_OK ? (size_t)c.total : 0;
+}
+
+mdn_status mdn_chunk_bwd_chunked(const mdn_params* p, const void* q, const void* k, const void* v, const float* beta,
+                                 const float* log_alpha, const float* log_mu, const float* eta,
+                                 const float* initial_S, const float* initial_M, const void* d_o,
+                                 const float* d_final_S, const float* d_final_M, float* dq, float* dk, float* dv,
+                                 float* dbeta, float* dlog_alpha, float* dlog_mu, float* deta, float* d_initial_S,
+                                 float* d_initial_M, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  t_last_launches = 0;
+  ChunkedBwdLayout c;
+  mdn_status st = chunked_bwd_layout(p, &c);
+  if (st != MDN_OK) return st;
+  if (p->o_dtype != MDN_BF16) return MDN_ERR_UNSUPPORTED;
+  if (!q || !k || !v || !d_o || !beta || !log_alpha || !log_mu || !dq || !dk || !dv || !dbeta || !dlog_alpha || !dlog_mu)
+    return MDN_ERR_INVALID_ARG;
+  if (!workspace || workspace_bytes < c.total || !aligned(workspace, 1024)) return MDN_ERR_WORKSPACE;
+  char* w = static_cast<char*>(workspace);
+  // 1. the forward's states (no output terms), kept per chunk; T, W and the coefficient vectors stay in ws_fwd
+  mdn_params pf = *p;
+  pf.segments = 1;
+  Plan fwd;
+  st = make_plan(&pf, nullptr, w + c.ws_fwd, c.lf.total_bytes, cuda_stream, &fwd);
+  if (st != MDN_OK) return st;
+  fwd.chain_dump = reinterpret_cast<uint8_t*>(w + c.fwd_states);
+  fwd.chain_state_only = 1;
+  st = run_forward(fwd, q, k, v, beta, log_alpha, log_mu, eta, initial_S, initial_M, w + c.stage /* o: never written */,
+                   nullptr, nullptr);
+  if (st != MDN_OK) return st;
+  const int launches_fwd = t_last_launches;
+  // 2. the adjoint state chain
+  st = mdn_bwd_state_chain(p, q, k, d_o, d_final_S, d_final_M, w + c.ws_fwd, c.lf.total_bytes, w + c.adj_states,
+                           d_initial_S, d_initial_M, w + c.stage, c.al.total, cuda_stream);
+  if (st != MDN_OK) return st;
+  t_last_launches += launches_fwd;
+  // 3. per (chunk, head): dq, dk, dv and the gate gradients
+  cudaError_t e = launch_bwd_chunk_par(fwd, q, k, v, d_o, beta, log_alpha, log_mu, eta, w + c.fwd_states,
+                                       w + c.adj_states, w + c.stage + c.al.v_ext, dq, dk, dv, dbeta, dlog_alpha,
+                                       dlog_mu, deta, &t_last_launches);
+  if (e != cudaSuccess) { t_last_cuda_error = (int)e; return MDN_ERR_CUDA; }
+  return MDN_OK;
+}
+
 // ---- the forward with layer operations
 static bool ops_active(const mdn_layer_ops* ops) {
   return ops && (ops->raw_gates || ops->qk_norm || ops->out_norm_gate);

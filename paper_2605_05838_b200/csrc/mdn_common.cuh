@@ -141,6 +141,11 @@ struct Plan {
 // Launchers (one per .cu file).  Each returns the CUDA error of its launches and adds
 // the number of kernels it enqueued to *launches.
 cudaError_t launch_chunk_map(const Plan& pl, int* launches);
+// bwd_chunk_par.cu: gradients of q, k, v and the gates per (chunk, head) from the kept states and the adjoint states
+cudaError_t launch_bwd_chunk_par(const Plan& fwd, const void* q, const void* k, const void* v, const void* d_o,
+                                 const float* beta, const float* log_alpha, const float* log_mu, const float* eta,
+                                 const void* fwd_states, const void* adj_states, const void* v_ext, float* dq, float* dk,
+                                 float* dv, float* dbeta, float* dlog_alpha, float* dlog_mu, float* deta, int* launches);
 // bwd_chunk.cu: builds the extended problem of the adjoint state chain from the forward's workspace
 cudaError_t launch_bwd_prep(const Plan& fwd, const void* q, const void* k, const void* d_o, void* k_ext, void* v_ext,
                             float* coef_ext, void* T_ext, int* launches);
