@@ -12,8 +12,10 @@
 // sum_j dR_rj X_rj = sum_d K_rd (dR S^T)_rd reuses a product that dK needs anyway), the adjoints of the two masks
 // d Geta = scale tril(dO V~^T) o (Q K^T), d G^- = dA o (K K^T), and from those the gate gradients by running the
 // coefficient recurrences of Eq. 10 in reverse.
-// All products are tf32 tensor-core MMAs (fp32 accumulate) on operands in shared memory: q, k, dO and the states as
-// the bf16 values they are, the intermediates (V~, dR, DW, DA, T, W) in fp32.  One 256-thread CTA per (chunk, head).
+// Every product is a warp-level bf16 tensor-core MMA (m16n8k16, fp32 accumulate) fed by ldmatrix from shared memory:
+// q, k, dO, T and the states are bf16 as they stand; every intermediate that comes out of an accumulator (R, dV~, V~,
+// dR, DW, DA) is kept as a bf16 hi + lo pair (16 mantissa bits through two MMAs), W as the hi + lo pair the forward
+// wrote.  One 256-thread CTA per (chunk, head).
 #include "mdn_common.cuh"
 #include "tc_utils.cuh"
 
@@ -21,75 +23,85 @@ namespace mdn {
 namespace {
 
 using namespace tc;
+typedef __nv_bfloat16 bf16;
 
 constexpr int kD = 128;
 constexpr int kThreads = 256;
-constexpr int LT = kD + 8;    // bf16 elements per row of a 64 x 128 bf16 tile and of a state (row = value index)
-constexpr int LF = kD + 4;    // floats per row of a 64 x 128 fp32 tile
-constexpr int L64 = C + 4;    // floats per row of a 64 x 64 matrix
+constexpr int LT = kD + 8;    // bf16 elements per row of a 64 x 128 tile and of a state (272 B: ldmatrix conflict-free)
+constexpr int L6 = C + 8;     // bf16 elements per row of a 64 x 64 matrix (144 B)
+constexpr int LG = C + 4;     // floats per row of a 64 x 64 fp32 matrix
 
 // shared memory map (bytes)
-constexpr uint32_t kOffSt = 0;                                   // state, bf16 [128 (value j)][LT (key d)]; later d Geta, d G^-
-constexpr uint32_t kOffK = kOffSt + kD * LT * 2;                 // k, q, dO tiles, bf16 [64][LT]
-constexpr uint32_t kOffQ = kOffK + C * LT * 2;
-constexpr uint32_t kOffDO = kOffQ + C * LT * 2;
-constexpr uint32_t kOffVt = kOffDO + C * LT * 2;                 // V~, fp32 [64][LF]; later DW
-constexpr uint32_t kOffDR = kOffVt + C * LF * 4;                 // dR, fp32 [64][LF]; later DA
-constexpr uint32_t kOffT = kOffDR + C * LF * 4;                  // T, fp32 [64][L64]
-constexpr uint32_t kOffTmp = kOffT + C * L64 * 4;                // R / dV~ (fp32 [64][LF]); later gamma and m ([64][L64] each)
-constexpr uint32_t kOffVec = kOffTmp + 2 * C * L64 * 4;          // vectors, 24 x [64] floats
+constexpr uint32_t kTile = C * LT * 2, kMat6 = C * L6 * 2, kMatF = C * LG * 4;
+constexpr uint32_t kOffSt = 0;                        // state, bf16 [128 (value j)][LT (key d)]; later d Geta, d G^- (fp32)
+constexpr uint32_t kOffK = kOffSt + kD * LT * 2;      // k, q, dO
+constexpr uint32_t kOffQ = kOffK + kTile;
+constexpr uint32_t kOffDO = kOffQ + kTile;
+constexpr uint32_t kOffVt = kOffDO + kTile;           // V~ hi, lo; later DW hi, lo
+constexpr uint32_t kOffDR = kOffVt + 2 * kTile;       // dR hi, lo; later DA hi, lo
+constexpr uint32_t kOffT = kOffDR + 2 * kTile;        // T, bf16 [64][L6]
+constexpr uint32_t kOffTmp = kOffT + kMat6;           // R / dV~ hi, lo; W hi, lo; later gamma, m (fp32 [64][LG] each)
+constexpr uint32_t kOffVec = kOffTmp + 2 * kTile;     // vectors, 24 x [64] floats
 constexpr uint32_t kSmem = kOffVec + 24 * C * 4;
-static_assert(2 * C * L64 * 4 >= C * LF * 4 && kD * LT * 2 >= 2 * C * L64 * 4, "overlays");
+static_assert(2 * kTile >= 2 * kMatF && kD * LT * 2 >= 2 * kMatF && 2 * kTile >= 2 * kMat6, "overlays");
 static_assert(kSmem <= 232448, "shared memory");
 
-// vectors
 enum Vec : int { vAbar = 0, vB, vP, vGS, vGM, vMubar, vAlpha, vBeta, vMu, vEta, vBprev,
                  vdAbar, vdB, vdP, vdGS, vdGM, vdMubar, vdAlpha, vdBeta, vdMu, vdEta, vRed };
 
 struct ParArgs {
   ChunkGeom g;
-  const __nv_bfloat16* q; const __nv_bfloat16* k; const __nv_bfloat16* v; const __nv_bfloat16* d_o;
+  const bf16* q; const bf16* k; const bf16* v; const bf16* d_o;
   const float* beta; const float* log_alpha; const float* log_mu; const float* eta;
-  const float* coef; const __nv_bfloat16* T; const __nv_bfloat16* W; size_t w_lo_offset;
-  const uint8_t* fwd_states; const uint8_t* adj_states; const __nv_bfloat16* v_ext;
+  const float* coef; const bf16* T; const bf16* W; size_t w_lo_offset;
+  const uint8_t* fwd_states; const uint8_t* adj_states;
   float scale;
   float* dq; float* dk; float* dv; float* dbeta; float* dlog_alpha; float* dlog_mu; float* deta;
 };
 
-__device__ __forceinline__ uint32_t tf32_of(float x) {
-  uint32_t r;
-  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
-  return r;
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
 }
-__device__ __forceinline__ void mma_tf32(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
   asm volatile(
-      "mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
       "{%0, %1, %2, %3};"
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
-// acc[mt][nt] (+)= A[m0 + 16 mt .., k] B[k, n0 + 8 nt ..] over k < K.  A(m, k), B(k, n) return floats from shared
-// memory (any layout: a transposed operand is an accessor with its indices exchanged).  g = lane / 4, t = lane % 4.
-template <int MT, int NT, class FA, class FB>
-__device__ __forceinline__ void warp_mma(float (&acc)[MT][NT][4], FA A, FB B, int K, int m0, int n0, int g, int t) {
-  for (int k0 = 0; k0 < K; k0 += 8) {
-    uint32_t af[MT][4], bf[NT][2];
+// A bf16 operand in shared memory: byte address of element (0, 0), row stride in bytes, and how it is stored:
+// for A, trans = false means [m][k] (k contiguous), true means [k][m]; for B, false means [n][k], true means [k][n].
+struct Opnd { uint32_t base; uint32_t ld; bool trans; };
+
+// acc[mt][nt] += A[m0 + 16 mt .., k] B[k, n0 + 8 nt ..] over k < K (a multiple of 16); NT even.
+template <int MT, int NT>
+__device__ __forceinline__ void warp_mma(float (&acc)[MT][NT][4], Opnd A, Opnd B, int K, int m0, int n0, int lane) {
+  const int l7 = lane & 7, q1 = (lane >> 3) & 1, q2 = lane >> 4;
+  for (int k0 = 0; k0 < K; k0 += 16) {
+    uint32_t af[MT][4], bfr[NT / 2][4];
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt) {
-      const int m = m0 + 16 * mt + g;
-      af[mt][0] = tf32_of(A(m, k0 + t)); af[mt][1] = tf32_of(A(m + 8, k0 + t));
-      af[mt][2] = tf32_of(A(m, k0 + t + 4)); af[mt][3] = tf32_of(A(m + 8, k0 + t + 4));
+      if (!A.trans) ldsm_x4(A.base + (m0 + 16 * mt + l7 + q1 * 8) * A.ld + (k0 + q2 * 8) * 2, af[mt]);
+      else ldsm_x4_t(A.base + (k0 + q2 * 8 + l7) * A.ld + (m0 + 16 * mt + q1 * 8) * 2, af[mt]);
     }
 #pragma unroll
-    for (int nt = 0; nt < NT; ++nt) {
-      const int n = n0 + 8 * nt + g;
-      bf[nt][0] = tf32_of(B(k0 + t, n)); bf[nt][1] = tf32_of(B(k0 + t + 4, n));
+    for (int p = 0; p < NT / 2; ++p) {
+      if (!B.trans) ldsm_x4(B.base + (n0 + 16 * p + l7 + q2 * 8) * B.ld + (k0 + q1 * 8) * 2, bfr[p]);
+      else ldsm_x4_t(B.base + (k0 + q1 * 8 + l7) * B.ld + (n0 + 16 * p + q2 * 8) * 2, bfr[p]);
     }
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
-      for (int nt = 0; nt < NT; ++nt) mma_tf32(acc[mt][nt], af[mt], bf[nt][0], bf[nt][1]);
+      for (int p = 0; p < NT / 2; ++p) {
+        mma_bf16(acc[mt][2 * p], af[mt], bfr[p][0], bfr[p][1]);
+        mma_bf16(acc[mt][2 * p + 1], af[mt], bfr[p][2], bfr[p][3]);
+      }
   }
 }
 
@@ -111,23 +123,40 @@ template <int MT, int NT, class F> __device__ __forceinline__ void for_frag(int 
 #pragma unroll
       for (int e = 0; e < 4; ++e) f(mt, nt, e, m0 + 16 * mt + g + 8 * (e >> 1), n0 + 8 * nt + 2 * t + (e & 1));
 }
+// ... and its column pairs: f(mt, nt, half, row, col) with the values acc[mt][nt][2 half], [2 half + 1] at col, col + 1
+template <int MT, int NT, class F> __device__ __forceinline__ void for_pair(int m0, int n0, int g, int t, F f) {
+#pragma unroll
+  for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+      for (int hf = 0; hf < 2; ++hf) f(mt, nt, hf, m0 + 16 * mt + g + 8 * hf, n0 + 8 * nt + 2 * t);
+}
 
 __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
   extern __shared__ __align__(16) uint8_t smem[];
-  __nv_bfloat16* sSt = reinterpret_cast<__nv_bfloat16*>(smem + kOffSt);
-  __nv_bfloat16* sK = reinterpret_cast<__nv_bfloat16*>(smem + kOffK);
-  __nv_bfloat16* sQ = reinterpret_cast<__nv_bfloat16*>(smem + kOffQ);
-  __nv_bfloat16* sDO = reinterpret_cast<__nv_bfloat16*>(smem + kOffDO);
-  float* sVt = reinterpret_cast<float*>(smem + kOffVt);
-  float* sDR = reinterpret_cast<float*>(smem + kOffDR);
-  float* sT = reinterpret_cast<float*>(smem + kOffT);
-  float* sTmp = reinterpret_cast<float*>(smem + kOffTmp);
-  float* sGam = sTmp;                       // gamma [64][L64] (after R / dV~ are done with the area)
-  float* sMm = sTmp + C * L64;              // m [64][L64]
-  float* sDW = sVt;                         // DW [64][L64] (after V~ is done)
-  float* sDA = sDR;                         // DA
-  float* sdGe = reinterpret_cast<float*>(smem + kOffSt);            // d Geta [64][L64] (after the states are done)
-  float* sdGm = sdGe + C * L64;             // d G^-
+  const uint32_t sb = smem_u32(smem);
+  bf16* sSt = reinterpret_cast<bf16*>(smem + kOffSt);
+  bf16* sK = reinterpret_cast<bf16*>(smem + kOffK);
+  bf16* sQ = reinterpret_cast<bf16*>(smem + kOffQ);
+  bf16* sDO = reinterpret_cast<bf16*>(smem + kOffDO);
+  bf16* sVtH = reinterpret_cast<bf16*>(smem + kOffVt);
+  bf16* sVtL = sVtH + C * LT;
+  bf16* sDRH = reinterpret_cast<bf16*>(smem + kOffDR);
+  bf16* sDRL = sDRH + C * LT;
+  bf16* sT = reinterpret_cast<bf16*>(smem + kOffT);
+  bf16* sTmpH = reinterpret_cast<bf16*>(smem + kOffTmp);      // R, then dV~ (hi, lo)
+  bf16* sTmpL = sTmpH + C * LT;
+  bf16* sWH = sTmpH;                                          // W (hi, lo) between R and dV~
+  bf16* sWL = sWH + C * L6;
+  float* sGam = reinterpret_cast<float*>(smem + kOffTmp);     // gamma, m (after dV~ is done with the area)
+  float* sMm = sGam + C * LG;
+  bf16* sDWH = reinterpret_cast<bf16*>(smem + kOffVt);        // DW, DA (after V~, dR are done)
+  bf16* sDWL = sDWH + C * L6;
+  bf16* sDAH = reinterpret_cast<bf16*>(smem + kOffDR);
+  bf16* sDAL = sDAH + C * L6;
+  float* sdGe = reinterpret_cast<float*>(smem + kOffSt);      // d Geta, d G^- (after the states are done)
+  float* sdGm = sdGe + C * LG;
   float* vec = reinterpret_cast<float*>(smem + kOffVec);
   auto V = [&](int which) { return vec + which * C; };
 
@@ -145,13 +174,35 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
   const uint8_t* imgdS = imgdM + 32768;
   const float scale = a.scale;
 
+  // operands
+  const Opnd oK{sb + kOffK, LT * 2, false}, oK_t{sb + kOffK, LT * 2, true};
+  const Opnd oQ{sb + kOffQ, LT * 2, false}, oQ_t{sb + kOffQ, LT * 2, true};
+  const Opnd oDO{sb + kOffDO, LT * 2, false}, oDO_t{sb + kOffDO, LT * 2, true};
+  const Opnd oSt_dk{sb + kOffSt, LT * 2, false};   // B(k = key d, n = value j) = S[d][j], stored [j][d]
+  const Opnd oSt_dv{sb + kOffSt, LT * 2, true};    // B(k = value j, n = key d)
+  const Opnd oVtH{sb + kOffVt, LT * 2, false}, oVtL{sb + kOffVt + kTile, LT * 2, false};
+  const Opnd oDRH{sb + kOffDR, LT * 2, false}, oDRL{sb + kOffDR + kTile, LT * 2, false};
+  const Opnd oT{sb + kOffT, L6 * 2, false}, oT_t{sb + kOffT, L6 * 2, true};
+  const Opnd oTmpH_t{sb + kOffTmp, LT * 2, true}, oTmpL_t{sb + kOffTmp + kTile, LT * 2, true};
+  const Opnd oWH_t{sb + kOffTmp, L6 * 2, true}, oWL_t{sb + kOffTmp + kMat6, L6 * 2, true};
+  const Opnd oDWH{sb + kOffVt, L6 * 2, false}, oDWL{sb + kOffVt + kMat6, L6 * 2, false};
+  const Opnd oDWH_t{sb + kOffVt, L6 * 2, true}, oDWL_t{sb + kOffVt + kMat6, L6 * 2, true};
+  const Opnd oDAH{sb + kOffDR, L6 * 2, false}, oDAL{sb + kOffDR + kMat6, L6 * 2, false};
+  const Opnd oDAH_t{sb + kOffDR, L6 * 2, true}, oDAL_t{sb + kOffDR + kMat6, L6 * 2, true};
+
   auto tok = [&](int r) { return (size_t)(si.tok0 + r) * H + h; };
-  auto load_tile = [&](__nv_bfloat16* dst, const __nv_bfloat16* src) {
+  auto load_tile = [&](bf16* dst, const bf16* src) {
     for (int idx = tid; idx < C * 16; idx += kThreads) {
       const int r = idx >> 4, c8 = (idx & 15) * 8;
       uint4 x = make_uint4(0u, 0u, 0u, 0u);
       if (r < n) x = *reinterpret_cast<const uint4*>(src + tok(r) * kD + c8);
       *reinterpret_cast<uint4*>(dst + r * LT + c8) = x;
+    }
+  };
+  auto load_mat64 = [&](bf16* dst, const bf16* src) {   // a [64][64] bf16 matrix -> [64][L6]
+    for (int idx = tid; idx < C * 8; idx += kThreads) {
+      const int r = idx >> 3, c8 = (idx & 7) * 8;
+      *reinterpret_cast<uint4*>(dst + r * L6 + c8) = *reinterpret_cast<const uint4*>(src + r * C + c8);
     }
   };
   // state image (value index j x key index d, two swizzled blocks) -> sSt[j][d]
@@ -176,16 +227,17 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
     for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
     return s;   // per warp; lane 0 adds it where it belongs
   };
-  auto bfv = [](const __nv_bfloat16* p, int i) { return __bfloat162float(p[i]); };
-  auto AK = [&](int m, int k) { return bfv(sK, m * LT + k); };
-  auto AQ = [&](int m, int k) { return bfv(sQ, m * LT + k); };
-  auto ADO = [&](int m, int k) { return bfv(sDO, m * LT + k); };
-  auto AVt = [&](int m, int k) { return sVt[m * LF + k]; };
-  auto ADR = [&](int m, int k) { return sDR[m * LF + k]; };
-  auto BSt_dk = [&](int k, int nn) { return bfv(sSt, nn * LT + k); };   // contraction over the key index: B(d, j) = S[d][j]
-  auto BSt_dv = [&](int k, int nn) { return bfv(sSt, k * LT + nn); };   // contraction over the value index: B(j, d) = S[d][j]
-  // row sums of G o X over the warp's 32 columns, added to a vector (X(r, c) from a tile)
-  auto add_rowsum = [&](float (&G)[2][4][4], auto X, float* dst, float sign) {
+  // a warp's 32 x 32 block of a 64 x 128 result -> bf16 hi + lo tiles (rows past the chunk's end are zero)
+  auto put_split = [&](float (&acc)[2][4][4], bf16* hi, bf16* lo) {
+    for_pair<2, 4>(m0, n0, g, t, [&](int mt, int nt, int hf, int r, int c) {
+      uint32_t ph = 0u, pl = 0u;
+      if (r < n) split_pack_bf16(acc[mt][nt][2 * hf], acc[mt][nt][2 * hf + 1], ph, pl);
+      *reinterpret_cast<uint32_t*>(hi + r * LT + c) = ph;
+      *reinterpret_cast<uint32_t*>(lo + r * LT + c) = pl;
+    });
+  };
+  // row sums of G o X over the warp's 32 columns, added to a vector (X: a bf16 tile, k or q)
+  auto add_rowsum = [&](float (&G)[2][4][4], const bf16* X, float* dst, float sign) {
 #pragma unroll
     for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
@@ -194,9 +246,9 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
         float s = 0.f;
 #pragma unroll
         for (int nt = 0; nt < 4; ++nt) {
-          const int c = n0 + 8 * nt + 2 * t;
-          s = fmaf(G[mt][nt][2 * hf], X(r, c), s);
-          s = fmaf(G[mt][nt][2 * hf + 1], X(r, c + 1), s);
+          const uint32_t x2 = *reinterpret_cast<const uint32_t*>(X + r * LT + n0 + 8 * nt + 2 * t);
+          s = fmaf(G[mt][nt][2 * hf], __uint_as_float(x2 << 16), s);
+          s = fmaf(G[mt][nt][2 * hf + 1], __uint_as_float(x2 & 0xffff0000u), s);
         }
         s += __shfl_xor_sync(0xffffffffu, s, 1);
         s += __shfl_xor_sync(0xffffffffu, s, 2);
@@ -220,7 +272,7 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
   load_tile(sK, a.k);
   load_tile(sQ, a.q);
   load_tile(sDO, a.d_o);
-  for (int idx = tid; idx < C * C; idx += kThreads) sT[(idx >> 6) * L64 + (idx & 63)] = __bfloat162float(a.T[mat + idx]);
+  load_mat64(sT, a.T + mat);
   load_state(imgS);
   __syncthreads();
   if (tid < C) V(vBprev)[tid] = tid > 0 ? V(vB)[tid - 1] : 0.f;
@@ -232,22 +284,26 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
   {
     float X[2][4][4], Y[2][4][4];
     zero(X); zero(Y);
-    warp_mma(X, AK, BSt_dk, kD, m0, n0, g, t);
+    warp_mma(X, oK, oSt_dk, kD, m0, n0, lane);
     __syncthreads();
     load_state(imgM);
     __syncthreads();
-    warp_mma(Y, AK, BSt_dk, kD, m0, n0, g, t);
+    warp_mma(Y, oK, oSt_dk, kD, m0, n0, lane);
     for_frag<2, 4>(m0, n0, g, t, [&](int mt, int nt, int e, int r, int c) {
       const float v = r < n ? __bfloat162float(a.v[tok(r) * kD + c]) : 0.f;
-      sTmp[r * LF + c] = v - V(vAbar)[r] * X[mt][nt][e] + V(vP)[r] * Y[mt][nt][e];
+      X[mt][nt][e] = v - V(vAbar)[r] * X[mt][nt][e] + V(vP)[r] * Y[mt][nt][e];
     });
+    put_split(X, sTmpH, sTmpL);
     __syncthreads();
     float Vt[2][4][4];
     zero(Vt);
-    warp_mma(Vt, [&](int m, int k) { return sT[m * L64 + k]; }, [&](int k, int nn) { return sTmp[k * LF + nn]; }, C, m0, n0, g, t);
-    for_frag<2, 4>(m0, n0, g, t, [&](int mt, int nt, int e, int r, int c) { sVt[r * LF + c] = r < n ? Vt[mt][nt][e] : 0.f; });
+    warp_mma(Vt, oT, oTmpH_t, C, m0, n0, lane);
+    warp_mma(Vt, oT, oTmpL_t, C, m0, n0, lane);
+    put_split(Vt, sVtH, sVtL);
   }
-  __syncthreads();
+  __syncthreads();   // V~ complete; R has been read
+  load_mat64(sWH, a.W + mat);
+  load_mat64(sWL, a.W + a.w_lo_offset + mat);
 
   // ---- with dM' (the end-of-chunk adjoint of M): K dM', the g_M term of dK and its coefficient adjoint
   float KdM[2][4][4];
@@ -258,49 +314,50 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
     if (lane == 0) atomicAdd(V(vdMubar) + n - 1, s);
   }
   __syncthreads();
-  warp_mma(KdM, AK, BSt_dk, kD, m0, n0, g, t);
+  warp_mma(KdM, oK, oSt_dk, kD, m0, n0, lane);
   {
     float G[2][4][4];
     zero(G);
-    warp_mma(G, AVt, BSt_dv, kD, m0, n0, g, t);                       // V~ dM'^T
+    warp_mma(G, oVtH, oSt_dv, kD, m0, n0, lane);                      // V~ dM'^T
+    warp_mma(G, oVtL, oSt_dv, kD, m0, n0, lane);
     for_frag<2, 4>(m0, n0, g, t, [&](int mt, int nt, int e, int r, int c) { dK[mt][nt][e] -= V(vGM)[r] * G[mt][nt][e]; });
-    add_rowsum(G, AK, V(vdGM), -1.f);
+    add_rowsum(G, sK, V(vdGM), -1.f);
   }
   __syncthreads();
-  // ---- with dS': K dS', the g_S term of dK, dV~ and dR
+  // ---- with dS': K dS', the g_S term of dK, dV~ = W^T dO + g_S.(K dS') - g_M.(K dM'), dR = T^T dV~
   load_state(imgdS);
   {
     const float s1 = dot_images(imgdS, imgS), s2 = dot_images(imgdS, imgM);   // d abar_C = <dS', S>, d b_C = -<dS', M>
     if (lane == 0) { atomicAdd(V(vdAbar) + n - 1, s1); atomicAdd(V(vdB) + n - 1, -s2); }
   }
   __syncthreads();
-  // W (hi + lo, fp32) into the free area: W^T dO is formed here in fp32 (the adjoint chain's bf16 copy of it would
-  // put one bf16 rounding of the dominant term into dV)
-  for (int idx = tid; idx < C * C; idx += kThreads)
-    sTmp[(idx >> 6) * L64 + (idx & 63)] = __bfloat162float(a.W[mat + idx]) + __bfloat162float(a.W[a.w_lo_offset + mat + idx]);
-  __syncthreads();
   {
-    float KdS[2][4][4], G[2][4][4], Vp[2][4][4];
-    zero(KdS); zero(G); zero(Vp);
-    warp_mma(Vp, [&](int m, int k) { return sTmp[k * L64 + m]; }, [&](int k, int nn) { return bfv(sDO, k * LT + nn); }, C, m0, n0, g, t);
-    __syncthreads();   // W has been read: the area takes dV~
-    warp_mma(KdS, AK, BSt_dk, kD, m0, n0, g, t);
-    warp_mma(G, AVt, BSt_dv, kD, m0, n0, g, t);                       // V~ dS'^T
-    for_frag<2, 4>(m0, n0, g, t, [&](int mt, int nt, int e, int r, int c) { dK[mt][nt][e] += V(vGS)[r] * G[mt][nt][e]; });
-    add_rowsum(G, AK, V(vdGS), 1.f);
+    float Z[2][4][4], G[2][4][4];
+    zero(Z); zero(G);
+    warp_mma(Z, oWH_t, oDO_t, C, m0, n0, lane);                       // W^T dO
+    warp_mma(Z, oWL_t, oDO_t, C, m0, n0, lane);
+    float KdS[2][4][4];
+    zero(KdS);
+    warp_mma(KdS, oK, oSt_dk, kD, m0, n0, lane);
+    warp_mma(G, oVtH, oSt_dv, kD, m0, n0, lane);                      // V~ dS'^T
+    warp_mma(G, oVtL, oSt_dv, kD, m0, n0, lane);
     for_frag<2, 4>(m0, n0, g, t, [&](int mt, int nt, int e, int r, int c) {
-      sTmp[r * LF + c] = Vp[mt][nt][e] + V(vGS)[r] * KdS[mt][nt][e] - V(vGM)[r] * KdM[mt][nt][e];
+      dK[mt][nt][e] += V(vGS)[r] * G[mt][nt][e];
+      Z[mt][nt][e] += V(vGS)[r] * KdS[mt][nt][e] - V(vGM)[r] * KdM[mt][nt][e];
     });
+    add_rowsum(G, sK, V(vdGS), 1.f);
+    __syncthreads();   // W has been read: the area takes dV~
+    put_split(Z, sTmpH, sTmpL);
   }
   __syncthreads();
   {
     float dR[2][4][4];
     zero(dR);
-    warp_mma(dR, [&](int m, int k) { return sT[k * L64 + m]; }, [&](int k, int nn) { return sTmp[k * LF + nn]; }, C, m0, n0, g, t);
+    warp_mma(dR, oT_t, oTmpH_t, C, m0, n0, lane);
+    warp_mma(dR, oT_t, oTmpL_t, C, m0, n0, lane);
+    put_split(dR, sDRH, sDRL);
     for_frag<2, 4>(m0, n0, g, t, [&](int mt, int nt, int e, int r, int c) {
-      const float x = r < n ? dR[mt][nt][e] : 0.f;
-      sDR[r * LF + c] = x;
-      if (r < n) a.dv[tok(r) * kD + c] = x;
+      if (r < n) a.dv[tok(r) * kD + c] = dR[mt][nt][e];
     });
   }
   __syncthreads();
@@ -311,13 +368,14 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
   {
     float G[2][4][4];
     zero(G);
-    warp_mma(G, ADO, BSt_dv, kD, m0, n0, g, t);
+    warp_mma(G, oDO, oSt_dv, kD, m0, n0, lane);
     for_frag<2, 4>(m0, n0, g, t, [&](int mt, int nt, int e, int r, int c) { dQ[mt][nt][e] += scale * V(vAbar)[r] * G[mt][nt][e]; });
-    add_rowsum(G, AQ, V(vdAbar), scale);
+    add_rowsum(G, sQ, V(vdAbar), scale);
     zero(G);
-    warp_mma(G, ADR, BSt_dv, kD, m0, n0, g, t);
+    warp_mma(G, oDRH, oSt_dv, kD, m0, n0, lane);
+    warp_mma(G, oDRL, oSt_dv, kD, m0, n0, lane);
     for_frag<2, 4>(m0, n0, g, t, [&](int mt, int nt, int e, int r, int c) { dK[mt][nt][e] -= V(vAbar)[r] * G[mt][nt][e]; });
-    add_rowsum(G, AK, V(vdAbar), -1.f);
+    add_rowsum(G, sK, V(vdAbar), -1.f);
   }
   __syncthreads();
   // ---- with M: dO M^T (dQ, d b), dR M^T (dK, d p)
@@ -326,13 +384,14 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
   {
     float G[2][4][4];
     zero(G);
-    warp_mma(G, ADO, BSt_dv, kD, m0, n0, g, t);
+    warp_mma(G, oDO, oSt_dv, kD, m0, n0, lane);
     for_frag<2, 4>(m0, n0, g, t, [&](int mt, int nt, int e, int r, int c) { dQ[mt][nt][e] -= scale * V(vB)[r] * G[mt][nt][e]; });
-    add_rowsum(G, AQ, V(vdB), -scale);
+    add_rowsum(G, sQ, V(vdB), -scale);
     zero(G);
-    warp_mma(G, ADR, BSt_dv, kD, m0, n0, g, t);
+    warp_mma(G, oDRH, oSt_dv, kD, m0, n0, lane);
+    warp_mma(G, oDRL, oSt_dv, kD, m0, n0, lane);
     for_frag<2, 4>(m0, n0, g, t, [&](int mt, int nt, int e, int r, int c) { dK[mt][nt][e] += V(vP)[r] * G[mt][nt][e]; });
-    add_rowsum(G, AK, V(vdP), 1.f);
+    add_rowsum(G, sK, V(vdP), 1.f);
   }
 
   // ---- gamma and m by the column recurrences of Eq. 10 (thread = column), into the area R / dV~ used
@@ -342,34 +401,54 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
     for (int r = 0; r < C; ++r) {
       if (r > i) m *= V(vMu)[r];
       if (r >= i) gam = V(vAlpha)[r] * gam + V(vBeta)[r] * m;
-      sGam[r * L64 + i] = r >= i ? gam : 0.f;
-      sMm[r * L64 + i] = r >= i ? m : 0.f;
+      sGam[r * LG + i] = r >= i ? gam : 0.f;
+      sMm[r * LG + i] = r >= i ? m : 0.f;
     }
   }
   // ---- the four 64 x 64 products
   float P1[2][2][4], P2[2][2][4], QK[2][2][4], KK[2][2][4];
   zero(P1); zero(P2); zero(QK); zero(KK);
-  warp_mma(P1, ADO, [&](int k, int nn) { return sVt[nn * LF + k]; }, kD, m0, n064, g, t);   // dO V~^T
-  warp_mma(P2, ADR, [&](int k, int nn) { return sVt[nn * LF + k]; }, kD, m0, n064, g, t);   // dR V~^T
-  warp_mma(QK, AQ, [&](int k, int nn) { return bfv(sK, nn * LT + k); }, kD, m0, n064, g, t);
-  warp_mma(KK, AK, [&](int k, int nn) { return bfv(sK, nn * LT + k); }, kD, m0, n064, g, t);
+  warp_mma(P1, oDO, oVtH, kD, m0, n064, lane);                        // dO V~^T
+  warp_mma(P1, oDO, oVtL, kD, m0, n064, lane);
+  warp_mma(P2, oDRH, oVtH, kD, m0, n064, lane);                       // dR V~^T
+  warp_mma(P2, oDRH, oVtL, kD, m0, n064, lane);
+  warp_mma(P2, oDRL, oVtH, kD, m0, n064, lane);
+  warp_mma(QK, oQ, oK, kD, m0, n064, lane);
+  warp_mma(KK, oK, oK, kD, m0, n064, lane);
   __syncthreads();   // V~, dR and the state are no longer read; gamma, m complete
-  for_frag<2, 2>(m0, n064, g, t, [&](int mt, int nt, int e, int r, int i) {
-    const bool live = r < n;
-    const float dOVt = (live && i <= r) ? P1[mt][nt][e] : 0.f;
-    const float dA = (live && i < r) ? -P2[mt][nt][e] : 0.f;
-    const float geta = sGam[r * L64 + i] * V(vEta)[i];
-    const float gmin = (r > 0) ? V(vAlpha)[r] * sGam[(r - 1) * L64 + i] * V(vEta)[i] : 0.f;
-    sDW[r * L64 + i] = scale * geta * dOVt;
-    sDA[r * L64 + i] = gmin * dA;
-    sdGe[r * L64 + i] = scale * dOVt * QK[mt][nt][e];
-    sdGm[r * L64 + i] = dA * KK[mt][nt][e];
+  for_pair<2, 2>(m0, n064, g, t, [&](int mt, int nt, int hf, int r, int i0) {
+    float dw[2], da[2];
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      const int i = i0 + e;
+      const bool live = r < n;
+      const float dOVt = (live && i <= r) ? P1[mt][nt][2 * hf + e] : 0.f;
+      const float dA = (live && i < r) ? -P2[mt][nt][2 * hf + e] : 0.f;
+      const float geta = sGam[r * LG + i] * V(vEta)[i];
+      const float gmin = (r > 0) ? V(vAlpha)[r] * sGam[(r - 1) * LG + i] * V(vEta)[i] : 0.f;
+      dw[e] = scale * geta * dOVt;
+      da[e] = gmin * dA;
+      sdGe[r * LG + i] = scale * dOVt * QK[mt][nt][2 * hf + e];
+      sdGm[r * LG + i] = dA * KK[mt][nt][2 * hf + e];
+    }
+    uint32_t ph, pl;
+    split_pack_bf16(dw[0], dw[1], ph, pl);
+    *reinterpret_cast<uint32_t*>(sDWH + r * L6 + i0) = ph;
+    *reinterpret_cast<uint32_t*>(sDWL + r * L6 + i0) = pl;
+    split_pack_bf16(da[0], da[1], ph, pl);
+    *reinterpret_cast<uint32_t*>(sDAH + r * L6 + i0) = ph;
+    *reinterpret_cast<uint32_t*>(sDAL + r * L6 + i0) = pl;
   });
   __syncthreads();
   // ---- dQ += DW K;  dK += DW^T Q + (DA + DA^T) K
-  warp_mma(dQ, [&](int m, int k) { return sDW[m * L64 + k]; }, [&](int k, int nn) { return bfv(sK, k * LT + nn); }, C, m0, n0, g, t);
-  warp_mma(dK, [&](int m, int k) { return sDW[k * L64 + m]; }, [&](int k, int nn) { return bfv(sQ, k * LT + nn); }, C, m0, n0, g, t);
-  warp_mma(dK, [&](int m, int k) { return sDA[m * L64 + k] + sDA[k * L64 + m]; }, [&](int k, int nn) { return bfv(sK, k * LT + nn); }, C, m0, n0, g, t);
+  warp_mma(dQ, oDWH, oK_t, C, m0, n0, lane);
+  warp_mma(dQ, oDWL, oK_t, C, m0, n0, lane);
+  warp_mma(dK, oDWH_t, oQ_t, C, m0, n0, lane);
+  warp_mma(dK, oDWL_t, oQ_t, C, m0, n0, lane);
+  warp_mma(dK, oDAH, oK_t, C, m0, n0, lane);
+  warp_mma(dK, oDAL, oK_t, C, m0, n0, lane);
+  warp_mma(dK, oDAH_t, oK_t, C, m0, n0, lane);
+  warp_mma(dK, oDAL_t, oK_t, C, m0, n0, lane);
   for_frag<2, 4>(m0, n0, g, t, [&](int mt, int nt, int e, int r, int c) {
     if (r < n) {
       a.dq[tok(r) * kD + c] = dQ[mt][nt][e];
@@ -379,15 +458,23 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
 
   // ---- gate gradients: the recurrences of Eq. 10 in reverse.  Thread i walks column i of gamma / m from the last
   // row up, carrying the adjoints of gamma_{r,i} and m_{r,i}; what belongs to a row goes to the row's accumulators.
-  __syncthreads();   // d Geta, d G^- written; all row sums in
+  __syncthreads();   // d Geta, d G^- written; all row sums in; DW, DA have been read
+  // per-(row, column) contributions to d alpha, d beta, d mu go to three matrices (the area DW, DA used) and are
+  // summed along the rows afterwards: all columns reach a row in the same step, shared-memory atomics would serialise
+  float* cAl = reinterpret_cast<float*>(smem + kOffVt);
+  float* cBe = cAl + C * LG;
+  float* cMu = cBe + C * LG;
+  static_assert(3 * kMatF <= 4 * kTile, "contribution matrices");
+  for (int idx = tid; idx < 3 * C * LG; idx += kThreads) cAl[idx] = 0.f;
+  __syncthreads();
   if (tid < C) {
     const int i = tid;
     const float eta_i = V(vEta)[i];
     float dg = 0.f, dm = 0.f, deta_i = 0.f;
     for (int r = C - 1; r >= i; --r) {
-      const float gam = sGam[r * L64 + i], mm = sMm[r * L64 + i];
-      const float gam_up = r > i ? sGam[(r - 1) * L64 + i] : 0.f;
-      const float al = V(vAlpha)[r], dge = sdGe[r * L64 + i], dgm = sdGm[r * L64 + i];
+      const float gam = sGam[r * LG + i], mm = sMm[r * LG + i];
+      const float gam_up = r > i ? sGam[(r - 1) * LG + i] : 0.f;
+      const float al = V(vAlpha)[r], dge = sdGe[r * LG + i], dgm = sdGm[r * LG + i];
       // gamma_{r,i} feeds Geta_{r,i}, G^-_{r+1,i} (carried in dg from the row below) and, in the last row, g_S
       float dgam = dg + dge * eta_i;
       float dmm = dm;
@@ -398,14 +485,24 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
       }
       deta_i += dge * gam + dgm * al * gam_up;
       dmm += dgam * V(vBeta)[r];
-      atomicAdd(V(vdAlpha) + r, dgam * gam_up + dgm * gam_up * eta_i);
-      atomicAdd(V(vdBeta) + r, dgam * mm);
-      if (r > i) atomicAdd(V(vdMu) + r, dmm * sMm[(r - 1) * L64 + i]);
+      cAl[r * LG + i] = dgam * gam_up + dgm * gam_up * eta_i;
+      cBe[r * LG + i] = dgam * mm;
+      if (r > i) cMu[r * LG + i] = dmm * sMm[(r - 1) * LG + i];
       // to the row above: gamma_{r-1,i} through the recurrence and through G^-_{r,i} = alpha_r gamma_{r-1,i} eta_i
       dg = dgam * al + dgm * al * eta_i;
       dm = dmm * V(vMu)[r];
     }
     V(vdEta)[i] = deta_i;
+  }
+  __syncthreads();
+  {   // row sums: four threads per row
+    const int r = tid >> 2, part = tid & 3;
+    float sa = 0.f, sbe = 0.f, sm = 0.f;
+    for (int i = part * 16; i < part * 16 + 16; ++i) { sa += cAl[r * LG + i]; sbe += cBe[r * LG + i]; sm += cMu[r * LG + i]; }
+    sa += __shfl_xor_sync(0xffffffffu, sa, 1); sa += __shfl_xor_sync(0xffffffffu, sa, 2);
+    sbe += __shfl_xor_sync(0xffffffffu, sbe, 1); sbe += __shfl_xor_sync(0xffffffffu, sbe, 2);
+    sm += __shfl_xor_sync(0xffffffffu, sm, 1); sm += __shfl_xor_sync(0xffffffffu, sm, 2);
+    if (part == 0) { V(vdAlpha)[r] += sa; V(vdBeta)[r] += sbe; V(vdMu)[r] += sm; }
   }
   __syncthreads();
   if (tid == 0) {   // the three vector recurrences (p_r = alpha_r b_{r-1}; b; the cumulative products), serial
@@ -457,7 +554,7 @@ cudaError_t launch_bwd_chunk_par(const Plan& fwd, const void* q, const void* k, 
   a.w_lo_offset = (size_t)fwd.geom.num_slots * fwd.p.H * C * C;
   a.fwd_states = static_cast<const uint8_t*>(fwd_states);
   a.adj_states = static_cast<const uint8_t*>(adj_states);
-  a.v_ext = static_cast<const __nv_bfloat16*>(v_ext);
+  (void)v_ext;
   a.scale = fwd.p.scale;
   a.dq = dq; a.dk = dk; a.dv = dv; a.dbeta = dbeta; a.dlog_alpha = dlog_alpha; a.dlog_mu = dlog_mu; a.deta = deta;
   cudaError_t e = cudaFuncSetAttribute(bwd_chunk_par_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmem);
