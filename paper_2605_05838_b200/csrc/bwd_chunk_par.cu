@@ -289,9 +289,11 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
     load_state(imgM);
     __syncthreads();
     warp_mma(Y, oK, oSt_dk, kD, m0, n0, lane);
-    for_frag<2, 4>(m0, n0, g, t, [&](int mt, int nt, int e, int r, int c) {
-      const float v = r < n ? __bfloat162float(a.v[tok(r) * kD + c]) : 0.f;
-      X[mt][nt][e] = v - V(vAbar)[r] * X[mt][nt][e] + V(vP)[r] * Y[mt][nt][e];
+    for_pair<2, 4>(m0, n0, g, t, [&](int mt, int nt, int hf, int r, int c) {
+      const uint32_t v2 = r < n ? *reinterpret_cast<const uint32_t*>(a.v + tok(r) * kD + c) : 0u;
+      const float ab = V(vAbar)[r], pp = V(vP)[r];
+      X[mt][nt][2 * hf] = __uint_as_float(v2 << 16) - ab * X[mt][nt][2 * hf] + pp * Y[mt][nt][2 * hf];
+      X[mt][nt][2 * hf + 1] = __uint_as_float(v2 & 0xffff0000u) - ab * X[mt][nt][2 * hf + 1] + pp * Y[mt][nt][2 * hf + 1];
     });
     put_split(X, sTmpH, sTmpL);
     __syncthreads();
@@ -356,8 +358,8 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
     warp_mma(dR, oT_t, oTmpH_t, C, m0, n0, lane);
     warp_mma(dR, oT_t, oTmpL_t, C, m0, n0, lane);
     put_split(dR, sDRH, sDRL);
-    for_frag<2, 4>(m0, n0, g, t, [&](int mt, int nt, int e, int r, int c) {
-      if (r < n) a.dv[tok(r) * kD + c] = dR[mt][nt][e];
+    for_pair<2, 4>(m0, n0, g, t, [&](int mt, int nt, int hf, int r, int c) {
+      if (r < n) *reinterpret_cast<float2*>(a.dv + tok(r) * kD + c) = make_float2(dR[mt][nt][2 * hf], dR[mt][nt][2 * hf + 1]);
     });
   }
   __syncthreads();
@@ -449,10 +451,10 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
   warp_mma(dK, oDAL, oK_t, C, m0, n0, lane);
   warp_mma(dK, oDAH_t, oK_t, C, m0, n0, lane);
   warp_mma(dK, oDAL_t, oK_t, C, m0, n0, lane);
-  for_frag<2, 4>(m0, n0, g, t, [&](int mt, int nt, int e, int r, int c) {
+  for_pair<2, 4>(m0, n0, g, t, [&](int mt, int nt, int hf, int r, int c) {
     if (r < n) {
-      a.dq[tok(r) * kD + c] = dQ[mt][nt][e];
-      a.dk[tok(r) * kD + c] = dK[mt][nt][e];
+      *reinterpret_cast<float2*>(a.dq + tok(r) * kD + c) = make_float2(dQ[mt][nt][2 * hf], dQ[mt][nt][2 * hf + 1]);
+      *reinterpret_cast<float2*>(a.dk + tok(r) * kD + c) = make_float2(dK[mt][nt][2 * hf], dK[mt][nt][2 * hf + 1]);
     }
   });
 
@@ -505,26 +507,49 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
     if (part == 0) { V(vdAlpha)[r] += sa; V(vdBeta)[r] += sbe; V(vdMu)[r] += sm; }
   }
   __syncthreads();
-  if (tid == 0) {   // the three vector recurrences (p_r = alpha_r b_{r-1}; b; the cumulative products), serial
+  // the three vector recurrences (p_r = alpha_r b_{r-1};  b_r = alpha_r b_{r-1} + beta_r mubar_r;  the cumulative
+  // products) in reverse: element-wise parts on 64 threads, the two 64-step chains on one thread each with the carry
+  // in a register
+  {
     float* dAl = V(vdAlpha); float* dBe = V(vdBeta); float* dMu = V(vdMu);
     float* dAb = V(vdAbar); float* dB = V(vdB); float* dMb = V(vdMubar);
-    for (int r = 0; r < C; ++r) {
+    if (tid < C) {
+      const int r = tid;
       dAl[r] += V(vdP)[r] * V(vBprev)[r];
-      if (r > 0) dB[r - 1] += V(vdP)[r] * V(vAlpha)[r];
+      if (r + 1 < C) dB[r] += V(vdP)[r + 1] * V(vAlpha)[r + 1];
     }
-    for (int r = C - 1; r >= 0; --r) {
+    __syncthreads();
+    if (tid == 0) {
+      float carry = 0.f;
+      for (int r = C - 1; r >= 0; --r) {
+        const float x = dB[r] + carry;
+        dB[r] = x;
+        carry = x * V(vAlpha)[r];
+      }
+    }
+    __syncthreads();
+    if (tid < C) {
+      const int r = tid;
       dAl[r] += dB[r] * V(vBprev)[r];
       dBe[r] += dB[r] * V(vMubar)[r];
       dMb[r] += dB[r] * V(vBeta)[r];
-      if (r > 0) dB[r - 1] += dB[r] * V(vAlpha)[r];
     }
-    for (int r = C - 1; r >= 0; --r) {
+    __syncthreads();
+    if (tid == 0 || tid == 32) {
+      float* d = tid == 0 ? dAb : dMb;
+      const float* mul = tid == 0 ? V(vAlpha) : V(vMu);
+      float carry = 0.f;
+      for (int r = C - 1; r >= 0; --r) {
+        const float x = d[r] + carry;
+        d[r] = x;
+        carry = x * mul[r];
+      }
+    }
+    __syncthreads();
+    if (tid < C) {
+      const int r = tid;
       dAl[r] += dAb[r] * (r > 0 ? V(vAbar)[r - 1] : 1.f);
       dMu[r] += dMb[r] * (r > 0 ? V(vMubar)[r - 1] : 1.f);
-      if (r > 0) {
-        dAb[r - 1] += dAb[r] * V(vAlpha)[r];
-        dMb[r - 1] += dMb[r] * V(vMu)[r];
-      }
     }
   }
   __syncthreads();
