@@ -15,6 +15,7 @@
 // holds the kernel that builds that problem from the forward's workspace (T, W, coefficient vectors) and q, k, dO.
 #include "mdn_common.cuh"
 #include "tc_utils.cuh"
+#include "warp_mma.cuh"
 
 namespace mdn {
 namespace {
@@ -23,7 +24,8 @@ using namespace tc;
 
 constexpr int kD = 128;
 constexpr int kPrepThreads = 256;
-constexpr int LWT = C + 4;   // floats per row of W^T in shared memory
+constexpr int LT = kD + 8;    // bf16 elements per row of the dO tile in shared memory (272 B: ldmatrix conflict-free)
+constexpr int L6 = C + 8;     // ... of a 64 x 64 matrix
 
 struct PrepArgs {
   ChunkGeom g;                      // the forward's geometry (fixed length)
@@ -41,45 +43,48 @@ struct PrepArgs {
 
 __global__ void __launch_bounds__(kPrepThreads) bwd_prep_kernel(PrepArgs a) {
   extern __shared__ __align__(16) uint8_t smem_raw[];
-  float* Wt = reinterpret_cast<float*>(smem_raw);                          // [64][LWT]: W^T, fp32 (hi + lo)
-  __nv_bfloat16* Tt = reinterpret_cast<__nv_bfloat16*>(Wt + C * LWT);      // [64][64 + 8]: T
+  __nv_bfloat16* sWH = reinterpret_cast<__nv_bfloat16*>(smem_raw);            // W hi, lo: [64][L6]
+  __nv_bfloat16* sWL = sWH + C * L6;
+  __nv_bfloat16* Tt = sWL + C * L6;                                           // T: [64][L6]
+  __nv_bfloat16* sDO = Tt + C * L6;                                           // dO: [64][LT]
   const int slot = blockIdx.x / a.g.H, h = blockIdx.x % a.g.H, H = a.g.H;
   const SlotInfo si = slot_info(a.g, slot);
   if (si.seq < 0) return;
-  const int tid = threadIdx.x;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
   const int nch = a.g.chunks_per_seq;
   // extended chunk indices of this forward chunk: the real step, then the injection step
   const int e_real = si.seq * 2 * nch + 2 * (nch - 1 - si.local), e_inj = e_real + 1;
   const size_t mat = ((size_t)slot * H + h) * C * C;
 
-  // ---- W^T (fp32) and T into shared memory
-  for (int idx = tid; idx < C * C; idx += kPrepThreads) {
-    const int r = idx >> 6, i = idx & 63;
-    Wt[i * LWT + r] = __bfloat162float(a.W[mat + idx]) + __bfloat162float(a.W[a.w_lo_offset + mat + idx]);
-    Tt[r * (C + 8) + i] = a.T[mat + idx];
+  // ---- W (hi, lo), T and the dO tile into shared memory; dO also goes out as the "V" of the injection step
+  for (int idx = tid; idx < C * 8; idx += kPrepThreads) {
+    const int r = idx >> 3, c8 = (idx & 7) * 8;
+    *reinterpret_cast<uint4*>(sWH + r * L6 + c8) = *reinterpret_cast<const uint4*>(a.W + mat + r * C + c8);
+    *reinterpret_cast<uint4*>(sWL + r * L6 + c8) = *reinterpret_cast<const uint4*>(a.W + a.w_lo_offset + mat + r * C + c8);
+    *reinterpret_cast<uint4*>(Tt + r * L6 + c8) = *reinterpret_cast<const uint4*>(a.T + mat + r * C + c8);
+  }
+  for (int idx = tid; idx < C * (kD / 8); idx += kPrepThreads) {
+    const int r = idx >> 4, c8 = (idx & 15) * 8;
+    uint4 x = make_uint4(0u, 0u, 0u, 0u);
+    if (r < si.n) x = *reinterpret_cast<const uint4*>(a.d_o + ((size_t)(si.tok0 + r) * H + h) * kD + c8);
+    *reinterpret_cast<uint4*>(sDO + r * LT + c8) = x;
+    *reinterpret_cast<uint4*>(a.v_ext + ((size_t)(e_inj * C + r) * H + h) * kD + c8) = x;
   }
   __syncthreads();
 
-  // ---- V' = W^T dO for the real step, dO itself for the injection step; thread = (value column j, half of the rows i)
+  // ---- V' = W^T dO for the real step: a 64 x 128 result, one 32 x 32 block per warp, bf16 MMAs (W as hi + lo)
   {
-    const int j = tid & (kD - 1), half = tid >> 7;
-    float docol[C];
-#pragma unroll
-    for (int r = 0; r < C; ++r)
-      docol[r] = r < si.n ? __bfloat162float(a.d_o[((size_t)(si.tok0 + r) * H + h) * kD + j]) : 0.f;
-    for (int i = half * 32; i < half * 32 + 32; ++i) {
-      float acc = 0.f;
-#pragma unroll
-      for (int r4 = 0; r4 < C; r4 += 4) {
-        const float4 w4 = *reinterpret_cast<const float4*>(Wt + i * LWT + r4);
-        acc = fmaf(w4.x, docol[r4], acc); acc = fmaf(w4.y, docol[r4 + 1], acc);
-        acc = fmaf(w4.z, docol[r4 + 2], acc); acc = fmaf(w4.w, docol[r4 + 3], acc);
-      }
-      a.v_ext[((size_t)(e_real * C + i) * H + h) * kD + j] = __float2bfloat16_rn(i < si.n ? acc : 0.f);
-    }
-#pragma unroll
-    for (int r = 0; r < C; ++r)
-      if ((r >> 5) == half) a.v_ext[((size_t)(e_inj * C + r) * H + h) * kD + j] = __float2bfloat16_rn(docol[r]);
+    const uint32_t sb = smem_u32(smem_raw);
+    const Opnd oWH_t{sb, L6 * 2, true}, oWL_t{sb + C * L6 * 2, L6 * 2, true}, oDO_t{sb + 3 * C * L6 * 2, LT * 2, true};
+    const int m0 = 32 * (warp & 1), n0 = 32 * (warp >> 1);
+    float Z[2][4][4];
+    zero(Z);
+    warp_mma(Z, oWH_t, oDO_t, C, m0, n0, lane);
+    warp_mma(Z, oWL_t, oDO_t, C, m0, n0, lane);
+    for_pair<2, 4>(m0, n0, g, t, [&](int mt, int nt, int hf, int i, int c) {
+      const uint32_t packed = i < si.n ? pack_bf16(Z[mt][nt][2 * hf], Z[mt][nt][2 * hf + 1]) : 0u;
+      *reinterpret_cast<uint32_t*>(a.v_ext + ((size_t)(e_real * C + i) * H + h) * kD + c) = packed;
+    });
   }
 
   // ---- keys of the two steps: k (real), q (injection); rows past the end of a short chunk are zero
@@ -98,7 +103,7 @@ __global__ void __launch_bounds__(kPrepThreads) bwd_prep_kernel(PrepArgs a) {
   const size_t mat_r = ((size_t)e_real * H + h) * C * C, mat_i = ((size_t)e_inj * H + h) * C * C;
   for (int idx = tid; idx < C * C; idx += kPrepThreads) {
     const int r = idx >> 6, i = idx & 63;
-    a.T_ext[mat_r + idx] = Tt[i * (C + 8) + r];
+    a.T_ext[mat_r + idx] = Tt[i * L6 + r];
     a.T_ext[mat_i + idx] = __float2bfloat16_rn(r == i ? 1.f : 0.f);
   }
 
@@ -130,7 +135,7 @@ __global__ void __launch_bounds__(kPrepThreads) bwd_prep_kernel(PrepArgs a) {
 
 }  // namespace
 
-size_t bwd_prep_smem_bytes() { return (size_t)C * LWT * 4 + (size_t)C * (C + 8) * 2; }
+size_t bwd_prep_smem_bytes() { return (size_t)3 * C * L6 * 2 + (size_t)C * LT * 2; }
 
 cudaError_t launch_bwd_prep(const Plan& fwd, const void* q, const void* k, const void* d_o, void* k_ext, void* v_ext,
                             float* coef_ext, void* T_ext, int* launches) {
