@@ -475,8 +475,10 @@ def run_layer_ops(args, w):
 
 
 def run_backward(args, w):
-    """Secondary benchmark (not the headline): mdn_chunk_bwd (all gradients) on the same workload, inputs and the
-    upstream gradient resident in HBM, CUDA events."""
+    """Secondary benchmark (not the headline): the backward (all gradients) on the same workload, inputs and the
+    upstream gradient resident in HBM, CUDA events.  --bwd-method chunked (default where it applies: bf16, dk = dv = 128,
+    fixed length): mdn_chunk_bwd_chunked, the chunk-parallel tensor-core backward; stepwise: mdn_chunk_bwd, the exact
+    token-level one."""
     import torch
     import paper_2605_05838_b200 as mdn
     mdn.lib()
@@ -488,12 +490,18 @@ def run_backward(args, w):
     gates = [dev(inp[n]) for n in ("beta", "log_alpha", "log_mu", "eta")]
     cu = None if inp["cu_seqlens"] is None else torch.from_numpy(inp["cu_seqlens"]).to("cuda")
     d_o = torch.randn(v.shape, device="cuda", generator=torch.Generator(device="cuda").manual_seed(1)).to(dt)
-    need = int(mdn.lib().mdn_chunk_bwd_workspace_bytes(ctypes.byref(mdn.make_params(q, v, num_seqs=0 if cu is None else cu.numel() - 1))))
+    can_chunk = w.dtype == "bf16" and w.dk == 128 and w.dv == 128 and cu is None
+    method = args.bwd_method if args.bwd_method != "auto" else ("chunked" if can_chunk else "stepwise")
+    if method == "chunked":
+        need = int(mdn.lib().mdn_chunk_bwd_chunked_workspace_bytes(ctypes.byref(mdn.make_params(q, v, path="tensor"))))
+    else:
+        need = int(mdn.lib().mdn_chunk_bwd_workspace_bytes(ctypes.byref(mdn.make_params(q, v, num_seqs=0 if cu is None else cu.numel() - 1))))
     ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+    S0, M0 = dev(inp["S0"]), dev(inp["M0"])
 
     def step():
-        return mdn.chunk_bwd(q, k, v, *gates, d_o, initial_S=dev(inp["S0"]), initial_M=dev(inp["M0"]), cu_seqlens=cu,
-                             scale=inp["scale"], workspace=ws)
+        return mdn.chunk_bwd(q, k, v, *gates, d_o, initial_S=S0, initial_M=M0, cu_seqlens=cu,
+                             scale=inp["scale"], workspace=ws, method=method)
 
     warm = max(args.warmup, 3)
     for _ in range(warm):
@@ -513,11 +521,14 @@ def run_backward(args, w):
     abytes = float(tokens * w.H * ((2 * w.dk + 2 * w.dv) * es + 16 + (2 * w.dk + w.dv) * 4 + 16))
     print(json.dumps({
         "metric": "MDN chunkwise bwd tokens/s", "value": tokens / (ms * 1e-3), "unit": "tokens/s", "n_gpus": 1,
-        "steps": args.steps, "warmup": warm, "ms_per_step": ms, "higher_is_better": True, "dtype": "f32",
-        "data": "synthetic", "config": {"workload": workload_desc(w), "form": "token-level adjoint recurrence, "
-                                        "per-chunk checkpoints and recomputation (fp32)"},
+        "steps": args.steps, "warmup": warm, "ms_per_step": ms, "higher_is_better": True,
+        "dtype": "bf16" if method == "chunked" else "f32",
+        "data": "synthetic", "config": {"workload": workload_desc(w), "form": (
+            "chunk-parallel: state-only forward keeping the chunk states, adjoint state chain, per-chunk kernel "
+            "(bf16 tensor-core products, fp32 accumulation)" if method == "chunked" else
+            "token-level adjoint recurrence, per-chunk checkpoints and recomputation (fp32)")},
         "gpu_launches": launches * args.steps, "workspace_bytes": need,
-        "roofline": {"bound": "hbm", "kernel": "bwd_stepwise", "achieved": abytes / (ms * 1e-3) / 1e9,
+        "roofline": {"bound": "hbm", "kernel": "whole backward" if method == "chunked" else "bwd_stepwise", "achieved": abytes / (ms * 1e-3) / 1e9,
                      "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": abytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
                      "traffic": None, "peak_source": peaks["source"], "algorithmic_bytes": abytes}}))
 
@@ -535,6 +546,7 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--decode", action="store_true", help="secondary benchmark: the recurrent decode step")
     ap.add_argument("--decode-batch", type=int, default=128)
+    ap.add_argument("--bwd-method", default="auto", choices=["auto", "chunked", "stepwise"])
     ap.add_argument("--backward", action="store_true", help="secondary benchmark: mdn_chunk_bwd (all gradients)")
     ap.add_argument("--layer-ops", action="store_true",
                     help="secondary benchmark: forward with the layer's element-wise operations, fused vs separate passes")

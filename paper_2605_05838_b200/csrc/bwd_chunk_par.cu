@@ -183,6 +183,20 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
       }
   };
 
+  // ---- everything this CTA will fetch later, towards L2 now (one CTA per SM: nothing else hides the latency)
+  for (int idx = tid; idx < 1024; idx += kThreads) {
+    const int which = idx >> 8, line = idx & 255;
+    const uint8_t* p = (which == 0 ? imgM : which == 1 ? imgdM : which == 2 ? imgdS : imgS) + line * 128;
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
+  }
+  if (tid < 128) {
+    const bf16* w = a.W + (tid >= 64 ? a.w_lo_offset : 0) + mat + (tid & 63) * C;
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(w));
+  }
+  if (tid < n) {
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(a.v + tok(tid) * kD));
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(a.v + tok(tid) * kD + 64));
+  }
   // ---- vectors: the chain's coefficient vectors, the gates, zeroed adjoints
   const float* cf = a.coef + ((size_t)slot * H + h) * MDN_NUM_COEF * C;
   for (int idx = tid; idx < 24 * C; idx += kThreads) vec[idx] = 0.f;
