@@ -1,7 +1,7 @@
 // Backward of the MDN recurrence (Section 3.1, Eq. 5-6): reverse-mode, token by token, with the states recomputed
 // chunk by chunk from checkpoints (the paper's training kernels also keep no per-token states and rebuild them in
 // the backward pass).  fp32 throughout; this is the exact CUDA form of the backward - every gradient, any dk, dv in
-// {64, 128}, fixed-length or packed input - not yet the chunk-parallel matrix form.
+// {64, 128}, fixed-length or packed input.  (The chunk-parallel matrix form on the tensor cores is bwd_chunk*.cu.)
 //
 // The value columns of S, M and of their adjoints GS, GM are independent; only dq, dk and the gate gradients sum over
 // columns.  One WARP owns 4 value columns of one (sequence, head): lane l holds rows l, l + 32, .. of those columns of
