@@ -44,6 +44,8 @@ constexpr uint32_t kOffT = kOffDR + 2 * kTile;        // T, bf16 [64][L6]
 constexpr uint32_t kOffTmp = kOffT + kMat6;           // R / dV~ hi, lo; W hi, lo; later gamma, m (fp32 [64][LG] each)
 constexpr uint32_t kOffVec = kOffTmp + 2 * kTile;     // vectors, 24 x [64] floats
 constexpr uint32_t kSmem = kOffVec + 24 * C * 4;
+constexpr uint32_t kR0 = kOffSt, kR1 = kOffVt, kR2 = kOffDR, kR3 = kOffTmp;   // the four reusable areas (see the kernel)
+static_assert(kD * LT * 2 == 2 * kTile, "a state and a hi + lo tile pair have the same size");
 static_assert(2 * kTile >= 2 * kMatF && kD * LT * 2 >= 2 * kMatF && 2 * kTile >= 2 * kMat6, "overlays");
 static_assert(kSmem <= 232448, "shared memory");
 
@@ -55,7 +57,7 @@ struct ParArgs {
   const bf16* q; const bf16* k; const bf16* v; const bf16* d_o;
   const float* beta; const float* log_alpha; const float* log_mu; const float* eta;
   const float* coef; const bf16* T; const bf16* W; size_t w_lo_offset;
-  const uint8_t* fwd_states; const uint8_t* adj_states;
+  const uint8_t* fwd_states; const uint8_t* adj_states; const bf16* v_ext;
   float scale;
   float* dq; float* dk; float* dv; float* dbeta; float* dlog_alpha; float* dlog_mu; float* deta;
 };
@@ -63,26 +65,17 @@ struct ParArgs {
 __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
   extern __shared__ __align__(16) uint8_t smem[];
   const uint32_t sb = smem_u32(smem);
-  bf16* sSt = reinterpret_cast<bf16*>(smem + kOffSt);
   bf16* sK = reinterpret_cast<bf16*>(smem + kOffK);
   bf16* sQ = reinterpret_cast<bf16*>(smem + kOffQ);
   bf16* sDO = reinterpret_cast<bf16*>(smem + kOffDO);
-  bf16* sVtH = reinterpret_cast<bf16*>(smem + kOffVt);
-  bf16* sVtL = sVtH + C * LT;
-  bf16* sDRH = reinterpret_cast<bf16*>(smem + kOffDR);
-  bf16* sDRL = sDRH + C * LT;
   bf16* sT = reinterpret_cast<bf16*>(smem + kOffT);
-  bf16* sTmpH = reinterpret_cast<bf16*>(smem + kOffTmp);      // R, then dV~ (hi, lo)
-  bf16* sTmpL = sTmpH + C * LT;
-  bf16* sWH = sTmpH;                                          // W (hi, lo) between R and dV~
-  bf16* sWL = sWH + C * L6;
-  float* sGam = reinterpret_cast<float*>(smem + kOffTmp);     // gamma, m (after dV~ is done with the area)
+  float* sGam = reinterpret_cast<float*>(smem + kR2);         // gamma, m
   float* sMm = sGam + C * LG;
-  bf16* sDWH = reinterpret_cast<bf16*>(smem + kOffVt);        // DW, DA (after V~, dR are done)
+  bf16* sDWH = reinterpret_cast<bf16*>(smem + kR1);           // DW, DA (hi, lo)
   bf16* sDWL = sDWH + C * L6;
-  bf16* sDAH = reinterpret_cast<bf16*>(smem + kOffDR);
+  bf16* sDAH = reinterpret_cast<bf16*>(smem + kR3);
   bf16* sDAL = sDAH + C * L6;
-  float* sdGe = reinterpret_cast<float*>(smem + kOffSt);      // d Geta, d G^- (after the states are done)
+  float* sdGe = reinterpret_cast<float*>(smem + kR0);         // d Geta, d G^-
   float* sdGm = sdGe + C * LG;
   float* vec = reinterpret_cast<float*>(smem + kOffVec);
   auto V = [&](int which) { return vec + which * C; };
@@ -105,17 +98,17 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
   const Opnd oK{sb + kOffK, LT * 2, false}, oK_t{sb + kOffK, LT * 2, true};
   const Opnd oQ{sb + kOffQ, LT * 2, false}, oQ_t{sb + kOffQ, LT * 2, true};
   const Opnd oDO{sb + kOffDO, LT * 2, false}, oDO_t{sb + kOffDO, LT * 2, true};
-  const Opnd oSt_dk{sb + kOffSt, LT * 2, false};   // B(k = key d, n = value j) = S[d][j], stored [j][d]
-  const Opnd oSt_dv{sb + kOffSt, LT * 2, true};    // B(k = value j, n = key d)
-  const Opnd oVtH{sb + kOffVt, LT * 2, false}, oVtL{sb + kOffVt + kTile, LT * 2, false};
-  const Opnd oDRH{sb + kOffDR, LT * 2, false}, oDRL{sb + kOffDR + kTile, LT * 2, false};
   const Opnd oT{sb + kOffT, L6 * 2, false}, oT_t{sb + kOffT, L6 * 2, true};
-  const Opnd oTmpH_t{sb + kOffTmp, LT * 2, true}, oTmpL_t{sb + kOffTmp + kTile, LT * 2, true};
-  const Opnd oWH_t{sb + kOffTmp, L6 * 2, true}, oWL_t{sb + kOffTmp + kMat6, L6 * 2, true};
-  const Opnd oDWH{sb + kOffVt, L6 * 2, false}, oDWL{sb + kOffVt + kMat6, L6 * 2, false};
-  const Opnd oDWH_t{sb + kOffVt, L6 * 2, true}, oDWL_t{sb + kOffVt + kMat6, L6 * 2, true};
-  const Opnd oDAH{sb + kOffDR, L6 * 2, false}, oDAL{sb + kOffDR + kMat6, L6 * 2, false};
-  const Opnd oDAH_t{sb + kOffDR, L6 * 2, true}, oDAL_t{sb + kOffDR + kMat6, L6 * 2, true};
+  // a state in an area: B(k = key d, n = value j) = S[d][j], stored [j][d]; or B(k = value j, n = key d)
+  auto st_dk = [&](uint32_t base) { return Opnd{sb + base, LT * 2, false}; };
+  auto st_dv = [&](uint32_t base) { return Opnd{sb + base, LT * 2, true}; };
+  // a 64 x 128 tile in an area, stored [row][column]: as A it is [m][k], as B it is [n][k]; tile_kn reads it as B [k][n]
+  auto tile_mk = [&](uint32_t base) { return Opnd{sb + base, LT * 2, false}; };
+  auto tile_kn = [&](uint32_t base) { return Opnd{sb + base, LT * 2, true}; };
+  const Opnd oDWH{sb + kR1, L6 * 2, false}, oDWL{sb + kR1 + kMat6, L6 * 2, false};
+  const Opnd oDWH_t{sb + kR1, L6 * 2, true}, oDWL_t{sb + kR1 + kMat6, L6 * 2, true};
+  const Opnd oDAH{sb + kR3, L6 * 2, false}, oDAL{sb + kR3 + kMat6, L6 * 2, false};
+  const Opnd oDAH_t{sb + kR3, L6 * 2, true}, oDAL_t{sb + kR3 + kMat6, L6 * 2, true};
 
   auto tok = [&](int r) { return (size_t)(si.tok0 + r) * H + h; };
   auto load_tile = [&](bf16* dst, const bf16* src) {
@@ -132,14 +125,16 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
       *reinterpret_cast<uint4*>(dst + r * L6 + c8) = *reinterpret_cast<const uint4*>(src + r * C + c8);
     }
   };
-  // state image (value index j x key index d, two swizzled blocks) -> sSt[j][d]
-  auto load_state = [&](const uint8_t* img) {
+  // state image (value index j x key index d, two swizzled blocks) -> [j][d] in an area, by cp.async
+  auto load_state = [&](const uint8_t* img, uint32_t base) {
     for (int idx = tid; idx < 2 * kD * 8; idx += kThreads) {
       const int half = idx >> 10, j = (idx >> 3) & 127, pp = idx & 7, c = pp ^ (j & 7);
-      *reinterpret_cast<uint4*>(sSt + j * LT + half * 64 + c * 8) =
-          *reinterpret_cast<const uint4*>(img + half * 16384 + j * 128 + pp * 16);
+      const uint32_t dst = sb + base + (j * LT + half * 64 + c * 8) * 2;
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(img + half * 16384 + j * 128 + pp * 16));
     }
   };
+  auto cp_async_commit = []() { asm volatile("cp.async.commit_group;" ::: "memory"); };
+  auto cp_async_wait = []() { asm volatile("cp.async.wait_group 0;" ::: "memory"); };
   auto dot_images = [&](const uint8_t* x, const uint8_t* y) {   // sum of the element-wise product (same layout)
     float s = 0.f;
     for (int idx = tid; idx < 2048; idx += kThreads) {
@@ -155,7 +150,9 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
     return s;   // per warp; lane 0 adds it where it belongs
   };
   // a warp's 32 x 32 block of a 64 x 128 result -> bf16 hi + lo tiles (rows past the chunk's end are zero)
-  auto put_split = [&](float (&acc)[2][4][4], bf16* hi, bf16* lo) {
+  auto put_split = [&](float (&acc)[2][4][4], uint32_t base) {
+    bf16* hi = reinterpret_cast<bf16*>(smem + base);
+    bf16* lo = hi + C * LT;
     for_pair<2, 4>(m0, n0, g, t, [&](int mt, int nt, int hf, int r, int c) {
       uint32_t ph = 0u, pl = 0u;
       if (r < n) split_pack_bf16(acc[mt][nt][2 * hf], acc[mt][nt][2 * hf + 1], ph, pl);
@@ -189,10 +186,7 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
     const uint8_t* p = (which == 0 ? imgM : which == 1 ? imgdM : which == 2 ? imgdS : imgS) + line * 128;
     asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
   }
-  if (tid < 128) {
-    const bf16* w = a.W + (tid >= 64 ? a.w_lo_offset : 0) + mat + (tid & 63) * C;
-    asm volatile("prefetch.global.L2 [%0];" ::"l"(w));
-  }
+  if (tid < C) asm volatile("prefetch.global.L2 [%0];" ::"l"(a.v_ext + ((size_t)(e_real * C + tid) * H + h) * kD));
   if (tid < n) {
     asm volatile("prefetch.global.L2 [%0];" ::"l"(a.v + tok(tid) * kD));
     asm volatile("prefetch.global.L2 [%0];" ::"l"(a.v + tok(tid) * kD + 64));
@@ -210,134 +204,129 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
     V(vAlpha)[r] = live ? expf(a.log_alpha[gi]) : 1.f; V(vMu)[r] = live ? expf(a.log_mu[gi]) : 1.f;
     V(vBeta)[r] = live ? a.beta[gi] : 0.f; V(vEta)[r] = live ? (a.eta ? a.eta[gi] : 1.f) : 0.f;
   }
+  // Four areas of 34816 bytes (a state, or the hi + lo pair of a 64 x 128 tile) are reused through the phases:
+  //   R0: S                              | later d Geta, d G^-
+  //   R1: M            | V~ (hi, lo)     | later DW (hi, lo), then two contribution matrices
+  //   R2: dM'          | dV~ (hi, lo)    | M again | gamma, m
+  //   R3: R (hi, lo)   | dS'             | dR (hi, lo) | DA (hi, lo), then a contribution matrix
+  // States arrive by cp.async (no registers in between), each as early as its area is free.
+  load_state(imgS, kR0);
+  load_state(imgM, kR1);
+  load_state(imgdM, kR2);
+  cp_async_commit();
   load_tile(sK, a.k);
   load_tile(sQ, a.q);
   load_tile(sDO, a.d_o);
   load_mat64(sT, a.T + mat);
-  load_state(imgS);
+  {
+    const float s = dot_images(imgdM, imgM);                         // d mubar_C = <dM', M>
+    if (lane == 0) atomicAdd(V(vdMubar) + n - 1, s);
+  }
+  cp_async_wait();
   __syncthreads();
   if (tid < C) V(vBprev)[tid] = tid > 0 ? V(vB)[tid - 1] : 0.f;
 
   float dQ[2][4][4], dK[2][4][4];
   zero(dQ); zero(dK);
 
-  // ---- forward quantities again: X = K S, Y = K M, R = V - abar.X + p.Y, V~ = T R
+  // ---- phase 1, with S and M: X = K S, Y = K M, R = V - abar.X + p.Y, V~ = T R; dO S^T, dO M^T (dQ, d abar, d b)
   {
     float X[2][4][4], Y[2][4][4];
     zero(X); zero(Y);
-    warp_mma(X, oK, oSt_dk, kD, m0, n0, lane);
-    __syncthreads();
-    load_state(imgM);
-    __syncthreads();
-    warp_mma(Y, oK, oSt_dk, kD, m0, n0, lane);
+    warp_mma(X, oK, st_dk(kR0), kD, m0, n0, lane);
+    warp_mma(Y, oK, st_dk(kR1), kD, m0, n0, lane);
     for_pair<2, 4>(m0, n0, g, t, [&](int mt, int nt, int hf, int r, int c) {
       const uint32_t v2 = r < n ? *reinterpret_cast<const uint32_t*>(a.v + tok(r) * kD + c) : 0u;
       const float ab = V(vAbar)[r], pp = V(vP)[r];
       X[mt][nt][2 * hf] = __uint_as_float(v2 << 16) - ab * X[mt][nt][2 * hf] + pp * Y[mt][nt][2 * hf];
       X[mt][nt][2 * hf + 1] = __uint_as_float(v2 & 0xffff0000u) - ab * X[mt][nt][2 * hf + 1] + pp * Y[mt][nt][2 * hf + 1];
     });
-    put_split(X, sTmpH, sTmpL);
-    __syncthreads();
+    put_split(X, kR3);
+    zero(Y);
+    warp_mma(Y, oDO, st_dv(kR0), kD, m0, n0, lane);                   // dO S^T
+    for_frag<2, 4>(m0, n0, g, t, [&](int mt, int nt, int e, int r, int c) { dQ[mt][nt][e] += scale * V(vAbar)[r] * Y[mt][nt][e]; });
+    add_rowsum(Y, sQ, V(vdAbar), scale);
+    zero(Y);
+    warp_mma(Y, oDO, st_dv(kR1), kD, m0, n0, lane);                   // dO M^T
+    for_frag<2, 4>(m0, n0, g, t, [&](int mt, int nt, int e, int r, int c) { dQ[mt][nt][e] -= scale * V(vB)[r] * Y[mt][nt][e]; });
+    add_rowsum(Y, sQ, V(vdB), -scale);
+    __syncthreads();   // R complete; M has been read
     float Vt[2][4][4];
     zero(Vt);
-    warp_mma(Vt, oT, oTmpH_t, C, m0, n0, lane);
-    warp_mma(Vt, oT, oTmpL_t, C, m0, n0, lane);
-    put_split(Vt, sVtH, sVtL);
+    warp_mma(Vt, oT, tile_kn(kR3), C, m0, n0, lane);
+    warp_mma(Vt, oT, tile_kn(kR3 + kTile), C, m0, n0, lane);
+    put_split(Vt, kR1);
   }
   __syncthreads();   // V~ complete; R has been read
-  load_mat64(sWH, a.W + mat);
-  load_mat64(sWL, a.W + a.w_lo_offset + mat);
+  load_state(imgdS, kR3);
+  cp_async_commit();
 
-  // ---- with dM' (the end-of-chunk adjoint of M): K dM', the g_M term of dK and its coefficient adjoint
-  float KdM[2][4][4];
-  zero(KdM);
-  load_state(imgdM);
+  // ---- phase 2, with dM' and dS': K dM', K dS', the g_S and g_M terms of dK, dV~ = W^T dO + g_S.(K dS') - g_M.(K dM'),
+  // dR = T^T dV~
   {
-    const float s = dot_images(imgdM, imgM);                         // d mubar_C = <dM', M>
-    if (lane == 0) atomicAdd(V(vdMubar) + n - 1, s);
-  }
-  __syncthreads();
-  warp_mma(KdM, oK, oSt_dk, kD, m0, n0, lane);
-  {
-    float G[2][4][4];
-    zero(G);
-    warp_mma(G, oVtH, oSt_dv, kD, m0, n0, lane);                      // V~ dM'^T
-    warp_mma(G, oVtL, oSt_dv, kD, m0, n0, lane);
+    float KdM[2][4][4], G[2][4][4];
+    zero(KdM); zero(G);
+    warp_mma(KdM, oK, st_dk(kR2), kD, m0, n0, lane);
+    warp_mma(G, tile_mk(kR1), st_dv(kR2), kD, m0, n0, lane);          // V~ dM'^T
+    warp_mma(G, tile_mk(kR1 + kTile), st_dv(kR2), kD, m0, n0, lane);
     for_frag<2, 4>(m0, n0, g, t, [&](int mt, int nt, int e, int r, int c) { dK[mt][nt][e] -= V(vGM)[r] * G[mt][nt][e]; });
     add_rowsum(G, sK, V(vdGM), -1.f);
-  }
-  __syncthreads();
-  // ---- with dS': K dS', the g_S term of dK, dV~ = W^T dO + g_S.(K dS') - g_M.(K dM'), dR = T^T dV~
-  load_state(imgdS);
-  {
-    const float s1 = dot_images(imgdS, imgS), s2 = dot_images(imgdS, imgM);   // d abar_C = <dS', S>, d b_C = -<dS', M>
-    if (lane == 0) { atomicAdd(V(vdAbar) + n - 1, s1); atomicAdd(V(vdB) + n - 1, -s2); }
-  }
-  __syncthreads();
-  {
-    float Z[2][4][4], G[2][4][4];
-    zero(Z); zero(G);
-    warp_mma(Z, oWH_t, oDO_t, C, m0, n0, lane);                       // W^T dO
-    warp_mma(Z, oWL_t, oDO_t, C, m0, n0, lane);
+    {
+      const float s1 = dot_images(imgdS, imgS), s2 = dot_images(imgdS, imgM);   // d abar_C = <dS', S>, d b_C = -<dS', M>
+      if (lane == 0) { atomicAdd(V(vdAbar) + n - 1, s1); atomicAdd(V(vdB) + n - 1, -s2); }
+    }
+    cp_async_wait();
+    __syncthreads();   // dS' has landed; dM' has been read
     float KdS[2][4][4];
-    zero(KdS);
-    warp_mma(KdS, oK, oSt_dk, kD, m0, n0, lane);
-    warp_mma(G, oVtH, oSt_dv, kD, m0, n0, lane);                      // V~ dS'^T
-    warp_mma(G, oVtL, oSt_dv, kD, m0, n0, lane);
-    for_frag<2, 4>(m0, n0, g, t, [&](int mt, int nt, int e, int r, int c) {
-      dK[mt][nt][e] += V(vGS)[r] * G[mt][nt][e];
-      Z[mt][nt][e] += V(vGS)[r] * KdS[mt][nt][e] - V(vGM)[r] * KdM[mt][nt][e];
-    });
+    zero(KdS); zero(G);
+    warp_mma(KdS, oK, st_dk(kR3), kD, m0, n0, lane);
+    warp_mma(G, tile_mk(kR1), st_dv(kR3), kD, m0, n0, lane);          // V~ dS'^T
+    warp_mma(G, tile_mk(kR1 + kTile), st_dv(kR3), kD, m0, n0, lane);
+    for_frag<2, 4>(m0, n0, g, t, [&](int mt, int nt, int e, int r, int c) { dK[mt][nt][e] += V(vGS)[r] * G[mt][nt][e]; });
     add_rowsum(G, sK, V(vdGS), 1.f);
-    __syncthreads();   // W has been read: the area takes dV~
-    put_split(Z, sTmpH, sTmpL);
+    for_pair<2, 4>(m0, n0, g, t, [&](int mt, int nt, int hf, int r, int c) {
+      // W^T dO as the adjoint chain's problem has it (bf16)
+      const uint32_t v2 = r < n ? *reinterpret_cast<const uint32_t*>(a.v_ext + ((size_t)(e_real * C + r) * H + h) * kD + c) : 0u;
+      const float gs = V(vGS)[r], gm = V(vGM)[r];
+      KdS[mt][nt][2 * hf] = __uint_as_float(v2 << 16) + gs * KdS[mt][nt][2 * hf] - gm * KdM[mt][nt][2 * hf];
+      KdS[mt][nt][2 * hf + 1] = __uint_as_float(v2 & 0xffff0000u) + gs * KdS[mt][nt][2 * hf + 1] - gm * KdM[mt][nt][2 * hf + 1];
+    });
+    put_split(KdS, kR2);
   }
-  __syncthreads();
+  __syncthreads();   // dV~ complete; dS' has been read
   {
     float dR[2][4][4];
     zero(dR);
-    warp_mma(dR, oT_t, oTmpH_t, C, m0, n0, lane);
-    warp_mma(dR, oT_t, oTmpL_t, C, m0, n0, lane);
-    put_split(dR, sDRH, sDRL);
+    warp_mma(dR, oT_t, tile_kn(kR2), C, m0, n0, lane);
+    warp_mma(dR, oT_t, tile_kn(kR2 + kTile), C, m0, n0, lane);
+    put_split(dR, kR3);
     for_pair<2, 4>(m0, n0, g, t, [&](int mt, int nt, int hf, int r, int c) {
       if (r < n) *reinterpret_cast<float2*>(a.dv + tok(r) * kD + c) = make_float2(dR[mt][nt][2 * hf], dR[mt][nt][2 * hf + 1]);
     });
   }
-  __syncthreads();
+  __syncthreads();   // dR complete; dV~ has been read
+  load_state(imgM, kR2);
+  cp_async_commit();
 
-  // ---- with S: dO S^T (dQ, d abar), dR S^T (dK, d abar)
-  load_state(imgS);
-  __syncthreads();
+  // ---- phase 3: dR S^T (dK, d abar) while M arrives again, then dR M^T (dK, d p)
   {
     float G[2][4][4];
     zero(G);
-    warp_mma(G, oDO, oSt_dv, kD, m0, n0, lane);
-    for_frag<2, 4>(m0, n0, g, t, [&](int mt, int nt, int e, int r, int c) { dQ[mt][nt][e] += scale * V(vAbar)[r] * G[mt][nt][e]; });
-    add_rowsum(G, sQ, V(vdAbar), scale);
-    zero(G);
-    warp_mma(G, oDRH, oSt_dv, kD, m0, n0, lane);
-    warp_mma(G, oDRL, oSt_dv, kD, m0, n0, lane);
+    warp_mma(G, tile_mk(kR3), st_dv(kR0), kD, m0, n0, lane);
+    warp_mma(G, tile_mk(kR3 + kTile), st_dv(kR0), kD, m0, n0, lane);
     for_frag<2, 4>(m0, n0, g, t, [&](int mt, int nt, int e, int r, int c) { dK[mt][nt][e] -= V(vAbar)[r] * G[mt][nt][e]; });
     add_rowsum(G, sK, V(vdAbar), -1.f);
-  }
-  __syncthreads();
-  // ---- with M: dO M^T (dQ, d b), dR M^T (dK, d p)
-  load_state(imgM);
-  __syncthreads();
-  {
-    float G[2][4][4];
+    cp_async_wait();
+    __syncthreads();
     zero(G);
-    warp_mma(G, oDO, oSt_dv, kD, m0, n0, lane);
-    for_frag<2, 4>(m0, n0, g, t, [&](int mt, int nt, int e, int r, int c) { dQ[mt][nt][e] -= scale * V(vB)[r] * G[mt][nt][e]; });
-    add_rowsum(G, sQ, V(vdB), -scale);
-    zero(G);
-    warp_mma(G, oDRH, oSt_dv, kD, m0, n0, lane);
-    warp_mma(G, oDRL, oSt_dv, kD, m0, n0, lane);
+    warp_mma(G, tile_mk(kR3), st_dv(kR2), kD, m0, n0, lane);
+    warp_mma(G, tile_mk(kR3 + kTile), st_dv(kR2), kD, m0, n0, lane);
     for_frag<2, 4>(m0, n0, g, t, [&](int mt, int nt, int e, int r, int c) { dK[mt][nt][e] += V(vP)[r] * G[mt][nt][e]; });
     add_rowsum(G, sK, V(vdP), 1.f);
   }
+  __syncthreads();   // M has been read: its area takes gamma and m
 
-  // ---- gamma and m by the column recurrences of Eq. 10 (thread = column), into the area R / dV~ used
+  // ---- gamma and m by the column recurrences of Eq. 10 (thread = column)
   if (tid < C) {
     const int i = tid;
     float m = 1.f, gam = 0.f;
@@ -351,14 +340,14 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
   // ---- the four 64 x 64 products
   float P1[2][2][4], P2[2][2][4], QK[2][2][4], KK[2][2][4];
   zero(P1); zero(P2); zero(QK); zero(KK);
-  warp_mma(P1, oDO, oVtH, kD, m0, n064, lane);                        // dO V~^T
-  warp_mma(P1, oDO, oVtL, kD, m0, n064, lane);
-  warp_mma(P2, oDRH, oVtH, kD, m0, n064, lane);                       // dR V~^T
-  warp_mma(P2, oDRH, oVtL, kD, m0, n064, lane);
-  warp_mma(P2, oDRL, oVtH, kD, m0, n064, lane);
+  warp_mma(P1, oDO, tile_mk(kR1), kD, m0, n064, lane);                        // dO V~^T  (V~ as B: [n][k])
+  warp_mma(P1, oDO, tile_mk(kR1 + kTile), kD, m0, n064, lane);
+  warp_mma(P2, tile_mk(kR3), tile_mk(kR1), kD, m0, n064, lane);               // dR V~^T
+  warp_mma(P2, tile_mk(kR3), tile_mk(kR1 + kTile), kD, m0, n064, lane);
+  warp_mma(P2, tile_mk(kR3 + kTile), tile_mk(kR1), kD, m0, n064, lane);
   warp_mma(QK, oQ, oK, kD, m0, n064, lane);
   warp_mma(KK, oK, oK, kD, m0, n064, lane);
-  __syncthreads();   // V~, dR and the state are no longer read; gamma, m complete
+  __syncthreads();   // V~, dR and S are no longer read; gamma, m complete
   for_pair<2, 2>(m0, n064, g, t, [&](int mt, int nt, int hf, int r, int i0) {
     float dw[2], da[2];
 #pragma unroll
@@ -404,11 +393,11 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
   __syncthreads();   // d Geta, d G^- written; all row sums in; DW, DA have been read
   // per-(row, column) contributions to d alpha, d beta, d mu go to three matrices (the area DW, DA used) and are
   // summed along the rows afterwards: all columns reach a row in the same step, shared-memory atomics would serialise
-  float* cAl = reinterpret_cast<float*>(smem + kOffVt);
+  float* cAl = reinterpret_cast<float*>(smem + kR1);
   float* cBe = cAl + C * LG;
-  float* cMu = cBe + C * LG;
-  static_assert(3 * kMatF <= 4 * kTile, "contribution matrices");
-  for (int idx = tid; idx < 3 * C * LG; idx += kThreads) cAl[idx] = 0.f;
+  float* cMu = reinterpret_cast<float*>(smem + kR3);
+  static_assert(2 * kMatF <= 2 * kTile, "contribution matrices");
+  for (int idx = tid; idx < C * LG; idx += kThreads) { cAl[idx] = 0.f; cBe[idx] = 0.f; cMu[idx] = 0.f; }
   __syncthreads();
   if (tid < C) {
     const int i = tid;
@@ -520,7 +509,7 @@ cudaError_t launch_bwd_chunk_par(const Plan& fwd, const void* q, const void* k, 
   a.w_lo_offset = (size_t)fwd.geom.num_slots * fwd.p.H * C * C;
   a.fwd_states = static_cast<const uint8_t*>(fwd_states);
   a.adj_states = static_cast<const uint8_t*>(adj_states);
-  (void)v_ext;
+  a.v_ext = static_cast<const bf16*>(v_ext);
   a.scale = fwd.p.scale;
   a.dq = dq; a.dk = dk; a.dv = dv; a.dbeta = dbeta; a.dlog_alpha = dlog_alpha; a.dlog_mu = dlog_mu; a.deta = deta;
   cudaError_t e = cudaFuncSetAttribute(bwd_chunk_par_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmem);
