@@ -135,10 +135,12 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
   };
   auto cp_async_commit = []() { asm volatile("cp.async.commit_group;" ::: "memory"); };
   auto cp_async_wait = []() { asm volatile("cp.async.wait_group 0;" ::: "memory"); };
-  auto dot_images = [&](const uint8_t* x, const uint8_t* y) {   // sum of the element-wise product (same layout)
+  // sum of the element-wise product of two states resident in two areas ([128][LT] each, 16 pieces of 16 B per row)
+  auto dot_areas = [&](uint32_t x, uint32_t y) {
     float s = 0.f;
-    for (int idx = tid; idx < 2048; idx += kThreads) {
-      const uint4 ux = *reinterpret_cast<const uint4*>(x + idx * 16), uy = *reinterpret_cast<const uint4*>(y + idx * 16);
+    for (int idx = tid; idx < kD * 16; idx += kThreads) {
+      const uint32_t off = ((idx >> 4) * LT + (idx & 15) * 8) * 2;
+      const uint4 ux = *reinterpret_cast<const uint4*>(smem + x + off), uy = *reinterpret_cast<const uint4*>(smem + y + off);
       const uint32_t xs[4] = {ux.x, ux.y, ux.z, ux.w}, ys[4] = {uy.x, uy.y, uy.z, uy.w};
 #pragma unroll
       for (int e = 0; e < 4; ++e)
@@ -180,13 +182,11 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
       }
   };
 
-  // ---- everything this CTA will fetch later, towards L2 now (one CTA per SM: nothing else hides the latency)
-  for (int idx = tid; idx < 1024; idx += kThreads) {
-    const int which = idx >> 8, line = idx & 255;
-    const uint8_t* p = (which == 0 ? imgM : which == 1 ? imgdM : which == 2 ? imgdS : imgS) + line * 128;
-    asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
+  // ---- what this CTA fetches later (V, W^T dO), towards L2 now (one CTA per SM: nothing else hides the latency)
+  if (tid < C) {
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(a.v_ext + ((size_t)(e_real * C + tid) * H + h) * kD));
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(a.v_ext + ((size_t)(e_real * C + tid) * H + h) * kD + 64));
   }
-  if (tid < C) asm volatile("prefetch.global.L2 [%0];" ::"l"(a.v_ext + ((size_t)(e_real * C + tid) * H + h) * kD));
   if (tid < n) {
     asm volatile("prefetch.global.L2 [%0];" ::"l"(a.v + tok(tid) * kD));
     asm volatile("prefetch.global.L2 [%0];" ::"l"(a.v + tok(tid) * kD + 64));
@@ -205,43 +205,50 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
     V(vBeta)[r] = live ? a.beta[gi] : 0.f; V(vEta)[r] = live ? (a.eta ? a.eta[gi] : 1.f) : 0.f;
   }
   // Four areas of 34816 bytes (a state, or the hi + lo pair of a 64 x 128 tile) are reused through the phases:
-  //   R0: S                              | later d Geta, d G^-
-  //   R1: M            | V~ (hi, lo)     | later DW (hi, lo), then two contribution matrices
-  //   R2: dM'          | dV~ (hi, lo)    | M again | gamma, m
-  //   R3: R (hi, lo)   | dS'             | dR (hi, lo) | DA (hi, lo), then a contribution matrix
-  // States arrive by cp.async (no registers in between), each as early as its area is free.
+  //   R0: S                                               | later d Geta, d G^-
+  //   R1: M    | R (hi, lo) | V~ (hi, lo)                 | later DW (hi, lo), then two contribution matrices
+  //   R2: dM'               | dV~ (hi, lo) | M again      | gamma, m
+  //   R3: dS'                              | dR (hi, lo)  | DA (hi, lo), then a contribution matrix
+  // All four states arrive at the start by cp.async (no registers in between); M is fetched a second time later.
   load_state(imgS, kR0);
   load_state(imgM, kR1);
   load_state(imgdM, kR2);
+  load_state(imgdS, kR3);
   cp_async_commit();
   load_tile(sK, a.k);
   load_tile(sQ, a.q);
   load_tile(sDO, a.d_o);
   load_mat64(sT, a.T + mat);
-  {
-    const float s = dot_images(imgdM, imgM);                         // d mubar_C = <dM', M>
-    if (lane == 0) atomicAdd(V(vdMubar) + n - 1, s);
-  }
   cp_async_wait();
   __syncthreads();
   if (tid < C) V(vBprev)[tid] = tid > 0 ? V(vB)[tid - 1] : 0.f;
+  {   // the end-of-chunk adjoints: d mubar_C = <dM', M>, d abar_C = <dS', S>, d b_C = -<dS', M>
+    const float s0 = dot_areas(kR2, kR1), s1 = dot_areas(kR3, kR0), s2 = dot_areas(kR3, kR1);
+    if (lane == 0) {
+      atomicAdd(V(vdMubar) + n - 1, s0);
+      atomicAdd(V(vdAbar) + n - 1, s1);
+      atomicAdd(V(vdB) + n - 1, -s2);
+    }
+  }
 
   float dQ[2][4][4], dK[2][4][4];
   zero(dQ); zero(dK);
 
-  // ---- phase 1, with S and M: X = K S, Y = K M, R = V - abar.X + p.Y, V~ = T R; dO S^T, dO M^T (dQ, d abar, d b)
+  // ---- phase 1, everything that needs only the four states and k, dO:
+  //   X = K S, Y = K M -> R = V - abar.X + p.Y;  dO S^T, dO M^T (dQ, d abar, d b);
+  //   K dM', K dS' -> dV~ = W^T dO + g_S.(K dS') - g_M.(K dM')
+  float Rf[2][4][4], dVf[2][4][4];
   {
-    float X[2][4][4], Y[2][4][4];
-    zero(X); zero(Y);
-    warp_mma(X, oK, st_dk(kR0), kD, m0, n0, lane);
+    float Y[2][4][4];
+    zero(Rf); zero(Y);
+    warp_mma(Rf, oK, st_dk(kR0), kD, m0, n0, lane);
     warp_mma(Y, oK, st_dk(kR1), kD, m0, n0, lane);
     for_pair<2, 4>(m0, n0, g, t, [&](int mt, int nt, int hf, int r, int c) {
       const uint32_t v2 = r < n ? *reinterpret_cast<const uint32_t*>(a.v + tok(r) * kD + c) : 0u;
       const float ab = V(vAbar)[r], pp = V(vP)[r];
-      X[mt][nt][2 * hf] = __uint_as_float(v2 << 16) - ab * X[mt][nt][2 * hf] + pp * Y[mt][nt][2 * hf];
-      X[mt][nt][2 * hf + 1] = __uint_as_float(v2 & 0xffff0000u) - ab * X[mt][nt][2 * hf + 1] + pp * Y[mt][nt][2 * hf + 1];
+      Rf[mt][nt][2 * hf] = __uint_as_float(v2 << 16) - ab * Rf[mt][nt][2 * hf] + pp * Y[mt][nt][2 * hf];
+      Rf[mt][nt][2 * hf + 1] = __uint_as_float(v2 & 0xffff0000u) - ab * Rf[mt][nt][2 * hf + 1] + pp * Y[mt][nt][2 * hf + 1];
     });
-    put_split(X, kR3);
     zero(Y);
     warp_mma(Y, oDO, st_dv(kR0), kD, m0, n0, lane);                   // dO S^T
     for_frag<2, 4>(m0, n0, g, t, [&](int mt, int nt, int e, int r, int c) { dQ[mt][nt][e] += scale * V(vAbar)[r] * Y[mt][nt][e]; });
@@ -250,60 +257,51 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
     warp_mma(Y, oDO, st_dv(kR1), kD, m0, n0, lane);                   // dO M^T
     for_frag<2, 4>(m0, n0, g, t, [&](int mt, int nt, int e, int r, int c) { dQ[mt][nt][e] -= scale * V(vB)[r] * Y[mt][nt][e]; });
     add_rowsum(Y, sQ, V(vdB), -scale);
-    __syncthreads();   // R complete; M has been read
-    float Vt[2][4][4];
-    zero(Vt);
-    warp_mma(Vt, oT, tile_kn(kR3), C, m0, n0, lane);
-    warp_mma(Vt, oT, tile_kn(kR3 + kTile), C, m0, n0, lane);
-    put_split(Vt, kR1);
-  }
-  __syncthreads();   // V~ complete; R has been read
-  load_state(imgdS, kR3);
-  cp_async_commit();
-
-  // ---- phase 2, with dM' and dS': K dM', K dS', the g_S and g_M terms of dK, dV~ = W^T dO + g_S.(K dS') - g_M.(K dM'),
-  // dR = T^T dV~
-  {
-    float KdM[2][4][4], G[2][4][4];
-    zero(KdM); zero(G);
-    warp_mma(KdM, oK, st_dk(kR2), kD, m0, n0, lane);
-    warp_mma(G, tile_mk(kR1), st_dv(kR2), kD, m0, n0, lane);          // V~ dM'^T
-    warp_mma(G, tile_mk(kR1 + kTile), st_dv(kR2), kD, m0, n0, lane);
-    for_frag<2, 4>(m0, n0, g, t, [&](int mt, int nt, int e, int r, int c) { dK[mt][nt][e] -= V(vGM)[r] * G[mt][nt][e]; });
-    add_rowsum(G, sK, V(vdGM), -1.f);
-    {
-      const float s1 = dot_images(imgdS, imgS), s2 = dot_images(imgdS, imgM);   // d abar_C = <dS', S>, d b_C = -<dS', M>
-      if (lane == 0) { atomicAdd(V(vdAbar) + n - 1, s1); atomicAdd(V(vdB) + n - 1, -s2); }
-    }
-    cp_async_wait();
-    __syncthreads();   // dS' has landed; dM' has been read
-    float KdS[2][4][4];
-    zero(KdS); zero(G);
-    warp_mma(KdS, oK, st_dk(kR3), kD, m0, n0, lane);
-    warp_mma(G, tile_mk(kR1), st_dv(kR3), kD, m0, n0, lane);          // V~ dS'^T
-    warp_mma(G, tile_mk(kR1 + kTile), st_dv(kR3), kD, m0, n0, lane);
-    for_frag<2, 4>(m0, n0, g, t, [&](int mt, int nt, int e, int r, int c) { dK[mt][nt][e] += V(vGS)[r] * G[mt][nt][e]; });
-    add_rowsum(G, sK, V(vdGS), 1.f);
+    zero(dVf); zero(Y);
+    warp_mma(dVf, oK, st_dk(kR3), kD, m0, n0, lane);                  // K dS'
+    warp_mma(Y, oK, st_dk(kR2), kD, m0, n0, lane);                    // K dM'
     for_pair<2, 4>(m0, n0, g, t, [&](int mt, int nt, int hf, int r, int c) {
       // W^T dO as the adjoint chain's problem has it (bf16)
       const uint32_t v2 = r < n ? *reinterpret_cast<const uint32_t*>(a.v_ext + ((size_t)(e_real * C + r) * H + h) * kD + c) : 0u;
       const float gs = V(vGS)[r], gm = V(vGM)[r];
-      KdS[mt][nt][2 * hf] = __uint_as_float(v2 << 16) + gs * KdS[mt][nt][2 * hf] - gm * KdM[mt][nt][2 * hf];
-      KdS[mt][nt][2 * hf + 1] = __uint_as_float(v2 & 0xffff0000u) + gs * KdS[mt][nt][2 * hf + 1] - gm * KdM[mt][nt][2 * hf + 1];
+      dVf[mt][nt][2 * hf] = __uint_as_float(v2 << 16) + gs * dVf[mt][nt][2 * hf] - gm * Y[mt][nt][2 * hf];
+      dVf[mt][nt][2 * hf + 1] = __uint_as_float(v2 & 0xffff0000u) + gs * dVf[mt][nt][2 * hf + 1] - gm * Y[mt][nt][2 * hf + 1];
     });
-    put_split(KdS, kR2);
   }
-  __syncthreads();   // dV~ complete; dS' has been read
+  __syncthreads();   // M has been read: R takes its place
+  put_split(Rf, kR1);
+  __syncthreads();
+  zero(Rf);
+  warp_mma(Rf, oT, tile_kn(kR1), C, m0, n0, lane);                    // V~ = T R
+  warp_mma(Rf, oT, tile_kn(kR1 + kTile), C, m0, n0, lane);
+  __syncthreads();   // R has been read: V~ takes its place
+  put_split(Rf, kR1);
+  __syncthreads();
+
+  // ---- phase 2: the g_M and g_S terms of dK from V~ dM'^T, V~ dS'^T; then dR = T^T dV~
   {
-    float dR[2][4][4];
-    zero(dR);
-    warp_mma(dR, oT_t, tile_kn(kR2), C, m0, n0, lane);
-    warp_mma(dR, oT_t, tile_kn(kR2 + kTile), C, m0, n0, lane);
-    put_split(dR, kR3);
-    for_pair<2, 4>(m0, n0, g, t, [&](int mt, int nt, int hf, int r, int c) {
-      if (r < n) *reinterpret_cast<float2*>(a.dv + tok(r) * kD + c) = make_float2(dR[mt][nt][2 * hf], dR[mt][nt][2 * hf + 1]);
-    });
+    float G[2][4][4];
+    zero(G);
+    warp_mma(G, tile_mk(kR1), st_dv(kR2), kD, m0, n0, lane);          // V~ dM'^T
+    warp_mma(G, tile_mk(kR1 + kTile), st_dv(kR2), kD, m0, n0, lane);
+    for_frag<2, 4>(m0, n0, g, t, [&](int mt, int nt, int e, int r, int c) { dK[mt][nt][e] -= V(vGM)[r] * G[mt][nt][e]; });
+    add_rowsum(G, sK, V(vdGM), -1.f);
+    zero(G);
+    warp_mma(G, tile_mk(kR1), st_dv(kR3), kD, m0, n0, lane);          // V~ dS'^T
+    warp_mma(G, tile_mk(kR1 + kTile), st_dv(kR3), kD, m0, n0, lane);
+    for_frag<2, 4>(m0, n0, g, t, [&](int mt, int nt, int e, int r, int c) { dK[mt][nt][e] += V(vGS)[r] * G[mt][nt][e]; });
+    add_rowsum(G, sK, V(vdGS), 1.f);
   }
+  __syncthreads();   // dM', dS' have been read: dV~ takes dM's place
+  put_split(dVf, kR2);
+  __syncthreads();
+  zero(dVf);
+  warp_mma(dVf, oT_t, tile_kn(kR2), C, m0, n0, lane);                 // dR = T^T dV~
+  warp_mma(dVf, oT_t, tile_kn(kR2 + kTile), C, m0, n0, lane);
+  put_split(dVf, kR3);
+  for_pair<2, 4>(m0, n0, g, t, [&](int mt, int nt, int hf, int r, int c) {
+    if (r < n) *reinterpret_cast<float2*>(a.dv + tok(r) * kD + c) = make_float2(dVf[mt][nt][2 * hf], dVf[mt][nt][2 * hf + 1]);
+  });
   __syncthreads();   // dR complete; dV~ has been read
   load_state(imgM, kR2);
   cp_async_commit();
