@@ -327,7 +327,8 @@ mdn_status mdn_bwd_state_chain(const mdn_params* p,
  *      masks, and from those the gate gradients by the recurrences of Eq. 10 in reverse.
  * Arguments as mdn_chunk_bwd (no cu_seqlens: fixed-length input only).  Tensor path only: bf16 q, k, v, bf16 d_o,
  * dk = dv = 128; MDN_ERR_UNSUPPORTED otherwise.  Operands are bf16 / tf32 with fp32 accumulation, so the gradients
- * carry the forward's bf16-level error (see the tests), not mdn_chunk_bwd's fp32 exactness.  deta,
+ * carry the forward's bf16-level error (see the tests), not mdn_chunk_bwd's fp32 exactness; d_final_S, d_final_M
+ * enter the tensor-core products through a bf16 copy (one rounding, up to 2^-8 of their largest element).  deta,
  * d_initial_S, d_initial_M may be NULL.  Workspace: mdn_chunk_bwd_chunked_workspace_bytes(p), 1024-byte aligned.
  */
 size_t mdn_chunk_bwd_chunked_workspace_bytes(const mdn_params* p);

@@ -114,17 +114,20 @@ def test_bwd_state_chain(mdn, T, with_final):
 
 NAMES = [("dq", "dq"), ("dk", "dk"), ("dv", "dv"), ("dbeta", "dbeta"), ("dlog_alpha", "dlog_alpha"),
          ("dlog_mu", "dlog_mu"), ("deta", "deta"), ("d_initial_S", "dS0"), ("d_initial_M", "dM0")]
-# bf16 / tf32 operands with fp32 accumulation, bf16 chunk states and adjoint states: the forward's bf16 bar,
-# max |g - ref| / RMS(ref) <= 2e-2 per gradient tensor.  With final-state gradients passed in (drawn as dense random
-# matrices of standard deviation 0.1) the chunk next to them sees one bf16 rounding of those matrices in its largest
-# term, which in this max-over-elements metric reaches 3e-2 there (nowhere else); for those cases the bound is 4e-2,
-# and every case also has to meet an RMS bound, |g - ref|_2 / |ref|_2 <= 5e-3.
+# bf16 operands with fp32 accumulation, bf16 chunk states and adjoint states: the forward's bf16 bar,
+# max |g - ref| / RMS(ref) <= 2e-2 per gradient tensor, plus an RMS bound |g - ref|_2 / |ref|_2 <= 5e-3.
+# Like q, k, v and dO, the final-state gradients of these cases are bf16-representable values: they enter tensor-core
+# products through a bf16 copy.  One case passes unrounded fp32 final-state gradients (dense random matrices of
+# standard deviation 0.1 that dominate the last chunk): that chunk then carries one bf16 rounding of its largest
+# term, up to 2^-8 of it, which this max-over-elements metric shows as 2-3e-2 there (RMS error unchanged).
 TOL_CHUNKED = 2e-2
-TOL_CHUNKED_FINAL = 4e-2
+TOL_CHUNKED_FP32_FINAL = 4e-2
 TOL_CHUNKED_RMS = 5e-3
 
 
-def chunked_vs_oracle(mdn, w, seed, with_final=True, eta_none=False, chains=None):
+def chunked_vs_oracle(mdn, w, seed, with_final=True, eta_none=False, chains=None, round_final=True):
+    """chains: indices of the (sequence, head) chains the oracle evaluates (the others are NaN in its output and
+    skipped by the error metrics): full-size configurations are checked on a sample."""
     import oracle
     import torch
     inp = wl.make_inputs(w)
@@ -132,6 +135,8 @@ def chunked_vs_oracle(mdn, w, seed, with_final=True, eta_none=False, chains=None
     d_o = wl.round_to_bf16(r.standard_normal((w.B, w.T, w.H, w.dv)).astype(np.float32))
     dS = (0.1 * r.standard_normal((w.B, w.H, w.dk, w.dv))).astype(np.float32) if with_final else None
     dM = (0.1 * r.standard_normal((w.B, w.H, w.dk, w.dv))).astype(np.float32) if with_final else None
+    if with_final and round_final:
+        dS, dM = wl.round_to_bf16(dS), wl.round_to_bf16(dM)
     eta = None if eta_none else inp["eta"]
     ref = oracle.stepwise_bwd(inp["q"], inp["k"], inp["v"], inp["beta"], inp["log_alpha"], inp["log_mu"], eta, d_o,
                               scale=inp["scale"], S0=inp["S0"], M0=inp["M0"], dS_final=dS, dM_final=dM,
@@ -148,7 +153,8 @@ def chunked_vs_oracle(mdn, w, seed, with_final=True, eta_none=False, chains=None
             continue
         x, y = got[gname].cpu().numpy().astype(np.float64), ref[rname]
         errs[gname] = rel_err(x, y)
-        rms[gname] = float(np.sqrt(np.mean((x - y) ** 2)) / np.sqrt(np.mean(y ** 2)))
+        m = ~np.isnan(y)
+        rms[gname] = float(np.sqrt(np.mean((x[m] - y[m]) ** 2)) / np.sqrt(np.mean(y[m] ** 2)))
     print(w.name, "max/RMS:", " ".join("%s %.2e" % kv for kv in errs.items()))
     print(w.name, "RMS    :", " ".join("%s %.2e" % kv for kv in rms.items()))
     assert max(rms.values()) <= TOL_CHUNKED_RMS, rms
@@ -159,7 +165,13 @@ def chunked_vs_oracle(mdn, w, seed, with_final=True, eta_none=False, chains=None
 def test_chunked_backward_lengths(mdn, T):
     w = wl.Workload("chunked_T%d" % T, B=2, T=T, H=2, dk=128, dv=128, dtype="bf16", init_state_std=0.1, seed=90 + T % 7)
     errs = chunked_vs_oracle(mdn, w, T)
-    assert max(errs.values()) <= TOL_CHUNKED_FINAL, errs
+    assert max(errs.values()) <= TOL_CHUNKED, errs
+
+
+def test_chunked_backward_fp32_final_state_gradients(mdn):
+    w = wl.Workload("chunked_fp32_final", B=2, T=64 * 3 + 20, H=2, dk=128, dv=128, dtype="bf16", init_state_std=0.1, seed=93)
+    errs = chunked_vs_oracle(mdn, w, 212, round_final=False)
+    assert max(errs.values()) <= TOL_CHUNKED_FP32_FINAL, errs
 
 
 def test_chunked_backward_no_eta_no_final(mdn):
@@ -183,3 +195,15 @@ def test_chunked_backward_matches_stepwise_kernel(mdn):
         e = rel_err(x, y)
         print(name, "%.2e" % e)
         assert e <= TOL_CHUNKED, (name, e)
+
+
+def test_chunked_backward_config1_sampled(mdn):
+    """400M-layer shape at full size (B=4, H=8, T=2048), four sampled chains, no final-state gradients."""
+    errs = chunked_vs_oracle(mdn, wl.CONFIGS[1], 11, with_final=False, chains=np.array([0, 9, 18, 31]))
+    assert max(errs.values()) <= TOL_CHUNKED, errs
+
+
+def test_chunked_backward_config2_sampled(mdn):
+    """The launch configuration bench.py --backward times (B=8, H=16, T=4096), two sampled chains."""
+    errs = chunked_vs_oracle(mdn, wl.CONFIGS[2], 12, with_final=True, chains=np.array([3, 126]))
+    assert max(errs.values()) <= TOL_CHUNKED, errs
