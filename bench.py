@@ -490,10 +490,11 @@ def run_backward(args, w):
     gates = [dev(inp[n]) for n in ("beta", "log_alpha", "log_mu", "eta")]
     cu = None if inp["cu_seqlens"] is None else torch.from_numpy(inp["cu_seqlens"]).to("cuda")
     d_o = torch.randn(v.shape, device="cuda", generator=torch.Generator(device="cuda").manual_seed(1)).to(dt)
-    can_chunk = w.dtype == "bf16" and w.dk == 128 and w.dv == 128 and cu is None
+    can_chunk = w.dtype == "bf16" and w.dk == 128 and w.dv == 128
     method = args.bwd_method if args.bwd_method != "auto" else ("chunked" if can_chunk else "stepwise")
     if method == "chunked":
-        need = int(mdn.lib().mdn_chunk_bwd_chunked_workspace_bytes(ctypes.byref(mdn.make_params(q, v, path="tensor"))))
+        need = int(mdn.lib().mdn_chunk_bwd_chunked_workspace_bytes(ctypes.byref(
+            mdn.make_params(q, v, num_seqs=0 if cu is None else cu.numel() - 1, path="tensor"))))
     else:
         need = int(mdn.lib().mdn_chunk_bwd_workspace_bytes(ctypes.byref(mdn.make_params(q, v, num_seqs=0 if cu is None else cu.numel() - 1))))
     ws = torch.empty(need, dtype=torch.uint8, device="cuda")

@@ -293,11 +293,12 @@ mdn_status mdn_chunk_fwd_keep_states(const mdn_params* p,
  * walk the chunks of every sequence from the last to the first.  This has the shape of the forward's own chunk step
  * with the roles of S and M exchanged, so it is run by the forward's chain kernel on an extended problem (per
  * chunk a real step and a step that adds the two Q terms) built from the forward's workspace.
- *   p, q, k: the forward call's (tensor path, fixed-length input, o_dtype bf16); d_o = dL/do, [B,T,H,dv] bf16;
- *   d_final_S, d_final_M: dL/d(final states), [B,H,dk,dv] float32 or NULL (zero);
+ *   p, q, k, cu_seqlens: the forward call's (tensor path, o_dtype bf16); d_o = dL/do, [B,T,H,dv] bf16;
+ *   d_final_S, d_final_M: dL/d(final states), [N,H,dk,dv] float32 or NULL (zero);
  *   fwd_workspace: the workspace of an mdn_chunk_fwd_keep_states call with the same p and inputs, untouched since
  *     (T, W and the coefficient vectors are read from it);
- *   adjoint_states: DEVICE buffer of mdn_bwd_adjoint_states_bytes(p) bytes, 1024-byte aligned.  Per sequence and
+ *   adjoint_states: DEVICE buffer of mdn_bwd_adjoint_states_bytes(p) bytes, 1024-byte aligned.  Per sequence (in
+ *     the workspace's slot order, entries of sequence s starting at twice its first chunk slot) and
  *     head it receives 2 x nchunks entries of 65536 bytes in the layout of mdn_chunk_fwd_keep_states with dM^T in
  *     the first half and dS^T in the second: entry 2 (nchunks - 1 - c) is the adjoint pair at the END of chunk c,
  *     entry 2 (nchunks - 1 - c) + 1 the pair after chunk c's K terms and before its Q terms;
@@ -312,6 +313,7 @@ size_t mdn_bwd_adjoint_states_bytes(const mdn_params* p);
 mdn_status mdn_bwd_state_chain(const mdn_params* p,
                                const void* q, const void* k, const void* d_o,
                                const float* d_final_S, const float* d_final_M,
+                               const int32_t* cu_seqlens,
                                void* fwd_workspace, size_t fwd_workspace_bytes,
                                void* adjoint_states,
                                float* d_initial_S, float* d_initial_M,
@@ -325,7 +327,7 @@ mdn_status mdn_bwd_state_chain(const mdn_params* p,
  *   2. the adjoint state recurrence (mdn_bwd_state_chain),
  *   3. per (chunk, head), in parallel: dV = dR, dQ, dK, the adjoints of the coefficient vectors and of the two
  *      masks, and from those the gate gradients by the recurrences of Eq. 10 in reverse.
- * Arguments as mdn_chunk_bwd (no cu_seqlens: fixed-length input only).  Tensor path only: bf16 q, k, v, bf16 d_o,
+ * Arguments as mdn_chunk_bwd (fixed-length or packed input).  Tensor path only: bf16 q, k, v, bf16 d_o,
  * dk = dv = 128; MDN_ERR_UNSUPPORTED otherwise.  Operands are bf16 / tf32 with fp32 accumulation, so the gradients
  * carry the forward's bf16-level error (see the tests), not mdn_chunk_bwd's fp32 exactness; d_final_S, d_final_M
  * enter the tensor-core products through a bf16 copy (one rounding, up to 2^-8 of their largest element).  deta,
@@ -337,6 +339,7 @@ mdn_status mdn_chunk_bwd_chunked(const mdn_params* p,
                                  const void* q, const void* k, const void* v,
                                  const float* beta, const float* log_alpha, const float* log_mu, const float* eta,
                                  const float* initial_S, const float* initial_M,
+                                 const int32_t* cu_seqlens,
                                  const void* d_o, const float* d_final_S, const float* d_final_M,
                                  float* dq, float* dk, float* dv,
                                  float* dbeta, float* dlog_alpha, float* dlog_mu, float* deta,

@@ -91,11 +91,11 @@ def lib() -> ctypes.CDLL:
         L.mdn_bwd_adjoint_states_bytes.restype = ctypes.c_size_t
         L.mdn_bwd_adjoint_states_bytes.argtypes = [P]
         L.mdn_bwd_state_chain.restype = ctypes.c_int
-        L.mdn_bwd_state_chain.argtypes = [P] + [vp] * 6 + [ctypes.c_size_t] + [vp] * 4 + [ctypes.c_size_t, vp]
+        L.mdn_bwd_state_chain.argtypes = [P] + [vp] * 7 + [ctypes.c_size_t] + [vp] * 4 + [ctypes.c_size_t, vp]
         L.mdn_chunk_bwd_chunked_workspace_bytes.restype = ctypes.c_size_t
         L.mdn_chunk_bwd_chunked_workspace_bytes.argtypes = [P]
         L.mdn_chunk_bwd_chunked.restype = ctypes.c_int
-        L.mdn_chunk_bwd_chunked.argtypes = [P] + [vp] * 21 + [vp, ctypes.c_size_t, vp]
+        L.mdn_chunk_bwd_chunked.argtypes = [P] + [vp] * 22 + [vp, ctypes.c_size_t, vp]
         L.mdn_chunk_bwd.restype = ctypes.c_int
         L.mdn_chunk_bwd.argtypes = [P] + [vp] * 22 + [vp, ctypes.c_size_t, vp]
         L.mdn_chunk_bwd_workspace_bytes.restype = ctypes.c_size_t
@@ -335,23 +335,25 @@ def unpack_chunk_states(states: torch.Tensor, H: int):
     return full[:, :, 0].contiguous(), full[:, :, 1].contiguous()
 
 
-def bwd_state_chain(q, k, d_o, fwd_workspace, *, v_dim: int, d_final_S=None, d_final_M=None,
+def bwd_state_chain(q, k, d_o, fwd_workspace, *, v_dim: int, d_final_S=None, d_final_M=None, cu_seqlens=None,
                     scale: Optional[float] = None, want_initial: bool = True):
     """mdn_bwd_state_chain after a chunk_fwd(..., keep_chunk_states=True) call whose workspace is `fwd_workspace`.
     Returns (adjoint_states, d_initial_S, d_initial_M): the raw adjoint-state buffer (2 entries per chunk, see
     include/mdn.h; unpack_chunk_states gives (dM, dS) per entry) and the initial states' gradients."""
     B, T, H, dk = q.shape
-    p = make_params(q, d_o, scale=scale, o_dtype=torch.bfloat16, path="tensor")
+    N = 0 if cu_seqlens is None else cu_seqlens.numel() - 1
+    nst = N if N > 0 else B
+    p = make_params(q, d_o, num_seqs=N, scale=scale, o_dtype=torch.bfloat16, path="tensor")
     nbytes = int(lib().mdn_bwd_adjoint_states_bytes(ctypes.byref(p)))
     need = int(lib().mdn_bwd_state_chain_workspace_bytes(ctypes.byref(p)))
     if nbytes == 0 or need == 0:
         raise MdnError(2, "mdn_bwd_state_chain_workspace_bytes")
     adj = torch.empty(nbytes, dtype=torch.uint8, device=q.device)
     ws = torch.empty(need, dtype=torch.uint8, device=q.device)
-    dS0 = torch.empty((B, H, dk, v_dim), dtype=torch.float32, device=q.device) if want_initial else None
-    dM0 = torch.empty((B, H, dk, v_dim), dtype=torch.float32, device=q.device) if want_initial else None
+    dS0 = torch.empty((nst, H, dk, v_dim), dtype=torch.float32, device=q.device) if want_initial else None
+    dM0 = torch.empty((nst, H, dk, v_dim), dtype=torch.float32, device=q.device) if want_initial else None
     st = lib().mdn_bwd_state_chain(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(d_o), _ptr(d_final_S), _ptr(d_final_M),
-                                   _ptr(fwd_workspace), fwd_workspace.numel(), _ptr(adj), _ptr(dS0), _ptr(dM0),
+                                   _ptr(cu_seqlens), _ptr(fwd_workspace), fwd_workspace.numel(), _ptr(adj), _ptr(dS0), _ptr(dM0),
                                    _ptr(ws), ws.numel(), _stream())
     if st != 0:
         raise MdnError(st, "mdn_bwd_state_chain")
@@ -384,9 +386,7 @@ def chunk_bwd(q, k, v, beta, log_alpha, log_mu, eta, d_o, *, initial_S=None, ini
         raise ValueError("method")
     chunked = method == "chunked"
     if chunked:
-        if cu_seqlens is not None:
-            raise MdnError(2, "mdn_chunk_bwd_chunked: fixed-length input only")
-        p = make_params(q, v, scale=scale, o_dtype=d_o.dtype, path="tensor")
+        p = make_params(q, v, num_seqs=N, scale=scale, o_dtype=d_o.dtype, path="tensor")
         need = int(lib().mdn_chunk_bwd_chunked_workspace_bytes(ctypes.byref(p)))
     else:
         need = int(lib().mdn_chunk_bwd_workspace_bytes(ctypes.byref(p)))
@@ -402,8 +402,8 @@ def chunk_bwd(q, k, v, beta, log_alpha, log_mu, eta, d_o, *, initial_S=None, ini
              d_initial_S=torch.empty((nst, H, dk, dv), **f32), d_initial_M=torch.empty((nst, H, dk, dv), **f32))
     if chunked:
         st = lib().mdn_chunk_bwd_chunked(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(beta), _ptr(log_alpha),
-                                         _ptr(log_mu), _ptr(eta), _ptr(initial_S), _ptr(initial_M), _ptr(d_o),
-                                         _ptr(d_final_S), _ptr(d_final_M), _ptr(g["dq"]), _ptr(g["dk"]), _ptr(g["dv"]),
+                                         _ptr(log_mu), _ptr(eta), _ptr(initial_S), _ptr(initial_M), _ptr(cu_seqlens),
+                                         _ptr(d_o), _ptr(d_final_S), _ptr(d_final_M), _ptr(g["dq"]), _ptr(g["dk"]), _ptr(g["dv"]),
                                          _ptr(g["dbeta"]), _ptr(g["dlog_alpha"]), _ptr(g["dlog_mu"]), _ptr(g["deta"]),
                                          _ptr(g["d_initial_S"]), _ptr(g["d_initial_M"]), _ptr(workspace),
                                          workspace.numel(), _stream())

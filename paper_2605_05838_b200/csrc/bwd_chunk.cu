@@ -51,9 +51,10 @@ __global__ void __launch_bounds__(kPrepThreads) bwd_prep_kernel(PrepArgs a) {
   const SlotInfo si = slot_info(a.g, slot);
   if (si.seq < 0) return;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
-  const int nch = a.g.chunks_per_seq;
+  int slot0, nch;
+  seq_chunks(a.g, si.seq, &slot0, &nch);
   // extended chunk indices of this forward chunk: the real step, then the injection step
-  const int e_real = si.seq * 2 * nch + 2 * (nch - 1 - si.local), e_inj = e_real + 1;
+  const int e_real = 2 * slot0 + 2 * (nch - 1 - si.local), e_inj = e_real + 1;
   const size_t mat = ((size_t)slot * H + h) * C * C;
 
   // ---- W (hi, lo), T and the dO tile into shared memory; dO also goes out as the "V" of the injection step
@@ -133,7 +134,18 @@ __global__ void __launch_bounds__(kPrepThreads) bwd_prep_kernel(PrepArgs a) {
   }
 }
 
+// cu_seqlens of the extended problem (packed input): sequence s has 2 x 64 tokens per chunk
+__global__ void bwd_ext_cu_kernel(const int32_t* __restrict__ chunk_off, int num_seqs, int32_t* __restrict__ cu_ext) {
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i <= num_seqs; i += gridDim.x * blockDim.x) cu_ext[i] = 2 * C * chunk_off[i];
+}
+
 }  // namespace
+
+cudaError_t launch_bwd_ext_cu(const Plan& fwd, int32_t* cu_ext, int* launches) {
+  bwd_ext_cu_kernel<<<1, 256, 0, fwd.stream>>>(fwd.geom.chunk_off, fwd.geom.num_seqs, cu_ext);
+  ++*launches;
+  return cudaGetLastError();
+}
 
 size_t bwd_prep_smem_bytes() { return (size_t)3 * C * L6 * 2 + (size_t)C * LT * 2; }
 

@@ -83,13 +83,15 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
   const int slot = blockIdx.x / a.g.H, h = blockIdx.x % a.g.H, H = a.g.H;
   const SlotInfo si = slot_info(a.g, slot);
   if (si.seq < 0) return;
-  const int n = si.n, nch = a.g.chunks_per_seq;
+  const int n = si.n;
+  int slot0, nch;
+  seq_chunks(a.g, si.seq, &slot0, &nch);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
   const int m0 = 32 * (warp & 1), n0 = 32 * (warp >> 1), n064 = 16 * (warp >> 1);   // the warp's block of a 64x128 / 64x64 result
   const size_t mat = ((size_t)slot * H + h) * C * C;
   const uint8_t* imgS = a.fwd_states + ((size_t)slot * H + h) * 65536;
   const uint8_t* imgM = imgS + 32768;
-  const int e_real = si.seq * 2 * nch + 2 * (nch - 1 - si.local);
+  const int e_real = 2 * slot0 + 2 * (nch - 1 - si.local);
   const uint8_t* imgdM = a.adj_states + ((size_t)e_real * H + h) * 65536;   // roles exchanged in the adjoint run
   const uint8_t* imgdS = imgdM + 32768;
   const float scale = a.scale;

@@ -30,7 +30,8 @@ __global__ void __launch_bounds__(1024) chunk_map_kernel(const int32_t* __restri
   const int tid = threadIdx.x;
   if (tid == 0) { s_carry = 0; s_bad = 0; }
   __syncthreads();
-  if (tid == 0 && (cu[0] != 0 || cu[num_seqs] != T)) s_bad = 1;
+  // T < 0: the total may fall short of -T (the caller pads its problem to a bound)
+  if (tid == 0 && (cu[0] != 0 || (T >= 0 ? cu[num_seqs] != T : cu[num_seqs] > -T))) s_bad = 1;
   for (int base = 0; base < num_seqs; base += 1024) {
     const int i = base + tid;
     int nch = 0;
@@ -78,7 +79,8 @@ __global__ void __launch_bounds__(1024) chunk_map_kernel(const int32_t* __restri
 
 cudaError_t launch_chunk_map(const Plan& pl, int* launches) {
   if (pl.geom.cu == nullptr) return cudaSuccess;
-  chunk_map_kernel<<<1, 1024, 0, pl.stream>>>(pl.geom.cu, pl.geom.num_seqs, pl.p.T, pl.geom.num_slots,
+  chunk_map_kernel<<<1, 1024, 0, pl.stream>>>(pl.geom.cu, pl.geom.num_seqs, pl.cu_total_may_be_short ? -pl.p.T : pl.p.T,
+                                              pl.geom.num_slots,
                                               const_cast<int32_t*>(pl.geom.chunk_off),
                                               const_cast<int32_t*>(pl.geom.slot_map),
                                               reinterpret_cast<int32_t*>(pl.ws + pl.lay.off_status));

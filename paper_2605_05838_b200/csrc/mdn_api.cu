@@ -221,22 +221,33 @@ mdn_status mdn_chunk_fwd_keep_states(const mdn_params* p, const void* q, const v
 }
 
 // ---- chunk-parallel backward, stage 1: the adjoint of the inter-chunk state recurrence
-struct AdjLayout { mdn_params pe; mdn_ws_layout le; uint64_t k_ext, v_ext, ws_ext, total; };
+struct AdjLayout { mdn_params pe; mdn_ws_layout le; uint64_t k_ext, v_ext, ws_ext, cu_ext, total; };
 
 static mdn_status adj_layout(const mdn_params* p, AdjLayout* a) {
   mdn_status st = check_params(p);
   if (st != MDN_OK) return st;
-  if (resolve_path(*p) != MDN_PATH_TENSOR || p->num_seqs > 0) return MDN_ERR_UNSUPPORTED;
+  if (resolve_path(*p) != MDN_PATH_TENSOR) return MDN_ERR_UNSUPPORTED;
   a->pe = *p;
-  a->pe.T = 2 * ((p->T + p->chunk - 1) / p->chunk) * p->chunk;   // a real and an injection step per chunk
   a->pe.segments = 1;
   a->pe.path = MDN_PATH_TENSOR;
+  if (p->num_seqs > 0) {   // packed: every chunk slot of the forward, padded to 64 rows, twice (host-side bound)
+    mdn_params pf = *p;
+    pf.segments = 1;
+    mdn_ws_layout lf;
+    st = make_layout(pf, &lf);
+    if (st != MDN_OK) return st;
+    a->pe.B = 1;
+    a->pe.T = 2 * p->chunk * (int)lf.num_slots;
+  } else {
+    a->pe.T = 2 * ((p->T + p->chunk - 1) / p->chunk) * p->chunk;   // a real and an injection step per chunk
+  }
   st = make_layout(a->pe, &a->le);
   if (st != MDN_OK) return st;
-  const uint64_t rows = (uint64_t)p->B * a->pe.T * p->H * p->dk * 2;
+  const uint64_t rows = (uint64_t)a->pe.B * a->pe.T * p->H * p->dk * 2;
   uint64_t off = 0;
   auto take = [&](uint64_t bytes) { uint64_t at = off; off = align_up(off + bytes, 1024); return at; };
-  a->k_ext = take(rows); a->v_ext = take(rows); a->ws_ext = take(a->le.total_bytes); a->total = off;
+  a->k_ext = take(rows); a->v_ext = take(rows); a->ws_ext = take(a->le.total_bytes);
+  a->cu_ext = take((uint64_t)(p->num_seqs + 1) * 4); a->total = off;
   return MDN_OK;
 }
 
@@ -251,8 +262,8 @@ size_t mdn_bwd_adjoint_states_bytes(const mdn_params* p) {
 }
 
 mdn_status mdn_bwd_state_chain(const mdn_params* p, const void* q, const void* k, const void* d_o,
-                               const float* d_final_S, const float* d_final_M, void* fwd_workspace,
-                               size_t fwd_workspace_bytes, void* adjoint_states, float* d_initial_S,
+                               const float* d_final_S, const float* d_final_M, const int32_t* cu_seqlens,
+                               void* fwd_workspace, size_t fwd_workspace_bytes, void* adjoint_states, float* d_initial_S,
                                float* d_initial_M, void* workspace, size_t workspace_bytes, void* cuda_stream) {
   t_last_launches = 0;
   AdjLayout al;
@@ -265,14 +276,20 @@ mdn_status mdn_bwd_state_chain(const mdn_params* p, const void* q, const void* k
   mdn_params pf = *p;
   pf.segments = 1;
   Plan fwd;
-  st = make_plan(&pf, nullptr, fwd_workspace, fwd_workspace_bytes, cuda_stream, &fwd);
+  st = make_plan(&pf, cu_seqlens, fwd_workspace, fwd_workspace_bytes, cuda_stream, &fwd);
   if (st != MDN_OK) return st;
   char* w = static_cast<char*>(workspace);
+  int32_t* cu_ext = p->num_seqs > 0 ? reinterpret_cast<int32_t*>(w + al.cu_ext) : nullptr;
   Plan ext;
-  st = make_plan(&al.pe, nullptr, w + al.ws_ext, al.le.total_bytes, cuda_stream, &ext);
+  st = make_plan(&al.pe, cu_ext, w + al.ws_ext, al.le.total_bytes, cuda_stream, &ext);
   if (st != MDN_OK) return st;
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   if (cudaMemsetAsync(ext.ws + ext.lay.off_status, 0, 16, s) != cudaSuccess) return MDN_ERR_CUDA;
+  if (cu_ext) {   // the chunk map of the extended problem: 2 x 64 tokens per chunk of every sequence
+    ext.cu_total_may_be_short = 1;
+    if (launch_bwd_ext_cu(fwd, cu_ext, &t_last_launches) != cudaSuccess || launch_chunk_map(ext, &t_last_launches) != cudaSuccess)
+      return MDN_ERR_CUDA;
+  }
   cudaError_t e = launch_bwd_prep(fwd, q, k, d_o, w + al.k_ext, w + al.v_ext,
                                   reinterpret_cast<float*>(ext.ws + ext.lay.off_coef), ext.ws + ext.lay.off_T,
                                   &t_last_launches);
@@ -314,11 +331,13 @@ size_t mdn_chunk_bwd_chunked_workspace_bytes(const mdn_params* p) {
 
 mdn_status mdn_chunk_bwd_chunked(const mdn_params* p, const void* q, const void* k, const void* v, const float* beta,
                                  const float* log_alpha, const float* log_mu, const float* eta,
-                                 const float* initial_S, const float* initial_M, const void* d_o,
-                                 const float* d_final_S, const float* d_final_M, float* dq, float* dk, float* dv,
+                                 const float* initial_S, const float* initial_M, const int32_t* cu_seqlens,
+                                 const void* d_o, const float* d_final_S, const float* d_final_M, float* dq, float* dk,
+                                 float* dv,
                                  float* dbeta, float* dlog_alpha, float* dlog_mu, float* deta, float* d_initial_S,
                                  float* d_initial_M, void* workspace, size_t workspace_bytes, void* cuda_stream) {
   t_last_launches = 0;
+  if (p && (p->num_seqs > 0) != (cu_seqlens != nullptr)) return MDN_ERR_INVALID_ARG;
   ChunkedBwdLayout c;
   mdn_status st = chunked_bwd_layout(p, &c);
   if (st != MDN_OK) return st;
@@ -331,7 +350,7 @@ mdn_status mdn_chunk_bwd_chunked(const mdn_params* p, const void* q, const void*
   mdn_params pf = *p;
   pf.segments = 1;
   Plan fwd;
-  st = make_plan(&pf, nullptr, w + c.ws_fwd, c.lf.total_bytes, cuda_stream, &fwd);
+  st = make_plan(&pf, cu_seqlens, w + c.ws_fwd, c.lf.total_bytes, cuda_stream, &fwd);
   if (st != MDN_OK) return st;
   fwd.chain_dump = reinterpret_cast<uint8_t*>(w + c.fwd_states);
   fwd.chain_state_only = 1;
@@ -340,7 +359,7 @@ mdn_status mdn_chunk_bwd_chunked(const mdn_params* p, const void* q, const void*
   if (st != MDN_OK) return st;
   const int launches_fwd = t_last_launches;
   // 2. the adjoint state chain
-  st = mdn_bwd_state_chain(p, q, k, d_o, d_final_S, d_final_M, w + c.ws_fwd, c.lf.total_bytes, w + c.adj_states,
+  st = mdn_bwd_state_chain(p, q, k, d_o, d_final_S, d_final_M, cu_seqlens, w + c.ws_fwd, c.lf.total_bytes, w + c.adj_states,
                            d_initial_S, d_initial_M, w + c.stage, c.al.total, cuda_stream);
   if (st != MDN_OK) return st;
   t_last_launches += launches_fwd;

@@ -66,6 +66,12 @@ __device__ __forceinline__ SlotInfo slot_info(const ChunkGeom& g, int slot) {
   return s;
 }
 
+// First chunk slot of a sequence and its chunk count (fixed-length or packed), for the per-chunk backward kernels.
+__device__ __forceinline__ void seq_chunks(const ChunkGeom& g, int seq, int* slot0, int* nch) {
+  if (g.cu == nullptr) { *slot0 = seq * g.chunks_per_seq; *nch = g.chunks_per_seq; }
+  else { *slot0 = g.chunk_off[seq]; *nch = g.chunk_off[seq + 1] - *slot0; }
+}
+
 // Range of chunk slots and tokens of one sequence (for the chain kernels).
 struct SeqInfo { int slot0, nchunks, tok0, len; };
 
@@ -136,6 +142,7 @@ struct Plan {
   uint8_t* chain_dump = nullptr;
   int chain_state_only = 0;
   int chain_end_scalars_in_rk = 0;
+  int cu_total_may_be_short = 0;   // packed: cu[N] <= T instead of == T (the adjoint chain's padded problem)
 };
 
 // Launchers (one per .cu file).  Each returns the CUDA error of its launches and adds
@@ -147,6 +154,7 @@ cudaError_t launch_bwd_chunk_par(const Plan& fwd, const void* q, const void* k, 
                                  const void* fwd_states, const void* adj_states, const void* v_ext, float* dq, float* dk,
                                  float* dv, float* dbeta, float* dlog_alpha, float* dlog_mu, float* deta, int* launches);
 // bwd_chunk.cu: builds the extended problem of the adjoint state chain from the forward's workspace
+cudaError_t launch_bwd_ext_cu(const Plan& fwd, int32_t* cu_ext, int* launches);
 cudaError_t launch_bwd_prep(const Plan& fwd, const void* q, const void* k, const void* d_o, void* k_ext, void* v_ext,
                             float* coef_ext, void* T_ext, int* launches);
 cudaError_t launch_coeff_scan(const Plan& pl, const float* beta, const float* log_alpha,

@@ -133,8 +133,9 @@ def chunked_vs_oracle(mdn, w, seed, with_final=True, eta_none=False, chains=None
     inp = wl.make_inputs(w)
     r = np.random.default_rng([seed, 78])
     d_o = wl.round_to_bf16(r.standard_normal((w.B, w.T, w.H, w.dv)).astype(np.float32))
-    dS = (0.1 * r.standard_normal((w.B, w.H, w.dk, w.dv))).astype(np.float32) if with_final else None
-    dM = (0.1 * r.standard_normal((w.B, w.H, w.dk, w.dv))).astype(np.float32) if with_final else None
+    N = len(inp["seq_len"])
+    dS = (0.1 * r.standard_normal((N, w.H, w.dk, w.dv))).astype(np.float32) if with_final else None
+    dM = (0.1 * r.standard_normal((N, w.H, w.dk, w.dv))).astype(np.float32) if with_final else None
     if with_final and round_final:
         dS, dM = wl.round_to_bf16(dS), wl.round_to_bf16(dM)
     eta = None if eta_none else inp["eta"]
@@ -145,6 +146,7 @@ def chunked_vs_oracle(mdn, w, seed, with_final=True, eta_none=False, chains=None
     dev = lambda x, d=torch.float32: None if x is None else torch.from_numpy(np.ascontiguousarray(x)).to("cuda").to(d)
     got = mdn.chunk_bwd(dev(inp["q"], bf), dev(inp["k"], bf), dev(inp["v"], bf), dev(inp["beta"]), dev(inp["log_alpha"]),
                         dev(inp["log_mu"]), dev(eta), dev(d_o, bf), initial_S=dev(inp["S0"]), initial_M=dev(inp["M0"]),
+                        cu_seqlens=None if inp["cu_seqlens"] is None else torch.from_numpy(inp["cu_seqlens"]).to("cuda"),
                         d_final_S=dev(dS), d_final_M=dev(dM), scale=inp["scale"], method="chunked")
     torch.cuda.synchronize()
     errs, rms = {}, {}
@@ -206,4 +208,12 @@ def test_chunked_backward_config1_sampled(mdn):
 def test_chunked_backward_config2_sampled(mdn):
     """The launch configuration bench.py --backward times (B=8, H=16, T=4096), two sampled chains."""
     errs = chunked_vs_oracle(mdn, wl.CONFIGS[2], 12, with_final=True, chains=np.array([3, 126]))
+    assert max(errs.values()) <= TOL_CHUNKED, errs
+
+
+def test_chunked_backward_packed(mdn):
+    """Packed sequences of uneven lengths (state and adjoint reset at every boundary, short last chunks)."""
+    w = wl.Workload("chunked_packed", B=1, T=900, H=2, dk=128, dv=128, dtype="bf16", varlen=True, len_lo=20, len_hi=330,
+                    init_state_std=0.1, seed=98)
+    errs = chunked_vs_oracle(mdn, w, 21)
     assert max(errs.values()) <= TOL_CHUNKED, errs
