@@ -113,18 +113,21 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
   const Opnd oDAH_t{sb + kR3, L6 * 2, true}, oDAL_t{sb + kR3 + kMat6, L6 * 2, true};
 
   auto tok = [&](int r) { return (size_t)(si.tok0 + r) * H + h; };
-  auto load_tile = [&](bf16* dst, const bf16* src) {
+  // everything arrives by cp.async (no registers in between, nothing blocks until the wait); rows past the chunk's
+  // end are zero-filled (source size 0)
+  auto cp16 = [&](uint32_t dst, const void* src, bool live) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(live ? 16 : 0));
+  };
+  auto load_tile = [&](uint32_t base, const bf16* src) {
     for (int idx = tid; idx < C * 16; idx += kThreads) {
       const int r = idx >> 4, c8 = (idx & 15) * 8;
-      uint4 x = make_uint4(0u, 0u, 0u, 0u);
-      if (r < n) x = *reinterpret_cast<const uint4*>(src + tok(r) * kD + c8);
-      *reinterpret_cast<uint4*>(dst + r * LT + c8) = x;
+      cp16(sb + base + (r * LT + c8) * 2, src + tok(r < n ? r : 0) * kD + c8, r < n);
     }
   };
-  auto load_mat64 = [&](bf16* dst, const bf16* src) {   // a [64][64] bf16 matrix -> [64][L6]
+  auto load_mat64 = [&](uint32_t base, const bf16* src) {   // a [64][64] bf16 matrix -> [64][L6]
     for (int idx = tid; idx < C * 8; idx += kThreads) {
       const int r = idx >> 3, c8 = (idx & 7) * 8;
-      *reinterpret_cast<uint4*>(dst + r * L6 + c8) = *reinterpret_cast<const uint4*>(src + r * C + c8);
+      cp16(sb + base + (r * L6 + c8) * 2, src + r * C + c8, true);
     }
   };
   // state image (value index j x key index d, two swizzled blocks) -> [j][d] in an area, by cp.async
@@ -193,6 +196,21 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
     asm volatile("prefetch.global.L2 [%0];" ::"l"(a.v + tok(tid) * kD));
     asm volatile("prefetch.global.L2 [%0];" ::"l"(a.v + tok(tid) * kD + 64));
   }
+  // Four areas of 34816 bytes (a state, or the hi + lo pair of a 64 x 128 tile) are reused through the phases:
+  //   R0: S                                               | later d Geta, d G^-
+  //   R1: M    | R (hi, lo) | V~ (hi, lo)                 | later DW (hi, lo), then two contribution matrices
+  //   R2: dM'               | dV~ (hi, lo) | M again      | gamma, m
+  //   R3: dS'                              | dR (hi, lo)  | DA (hi, lo), then a contribution matrix
+  // All four states arrive at the start by cp.async (no registers in between); M is fetched a second time later.
+  load_state(imgS, kR0);
+  load_state(imgM, kR1);
+  load_state(imgdM, kR2);
+  load_state(imgdS, kR3);
+  load_tile(kOffK, a.k);
+  load_tile(kOffQ, a.q);
+  load_tile(kOffDO, a.d_o);
+  load_mat64(kOffT, a.T + mat);
+  cp_async_commit();
   // ---- vectors: the chain's coefficient vectors, the gates, zeroed adjoints
   const float* cf = a.coef + ((size_t)slot * H + h) * MDN_NUM_COEF * C;
   for (int idx = tid; idx < 24 * C; idx += kThreads) vec[idx] = 0.f;
@@ -206,21 +224,6 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
     V(vAlpha)[r] = live ? expf(a.log_alpha[gi]) : 1.f; V(vMu)[r] = live ? expf(a.log_mu[gi]) : 1.f;
     V(vBeta)[r] = live ? a.beta[gi] : 0.f; V(vEta)[r] = live ? (a.eta ? a.eta[gi] : 1.f) : 0.f;
   }
-  // Four areas of 34816 bytes (a state, or the hi + lo pair of a 64 x 128 tile) are reused through the phases:
-  //   R0: S                                               | later d Geta, d G^-
-  //   R1: M    | R (hi, lo) | V~ (hi, lo)                 | later DW (hi, lo), then two contribution matrices
-  //   R2: dM'               | dV~ (hi, lo) | M again      | gamma, m
-  //   R3: dS'                              | dR (hi, lo)  | DA (hi, lo), then a contribution matrix
-  // All four states arrive at the start by cp.async (no registers in between); M is fetched a second time later.
-  load_state(imgS, kR0);
-  load_state(imgM, kR1);
-  load_state(imgdM, kR2);
-  load_state(imgdS, kR3);
-  cp_async_commit();
-  load_tile(sK, a.k);
-  load_tile(sQ, a.q);
-  load_tile(sDO, a.d_o);
-  load_mat64(sT, a.T + mat);
   cp_async_wait();
   __syncthreads();
   if (tid < C) V(vBprev)[tid] = tid > 0 ? V(vB)[tid - 1] : 0.f;
