@@ -347,6 +347,26 @@ mdn_status mdn_chunk_bwd_chunked(const mdn_params* p,
                                  void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * The same backward for a caller that kept what the forward produced (the usual save-for-backward trade): steps 2
+ * and 3 of mdn_chunk_bwd_chunked on the workspace and the chunk states of an mdn_chunk_fwd_keep_states call with the
+ * same p and inputs, both untouched since.  Saves the second intra-chunk pass and the state-only forward; the price
+ * is keeping that workspace and mdn_chunk_states_bytes(p) alive between the two calls.  Other arguments and the
+ * results as mdn_chunk_bwd_chunked; workspace: mdn_chunk_bwd_saved_workspace_bytes(p), 1024-byte aligned.
+ */
+size_t mdn_chunk_bwd_saved_workspace_bytes(const mdn_params* p);
+
+mdn_status mdn_chunk_bwd_saved(const mdn_params* p,
+                               const void* q, const void* k, const void* v,
+                               const float* beta, const float* log_alpha, const float* log_mu, const float* eta,
+                               const int32_t* cu_seqlens,
+                               void* fwd_workspace, size_t fwd_workspace_bytes, const void* chunk_states,
+                               const void* d_o, const float* d_final_S, const float* d_final_M,
+                               float* dq, float* dk, float* dv,
+                               float* dbeta, float* dlog_alpha, float* dlog_mu, float* deta,
+                               float* d_initial_S, float* d_initial_M,
+                               void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * Backward of mdn_chunk_fwd (Section 3.1: the training pass differentiates the same recurrence; like the paper's
  * kernels this keeps no per-token states and rebuilds them from per-chunk checkpoints):
  * given d_o = dL/do ([B,T,H,dv], o_dtype) and optionally dL/d(final_S), dL/d(final_M) ([N,H,dk,dv] float32, NULL =

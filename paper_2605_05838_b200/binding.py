@@ -96,6 +96,10 @@ def lib() -> ctypes.CDLL:
         L.mdn_chunk_bwd_chunked_workspace_bytes.argtypes = [P]
         L.mdn_chunk_bwd_chunked.restype = ctypes.c_int
         L.mdn_chunk_bwd_chunked.argtypes = [P] + [vp] * 22 + [vp, ctypes.c_size_t, vp]
+        L.mdn_chunk_bwd_saved_workspace_bytes.restype = ctypes.c_size_t
+        L.mdn_chunk_bwd_saved_workspace_bytes.argtypes = [P]
+        L.mdn_chunk_bwd_saved.restype = ctypes.c_int
+        L.mdn_chunk_bwd_saved.argtypes = [P] + [vp] * 9 + [ctypes.c_size_t] + [vp] * 13 + [vp, ctypes.c_size_t, vp]
         L.mdn_chunk_bwd.restype = ctypes.c_int
         L.mdn_chunk_bwd.argtypes = [P] + [vp] * 22 + [vp, ctypes.c_size_t, vp]
         L.mdn_chunk_bwd_workspace_bytes.restype = ctypes.c_size_t
@@ -362,10 +366,11 @@ def bwd_state_chain(q, k, d_o, fwd_workspace, *, v_dim: int, d_final_S=None, d_f
 
 def chunk_bwd(q, k, v, beta, log_alpha, log_mu, eta, d_o, *, initial_S=None, initial_M=None, cu_seqlens=None,
               d_final_S=None, d_final_M=None, scale: Optional[float] = None, workspace: Optional[torch.Tensor] = None,
-              method: str = "stepwise"):
+              method: str = "stepwise", saved=None):
     """mdn_chunk_bwd (method="stepwise": exact, fp32, token by token) or mdn_chunk_bwd_chunked (method="chunked":
     chunk-parallel on the tensor cores; bf16 inputs, dk = dv = 128, fixed length) on CUDA tensors (current stream):
-    gradients of mdn_chunk_fwd's outputs' loss.
+    gradients of mdn_chunk_fwd's outputs' loss.  saved = (fwd_workspace, chunk_states) of a chunk_fwd(...,
+    keep_chunk_states=True) call with the same inputs: mdn_chunk_bwd_saved (method="chunked" only).
     d_o: [B,T,H,dv] (its dtype is taken as the forward's o_dtype).  Returns a dict of float32 tensors
     dq, dk, dv, dbeta, dlog_alpha, dlog_mu, deta (None when eta is None), d_initial_S, d_initial_M."""
     _check_inputs(q, k, v, (("beta", beta), ("log_alpha", log_alpha), ("log_mu", log_mu), ("eta", eta)), "cuda")
@@ -387,7 +392,8 @@ def chunk_bwd(q, k, v, beta, log_alpha, log_mu, eta, d_o, *, initial_S=None, ini
     chunked = method == "chunked"
     if chunked:
         p = make_params(q, v, num_seqs=N, scale=scale, o_dtype=d_o.dtype, path="tensor")
-        need = int(lib().mdn_chunk_bwd_chunked_workspace_bytes(ctypes.byref(p)))
+        need = int(lib().mdn_chunk_bwd_saved_workspace_bytes(ctypes.byref(p)) if saved is not None
+                   else lib().mdn_chunk_bwd_chunked_workspace_bytes(ctypes.byref(p)))
     else:
         need = int(lib().mdn_chunk_bwd_workspace_bytes(ctypes.byref(p)))
     if need == 0:
@@ -400,6 +406,17 @@ def chunk_bwd(q, k, v, beta, log_alpha, log_mu, eta, d_o, *, initial_S=None, ini
              dlog_alpha=torch.empty((B, T, H), **f32), dlog_mu=torch.empty((B, T, H), **f32),
              deta=torch.empty((B, T, H), **f32) if eta is not None else None,
              d_initial_S=torch.empty((nst, H, dk, dv), **f32), d_initial_M=torch.empty((nst, H, dk, dv), **f32))
+    if chunked and saved is not None:
+        fws, fstates = saved
+        st = lib().mdn_chunk_bwd_saved(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(beta), _ptr(log_alpha), _ptr(log_mu),
+                                       _ptr(eta), _ptr(cu_seqlens), _ptr(fws), fws.numel(), _ptr(fstates), _ptr(d_o),
+                                       _ptr(d_final_S), _ptr(d_final_M), _ptr(g["dq"]), _ptr(g["dk"]), _ptr(g["dv"]),
+                                       _ptr(g["dbeta"]), _ptr(g["dlog_alpha"]), _ptr(g["dlog_mu"]), _ptr(g["deta"]),
+                                       _ptr(g["d_initial_S"]), _ptr(g["d_initial_M"]), _ptr(workspace),
+                                       workspace.numel(), _stream())
+        if st != 0:
+            raise MdnError(st, "mdn_chunk_bwd_saved")
+        return g
     if chunked:
         st = lib().mdn_chunk_bwd_chunked(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(beta), _ptr(log_alpha),
                                          _ptr(log_mu), _ptr(eta), _ptr(initial_S), _ptr(initial_M), _ptr(cu_seqlens),

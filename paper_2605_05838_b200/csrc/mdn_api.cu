@@ -329,6 +329,58 @@ size_t mdn_chunk_bwd_chunked_workspace_bytes(const mdn_params* p) {
   return chunked_bwd_layout(p, &c) == MDN_OK ? (size_t)c.total : 0;
 }
 
+size_t mdn_chunk_bwd_saved_workspace_bytes(const mdn_params* p) {
+  ChunkedBwdLayout c;
+  return chunked_bwd_layout(p, &c) == MDN_OK ? (size_t)(c.total - c.adj_states) : 0;
+}
+
+// Steps 2 and 3 on states and a workspace that a mdn_chunk_fwd_keep_states call left behind.
+static mdn_status bwd_from_states(const mdn_params* p, const ChunkedBwdLayout& c, const void* q, const void* k,
+                                  const void* v, const float* beta, const float* log_alpha, const float* log_mu,
+                                  const float* eta, const int32_t* cu_seqlens, const void* d_o, const float* d_final_S,
+                                  const float* d_final_M, void* fwd_ws, const void* fwd_states, char* adj_states,
+                                  char* stage, float* dq, float* dk, float* dv, float* dbeta, float* dlog_alpha,
+                                  float* dlog_mu, float* deta, float* d_initial_S, float* d_initial_M,
+                                  void* cuda_stream, int launches_before) {
+  mdn_status st = mdn_bwd_state_chain(p, q, k, d_o, d_final_S, d_final_M, cu_seqlens, fwd_ws, c.lf.total_bytes, adj_states,
+                                      d_initial_S, d_initial_M, stage, c.al.total, cuda_stream);
+  if (st != MDN_OK) return st;
+  t_last_launches += launches_before;
+  mdn_params pf = *p;
+  pf.segments = 1;
+  Plan fwd;
+  st = make_plan(&pf, cu_seqlens, fwd_ws, c.lf.total_bytes, cuda_stream, &fwd);
+  if (st != MDN_OK) return st;
+  cudaError_t e = launch_bwd_chunk_par(fwd, q, k, v, d_o, beta, log_alpha, log_mu, eta, fwd_states, adj_states,
+                                       stage + c.al.v_ext, dq, dk, dv, dbeta, dlog_alpha, dlog_mu, deta, &t_last_launches);
+  if (e != cudaSuccess) { t_last_cuda_error = (int)e; return MDN_ERR_CUDA; }
+  return MDN_OK;
+}
+
+mdn_status mdn_chunk_bwd_saved(const mdn_params* p, const void* q, const void* k, const void* v, const float* beta,
+                               const float* log_alpha, const float* log_mu, const float* eta,
+                               const int32_t* cu_seqlens, void* fwd_workspace, size_t fwd_workspace_bytes,
+                               const void* chunk_states, const void* d_o, const float* d_final_S,
+                               const float* d_final_M, float* dq, float* dk, float* dv, float* dbeta,
+                               float* dlog_alpha, float* dlog_mu, float* deta, float* d_initial_S,
+                               float* d_initial_M, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  t_last_launches = 0;
+  if (p && (p->num_seqs > 0) != (cu_seqlens != nullptr)) return MDN_ERR_INVALID_ARG;
+  ChunkedBwdLayout c;
+  mdn_status st = chunked_bwd_layout(p, &c);
+  if (st != MDN_OK) return st;
+  if (p->o_dtype != MDN_BF16) return MDN_ERR_UNSUPPORTED;
+  if (!q || !k || !v || !d_o || !beta || !log_alpha || !log_mu || !dq || !dk || !dv || !dbeta || !dlog_alpha || !dlog_mu)
+    return MDN_ERR_INVALID_ARG;
+  if (!fwd_workspace || fwd_workspace_bytes < c.lf.total_bytes || !aligned(fwd_workspace, 256)) return MDN_ERR_WORKSPACE;
+  if (!chunk_states || !aligned(chunk_states, 1024)) return MDN_ERR_INVALID_ARG;
+  if (!workspace || workspace_bytes < c.total - c.adj_states || !aligned(workspace, 1024)) return MDN_ERR_WORKSPACE;
+  char* w = static_cast<char*>(workspace);   // [adjoint states | stage scratch], as in the full layout from adj_states on
+  return bwd_from_states(p, c, q, k, v, beta, log_alpha, log_mu, eta, cu_seqlens, d_o, d_final_S, d_final_M,
+                         fwd_workspace, chunk_states, w, w + (c.stage - c.adj_states), dq, dk, dv, dbeta, dlog_alpha,
+                         dlog_mu, deta, d_initial_S, d_initial_M, cuda_stream, 0);
+}
+
 mdn_status mdn_chunk_bwd_chunked(const mdn_params* p, const void* q, const void* k, const void* v, const float* beta,
                                  const float* log_alpha, const float* log_mu, const float* eta,
                                  const float* initial_S, const float* initial_M, const int32_t* cu_seqlens,
@@ -357,18 +409,10 @@ mdn_status mdn_chunk_bwd_chunked(const mdn_params* p, const void* q, const void*
   st = run_forward(fwd, q, k, v, beta, log_alpha, log_mu, eta, initial_S, initial_M, w + c.stage /* o: never written */,
                    nullptr, nullptr);
   if (st != MDN_OK) return st;
-  const int launches_fwd = t_last_launches;
-  // 2. the adjoint state chain
-  st = mdn_bwd_state_chain(p, q, k, d_o, d_final_S, d_final_M, cu_seqlens, w + c.ws_fwd, c.lf.total_bytes, w + c.adj_states,
-                           d_initial_S, d_initial_M, w + c.stage, c.al.total, cuda_stream);
-  if (st != MDN_OK) return st;
-  t_last_launches += launches_fwd;
-  // 3. per (chunk, head): dq, dk, dv and the gate gradients
-  cudaError_t e = launch_bwd_chunk_par(fwd, q, k, v, d_o, beta, log_alpha, log_mu, eta, w + c.fwd_states,
-                                       w + c.adj_states, w + c.stage + c.al.v_ext, dq, dk, dv, dbeta, dlog_alpha,
-                                       dlog_mu, deta, &t_last_launches);
-  if (e != cudaSuccess) { t_last_cuda_error = (int)e; return MDN_ERR_CUDA; }
-  return MDN_OK;
+  // 2. the adjoint state chain;  3. per (chunk, head): dq, dk, dv and the gate gradients
+  return bwd_from_states(p, c, q, k, v, beta, log_alpha, log_mu, eta, cu_seqlens, d_o, d_final_S, d_final_M, w + c.ws_fwd,
+                         w + c.fwd_states, w + c.adj_states, w + c.stage, dq, dk, dv, dbeta, dlog_alpha, dlog_mu, deta,
+                         d_initial_S, d_initial_M, cuda_stream, t_last_launches);
 }
 
 // ---- the forward with layer operations

@@ -217,3 +217,24 @@ def test_chunked_backward_packed(mdn):
                     init_state_std=0.1, seed=98)
     errs = chunked_vs_oracle(mdn, w, 21)
     assert max(errs.values()) <= TOL_CHUNKED, errs
+
+
+def test_backward_from_saved_forward(mdn):
+    """mdn_chunk_bwd_saved on the workspace and the chunk states a keep-states forward left behind: the same numbers
+    as the self-contained call (which redoes that part of the forward without the output terms)."""
+    import torch
+    w = wl.Workload("saved", B=2, T=64 * 5 + 9, H=2, dk=128, dv=128, dtype="bf16", init_state_std=0.1, seed=99)
+    inp = wl.make_inputs(w)
+    t = to_torch(inp)
+    d_o = torch.randn((w.B, w.T, w.H, w.dv), generator=torch.Generator().manual_seed(4)).to(torch.bfloat16).cuda()
+    args = (t["q"], t["k"], t["v"], t["beta"], t["log_alpha"], t["log_mu"], t["eta"])
+    kw = dict(initial_S=t["initial_S"], initial_M=t["initial_M"], scale=inp["scale"])
+    _, _, _, states, ws = mdn.chunk_fwd(*args, path="tensor", keep_chunk_states=True, **kw)
+    a = mdn.chunk_bwd(*args, d_o, method="chunked", saved=(ws, states), **kw)
+    b = mdn.chunk_bwd(*args, d_o, method="chunked", **kw)
+    # dq, dk, dv and the initial states' gradients have a fixed summation order; the gate gradients sum four warps'
+    # row sums through shared-memory atomics, so their last bits can differ from run to run
+    for name in ("dq", "dk", "dv", "d_initial_S", "d_initial_M"):
+        assert torch.equal(a[name], b[name]), name
+    for name in ("dbeta", "dlog_alpha", "dlog_mu", "deta"):
+        assert torch.allclose(a[name], b[name], rtol=1e-4, atol=1e-5 * float(b[name].abs().max())), name
