@@ -437,6 +437,38 @@ def chunk_bwd(q, k, v, beta, log_alpha, log_mu, eta, d_o, *, initial_S=None, ini
     return g
 
 
+class _ChunkAttention(torch.autograd.Function):
+    """Autograd glue around mdn_chunk_fwd_keep_states / mdn_chunk_bwd_saved (no arithmetic here)."""
+
+    @staticmethod
+    def forward(ctx, q, k, v, beta, log_alpha, log_mu, eta, initial_S, initial_M, cu_seqlens, scale):
+        o, Sf, Mf, states, ws = chunk_fwd(q, k, v, beta, log_alpha, log_mu, eta, initial_S=initial_S,
+                                          initial_M=initial_M, cu_seqlens=cu_seqlens, scale=scale, path="tensor",
+                                          keep_chunk_states=True)
+        ctx.save_for_backward(q, k, v, beta, log_alpha, log_mu, eta, initial_S, initial_M, cu_seqlens, states, ws)
+        ctx.scale = scale
+        return o, Sf, Mf
+
+    @staticmethod
+    def backward(ctx, d_o, d_Sf, d_Mf):
+        q, k, v, beta, log_alpha, log_mu, eta, initial_S, initial_M, cu_seqlens, states, ws = ctx.saved_tensors
+        g = chunk_bwd(q, k, v, beta, log_alpha, log_mu, eta, d_o.contiguous().to(q.dtype), initial_S=initial_S,
+                      initial_M=initial_M, cu_seqlens=cu_seqlens,
+                      d_final_S=None if d_Sf is None else d_Sf.contiguous().float(),
+                      d_final_M=None if d_Mf is None else d_Mf.contiguous().float(), scale=ctx.scale,
+                      method="chunked", saved=(ws, states))
+        return (g["dq"].to(q.dtype), g["dk"].to(k.dtype), g["dv"].to(v.dtype), g["dbeta"], g["dlog_alpha"], g["dlog_mu"],
+                g["deta"], None if initial_S is None else g["d_initial_S"], None if initial_M is None else g["d_initial_M"],
+                None, None)
+
+
+def chunk_attention(q, k, v, beta, log_alpha, log_mu, eta, *, initial_S=None, initial_M=None, cu_seqlens=None,
+                    scale: Optional[float] = None):
+    """The forward as a differentiable torch function (tensor path: bf16 q, k, v, dk = dv = 128): returns
+    (o, final_S, final_M); gradients come from the chunk-parallel backward on the states the forward kept."""
+    return _ChunkAttention.apply(q, k, v, beta, log_alpha, log_mu, eta, initial_S, initial_M, cu_seqlens, scale)
+
+
 def decode_step(q, k, v, beta, log_alpha, log_mu, eta, S, M, *, scale: Optional[float] = None,
                 o_dtype: Optional[torch.dtype] = None, out: Optional[torch.Tensor] = None,
                 layer_ops: Optional[MdnLayerOps] = None) -> torch.Tensor:

@@ -238,3 +238,21 @@ def test_backward_from_saved_forward(mdn):
         assert torch.equal(a[name], b[name]), name
     for name in ("dbeta", "dlog_alpha", "dlog_mu", "deta"):
         assert torch.allclose(a[name], b[name], rtol=1e-4, atol=1e-5 * float(b[name].abs().max())), name
+
+
+def test_autograd_function(mdn):
+    """chunk_attention under torch.autograd: the same gradients as the explicit backward call."""
+    import torch
+    w = wl.Workload("autograd", B=2, T=64 * 3 + 11, H=2, dk=128, dv=128, dtype="bf16", seed=101)
+    inp = wl.make_inputs(w)
+    t = to_torch(inp)
+    leaves = [t[n].clone().requires_grad_(True) for n in ("q", "k", "v", "beta", "log_alpha", "log_mu", "eta")]
+    o, Sf, Mf = mdn.chunk_attention(*leaves, scale=inp["scale"])
+    d_o = torch.randn(o.shape, generator=torch.Generator().manual_seed(6)).to(torch.bfloat16).cuda()
+    dS = (0.1 * torch.randn(Sf.shape, generator=torch.Generator().manual_seed(7))).to(torch.bfloat16).float().cuda()
+    ((o.float() * d_o.float()).sum() + (Sf * dS).sum()).backward()
+    ref = mdn.chunk_bwd(t["q"], t["k"], t["v"], t["beta"], t["log_alpha"], t["log_mu"], t["eta"], d_o, d_final_S=dS,
+                        d_final_M=torch.zeros_like(dS), scale=inp["scale"], method="chunked")
+    for leaf, name in zip(leaves, ("dq", "dk", "dv", "dbeta", "dlog_alpha", "dlog_mu", "deta")):
+        x, y = leaf.grad.float(), ref[name].to(leaf.dtype).float()
+        assert torch.allclose(x, y, rtol=1e-3, atol=1e-4 * float(y.abs().max())), name
