@@ -516,6 +516,32 @@ def run_backward(args, w):
     e1.record()
     torch.cuda.synchronize()
     ms = e0.elapsed_time(e1) / args.steps
+    train = None
+    if method == "chunked":
+        # the save-for-backward split: a forward that keeps its chunk states, then the backward on what it kept
+        fkw = dict(initial_S=S0, initial_M=M0, cu_seqlens=cu, scale=inp["scale"], path="tensor")
+        o_buf = torch.empty_like(v)
+
+        def timed(fn, n):
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            t0.record()
+            for _ in range(n):
+                fn()
+            t1.record()
+            torch.cuda.synchronize()
+            return t0.elapsed_time(t1) / n
+
+        _, _, _, states, fws = mdn.chunk_fwd(q, k, v, *gates, keep_chunk_states=True, out=o_buf, **fkw)
+        f_ms = timed(lambda: mdn.chunk_fwd(q, k, v, *gates, keep_chunk_states=True, out=o_buf, workspace=fws, **fkw), args.steps)
+        ws2 = torch.empty(int(mdn.lib().mdn_chunk_bwd_saved_workspace_bytes(ctypes.byref(
+            mdn.make_params(q, v, num_seqs=0 if cu is None else cu.numel() - 1, path="tensor")))), dtype=torch.uint8, device="cuda")
+        b_ms = timed(lambda: mdn.chunk_bwd(q, k, v, *gates, d_o, initial_S=S0, initial_M=M0, cu_seqlens=cu, scale=inp["scale"],
+                                           workspace=ws2, method="chunked", saved=(fws, states)), args.steps)
+        train = {"forward_keep_states_ms": f_ms, "backward_on_saved_states_ms": b_ms,
+                 "tokens_per_s": w.B * w.T / ((f_ms + b_ms) * 1e-3)}
     peaks = load_peaks()
     tokens, es = w.B * w.T, (2 if w.dtype == "bf16" else 4)
     # reads q, k, v, dO and four gates; writes dq, dk, dv (fp32) and four gate gradients
@@ -528,7 +554,7 @@ def run_backward(args, w):
             "chunk-parallel: state-only forward keeping the chunk states, adjoint state chain, per-chunk kernel "
             "(bf16 tensor-core products, fp32 accumulation)" if method == "chunked" else
             "token-level adjoint recurrence, per-chunk checkpoints and recomputation (fp32)")},
-        "gpu_launches": launches * args.steps, "workspace_bytes": need,
+        "gpu_launches": launches * args.steps, "workspace_bytes": need, "training_step": train,
         "roofline": {"bound": "hbm", "kernel": "whole backward" if method == "chunked" else "bwd_stepwise", "achieved": abytes / (ms * 1e-3) / 1e9,
                      "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": abytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
                      "traffic": None, "peak_source": peaks["source"], "algorithmic_bytes": abytes}}))
