@@ -268,7 +268,9 @@ mdn_status mdn_chunk_fwd_fused(const mdn_params* p, const mdn_layer_ops* ops /* 
  * (value index x key index, 128 x 128) and then that of M^T, each as two blocks (key index 0..63, 64..127) of 128
  * rows x 128 bytes whose 16-byte pieces are XOR-swizzled with (row mod 8) - the image a K-major tcgen05 operand
  * has in shared memory, so a later kernel can fetch a block with one untiled bulk copy.  These are the copies the
- * forward's own tensor-core products read (the fp32 masters stay on chip).
+ * forward's own tensor-core products read (the fp32 masters stay on chip).  Behind the images of all slots lies a
+ * second part: V~ = T (V - abar.(K S) + p.(K M)) of every chunk as float32 [chunk slot][64][H][dv] (rows past the end
+ * of a short chunk are not written), which the chunk-parallel backward reads instead of rebuilding it.
  * Tensor path only (bf16 input, dk = dv = 128): MDN_ERR_UNSUPPORTED otherwise.  The serial chain is used
  * (p->segments is ignored).  Workspace as for mdn_chunk_fwd.
  */
@@ -301,7 +303,8 @@ mdn_status mdn_chunk_fwd_keep_states(const mdn_params* p,
  *     the workspace's slot order, entries of sequence s starting at twice its first chunk slot) and
  *     head it receives 2 x nchunks entries of 65536 bytes in the layout of mdn_chunk_fwd_keep_states with dM^T in
  *     the first half and dS^T in the second: entry 2 (nchunks - 1 - c) is the adjoint pair at the END of chunk c,
- *     entry 2 (nchunks - 1 - c) + 1 the pair after chunk c's K terms and before its Q terms;
+ *     entry 2 (nchunks - 1 - c) + 1 the pair after chunk c's K terms and before its Q terms; behind all entries, as
+ *     float32 [entry / 2][64][H][dv], dR = T^T dV~ (= dL/dv) of the chunk whose real step is entry 2 (nchunks-1-c);
  *   d_initial_S, d_initial_M: dL/d(initial states), [B,H,dk,dv] float32, or NULL;
  *   workspace: mdn_bwd_state_chain_workspace_bytes(p) bytes, 1024-byte aligned, scratch.
  * The gradients of q, k, v and the gates follow from these adjoint states and the kept forward states chunk by chunk,
@@ -325,8 +328,9 @@ mdn_status mdn_bwd_state_chain(const mdn_params* p,
  *   1. the forward's state recurrence again, keeping (S, M) at the start of every chunk (mdn_chunk_fwd_keep_states
  *      without the output terms),
  *   2. the adjoint state recurrence (mdn_bwd_state_chain),
- *   3. per (chunk, head), in parallel: dV = dR, dQ, dK, the adjoints of the coefficient vectors and of the two
- *      masks, and from those the gate gradients by the recurrences of Eq. 10 in reverse.
+ *   3. per (chunk, head), in parallel: dQ, dK, the adjoints of the coefficient vectors and of the two masks, and
+ *      from those the gate gradients by the recurrences of Eq. 10 in reverse (V~ and dR = dV are left behind by the
+ *      chain runs of steps 1 and 2).
  * Arguments as mdn_chunk_bwd (fixed-length or packed input).  Tensor path only: bf16 q, k, v, bf16 d_o,
  * dk = dv = 128; MDN_ERR_UNSUPPORTED otherwise.  Operands are bf16 / tf32 with fp32 accumulation, so the gradients
  * carry the forward's bf16-level error (see the tests), not mdn_chunk_bwd's fp32 exactness; d_final_S, d_final_M

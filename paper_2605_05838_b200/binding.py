@@ -325,10 +325,32 @@ def chunk_fwd(q, k, v, beta, log_alpha, log_mu, eta=None, *, initial_S=None, ini
     return o, Sf, Mf
 
 
-def unpack_chunk_states(states: torch.Tensor, H: int):
-    """The buffer of mdn_chunk_fwd_keep_states as float32 tensors (S, M) of shape [slots, H, dk, dv] (dk = dv = 128):
-    undoes the transposition and the 128-byte swizzle of the shared-memory image."""
-    raw = states.view(torch.bfloat16).view(-1, H, 2, 2, 128, 8, 8)          # slot, head, S|M, key half, row, piece, elem
+_IMAGE_BYTES, _VT_BYTES = 65536, 64 * 128 * 4
+
+
+def _states_parts(states: torch.Tensor, H: int, adjoint: bool):
+    """(state images, V~ part, slots) of a kept-states buffer: per (slot, head) a 64 KB state image, and behind all
+    images one fp32 [64, H, 128] block per slot (forward) or per pair of slots (adjoint chain)."""
+    nbytes = states.numel()
+    if not adjoint:
+        slots = nbytes // (H * (_IMAGE_BYTES + _VT_BYTES))
+        vt_slots = slots
+    else:
+        pair = H * (2 * _IMAGE_BYTES + _VT_BYTES)
+        slots = 2 * (nbytes // pair) + (1 if nbytes % pair else 0)
+        vt_slots = (slots + 1) // 2
+    if slots * H * _IMAGE_BYTES + vt_slots * H * _VT_BYTES != nbytes:
+        raise ValueError("not a kept-states buffer for H = %d" % H)
+    cut = slots * H * _IMAGE_BYTES
+    return states[:cut], states[cut:], slots
+
+
+def unpack_chunk_states(states: torch.Tensor, H: int, adjoint: bool = False):
+    """The state images of a mdn_chunk_fwd_keep_states (or, adjoint=True, mdn_bwd_state_chain) buffer as float32
+    tensors (S, M) of shape [slots, H, dk, dv] (dk = dv = 128): undoes the transposition and the 128-byte swizzle of
+    the shared-memory image."""
+    images, _, _ = _states_parts(states, H, adjoint)
+    raw = images.view(torch.bfloat16).view(-1, H, 2, 2, 128, 8, 8)          # slot, head, S|M, key half, row, piece, elem
     rows = torch.arange(128, device=states.device)
     piece = torch.arange(8, device=states.device)
     src = (piece[None, :] ^ (rows[:, None] & 7))                            # where logical piece c of row r lies
@@ -337,6 +359,13 @@ def unpack_chunk_states(states: torch.Tensor, H: int):
     full = torch.cat([logical[:, :, :, 0], logical[:, :, :, 1]], dim=-1)    # [slot, H, 2, value, key]
     full = full.transpose(-1, -2).float()                                   # [slot, H, 2, key, value]
     return full[:, :, 0].contiguous(), full[:, :, 1].contiguous()
+
+
+def unpack_chunk_vt(states: torch.Tensor, H: int, adjoint: bool = False):
+    """The second part of a kept-states buffer: V~ of every chunk slot as float32 [slots, 64, H, 128] (rows past a
+    short chunk's end are unwritten); with adjoint=True, dR = T^T dV~ at half the extended slot index."""
+    _, vt, _ = _states_parts(states, H, adjoint)
+    return vt.view(torch.float32).view(-1, 64, H, 128)
 
 
 def bwd_state_chain(q, k, d_o, fwd_workspace, *, v_dim: int, d_final_S=None, d_final_M=None, cu_seqlens=None,

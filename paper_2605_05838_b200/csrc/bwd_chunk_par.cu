@@ -12,10 +12,11 @@
 // sum_j dR_rj X_rj = sum_d K_rd (dR S^T)_rd reuses a product that dK needs anyway), the adjoints of the two masks
 // d Geta = scale tril(dO V~^T) o (Q K^T), d G^- = dA o (K K^T), and from those the gate gradients by running the
 // coefficient recurrences of Eq. 10 in reverse.
+// V~ and dR are not recomputed here: the two chain runs (the forward that keeps its states, the adjoint chain) have
+// both in their epilogues and leave them in global memory as fp32, so X, Y, R, T R, K dS', K dM' and T^T dV~ cost nothing.
 // Every product is a warp-level bf16 tensor-core MMA (m16n8k16, fp32 accumulate) fed by ldmatrix from shared memory:
-// q, k, dO, T and the states are bf16 as they stand; every intermediate that comes out of an accumulator (R, dV~, V~,
-// dR, DW, DA) is kept as a bf16 hi + lo pair (16 mantissa bits through two MMAs), W as the hi + lo pair the forward
-// wrote.  One 256-thread CTA per (chunk, head).
+// q, k, dO and the states are bf16 as they stand; V~, dR and every intermediate that comes out of an accumulator (DW,
+// DA) is kept as a bf16 hi + lo pair (16 mantissa bits through two MMAs).  One 256-thread CTA per (chunk, head).
 #include "mdn_common.cuh"
 #include "tc_utils.cuh"
 #include "warp_mma.cuh"
@@ -40,8 +41,7 @@ constexpr uint32_t kOffQ = kOffK + kTile;
 constexpr uint32_t kOffDO = kOffQ + kTile;
 constexpr uint32_t kOffVt = kOffDO + kTile;           // V~ hi, lo; later DW hi, lo
 constexpr uint32_t kOffDR = kOffVt + 2 * kTile;       // dR hi, lo; later DA hi, lo
-constexpr uint32_t kOffT = kOffDR + 2 * kTile;        // T, bf16 [64][L6]
-constexpr uint32_t kOffTmp = kOffT + kMat6;           // R / dV~ hi, lo; W hi, lo; later gamma, m (fp32 [64][LG] each)
+constexpr uint32_t kOffTmp = kOffDR + 2 * kTile;      // dS', then M again; later gamma, m (fp32 [64][LG] each)
 constexpr uint32_t kOffVec = kOffTmp + 2 * kTile;     // vectors, 24 x [64] floats
 constexpr uint32_t kSmem = kOffVec + 24 * C * 4;
 constexpr uint32_t kR0 = kOffSt, kR1 = kOffVt, kR2 = kOffDR, kR3 = kOffTmp;   // the four reusable areas (see the kernel)
@@ -54,10 +54,11 @@ enum Vec : int { vAbar = 0, vB, vP, vGS, vGM, vMubar, vAlpha, vBeta, vMu, vEta, 
 
 struct ParArgs {
   ChunkGeom g;
-  const bf16* q; const bf16* k; const bf16* v; const bf16* d_o;
+  const bf16* q; const bf16* k; const bf16* d_o;
   const float* beta; const float* log_alpha; const float* log_mu; const float* eta;
-  const float* coef; const bf16* T; const bf16* W; size_t w_lo_offset;
-  const uint8_t* fwd_states; const uint8_t* adj_states; const bf16* v_ext;
+  const float* coef;
+  const uint8_t* fwd_states; const uint8_t* adj_states;   // state images per chunk slot
+  const float* fwd_vt; const float* adj_dr;               // V~ and dR per chunk slot, fp32 [slot][64][H][dv]
   float scale;
   float* dq; float* dk; float* dv; float* dbeta; float* dlog_alpha; float* dlog_mu; float* deta;
 };
@@ -68,7 +69,6 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
   bf16* sK = reinterpret_cast<bf16*>(smem + kOffK);
   bf16* sQ = reinterpret_cast<bf16*>(smem + kOffQ);
   bf16* sDO = reinterpret_cast<bf16*>(smem + kOffDO);
-  bf16* sT = reinterpret_cast<bf16*>(smem + kOffT);
   float* sGam = reinterpret_cast<float*>(smem + kR2);         // gamma, m
   float* sMm = sGam + C * LG;
   bf16* sDWH = reinterpret_cast<bf16*>(smem + kR1);           // DW, DA (hi, lo)
@@ -88,7 +88,6 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
   seq_chunks(a.g, si.seq, &slot0, &nch);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
   const int m0 = 32 * (warp & 1), n0 = 32 * (warp >> 1), n064 = 16 * (warp >> 1);   // the warp's block of a 64x128 / 64x64 result
-  const size_t mat = ((size_t)slot * H + h) * C * C;
   const uint8_t* imgS = a.fwd_states + ((size_t)slot * H + h) * 65536;
   const uint8_t* imgM = imgS + 32768;
   const int e_real = 2 * slot0 + 2 * (nch - 1 - si.local);
@@ -100,7 +99,6 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
   const Opnd oK{sb + kOffK, LT * 2, false}, oK_t{sb + kOffK, LT * 2, true};
   const Opnd oQ{sb + kOffQ, LT * 2, false}, oQ_t{sb + kOffQ, LT * 2, true};
   const Opnd oDO{sb + kOffDO, LT * 2, false}, oDO_t{sb + kOffDO, LT * 2, true};
-  const Opnd oT{sb + kOffT, L6 * 2, false}, oT_t{sb + kOffT, L6 * 2, true};
   // a state in an area: B(k = key d, n = value j) = S[d][j], stored [j][d]; or B(k = value j, n = key d)
   auto st_dk = [&](uint32_t base) { return Opnd{sb + base, LT * 2, false}; };
   auto st_dv = [&](uint32_t base) { return Opnd{sb + base, LT * 2, true}; };
@@ -124,10 +122,31 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
       cp16(sb + base + (r * LT + c8) * 2, src + tok(r < n ? r : 0) * kD + c8, r < n);
     }
   };
-  auto load_mat64 = [&](uint32_t base, const bf16* src) {   // a [64][64] bf16 matrix -> [64][L6]
-    for (int idx = tid; idx < C * 8; idx += kThreads) {
-      const int r = idx >> 3, c8 = (idx & 7) * 8;
-      cp16(sb + base + (r * L6 + c8) * 2, src + r * C + c8, true);
+  // a chunk's V~ or dR (fp32 rows of one head, H * dv floats apart) -> [64][128] fp32 at the start of an area
+  auto load_f32 = [&](uint32_t base, const float* src) {
+    for (int idx = tid; idx < C * 32; idx += kThreads) {
+      const int r = idx >> 5, c4 = (idx & 31) * 4;
+      cp16(sb + base + idx * 16, src + (size_t)(r < n ? r : 0) * H * kD + c4, r < n);
+    }
+  };
+  // ... and from there, in place, to the bf16 hi + lo tiles the products read (every thread holds its 32 values across
+  // the barrier); `out`, if given, receives the fp32 values of the live rows (dv = dR)
+  auto split_in_place = [&](uint32_t base, float* out) {
+    float4 x[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) x[i] = *reinterpret_cast<const float4*>(smem + base + (tid + kThreads * i) * 16);
+    __syncthreads();
+    bf16* hi = reinterpret_cast<bf16*>(smem + base);
+    bf16* lo = hi + C * LT;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int idx = tid + kThreads * i, r = idx >> 5, c4 = (idx & 31) * 4;
+      uint2 ph, pl;
+      split_pack_bf16(x[i].x, x[i].y, ph.x, pl.x);
+      split_pack_bf16(x[i].z, x[i].w, ph.y, pl.y);
+      *reinterpret_cast<uint2*>(hi + r * LT + c4) = ph;
+      *reinterpret_cast<uint2*>(lo + r * LT + c4) = pl;
+      if (out != nullptr && r < n) *reinterpret_cast<float4*>(out + tok(r) * kD + c4) = x[i];
     }
   };
   // state image (value index j x key index d, two swizzled blocks) -> [j][d] in an area, by cp.async
@@ -156,17 +175,6 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
     for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
     return s;   // per warp; lane 0 adds it where it belongs
   };
-  // a warp's 32 x 32 block of a 64 x 128 result -> bf16 hi + lo tiles (rows past the chunk's end are zero)
-  auto put_split = [&](float (&acc)[2][4][4], uint32_t base) {
-    bf16* hi = reinterpret_cast<bf16*>(smem + base);
-    bf16* lo = hi + C * LT;
-    for_pair<2, 4>(m0, n0, g, t, [&](int mt, int nt, int hf, int r, int c) {
-      uint32_t ph = 0u, pl = 0u;
-      if (r < n) split_pack_bf16(acc[mt][nt][2 * hf], acc[mt][nt][2 * hf + 1], ph, pl);
-      *reinterpret_cast<uint32_t*>(hi + r * LT + c) = ph;
-      *reinterpret_cast<uint32_t*>(lo + r * LT + c) = pl;
-    });
-  };
   // row sums of G o X over the warp's 32 columns, added to a vector (X: a bf16 tile, k or q)
   auto add_rowsum = [&](float (&G)[2][4][4], const bf16* X, float* dst, float sign) {
 #pragma unroll
@@ -187,29 +195,29 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
       }
   };
 
-  // ---- what this CTA fetches later (V, W^T dO), towards L2 now (one CTA per SM: nothing else hides the latency)
-  if (tid < C) {
-    asm volatile("prefetch.global.L2 [%0];" ::"l"(a.v_ext + ((size_t)(e_real * C + tid) * H + h) * kD));
-    asm volatile("prefetch.global.L2 [%0];" ::"l"(a.v_ext + ((size_t)(e_real * C + tid) * H + h) * kD + 64));
-  }
-  if (tid < n) {
-    asm volatile("prefetch.global.L2 [%0];" ::"l"(a.v + tok(tid) * kD));
-    asm volatile("prefetch.global.L2 [%0];" ::"l"(a.v + tok(tid) * kD + 64));
+  const float* vt_rows = a.fwd_vt + (((size_t)slot * C) * H + h) * kD;
+  const float* dr_rows = a.adj_dr + (((size_t)(e_real >> 1) * C) * H + h) * kD;
+  // ---- what this CTA fetches later (V~, dR), towards L2 now (one CTA per SM: nothing else hides the latency)
+  {
+    const int r = tid >> 2, part = (tid & 3) * 32;
+    if (r < n) {
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(vt_rows + (size_t)r * H * kD + part));
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(dr_rows + (size_t)r * H * kD + part));
+    }
   }
   // Four areas of 34816 bytes (a state, or the hi + lo pair of a 64 x 128 tile) are reused through the phases:
   //   R0: S                                               | later d Geta, d G^-
-  //   R1: M    | R (hi, lo) | V~ (hi, lo)                 | later DW (hi, lo), then two contribution matrices
-  //   R2: dM'               | dV~ (hi, lo) | M again      | gamma, m
-  //   R3: dS'                              | dR (hi, lo)  | DA (hi, lo), then a contribution matrix
+  //   R1: M    | V~ (fp32, then hi, lo)                   | later DW (hi, lo), then two contribution matrices
+  //   R2: dS'  | M again                                  | gamma, m
+  //   R3: dM'  | dR (fp32, then hi, lo)                   | DA (hi, lo), then a contribution matrix
   // All four states arrive at the start by cp.async (no registers in between); M is fetched a second time later.
   load_state(imgS, kR0);
   load_state(imgM, kR1);
-  load_state(imgdM, kR2);
-  load_state(imgdS, kR3);
+  load_state(imgdS, kR2);
+  load_state(imgdM, kR3);
   load_tile(kOffK, a.k);
   load_tile(kOffQ, a.q);
   load_tile(kOffDO, a.d_o);
-  load_mat64(kOffT, a.T + mat);
   cp_async_commit();
   // ---- vectors: the chain's coefficient vectors, the gates, zeroed adjoints
   const float* cf = a.coef + ((size_t)slot * H + h) * MDN_NUM_COEF * C;
@@ -228,7 +236,7 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
   __syncthreads();
   if (tid < C) V(vBprev)[tid] = tid > 0 ? V(vB)[tid - 1] : 0.f;
   {   // the end-of-chunk adjoints: d mubar_C = <dM', M>, d abar_C = <dS', S>, d b_C = -<dS', M>
-    const float s0 = dot_areas(kR2, kR1), s1 = dot_areas(kR3, kR0), s2 = dot_areas(kR3, kR1);
+    const float s0 = dot_areas(kR3, kR1), s1 = dot_areas(kR2, kR0), s2 = dot_areas(kR2, kR1);
     if (lane == 0) {
       atomicAdd(V(vdMubar) + n - 1, s0);
       atomicAdd(V(vdAbar) + n - 1, s1);
@@ -239,21 +247,9 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
   float dQ[2][4][4], dK[2][4][4];
   zero(dQ); zero(dK);
 
-  // ---- phase 1, everything that needs only the four states and k, dO:
-  //   X = K S, Y = K M -> R = V - abar.X + p.Y;  dO S^T, dO M^T (dQ, d abar, d b);
-  //   K dM', K dS' -> dV~ = W^T dO + g_S.(K dS') - g_M.(K dM')
-  float Rf[2][4][4], dVf[2][4][4];
+  // ---- phase 1: dO S^T, dO M^T (dQ, d abar, d b)
   {
     float Y[2][4][4];
-    zero(Rf); zero(Y);
-    warp_mma(Rf, oK, st_dk(kR0), kD, m0, n0, lane);
-    warp_mma(Y, oK, st_dk(kR1), kD, m0, n0, lane);
-    for_pair<2, 4>(m0, n0, g, t, [&](int mt, int nt, int hf, int r, int c) {
-      const uint32_t v2 = r < n ? *reinterpret_cast<const uint32_t*>(a.v + tok(r) * kD + c) : 0u;
-      const float ab = V(vAbar)[r], pp = V(vP)[r];
-      Rf[mt][nt][2 * hf] = __uint_as_float(v2 << 16) - ab * Rf[mt][nt][2 * hf] + pp * Y[mt][nt][2 * hf];
-      Rf[mt][nt][2 * hf + 1] = __uint_as_float(v2 & 0xffff0000u) - ab * Rf[mt][nt][2 * hf + 1] + pp * Y[mt][nt][2 * hf + 1];
-    });
     zero(Y);
     warp_mma(Y, oDO, st_dv(kR0), kD, m0, n0, lane);                   // dO S^T
     for_frag<2, 4>(m0, n0, g, t, [&](int mt, int nt, int e, int r, int c) { dQ[mt][nt][e] += scale * V(vAbar)[r] * Y[mt][nt][e]; });
@@ -262,54 +258,43 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
     warp_mma(Y, oDO, st_dv(kR1), kD, m0, n0, lane);                   // dO M^T
     for_frag<2, 4>(m0, n0, g, t, [&](int mt, int nt, int e, int r, int c) { dQ[mt][nt][e] -= scale * V(vB)[r] * Y[mt][nt][e]; });
     add_rowsum(Y, sQ, V(vdB), -scale);
-    zero(dVf); zero(Y);
-    warp_mma(dVf, oK, st_dk(kR3), kD, m0, n0, lane);                  // K dS'
-    warp_mma(Y, oK, st_dk(kR2), kD, m0, n0, lane);                    // K dM'
-    for_pair<2, 4>(m0, n0, g, t, [&](int mt, int nt, int hf, int r, int c) {
-      // W^T dO as the adjoint chain's problem has it (bf16)
-      const uint32_t v2 = r < n ? *reinterpret_cast<const uint32_t*>(a.v_ext + ((size_t)(e_real * C + r) * H + h) * kD + c) : 0u;
-      const float gs = V(vGS)[r], gm = V(vGM)[r];
-      dVf[mt][nt][2 * hf] = __uint_as_float(v2 << 16) + gs * dVf[mt][nt][2 * hf] - gm * Y[mt][nt][2 * hf];
-      dVf[mt][nt][2 * hf + 1] = __uint_as_float(v2 & 0xffff0000u) + gs * dVf[mt][nt][2 * hf + 1] - gm * Y[mt][nt][2 * hf + 1];
-    });
   }
-  __syncthreads();   // M has been read: R takes its place
-  put_split(Rf, kR1);
+  __syncthreads();   // M has been read: V~ takes its place
+  load_f32(kR1, vt_rows);
+  cp_async_commit();
+  float QK[2][2][4], KK[2][2][4];   // Q K^T, K K^T while V~ arrives
+  zero(QK); zero(KK);
+  warp_mma(QK, oQ, oK, kD, m0, n064, lane);
+  warp_mma(KK, oK, oK, kD, m0, n064, lane);
+  cp_async_wait();
   __syncthreads();
-  zero(Rf);
-  warp_mma(Rf, oT, tile_kn(kR1), C, m0, n0, lane);                    // V~ = T R
-  warp_mma(Rf, oT, tile_kn(kR1 + kTile), C, m0, n0, lane);
-  __syncthreads();   // R has been read: V~ takes its place
-  put_split(Rf, kR1);
+  split_in_place(kR1, nullptr);
   __syncthreads();
 
-  // ---- phase 2: the g_M and g_S terms of dK from V~ dM'^T, V~ dS'^T; then dR = T^T dV~
+  // ---- phase 2: the g_M and g_S terms of dK from V~ dM'^T, V~ dS'^T; dR arrives under the second
   {
     float G[2][4][4];
     zero(G);
-    warp_mma(G, tile_mk(kR1), st_dv(kR2), kD, m0, n0, lane);          // V~ dM'^T
-    warp_mma(G, tile_mk(kR1 + kTile), st_dv(kR2), kD, m0, n0, lane);
+    warp_mma(G, tile_mk(kR1), st_dv(kR3), kD, m0, n0, lane);          // V~ dM'^T
+    warp_mma(G, tile_mk(kR1 + kTile), st_dv(kR3), kD, m0, n0, lane);
     for_frag<2, 4>(m0, n0, g, t, [&](int mt, int nt, int e, int r, int c) { dK[mt][nt][e] -= V(vGM)[r] * G[mt][nt][e]; });
     add_rowsum(G, sK, V(vdGM), -1.f);
+    __syncthreads();   // dM' has been read: dR takes its place
+    load_f32(kR3, dr_rows);
+    cp_async_commit();
     zero(G);
-    warp_mma(G, tile_mk(kR1), st_dv(kR3), kD, m0, n0, lane);          // V~ dS'^T
-    warp_mma(G, tile_mk(kR1 + kTile), st_dv(kR3), kD, m0, n0, lane);
+    warp_mma(G, tile_mk(kR1), st_dv(kR2), kD, m0, n0, lane);          // V~ dS'^T
+    warp_mma(G, tile_mk(kR1 + kTile), st_dv(kR2), kD, m0, n0, lane);
     for_frag<2, 4>(m0, n0, g, t, [&](int mt, int nt, int e, int r, int c) { dK[mt][nt][e] += V(vGS)[r] * G[mt][nt][e]; });
     add_rowsum(G, sK, V(vdGS), 1.f);
   }
-  __syncthreads();   // dM', dS' have been read: dV~ takes dM's place
-  put_split(dVf, kR2);
-  __syncthreads();
-  zero(dVf);
-  warp_mma(dVf, oT_t, tile_kn(kR2), C, m0, n0, lane);                 // dR = T^T dV~
-  warp_mma(dVf, oT_t, tile_kn(kR2 + kTile), C, m0, n0, lane);
-  put_split(dVf, kR3);
-  for_pair<2, 4>(m0, n0, g, t, [&](int mt, int nt, int hf, int r, int c) {
-    if (r < n) *reinterpret_cast<float2*>(a.dv + tok(r) * kD + c) = make_float2(dVf[mt][nt][2 * hf], dVf[mt][nt][2 * hf + 1]);
-  });
-  __syncthreads();   // dR complete; dV~ has been read
+  __syncthreads();   // dS' has been read: M takes its place
   load_state(imgM, kR2);
   cp_async_commit();
+  asm volatile("cp.async.wait_group 1;" ::: "memory");   // dR is in (M may still be on its way)
+  __syncthreads();
+  split_in_place(kR3, a.dv);
+  __syncthreads();
 
   // ---- phase 3: dR S^T (dK, d abar) while M arrives again, then dR M^T (dK, d p)
   {
@@ -341,15 +326,13 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
     }
   }
   // ---- the four 64 x 64 products
-  float P1[2][2][4], P2[2][2][4], QK[2][2][4], KK[2][2][4];
-  zero(P1); zero(P2); zero(QK); zero(KK);
+  float P1[2][2][4], P2[2][2][4];
+  zero(P1); zero(P2);
   warp_mma(P1, oDO, tile_mk(kR1), kD, m0, n064, lane);                        // dO V~^T  (V~ as B: [n][k])
   warp_mma(P1, oDO, tile_mk(kR1 + kTile), kD, m0, n064, lane);
   warp_mma(P2, tile_mk(kR3), tile_mk(kR1), kD, m0, n064, lane);               // dR V~^T
   warp_mma(P2, tile_mk(kR3), tile_mk(kR1 + kTile), kD, m0, n064, lane);
   warp_mma(P2, tile_mk(kR3 + kTile), tile_mk(kR1), kD, m0, n064, lane);
-  warp_mma(QK, oQ, oK, kD, m0, n064, lane);
-  warp_mma(KK, oK, oK, kD, m0, n064, lane);
   __syncthreads();   // V~, dR and S are no longer read; gamma, m complete
   for_pair<2, 2>(m0, n064, g, t, [&](int mt, int nt, int hf, int r, int i0) {
     float dw[2], da[2];
@@ -497,22 +480,19 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
 
 }  // namespace
 
-cudaError_t launch_bwd_chunk_par(const Plan& fwd, const void* q, const void* k, const void* v, const void* d_o,
-                                 const float* beta, const float* log_alpha, const float* log_mu, const float* eta,
-                                 const void* fwd_states, const void* adj_states, const void* v_ext, float* dq, float* dk,
+cudaError_t launch_bwd_chunk_par(const Plan& fwd, const void* q, const void* k, const void* d_o, const float* beta,
+                                 const float* log_alpha, const float* log_mu, const float* eta, const void* fwd_states,
+                                 const float* fwd_vt, const void* adj_states, const float* adj_dr, float* dq, float* dk,
                                  float* dv, float* dbeta, float* dlog_alpha, float* dlog_mu, float* deta, int* launches) {
   ParArgs a;
   a.g = fwd.geom;
   a.q = static_cast<const __nv_bfloat16*>(q); a.k = static_cast<const __nv_bfloat16*>(k);
-  a.v = static_cast<const __nv_bfloat16*>(v); a.d_o = static_cast<const __nv_bfloat16*>(d_o);
+  a.d_o = static_cast<const __nv_bfloat16*>(d_o);
   a.beta = beta; a.log_alpha = log_alpha; a.log_mu = log_mu; a.eta = eta;
   a.coef = reinterpret_cast<const float*>(fwd.ws + fwd.lay.off_coef);
-  a.T = reinterpret_cast<const __nv_bfloat16*>(fwd.ws + fwd.lay.off_T);
-  a.W = reinterpret_cast<const __nv_bfloat16*>(fwd.ws + fwd.lay.off_W);
-  a.w_lo_offset = (size_t)fwd.geom.num_slots * fwd.p.H * C * C;
   a.fwd_states = static_cast<const uint8_t*>(fwd_states);
   a.adj_states = static_cast<const uint8_t*>(adj_states);
-  a.v_ext = static_cast<const bf16*>(v_ext);
+  a.fwd_vt = fwd_vt; a.adj_dr = adj_dr;
   a.scale = fwd.p.scale;
   a.dq = dq; a.dk = dk; a.dv = dv; a.dbeta = dbeta; a.dlog_alpha = dlog_alpha; a.dlog_mu = dlog_mu; a.deta = deta;
   cudaError_t e = cudaFuncSetAttribute(bwd_chunk_par_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmem);

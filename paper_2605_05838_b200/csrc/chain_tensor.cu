@@ -119,6 +119,8 @@ struct ChainArgs {
   int state_only;             // no output terms (no Q, W loads, no output MMAs): states (and the dump) only
   int end_scalars_in_rk;      // (abar_C, b_C, mubar_C) of a chunk are entries 0..2 of coefficient vector 6, not the
                               // last entries of vectors 0, 1, 5 (the adjoint chain decouples them)
+  float* vt_dump;             // NULL, or [chunk slot][64][H][dv] fp32: V~ of every chunk as EPI-2 reads it
+  int vt_dump_even_only;      // only the even chunk slots, written at slot / 2 (the adjoint chain: its real steps)
   uint32_t drop_lo;           // debug: bit 0 R, 1 V~_S/V~_M, 2 V~ (output), 3 W: leave that operand's lo part out
   long long* timeline;        // debug: CTA 0 writes clock64() at [chunk*32 + event] (NULL = off)
 };
@@ -853,6 +855,23 @@ __global__ void __launch_bounds__(Roles<token_groups(kLayer)>::kThreads, 1) chai
           MDN_WARP_ARRIVE(b_v2);
         }
         MDN_MARK(c, kEvV2Arrive);
+        if constexpr (kTrain) {   // off the chain's critical path: MMA-3 is running
+          int slot_c = sq.slot0 + c;
+          if (a.vt_dump != nullptr && !(a.vt_dump_even_only && (slot_c & 1))) {
+            if (a.vt_dump_even_only) slot_c >>= 1;
+            const int live = min(C, sq.len - c * C) - r0;   // this thread's tokens inside the chunk
+            float* dst = a.vt_dump + (((size_t)slot_c * C + r0) * H + h) * kD + d;
+            const size_t stride = (size_t)H * kD;
+            if (live >= kTok) {   // the usual case: no per-store predicate
+#pragma unroll
+              for (int j = 0; j < kTok; ++j, dst += stride) *dst = __uint_as_float(vt[j]);
+            } else {
+#pragma unroll
+              for (int j = 0; j < kTok; ++j, dst += stride)
+                if (j < live) *dst = __uint_as_float(vt[j]);
+            }
+          }
+        }
       }
     }
   }
@@ -908,6 +927,7 @@ cudaError_t launch_chain_tensor(const Plan& pl, const void* q, const void* k, co
   const char* tl = getenv("MDN_DEBUG_TIMELINE");   // device address of an int64 buffer, [chunks][32]
   a.timeline = tl ? reinterpret_cast<long long*>(strtoull(tl, nullptr, 0)) : nullptr;
   a.dump = pl.chain_dump; a.state_only = pl.chain_state_only; a.end_scalars_in_rk = pl.chain_end_scalars_in_rk;
+  a.vt_dump = pl.chain_vt_dump; a.vt_dump_even_only = pl.chain_vt_dump_even_only;
   a.seg_G = 0; a.seg_phase = 0;
   a.seg_E = a.seg_Psi = a.seg_PhiS = a.seg_PhiM = nullptr;
   const unsigned chains = (unsigned)pl.geom.num_seqs * p.H;
@@ -922,7 +942,7 @@ cudaError_t launch_chain_tensor(const Plan& pl, const void* q, const void* k, co
     return e;
   };
   auto launch = [&](unsigned grid) -> cudaError_t {
-    const bool train = a.dump != nullptr || a.state_only || a.end_scalars_in_rk;
+    const bool train = a.dump != nullptr || a.state_only || a.end_scalars_in_rk || a.vt_dump != nullptr;
     if (train) {   // plain forward with the training options (no layer operations there)
       if (layer) return cudaErrorInvalidValue;
       return p.o_dtype == MDN_BF16 ? launch_as(chain_tensor_kernel<__nv_bfloat16, false, true>, grid)

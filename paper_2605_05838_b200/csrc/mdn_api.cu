@@ -194,11 +194,15 @@ mdn_status mdn_chunk_fwd(const mdn_params* p, const void* q, const void* k, cons
 }
 
 // ---- the forward that keeps the chunk-start states (tensor path, serial chain)
+// Per (chunk slot, head): the bf16 state images S_b^T | M_b^T (2 x 32 KB), and behind all of them V~ of every chunk
+// slot as fp32 [slot][64][H][dv] (32 KB per slot and head).  The adjoint chain's buffer has the same two parts, with
+// dR = T^T dV~ (the V~ of its real steps) at half the extended slot index.
+constexpr uint64_t kStateImageBytes = 65536, kVtSlotBytes = 64 * 128 * 4;
 size_t mdn_chunk_states_bytes(const mdn_params* p) {
   mdn_ws_layout lay;
   if (check_params(p) != MDN_OK || make_layout(*p, &lay) != MDN_OK) return 0;
   if (resolve_path(*p) != MDN_PATH_TENSOR) return 0;
-  return (size_t)lay.num_slots * p->H * 65536;
+  return (size_t)lay.num_slots * p->H * (kStateImageBytes + kVtSlotBytes);
 }
 
 mdn_status mdn_chunk_fwd_keep_states(const mdn_params* p, const void* q, const void* k, const void* v,
@@ -217,11 +221,16 @@ mdn_status mdn_chunk_fwd_keep_states(const mdn_params* p, const void* q, const v
   mdn_status st = make_plan(&ps, cu_seqlens, workspace, workspace_bytes, cuda_stream, &pl);
   if (st != MDN_OK) return st;
   pl.chain_dump = static_cast<uint8_t*>(chunk_states);
+  pl.chain_vt_dump = reinterpret_cast<float*>(pl.chain_dump + (uint64_t)pl.lay.num_slots * p->H * kStateImageBytes);
   return run_forward(pl, q, k, v, beta, log_alpha, log_mu, eta, initial_S, initial_M, o, final_S, final_M);
 }
 
 // ---- chunk-parallel backward, stage 1: the adjoint of the inter-chunk state recurrence
-struct AdjLayout { mdn_params pe; mdn_ws_layout le; uint64_t k_ext, v_ext, ws_ext, cu_ext, total; };
+struct AdjLayout {
+  mdn_params pe; mdn_ws_layout le; uint64_t k_ext, v_ext, ws_ext, cu_ext, total;
+  uint64_t image_bytes() const { return (uint64_t)le.num_slots * pe.H * kStateImageBytes; }
+  uint64_t states_bytes() const { return image_bytes() + (uint64_t)((le.num_slots + 1) / 2) * pe.H * kVtSlotBytes; }
+};
 
 static mdn_status adj_layout(const mdn_params* p, AdjLayout* a) {
   mdn_status st = check_params(p);
@@ -258,7 +267,7 @@ size_t mdn_bwd_state_chain_workspace_bytes(const mdn_params* p) {
 
 size_t mdn_bwd_adjoint_states_bytes(const mdn_params* p) {
   AdjLayout a;
-  return adj_layout(p, &a) == MDN_OK ? (size_t)a.le.num_slots * p->H * 65536 : 0;
+  return adj_layout(p, &a) == MDN_OK ? (size_t)a.states_bytes() : 0;
 }
 
 mdn_status mdn_bwd_state_chain(const mdn_params* p, const void* q, const void* k, const void* d_o,
@@ -296,6 +305,8 @@ mdn_status mdn_bwd_state_chain(const mdn_params* p, const void* q, const void* k
   if (e != cudaSuccess) { t_last_cuda_error = (int)e; return MDN_ERR_CUDA; }
   // the forward's chain kernel on the extended problem, roles exchanged: its "S" is dM, its "M" is dS
   ext.chain_dump = static_cast<uint8_t*>(adjoint_states);
+  ext.chain_vt_dump = reinterpret_cast<float*>(ext.chain_dump + al.image_bytes());
+  ext.chain_vt_dump_even_only = 1;
   ext.chain_state_only = 1;
   ext.chain_end_scalars_in_rk = 1;
   e = launch_chain_tensor(ext, w + al.k_ext, w + al.k_ext, w + al.v_ext, d_final_M, d_final_S, w + al.v_ext,
@@ -317,8 +328,8 @@ static mdn_status chunked_bwd_layout(const mdn_params* p, ChunkedBwdLayout* c) {
   uint64_t off = 0;
   auto take = [&](uint64_t bytes) { uint64_t at = off; off = align_up(off + bytes, 1024); return at; };
   c->ws_fwd = take(c->lf.total_bytes);
-  c->fwd_states = take((uint64_t)c->lf.num_slots * p->H * 65536);
-  c->adj_states = take((uint64_t)c->al.le.num_slots * p->H * 65536);
+  c->fwd_states = take((uint64_t)c->lf.num_slots * p->H * (kStateImageBytes + kVtSlotBytes));
+  c->adj_states = take(c->al.states_bytes());
   c->stage = take(c->al.total);
   c->total = off;
   return MDN_OK;
@@ -351,8 +362,12 @@ static mdn_status bwd_from_states(const mdn_params* p, const ChunkedBwdLayout& c
   Plan fwd;
   st = make_plan(&pf, cu_seqlens, fwd_ws, c.lf.total_bytes, cuda_stream, &fwd);
   if (st != MDN_OK) return st;
-  cudaError_t e = launch_bwd_chunk_par(fwd, q, k, v, d_o, beta, log_alpha, log_mu, eta, fwd_states, adj_states,
-                                       stage + c.al.v_ext, dq, dk, dv, dbeta, dlog_alpha, dlog_mu, deta, &t_last_launches);
+  const char* fs = static_cast<const char*>(fwd_states);
+  cudaError_t e = launch_bwd_chunk_par(
+      fwd, q, k, d_o, beta, log_alpha, log_mu, eta, fs,
+      reinterpret_cast<const float*>(fs + (uint64_t)c.lf.num_slots * p->H * kStateImageBytes), adj_states,
+      reinterpret_cast<const float*>(adj_states + c.al.image_bytes()), dq, dk, dv, dbeta, dlog_alpha, dlog_mu, deta,
+      &t_last_launches);
   if (e != cudaSuccess) { t_last_cuda_error = (int)e; return MDN_ERR_CUDA; }
   return MDN_OK;
 }
@@ -405,6 +420,7 @@ mdn_status mdn_chunk_bwd_chunked(const mdn_params* p, const void* q, const void*
   st = make_plan(&pf, cu_seqlens, w + c.ws_fwd, c.lf.total_bytes, cuda_stream, &fwd);
   if (st != MDN_OK) return st;
   fwd.chain_dump = reinterpret_cast<uint8_t*>(w + c.fwd_states);
+  fwd.chain_vt_dump = reinterpret_cast<float*>(w + c.fwd_states + (uint64_t)c.lf.num_slots * p->H * kStateImageBytes);
   fwd.chain_state_only = 1;
   st = run_forward(fwd, q, k, v, beta, log_alpha, log_mu, eta, initial_S, initial_M, w + c.stage /* o: never written */,
                    nullptr, nullptr);

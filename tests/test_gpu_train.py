@@ -64,6 +64,31 @@ def test_keep_chunk_states(mdn, name, kw):
     fs, fm = bf16_floor(S_ref), bf16_floor(M_ref)
     print("chunk-start states (%s, %d slots): S %.3e (bf16 floor %.3e) M %.3e (floor %.3e)" % (name, n, es, fs, em, fm))
     assert es <= fs + TOL_OVER_FLOOR and em <= fm + TOL_OVER_FLOOR
+    # V~ = T (V - abar.(K S) + p.(K M)) of every chunk (Section 3.2), kept beside the states for the backward: against
+    # the fp64 chunk form evaluated on the oracle's own chunk-start states
+    from oracle import chunkwise_bwd as ob
+    Vt = mdn.unpack_chunk_vt(states, w.H).cpu().numpy()
+    lens = np.asarray(inp["seq_len"])
+    cu = inp.get("cu_seqlens")
+    f64 = lambda x: np.asarray(x, dtype=np.float64)
+    slot, got, ref = 0, [], []
+    for s_i in range(len(lens)):
+        b_i, base = (0, int(cu[s_i])) if cu is not None else (s_i, 0)
+        for c in range((int(lens[s_i]) + 63) // 64):
+            t0, nn = base + 64 * c, min(64, int(lens[s_i]) - 64 * c)
+            sl = slice(t0, t0 + nn)
+            for h in range(w.H):
+                eta = inp["eta"][b_i, sl, h] if inp.get("eta") is not None else np.ones(nn)
+                co = ob.chunk_coefficients(np.exp(f64(inp["log_alpha"][b_i, sl, h])), np.exp(f64(inp["log_mu"][b_i, sl, h])),
+                                           f64(inp["beta"][b_i, sl, h]), f64(eta))
+                fw = ob.chunk_forward(f64(inp["q"][b_i, sl, h]), f64(inp["k"][b_i, sl, h]), f64(inp["v"][b_i, sl, h]),
+                                      S_ref[slot, h], M_ref[slot, h], co, inp["scale"])
+                ref.append(fw["Vt"])
+                got.append(Vt[slot, :nn, h])
+            slot += 1
+    ev = rel_err(np.concatenate(got), np.concatenate(ref))
+    print("kept V~ (%s): %.3e" % (name, ev))
+    assert ev <= 2e-2
 
 
 @pytest.mark.parametrize("T, with_final", [(64 * 4 + 20, True), (64 * 3, False)])
@@ -86,7 +111,7 @@ def test_bwd_state_chain(mdn, T, with_final):
     adj, dS0, dM0 = mdn.bwd_state_chain(t["q"], t["k"], dev(d_o, torch.bfloat16), ws, v_dim=w.dv, d_final_S=dev(dSf),
                                         d_final_M=dev(dMf), scale=inp["scale"])
     torch.cuda.synchronize()
-    dM_e, dS_e = mdn.unpack_chunk_states(adj, w.H)       # entries: first half = dM, second half = dS
+    dM_e, dS_e = mdn.unpack_chunk_states(adj, w.H, adjoint=True)       # entries: first half = dM, second half = dS
     dM_e, dS_e = dM_e.cpu().numpy(), dS_e.cpu().numpy()
     nch = (T + 63) // 64
     ref_S, ref_M, got_S, got_M = [], [], [], []
