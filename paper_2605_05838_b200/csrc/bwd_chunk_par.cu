@@ -68,7 +68,6 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
   const uint32_t sb = smem_u32(smem);
   bf16* sK = reinterpret_cast<bf16*>(smem + kOffK);
   bf16* sQ = reinterpret_cast<bf16*>(smem + kOffQ);
-  bf16* sDO = reinterpret_cast<bf16*>(smem + kOffDO);
   float* sGam = reinterpret_cast<float*>(smem + kR2);         // gamma, m
   float* sMm = sGam + C * LG;
   bf16* sDWH = reinterpret_cast<bf16*>(smem + kR1);           // DW, DA (hi, lo)
@@ -98,13 +97,11 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
   // operands
   const Opnd oK{sb + kOffK, LT * 2, false}, oK_t{sb + kOffK, LT * 2, true};
   const Opnd oQ{sb + kOffQ, LT * 2, false}, oQ_t{sb + kOffQ, LT * 2, true};
-  const Opnd oDO{sb + kOffDO, LT * 2, false}, oDO_t{sb + kOffDO, LT * 2, true};
+  const Opnd oDO{sb + kOffDO, LT * 2, false};
   // a state in an area: B(k = key d, n = value j) = S[d][j], stored [j][d]; or B(k = value j, n = key d)
-  auto st_dk = [&](uint32_t base) { return Opnd{sb + base, LT * 2, false}; };
   auto st_dv = [&](uint32_t base) { return Opnd{sb + base, LT * 2, true}; };
   // a 64 x 128 tile in an area, stored [row][column]: as A it is [m][k], as B it is [n][k]; tile_kn reads it as B [k][n]
   auto tile_mk = [&](uint32_t base) { return Opnd{sb + base, LT * 2, false}; };
-  auto tile_kn = [&](uint32_t base) { return Opnd{sb + base, LT * 2, true}; };
   const Opnd oDWH{sb + kR1, L6 * 2, false}, oDWL{sb + kR1 + kMat6, L6 * 2, false};
   const Opnd oDWH_t{sb + kR1, L6 * 2, true}, oDWL_t{sb + kR1 + kMat6, L6 * 2, true};
   const Opnd oDAH{sb + kR3, L6 * 2, false}, oDAL{sb + kR3 + kMat6, L6 * 2, false};
@@ -374,107 +371,125 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
     }
   });
 
-  // ---- gate gradients: the recurrences of Eq. 10 in reverse.  Thread i walks column i of gamma / m from the last
-  // row up, carrying the adjoints of gamma_{r,i} and m_{r,i}; what belongs to a row goes to the row's accumulators.
+  // ---- gate gradients: the recurrences of Eq. 10 in reverse, column i of gamma / m from the last row up, carrying
+  // the adjoints of gamma_{r,i} and m_{r,i}.
   __syncthreads();   // d Geta, d G^- written; all row sums in; DW, DA have been read
-  // per-(row, column) contributions to d alpha, d beta, d mu go to three matrices (the area DW, DA used) and are
-  // summed along the rows afterwards: all columns reach a row in the same step, shared-memory atomics would serialise
-  float* cAl = reinterpret_cast<float*>(smem + kR1);
-  float* cBe = cAl + C * LG;
-  float* cMu = reinterpret_cast<float*>(smem + kR3);
-  static_assert(2 * kMatF <= 2 * kTile, "contribution matrices");
-  for (int idx = tid; idx < C * LG; idx += kThreads) { cAl[idx] = 0.f; cBe[idx] = 0.f; cMu[idx] = 0.f; }
-  __syncthreads();
+  // In two passes.  Serial (thread i = column i, from the last row up): only the two carried adjoints
+  //     d gamma_{r,i} = dg + dGeta_{r,i} eta_i,      dg <- alpha_r (d gamma_{r,i} + dG^-_{r,i} eta_i)
+  //     d m_{r,i}     = dm + d gamma_{r,i} beta_r,   dm <- mu_r d m_{r,i}
+  // (g_S, g_M enter in the last row), written to two matrices in the area DW used.  Everything that is a sum over a
+  // row (d alpha_r, d beta_r, d mu_r) or over a column (d eta_i) of products with these follows on all threads:
+  // shared-memory atomics from the serial walk would serialise 64-way, and the walk itself is one instruction stream.
+  float* sDg = reinterpret_cast<float*>(smem + kR1);
+  float* sDm = sDg + C * LG;
+  float* sPart = reinterpret_cast<float*>(smem + kR3);   // [3][64] partial column sums
+  static_assert(2 * kMatF <= 2 * kTile, "adjoint matrices");
   if (tid < C) {
     const int i = tid;
     const float eta_i = V(vEta)[i];
-    float dg = 0.f, dm = 0.f, deta_i = 0.f;
-    for (int r = C - 1; r >= i; --r) {
-      const float gam = sGam[r * LG + i], mm = sMm[r * LG + i];
-      const float gam_up = r > i ? sGam[(r - 1) * LG + i] : 0.f;
-      const float al = V(vAlpha)[r], dge = sdGe[r * LG + i], dgm = sdGm[r * LG + i];
-      // gamma_{r,i} feeds Geta_{r,i}, G^-_{r+1,i} (carried in dg from the row below) and, in the last row, g_S
-      float dgam = dg + dge * eta_i;
-      float dmm = dm;
-      if (r == C - 1) {
-        dgam += V(vdGS)[i] * eta_i;
-        dmm += V(vdGM)[i] * eta_i;
-        deta_i += V(vdGS)[i] * gam + V(vdGM)[i] * mm;
+    float dg = V(vdGS)[i] * eta_i, dm = V(vdGM)[i] * eta_i;   // what g_S, g_M give to the last row
+    for (int rb = C - 4; rb >= 0; rb -= 4) {   // four rows' loads first: the walk itself is a chain of three FMAs per row
+      float dge[4], dgm[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) { dge[u] = sdGe[(rb + u) * LG + i]; dgm[u] = sdGm[(rb + u) * LG + i]; }   // zero above the diagonal
+      const float4 al4 = *reinterpret_cast<const float4*>(V(vAlpha) + rb), be4 = *reinterpret_cast<const float4*>(V(vBeta) + rb);
+      const float4 mu4 = *reinterpret_cast<const float4*>(V(vMu) + rb);
+      const float al[4] = {al4.x, al4.y, al4.z, al4.w}, be[4] = {be4.x, be4.y, be4.z, be4.w}, mu[4] = {mu4.x, mu4.y, mu4.z, mu4.w};
+#pragma unroll
+      for (int u = 3; u >= 0; --u) {
+        const float dgam = fmaf(dge[u], eta_i, dg);
+        const float dmm = fmaf(dgam, be[u], dm);
+        sDg[(rb + u) * LG + i] = dgam;
+        sDm[(rb + u) * LG + i] = dmm;
+        dg = al[u] * fmaf(dgm[u], eta_i, dgam);
+        dm = dmm * mu[u];
       }
-      deta_i += dge * gam + dgm * al * gam_up;
-      dmm += dgam * V(vBeta)[r];
-      cAl[r * LG + i] = dgam * gam_up + dgm * gam_up * eta_i;
-      cBe[r * LG + i] = dgam * mm;
-      if (r > i) cMu[r * LG + i] = dmm * sMm[(r - 1) * LG + i];
-      // to the row above: gamma_{r-1,i} through the recurrence and through G^-_{r,i} = alpha_r gamma_{r-1,i} eta_i
-      dg = dgam * al + dgm * al * eta_i;
-      dm = dmm * V(vMu)[r];
     }
-    V(vdEta)[i] = deta_i;
+  } else {
+    // meanwhile on the other six warps, column sums that do not need the walk: d eta_i = sum_r dGeta gamma_{r,i} +
+    // dG^- alpha_r gamma_{r-1,i}, and the last row's g_S, g_M terms (three threads per column, a third of the rows each)
+    const int i = (tid - C) & 63, part = (tid - C) >> 6, r0 = 22 * part, r1 = min(C, r0 + 22);
+    float s = 0.f;
+#pragma unroll 4
+    for (int r = max(r0, i); r < r1; ++r) {
+      s = fmaf(sdGe[r * LG + i], sGam[r * LG + i], s);
+      if (r > i) s = fmaf(sdGm[r * LG + i] * V(vAlpha)[r], sGam[(r - 1) * LG + i], s);
+    }
+    if (part == 2) s += V(vdGS)[i] * sGam[(C - 1) * LG + i] + V(vdGM)[i] * sMm[(C - 1) * LG + i];
+    sPart[part * C + i] = s;
   }
   __syncthreads();
-  {   // row sums: four threads per row
+  {   // row sums, four threads per row: d alpha_r += sum_i gamma_{r-1,i} (d gamma + dG^- eta_i), d beta_r += sum_i
+      // d gamma m_{r,i}, d mu_r += sum_i d m m_{r-1,i}   (columns i <= r; the terms with gamma_{r-1,i}, m_{r-1,i}: i < r)
     const int r = tid >> 2, part = tid & 3;
     float sa = 0.f, sbe = 0.f, sm = 0.f;
-    for (int i = part * 16; i < part * 16 + 16; ++i) { sa += cAl[r * LG + i]; sbe += cBe[r * LG + i]; sm += cMu[r * LG + i]; }
+#pragma unroll 4
+    for (int i = part; i < C; i += 4) {   // columns interleaved over the row's four threads: conflict-free
+      if (i <= r) {
+        const float dgam = sDg[r * LG + i], dmm = sDm[r * LG + i];
+        sbe = fmaf(dgam, sMm[r * LG + i], sbe);
+        if (i < r) {
+          sa = fmaf(sGam[(r - 1) * LG + i], fmaf(sdGm[r * LG + i], V(vEta)[i], dgam), sa);
+          sm = fmaf(dmm, sMm[(r - 1) * LG + i], sm);
+        }
+      }
+    }
     sa += __shfl_xor_sync(0xffffffffu, sa, 1); sa += __shfl_xor_sync(0xffffffffu, sa, 2);
     sbe += __shfl_xor_sync(0xffffffffu, sbe, 1); sbe += __shfl_xor_sync(0xffffffffu, sbe, 2);
     sm += __shfl_xor_sync(0xffffffffu, sm, 1); sm += __shfl_xor_sync(0xffffffffu, sm, 2);
     if (part == 0) { V(vdAlpha)[r] += sa; V(vdBeta)[r] += sbe; V(vdMu)[r] += sm; }
   }
   __syncthreads();
-  // the three vector recurrences (p_r = alpha_r b_{r-1};  b_r = alpha_r b_{r-1} + beta_r mubar_r;  the cumulative
-  // products) in reverse: element-wise parts on 64 threads, the two 64-step chains on one thread each with the carry
-  // in a register
-  {
-    float* dAl = V(vdAlpha); float* dBe = V(vdBeta); float* dMu = V(vdMu);
-    float* dAb = V(vdAbar); float* dB = V(vdB); float* dMb = V(vdMubar);
-    if (tid < C) {
-      const int r = tid;
-      dAl[r] += V(vdP)[r] * V(vBprev)[r];
-      if (r + 1 < C) dB[r] += V(vdP)[r + 1] * V(vAlpha)[r + 1];
-    }
-    __syncthreads();
-    if (tid == 0) {
-      float carry = 0.f;
-      for (int r = C - 1; r >= 0; --r) {
-        const float x = dB[r] + carry;
-        dB[r] = x;
-        carry = x * V(vAlpha)[r];
+  // The three vector recurrences (p_r = alpha_r b_{r-1};  b_r = alpha_r b_{r-1} + beta_r mubar_r;  the cumulative
+  // products) in reverse, on one warp with two rows per lane and everything in registers.  Each reverse chain
+  // x_{r-1} = d_{r-1} + c_r x_r is a suffix scan of affine maps: the lane's two rows compose to x_{2l} = B + A x_{2l+2},
+  // five shuffle steps compose the lanes.
+  if (warp == 0) {
+    const int e0 = 2 * lane, e1 = e0 + 1;
+    auto rev_scan = [&](float& d0, float& d1, float c1, float c2) {   // c1 = c_{e1}, c2 = c_{e1+1} (0 past the end)
+      float A = c1 * c2, B = fmaf(c1, d1, d0);
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const float A2 = __shfl_down_sync(0xffffffffu, A, o), B2 = __shfl_down_sync(0xffffffffu, B, o);
+        if (lane + o < 32) { B = fmaf(A, B2, B); A *= A2; }
       }
+      float xn = __shfl_down_sync(0xffffffffu, B, 1);
+      if (lane == 31) xn = 0.f;
+      d1 = fmaf(c2, xn, d1);
+      d0 = B;
+    };
+    const float2 al = *reinterpret_cast<const float2*>(V(vAlpha) + e0), mu = *reinterpret_cast<const float2*>(V(vMu) + e0);
+    const float al2 = lane < 31 ? V(vAlpha)[e0 + 2] : 0.f, mu2 = lane < 31 ? V(vMu)[e0 + 2] : 0.f;
+    const float2 be = *reinterpret_cast<const float2*>(V(vBeta) + e0), bp = *reinterpret_cast<const float2*>(V(vBprev) + e0);
+    const float2 mb = *reinterpret_cast<const float2*>(V(vMubar) + e0), dP = *reinterpret_cast<const float2*>(V(vdP) + e0);
+    const float dP2 = lane < 31 ? V(vdP)[e0 + 2] : 0.f;
+    float2 dAl = *reinterpret_cast<const float2*>(V(vdAlpha) + e0), dBe = *reinterpret_cast<const float2*>(V(vdBeta) + e0);
+    float2 dMu = *reinterpret_cast<const float2*>(V(vdMu) + e0), dAb = *reinterpret_cast<const float2*>(V(vdAbar) + e0);
+    float2 dB = *reinterpret_cast<const float2*>(V(vdB) + e0), dMb = *reinterpret_cast<const float2*>(V(vdMubar) + e0);
+    const float ab_prev0 = lane > 0 ? V(vAbar)[e0 - 1] : 1.f, mb_prev0 = lane > 0 ? V(vMubar)[e0 - 1] : 1.f;
+    const float ab0 = V(vAbar)[e0];
+    // p_r = alpha_r b_{r-1}
+    dAl.x = fmaf(dP.x, bp.x, dAl.x); dAl.y = fmaf(dP.y, bp.y, dAl.y);
+    dB.x = fmaf(dP.y, al.y, dB.x); dB.y = fmaf(dP2, al2, dB.y);
+    rev_scan(dB.x, dB.y, al.y, al2);                      // b_r = alpha_r b_{r-1} + beta_r mubar_r
+    dAl.x = fmaf(dB.x, bp.x, dAl.x); dAl.y = fmaf(dB.y, bp.y, dAl.y);
+    dBe.x = fmaf(dB.x, mb.x, dBe.x); dBe.y = fmaf(dB.y, mb.y, dBe.y);
+    dMb.x = fmaf(dB.x, be.x, dMb.x); dMb.y = fmaf(dB.y, be.y, dMb.y);
+    rev_scan(dAb.x, dAb.y, al.y, al2);                    // abar_r = alpha_r abar_{r-1},  mubar_r = mu_r mubar_{r-1}
+    rev_scan(dMb.x, dMb.y, mu.y, mu2);
+    dAl.x = fmaf(dAb.x, ab_prev0, dAl.x); dAl.y = fmaf(dAb.y, ab0, dAl.y);
+    dMu.x = fmaf(dMb.x, mb_prev0, dMu.x); dMu.y = fmaf(dMb.y, mb.x, dMu.y);
+    const float de0 = sPart[e0] + sPart[C + e0] + sPart[2 * C + e0], de1 = sPart[e1] + sPart[C + e1] + sPart[2 * C + e1];
+    if (e0 < n) {
+      const size_t gi = tok(e0);
+      a.dbeta[gi] = dBe.x; a.dlog_alpha[gi] = al.x * dAl.x; a.dlog_mu[gi] = mu.x * dMu.x;
+      if (a.deta) a.deta[gi] = de0;
     }
-    __syncthreads();
-    if (tid < C) {
-      const int r = tid;
-      dAl[r] += dB[r] * V(vBprev)[r];
-      dBe[r] += dB[r] * V(vMubar)[r];
-      dMb[r] += dB[r] * V(vBeta)[r];
+    if (e1 < n) {
+      const size_t gi = tok(e1);
+      a.dbeta[gi] = dBe.y; a.dlog_alpha[gi] = al.y * dAl.y; a.dlog_mu[gi] = mu.y * dMu.y;
+      if (a.deta) a.deta[gi] = de1;
     }
-    __syncthreads();
-    if (tid == 0 || tid == 32) {
-      float* d = tid == 0 ? dAb : dMb;
-      const float* mul = tid == 0 ? V(vAlpha) : V(vMu);
-      float carry = 0.f;
-      for (int r = C - 1; r >= 0; --r) {
-        const float x = d[r] + carry;
-        d[r] = x;
-        carry = x * mul[r];
-      }
-    }
-    __syncthreads();
-    if (tid < C) {
-      const int r = tid;
-      dAl[r] += dAb[r] * (r > 0 ? V(vAbar)[r - 1] : 1.f);
-      dMu[r] += dMb[r] * (r > 0 ? V(vMubar)[r - 1] : 1.f);
-    }
-  }
-  __syncthreads();
-  if (tid < n) {
-    const size_t gi = tok(tid);
-    a.dbeta[gi] = V(vdBeta)[tid];
-    a.dlog_alpha[gi] = V(vAlpha)[tid] * V(vdAlpha)[tid];
-    a.dlog_mu[gi] = V(vMu)[tid] * V(vdMu)[tid];
-    if (a.deta) a.deta[gi] = V(vdEta)[tid];
   }
 }
 
