@@ -43,7 +43,8 @@ constexpr uint32_t kOffVt = kOffDO + kTile;           // V~ hi, lo; later DW hi,
 constexpr uint32_t kOffDR = kOffVt + 2 * kTile;       // dR hi, lo; later DA hi, lo
 constexpr uint32_t kOffTmp = kOffDR + 2 * kTile;      // dS', then M again; later gamma, m (fp32 [64][LG] each)
 constexpr uint32_t kOffVec = kOffTmp + 2 * kTile;     // vectors, 24 x [64] floats
-constexpr uint32_t kSmem = kOffVec + 24 * C * 4;
+constexpr uint32_t kOffGam = kOffVec + 24 * C * 4;    // gamma, fp32 [64][LG]: built while the first loads are in flight
+constexpr uint32_t kSmem = kOffGam + kMatF;
 constexpr uint32_t kR0 = kOffSt, kR1 = kOffVt, kR2 = kOffDR, kR3 = kOffTmp;   // the four reusable areas (see the kernel)
 static_assert(kD * LT * 2 == 2 * kTile, "a state and a hi + lo tile pair have the same size");
 static_assert(2 * kTile >= 2 * kMatF && kD * LT * 2 >= 2 * kMatF && 2 * kTile >= 2 * kMat6, "overlays");
@@ -68,8 +69,8 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
   const uint32_t sb = smem_u32(smem);
   bf16* sK = reinterpret_cast<bf16*>(smem + kOffK);
   bf16* sQ = reinterpret_cast<bf16*>(smem + kOffQ);
-  float* sGam = reinterpret_cast<float*>(smem + kR2);         // gamma, m
-  float* sMm = sGam + C * LG;
+  float* sGam = reinterpret_cast<float*>(smem + kOffGam);     // gamma (own place), m
+  float* sMm = reinterpret_cast<float*>(smem + kR2);
   bf16* sDWH = reinterpret_cast<bf16*>(smem + kR1);           // DW, DA (hi, lo)
   bf16* sDWL = sDWH + C * L6;
   bf16* sDAH = reinterpret_cast<bf16*>(smem + kR3);
@@ -156,21 +157,35 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
   };
   auto cp_async_commit = []() { asm volatile("cp.async.commit_group;" ::: "memory"); };
   auto cp_async_wait = []() { asm volatile("cp.async.wait_group 0;" ::: "memory"); };
-  // sum of the element-wise product of two states resident in two areas ([128][LT] each, 16 pieces of 16 B per row)
-  auto dot_areas = [&](uint32_t x, uint32_t y) {
-    float s = 0.f;
-    for (int idx = tid; idx < kD * 16; idx += kThreads) {
+  // the three inner products of state images that the end-of-chunk adjoints need, in one pass over the four areas
+  // ([128][LT] each, 16 pieces of 16 B per row): <dM', M>, <dS', S>, <dS', M>, summed per warp
+  auto state_dots = [&](float& dmm, float& dss, float& dsm) {
+    float s0 = 0.f, s1 = 0.f, s2 = 0.f;
+#pragma unroll 2
+    for (int idx = tid - C; idx < kD * 16; idx += kThreads - C) {   // threads C.. (the first two warps are elsewhere)
       const uint32_t off = ((idx >> 4) * LT + (idx & 15) * 8) * 2;
-      const uint4 ux = *reinterpret_cast<const uint4*>(smem + x + off), uy = *reinterpret_cast<const uint4*>(smem + y + off);
-      const uint32_t xs[4] = {ux.x, ux.y, ux.z, ux.w}, ys[4] = {uy.x, uy.y, uy.z, uy.w};
+      const uint4 uS = *reinterpret_cast<const uint4*>(smem + kR0 + off), uM = *reinterpret_cast<const uint4*>(smem + kR1 + off);
+      const uint4 udS = *reinterpret_cast<const uint4*>(smem + kR2 + off), udM = *reinterpret_cast<const uint4*>(smem + kR3 + off);
+      const uint32_t xS[4] = {uS.x, uS.y, uS.z, uS.w}, xM[4] = {uM.x, uM.y, uM.z, uM.w};
+      const uint32_t xdS[4] = {udS.x, udS.y, udS.z, udS.w}, xdM[4] = {udM.x, udM.y, udM.z, udM.w};
 #pragma unroll
-      for (int e = 0; e < 4; ++e)
-        s += __uint_as_float(xs[e] << 16) * __uint_as_float(ys[e] << 16) +
-             __uint_as_float(xs[e] & 0xffff0000u) * __uint_as_float(ys[e] & 0xffff0000u);
+      for (int e = 0; e < 4; ++e) {
+        const float S0 = __uint_as_float(xS[e] << 16), S1 = __uint_as_float(xS[e] & 0xffff0000u);
+        const float M0 = __uint_as_float(xM[e] << 16), M1 = __uint_as_float(xM[e] & 0xffff0000u);
+        const float dS0 = __uint_as_float(xdS[e] << 16), dS1 = __uint_as_float(xdS[e] & 0xffff0000u);
+        const float dM0 = __uint_as_float(xdM[e] << 16), dM1 = __uint_as_float(xdM[e] & 0xffff0000u);
+        s0 = fmaf(dM0, M0, fmaf(dM1, M1, s0));
+        s1 = fmaf(dS0, S0, fmaf(dS1, S1, s1));
+        s2 = fmaf(dS0, M0, fmaf(dS1, M1, s2));
+      }
     }
 #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
-    return s;   // per warp; lane 0 adds it where it belongs
+    for (int off = 16; off > 0; off >>= 1) {
+      s0 += __shfl_xor_sync(0xffffffffu, s0, off);
+      s1 += __shfl_xor_sync(0xffffffffu, s1, off);
+      s2 += __shfl_xor_sync(0xffffffffu, s2, off);
+    }
+    dmm = s0; dss = s1; dsm = s2;   // per warp; lane 0 adds them where they belong
   };
   // row sums of G o X over the warp's 32 columns, added to a vector (X: a bf16 tile, k or q)
   auto add_rowsum = [&](float (&G)[2][4][4], const bf16* X, float* dst, float sign) {
@@ -205,7 +220,7 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
   // Four areas of 34816 bytes (a state, or the hi + lo pair of a 64 x 128 tile) are reused through the phases:
   //   R0: S                                               | later d Geta, d G^-
   //   R1: M    | V~ (fp32, then hi, lo)                   | later DW (hi, lo), then two contribution matrices
-  //   R2: dS'  | M again                                  | gamma, m
+  //   R2: dS'  | M again                                  | m
   //   R3: dM'  | dR (fp32, then hi, lo)                   | DA (hi, lo), then a contribution matrix
   // All four states arrive at the start by cp.async (no registers in between); M is fetched a second time later.
   load_state(imgS, kR0);
@@ -231,9 +246,27 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
   }
   cp_async_wait();
   __syncthreads();
-  if (tid < C) V(vBprev)[tid] = tid > 0 ? V(vB)[tid - 1] : 0.f;
-  {   // the end-of-chunk adjoints: d mubar_C = <dM', M>, d abar_C = <dS', S>, d b_C = -<dS', M>
-    const float s0 = dot_areas(kR3, kR1), s1 = dot_areas(kR2, kR0), s2 = dot_areas(kR2, kR1);
+  if (tid < C) {
+    // two warps: gamma by the column recurrence of Eq. 10 (thread = column) ...
+    V(vBprev)[tid] = tid > 0 ? V(vB)[tid - 1] : 0.f;
+    const int i = tid;
+    float m = 1.f, gam = 0.f;
+    for (int rb = 0; rb < C; rb += 4) {
+      const float4 al = *reinterpret_cast<const float4*>(V(vAlpha) + rb), be = *reinterpret_cast<const float4*>(V(vBeta) + rb);
+      const float4 mu = *reinterpret_cast<const float4*>(V(vMu) + rb);
+      const float a4[4] = {al.x, al.y, al.z, al.w}, b4[4] = {be.x, be.y, be.z, be.w}, m4[4] = {mu.x, mu.y, mu.z, mu.w};
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int rr = rb + u;
+        if (rr > i) m *= m4[u];
+        if (rr >= i) gam = fmaf(a4[u], gam, b4[u] * m);
+        sGam[rr * LG + i] = rr >= i ? gam : 0.f;
+      }
+    }
+  } else {
+    // ... six warps: the end-of-chunk adjoints d mubar_C = <dM', M>, d abar_C = <dS', S>, d b_C = -<dS', M>
+    float s0, s1, s2;
+    state_dots(s0, s1, s2);
     if (lane == 0) {
       atomicAdd(V(vdMubar) + n - 1, s0);
       atomicAdd(V(vdAbar) + n - 1, s1);
@@ -309,17 +342,21 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
     for_frag<2, 4>(m0, n0, g, t, [&](int mt, int nt, int e, int r, int c) { dK[mt][nt][e] += V(vP)[r] * G[mt][nt][e]; });
     add_rowsum(G, sK, V(vdP), 1.f);
   }
-  __syncthreads();   // M has been read: its area takes gamma and m
+  __syncthreads();   // M has been read: its area takes m
 
-  // ---- gamma and m by the column recurrences of Eq. 10 (thread = column)
+  // ---- m by its column recurrence (thread = column): m_{r,i} = mu_{i+1} .. mu_r
   if (tid < C) {
     const int i = tid;
-    float m = 1.f, gam = 0.f;
-    for (int r = 0; r < C; ++r) {
-      if (r > i) m *= V(vMu)[r];
-      if (r >= i) gam = V(vAlpha)[r] * gam + V(vBeta)[r] * m;
-      sGam[r * LG + i] = r >= i ? gam : 0.f;
-      sMm[r * LG + i] = r >= i ? m : 0.f;
+    float m = 1.f;
+    for (int rb = 0; rb < C; rb += 4) {
+      const float4 mu = *reinterpret_cast<const float4*>(V(vMu) + rb);
+      const float m4[4] = {mu.x, mu.y, mu.z, mu.w};
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int rr = rb + u;
+        if (rr > i) m *= m4[u];
+        sMm[rr * LG + i] = rr >= i ? m : 0.f;
+      }
     }
   }
   // ---- the four 64 x 64 products
