@@ -50,6 +50,7 @@ static_assert(kD * LT * 2 == 2 * kTile, "a state and a hi + lo tile pair have th
 static_assert(2 * kTile >= 2 * kMatF && kD * LT * 2 >= 2 * kMatF && 2 * kTile >= 2 * kMat6, "overlays");
 static_assert(kSmem <= 232448, "shared memory");
 
+constexpr int kBarSlot = 22;   // vector slot that holds the two mbarriers and the abort flag instead
 enum Vec : int { vAbar = 0, vB, vP, vGS, vGM, vMubar, vAlpha, vBeta, vMu, vEta, vBprev,
                  vdAbar, vdB, vdP, vdGS, vdGM, vdMubar, vdAlpha, vdBeta, vdMu, vdEta, vRed };
 
@@ -60,6 +61,7 @@ struct ParArgs {
   const float* coef;
   const uint8_t* fwd_states; const uint8_t* adj_states;   // state images per chunk slot
   const float* fwd_vt; const float* adj_dr;               // V~ and dR per chunk slot, fp32 [slot][64][H][dv]
+  int32_t* status;                                        // the forward workspace's status word
   float scale;
   float* dq; float* dk; float* dv; float* dbeta; float* dlog_alpha; float* dlog_mu; float* deta;
 };
@@ -100,7 +102,7 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
   const Opnd oQ{sb + kOffQ, LT * 2, false}, oQ_t{sb + kOffQ, LT * 2, true};
   const Opnd oDO{sb + kOffDO, LT * 2, false};
   // a state in an area: B(k = key d, n = value j) = S[d][j], stored [j][d]; or B(k = value j, n = key d)
-  auto st_dv = [&](uint32_t base) { return Opnd{sb + base, LT * 2, true}; };
+  auto st_dv = [&](uint32_t base) { return Opnd{sb + base, 0, true, true}; };
   // a 64 x 128 tile in an area, stored [row][column]: as A it is [m][k], as B it is [n][k]; tile_kn reads it as B [k][n]
   auto tile_mk = [&](uint32_t base) { return Opnd{sb + base, LT * 2, false}; };
   const Opnd oDWH{sb + kR1, L6 * 2, false}, oDWL{sb + kR1 + kMat6, L6 * 2, false};
@@ -147,23 +149,21 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
       if (out != nullptr && r < n) *reinterpret_cast<float4*>(out + tok(r) * kD + c4) = x[i];
     }
   };
-  // state image (value index j x key index d, two swizzled blocks) -> [j][d] in an area, by cp.async
-  auto load_state = [&](const uint8_t* img, uint32_t base) {
-    for (int idx = tid; idx < 2 * kD * 8; idx += kThreads) {
-      const int half = idx >> 10, j = (idx >> 3) & 127, pp = idx & 7, c = pp ^ (j & 7);
-      const uint32_t dst = sb + base + (j * LT + half * 64 + c * 8) * 2;
-      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(img + half * 16384 + j * 128 + pp * 16));
-    }
+  // a state image (value index j x key index d, two swizzled blocks) goes into an area as it is, by two bulk copies
+  // from one thread; the products address it through the swizzle (Opnd::swz)
+  auto load_state = [&](const uint8_t* img, uint32_t base, uint32_t bar) {
+    bulk_load(sb + base, img, 16384, bar);
+    bulk_load(sb + base + 16384, img + 16384, 16384, bar);
   };
   auto cp_async_commit = []() { asm volatile("cp.async.commit_group;" ::: "memory"); };
   auto cp_async_wait = []() { asm volatile("cp.async.wait_group 0;" ::: "memory"); };
   // the three inner products of state images that the end-of-chunk adjoints need, in one pass over the four areas
-  // ([128][LT] each, 16 pieces of 16 B per row): <dM', M>, <dS', S>, <dS', M>, summed per warp
+  // (32768-byte images): <dM', M>, <dS', S>, <dS', M>, summed per warp
   auto state_dots = [&](float& dmm, float& dss, float& dsm) {
     float s0 = 0.f, s1 = 0.f, s2 = 0.f;
 #pragma unroll 2
     for (int idx = tid - C; idx < kD * 16; idx += kThreads - C) {   // threads C.. (the first two warps are elsewhere)
-      const uint32_t off = ((idx >> 4) * LT + (idx & 15) * 8) * 2;
+      const uint32_t off = idx * 16;   // the four images have the same layout: any common order will do
       const uint4 uS = *reinterpret_cast<const uint4*>(smem + kR0 + off), uM = *reinterpret_cast<const uint4*>(smem + kR1 + off);
       const uint4 udS = *reinterpret_cast<const uint4*>(smem + kR2 + off), udM = *reinterpret_cast<const uint4*>(smem + kR3 + off);
       const uint32_t xS[4] = {uS.x, uS.y, uS.z, uS.w}, xM[4] = {uM.x, uM.y, uM.z, uM.w};
@@ -223,17 +223,26 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
   //   R2: dS'  | M again                                  | m
   //   R3: dM'  | dR (fp32, then hi, lo)                   | DA (hi, lo), then a contribution matrix
   // All four states arrive at the start by cp.async (no registers in between); M is fetched a second time later.
-  load_state(imgS, kR0);
-  load_state(imgM, kR1);
-  load_state(imgdS, kR2);
-  load_state(imgdM, kR3);
+  const uint32_t bar0 = smem_u32(vec + kBarSlot * C), bar1 = bar0 + 8;   // mbarriers: the four states; M again
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(vec + kBarSlot * C + 4);
+  if (tid == 0) {
+    *abort_flag = 0;
+    mbar_init(bar0, 1);
+    mbar_init(bar1, 1);
+    mbar_fence_init();
+    mbar_arrive_expect_tx(bar0, 4 * 32768);
+    load_state(imgS, kR0, bar0);
+    load_state(imgM, kR1, bar0);
+    load_state(imgdS, kR2, bar0);
+    load_state(imgdM, kR3, bar0);
+  }
   load_tile(kOffK, a.k);
   load_tile(kOffQ, a.q);
   load_tile(kOffDO, a.d_o);
   cp_async_commit();
   // ---- vectors: the chain's coefficient vectors, the gates, zeroed adjoints
   const float* cf = a.coef + ((size_t)slot * H + h) * MDN_NUM_COEF * C;
-  for (int idx = tid; idx < 24 * C; idx += kThreads) vec[idx] = 0.f;
+  for (int idx = tid; idx < kBarSlot * C; idx += kThreads) vec[idx] = 0.f;
   __syncthreads();
   if (tid < C) {
     const int r = tid;
@@ -245,7 +254,13 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
     V(vBeta)[r] = live ? a.beta[gi] : 0.f; V(vEta)[r] = live ? (a.eta ? a.eta[gi] : 1.f) : 0.f;
   }
   cp_async_wait();
-  __syncthreads();
+  {   // the states: a bounded wait; if it runs out the CTA reports it and leaves (all threads together)
+    const bool ok = mbar_wait(bar0, 0, abort_flag);
+    if (!__syncthreads_and(ok)) {
+      if (tid == 0) atomicCAS(a.status, kDevOk, kDevTimeout);
+      return;
+    }
+  }
   if (tid < C) {
     // two warps: gamma by the column recurrence of Eq. 10 (thread = column) ...
     V(vBprev)[tid] = tid > 0 ? V(vB)[tid - 1] : 0.f;
@@ -319,9 +334,12 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
     add_rowsum(G, sK, V(vdGS), 1.f);
   }
   __syncthreads();   // dS' has been read: M takes its place
-  load_state(imgM, kR2);
-  cp_async_commit();
-  asm volatile("cp.async.wait_group 1;" ::: "memory");   // dR is in (M may still be on its way)
+  if (tid == 0) {
+    fence_proxy_async_smem();
+    mbar_arrive_expect_tx(bar1, 32768);
+    load_state(imgM, kR2, bar1);
+  }
+  cp_async_wait();   // dR is in (M may still be on its way)
   __syncthreads();
   split_in_place(kR3, a.dv);
   __syncthreads();
@@ -334,8 +352,13 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
     warp_mma(G, tile_mk(kR3 + kTile), st_dv(kR0), kD, m0, n0, lane);
     for_frag<2, 4>(m0, n0, g, t, [&](int mt, int nt, int e, int r, int c) { dK[mt][nt][e] -= V(vAbar)[r] * G[mt][nt][e]; });
     add_rowsum(G, sK, V(vdAbar), -1.f);
-    cp_async_wait();
-    __syncthreads();
+    {
+      const bool ok = mbar_wait(bar1, 0, abort_flag);
+      if (!__syncthreads_and(ok)) {
+        if (tid == 0) atomicCAS(a.status, kDevOk, kDevTimeout);
+        return;
+      }
+    }
     zero(G);
     warp_mma(G, tile_mk(kR3), st_dv(kR2), kD, m0, n0, lane);
     warp_mma(G, tile_mk(kR3 + kTile), st_dv(kR2), kD, m0, n0, lane);
@@ -545,6 +568,7 @@ cudaError_t launch_bwd_chunk_par(const Plan& fwd, const void* q, const void* k, 
   a.fwd_states = static_cast<const uint8_t*>(fwd_states);
   a.adj_states = static_cast<const uint8_t*>(adj_states);
   a.fwd_vt = fwd_vt; a.adj_dr = adj_dr;
+  a.status = reinterpret_cast<int32_t*>(fwd.ws + fwd.lay.off_status);
   a.scale = fwd.p.scale;
   a.dq = dq; a.dk = dk; a.dv = dv; a.dbeta = dbeta; a.dlog_alpha = dlog_alpha; a.dlog_mu = dlog_mu; a.deta = deta;
   cudaError_t e = cudaFuncSetAttribute(bwd_chunk_par_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmem);

@@ -23,7 +23,15 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], 
 
 // A bf16 operand in shared memory: byte address of element (0, 0), row stride in bytes, and how it is stored:
 // for A, trans = false means [m][k] (k contiguous), true means [k][m]; for B, false means [n][k], true means [k][n].
-struct Opnd { uint32_t base; uint32_t ld; bool trans; };
+// swz: the operand is a raw 128-byte-swizzled image instead ([.. x 128] bf16 as two blocks of [rows][64 columns],
+// 128-byte rows, 16384 bytes per block, the 16-byte piece index XORed with row mod 8); ld is then unused.
+struct Opnd { uint32_t base; uint32_t ld; bool trans; bool swz = false; };
+
+// byte address of the 8-element row segment (row, col .. col + 7), col a multiple of 8
+__device__ __forceinline__ uint32_t opnd_addr(const Opnd& o, int row, int col) {
+  if (!o.swz) return o.base + row * o.ld + col * 2;
+  return o.base + (col >> 6) * 16384 + row * 128 + ((((col >> 3) ^ row) & 7) << 4);
+}
 
 // acc[mt][nt] += A[m0 + 16 mt .., k] B[k, n0 + 8 nt ..] over k < K (a multiple of 16); NT even.
 template <int MT, int NT>
@@ -33,13 +41,13 @@ __device__ __forceinline__ void warp_mma(float (&acc)[MT][NT][4], Opnd A, Opnd B
     uint32_t af[MT][4], bfr[NT / 2][4];
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt) {
-      if (!A.trans) ldsm_x4(A.base + (m0 + 16 * mt + l7 + q1 * 8) * A.ld + (k0 + q2 * 8) * 2, af[mt]);
-      else ldsm_x4_t(A.base + (k0 + q2 * 8 + l7) * A.ld + (m0 + 16 * mt + q1 * 8) * 2, af[mt]);
+      if (!A.trans) ldsm_x4(opnd_addr(A, m0 + 16 * mt + l7 + q1 * 8, k0 + q2 * 8), af[mt]);
+      else ldsm_x4_t(opnd_addr(A, k0 + q2 * 8 + l7, m0 + 16 * mt + q1 * 8), af[mt]);
     }
 #pragma unroll
     for (int p = 0; p < NT / 2; ++p) {
-      if (!B.trans) ldsm_x4(B.base + (n0 + 16 * p + l7 + q2 * 8) * B.ld + (k0 + q1 * 8) * 2, bfr[p]);
-      else ldsm_x4_t(B.base + (k0 + q1 * 8 + l7) * B.ld + (n0 + 16 * p + q2 * 8) * 2, bfr[p]);
+      if (!B.trans) ldsm_x4(opnd_addr(B, n0 + 16 * p + l7 + q2 * 8, k0 + q1 * 8), bfr[p]);
+      else ldsm_x4_t(opnd_addr(B, k0 + q1 * 8 + l7, n0 + 16 * p + q2 * 8), bfr[p]);
     }
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt)
