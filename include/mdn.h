@@ -293,18 +293,17 @@ mdn_status mdn_chunk_fwd_keep_states(const mdn_params* p,
  *     dS  = abar_C dS' - K^T (abar . dR) + scale Q^T (abar . dO),
  *     dM  = -b_C dS' + mubar_C dM' + K^T (p . dR) - scale Q^T (b . dO)
  * walk the chunks of every sequence from the last to the first.  This has the shape of the forward's own chunk step
- * with the roles of S and M exchanged, so it is run by the forward's chain kernel on an extended problem (per
- * chunk a real step and a step that adds the two Q terms) built from the forward's workspace.
+ * with the roles of S and M exchanged plus a second rank-64 update for the two Q terms, so it is run by the forward's
+ * chain kernel on a mirrored problem (every sequence's chunks in reverse order) built from the forward's workspace.
  *   p, q, k, cu_seqlens: the forward call's (tensor path, o_dtype bf16); d_o = dL/do, [B,T,H,dv] bf16;
  *   d_final_S, d_final_M: dL/d(final states), [N,H,dk,dv] float32 or NULL (zero);
  *   fwd_workspace: the workspace of an mdn_chunk_fwd_keep_states call with the same p and inputs, untouched since
  *     (T, W and the coefficient vectors are read from it);
  *   adjoint_states: DEVICE buffer of mdn_bwd_adjoint_states_bytes(p) bytes, 1024-byte aligned.  Per sequence (in
- *     the workspace's slot order, entries of sequence s starting at twice its first chunk slot) and
- *     head it receives 2 x nchunks entries of 65536 bytes in the layout of mdn_chunk_fwd_keep_states with dM^T in
- *     the first half and dS^T in the second: entry 2 (nchunks - 1 - c) is the adjoint pair at the END of chunk c,
- *     entry 2 (nchunks - 1 - c) + 1 the pair after chunk c's K terms and before its Q terms; behind all entries, as
- *     float32 [entry / 2][64][H][dv], dR = T^T dV~ (= dL/dv) of the chunk whose real step is entry 2 (nchunks-1-c);
+ *     the workspace's slot order, entries of sequence s starting at its first chunk slot) and head it receives
+ *     nchunks entries of 65536 bytes in the layout of mdn_chunk_fwd_keep_states with dM^T in the first half and
+ *     dS^T in the second: entry nchunks - 1 - c is the adjoint pair at the END of chunk c; behind all entries, as
+ *     float32 [entry][64][H][dv], dR = T^T dV~ (= dL/dv) of the same chunk;
  *   d_initial_S, d_initial_M: dL/d(initial states), [B,H,dk,dv] float32, or NULL;
  *   workspace: mdn_bwd_state_chain_workspace_bytes(p) bytes, 1024-byte aligned, scratch.
  * The gradients of q, k, v and the gates follow from these adjoint states and the kept forward states chunk by chunk,

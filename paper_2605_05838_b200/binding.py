@@ -328,28 +328,22 @@ def chunk_fwd(q, k, v, beta, log_alpha, log_mu, eta=None, *, initial_S=None, ini
 _IMAGE_BYTES, _VT_BYTES = 65536, 64 * 128 * 4
 
 
-def _states_parts(states: torch.Tensor, H: int, adjoint: bool):
+def _states_parts(states: torch.Tensor, H: int):
     """(state images, V~ part, slots) of a kept-states buffer: per (slot, head) a 64 KB state image, and behind all
-    images one fp32 [64, H, 128] block per slot (forward) or per pair of slots (adjoint chain)."""
+    images one fp32 [64, H, 128] block per slot."""
     nbytes = states.numel()
-    if not adjoint:
-        slots = nbytes // (H * (_IMAGE_BYTES + _VT_BYTES))
-        vt_slots = slots
-    else:
-        pair = H * (2 * _IMAGE_BYTES + _VT_BYTES)
-        slots = 2 * (nbytes // pair) + (1 if nbytes % pair else 0)
-        vt_slots = (slots + 1) // 2
-    if slots * H * _IMAGE_BYTES + vt_slots * H * _VT_BYTES != nbytes:
+    slots = nbytes // (H * (_IMAGE_BYTES + _VT_BYTES))
+    if slots * H * (_IMAGE_BYTES + _VT_BYTES) != nbytes:
         raise ValueError("not a kept-states buffer for H = %d" % H)
     cut = slots * H * _IMAGE_BYTES
     return states[:cut], states[cut:], slots
 
 
-def unpack_chunk_states(states: torch.Tensor, H: int, adjoint: bool = False):
-    """The state images of a mdn_chunk_fwd_keep_states (or, adjoint=True, mdn_bwd_state_chain) buffer as float32
-    tensors (S, M) of shape [slots, H, dk, dv] (dk = dv = 128): undoes the transposition and the 128-byte swizzle of
-    the shared-memory image."""
-    images, _, _ = _states_parts(states, H, adjoint)
+def unpack_chunk_states(states: torch.Tensor, H: int):
+    """The state images of a mdn_chunk_fwd_keep_states (or mdn_bwd_state_chain) buffer as float32 tensors (S, M) of
+    shape [slots, H, dk, dv] (dk = dv = 128): undoes the transposition and the 128-byte swizzle of the shared-memory
+    image."""
+    images, _, _ = _states_parts(states, H)
     raw = images.view(torch.bfloat16).view(-1, H, 2, 2, 128, 8, 8)          # slot, head, S|M, key half, row, piece, elem
     rows = torch.arange(128, device=states.device)
     piece = torch.arange(8, device=states.device)
@@ -361,18 +355,19 @@ def unpack_chunk_states(states: torch.Tensor, H: int, adjoint: bool = False):
     return full[:, :, 0].contiguous(), full[:, :, 1].contiguous()
 
 
-def unpack_chunk_vt(states: torch.Tensor, H: int, adjoint: bool = False):
+def unpack_chunk_vt(states: torch.Tensor, H: int):
     """The second part of a kept-states buffer: V~ of every chunk slot as float32 [slots, 64, H, 128] (rows past a
-    short chunk's end are unwritten); with adjoint=True, dR = T^T dV~ at half the extended slot index."""
-    _, vt, _ = _states_parts(states, H, adjoint)
+    short chunk's end are unwritten); for the adjoint chain's buffer, dR = T^T dV~ in the chain's mirrored order."""
+    _, vt, _ = _states_parts(states, H)
     return vt.view(torch.float32).view(-1, 64, H, 128)
 
 
 def bwd_state_chain(q, k, d_o, fwd_workspace, *, v_dim: int, d_final_S=None, d_final_M=None, cu_seqlens=None,
                     scale: Optional[float] = None, want_initial: bool = True):
     """mdn_bwd_state_chain after a chunk_fwd(..., keep_chunk_states=True) call whose workspace is `fwd_workspace`.
-    Returns (adjoint_states, d_initial_S, d_initial_M): the raw adjoint-state buffer (2 entries per chunk, see
-    include/mdn.h; unpack_chunk_states gives (dM, dS) per entry) and the initial states' gradients."""
+    Returns (adjoint_states, d_initial_S, d_initial_M): the raw adjoint-state buffer (one entry per chunk, a
+    sequence's chunks in reverse order, see include/mdn.h; unpack_chunk_states gives (dM, dS) per entry) and the
+    initial states' gradients."""
     B, T, H, dk = q.shape
     N = 0 if cu_seqlens is None else cu_seqlens.numel() - 1
     nst = N if N > 0 else B

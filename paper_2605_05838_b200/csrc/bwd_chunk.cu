@@ -9,10 +9,11 @@
 // This has the shape of the forward's own chunk step with the roles exchanged (dM for S, dS for M):
 //     X = K dM', Y = K dS',  "R" = V' - g_M . X + g_S . Y  with V' = W^T dO,  "V~" = T^T "R" = dR,
 //     dM = mubar_C dM' - b_C dS' + K^T (p . dR),   dS = abar_C dS' - K^T (abar . dR),
-// followed by a second, state-only step that adds the two Q terms (K := Q, V := dO, T := I, no decay).
-// So the adjoint chain is run by the forward's chain kernel itself (chain_tensor.cu, training instantiation) on an
-// "extended" problem built here: per chunk, in REVERSE chunk order, a real step and an injection step.  This file
-// holds the kernel that builds that problem from the forward's workspace (T, W, coefficient vectors) and q, k, dO.
+// plus the two Q terms, a second rank-64 update of the pair: dM -= Q^T ((scale b) . dO), dS += Q^T ((scale abar) . dO).
+// So the adjoint chain is run by the forward's chain kernel itself (chain_tensor.cu, training instantiation with the
+// second update switched on) on a "mirrored" problem built here: the chunks of every sequence in REVERSE order,
+// short chunks padded to 64 rows.  This file holds the kernel that builds that problem from the forward's workspace
+// (T, W, coefficient vectors) and q, k, dO.
 #include "mdn_common.cuh"
 #include "tc_utils.cuh"
 #include "warp_mma.cuh"
@@ -35,10 +36,10 @@ struct PrepArgs {
   const __nv_bfloat16* W;           // forward: hi part, lo part w_lo_offset elements later
   size_t w_lo_offset;
   float scale;
-  // the extended problem: 2 chunks per forward chunk, sequence s = rows [s * 2 nch * 64, ..) of k_ext, v_ext
-  __nv_bfloat16* k_ext; __nv_bfloat16* v_ext;   // [B][2 nch 64][H][128]
-  float* coef_ext;                  // [2 slots][H][MDN_NUM_COEF][64]
-  __nv_bfloat16* T_ext;             // [2 slots][H][64][64]
+  // the mirrored problem: sequence s = rows [chunk_off[s] * 64, ..) of k_ext, q_ext, v_ext, do_ext
+  __nv_bfloat16* k_ext; __nv_bfloat16* q_ext; __nv_bfloat16* v_ext; __nv_bfloat16* do_ext;   // [slots 64][H][128]
+  float* coef_ext;                  // [slots][H][MDN_NUM_COEF][64]
+  __nv_bfloat16* T_ext;             // [slots][H][64][64]
 };
 
 __global__ void __launch_bounds__(kPrepThreads) bwd_prep_kernel(PrepArgs a) {
@@ -53,11 +54,11 @@ __global__ void __launch_bounds__(kPrepThreads) bwd_prep_kernel(PrepArgs a) {
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
   int slot0, nch;
   seq_chunks(a.g, si.seq, &slot0, &nch);
-  // extended chunk indices of this forward chunk: the real step, then the injection step
-  const int e_real = 2 * slot0 + 2 * (nch - 1 - si.local), e_inj = e_real + 1;
+  // where this forward chunk lies in the mirrored problem
+  const int e_real = slot0 + (nch - 1 - si.local);
   const size_t mat = ((size_t)slot * H + h) * C * C;
 
-  // ---- W (hi, lo), T and the dO tile into shared memory; dO also goes out as the "V" of the injection step
+  // ---- W (hi, lo), T and the dO tile into shared memory; dO also goes out in the mirrored order
   for (int idx = tid; idx < C * 8; idx += kPrepThreads) {
     const int r = idx >> 3, c8 = (idx & 7) * 8;
     *reinterpret_cast<uint4*>(sWH + r * L6 + c8) = *reinterpret_cast<const uint4*>(a.W + mat + r * C + c8);
@@ -69,7 +70,7 @@ __global__ void __launch_bounds__(kPrepThreads) bwd_prep_kernel(PrepArgs a) {
     uint4 x = make_uint4(0u, 0u, 0u, 0u);
     if (r < si.n) x = *reinterpret_cast<const uint4*>(a.d_o + ((size_t)(si.tok0 + r) * H + h) * kD + c8);
     *reinterpret_cast<uint4*>(sDO + r * LT + c8) = x;
-    *reinterpret_cast<uint4*>(a.v_ext + ((size_t)(e_inj * C + r) * H + h) * kD + c8) = x;
+    *reinterpret_cast<uint4*>(a.do_ext + ((size_t)(e_real * C + r) * H + h) * kD + c8) = x;
   }
   __syncthreads();
 
@@ -88,7 +89,7 @@ __global__ void __launch_bounds__(kPrepThreads) bwd_prep_kernel(PrepArgs a) {
     });
   }
 
-  // ---- keys of the two steps: k (real), q (injection); rows past the end of a short chunk are zero
+  // ---- k and q in the mirrored order; rows past the end of a short chunk are zero
   for (int idx = tid; idx < C * (kD / 8); idx += kPrepThreads) {
     const int r = idx >> 4, c8 = (idx & 15) * 8;
     uint4 kv = make_uint4(0u, 0u, 0u, 0u), qv = kv;
@@ -97,46 +98,43 @@ __global__ void __launch_bounds__(kPrepThreads) bwd_prep_kernel(PrepArgs a) {
       qv = *reinterpret_cast<const uint4*>(a.q + ((size_t)(si.tok0 + r) * H + h) * kD + c8);
     }
     *reinterpret_cast<uint4*>(a.k_ext + ((size_t)(e_real * C + r) * H + h) * kD + c8) = kv;
-    *reinterpret_cast<uint4*>(a.k_ext + ((size_t)(e_inj * C + r) * H + h) * kD + c8) = qv;
+    *reinterpret_cast<uint4*>(a.q_ext + ((size_t)(e_real * C + r) * H + h) * kD + c8) = qv;
   }
 
-  // ---- T^T (real), I (injection)
-  const size_t mat_r = ((size_t)e_real * H + h) * C * C, mat_i = ((size_t)e_inj * H + h) * C * C;
+  // ---- T^T
+  const size_t mat_r = ((size_t)e_real * H + h) * C * C;
   for (int idx = tid; idx < C * C; idx += kPrepThreads) {
     const int r = idx >> 6, i = idx & 63;
     a.T_ext[mat_r + idx] = Tt[i * L6 + r];
-    a.T_ext[mat_i + idx] = __float2bfloat16_rn(r == i ? 1.f : 0.f);
   }
 
-  // ---- coefficient vectors.  Real step: abar' = g_M, p' = g_S, g_S' = p, g_M' = abar, end-of-chunk scalars
-  // (mubar_C, b_C, abar_C) in vector 6.  Injection step: no decay, g_S' = -scale b, g_M' = -scale abar.
+  // ---- coefficient vectors: abar' = g_M, p' = g_S, g_S' = p, g_M' = abar, end-of-chunk scalars (mubar_C, b_C,
+  // abar_C) in vector 6; b stays where it is: with g_M' = abar it scales dO in the second update
   const float* cf = a.coef + ((size_t)slot * H + h) * MDN_NUM_COEF * C;
   float* cr = a.coef_ext + ((size_t)e_real * H + h) * MDN_NUM_COEF * C;
-  float* ci = a.coef_ext + ((size_t)e_inj * H + h) * MDN_NUM_COEF * C;
   for (int idx = tid; idx < MDN_NUM_COEF * C; idx += kPrepThreads) {
     const int vec = idx >> 6, r = idx & 63;
     const bool live = r < si.n;
-    float xr = 0.f, xi = 0.f;
+    float xr = 0.f;
     switch (vec) {
       case kAbar: xr = live ? cf[kGM * C + r] : 0.f; break;
+      case kB: xr = live ? cf[kB * C + r] : 0.f; break;
       case kAlphaBPrev: xr = live ? cf[kGS * C + r] : 0.f; break;
-      case kGS: xr = live ? cf[kAlphaBPrev * C + r] : 0.f; xi = live ? -a.scale * cf[kB * C + r] : 0.f; break;
-      case kGM: xr = live ? cf[kAbar * C + r] : 0.f; xi = live ? -a.scale * cf[kAbar * C + r] : 0.f; break;
+      case kGS: xr = live ? cf[kAlphaBPrev * C + r] : 0.f; break;
+      case kGM: xr = live ? cf[kAbar * C + r] : 0.f; break;
       case kRk:
         xr = r == 0 ? cf[kMubar * C + C - 1] : r == 1 ? cf[kB * C + C - 1] : r == 2 ? cf[kAbar * C + C - 1] : 1.f;
-        xi = r == 1 ? 0.f : 1.f;
         break;
-      case kRq: xr = 1.f; xi = 1.f; break;
-      default: break;   // b, mubar and the per-token gates are not read by a state-only run
+      case kRq: xr = 1.f; break;
+      default: break;   // mubar and the per-token gates are not read by a state-only run
     }
     cr[idx] = xr;
-    ci[idx] = xi;
   }
 }
 
-// cu_seqlens of the extended problem (packed input): sequence s has 2 x 64 tokens per chunk
+// cu_seqlens of the mirrored problem (packed input): sequence s has 64 tokens per chunk
 __global__ void bwd_ext_cu_kernel(const int32_t* __restrict__ chunk_off, int num_seqs, int32_t* __restrict__ cu_ext) {
-  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i <= num_seqs; i += gridDim.x * blockDim.x) cu_ext[i] = 2 * C * chunk_off[i];
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i <= num_seqs; i += gridDim.x * blockDim.x) cu_ext[i] = C * chunk_off[i];
 }
 
 }  // namespace
@@ -149,8 +147,8 @@ cudaError_t launch_bwd_ext_cu(const Plan& fwd, int32_t* cu_ext, int* launches) {
 
 size_t bwd_prep_smem_bytes() { return (size_t)3 * C * L6 * 2 + (size_t)C * LT * 2; }
 
-cudaError_t launch_bwd_prep(const Plan& fwd, const void* q, const void* k, const void* d_o, void* k_ext, void* v_ext,
-                            float* coef_ext, void* T_ext, int* launches) {
+cudaError_t launch_bwd_prep(const Plan& fwd, const void* q, const void* k, const void* d_o, void* k_ext, void* q_ext,
+                            void* v_ext, void* do_ext, float* coef_ext, void* T_ext, int* launches) {
   PrepArgs a;
   a.g = fwd.geom;
   a.q = static_cast<const __nv_bfloat16*>(q);
@@ -163,6 +161,8 @@ cudaError_t launch_bwd_prep(const Plan& fwd, const void* q, const void* k, const
   a.scale = fwd.p.scale;
   a.k_ext = static_cast<__nv_bfloat16*>(k_ext);
   a.v_ext = static_cast<__nv_bfloat16*>(v_ext);
+  a.q_ext = static_cast<__nv_bfloat16*>(q_ext);
+  a.do_ext = static_cast<__nv_bfloat16*>(do_ext);
   a.coef_ext = coef_ext;
   a.T_ext = static_cast<__nv_bfloat16*>(T_ext);
   const size_t smem = bwd_prep_smem_bytes();

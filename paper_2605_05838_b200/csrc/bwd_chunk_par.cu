@@ -92,7 +92,7 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
   const int m0 = 32 * (warp & 1), n0 = 32 * (warp >> 1), n064 = 16 * (warp >> 1);   // the warp's block of a 64x128 / 64x64 result
   const uint8_t* imgS = a.fwd_states + ((size_t)slot * H + h) * 65536;
   const uint8_t* imgM = imgS + 32768;
-  const int e_real = 2 * slot0 + 2 * (nch - 1 - si.local);
+  const int e_real = slot0 + (nch - 1 - si.local);   // this chunk in the adjoint chain's mirrored order
   const uint8_t* imgdM = a.adj_states + ((size_t)e_real * H + h) * 65536;   // roles exchanged in the adjoint run
   const uint8_t* imgdS = imgdM + 32768;
   const float scale = a.scale;
@@ -208,7 +208,7 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
   };
 
   const float* vt_rows = a.fwd_vt + (((size_t)slot * C) * H + h) * kD;
-  const float* dr_rows = a.adj_dr + (((size_t)(e_real >> 1) * C) * H + h) * kD;
+  const float* dr_rows = a.adj_dr + (((size_t)e_real * C) * H + h) * kD;
   // ---- what this CTA fetches later (V~, dR), towards L2 now (one CTA per SM: nothing else hides the latency)
   {
     const int r = tid >> 2, part = (tid & 3) * 32;

@@ -120,7 +120,10 @@ struct ChainArgs {
   int end_scalars_in_rk;      // (abar_C, b_C, mubar_C) of a chunk are entries 0..2 of coefficient vector 6, not the
                               // last entries of vectors 0, 1, 5 (the adjoint chain decouples them)
   float* vt_dump;             // NULL, or [chunk slot][64][H][dv] fp32: V~ of every chunk as EPI-2 reads it
-  int vt_dump_even_only;      // only the even chunk slots, written at slot / 2 (the adjoint chain: its real steps)
+  int inject;                 // state-only runs: a second rank-64 update of the pair per chunk, S^T += G_S^T Q,
+                              // M^T -= G_M^T Q with G_S = (-scale b) . G, G_M = (-scale g_M) . G (b, g_M: coefficient
+                              // vectors 1 and 4), G the [B,T,H,dv] bf16 tensor passed as `o`, Q the q tensor: the two Q
+                              // terms of the adjoint state recurrence
   uint32_t drop_lo;           // debug: bit 0 R, 1 V~_S/V~_M, 2 V~ (output), 3 W: leave that operand's lo part out
   long long* timeline;        // debug: CTA 0 writes clock64() at [chunk*32 + event] (NULL = off)
 };
@@ -313,7 +316,8 @@ __global__ void __launch_bounds__(Roles<token_groups(kLayer)>::kThreads, 1) chai
           const int tok0 = sq.tok0 + c * C;
           const int mat = (sq.slot0 + c) * H + h;
           // state-only runs need neither Q nor W, and the V = 0 runs no V either
-          mbar_arrive_expect_tx(fb, kTxBytes - (write_o ? 0u : kTxQW) - (v_zero ? kTxV : 0u));
+          const bool inj = kTrain && a.inject;   // Q and G (into the W area) instead of Q and W
+          mbar_arrive_expect_tx(fb, kTxBytes - ((write_o || inj) ? 0u : kTxQW) - (v_zero ? kTxV : 0u));
           tma_load_2d(st + kStK, &map_k, h * kD, tok0, fb);
           tma_load_2d(st + kStK + 8192, &map_k, h * kD + 64, tok0, fb);
           bulk_load(st + kStCoef, a.coef + (size_t)mat * MDN_NUM_COEF * C, kCoefBytes, fb);
@@ -324,6 +328,10 @@ __global__ void __launch_bounds__(Roles<token_groups(kLayer)>::kThreads, 1) chai
             tma_load_2d(st + kStQ + 8192, &map_q, h * kD + 64, tok0, fb);
             tma_load_2d(st + kStWh, &map_w, 0, mat * C, fb);
             tma_load_2d(st + kStWl, &map_w, 0, mat * C + (int)a.w_lo_row_offset, fb);
+          } else if (inj) {
+            tma_load_2d(st + kStQ, &map_q, h * kD, tok0, fb);
+            tma_load_2d(st + kStQ + 8192, &map_q, h * kD + 64, tok0, fb);
+            tma_load_2d(st + kStWh, &map_o, h * kD, tok0, fb);   // G: the tensor map of `o`, used for a load
           }
           MDN_MARK(c, kEvTmaIssued);
           issued = c + 1;
@@ -435,6 +443,17 @@ __global__ void __launch_bounds__(Roles<token_groups(kLayer)>::kThreads, 1) chai
           umma_ts(tmem + kColS, tmem + kColX + a_col(k >> 2, k & 3), dKmn + 128 * (k & 3), id128_mn, true);
         for (int k = 0; k < n3; ++k)
           umma_ts(tmem + kColM, tmem + kColY + a_col(k >> 2, k & 3), dKmn + 128 * (k & 3), id128_mn_neg, true);
+        if constexpr (kTrain) {
+          if (a.inject) {   // the second update, operands in Z, U (ready since the start of the chunk), Q read MN-major
+            const uint64_t dQmn = smem_desc_sw128(st + kStQ, 8192, 1024);
+            MDN_WAIT(b_v2, ph);
+            tc_fence_after_sync();
+            for (int k = 0; k < 8; ++k)
+              umma_ts(tmem + kColS, tmem + kColZ + a_col(k >> 2, k & 3), dQmn + 128 * (k & 3), id128_mn, true);
+            for (int k = 0; k < 8; ++k)
+              umma_ts(tmem + kColM, tmem + kColU + a_col(k >> 2, k & 3), dQmn + 128 * (k & 3), id128_mn_neg, true);
+          }
+        }
         umma_commit(b_m3);
         if (!write_o) continue;   // state-only run: no output terms
         // ---- MMA-3': U = V~^T W^T  with  V~ = hi + lo, W = hi + lo (lo*lo dropped)
@@ -686,6 +705,33 @@ __global__ void __launch_bounds__(Roles<token_groups(kLayer)>::kThreads, 1) chai
       const uint8_t* stg = smem + kOffStage + (c & 1) * kStageBytes;
       const float* cf = reinterpret_cast<const float*>(stg + kStCoef);
       const __nv_bfloat16* sV = reinterpret_cast<const __nv_bfloat16*>(stg + kStV);
+      if constexpr (kTrain) {
+        if (a.inject) {
+          // operands of the second update: they depend on nothing the chain computes, so they are made here, while
+          // MMA-1a runs.  Z, U are free in a state-only run; the previous chunk's MMA-3 (waited for in P) was their
+          // last reader.
+          const __nv_bfloat16* sG = reinterpret_cast<const __nv_bfloat16*>(stg + kStWh);
+          float gv[kTok];
+#pragma unroll
+          for (int j = 0; j < kTok; ++j) gv[j] = __bfloat162float(sG[(r0 + j) * kD + d]);
+#pragma unroll
+          for (int which = 0; which < 2; ++which) {
+            uint32_t oh[kPk], ol[kPk];
+            const float* vecp = cf + (which ? kGM : kB) * C + r0;
+#pragma unroll
+            for (int j = 0; j < kTok; j += 4) {
+              const float4 w4 = *reinterpret_cast<const float4*>(vecp + j);
+              split_pack_bf16(-a.scale * w4.x * gv[j], -a.scale * w4.y * gv[j + 1], oh[j >> 1], ol[j >> 1]);
+              split_pack_bf16(-a.scale * w4.z * gv[j + 2], -a.scale * w4.w * gv[j + 3], oh[(j >> 1) + 1], ol[(j >> 1) + 1]);
+            }
+            tmem_st_n<kPk>(tl + (which ? kColU : kColZ) + r0, oh);
+            tmem_st_n<kPk>(tl + (which ? kColU : kColZ) + r0 + kPk, ol);
+          }
+          tmem_wait_st();
+          tc_fence_before_sync();
+          MDN_WARP_ARRIVE(b_v2);
+        }
+      }
       // ---------------- EPI-1: R^T = V^T - abar .* X + (alpha b^-) .* Y  -> bf16 hi, lo in X
       {
         // V and the coefficients do not depend on the MMA: fetch them while MMA-1a runs
@@ -856,9 +902,8 @@ __global__ void __launch_bounds__(Roles<token_groups(kLayer)>::kThreads, 1) chai
         }
         MDN_MARK(c, kEvV2Arrive);
         if constexpr (kTrain) {   // off the chain's critical path: MMA-3 is running
-          int slot_c = sq.slot0 + c;
-          if (a.vt_dump != nullptr && !(a.vt_dump_even_only && (slot_c & 1))) {
-            if (a.vt_dump_even_only) slot_c >>= 1;
+          const int slot_c = sq.slot0 + c;
+          if (a.vt_dump != nullptr) {
             const int live = min(C, sq.len - c * C) - r0;   // this thread's tokens inside the chunk
             float* dst = a.vt_dump + (((size_t)slot_c * C + r0) * H + h) * kD + d;
             const size_t stride = (size_t)H * kD;
@@ -927,7 +972,7 @@ cudaError_t launch_chain_tensor(const Plan& pl, const void* q, const void* k, co
   const char* tl = getenv("MDN_DEBUG_TIMELINE");   // device address of an int64 buffer, [chunks][32]
   a.timeline = tl ? reinterpret_cast<long long*>(strtoull(tl, nullptr, 0)) : nullptr;
   a.dump = pl.chain_dump; a.state_only = pl.chain_state_only; a.end_scalars_in_rk = pl.chain_end_scalars_in_rk;
-  a.vt_dump = pl.chain_vt_dump; a.vt_dump_even_only = pl.chain_vt_dump_even_only;
+  a.vt_dump = pl.chain_vt_dump; a.inject = pl.chain_inject;
   a.seg_G = 0; a.seg_phase = 0;
   a.seg_E = a.seg_Psi = a.seg_PhiS = a.seg_PhiM = nullptr;
   const unsigned chains = (unsigned)pl.geom.num_seqs * p.H;
@@ -942,7 +987,8 @@ cudaError_t launch_chain_tensor(const Plan& pl, const void* q, const void* k, co
     return e;
   };
   auto launch = [&](unsigned grid) -> cudaError_t {
-    const bool train = a.dump != nullptr || a.state_only || a.end_scalars_in_rk || a.vt_dump != nullptr;
+    const bool train = a.dump != nullptr || a.state_only || a.end_scalars_in_rk || a.vt_dump != nullptr || a.inject;
+    if (a.inject && !a.state_only) return cudaErrorInvalidValue;
     if (train) {   // plain forward with the training options (no layer operations there)
       if (layer) return cudaErrorInvalidValue;
       return p.o_dtype == MDN_BF16 ? launch_as(chain_tensor_kernel<__nv_bfloat16, false, true>, grid)

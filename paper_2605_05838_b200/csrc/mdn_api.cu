@@ -196,7 +196,7 @@ mdn_status mdn_chunk_fwd(const mdn_params* p, const void* q, const void* k, cons
 // ---- the forward that keeps the chunk-start states (tensor path, serial chain)
 // Per (chunk slot, head): the bf16 state images S_b^T | M_b^T (2 x 32 KB), and behind all of them V~ of every chunk
 // slot as fp32 [slot][64][H][dv] (32 KB per slot and head).  The adjoint chain's buffer has the same two parts, with
-// dR = T^T dV~ (the V~ of its real steps) at half the extended slot index.
+// dR = T^T dV~ in the place of V~.
 constexpr uint64_t kStateImageBytes = 65536, kVtSlotBytes = 64 * 128 * 4;
 size_t mdn_chunk_states_bytes(const mdn_params* p) {
   mdn_ws_layout lay;
@@ -227,9 +227,9 @@ mdn_status mdn_chunk_fwd_keep_states(const mdn_params* p, const void* q, const v
 
 // ---- chunk-parallel backward, stage 1: the adjoint of the inter-chunk state recurrence
 struct AdjLayout {
-  mdn_params pe; mdn_ws_layout le; uint64_t k_ext, v_ext, ws_ext, cu_ext, total;
+  mdn_params pe; mdn_ws_layout le; uint64_t k_ext, q_ext, v_ext, do_ext, ws_ext, cu_ext, total;
   uint64_t image_bytes() const { return (uint64_t)le.num_slots * pe.H * kStateImageBytes; }
-  uint64_t states_bytes() const { return image_bytes() + (uint64_t)((le.num_slots + 1) / 2) * pe.H * kVtSlotBytes; }
+  uint64_t states_bytes() const { return image_bytes() + (uint64_t)le.num_slots * pe.H * kVtSlotBytes; }
 };
 
 static mdn_status adj_layout(const mdn_params* p, AdjLayout* a) {
@@ -239,23 +239,24 @@ static mdn_status adj_layout(const mdn_params* p, AdjLayout* a) {
   a->pe = *p;
   a->pe.segments = 1;
   a->pe.path = MDN_PATH_TENSOR;
-  if (p->num_seqs > 0) {   // packed: every chunk slot of the forward, padded to 64 rows, twice (host-side bound)
+  if (p->num_seqs > 0) {   // packed: every chunk slot of the forward, padded to 64 rows (host-side bound)
     mdn_params pf = *p;
     pf.segments = 1;
     mdn_ws_layout lf;
     st = make_layout(pf, &lf);
     if (st != MDN_OK) return st;
     a->pe.B = 1;
-    a->pe.T = 2 * p->chunk * (int)lf.num_slots;
+    a->pe.T = p->chunk * (int)lf.num_slots;
   } else {
-    a->pe.T = 2 * ((p->T + p->chunk - 1) / p->chunk) * p->chunk;   // a real and an injection step per chunk
+    a->pe.T = ((p->T + p->chunk - 1) / p->chunk) * p->chunk;   // short chunks padded to 64 rows
   }
   st = make_layout(a->pe, &a->le);
   if (st != MDN_OK) return st;
   const uint64_t rows = (uint64_t)a->pe.B * a->pe.T * p->H * p->dk * 2;
   uint64_t off = 0;
   auto take = [&](uint64_t bytes) { uint64_t at = off; off = align_up(off + bytes, 1024); return at; };
-  a->k_ext = take(rows); a->v_ext = take(rows); a->ws_ext = take(a->le.total_bytes);
+  a->k_ext = take(rows); a->q_ext = take(rows); a->v_ext = take(rows); a->do_ext = take(rows);
+  a->ws_ext = take(a->le.total_bytes);
   a->cu_ext = take((uint64_t)(p->num_seqs + 1) * 4); a->total = off;
   return MDN_OK;
 }
@@ -294,22 +295,22 @@ mdn_status mdn_bwd_state_chain(const mdn_params* p, const void* q, const void* k
   if (st != MDN_OK) return st;
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   if (cudaMemsetAsync(ext.ws + ext.lay.off_status, 0, 16, s) != cudaSuccess) return MDN_ERR_CUDA;
-  if (cu_ext) {   // the chunk map of the extended problem: 2 x 64 tokens per chunk of every sequence
+  if (cu_ext) {   // the chunk map of the mirrored problem: 64 tokens per chunk of every sequence
     ext.cu_total_may_be_short = 1;
     if (launch_bwd_ext_cu(fwd, cu_ext, &t_last_launches) != cudaSuccess || launch_chunk_map(ext, &t_last_launches) != cudaSuccess)
       return MDN_ERR_CUDA;
   }
-  cudaError_t e = launch_bwd_prep(fwd, q, k, d_o, w + al.k_ext, w + al.v_ext,
+  cudaError_t e = launch_bwd_prep(fwd, q, k, d_o, w + al.k_ext, w + al.q_ext, w + al.v_ext, w + al.do_ext,
                                   reinterpret_cast<float*>(ext.ws + ext.lay.off_coef), ext.ws + ext.lay.off_T,
                                   &t_last_launches);
   if (e != cudaSuccess) { t_last_cuda_error = (int)e; return MDN_ERR_CUDA; }
   // the forward's chain kernel on the extended problem, roles exchanged: its "S" is dM, its "M" is dS
   ext.chain_dump = static_cast<uint8_t*>(adjoint_states);
   ext.chain_vt_dump = reinterpret_cast<float*>(ext.chain_dump + al.image_bytes());
-  ext.chain_vt_dump_even_only = 1;
+  ext.chain_inject = 1;   // the two Q terms: q and dO (passed in the place of o) give a second update per chunk
   ext.chain_state_only = 1;
   ext.chain_end_scalars_in_rk = 1;
-  e = launch_chain_tensor(ext, w + al.k_ext, w + al.k_ext, w + al.v_ext, d_final_M, d_final_S, w + al.v_ext,
+  e = launch_chain_tensor(ext, w + al.q_ext, w + al.k_ext, w + al.v_ext, d_final_M, d_final_S, w + al.do_ext,
                           d_initial_M, d_initial_S, &t_last_launches);
   if (e != cudaSuccess) { t_last_cuda_error = (int)e; return MDN_ERR_CUDA; }
   return MDN_OK;

@@ -143,7 +143,7 @@ struct Plan {
   int chain_state_only = 0;
   int chain_end_scalars_in_rk = 0;
   float* chain_vt_dump = nullptr;        // V~ per chunk slot, fp32 [slot][64][H][dv]
-  int chain_vt_dump_even_only = 0;
+  int chain_inject = 0;                  // second update per chunk from q and the tensor passed as o (adjoint chain)
   int cu_total_may_be_short = 0;   // packed: cu[N] <= T instead of == T (the adjoint chain's padded problem)
 };
 
@@ -151,16 +151,16 @@ struct Plan {
 // the number of kernels it enqueued to *launches.
 cudaError_t launch_chunk_map(const Plan& pl, int* launches);
 // bwd_chunk_par.cu: gradients of q, k, v and the gates per (chunk, head) from the kept states and the adjoint states
-// (state images per chunk slot; fwd_vt = V~, adj_dr = dR per chunk slot as fp32 [slot][64][H][dv], adj_* indexed by the
-// adjoint chain's extended slots: images at 2 e, dR at e)
+// (state images per chunk slot; fwd_vt = V~, adj_dr = dR per chunk slot as fp32 [slot][64][H][dv]; adj_* in the adjoint
+// chain's mirrored order: chunk c of a sequence with n chunks at the sequence's slot n - 1 - c)
 cudaError_t launch_bwd_chunk_par(const Plan& fwd, const void* q, const void* k, const void* d_o, const float* beta,
                                  const float* log_alpha, const float* log_mu, const float* eta, const void* fwd_states,
                                  const float* fwd_vt, const void* adj_states, const float* adj_dr, float* dq, float* dk,
                                  float* dv, float* dbeta, float* dlog_alpha, float* dlog_mu, float* deta, int* launches);
 // bwd_chunk.cu: builds the extended problem of the adjoint state chain from the forward's workspace
 cudaError_t launch_bwd_ext_cu(const Plan& fwd, int32_t* cu_ext, int* launches);
-cudaError_t launch_bwd_prep(const Plan& fwd, const void* q, const void* k, const void* d_o, void* k_ext, void* v_ext,
-                            float* coef_ext, void* T_ext, int* launches);
+cudaError_t launch_bwd_prep(const Plan& fwd, const void* q, const void* k, const void* d_o, void* k_ext, void* q_ext,
+                            void* v_ext, void* do_ext, float* coef_ext, void* T_ext, int* launches);
 cudaError_t launch_coeff_scan(const Plan& pl, const float* beta, const float* log_alpha,
                               const float* log_mu, const float* eta, int* launches);
 // The layer operations as passes of their own (layer_ops.cu).

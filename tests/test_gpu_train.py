@@ -111,7 +111,7 @@ def test_bwd_state_chain(mdn, T, with_final):
     adj, dS0, dM0 = mdn.bwd_state_chain(t["q"], t["k"], dev(d_o, torch.bfloat16), ws, v_dim=w.dv, d_final_S=dev(dSf),
                                         d_final_M=dev(dMf), scale=inp["scale"])
     torch.cuda.synchronize()
-    dM_e, dS_e = mdn.unpack_chunk_states(adj, w.H, adjoint=True)       # entries: first half = dM, second half = dS
+    dM_e, dS_e = mdn.unpack_chunk_states(adj, w.H)       # entries: first half = dM, second half = dS
     dM_e, dS_e = dM_e.cpu().numpy(), dS_e.cpu().numpy()
     nch = (T + 63) // 64
     ref_S, ref_M, got_S, got_M = [], [], [], []
@@ -124,7 +124,7 @@ def test_bwd_state_chain(mdn, T, with_final):
                                   dS_final=None if dSf is None else dSf[b, h], dM_final=None if dMf is None else dMf[b, h])
             ref_S0[b, h], ref_M0[b, h] = g["dS0"], g["dM0"]
             for c in range(nch):
-                e = b * 2 * nch + 2 * (nch - 1 - c)
+                e = b * nch + (nch - 1 - c)       # a sequence's chunks lie in reverse order
                 ref_S.append(g["adj_end"][c][0]); ref_M.append(g["adj_end"][c][1])
                 got_S.append(dS_e[e, h]); got_M.append(dM_e[e, h])
     ref_S, ref_M, got_S, got_M = map(np.stack, (ref_S, ref_M, got_S, got_M))
