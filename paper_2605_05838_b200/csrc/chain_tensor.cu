@@ -434,17 +434,10 @@ __global__ void __launch_bounds__(Roles<token_groups(kLayer)>::kThreads, 1) chai
         } else {
           if (write_o && qk_on) MDN_MMA_1B(true);
         }
-        // ---- MMA-3: S^T += V~_S^T K, M^T -= V~_M^T K   (K tile read MN-major: N = dk, K = tokens)
-        MDN_WAIT(b_v1, ph);
-        tc_fence_after_sync();
-        MDN_MARK(c, kEvVSeen);
-        const int n3 = (a.drop_lo & 2u) ? 4 : 8;
-        for (int k = 0; k < n3; ++k)
-          umma_ts(tmem + kColS, tmem + kColX + a_col(k >> 2, k & 3), dKmn + 128 * (k & 3), id128_mn, true);
-        for (int k = 0; k < n3; ++k)
-          umma_ts(tmem + kColM, tmem + kColY + a_col(k >> 2, k & 3), dKmn + 128 * (k & 3), id128_mn_neg, true);
         if constexpr (kTrain) {
-          if (a.inject) {   // the second update, operands in Z, U (ready since the start of the chunk), Q read MN-major
+          if (a.inject) {
+            // the second update (operands in Z, U and the pre-scaled masters ready since the start of the chunk, Q
+            // read MN-major) needs nothing of this chunk's V~: issued here it runs while EPI-2 works, before MMA-3
             const uint64_t dQmn = smem_desc_sw128(st + kStQ, 8192, 1024);
             MDN_WAIT(b_v2, ph);
             tc_fence_after_sync();
@@ -454,6 +447,15 @@ __global__ void __launch_bounds__(Roles<token_groups(kLayer)>::kThreads, 1) chai
               umma_ts(tmem + kColM, tmem + kColU + a_col(k >> 2, k & 3), dQmn + 128 * (k & 3), id128_mn_neg, true);
           }
         }
+        // ---- MMA-3: S^T += V~_S^T K, M^T -= V~_M^T K   (K tile read MN-major: N = dk, K = tokens)
+        MDN_WAIT(b_v1, ph);
+        tc_fence_after_sync();
+        MDN_MARK(c, kEvVSeen);
+        const int n3 = (a.drop_lo & 2u) ? 4 : 8;
+        for (int k = 0; k < n3; ++k)
+          umma_ts(tmem + kColS, tmem + kColX + a_col(k >> 2, k & 3), dKmn + 128 * (k & 3), id128_mn, true);
+        for (int k = 0; k < n3; ++k)
+          umma_ts(tmem + kColM, tmem + kColY + a_col(k >> 2, k & 3), dKmn + 128 * (k & 3), id128_mn_neg, true);
         umma_commit(b_m3);
         if (!write_o) continue;   // state-only run: no output terms
         // ---- MMA-3': U = V~^T W^T  with  V~ = hi + lo, W = hi + lo (lo*lo dropped)
