@@ -11,9 +11,10 @@
 //     dM = mubar_C dM' - b_C dS' + K^T (p . dR),   dS = abar_C dS' - K^T (abar . dR),
 // plus the two Q terms, a second rank-64 update of the pair: dM -= Q^T ((scale b) . dO), dS += Q^T ((scale abar) . dO).
 // So the adjoint chain is run by the forward's chain kernel itself (chain_tensor.cu, training instantiation with the
-// second update switched on) on a "mirrored" problem built here: the chunks of every sequence in REVERSE order,
-// short chunks padded to 64 rows.  This file holds the kernel that builds that problem from the forward's workspace
-// (T, W, coefficient vectors) and q, k, dO.
+// second update switched on) on a "mirrored" problem: the chunks of every sequence in REVERSE order, short chunks
+// padded to 64 rows.  q, k and dO are read in place (the chain kernel mirrors the chunk index itself; rows past a
+// short chunk's end meet zero coefficients); this file holds the kernel that builds the rest of that problem (W^T dO,
+// T^T, the coefficient vectors) from the forward's workspace.
 #include "mdn_common.cuh"
 #include "tc_utils.cuh"
 #include "warp_mma.cuh"
@@ -30,14 +31,14 @@ constexpr int L6 = C + 8;     // ... of a 64 x 64 matrix
 
 struct PrepArgs {
   ChunkGeom g;                      // the forward's geometry (fixed length)
-  const __nv_bfloat16* q; const __nv_bfloat16* k; const __nv_bfloat16* d_o;
+  const __nv_bfloat16* d_o;
   const float* coef;                // forward: [slot][H][MDN_NUM_COEF][64]
   const __nv_bfloat16* T;           // forward: [slot][H][64][64]
   const __nv_bfloat16* W;           // forward: hi part, lo part w_lo_offset elements later
   size_t w_lo_offset;
   float scale;
-  // the mirrored problem: sequence s = rows [chunk_off[s] * 64, ..) of k_ext, q_ext, v_ext, do_ext
-  __nv_bfloat16* k_ext; __nv_bfloat16* q_ext; __nv_bfloat16* v_ext; __nv_bfloat16* do_ext;   // [slots 64][H][128]
+  // the mirrored problem: sequence s = rows [chunk_off[s] * 64, ..) of v_ext
+  __nv_bfloat16* v_ext;             // [slots 64][H][128]
   float* coef_ext;                  // [slots][H][MDN_NUM_COEF][64]
   __nv_bfloat16* T_ext;             // [slots][H][64][64]
 };
@@ -58,7 +59,7 @@ __global__ void __launch_bounds__(kPrepThreads) bwd_prep_kernel(PrepArgs a) {
   const int e_real = slot0 + (nch - 1 - si.local);
   const size_t mat = ((size_t)slot * H + h) * C * C;
 
-  // ---- W (hi, lo), T and the dO tile into shared memory; dO also goes out in the mirrored order
+  // ---- W (hi, lo), T and the dO tile into shared memory
   for (int idx = tid; idx < C * 8; idx += kPrepThreads) {
     const int r = idx >> 3, c8 = (idx & 7) * 8;
     *reinterpret_cast<uint4*>(sWH + r * L6 + c8) = *reinterpret_cast<const uint4*>(a.W + mat + r * C + c8);
@@ -70,7 +71,6 @@ __global__ void __launch_bounds__(kPrepThreads) bwd_prep_kernel(PrepArgs a) {
     uint4 x = make_uint4(0u, 0u, 0u, 0u);
     if (r < si.n) x = *reinterpret_cast<const uint4*>(a.d_o + ((size_t)(si.tok0 + r) * H + h) * kD + c8);
     *reinterpret_cast<uint4*>(sDO + r * LT + c8) = x;
-    *reinterpret_cast<uint4*>(a.do_ext + ((size_t)(e_real * C + r) * H + h) * kD + c8) = x;
   }
   __syncthreads();
 
@@ -87,18 +87,6 @@ __global__ void __launch_bounds__(kPrepThreads) bwd_prep_kernel(PrepArgs a) {
       const uint32_t packed = i < si.n ? pack_bf16(Z[mt][nt][2 * hf], Z[mt][nt][2 * hf + 1]) : 0u;
       *reinterpret_cast<uint32_t*>(a.v_ext + ((size_t)(e_real * C + i) * H + h) * kD + c) = packed;
     });
-  }
-
-  // ---- k and q in the mirrored order; rows past the end of a short chunk are zero
-  for (int idx = tid; idx < C * (kD / 8); idx += kPrepThreads) {
-    const int r = idx >> 4, c8 = (idx & 15) * 8;
-    uint4 kv = make_uint4(0u, 0u, 0u, 0u), qv = kv;
-    if (r < si.n) {
-      kv = *reinterpret_cast<const uint4*>(a.k + ((size_t)(si.tok0 + r) * H + h) * kD + c8);
-      qv = *reinterpret_cast<const uint4*>(a.q + ((size_t)(si.tok0 + r) * H + h) * kD + c8);
-    }
-    *reinterpret_cast<uint4*>(a.k_ext + ((size_t)(e_real * C + r) * H + h) * kD + c8) = kv;
-    *reinterpret_cast<uint4*>(a.q_ext + ((size_t)(e_real * C + r) * H + h) * kD + c8) = qv;
   }
 
   // ---- T^T
@@ -147,22 +135,16 @@ cudaError_t launch_bwd_ext_cu(const Plan& fwd, int32_t* cu_ext, int* launches) {
 
 size_t bwd_prep_smem_bytes() { return (size_t)3 * C * L6 * 2 + (size_t)C * LT * 2; }
 
-cudaError_t launch_bwd_prep(const Plan& fwd, const void* q, const void* k, const void* d_o, void* k_ext, void* q_ext,
-                            void* v_ext, void* do_ext, float* coef_ext, void* T_ext, int* launches) {
+cudaError_t launch_bwd_prep(const Plan& fwd, const void* d_o, void* v_ext, float* coef_ext, void* T_ext, int* launches) {
   PrepArgs a;
   a.g = fwd.geom;
-  a.q = static_cast<const __nv_bfloat16*>(q);
-  a.k = static_cast<const __nv_bfloat16*>(k);
   a.d_o = static_cast<const __nv_bfloat16*>(d_o);
   a.coef = reinterpret_cast<const float*>(fwd.ws + fwd.lay.off_coef);
   a.T = reinterpret_cast<const __nv_bfloat16*>(fwd.ws + fwd.lay.off_T);
   a.W = reinterpret_cast<const __nv_bfloat16*>(fwd.ws + fwd.lay.off_W);
   a.w_lo_offset = (size_t)fwd.geom.num_slots * fwd.p.H * C * C;
   a.scale = fwd.p.scale;
-  a.k_ext = static_cast<__nv_bfloat16*>(k_ext);
   a.v_ext = static_cast<__nv_bfloat16*>(v_ext);
-  a.q_ext = static_cast<__nv_bfloat16*>(q_ext);
-  a.do_ext = static_cast<__nv_bfloat16*>(do_ext);
   a.coef_ext = coef_ext;
   a.T_ext = static_cast<__nv_bfloat16*>(T_ext);
   const size_t smem = bwd_prep_smem_bytes();

@@ -120,6 +120,9 @@ struct ChainArgs {
   int end_scalars_in_rk;      // (abar_C, b_C, mubar_C) of a chunk are entries 0..2 of coefficient vector 6, not the
                               // last entries of vectors 0, 1, 5 (the adjoint chain decouples them)
   float* vt_dump;             // NULL, or [chunk slot][64][H][dv] fp32: V~ of every chunk as EPI-2 reads it
+  int mirror;                 // with inject: q, k and G are the ORIGINAL tensors of a problem whose chunks this run walks
+  ChunkGeom mirror_g;         // in reverse order (geometry mirror_g): chunk c of this run reads the rows of original
+                              // chunk nchunks - 1 - c; rows past a short chunk's end meet zero coefficients
   int inject;                 // state-only runs: a second rank-64 update of the pair per chunk, S^T += G_S^T Q,
                               // M^T -= G_M^T Q with G_S = (-scale b) . G, G_M = (-scale g_M) . G (b, g_M: coefficient
                               // vectors 1 and 4), G the [B,T,H,dv] bf16 tensor passed as `o`, Q the q tensor: the two Q
@@ -317,9 +320,11 @@ __global__ void __launch_bounds__(Roles<token_groups(kLayer)>::kThreads, 1) chai
           const int mat = (sq.slot0 + c) * H + h;
           // state-only runs need neither Q nor W, and the V = 0 runs no V either
           const bool inj = kTrain && a.inject;   // Q and G (into the W area) instead of Q and W
+          int tok0k = tok0;                      // rows of k, q, G
+          if (kTrain && a.mirror) tok0k = seq_info(a.mirror_g, seq).tok0 + (nch - 1 - c) * C;
           mbar_arrive_expect_tx(fb, kTxBytes - ((write_o || inj) ? 0u : kTxQW) - (v_zero ? kTxV : 0u));
-          tma_load_2d(st + kStK, &map_k, h * kD, tok0, fb);
-          tma_load_2d(st + kStK + 8192, &map_k, h * kD + 64, tok0, fb);
+          tma_load_2d(st + kStK, &map_k, h * kD, tok0k, fb);
+          tma_load_2d(st + kStK + 8192, &map_k, h * kD + 64, tok0k, fb);
           bulk_load(st + kStCoef, a.coef + (size_t)mat * MDN_NUM_COEF * C, kCoefBytes, fb);
           if (!v_zero) tma_load_2d(st + kStV, &map_v, h * kD, tok0, fb);
           tma_load_2d(st + kStT, &map_t, 0, mat * C, fb);
@@ -329,9 +334,9 @@ __global__ void __launch_bounds__(Roles<token_groups(kLayer)>::kThreads, 1) chai
             tma_load_2d(st + kStWh, &map_w, 0, mat * C, fb);
             tma_load_2d(st + kStWl, &map_w, 0, mat * C + (int)a.w_lo_row_offset, fb);
           } else if (inj) {
-            tma_load_2d(st + kStQ, &map_q, h * kD, tok0, fb);
-            tma_load_2d(st + kStQ + 8192, &map_q, h * kD + 64, tok0, fb);
-            tma_load_2d(st + kStWh, &map_o, h * kD, tok0, fb);   // G: the tensor map of `o`, used for a load
+            tma_load_2d(st + kStQ, &map_q, h * kD, tok0k, fb);
+            tma_load_2d(st + kStQ + 8192, &map_q, h * kD + 64, tok0k, fb);
+            tma_load_2d(st + kStWh, &map_o, h * kD, tok0k, fb);   // G: the tensor map of `o`, used for a load
           }
           MDN_MARK(c, kEvTmaIssued);
           issued = c + 1;
@@ -948,17 +953,19 @@ cudaError_t launch_chain_tensor(const Plan& pl, const void* q, const void* k, co
                                 const float* M0, void* o, float* Sf, float* Mf, int* launches) {
   const mdn_params& p = pl.p;
   const uint64_t tokens = (uint64_t)p.B * p.T;
+  // mirrored run: q, k, o are another problem's tensors (its geometry in chain_mirror_geom)
+  const uint64_t tokens_qko = pl.chain_mirror_geom ? (uint64_t)pl.chain_mirror_geom->B * pl.chain_mirror_geom->T : tokens;
   const uint64_t mats = (uint64_t)pl.geom.num_slots * p.H;
   CUtensorMap mq, mk, mv, mt, mw, mo;
   const uint64_t row = (uint64_t)p.H * kD;
-  if (!encode_tma_2d_bf16(&mq, TmaMap2D{q, row, tokens, row * 2, 64, 64, true}) ||
-      !encode_tma_2d_bf16(&mk, TmaMap2D{k, row, tokens, row * 2, 64, 64, true}) ||
+  if (!encode_tma_2d_bf16(&mq, TmaMap2D{q, row, tokens_qko, row * 2, 64, 64, true}) ||
+      !encode_tma_2d_bf16(&mk, TmaMap2D{k, row, tokens_qko, row * 2, 64, 64, true}) ||
       !encode_tma_2d_bf16(&mv, TmaMap2D{v, row, tokens, row * 2, 128, 64, false}) ||
       !encode_tma_2d_bf16(&mt, TmaMap2D{pl.ws + pl.lay.off_T, 64, mats * C, 128, 64, 64, true}) ||
       !encode_tma_2d_bf16(&mw, TmaMap2D{pl.ws + pl.lay.off_W, 64, 2 * mats * C, 128, 64, 64, true}))
     return cudaErrorInvalidValue;
   const bool o_bf16 = p.o_dtype == MDN_BF16;
-  if (!encode_tma_2d(&mo, TmaMap2D{o, row, tokens, row * (o_bf16 ? 2u : 4u), 128, 64, false}, !o_bf16))
+  if (!encode_tma_2d(&mo, TmaMap2D{o, row, tokens_qko, row * (o_bf16 ? 2u : 4u), 128, 64, false}, !o_bf16))
     return cudaErrorInvalidValue;
   ChainArgs a;
   a.qk_on = pl.qk.on; a.qk_d = pl.qk.d;
@@ -975,6 +982,8 @@ cudaError_t launch_chain_tensor(const Plan& pl, const void* q, const void* k, co
   a.timeline = tl ? reinterpret_cast<long long*>(strtoull(tl, nullptr, 0)) : nullptr;
   a.dump = pl.chain_dump; a.state_only = pl.chain_state_only; a.end_scalars_in_rk = pl.chain_end_scalars_in_rk;
   a.vt_dump = pl.chain_vt_dump; a.inject = pl.chain_inject;
+  a.mirror = pl.chain_mirror_geom != nullptr;
+  if (a.mirror) a.mirror_g = *pl.chain_mirror_geom; else a.mirror_g = pl.geom;
   a.seg_G = 0; a.seg_phase = 0;
   a.seg_E = a.seg_Psi = a.seg_PhiS = a.seg_PhiM = nullptr;
   const unsigned chains = (unsigned)pl.geom.num_seqs * p.H;
@@ -990,7 +999,7 @@ cudaError_t launch_chain_tensor(const Plan& pl, const void* q, const void* k, co
   };
   auto launch = [&](unsigned grid) -> cudaError_t {
     const bool train = a.dump != nullptr || a.state_only || a.end_scalars_in_rk || a.vt_dump != nullptr || a.inject;
-    if (a.inject && !a.state_only) return cudaErrorInvalidValue;
+    if ((a.inject && !a.state_only) || (a.mirror && !a.inject)) return cudaErrorInvalidValue;
     if (train) {   // plain forward with the training options (no layer operations there)
       if (layer) return cudaErrorInvalidValue;
       return p.o_dtype == MDN_BF16 ? launch_as(chain_tensor_kernel<__nv_bfloat16, false, true>, grid)

@@ -227,7 +227,7 @@ mdn_status mdn_chunk_fwd_keep_states(const mdn_params* p, const void* q, const v
 
 // ---- chunk-parallel backward, stage 1: the adjoint of the inter-chunk state recurrence
 struct AdjLayout {
-  mdn_params pe; mdn_ws_layout le; uint64_t k_ext, q_ext, v_ext, do_ext, ws_ext, cu_ext, total;
+  mdn_params pe; mdn_ws_layout le; uint64_t v_ext, ws_ext, cu_ext, total;
   uint64_t image_bytes() const { return (uint64_t)le.num_slots * pe.H * kStateImageBytes; }
   uint64_t states_bytes() const { return image_bytes() + (uint64_t)le.num_slots * pe.H * kVtSlotBytes; }
 };
@@ -255,8 +255,7 @@ static mdn_status adj_layout(const mdn_params* p, AdjLayout* a) {
   const uint64_t rows = (uint64_t)a->pe.B * a->pe.T * p->H * p->dk * 2;
   uint64_t off = 0;
   auto take = [&](uint64_t bytes) { uint64_t at = off; off = align_up(off + bytes, 1024); return at; };
-  a->k_ext = take(rows); a->q_ext = take(rows); a->v_ext = take(rows); a->do_ext = take(rows);
-  a->ws_ext = take(a->le.total_bytes);
+  a->v_ext = take(rows); a->ws_ext = take(a->le.total_bytes);
   a->cu_ext = take((uint64_t)(p->num_seqs + 1) * 4); a->total = off;
   return MDN_OK;
 }
@@ -300,18 +299,18 @@ mdn_status mdn_bwd_state_chain(const mdn_params* p, const void* q, const void* k
     if (launch_bwd_ext_cu(fwd, cu_ext, &t_last_launches) != cudaSuccess || launch_chunk_map(ext, &t_last_launches) != cudaSuccess)
       return MDN_ERR_CUDA;
   }
-  cudaError_t e = launch_bwd_prep(fwd, q, k, d_o, w + al.k_ext, w + al.q_ext, w + al.v_ext, w + al.do_ext,
-                                  reinterpret_cast<float*>(ext.ws + ext.lay.off_coef), ext.ws + ext.lay.off_T,
-                                  &t_last_launches);
+  cudaError_t e = launch_bwd_prep(fwd, d_o, w + al.v_ext, reinterpret_cast<float*>(ext.ws + ext.lay.off_coef),
+                                  ext.ws + ext.lay.off_T, &t_last_launches);
   if (e != cudaSuccess) { t_last_cuda_error = (int)e; return MDN_ERR_CUDA; }
   // the forward's chain kernel on the extended problem, roles exchanged: its "S" is dM, its "M" is dS
   ext.chain_dump = static_cast<uint8_t*>(adjoint_states);
   ext.chain_vt_dump = reinterpret_cast<float*>(ext.chain_dump + al.image_bytes());
   ext.chain_inject = 1;   // the two Q terms: q and dO (passed in the place of o) give a second update per chunk
+  ext.chain_mirror_geom = &fwd.geom;   // q, k, dO are read in place, chunk index mirrored
   ext.chain_state_only = 1;
   ext.chain_end_scalars_in_rk = 1;
-  e = launch_chain_tensor(ext, w + al.q_ext, w + al.k_ext, w + al.v_ext, d_final_M, d_final_S, w + al.do_ext,
-                          d_initial_M, d_initial_S, &t_last_launches);
+  e = launch_chain_tensor(ext, q, k, w + al.v_ext, d_final_M, d_final_S, const_cast<void*>(d_o), d_initial_M,
+                          d_initial_S, &t_last_launches);
   if (e != cudaSuccess) { t_last_cuda_error = (int)e; return MDN_ERR_CUDA; }
   return MDN_OK;
 }
