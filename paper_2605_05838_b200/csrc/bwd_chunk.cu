@@ -13,8 +13,8 @@
 // So the adjoint chain is run by the forward's chain kernel itself (chain_tensor.cu, training instantiation with the
 // second update switched on) on a "mirrored" problem: the chunks of every sequence in REVERSE order, short chunks
 // padded to 64 rows.  q, k and dO are read in place (the chain kernel mirrors the chunk index itself; rows past a
-// short chunk's end meet zero coefficients); this file holds the kernel that builds the rest of that problem (W^T dO,
-// T^T, the coefficient vectors) from the forward's workspace.
+// short chunk's end meet zero coefficients), and so is T (its tile is read transposed); this file holds the kernel
+// that builds the rest of that problem (W^T dO and the coefficient vectors) from the forward's workspace.
 #include "mdn_common.cuh"
 #include "tc_utils.cuh"
 #include "warp_mma.cuh"
@@ -33,22 +33,19 @@ struct PrepArgs {
   ChunkGeom g;                      // the forward's geometry (fixed length)
   const __nv_bfloat16* d_o;
   const float* coef;                // forward: [slot][H][MDN_NUM_COEF][64]
-  const __nv_bfloat16* T;           // forward: [slot][H][64][64]
   const __nv_bfloat16* W;           // forward: hi part, lo part w_lo_offset elements later
   size_t w_lo_offset;
   float scale;
   // the mirrored problem: sequence s = rows [chunk_off[s] * 64, ..) of v_ext
   __nv_bfloat16* v_ext;             // [slots 64][H][128]
   float* coef_ext;                  // [slots][H][MDN_NUM_COEF][64]
-  __nv_bfloat16* T_ext;             // [slots][H][64][64]
 };
 
 __global__ void __launch_bounds__(kPrepThreads) bwd_prep_kernel(PrepArgs a) {
   extern __shared__ __align__(16) uint8_t smem_raw[];
   __nv_bfloat16* sWH = reinterpret_cast<__nv_bfloat16*>(smem_raw);            // W hi, lo: [64][L6]
   __nv_bfloat16* sWL = sWH + C * L6;
-  __nv_bfloat16* Tt = sWL + C * L6;                                           // T: [64][L6]
-  __nv_bfloat16* sDO = Tt + C * L6;                                           // dO: [64][LT]
+  __nv_bfloat16* sDO = sWL + C * L6;                                          // dO: [64][LT]
   const int slot = blockIdx.x / a.g.H, h = blockIdx.x % a.g.H, H = a.g.H;
   const SlotInfo si = slot_info(a.g, slot);
   if (si.seq < 0) return;
@@ -59,12 +56,11 @@ __global__ void __launch_bounds__(kPrepThreads) bwd_prep_kernel(PrepArgs a) {
   const int e_real = slot0 + (nch - 1 - si.local);
   const size_t mat = ((size_t)slot * H + h) * C * C;
 
-  // ---- W (hi, lo), T and the dO tile into shared memory
+  // ---- W (hi, lo) and the dO tile into shared memory
   for (int idx = tid; idx < C * 8; idx += kPrepThreads) {
     const int r = idx >> 3, c8 = (idx & 7) * 8;
     *reinterpret_cast<uint4*>(sWH + r * L6 + c8) = *reinterpret_cast<const uint4*>(a.W + mat + r * C + c8);
     *reinterpret_cast<uint4*>(sWL + r * L6 + c8) = *reinterpret_cast<const uint4*>(a.W + a.w_lo_offset + mat + r * C + c8);
-    *reinterpret_cast<uint4*>(Tt + r * L6 + c8) = *reinterpret_cast<const uint4*>(a.T + mat + r * C + c8);
   }
   for (int idx = tid; idx < C * (kD / 8); idx += kPrepThreads) {
     const int r = idx >> 4, c8 = (idx & 15) * 8;
@@ -77,7 +73,7 @@ __global__ void __launch_bounds__(kPrepThreads) bwd_prep_kernel(PrepArgs a) {
   // ---- V' = W^T dO for the real step: a 64 x 128 result, one 32 x 32 block per warp, bf16 MMAs (W as hi + lo)
   {
     const uint32_t sb = smem_u32(smem_raw);
-    const Opnd oWH_t{sb, L6 * 2, true}, oWL_t{sb + C * L6 * 2, L6 * 2, true}, oDO_t{sb + 3 * C * L6 * 2, LT * 2, true};
+    const Opnd oWH_t{sb, L6 * 2, true}, oWL_t{sb + C * L6 * 2, L6 * 2, true}, oDO_t{sb + 2 * C * L6 * 2, LT * 2, true};
     const int m0 = 32 * (warp & 1), n0 = 32 * (warp >> 1);
     float Z[2][4][4];
     zero(Z);
@@ -87,13 +83,6 @@ __global__ void __launch_bounds__(kPrepThreads) bwd_prep_kernel(PrepArgs a) {
       const uint32_t packed = i < si.n ? pack_bf16(Z[mt][nt][2 * hf], Z[mt][nt][2 * hf + 1]) : 0u;
       *reinterpret_cast<uint32_t*>(a.v_ext + ((size_t)(e_real * C + i) * H + h) * kD + c) = packed;
     });
-  }
-
-  // ---- T^T
-  const size_t mat_r = ((size_t)e_real * H + h) * C * C;
-  for (int idx = tid; idx < C * C; idx += kPrepThreads) {
-    const int r = idx >> 6, i = idx & 63;
-    a.T_ext[mat_r + idx] = Tt[i * L6 + r];
   }
 
   // ---- coefficient vectors: abar' = g_M, p' = g_S, g_S' = p, g_M' = abar, end-of-chunk scalars (mubar_C, b_C,
@@ -133,20 +122,18 @@ cudaError_t launch_bwd_ext_cu(const Plan& fwd, int32_t* cu_ext, int* launches) {
   return cudaGetLastError();
 }
 
-size_t bwd_prep_smem_bytes() { return (size_t)3 * C * L6 * 2 + (size_t)C * LT * 2; }
+size_t bwd_prep_smem_bytes() { return (size_t)2 * C * L6 * 2 + (size_t)C * LT * 2; }
 
-cudaError_t launch_bwd_prep(const Plan& fwd, const void* d_o, void* v_ext, float* coef_ext, void* T_ext, int* launches) {
+cudaError_t launch_bwd_prep(const Plan& fwd, const void* d_o, void* v_ext, float* coef_ext, int* launches) {
   PrepArgs a;
   a.g = fwd.geom;
   a.d_o = static_cast<const __nv_bfloat16*>(d_o);
   a.coef = reinterpret_cast<const float*>(fwd.ws + fwd.lay.off_coef);
-  a.T = reinterpret_cast<const __nv_bfloat16*>(fwd.ws + fwd.lay.off_T);
   a.W = reinterpret_cast<const __nv_bfloat16*>(fwd.ws + fwd.lay.off_W);
   a.w_lo_offset = (size_t)fwd.geom.num_slots * fwd.p.H * C * C;
   a.scale = fwd.p.scale;
   a.v_ext = static_cast<__nv_bfloat16*>(v_ext);
   a.coef_ext = coef_ext;
-  a.T_ext = static_cast<__nv_bfloat16*>(T_ext);
   const size_t smem = bwd_prep_smem_bytes();
   cudaError_t e = cudaFuncSetAttribute(bwd_prep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;

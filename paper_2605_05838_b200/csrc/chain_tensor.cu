@@ -120,9 +120,10 @@ struct ChainArgs {
   int end_scalars_in_rk;      // (abar_C, b_C, mubar_C) of a chunk are entries 0..2 of coefficient vector 6, not the
                               // last entries of vectors 0, 1, 5 (the adjoint chain decouples them)
   float* vt_dump;             // NULL, or [chunk slot][64][H][dv] fp32: V~ of every chunk as EPI-2 reads it
-  int mirror;                 // with inject: q, k and G are the ORIGINAL tensors of a problem whose chunks this run walks
-  ChunkGeom mirror_g;         // in reverse order (geometry mirror_g): chunk c of this run reads the rows of original
-                              // chunk nchunks - 1 - c; rows past a short chunk's end meet zero coefficients
+  int mirror;                 // with inject: q, k, G and T are the ORIGINAL tensors of a problem whose chunks this run
+  ChunkGeom mirror_g;         // walks in reverse order (geometry mirror_g): chunk c of this run reads the rows of
+                              // original chunk nchunks - 1 - c (rows past a short chunk's end meet zero coefficients)
+                              // and uses that chunk's T transposed (the tile is read MN-major)
   int inject;                 // state-only runs: a second rank-64 update of the pair per chunk, S^T += G_S^T Q,
                               // M^T -= G_M^T Q with G_S = (-scale b) . G, G_M = (-scale g_M) . G (b, g_M: coefficient
                               // vectors 1 and 4), G the [B,T,H,dv] bf16 tensor passed as `o`, Q the q tensor: the two Q
@@ -321,13 +322,17 @@ __global__ void __launch_bounds__(Roles<token_groups(kLayer)>::kThreads, 1) chai
           // state-only runs need neither Q nor W, and the V = 0 runs no V either
           const bool inj = kTrain && a.inject;   // Q and G (into the W area) instead of Q and W
           int tok0k = tok0;                      // rows of k, q, G
-          if (kTrain && a.mirror) tok0k = seq_info(a.mirror_g, seq).tok0 + (nch - 1 - c) * C;
+          int mat_t = mat;                       // which T
+          if (kTrain && a.mirror) {
+            tok0k = seq_info(a.mirror_g, seq).tok0 + (nch - 1 - c) * C;
+            mat_t = (sq.slot0 + nch - 1 - c) * H + h;
+          }
           mbar_arrive_expect_tx(fb, kTxBytes - ((write_o || inj) ? 0u : kTxQW) - (v_zero ? kTxV : 0u));
           tma_load_2d(st + kStK, &map_k, h * kD, tok0k, fb);
           tma_load_2d(st + kStK + 8192, &map_k, h * kD + 64, tok0k, fb);
           bulk_load(st + kStCoef, a.coef + (size_t)mat * MDN_NUM_COEF * C, kCoefBytes, fb);
           if (!v_zero) tma_load_2d(st + kStV, &map_v, h * kD, tok0, fb);
-          tma_load_2d(st + kStT, &map_t, 0, mat * C, fb);
+          tma_load_2d(st + kStT, &map_t, 0, mat_t * C, fb);
           if (write_o) {
             tma_load_2d(st + kStQ, &map_q, h * kD, tok0, fb);
             tma_load_2d(st + kStQ + 8192, &map_q, h * kD + 64, tok0, fb);
@@ -419,11 +424,18 @@ __global__ void __launch_bounds__(Roles<token_groups(kLayer)>::kThreads, 1) chai
         MDN_WAIT(b_r, ph);
         tc_fence_after_sync();
         MDN_MARK(c, kEvRSeen);
+        if (kTrain && a.mirror) {   // T^T: the same tile read MN-major (16 rows = 2048 bytes per K step)
+          const uint64_t dTmn = smem_desc_sw128(st + kStT, 8192, 1024);
+          const uint32_t id64_mn = idesc_bf16(128, 64, false, true, false);
+          for (int k = 0; k < 8; ++k)
+            umma_ts(tmem + kColY, tmem + kColX + a_col(k >> 2, k & 3), dTmn + 128 * (k & 3), id64_mn, k > 0);
+        } else {
 #pragma unroll
-        for (int k = 0; k < 4; ++k) umma_ts(tmem + kColY, tmem + kColX + a_col(0, k), dT + 2 * k, id64, k > 0);
-        if (!(a.drop_lo & 1u)) {
+          for (int k = 0; k < 4; ++k) umma_ts(tmem + kColY, tmem + kColX + a_col(0, k), dT + 2 * k, id64, k > 0);
+          if (!(a.drop_lo & 1u)) {
 #pragma unroll
-          for (int k = 0; k < 4; ++k) umma_ts(tmem + kColY, tmem + kColX + a_col(1, k), dT + 2 * k, id64, true);
+            for (int k = 0; k < 4; ++k) umma_ts(tmem + kColY, tmem + kColX + a_col(1, k), dT + 2 * k, id64, true);
+          }
         }
         umma_commit(b_m2);
         // ... and U = M_b Q^T here: it fits under EPI-2 and is done before MMA-3 can start
@@ -961,7 +973,8 @@ cudaError_t launch_chain_tensor(const Plan& pl, const void* q, const void* k, co
   if (!encode_tma_2d_bf16(&mq, TmaMap2D{q, row, tokens_qko, row * 2, 64, 64, true}) ||
       !encode_tma_2d_bf16(&mk, TmaMap2D{k, row, tokens_qko, row * 2, 64, 64, true}) ||
       !encode_tma_2d_bf16(&mv, TmaMap2D{v, row, tokens, row * 2, 128, 64, false}) ||
-      !encode_tma_2d_bf16(&mt, TmaMap2D{pl.ws + pl.lay.off_T, 64, mats * C, 128, 64, 64, true}) ||
+      !encode_tma_2d_bf16(&mt, TmaMap2D{pl.chain_mirror_T ? pl.chain_mirror_T : pl.ws + pl.lay.off_T, 64, mats * C, 128, 64,
+                                        64, true}) ||
       !encode_tma_2d_bf16(&mw, TmaMap2D{pl.ws + pl.lay.off_W, 64, 2 * mats * C, 128, 64, 64, true}))
     return cudaErrorInvalidValue;
   const bool o_bf16 = p.o_dtype == MDN_BF16;

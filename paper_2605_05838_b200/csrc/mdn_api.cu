@@ -300,13 +300,14 @@ mdn_status mdn_bwd_state_chain(const mdn_params* p, const void* q, const void* k
       return MDN_ERR_CUDA;
   }
   cudaError_t e = launch_bwd_prep(fwd, d_o, w + al.v_ext, reinterpret_cast<float*>(ext.ws + ext.lay.off_coef),
-                                  ext.ws + ext.lay.off_T, &t_last_launches);
+                                  &t_last_launches);
   if (e != cudaSuccess) { t_last_cuda_error = (int)e; return MDN_ERR_CUDA; }
   // the forward's chain kernel on the extended problem, roles exchanged: its "S" is dM, its "M" is dS
   ext.chain_dump = static_cast<uint8_t*>(adjoint_states);
   ext.chain_vt_dump = reinterpret_cast<float*>(ext.chain_dump + al.image_bytes());
   ext.chain_inject = 1;   // the two Q terms: q and dO (passed in the place of o) give a second update per chunk
-  ext.chain_mirror_geom = &fwd.geom;   // q, k, dO are read in place, chunk index mirrored
+  ext.chain_mirror_geom = &fwd.geom;   // q, k, dO and T are read in place, chunk index mirrored
+  ext.chain_mirror_T = fwd.ws + fwd.lay.off_T;
   ext.chain_state_only = 1;
   ext.chain_end_scalars_in_rk = 1;
   e = launch_chain_tensor(ext, q, k, w + al.v_ext, d_final_M, d_final_S, const_cast<void*>(d_o), d_initial_M,

@@ -145,6 +145,7 @@ struct Plan {
   float* chain_vt_dump = nullptr;        // V~ per chunk slot, fp32 [slot][64][H][dv]
   int chain_inject = 0;                  // second update per chunk from q and the tensor passed as o (adjoint chain)
   const ChunkGeom* chain_mirror_geom = nullptr;   // q, k, o belong to this geometry, walked in reverse chunk order
+  const char* chain_mirror_T = nullptr;           // ... and T ([slot][H][64][64] bf16 of that problem), used transposed
   int cu_total_may_be_short = 0;   // packed: cu[N] <= T instead of == T (the adjoint chain's padded problem)
 };
 
@@ -160,7 +161,7 @@ cudaError_t launch_bwd_chunk_par(const Plan& fwd, const void* q, const void* k, 
                                  float* dv, float* dbeta, float* dlog_alpha, float* dlog_mu, float* deta, int* launches);
 // bwd_chunk.cu: builds the extended problem of the adjoint state chain from the forward's workspace
 cudaError_t launch_bwd_ext_cu(const Plan& fwd, int32_t* cu_ext, int* launches);
-cudaError_t launch_bwd_prep(const Plan& fwd, const void* d_o, void* v_ext, float* coef_ext, void* T_ext, int* launches);
+cudaError_t launch_bwd_prep(const Plan& fwd, const void* d_o, void* v_ext, float* coef_ext, int* launches);
 cudaError_t launch_coeff_scan(const Plan& pl, const float* beta, const float* log_alpha,
                               const float* log_mu, const float* eta, int* launches);
 // The layer operations as passes of their own (layer_ops.cu).
