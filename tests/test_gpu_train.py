@@ -244,6 +244,18 @@ def test_chunked_backward_packed(mdn):
     assert max(errs.values()) <= TOL_CHUNKED, errs
 
 
+def test_chunked_backward_tiny_sequences(mdn):
+    """Degenerate shapes: packed sequences of 1 to 70 tokens (most chunks short, many one-chunk sequences: the
+    adjoint chain reads q, k, dO past every short chunk's end) and a fixed-length batch shorter than one chunk."""
+    w = wl.Workload("chunked_tiny_packed", B=1, T=400, H=2, dk=128, dv=128, dtype="bf16", varlen=True, len_lo=1, len_hi=70,
+                    init_state_std=0.1, seed=101)
+    errs = chunked_vs_oracle(mdn, w, 31)
+    assert max(errs.values()) <= TOL_CHUNKED, errs
+    w = wl.Workload("chunked_T23", B=3, T=23, H=2, dk=128, dv=128, dtype="bf16", init_state_std=0.1, seed=102)
+    errs = chunked_vs_oracle(mdn, w, 32)
+    assert max(errs.values()) <= TOL_CHUNKED, errs
+
+
 def test_backward_from_saved_forward(mdn):
     """mdn_chunk_bwd_saved on the workspace and the chunk states a keep-states forward left behind: the same numbers
     as the self-contained call (which redoes that part of the forward without the output terms)."""
