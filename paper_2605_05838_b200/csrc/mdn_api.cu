@@ -302,7 +302,7 @@ mdn_status mdn_bwd_state_chain(const mdn_params* p, const void* q, const void* k
   cudaError_t e = launch_bwd_prep(fwd, d_o, w + al.v_ext, reinterpret_cast<float*>(ext.ws + ext.lay.off_coef),
                                   &t_last_launches);
   if (e != cudaSuccess) { t_last_cuda_error = (int)e; return MDN_ERR_CUDA; }
-  // the forward's chain kernel on the extended problem, roles exchanged: its "S" is dM, its "M" is dS
+  // the forward's chain kernel on the mirrored problem, roles exchanged: its "S" is dM, its "M" is dS
   ext.chain_dump = static_cast<uint8_t*>(adjoint_states);
   ext.chain_vt_dump = reinterpret_cast<float*>(ext.chain_dump + al.image_bytes());
   ext.chain_inject = 1;   // the two Q terms: q and dO (passed in the place of o) give a second update per chunk

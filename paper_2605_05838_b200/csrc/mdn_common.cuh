@@ -159,7 +159,7 @@ cudaError_t launch_bwd_chunk_par(const Plan& fwd, const void* q, const void* k, 
                                  const float* log_alpha, const float* log_mu, const float* eta, const void* fwd_states,
                                  const float* fwd_vt, const void* adj_states, const float* adj_dr, float* dq, float* dk,
                                  float* dv, float* dbeta, float* dlog_alpha, float* dlog_mu, float* deta, int* launches);
-// bwd_chunk.cu: builds the extended problem of the adjoint state chain from the forward's workspace
+// bwd_chunk.cu: W^T dO and the coefficient vectors of the adjoint state chain's mirrored problem, from the forward's workspace
 cudaError_t launch_bwd_ext_cu(const Plan& fwd, int32_t* cu_ext, int* launches);
 cudaError_t launch_bwd_prep(const Plan& fwd, const void* d_o, void* v_ext, float* coef_ext, int* launches);
 cudaError_t launch_coeff_scan(const Plan& pl, const float* beta, const float* log_alpha,
