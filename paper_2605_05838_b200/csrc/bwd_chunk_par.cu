@@ -50,6 +50,7 @@ static_assert(kD * LT * 2 == 2 * kTile, "a state and a hi + lo tile pair have th
 static_assert(2 * kTile >= 2 * kMatF && kD * LT * 2 >= 2 * kMatF && 2 * kTile >= 2 * kMat6, "overlays");
 static_assert(kSmem <= 232448, "shared memory");
 
+constexpr int kIssuer = kThreads - 32;   // the thread that issues the bulk copies
 constexpr int kBarSlot = 22;   // vector slot that holds the two mbarriers and the abort flag instead
 enum Vec : int { vAbar = 0, vB, vP, vGS, vGM, vMubar, vAlpha, vBeta, vMu, vEta, vBprev,
                  vdAbar, vdB, vdP, vdGS, vdGM, vdMubar, vdAlpha, vdBeta, vdMu, vdEta, vRed };
@@ -225,7 +226,7 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
   // All four states arrive at the start by cp.async (no registers in between); M is fetched a second time later.
   const uint32_t bar0 = smem_u32(vec + kBarSlot * C), bar1 = bar0 + 8;   // mbarriers: the four states; M again
   volatile int* abort_flag = reinterpret_cast<volatile int*>(vec + kBarSlot * C + 4);
-  if (tid == 0) {
+  if (tid == kIssuer) {   // a thread of the last warp: the first two warps have the vectors and gamma to set up
     *abort_flag = 0;
     mbar_init(bar0, 1);
     mbar_init(bar1, 1);
@@ -334,7 +335,7 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
     add_rowsum(G, sK, V(vdGS), 1.f);
   }
   __syncthreads();   // dS' has been read: M takes its place
-  if (tid == 0) {
+  if (tid == kIssuer) {
     fence_proxy_async_smem();
     mbar_arrive_expect_tx(bar1, 32768);
     load_state(imgM, kR2, bar1);
