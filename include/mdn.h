@@ -465,6 +465,8 @@ mdn_status mdn_set_stage_events(void* const* events /* host */, int32_t n);
  *   mode 2: out[128 x 64]  = a[128 x 64]  * b[64 x 64]^T      (A from tensor memory)
  *   mode 3: out[128 x 128] = 1 - a[128 x 64] * b[64 x 128]    (A from tensor memory, negated; B MN-major via TMA;
  *                                                              accumulating onto a preloaded D)
+ *   mode 4: M = 64: a[64 x 128] * b[128 x 128]^T from shared memory into tensor memory pre-filled with -777;
+ *           out[128 x 128] = all 128 lanes x 128 columns (shows which lanes the 64 rows of the result occupy)
  * a, b: bf16 row-major device buffers; out: float32 device buffer; status: device int32 (0 = ok).
  */
 mdn_status mdn_selftest_umma(int32_t mode, const void* a, const void* b, float* out, int32_t* status,

@@ -107,6 +107,40 @@ __global__ void __launch_bounds__(128) umma_probe_kernel(int mode, const __nv_bf
         for (int j = 0; j < 32; ++j) out[tid * 64 + c0 + j] = __uint_as_float(r[j]);
       }
     }
+  } else if (mode == 4) {     // SS with M = 64: D[64x128] = A[64x128] * B[128x128]^T; out = all 128 lanes x 128 columns
+    // tensor memory is filled with a sentinel first, so the lanes the 64 rows land in can be read off the result
+    {
+      uint32_t r[32];
+      for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(-777.0f);
+      for (int c0 = 0; c0 < 128; c0 += 32) tmem_st32(tmem + lane_base + c0, r);
+      tmem_wait_st();
+    }
+    fill_kmajor(sB, a, 64, 128, tid, 128);    // A: two [64 x 64] blocks (16 KB) in the smaller area
+    fill_kmajor(sA, b, 128, 128, tid, 128);   // B: two [128 x 64] blocks (32 KB)
+    fence_proxy_async_smem();
+    tc_fence_before_sync();
+    __syncthreads();
+    if (tid == 0) {
+      tc_fence_after_sync();
+      const uint32_t id = idesc_bf16(64, 128, false, false, false);
+      for (int k = 0; k < 8; ++k) {
+        const uint64_t da = smem_desc_sw128(smem_u32(sB) + (k / 4) * 8192 + (k % 4) * 32, 16, 1024);
+        const uint64_t db = smem_desc_sw128(smem_u32(sA) + (k / 4) * 16384 + (k % 4) * 32, 16, 1024);
+        umma_ss(tmem, da, db, id, k > 0);
+      }
+      umma_commit(bar_mma);
+    }
+    ok = mbar_wait(bar_mma, 0, &abort_flag);
+    __syncwarp();
+    tc_fence_after_sync();
+    if (ok) {
+      for (int c0 = 0; c0 < 128; c0 += 32) {
+        uint32_t r[32];
+        tmem_ld32(tmem + lane_base + c0, r);
+        tmem_wait_ld();
+        for (int j = 0; j < 32; ++j) out[tid * 128 + c0 + j] = __uint_as_float(r[j]);
+      }
+    }
   } else if (mode == 2 || mode == 3) {
     // A [128 x 64] bf16 -> TMEM columns 128..159, two elements per column (even k in the low half)
     {
@@ -190,7 +224,7 @@ __global__ void __launch_bounds__(128) umma_probe_kernel(int mode, const __nv_bf
 extern "C" mdn_status mdn_selftest_umma(int32_t mode, const void* a, const void* b, float* out, int32_t* status,
                                         void* cuda_stream) {
   using namespace mdn;
-  if (mode < 0 || mode > 3 || !a || !out || !status || (mode != 0 && !b)) return MDN_ERR_INVALID_ARG;
+  if (mode < 0 || mode > 4 || !a || !out || !status || (mode != 0 && !b)) return MDN_ERR_INVALID_ARG;
   CUtensorMap map;
   std::memset(&map, 0, sizeof(map));
   const void* tma_src = mode == 3 ? b : a;      // [64 x 128] bf16

@@ -63,3 +63,18 @@ def test_mma_tmem_a_mnmajor_b_negate_accumulate(mdn):
     out = run(mdn, 3, a, b, (128, 128))
     ref = 1.0 - a.float() @ b.float()
     assert (out - ref).abs().max() < 1e-3
+
+
+def test_mma_m64_data_path_layout(mdn):
+    """M = 64 (a 64-row product, e.g. the 64 tokens of a chunk as rows): row r of the result lies in tensor-memory
+    lane 32 (r // 16) + r % 16 - sixteen lanes of each 32-lane quarter - and the other lanes are left untouched."""
+    rng = np.random.default_rng(5)
+    a, b = bf16_mat(rng, (64, 128)), bf16_mat(rng, (128, 128))
+    out = run(mdn, 4, a, b, (128, 128)).numpy()
+    ref = (a.float() @ b.float().T).numpy()
+    for lane in range(128):
+        q, i = divmod(lane, 32)
+        if i < 16:
+            assert np.abs(out[lane] - ref[16 * q + i]).max() < 1e-3, lane
+        else:
+            assert np.all(out[lane] == -777.0), lane
