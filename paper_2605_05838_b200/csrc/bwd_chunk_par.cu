@@ -349,8 +349,9 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
   {
     float G[2][4][4];
     zero(G);
+    // dR enters these two products as its hi part alone: S and M are single bf16 values themselves, and the lo part
+    // changes no gradient's error (measured; V~ in the two products above does need its lo part)
     warp_mma(G, tile_mk(kR3), st_dv(kR0), kD, m0, n0, lane);
-    warp_mma(G, tile_mk(kR3 + kTile), st_dv(kR0), kD, m0, n0, lane);
     for_frag<2, 4>(m0, n0, g, t, [&](int mt, int nt, int e, int r, int c) { dK[mt][nt][e] -= V(vAbar)[r] * G[mt][nt][e]; });
     add_rowsum(G, sK, V(vdAbar), -1.f);
     {
@@ -362,7 +363,6 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
     }
     zero(G);
     warp_mma(G, tile_mk(kR3), st_dv(kR2), kD, m0, n0, lane);
-    warp_mma(G, tile_mk(kR3 + kTile), st_dv(kR2), kD, m0, n0, lane);
     for_frag<2, 4>(m0, n0, g, t, [&](int mt, int nt, int e, int r, int c) { dK[mt][nt][e] += V(vP)[r] * G[mt][nt][e]; });
     add_rowsum(G, sK, V(vdP), 1.f);
   }
