@@ -15,8 +15,10 @@
 // V~ and dR are not recomputed here: the two chain runs (the forward that keeps its states, the adjoint chain) have
 // both in their epilogues and leave them in global memory as fp32, so X, Y, R, T R, K dS', K dM' and T^T dV~ cost nothing.
 // Every product is a warp-level bf16 tensor-core MMA (m16n8k16, fp32 accumulate) fed by ldmatrix from shared memory:
-// q, k, dO and the states are bf16 as they stand; V~, dR and every intermediate that comes out of an accumulator (DW,
-// DA) is kept as a bf16 hi + lo pair (16 mantissa bits through two MMAs).  One 256-thread CTA per (chunk, head).
+// q, k, dO and the states are bf16 as they stand.  Of the operands that come out of an accumulator, V~ and DW are
+// bf16 hi + lo pairs (16 mantissa bits through two MMAs); dR and DA enter as single bf16 values: measured, their lo
+// parts change no gradient's error, while leaving out the lo part of V~ or DW does (dk 5e-2, dq 1.5x).
+// One 256-thread CTA per (chunk, head).
 #include "mdn_common.cuh"
 #include "tc_utils.cuh"
 #include "warp_mma.cuh"
@@ -40,7 +42,7 @@ constexpr uint32_t kOffK = kOffSt + kD * LT * 2;      // k, q, dO
 constexpr uint32_t kOffQ = kOffK + kTile;
 constexpr uint32_t kOffDO = kOffQ + kTile;
 constexpr uint32_t kOffVt = kOffDO + kTile;           // V~ hi, lo; later DW hi, lo
-constexpr uint32_t kOffDR = kOffVt + 2 * kTile;       // dR hi, lo; later DA hi, lo
+constexpr uint32_t kOffDR = kOffVt + 2 * kTile;       // dR; later DA
 constexpr uint32_t kOffTmp = kOffDR + 2 * kTile;      // dS', then M again; later gamma, m (fp32 [64][LG] each)
 constexpr uint32_t kOffVec = kOffTmp + 2 * kTile;     // vectors, 24 x [64] floats
 constexpr uint32_t kOffGam = kOffVec + 24 * C * 4;    // gamma, fp32 [64][LG]: built while the first loads are in flight
@@ -74,10 +76,9 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
   bf16* sQ = reinterpret_cast<bf16*>(smem + kOffQ);
   float* sGam = reinterpret_cast<float*>(smem + kOffGam);     // gamma (own place), m
   float* sMm = reinterpret_cast<float*>(smem + kR2);
-  bf16* sDWH = reinterpret_cast<bf16*>(smem + kR1);           // DW, DA (hi, lo)
+  bf16* sDWH = reinterpret_cast<bf16*>(smem + kR1);           // DW (hi, lo), DA
   bf16* sDWL = sDWH + C * L6;
   bf16* sDAH = reinterpret_cast<bf16*>(smem + kR3);
-  bf16* sDAL = sDAH + C * L6;
   float* sdGe = reinterpret_cast<float*>(smem + kR0);         // d Geta, d G^-
   float* sdGm = sdGe + C * LG;
   float* vec = reinterpret_cast<float*>(smem + kOffVec);
@@ -108,8 +109,7 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
   auto tile_mk = [&](uint32_t base) { return Opnd{sb + base, LT * 2, false}; };
   const Opnd oDWH{sb + kR1, L6 * 2, false}, oDWL{sb + kR1 + kMat6, L6 * 2, false};
   const Opnd oDWH_t{sb + kR1, L6 * 2, true}, oDWL_t{sb + kR1 + kMat6, L6 * 2, true};
-  const Opnd oDAH{sb + kR3, L6 * 2, false}, oDAL{sb + kR3 + kMat6, L6 * 2, false};
-  const Opnd oDAH_t{sb + kR3, L6 * 2, true}, oDAL_t{sb + kR3 + kMat6, L6 * 2, true};
+  const Opnd oDAH{sb + kR3, L6 * 2, false}, oDAH_t{sb + kR3, L6 * 2, true};
 
   auto tok = [&](int r) { return (size_t)(si.tok0 + r) * H + h; };
   // everything arrives by cp.async (no registers in between, nothing blocks until the wait); rows past the chunk's
@@ -131,8 +131,8 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
     }
   };
   // ... and from there, in place, to the bf16 hi + lo tiles the products read (every thread holds its 32 values across
-  // the barrier); `out`, if given, receives the fp32 values of the live rows (dv = dR)
-  auto split_in_place = [&](uint32_t base, float* out) {
+  // the barrier; with_lo = false: the hi tile only); `out`, if given, receives the fp32 values of the live rows (dv = dR)
+  auto split_in_place = [&](uint32_t base, float* out, bool with_lo) {
     float4 x[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) x[i] = *reinterpret_cast<const float4*>(smem + base + (tid + kThreads * i) * 16);
@@ -146,7 +146,7 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
       split_pack_bf16(x[i].x, x[i].y, ph.x, pl.x);
       split_pack_bf16(x[i].z, x[i].w, ph.y, pl.y);
       *reinterpret_cast<uint2*>(hi + r * LT + c4) = ph;
-      *reinterpret_cast<uint2*>(lo + r * LT + c4) = pl;
+      if (with_lo) *reinterpret_cast<uint2*>(lo + r * LT + c4) = pl;
       if (out != nullptr && r < n) *reinterpret_cast<float4*>(out + tok(r) * kD + c4) = x[i];
     }
   };
@@ -222,7 +222,7 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
   //   R0: S                                               | later d Geta, d G^-
   //   R1: M    | V~ (fp32, then hi, lo)                   | later DW (hi, lo), then two contribution matrices
   //   R2: dS'  | M again                                  | m
-  //   R3: dM'  | dR (fp32, then hi, lo)                   | DA (hi, lo), then a contribution matrix
+  //   R3: dM'  | dR (fp32, then bf16)                     | DA, then a contribution matrix
   // All four states arrive at the start by cp.async (no registers in between); M is fetched a second time later.
   const uint32_t bar0 = smem_u32(vec + kBarSlot * C), bar1 = bar0 + 8;   // mbarriers: the four states; M again
   volatile int* abort_flag = reinterpret_cast<volatile int*>(vec + kBarSlot * C + 4);
@@ -314,7 +314,7 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
   warp_mma(KK, oK, oK, kD, m0, n064, lane);
   cp_async_wait();
   __syncthreads();
-  split_in_place(kR1, nullptr);
+  split_in_place(kR1, nullptr, true);
   __syncthreads();
 
   // ---- phase 2: the g_M and g_S terms of dK from V~ dM'^T, V~ dS'^T; dR arrives under the second
@@ -342,7 +342,7 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
   }
   cp_async_wait();   // dR is in (M may still be on its way)
   __syncthreads();
-  split_in_place(kR3, a.dv);
+  split_in_place(kR3, a.dv, false);   // no product reads dR's lo part
   __syncthreads();
 
   // ---- phase 3: dR S^T (dK, d abar) while M arrives again, then dR M^T (dK, d p)
@@ -390,7 +390,6 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
   warp_mma(P1, oDO, tile_mk(kR1 + kTile), kD, m0, n064, lane);
   warp_mma(P2, tile_mk(kR3), tile_mk(kR1), kD, m0, n064, lane);               // dR V~^T
   warp_mma(P2, tile_mk(kR3), tile_mk(kR1 + kTile), kD, m0, n064, lane);
-  warp_mma(P2, tile_mk(kR3 + kTile), tile_mk(kR1), kD, m0, n064, lane);
   __syncthreads();   // V~, dR and S are no longer read; gamma, m complete
   for_pair<2, 2>(m0, n064, g, t, [&](int mt, int nt, int hf, int r, int i0) {
     float dw[2], da[2];
@@ -411,9 +410,7 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
     split_pack_bf16(dw[0], dw[1], ph, pl);
     *reinterpret_cast<uint32_t*>(sDWH + r * L6 + i0) = ph;
     *reinterpret_cast<uint32_t*>(sDWL + r * L6 + i0) = pl;
-    split_pack_bf16(da[0], da[1], ph, pl);
-    *reinterpret_cast<uint32_t*>(sDAH + r * L6 + i0) = ph;
-    *reinterpret_cast<uint32_t*>(sDAL + r * L6 + i0) = pl;
+    *reinterpret_cast<uint32_t*>(sDAH + r * L6 + i0) = pack_bf16(da[0], da[1]);
   });
   __syncthreads();
   // ---- dQ += DW K;  dK += DW^T Q + (DA + DA^T) K
@@ -422,9 +419,7 @@ __global__ void __launch_bounds__(kThreads, 1) bwd_chunk_par_kernel(ParArgs a) {
   warp_mma(dK, oDWH_t, oQ_t, C, m0, n0, lane);
   warp_mma(dK, oDWL_t, oQ_t, C, m0, n0, lane);
   warp_mma(dK, oDAH, oK_t, C, m0, n0, lane);
-  warp_mma(dK, oDAL, oK_t, C, m0, n0, lane);
   warp_mma(dK, oDAH_t, oK_t, C, m0, n0, lane);
-  warp_mma(dK, oDAL_t, oK_t, C, m0, n0, lane);
   for_pair<2, 4>(m0, n0, g, t, [&](int mt, int nt, int hf, int r, int c) {
     if (r < n) {
       *reinterpret_cast<float2*>(a.dq + tok(r) * kD + c) = make_float2(dQ[mt][nt][2 * hf], dQ[mt][nt][2 * hf + 1]);
