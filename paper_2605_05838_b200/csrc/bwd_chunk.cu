@@ -43,9 +43,7 @@ struct PrepArgs {
 
 __global__ void __launch_bounds__(kPrepThreads) bwd_prep_kernel(PrepArgs a) {
   extern __shared__ __align__(16) uint8_t smem_raw[];
-  __nv_bfloat16* sWH = reinterpret_cast<__nv_bfloat16*>(smem_raw);            // W hi, lo: [64][L6]
-  __nv_bfloat16* sWL = sWH + C * L6;
-  __nv_bfloat16* sDO = sWL + C * L6;                                          // dO: [64][LT]
+  // shared memory: W hi, W lo ([64][L6] each), then the dO tile ([64][LT])
   const int slot = blockIdx.x / a.g.H, h = blockIdx.x % a.g.H, H = a.g.H;
   const SlotInfo si = slot_info(a.g, slot);
   if (si.seq < 0) return;
@@ -56,33 +54,23 @@ __global__ void __launch_bounds__(kPrepThreads) bwd_prep_kernel(PrepArgs a) {
   const int e_real = slot0 + (nch - 1 - si.local);
   const size_t mat = ((size_t)slot * H + h) * C * C;
 
-  // ---- W (hi, lo) and the dO tile into shared memory
-  for (int idx = tid; idx < C * 8; idx += kPrepThreads) {
-    const int r = idx >> 3, c8 = (idx & 7) * 8;
-    *reinterpret_cast<uint4*>(sWH + r * L6 + c8) = *reinterpret_cast<const uint4*>(a.W + mat + r * C + c8);
-    *reinterpret_cast<uint4*>(sWL + r * L6 + c8) = *reinterpret_cast<const uint4*>(a.W + a.w_lo_offset + mat + r * C + c8);
-  }
-  for (int idx = tid; idx < C * (kD / 8); idx += kPrepThreads) {
-    const int r = idx >> 4, c8 = (idx & 15) * 8;
-    uint4 x = make_uint4(0u, 0u, 0u, 0u);
-    if (r < si.n) x = *reinterpret_cast<const uint4*>(a.d_o + ((size_t)(si.tok0 + r) * H + h) * kD + c8);
-    *reinterpret_cast<uint4*>(sDO + r * LT + c8) = x;
-  }
-  __syncthreads();
-
-  // ---- V' = W^T dO for the real step: a 64 x 128 result, one 32 x 32 block per warp, bf16 MMAs (W as hi + lo)
+  // ---- W (hi, lo) and the dO tile into shared memory by cp.async (rows past the chunk's end zero-filled); the
+  // coefficient vectors are remapped while the copies are in flight
   {
     const uint32_t sb = smem_u32(smem_raw);
-    const Opnd oWH_t{sb, L6 * 2, true}, oWL_t{sb + C * L6 * 2, L6 * 2, true}, oDO_t{sb + 2 * C * L6 * 2, LT * 2, true};
-    const int m0 = 32 * (warp & 1), n0 = 32 * (warp >> 1);
-    float Z[2][4][4];
-    zero(Z);
-    warp_mma(Z, oWH_t, oDO_t, C, m0, n0, lane);
-    warp_mma(Z, oWL_t, oDO_t, C, m0, n0, lane);
-    for_pair<2, 4>(m0, n0, g, t, [&](int mt, int nt, int hf, int i, int c) {
-      const uint32_t packed = i < si.n ? pack_bf16(Z[mt][nt][2 * hf], Z[mt][nt][2 * hf + 1]) : 0u;
-      *reinterpret_cast<uint32_t*>(a.v_ext + ((size_t)(e_real * C + i) * H + h) * kD + c) = packed;
-    });
+    auto cp16 = [&](uint32_t dst, const void* src, bool live) {
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(live ? 16 : 0));
+    };
+    for (int idx = tid; idx < C * 8; idx += kPrepThreads) {
+      const int r = idx >> 3, c8 = (idx & 7) * 8;
+      cp16(sb + (r * L6 + c8) * 2, a.W + mat + r * C + c8, true);
+      cp16(sb + (C * L6 + r * L6 + c8) * 2, a.W + a.w_lo_offset + mat + r * C + c8, true);
+    }
+    for (int idx = tid; idx < C * (kD / 8); idx += kPrepThreads) {
+      const int r = idx >> 4, c8 = (idx & 15) * 8;
+      cp16(sb + (2 * C * L6 + r * LT + c8) * 2, a.d_o + ((size_t)(si.tok0 + (r < si.n ? r : 0)) * H + h) * kD + c8, r < si.n);
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
   }
 
   // ---- coefficient vectors: abar' = g_M, p' = g_S, g_S' = p, g_M' = abar, end-of-chunk scalars (mubar_C, b_C,
@@ -106,6 +94,23 @@ __global__ void __launch_bounds__(kPrepThreads) bwd_prep_kernel(PrepArgs a) {
       default: break;   // mubar and the per-token gates are not read by a state-only run
     }
     cr[idx] = xr;
+  }
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
+  __syncthreads();
+
+  // ---- V' = W^T dO for the real step: a 64 x 128 result, one 32 x 32 block per warp, bf16 MMAs (W as hi + lo)
+  {
+    const uint32_t sb = smem_u32(smem_raw);
+    const Opnd oWH_t{sb, L6 * 2, true}, oWL_t{sb + C * L6 * 2, L6 * 2, true}, oDO_t{sb + 2 * C * L6 * 2, LT * 2, true};
+    const int m0 = 32 * (warp & 1), n0 = 32 * (warp >> 1);
+    float Z[2][4][4];
+    zero(Z);
+    warp_mma(Z, oWH_t, oDO_t, C, m0, n0, lane);
+    warp_mma(Z, oWL_t, oDO_t, C, m0, n0, lane);
+    for_pair<2, 4>(m0, n0, g, t, [&](int mt, int nt, int hf, int i, int c) {
+      const uint32_t packed = i < si.n ? pack_bf16(Z[mt][nt][2 * hf], Z[mt][nt][2 * hf + 1]) : 0u;
+      *reinterpret_cast<uint32_t*>(a.v_ext + ((size_t)(e_real * C + i) * H + h) * kD + c) = packed;
+    });
   }
 }
 
