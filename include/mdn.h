@@ -467,6 +467,8 @@ mdn_status mdn_set_stage_events(void* const* events /* host */, int32_t n);
  *                                                              accumulating onto a preloaded D)
  *   mode 4: M = 64: a[64 x 128] * b[128 x 128]^T from shared memory into tensor memory pre-filled with -777;
  *           out[128 x 128] = all 128 lanes x 128 columns (shows which lanes the 64 rows of the result occupy)
+ *   mode 5: M = 64 with an MN-major B: out[64 x 128] = a[64 x 128] * b[128 x 128], b laid out in shared memory as
+ *           mdn_chunk_fwd_keep_states keeps a chunk state (value index x key index, two swizzled blocks)
  * a, b: bf16 row-major device buffers; out: float32 device buffer; status: device int32 (0 = ok).
  */
 mdn_status mdn_selftest_umma(int32_t mode, const void* a, const void* b, float* out, int32_t* status,

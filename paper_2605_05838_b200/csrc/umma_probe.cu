@@ -107,6 +107,37 @@ __global__ void __launch_bounds__(128) umma_probe_kernel(int mode, const __nv_bf
         for (int j = 0; j < 32; ++j) out[tid * 64 + c0 + j] = __uint_as_float(r[j]);
       }
     }
+  } else if (mode == 5) {     // SS with M = 64 and an MN-major B: D[64x128] = A[64x128] * B[128x128], B a kept chunk state
+    // B[j][d] (value index j = K, key index d = N) lies as the chain kernel keeps a state: two blocks (d halves) of
+    // [128 rows j][64 d], 128-byte swizzle; read MN-major it needs no transposition.  out[64 x 128], rows from the
+    // lanes the M = 64 data path uses
+    fill_kmajor(sB, a, 64, 128, tid, 128);
+    fill_kmajor(sA, b, 128, 128, tid, 128);
+    fence_proxy_async_smem();
+    tc_fence_before_sync();
+    __syncthreads();
+    if (tid == 0) {
+      tc_fence_after_sync();
+      const uint32_t id = idesc_bf16(64, 128, false, true, false);
+      for (int k = 0; k < 8; ++k) {
+        const uint64_t da = smem_desc_sw128(smem_u32(sB) + (k / 4) * 8192 + (k % 4) * 32, 16, 1024);
+        const uint64_t db = smem_desc_sw128(smem_u32(sA) + k * 2048, 16384, 1024);   // 16 rows of j per K step
+        umma_ss(tmem, da, db, id, k > 0);
+      }
+      umma_commit(bar_mma);
+    }
+    ok = mbar_wait(bar_mma, 0, &abort_flag);
+    __syncwarp();
+    tc_fence_after_sync();
+    if (ok) {
+      for (int c0 = 0; c0 < 128; c0 += 32) {
+        uint32_t r[32];
+        tmem_ld32(tmem + lane_base + c0, r);
+        tmem_wait_ld();
+        if ((tid & 31) < 16)
+          for (int j = 0; j < 32; ++j) out[(16 * warp + (tid & 31)) * 128 + c0 + j] = __uint_as_float(r[j]);
+      }
+    }
   } else if (mode == 4) {     // SS with M = 64: D[64x128] = A[64x128] * B[128x128]^T; out = all 128 lanes x 128 columns
     // tensor memory is filled with a sentinel first, so the lanes the 64 rows land in can be read off the result
     {
@@ -224,7 +255,7 @@ __global__ void __launch_bounds__(128) umma_probe_kernel(int mode, const __nv_bf
 extern "C" mdn_status mdn_selftest_umma(int32_t mode, const void* a, const void* b, float* out, int32_t* status,
                                         void* cuda_stream) {
   using namespace mdn;
-  if (mode < 0 || mode > 4 || !a || !out || !status || (mode != 0 && !b)) return MDN_ERR_INVALID_ARG;
+  if (mode < 0 || mode > 5 || !a || !out || !status || (mode != 0 && !b)) return MDN_ERR_INVALID_ARG;
   CUtensorMap map;
   std::memset(&map, 0, sizeof(map));
   const void* tma_src = mode == 3 ? b : a;      // [64 x 128] bf16

@@ -78,3 +78,13 @@ def test_mma_m64_data_path_layout(mdn):
             assert np.abs(out[lane] - ref[16 * q + i]).max() < 1e-3, lane
         else:
             assert np.all(out[lane] == -777.0), lane
+
+
+def test_mma_m64_state_image_as_mn_major_b(mdn):
+    """A 64-row product against a kept chunk state read in place: B[j][d] in the state's shared-memory image (two
+    blocks of key-index halves, 128-byte swizzle) through an MN-major descriptor, sixteen rows of j per K step."""
+    rng = np.random.default_rng(6)
+    a, b = bf16_mat(rng, (64, 128)), bf16_mat(rng, (128, 128))
+    out = run(mdn, 5, a, b, (64, 128))
+    ref = a.float() @ b.float()
+    assert (out - ref).abs().max() < 1e-3
