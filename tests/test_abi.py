@@ -101,3 +101,39 @@ def test_null_and_workspace_errors_before_any_launch(mdn):
     a2 = list(args); a2[9] = fake
     st = L.mdn_chunk_fwd(ctypes.byref(p), *a2, fake, 1 << 40, null)
     assert mdn.status_string(st) == "invalid argument"
+
+
+def test_training_buffer_sizes_and_state_image_unpacking(mdn):
+    """Host-side arithmetic of the training entry points: per (chunk slot, head) a 64 KB state image and 32 KB of
+    fp32 V~ (dR for the adjoint chain, one entry per chunk); and the binding's reading of a state image, checked on a
+    hand-built image (value index x key index, two key-index blocks, 16-byte pieces XOR-swizzled with the row)."""
+    import numpy as np
+    import torch
+    L = mdn.lib()
+    bf = dict(dk=128, dv=128, io_dtype=1, o_dtype=1)
+    p = params(mdn, B=2, T=130, H=3, **bf)                   # 3 chunks per sequence: 6 slots
+    per = 3 * (65536 + 64 * 128 * 4)
+    assert L.mdn_chunk_states_bytes(ctypes.byref(p)) == 6 * per
+    assert L.mdn_bwd_adjoint_states_bytes(ctypes.byref(p)) == 6 * per
+    assert L.mdn_chunk_bwd_chunked_workspace_bytes(ctypes.byref(p)) > L.mdn_chunk_bwd_saved_workspace_bytes(ctypes.byref(p)) > 0
+    f32 = params(mdn, B=2, T=130, H=3)                      # SIMT path: no chunk-parallel backward
+    assert L.mdn_chunk_states_bytes(ctypes.byref(f32)) == 0 and L.mdn_chunk_bwd_chunked_workspace_bytes(ctypes.byref(f32)) == 0
+
+    H, slots = 2, 3
+    rng = np.random.default_rng(0)
+    S = torch.from_numpy(rng.standard_normal((slots, H, 2, 128, 128)).astype(np.float32)).to(torch.bfloat16)   # [.., S|M, key d, value j]
+    img = torch.zeros((slots, H, 2, 2, 128, 64), dtype=torch.bfloat16)        # [.., S|M, key half, row j, 64 keys in swizzled order]
+    for j in range(128):
+        for piece in range(8):
+            for half in range(2):
+                src = S[:, :, :, half * 64 + piece * 8: half * 64 + piece * 8 + 8, j]          # logical piece of row j
+                phys = piece ^ (j & 7)
+                img[:, :, :, half, j, phys * 8: phys * 8 + 8] = src
+    vt = torch.from_numpy(rng.standard_normal((slots, 64, H, 128)).astype(np.float32))
+    buf = torch.cat([img.view(torch.uint8).reshape(-1), vt.view(torch.uint8).reshape(-1)])
+    assert buf.numel() == slots * H * (65536 + 32768)
+    Sg, Mg = mdn.unpack_chunk_states(buf, H)
+    assert torch.equal(Sg, S[:, :, 0].float()) and torch.equal(Mg, S[:, :, 1].float())
+    assert torch.equal(mdn.unpack_chunk_vt(buf, H), vt)
+    with pytest.raises(ValueError):
+        mdn.unpack_chunk_states(buf[:-4], H)
