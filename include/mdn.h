@@ -25,8 +25,13 @@
  *    restarts at every sequence; chunks never straddle sequences; the last chunk
  *    of a sequence may be short.
  *  - The caller owns every buffer, including the workspace.  The library
- *    allocates no device memory, keeps no state between calls, and only
- *    enqueues work on the given stream (it never synchronises).
+ *    allocates no device memory and only enqueues work on the given stream
+ *    (it never synchronises).  It keeps no state between calls, with three
+ *    documented exceptions: mdn_chunk_fwd_host keeps two internal streams and
+ *    their events per host thread and device; mdn_chunk_fwd_static_scratch
+ *    keeps the device address of its built-in scratch array (and the array
+ *    keeps the last call's contents); mdn_set_stage_events keeps the event
+ *    handles of the calling host thread until cleared.
  *  - Errors are returned as mdn_status; nothing throws, aborts or traps.
  *    Invalid arguments are rejected on the host before anything is launched.
  */
@@ -456,23 +461,6 @@ const char* mdn_status_string(mdn_status s);
  */
 #define MDN_NUM_STAGE_EVENTS 4
 mdn_status mdn_set_stage_events(void* const* events /* host */, int32_t n);
-
-/*
- * Diagnostic: runs one small tcgen05 / TMA case on one CTA (the operand configurations the
- * tensor-core chain kernel uses) so that each can be checked against a host matmul.
- *   mode 0: TMA 128-byte-swizzled load of a [64 x 128] bf16 matrix `a`; out = the raw 16 KB of shared memory
- *   mode 1: out[128 x 64]  = a[128 x 128] * b[64 x 128]^T     (A and B from shared memory, K-major)
- *   mode 2: out[128 x 64]  = a[128 x 64]  * b[64 x 64]^T      (A from tensor memory)
- *   mode 3: out[128 x 128] = 1 - a[128 x 64] * b[64 x 128]    (A from tensor memory, negated; B MN-major via TMA;
- *                                                              accumulating onto a preloaded D)
- *   mode 4: M = 64: a[64 x 128] * b[128 x 128]^T from shared memory into tensor memory pre-filled with -777;
- *           out[128 x 128] = all 128 lanes x 128 columns (shows which lanes the 64 rows of the result occupy)
- *   mode 5: M = 64 with an MN-major B: out[64 x 128] = a[64 x 128] * b[128 x 128], b laid out in shared memory as
- *           mdn_chunk_fwd_keep_states keeps a chunk state (value index x key index, two swizzled blocks)
- * a, b: bf16 row-major device buffers; out: float32 device buffer; status: device int32 (0 = ok).
- */
-mdn_status mdn_selftest_umma(int32_t mode, const void* a, const void* b, float* out, int32_t* status,
-                             void* cuda_stream);
 
 /* Text of the CUDA runtime error behind the last MDN_ERR_CUDA returned on this host thread by the
  * intra-chunk or chain launches (static string, host pointer). */

@@ -124,8 +124,6 @@ def lib() -> ctypes.CDLL:
         L.mdn_status_string.argtypes = [ctypes.c_int]
         L.mdn_set_stage_events.restype = ctypes.c_int
         L.mdn_set_stage_events.argtypes = [ctypes.POINTER(vp), ctypes.c_int32]
-        L.mdn_selftest_umma.restype = ctypes.c_int
-        L.mdn_selftest_umma.argtypes = [ctypes.c_int32, vp, vp, vp, vp, vp]
         L.mdn_last_cuda_error_string.restype = ctypes.c_char_p
         L.mdn_last_cuda_error_string.argtypes = []
         L.mdn_last_launch_count.restype = ctypes.c_int32
@@ -593,12 +591,6 @@ def intra_chunk(p: MdnParams, q, k, cu_seqlens, workspace) -> None:
                                workspace.numel(), _stream())
     if st != 0:
         raise MdnError(st, "mdn_intra_chunk")
-
-
-def selftest_umma(mode: int, a, b, out, status) -> None:
-    st = lib().mdn_selftest_umma(int(mode), _ptr(a), _ptr(b), _ptr(out), _ptr(status), _stream())
-    if st != 0:
-        raise MdnError(st, "mdn_selftest_umma")
 
 
 def read_status(p: MdnParams, workspace) -> int:

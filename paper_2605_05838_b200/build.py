@@ -16,7 +16,9 @@ CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libmdn.so")
 OBJ_DIR = os.path.join(PKG, "build")
 
-NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
+# MDN_BUILD_DEBUG=1 in the environment of the BUILD compiles the debug knobs in (-DMDN_DEBUG: precision ablation
+# switch and the per-chunk clock stamps of the chain kernels); the default library has none of them.
+NVCC_FLAGS = (["-DMDN_DEBUG"] if os.environ.get("MDN_BUILD_DEBUG") == "1" else []) + ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 
 

@@ -271,7 +271,9 @@ __global__ void __launch_bounds__(Roles<token_groups(kLayer)>::kThreads, 1) chai
     ok = false;                                    \
     break;                                         \
   }
+#ifdef MDN_DEBUG
   long long* const tline = (blockIdx.x == 0) ? a.timeline : nullptr;
+#endif
   // Hand-over arrivals of the epilogue.  With 16 epilogue warps (layer variant) one arrival per warp, after the warp
   // has converged (every lane's stores and fences precede it): 32 x fewer shared-memory atomics in front of every
   // hand-over, 2 % of the step.  The 8-warp plain forward measured 1 % slower that way and keeps one per thread.
@@ -284,8 +286,12 @@ __global__ void __launch_bounds__(Roles<token_groups(kLayer)>::kThreads, 1) chai
       mbar_arrive(bar);                  \
     }                                    \
   }
+#ifdef MDN_DEBUG
 #define MDN_MARK(c, ev) \
   if (tline != nullptr && lane == 0 && (warp == 0 || warp >= kEpiWarps)) tline[(c) * 32 + (ev)] = clock64();
+#else
+#define MDN_MARK(c, ev)
+#endif
 
   if (warp == kWarpTma) {
     // ================================================================== TMA producer + output stores
@@ -989,10 +995,14 @@ cudaError_t launch_chain_tensor(const Plan& pl, const void* q, const void* k, co
   a.status = reinterpret_cast<int32_t*>(pl.ws + pl.lay.off_status);
   a.scale = p.scale;
   a.w_lo_row_offset = (uint32_t)(mats * C);
+  a.drop_lo = 0u;
+  a.timeline = nullptr;
+#ifdef MDN_DEBUG   // debug builds only (-DMDN_DEBUG): the product library reads nothing from the environment
   const char* drop = getenv("MDN_DEBUG_DROP_LO");
   a.drop_lo = drop ? (uint32_t)atoi(drop) : 0u;
   const char* tl = getenv("MDN_DEBUG_TIMELINE");   // device address of an int64 buffer, [chunks][32]
   a.timeline = tl ? reinterpret_cast<long long*>(strtoull(tl, nullptr, 0)) : nullptr;
+#endif
   a.dump = pl.chain_dump; a.state_only = pl.chain_state_only; a.end_scalars_in_rk = pl.chain_end_scalars_in_rk;
   a.vt_dump = pl.chain_vt_dump; a.inject = pl.chain_inject;
   a.mirror = pl.chain_mirror_geom != nullptr;

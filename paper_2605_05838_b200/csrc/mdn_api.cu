@@ -663,11 +663,16 @@ static bool host_arena(const mdn_params* p, HostArena* a) {
   if (check_params(p) != MDN_OK) return false;
   a->slices = host_slices(*p);
   a->rows_max = (p->B + a->slices - 1) / a->slices;
-  mdn_params ps = *p;
-  ps.B = a->rows_max;
-  mdn_ws_layout lay;
-  if (make_layout(ps, &lay) != MDN_OK) return false;
-  a->ws_slice = align_up(lay.total_bytes, 256);
+  // a slice holds rows_max or rows_max - 1 rows, and the smaller one may need the LARGER workspace (with fewer
+  // chains the parallel inter-chunk scan can switch on and bring its segment scratch): size for both
+  a->ws_slice = 0;
+  for (int rows = a->rows_max; rows >= 1 && rows >= p->B / a->slices; --rows) {
+    mdn_params ps = *p;
+    ps.B = rows;
+    mdn_ws_layout lay;
+    if (make_layout(ps, &lay) != MDN_OK) return false;
+    if (align_up(lay.total_bytes, 256) > a->ws_slice) a->ws_slice = align_up(lay.total_bytes, 256);
+  }
   const uint64_t es = p->io_dtype == MDN_BF16 ? 2 : 4, eo = p->o_dtype == MDN_BF16 ? 2 : 4;
   const uint64_t rows = (uint64_t)p->B, nseq = (uint64_t)(p->num_seqs > 0 ? p->num_seqs : p->B);
   a->qk_row = (uint64_t)p->T * p->H * p->dk * es; a->v_row = (uint64_t)p->T * p->H * p->dv * es;

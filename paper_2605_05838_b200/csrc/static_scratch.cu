@@ -50,9 +50,13 @@ extern "C" mdn_status mdn_chunk_fwd_static_scratch(const mdn_params* p, const vo
                                                    const float* eta, const float* initial_S, const float* initial_M,
                                                    const int32_t* cu_seqlens, void* o, float* final_S, float* final_M,
                                                    void* cuda_stream) {
-  const size_t need = mdn_chunk_fwd_workspace_bytes(p);
-  if (need == 0) return p ? MDN_ERR_UNSUPPORTED : MDN_ERR_INVALID_ARG;
-  if (need > (size_t)MDN_STATIC_SCRATCH_BYTES) return MDN_ERR_STATIC_SCRATCH;
+  // Parameters the workspace entry point would refuse get the same status here; only a valid problem
+  // that needs more scratch than the array holds is answered with MDN_ERR_STATIC_SCRATCH.
+  mdn_ws_layout lay;
+  const mdn_status ps = mdn_workspace_layout(p, &lay);
+  if (ps != MDN_OK) return ps;
+  if (p->num_seqs > 0 ? cu_seqlens == nullptr : cu_seqlens != nullptr) return MDN_ERR_INVALID_ARG;
+  if (lay.total_bytes > (uint64_t)MDN_STATIC_SCRATCH_BYTES) return MDN_ERR_STATIC_SCRATCH;
   void* scratch = nullptr;
   const mdn_status st = scratch_address(&scratch);
   if (st != MDN_OK) return st;

@@ -54,8 +54,9 @@ constexpr uint32_t kSpinLimit = 1u << 22;   // try_wait suspends internally; thi
 
 // Bounded wait.  Returns false when the limit ran out or another thread already gave up
 // (*abort_flag != 0); the caller then unwinds to the kernel's common exit.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  for (uint32_t it = 0; it < kSpinLimit; ++it) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          uint32_t limit = kSpinLimit) {
+  for (uint32_t it = 0; it < limit; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((it & 255u) == 255u && *abort_flag != 0) return false;
   }
@@ -140,6 +141,23 @@ __device__ __host__ constexpr uint32_t idesc_bf16(int M, int N, bool a_mn_major,
          | (static_cast<uint32_t>(N >> 3) << 17) | (static_cast<uint32_t>(M >> 4) << 24);
 }
 
+// Instruction descriptor for kind::tf32 (fp32 storage read as tf32: the low 13 mantissa bits are ignored) with fp32
+// accumulation.  One instruction covers K = 8.
+__device__ __host__ constexpr uint32_t idesc_tf32(int M, int N, bool a_mn_major, bool b_mn_major, bool negate_a) {
+  return (1u << 4)                          // D format: fp32
+         | (2u << 7) | (2u << 10)           // A, B format: tf32
+         | (negate_a ? (1u << 13) : 0u)
+         | (a_mn_major ? (1u << 15) : 0u) | (b_mn_major ? (1u << 16) : 0u)
+         | (static_cast<uint32_t>(N >> 3) << 17) | (static_cast<uint32_t>(M >> 4) << 24);
+}
+
+// Byte offset of element (row, col) of a [rows x 32] fp32 block (128-byte rows, 8-row / 1024-byte atoms) in the
+// 128-byte swizzle.  The block base must be 1024-byte aligned.
+__device__ __host__ __forceinline__ uint32_t sw128_offset_f32(uint32_t row, uint32_t col_f32) {
+  const uint32_t chunk = (col_f32 >> 2) ^ (row & 7u);
+  return row * 128u + chunk * 16u + (col_f32 & 3u) * 4u;
+}
+
 // D[tmem] (+)= A[smem] * B[smem]; issued by ONE thread.
 __device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, bool accumulate) {
   asm volatile(
@@ -156,6 +174,23 @@ __device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64
       "setp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}\n"
       ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(static_cast<uint32_t>(accumulate))
+      : "memory");
+}
+// kind::tf32 forms: A from tensor memory (one 32-bit column per K element) or from shared memory.
+__device__ __forceinline__ void umma_ts_tf32(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, bool accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, p;\n\t}\n"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(static_cast<uint32_t>(accumulate))
+      : "memory");
+}
+__device__ __forceinline__ void umma_ss_tf32(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, bool accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}\n"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(static_cast<uint32_t>(accumulate))
       : "memory");
 }
 // Make `bar` complete once every tcgen05.mma this thread issued so far has finished.
@@ -266,7 +301,28 @@ __device__ __forceinline__ void split_pack_bf16(float x0, float x1, uint32_t& hi
 struct TmaMap2D {
   const void* base; uint64_t inner, outer; uint64_t row_stride_bytes; uint32_t box_inner, box_outer; bool swizzle128;
 };
-bool encode_tma_2d(CUtensorMap* out, const TmaMap2D& d, bool f32);   // element type bf16, or float32 when f32
+// Element type bf16, or float32 when f32.
+inline bool encode_tma_2d(CUtensorMap* out, const TmaMap2D& d, bool f32) {
+  typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                               const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                               CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+  static EncodeFn fn = nullptr;
+  if (fn == nullptr) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess || p == nullptr)
+      return false;
+    fn = reinterpret_cast<EncodeFn>(p);
+  }
+  const cuuint64_t dims[2] = {d.inner, d.outer};
+  const cuuint64_t strides[1] = {d.row_stride_bytes};
+  const cuuint32_t box[2] = {d.box_inner, d.box_outer};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(out, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(d.base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, d.swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
 inline bool encode_tma_2d_bf16(CUtensorMap* out, const TmaMap2D& d) { return encode_tma_2d(out, d, false); }
 
 }  // namespace mdn

@@ -1,35 +1,14 @@
-// Bring-up probe for the sm_100a building blocks of the tensor-core chain kernel: one CTA runs
+// Test-only bring-up probe for the sm_100a building blocks of the tensor-core kernels: one CTA runs
 // one small tcgen05 / TMA case per mode so that descriptor, swizzle and TMEM-layout mistakes show
-// up in isolation (checked against a host matmul by the tests).  Also home of the host-side
-// tensor-map encoder.
+// up in isolation (checked against a host matmul by the tests).  Built into its own library
+// (libmdn_probe.so) by tests/probe/build_probe.py; nothing of it is part of libmdn.so.
 #include <cstring>
 
 #include "mdn_common.cuh"
+#include "mdn_probe.h"
 #include "tc_utils.cuh"
 
 namespace mdn {
-
-bool encode_tma_2d(CUtensorMap* out, const TmaMap2D& d, bool f32) {
-  typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                               const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                               CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-  static EncodeFn fn = nullptr;
-  if (fn == nullptr) {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
-        qres != cudaDriverEntryPointSuccess || p == nullptr)
-      return false;
-    fn = reinterpret_cast<EncodeFn>(p);
-  }
-  const cuuint64_t dims[2] = {d.inner, d.outer};
-  const cuuint64_t strides[1] = {d.row_stride_bytes};
-  const cuuint32_t box[2] = {d.box_inner, d.box_outer};
-  const cuuint32_t estr[2] = {1, 1};
-  return fn(out, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(d.base), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, d.swizzle128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
-            CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
 
 namespace {
 

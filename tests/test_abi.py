@@ -55,6 +55,28 @@ def test_workspace_layout_and_bounds(mdn):
     assert mdn.host_arena_bytes(p) > mdn.workspace_bytes(p)
 
 
+def test_host_arena_covers_every_slice_workspace(mdn):
+    """mdn_chunk_fwd_host cuts the batch into up to eight slices with B // 8 or B // 8 + 1 rows and calls
+    mdn_chunk_fwd on each with its own workspace: the arena's workspace part must cover the LARGEST of the slices'
+    needs - a slice with fewer rows can need more (with fewer chains the parallel inter-chunk scan switches on)."""
+    up = lambda x: (x + 255) // 256 * 256
+    bf = dict(dk=128, dv=128, io_dtype=1, o_dtype=1)
+    checked = shrinking = 0
+    for B in (1, 2, 7, 8, 9, 15, 17, 33, 40, 64):
+        for H in (1, 2, 5, 16):
+            for T in (64, 1000, 4096, 16384):
+                p = params(mdn, B=B, H=H, T=T, **bf)
+                slices = min(B, 8)
+                rows, st = B * T * H, H * 128 * 128 * 4
+                io = 3 * up(rows * 128 * 2) + 4 * up(rows * 4) + 2 * up(B * st) + up(0) + up(rows * 128 * 2) + 2 * up(B * st)
+                ws_part = mdn.host_arena_bytes(p) - io
+                need = [mdn.workspace_bytes(params(mdn, B=b, H=H, T=T, **bf)) for b in {B // slices, -(-B // slices)} if b > 0]
+                assert ws_part >= slices * up(max(need)), (B, H, T)
+                checked += 1
+                shrinking += len(need) == 2 and need[0] != need[1] and (need[0] > need[1]) != (B // slices > -(-B // slices))
+    assert checked == 160
+
+
 def test_segment_choice_for_the_parallel_inter_chunk_scan(mdn):
     """Host-side rule only: few long chains are split, anything that already fills the GPU is not."""
     bf = dict(dk=128, dv=128, io_dtype=1, o_dtype=1)

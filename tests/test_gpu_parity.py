@@ -49,9 +49,9 @@ def check_bf16_store(o_bf16, o_ref, label):
     assert excess.max() <= TOL_BF16 * rms
 
 
-def compare(mdn, inp, path, chains=None, tol=None, label=""):
+def compare(mdn, inp, path, chains=None, tol=None, label="", ref=None):
     w = inp["workload"]
-    o_ref, S_ref, M_ref = run_oracle(inp, chains)
+    o_ref, S_ref, M_ref = ref if ref is not None else run_oracle(inp, chains)
     if w.dtype == "f32":
         o, S, M = run_gpu(mdn, inp, path=path)
         errs = rel_err(o, o_ref), rel_err(S, S_ref), rel_err(M, M_ref)
@@ -69,6 +69,38 @@ def compare(mdn, inp, path, chains=None, tol=None, label=""):
 
 
 # ------------------------------------------------------------------------------------------ stages
+@pytest.mark.parametrize("lens", [[1, 63, 64, 65, 129, 300], [64], [1], [5, 1, 1, 200, 64, 127, 128, 2, 640],
+                                  list(range(1, 41)), [0, 7, 0, 130, 0]])
+def test_chunk_map_is_bit_exact(mdn, lens):
+    """a0: the chunk map the prep kernel writes from cu_seqlens - first slot of every sequence and, per slot,
+    (sequence, first token, valid tokens, chunk index inside the sequence); unused slots up to the host-side bound
+    T/64 + num_seqs carry sequence -1 - equals the integers computed here from the lengths, bit for bit."""
+    import torch
+    lens = np.asarray(lens, dtype=np.int64)
+    N, T, H = len(lens), int(lens.sum()), 2
+    cu = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    z = torch.zeros((1, T, H), dtype=torch.float32, device="cuda")
+    qv = torch.zeros((1, T, H, 64), dtype=torch.float32, device="cuda")
+    p = mdn.make_params(qv, qv, num_seqs=N)
+    lay = mdn.workspace_layout(p)
+    assert lay.num_slots == T // 64 + N
+    ws = torch.full((lay.total_bytes,), 0x5A, dtype=torch.uint8, device="cuda")       # stale bytes everywhere
+    mdn.coeff_scan(p, z, z, z, None, torch.from_numpy(cu).cuda(), ws)
+    torch.cuda.synchronize()
+    assert mdn.read_status(p, ws) == 0
+    chunk_off = ws[lay.off_chunk_off: lay.off_chunk_off + 4 * (N + 1)].view(torch.int32).cpu().numpy()
+    slot_map = ws[lay.off_slot_map: lay.off_slot_map + 16 * lay.num_slots].view(torch.int32).cpu().numpy().reshape(-1, 4)
+    nch = (lens + 63) // 64
+    want_off = np.concatenate([[0], np.cumsum(nch)]).astype(np.int32)
+    want_map = np.zeros((lay.num_slots, 4), dtype=np.int32)
+    want_map[:, 0] = -1
+    for n in range(N):
+        for c in range(int(nch[n])):
+            want_map[want_off[n] + c] = (n, cu[n] + 64 * c, min(64, lens[n] - 64 * c), c)
+    assert np.array_equal(chunk_off, want_off)
+    assert np.array_equal(slot_map, want_map)
+
+
 def test_coefficient_scan_matches_eq10(mdn):
     import torch
     from oracle import chunkwise as cw
@@ -191,21 +223,13 @@ def test_config0_tiny_fp32(mdn):
 
 @pytest.mark.parametrize("cfg", [1, 2, 3, 4])
 def test_named_bf16_configs_full_size(mdn, cfg):
+    """Every (sequence, head) chain of the named bf16 configurations at full size, element by element, on the path
+    bench.py times (tensor) and on the fp32 SIMT path."""
     w = wl.CONFIGS[cfg]
     inp = wl.make_inputs(w)
-    N = len(inp["seq_len"])
-    rng = np.random.default_rng(cfg)
-    all_chains = np.arange(N * w.H)
-    if cfg == 1:
-        chains = all_chains
-    elif cfg == 2:      # first, last and 14 random chains of 128
-        chains = np.unique(np.concatenate([[0, N * w.H - 1], rng.choice(all_chains, 14, replace=False)]))
-    elif cfg == 3:      # 4 of 16 heads, all 65536 tokens (1024 serial chunk steps)
-        chains = np.array([0, 5, 10, 15])
-    else:               # every sequence, two heads each
-        chains = np.array([n * w.H + h for n in range(N) for h in (n % w.H, (n + 7) % w.H)])
+    ref = run_oracle(inp)           # all chains, once for both paths
     for path in paths_for(mdn, w):
-        compare(mdn, inp, path, chains=chains, label=w.name)
+        compare(mdn, inp, path, label=w.name, ref=ref)
 
 
 # ------------------------------------------------------------------------------------------ edge cases
