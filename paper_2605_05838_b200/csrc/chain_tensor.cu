@@ -967,8 +967,16 @@ cudaError_t launch_intra_tensor(const Plan& pl, const void* q, const void* k, co
   return launch_intra_mma(pl, q, k, gates, launches);
 }
 
+bool chain_uses_tf32_kernel(const Plan& pl) {
+  const bool layer = pl.qk.on || pl.post.on;
+  const bool train = pl.chain_dump != nullptr || pl.chain_state_only || pl.chain_end_scalars_in_rk ||
+                     pl.chain_vt_dump != nullptr || pl.chain_inject || pl.chain_mirror_geom != nullptr;
+  return pl.p.path == MDN_PATH_TENSOR && !layer && !train;
+}
+
 cudaError_t launch_chain_tensor(const Plan& pl, const void* q, const void* k, const void* v, const float* S0,
                                 const float* M0, void* o, float* Sf, float* Mf, int* launches) {
+  if (pl.w_f32) return launch_chain_tf32(pl, q, k, v, S0, M0, o, Sf, Mf, launches);
   const mdn_params& p = pl.p;
   const uint64_t tokens = (uint64_t)p.B * p.T;
   // mirrored run: q, k, o are another problem's tensors (its geometry in chain_mirror_geom)

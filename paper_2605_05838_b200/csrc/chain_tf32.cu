@@ -1,0 +1,834 @@
+// a3 + a4 of the plain forward on the 5th-generation tensor cores (tcgen05, sm_100a), second design: one CTA walks
+// the chunks of one (sequence, head) in order; bf16 q/k/v, dk = dv = 128, chunk 64.  (The first design,
+// chain_tensor.cu, stays for the forward with layer operations and for the training / backward runs.)
+//
+// Everything is kept TRANSPOSED: the value dimension (128) is the MMA M dimension and fills the 128 tensor-memory
+// lanes, tokens are N (or K).  What is different here:
+//
+//  * No per-chunk pass over the state.  The fp32 masters S^T, M^T in tensor memory are read by the tensor core as
+//    they are, as the A operand of kind::tf32 products (fp32 storage read as tf32), against fp32 copies of the K and
+//    Q tiles that two converter warps write one chunk ahead.  No bf16 copy of the state is ever made.
+//  * Lazy scaling of the state.  The chunk hand-over  S' = abar_C S - b_C M + dS,  M' = mubar_C M - dM  (state equations
+//    below Eq. 12) is a 2 x 2 upper-triangular scalar map D_c on the pair [S; M].  Instead of rescaling the masters
+//    every chunk, the masters hold [Sh; Mh] with  [S; M] = G [Sh; Mh],  G = [[g11, g12], [0, g22]]  kept as three
+//    scalars:  G' = D_c G  and the update is added in hat coordinates,  [Sh'; Mh'] = [Sh; Mh] + G'^-1 [dS; -dM].
+//    Every use of the state then only changes per-token coefficients (all products are linear in the state):
+//        K S = g11 (K Sh) + g12 (K Mh),  K M = g22 (K Mh)        ->  R = V - cX .* X + cY .* Y
+//        Q S, Q M likewise                                       ->  o_inter = cZ .* Z + cU .* U
+//        dS / g11' + (g12' / (g11' g22')) dM,  dM / g22'         ->  per-token weights wS, wM of V~ in the updates
+//    with cX = abar g11, cY = (alpha b^-) g22 - abar g12, cZ = scale abar g11, cU = scale (abar g12 - b g22),
+//    wS = (gS + (g12'/g22') gM) / g11', wM = gM / g22' (gS = gamma_C eta, gM = (mubar_C/mubar) eta).  The converter
+//    warps run the scalar recurrence of G and write these six vectors per chunk.  When G' would leave a safe range
+//    (g11' or g22' below 2^-64, or |g12'| above g22': fast-decaying gates, mu = 0 tokens, S decaying slower than M) the chunk is "eager":
+//    the epilogue warps rescale the masters once by G' (the first design's pre-scaling, with G folded in) and G
+//    returns to the identity.  The result is the same recurrence either way; only rounding differs.
+//  * One product gives the state terms of the correction AND of the output: B = the K tile stacked on the Q tile
+//    (128 rows), so [X | Z] = Sh [K; Q]^T and [Y | U] = Mh [K; Q]^T are two N = 128 products (a product costs the
+//    same up to N = 128: measured 54 / 54 / 64 / 128 cycles at N = 32 / 64 / 128 / 256 with A in tensor memory).
+//  * The intra-chunk output product reads V~ straight from the accumulator of V~ = T R (kind::tf32 against an fp32 W
+//    tile the intra-chunk kernel writes), accumulating onto the inter-chunk terms the epilogue has left there: no
+//    operand conversion for it, and it runs under the epilogue's work on the state update.
+//
+// Per chunk:  MMA-1 [X|Z], [Y|U]  ->  EPI-1 R^T (bf16 hi + lo)  ->  MMA-2 Y = R^T T^T  ->  EPI-2 wS .* V~, wM .* V~ (bf16 hi + lo)
+//             ->  MMA-3 Sh^T += (wS V~)^T K, Mh^T -= (wM V~)^T K (K tile read MN-major)  ->  next chunk's MMA-1.
+// Off that path: o_inter into U (under MMA-2), MMA-3' U += V~^T W^T (under EPI-2), output tile + TMA store (under MMA-3).
+//
+// Warps: MMA issuer (one elected lane, tensor-memory owner), TMA producer (also issues the output stores), 8 epilogue
+// warps (lane quarter x token half), 2 converter warps.  All hand-offs are mbarriers with bounded waits.
+#include <cstdlib>
+#include <cstring>
+
+#include "mdn_common.cuh"
+#include "tc_utils.cuh"
+
+namespace mdn {
+namespace {
+
+using namespace tc;
+
+constexpr int kD = 128;
+constexpr int kEpiWarps = 8, kTok = 32, kPk = 16;
+// Warp roles.  The hardware schedulers favour the older (lower-numbered) of their ready warps, and the MMA issuer must
+// never wait for an issue slot behind an epilogue warp that is busy with arithmetic (measured: as the youngest warp of
+// its scheduler it reacted 500-800 cycles late to every hand-over that fell into an epilogue step).  So: warp 0 MMA
+// issuer, warp 1 TMA producer, warps 2..9 epilogue (lane quarter = warp % 4, as tensor memory demands), warps 10 and 11
+// converters (the youngest on the two schedulers that hold neither the MMA nor the TMA warp).  Three warps per
+// scheduler: 168 registers each.
+constexpr int kWarpMma = 0, kWarpTma = 1, kWarpEpi = 2, kWarpCvt = 10, kCvtWarps = 2;
+constexpr int kThreads = (kEpiWarps + 2 + kCvtWarps) * 32;
+constexpr int kEpiThreads = kEpiWarps * 32, kCvtThreads = kCvtWarps * 32;
+
+// shared memory (offsets from a 1024-byte aligned base)
+// The K tile is read twice: by the converter warps, as rows from global memory a chunk ahead (with the Q rows), for its
+// fp32 copy; and by TMA into the stage, where MMA-3 reads it (MN-major) at the end of the chunk (an L2 hit).
+constexpr uint32_t kOffKQ32 = 0;        // fp32 [K; Q]: four dk quarters x [128 rows (K tokens, then Q tokens) x 128 B], swizzled
+constexpr uint32_t kOffStage = 65536;
+constexpr uint32_t kStK = 0, kStV = 16384, kStT = 32768, kStW = 40960, kStCoef = 57344;
+constexpr uint32_t kCoefBytes = kChainCoefs * C * sizeof(float);
+constexpr uint32_t kStageBytes = 59392;
+constexpr uint32_t kTxBytes = 2 * 16384 + 8192 + 16384 + kCoefBytes;
+constexpr uint32_t kTxW = 16384, kTxV = 16384;   // bytes of the W tile, of the V tile
+constexpr uint32_t kStOut = kStV;       // the finished output tile: V area (bf16), V + T + half of W (fp32); all dead by then
+constexpr uint32_t kOffAdj = kOffStage + 2 * kStageBytes;
+constexpr uint32_t kAdjBytes = 2048;
+constexpr uint32_t kSmemBytes = kOffAdj + 2 * kAdjBytes + 1024;
+static_assert(kStCoef + kCoefBytes <= kStageBytes && kSmemBytes <= 232448, "shared-memory layout");
+
+// per-chunk block the converter warps publish (float indices)
+enum Adj : int { kCx = 0, kCy = 64, kCz = 128, kCu = 192, kWs = 256, kWm = 320, kN11 = 384, kN12, kN22, kLazy };
+constexpr float kLazyMin = 5.421010862427522e-20f;   // 2^-64: smallest g11', g22' a lazy chunk may leave
+constexpr float kLazyMix = 1.f;                      // largest |g12'| / g22' (beyond it the two hat terms of S cancel too much)
+
+// tensor memory columns (512 x 128 lanes x 32 bit)
+constexpr uint32_t kColS = 0, kColM = 128, kColX = 256, kColZ = 320, kColY = 384, kColU = 448;
+
+struct Bars {
+  uint64_t full[2];   // TMA loads of a stage landed                                      (1 + tx bytes)
+  uint64_t go[2];     // a stage's output tile is staged and nothing reads the stage any more (256)
+  uint64_t kq;        // fp32 [K; Q] of a chunk written                                   (64)
+  uint64_t adj[2];    // a chunk's coefficient block written                              (64)
+  uint64_t fin;       // G after the last chunk written                                   (64)
+  uint64_t init;      // masters of chunk 0 stored                                        (256)
+  uint64_t mx;        // first half of MMA-1 done: X, Z                                    (commit)
+  uint64_t m1;        // MMA-1 done: X, Z, Y, U                                            (commit)
+  uint64_t r;         // EPI-1 done: R^T hi/lo in X                                        (256)
+  uint64_t m2;        // MMA-2 done                                                       (commit)
+  uint64_t oi;        // inter-chunk output terms stored in U                             (256)
+  uint64_t v1a;       // EPI-2, first part: wS V~ in X (eager chunks: Sh rescaled)         (256)
+  uint64_t v1b;       // EPI-2, second part: wM V~ in Y (eager chunks: Mh rescaled)        (256)
+  uint64_t m3s;       // MMA-3, Sh part done                                              (commit)
+  uint64_t m3;        // MMA-3 done                                                       (commit)
+  uint64_t mo;        // MMA-3' done                                                      (commit)
+  uint64_t zu;        // U (the chunk's output) has been read                              (256)
+};
+
+struct Args {
+  ChunkGeom g;
+  const float* coef;
+  const __nv_bfloat16* q;   // the converters read the K and Q rows straight from global memory
+  const __nv_bfloat16* k;
+  long long tokens;         // B * T: rows past the end of the tensor read as zeros
+  const float* S0;
+  const float* M0;
+  void* o;
+  float* Sf;
+  float* Mf;
+  int32_t* status;
+  float scale;
+  // parallel inter-chunk scan (seg_G = 0: off, one CTA walks all chunks of its chain)
+  int seg_G;
+  int seg_phase;
+  float* seg_E;
+  float* seg_Psi;
+  float* seg_PhiS;
+  float* seg_PhiM;
+  long long* timeline;   // debug builds: CTA 0 writes clock64() at [chunk * 32 + event]
+};
+
+enum Ev : int { kEvMma1 = 0, kEvM1Seen, kEvRArrive, kEvOiArrive, kEvM2Seen, kEvV1Arrive, kEvOutDone, kEvM3Seen, kEvRSeen,
+                kEvV1Seen, kEvCvtStart, kEvCvtDone, kEvTmaIssued, kEvStoresDone, kEvM2Own, kEvEager,
+                kEvXzIssued, kEvYuIssued, kEvM2Issued, kEvSIssued, kEvMIssued, kEvV1bSeen, kEvV1bArrive, kEvZuArrive, kEvMoIssued, kEvM3sOwn, kEvKqSeen, kEvLoopTop, kEvRArrive2, kEvV1Arrive2 };
+
+template <typename TO> __device__ __forceinline__ void stage_o(uint8_t* tile, int r, int d, float x);
+template <> __device__ __forceinline__ void stage_o<float>(uint8_t* tile, int r, int d, float x) {
+  reinterpret_cast<float*>(tile)[r * kD + d] = x;
+}
+template <> __device__ __forceinline__ void stage_o<__nv_bfloat16>(uint8_t* tile, int r, int d, float x) {
+  reinterpret_cast<__nv_bfloat16*>(tile)[r * kD + d] = __float2bfloat16_rn(x);
+}
+
+template <typename TO>
+__global__ void __launch_bounds__(kThreads, 1) chain_tf32_kernel(const Args a, const __grid_constant__ CUtensorMap map_q,
+                                                                const __grid_constant__ CUtensorMap map_k,
+                                                                const __grid_constant__ CUtensorMap map_v,
+                                                                const __grid_constant__ CUtensorMap map_t,
+                                                                const __grid_constant__ CUtensorMap map_w,
+                                                                const __grid_constant__ CUtensorMap map_o) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  __shared__ __align__(8) Bars bars;
+  __shared__ uint32_t tmem_slot;
+  __shared__ int abort_flag;
+  __shared__ float g_final[4];   // G after the last chunk: what the final states are read through
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int H = a.g.H;
+  // ---- work item: which chain, which segment of it, which kind of run
+  int chain = blockIdx.x, seg = 0, run = 0;   // run 0: the real thing; 1: Psi; 2: Phi from (I, 0); 3: Phi from (0, I)
+  if (a.seg_G > 0) {
+    if (a.seg_phase == 1) {
+      const int items = 1 + 3 * (a.seg_G - 2);
+      chain = blockIdx.x / items;
+      const int w = blockIdx.x % items;
+      if (w > 0) { seg = 1 + (w - 1) / 3; run = 1 + (w - 1) % 3; }
+    } else {
+      chain = blockIdx.x / (a.seg_G - 1);
+      seg = 1 + blockIdx.x % (a.seg_G - 1);
+    }
+  }
+  const int seq = chain / H, h = chain % H;
+  grid_dependency_wait();   // chunk map, coefficients, T and W (and segment states) come from the previous kernels
+  SeqInfo sq = seq_info(a.g, seq);
+  if (a.seg_G > 0) {        // restrict the view to this segment's chunks
+    const int per = (sq.nchunks + a.seg_G - 1) / a.seg_G;
+    const int cb = min(sq.nchunks, seg * per), ce = min(sq.nchunks, (seg + 1) * per);
+    sq.slot0 += cb;
+    sq.tok0 += cb * C;
+    sq.len = (ce > cb) ? min(sq.len - cb * C, (ce - cb) * C) : 0;
+    sq.nchunks = ce - cb;
+  }
+  const int nch = sq.nchunks;
+  const size_t st_off = (size_t)chain * kD * kD;
+  // ---- where the start state comes from, where the end state goes, whether V counts, whether o is written
+  const float* S0p = a.S0 ? a.S0 + st_off : nullptr;
+  const float* M0p = a.M0 ? a.M0 + st_off : nullptr;
+  float* Sfp = a.Sf ? a.Sf + st_off : nullptr;
+  float* Mfp = a.Mf ? a.Mf + st_off : nullptr;
+  bool id_s = false, id_m = false, v_zero = false, write_o = true;
+  if (a.seg_G > 0) {
+    constexpr size_t kMat = (size_t)kD * kD;
+    auto e_ptr = [&](int gi, int which) { return a.seg_E + (((size_t)chain * (a.seg_G - 1) + gi) * 2 + which) * kMat; };
+    if (run == 0) {
+      if (seg > 0) { S0p = e_ptr(seg - 1, 0); M0p = e_ptr(seg - 1, 1); }
+      if (seg < a.seg_G - 1) {
+        Sfp = (seg == 0) ? e_ptr(0, 0) : nullptr;
+        Mfp = (seg == 0) ? e_ptr(0, 1) : nullptr;
+      }
+    } else {
+      write_o = false;
+      S0p = M0p = nullptr;
+      id_s = run == 2; id_m = run == 3; v_zero = run >= 2;
+      float* base = (run == 1 ? a.seg_Psi : run == 2 ? a.seg_PhiS : a.seg_PhiM) +
+                    (((size_t)chain * (a.seg_G - 2) + (seg - 1)) * 2) * kMat;
+      Sfp = base; Mfp = base + kMat;
+    }
+  }
+
+  const uint32_t s_base = smem_u32(smem);
+  const uint32_t b_full0 = smem_u32(&bars.full[0]), b_full1 = smem_u32(&bars.full[1]);
+  const uint32_t b_go0 = smem_u32(&bars.go[0]), b_go1 = smem_u32(&bars.go[1]);
+  const uint32_t b_kq = smem_u32(&bars.kq), b_adj0 = smem_u32(&bars.adj[0]), b_adj1 = smem_u32(&bars.adj[1]);
+  const uint32_t b_init = smem_u32(&bars.init), b_m1 = smem_u32(&bars.m1), b_r = smem_u32(&bars.r);
+  const uint32_t b_m2 = smem_u32(&bars.m2), b_oi = smem_u32(&bars.oi), b_v1a = smem_u32(&bars.v1a);
+  const uint32_t b_v1b = smem_u32(&bars.v1b), b_mx = smem_u32(&bars.mx), b_m3s = smem_u32(&bars.m3s);
+  const uint32_t b_m3 = smem_u32(&bars.m3), b_mo = smem_u32(&bars.mo), b_zu = smem_u32(&bars.zu);
+  const uint32_t b_fin = smem_u32(&bars.fin);
+
+  if (tid == 0) {
+    abort_flag = 0;
+    mbar_init(b_full0, 1); mbar_init(b_full1, 1);
+    mbar_init(b_go0, kEpiThreads); mbar_init(b_go1, kEpiThreads);
+    mbar_init(b_kq, kCvtThreads); mbar_init(b_adj0, kCvtThreads); mbar_init(b_adj1, kCvtThreads);
+    mbar_init(b_fin, kCvtThreads);
+    mbar_init(b_init, kEpiThreads); mbar_init(b_r, kEpiThreads); mbar_init(b_oi, kEpiThreads);
+    mbar_init(b_v1a, kEpiThreads); mbar_init(b_v1b, kEpiThreads); mbar_init(b_zu, kEpiThreads);
+    mbar_init(b_m1, 1); mbar_init(b_m2, 1); mbar_init(b_m3, 1); mbar_init(b_mo, 1); mbar_init(b_mx, 1); mbar_init(b_m3s, 1);
+    mbar_fence_init();
+  }
+  if (warp == kWarpMma) tmem_alloc(smem_u32(&tmem_slot), 512);
+  if (warp == kWarpTma && lane == 0) {
+    prefetch_tensormap(&map_q); prefetch_tensormap(&map_k); prefetch_tensormap(&map_v);
+    prefetch_tensormap(&map_t); prefetch_tensormap(&map_w); prefetch_tensormap(&map_o);
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem = tmem_slot;
+  bool ok = true;
+  volatile int* abortp = &abort_flag;
+#define MDN_WAIT(bar, par)                         \
+  if (!mbar_wait((bar), (par), abortp)) {          \
+    ok = false;                                    \
+    break;                                         \
+  }
+  // waits on the chain's critical path poll without suspending
+#define MDN_SPIN(bar, par)                         \
+  if (!mbar_wait_spin((bar), (par), abortp)) {     \
+    ok = false;                                    \
+    break;                                         \
+  }
+#ifdef MDN_DEBUG
+  // Stamps go to shared memory (a global store per stamp slows the stamping thread by hundreds of cycles) for the
+  // chunks kTlFirst .. kTlFirst + 7 and are copied out when the kernel ends.
+  long long* const tline = (blockIdx.x == 0) ? a.timeline : nullptr;
+  constexpr int kTlFirst = 16;
+  __shared__ long long tl_sm[8][32];
+#define MDN_MARK(c, ev) \
+  if (tline != nullptr && lane == 0 && (c) >= kTlFirst && (c) < kTlFirst + 8 && \
+      (warp < kWarpEpi || warp == kWarpEpi + 2 || warp >= kWarpCvt)) tl_sm[(c) - kTlFirst][(ev)] = clock64();
+#define MDN_MARK2(c, ev) \
+  if (tline != nullptr && lane == 0 && (c) >= kTlFirst && (c) < kTlFirst + 8 && warp == 7) tl_sm[(c) - kTlFirst][(ev)] = clock64();
+#else
+#define MDN_MARK(c, ev)
+#define MDN_MARK2(c, ev)
+#endif
+
+#ifdef MDN_DEBUG
+  if (tline != nullptr && tid == 0) {   // clock rate of this run: cycle and nanosecond stamps at both ends
+    unsigned long long ns;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ns));
+    tline[30] = clock64(); tline[31] = (long long)ns;
+  }
+#endif
+  if (warp == kWarpTma) {
+    // ================================================================== TMA producer + output stores
+    // Stage s = c & 1 serves chunk c, then (as the staged output tile) is written out and refilled for chunk c + 2.
+    if (lane == 0) {
+      int issued = 0;
+      for (int c = 0; c < nch + 2; ++c) {
+        const int s = c & 1;
+        const uint32_t st = s_base + kOffStage + s * kStageBytes;
+        if (c >= 2) {
+          const int co = c - 2;
+          MDN_WAIT(s ? b_go1 : b_go0, (co >> 1) & 1);
+          const int n = min(C, sq.len - co * C);
+          const int tok0 = sq.tok0 + co * C;
+          const uint32_t src = st + kStOut;
+          if (!write_o) {
+            // Psi / Phi runs of the parallel scan produce states only
+          } else if (n == C) {
+            tma_store_2d(&map_o, h * kD, tok0, src);
+          } else {   // short chunk: rows >= n belong to another sequence; one bulk copy per valid row
+            for (int r = 0; r < n; ++r)
+              bulk_store(static_cast<uint8_t*>(a.o) + (((size_t)(tok0 + r) * H + h) * kD) * sizeof(TO),
+                         src + r * kD * (uint32_t)sizeof(TO), kD * (uint32_t)sizeof(TO));
+          }
+          tma_store_commit();
+          tma_store_wait_read();
+          MDN_MARK(co, kEvStoresDone);
+        }
+        if (c < nch) {
+          const uint32_t fb = s ? b_full1 : b_full0;
+          const int tok0 = sq.tok0 + c * C;
+          const int mat = (sq.slot0 + c) * H + h;
+          mbar_arrive_expect_tx(fb, kTxBytes - (write_o ? 0u : kTxW) - (v_zero ? kTxV : 0u));
+          bulk_load(st + kStCoef, a.coef + (size_t)mat * MDN_NUM_COEF * C, kCoefBytes, fb);
+          if (!v_zero) tma_load_2d(st + kStV, &map_v, h * kD, tok0, fb);
+          tma_load_2d(st + kStT, &map_t, 0, mat * C, fb);
+          if (write_o) {
+            tma_load_2d(st + kStW, &map_w, 0, mat * C, fb);
+            tma_load_2d(st + kStW + 8192, &map_w, 32, mat * C, fb);
+          }
+          tma_load_2d(st + kStK, &map_k, h * kD, tok0, fb);          // for MMA-3 at the end of the chunk (L2 hit)
+          tma_load_2d(st + kStK + 8192, &map_k, h * kD + 64, tok0, fb);
+          MDN_MARK(c, kEvTmaIssued);
+          issued = c + 1;
+        }
+      }
+      if (!ok) {   // giving up: let the copies already in flight land before the CTA exits
+        for (int c = max(0, issued - 2); c < issued; ++c)
+          for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait((c & 1) ? b_full1 : b_full0, (c >> 1) & 1); ++it) {}
+      }
+      tma_store_wait_all();
+    }
+  } else if (warp == kWarpMma) {
+    // ================================================================== MMA issuer
+    // The whole warp walks the loop and waits (warp-uniform control flow and operands: the descriptors can live in
+    // uniform registers); one elected lane issues the products and the commits.
+    {
+      const uint32_t tm = __shfl_sync(0xffffffffu, tmem, 0);
+      const uint32_t sb = __shfl_sync(0xffffffffu, s_base, 0);
+      const bool lead = elect_one();
+      // Column of the bf16 A operands the epilogue leaves in X, Y: K-step k covers tokens 16k .. 16k + 15; the
+      // epilogue warp that owns those tokens keeps hi (part 0) and lo (part 1) inside its own kTok columns
+      auto a_col = [](int part, int k) {
+        return static_cast<uint32_t>(kTok * ((16 * k) / kTok) + kPk * part + ((16 * k) % kTok) / 2);
+      };
+      const uint32_t id64 = idesc_bf16(128, 64, false, false, false);
+      const uint32_t id128_mn = idesc_bf16(128, 128, false, true, false);
+      const uint32_t id128_mn_neg = idesc_bf16(128, 128, false, true, true);
+      const uint32_t id1 = idesc_tf32(128, write_o ? 128 : 64, false, false, false);
+      const uint32_t id64_tf32 = idesc_tf32(128, 64, false, false, false);
+      const uint64_t dKQ = smem_desc_sw128(sb + kOffKQ32, 16, 1024);   // + (j >> 2) * 16384 bytes + (j & 3) * 32 bytes per K step
+      // per stage: T, the two halves of W, the K tile read MN-major (+2048 B per 16 tokens)
+      const uint64_t dT_0 = smem_desc_sw128(sb + kOffStage + kStT, 16, 1024), dT_1 = dT_0 + (kStageBytes >> 4);
+      const uint64_t dW0_0 = smem_desc_sw128(sb + kOffStage + kStW, 16, 1024), dW0_1 = dW0_0 + (kStageBytes >> 4);
+      const uint64_t dKmn_0 = smem_desc_sw128(sb + kOffStage + kStK, 8192, 1024), dKmn_1 = dKmn_0 + (kStageBytes >> 4);
+      for (int c = 0; c < nch; ++c) {
+        const int s = c & 1;
+        const uint32_t ph = c & 1;
+        const uint64_t dT = s ? dT_1 : dT_0, dW0 = s ? dW0_1 : dW0_0, dW1 = dW0 + (8192 >> 4), dKmn = s ? dKmn_1 : dKmn_0;
+        MDN_MARK(c, kEvLoopTop);
+        MDN_SPIN(b_kq, ph);
+        MDN_MARK(c, kEvKqSeen);
+        if (c == 0) MDN_WAIT(b_init, 0);
+        tc_fence_after_sync();
+        MDN_MARK(c, kEvMma1);
+        // ---- MMA-1: [X | Z] = Sh [K; Q]^T, [Y | U] = Mh [K; Q]^T  (state-only runs: X, Y against K alone).  Issued right
+        // behind the previous chunk's updates of Sh, Mh, without waiting for their commits: the tensor pipe runs this
+        // thread's products in issue order, a product that reads another's accumulator (or overwrites another's
+        // operand) included - the probe library's chained-product tests show it.  Commits are for the epilogue.
+        if (lead) {
+#pragma unroll
+          for (int j = 0; j < 16; ++j)
+            umma_ts_tf32(tm + kColX, tm + kColS + 8 * j, dKQ + (uint64_t)((j >> 2) * 1024 + (j & 3) * 2), id1, j > 0);
+          umma_commit(b_mx);
+        }
+        MDN_MARK(c, kEvXzIssued);
+        if (write_o) MDN_SPIN(b_zu, ph ^ 1);   // the previous chunk's output has been read out of U
+        tc_fence_after_sync();
+        if (lead) {
+#pragma unroll
+          for (int j = 0; j < 16; ++j)
+            umma_ts_tf32(tm + kColY, tm + kColM + 8 * j, dKQ + (uint64_t)((j >> 2) * 1024 + (j & 3) * 2), id1, j > 0);
+          umma_commit(b_m1);
+        }
+        MDN_MARK(c, kEvYuIssued);
+        // (T, W and the bf16 K tile of the stage have landed: the converters waited for them before they published the
+        // coefficients the epilogue has used by the time it hands R over)
+        // ---- MMA-2: Y = (R_hi + R_lo)^T T^T
+        MDN_SPIN(b_r, ph);
+        tc_fence_after_sync();
+        MDN_MARK(c, kEvRSeen);
+        if (lead) {
+#pragma unroll
+          for (int k = 0; k < 4; ++k) umma_ts(tm + kColY, tm + kColX + a_col(0, k), dT + 2 * k, id64, k > 0);
+#pragma unroll
+          for (int k = 0; k < 4; ++k) umma_ts(tm + kColY, tm + kColX + a_col(1, k), dT + 2 * k, id64, true);
+          umma_commit(b_m2);
+        }
+        MDN_MARK(c, kEvM2Issued);
+        // ---- MMA-3': U += V~^T W^T, V~ read as tf32 from the accumulator MMA-2 has just filled, W an fp32 tile;
+        // U holds the inter-chunk terms.  Runs while the epilogue makes the state-update operands.
+        if (write_o) {
+          MDN_SPIN(b_oi, ph);
+          tc_fence_after_sync();
+          MDN_MARK(c, kEvM2Own);
+          if (lead) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+              umma_ts_tf32(tm + kColU, tm + kColY + 8 * j, ((j >> 2) ? dW1 : dW0) + 2 * (j & 3), id64_tf32, true);
+            umma_commit(b_mo);
+          }
+          MDN_MARK(c, kEvMoIssued);
+        }
+        // ---- MMA-3: Sh^T += (wS V~)^T K, then Mh^T -= (wM V~)^T K   (K tile read MN-major: N = dk, K = tokens); the
+        // first starts while the epilogue still makes the second one's operand
+        MDN_SPIN(b_v1a, ph);
+        tc_fence_after_sync();
+        MDN_MARK(c, kEvV1Seen);
+        if (lead) {
+#pragma unroll
+          for (int k = 0; k < 8; ++k)
+            umma_ts(tm + kColS, tm + kColX + a_col(k >> 2, k & 3), dKmn + 128 * (k & 3), id128_mn, true);
+          umma_commit(b_m3s);
+        }
+        MDN_MARK(c, kEvSIssued);
+        MDN_SPIN(b_v1b, ph);
+        tc_fence_after_sync();
+        MDN_MARK(c, kEvV1bSeen);
+        if (lead) {
+#pragma unroll
+          for (int k = 0; k < 8; ++k)
+            umma_ts(tm + kColM, tm + kColY + a_col(k >> 2, k & 3), dKmn + 128 * (k & 3), id128_mn_neg, true);
+          umma_commit(b_m3);
+        }
+        MDN_MARK(c, kEvMIssued);
+      }
+    }
+  } else if (warp >= kWarpCvt) {
+    // ================================================================== converter warps
+    // One chunk ahead of the chain: the fp32 copies of the K and Q tiles, then the scalar recurrence of G and the
+    // chunk's six coefficient vectors.
+    const int t = tid - kWarpCvt * 32;   // 0..63: the token whose coefficients this thread writes
+    float g11 = 1.f, g12 = 0.f, g22 = 1.f;
+    // Rows of the K and Q tiles: in step i a warp reads two whole rows (sixteen 16-byte pieces each: coalesced), the two
+    // warps four; row = 4 i + 2 warp + lane / 16, piece = lane % 16.  The fp32 stores of one such step spread evenly
+    // over the banks in the swizzled layout.
+    const int cw = warp - kWarpCvt, piece = lane & 15;
+    const size_t row_stride = (size_t)H * kD;   // elements between consecutive tokens
+    uint4 kq[2][16];
+    auto load_rows = [&](int c) {
+      const long long tok0 = (long long)sq.tok0 + (long long)c * C;
+#pragma unroll
+      for (int which = 0; which < 2; ++which) {
+        const __nv_bfloat16* base = (which ? a.q : a.k) + (size_t)h * kD + piece * 8;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          const long long tok = tok0 + 4 * i + 2 * cw + (lane >> 4);
+          kq[which][i] = make_uint4(0u, 0u, 0u, 0u);
+          if (tok < a.tokens && (which == 0 || write_o)) {
+            // volatile: the loads must be ISSUED here, a chunk ahead of their use, not sunk down to the stores
+            asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+                         : "=r"(kq[which][i].x), "=r"(kq[which][i].y), "=r"(kq[which][i].z), "=r"(kq[which][i].w)
+                         : "l"(base + (size_t)tok * row_stride));
+          }
+        }
+      }
+    };
+    if (nch > 0) load_rows(0);
+    for (int c = 0; c <= nch; ++c) {
+      if (c < nch) {
+        // ---- fp32 copies of this chunk's K and Q tiles (the chain needs them first); the rows are in registers
+        if (c > 0) MDN_WAIT(b_m1, (c - 1) & 1);   // the previous chunk's products have read the fp32 tiles
+        MDN_MARK(c, kEvCvtStart);
+#pragma unroll
+        for (int which = 0; which < 2; ++which) {
+          if (which == 0 || write_o) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              const int row = 4 * i + 2 * cw + (lane >> 4);
+              const uint32_t sw = static_cast<uint32_t>(row & 7);
+              const uint32_t d0 = s_base + kOffKQ32 + (piece >> 2) * 16384 + (which * 64 + row) * 128;
+              const uint32_t ch = static_cast<uint32_t>((piece & 3) * 2);
+              const uint4 u = kq[which][i];
+              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(d0 + ((ch ^ sw) << 4)), "r"(u.x << 16),
+                           "r"(u.x & 0xffff0000u), "r"(u.y << 16), "r"(u.y & 0xffff0000u) : "memory");
+              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(d0 + (((ch + 1) ^ sw) << 4)), "r"(u.z << 16),
+                           "r"(u.z & 0xffff0000u), "r"(u.w << 16), "r"(u.w & 0xffff0000u) : "memory");
+            }
+          }
+          if (which == 0) MDN_MARK(c, kEvM3sOwn);
+        }
+        MDN_MARK(c, kEvEager);
+        fence_proxy_async_smem();
+        mbar_arrive(b_kq);
+        MDN_MARK(c, kEvCvtDone);
+        // ---- the scalar recurrence of G and the chunk's six coefficient vectors
+        float* aj = reinterpret_cast<float*>(smem + kOffAdj + (c & 1) * kAdjBytes);
+        MDN_WAIT((c & 1) ? b_full1 : b_full0, (c >> 1) & 1);
+        const float* cf = reinterpret_cast<const float*>(smem + kOffStage + (c & 1) * kStageBytes + kStCoef);
+        const float aC = cf[kAbar * C + C - 1], bC = cf[kB * C + C - 1], mC = cf[kMubar * C + C - 1];
+        const float n11 = __fmul_rn(aC, g11), n12 = __fsub_rn(__fmul_rn(aC, g12), __fmul_rn(bC, g22)), n22 = __fmul_rn(mC, g22);
+        const bool lazy = n11 >= kLazyMin && n22 >= kLazyMin && fabsf(n12) <= kLazyMix * n22;
+        const float ab = cf[kAbar * C + t], bb = cf[kB * C + t], pp = cf[kAlphaBPrev * C + t];
+        const float gs = cf[kGS * C + t], gm = cf[kGM * C + t];
+        const float cx = ab * g11, cy = pp * g22 - ab * g12;
+        aj[kCx + t] = cx;
+        aj[kCy + t] = cy;
+        aj[kCz + t] = a.scale * cx;
+        aj[kCu + t] = a.scale * (ab * g12 - bb * g22);
+        if (lazy) {
+          aj[kWs + t] = (gs + (n12 / n22) * gm) / n11;
+          aj[kWm + t] = gm / n22;
+        } else {
+          aj[kWs + t] = gs;
+          aj[kWm + t] = gm;
+        }
+        if (t == 0) { aj[kN11] = n11; aj[kN12] = n12; aj[kN22] = n22; aj[kLazy] = lazy ? 1.f : 0.f; }
+        if (lazy) { g11 = n11; g12 = n12; g22 = n22; } else { g11 = 1.f; g12 = 0.f; g22 = 1.f; }
+        mbar_arrive((c & 1) ? b_adj1 : b_adj0);
+        // the next chunk's rows: in flight while the chain works on this chunk (issued last: nothing this thread
+        // still has to do for the current chunk may queue up behind thirty-two outstanding loads)
+        if (c + 1 < nch) load_rows(c + 1);
+      } else {
+        if (t == 0) { g_final[0] = g11; g_final[1] = g12; g_final[2] = g22; }
+        mbar_arrive(b_fin);
+      }
+    }
+  } else {
+    // ================================================================== epilogue warps
+    // lane quarter q4 = warp & 3 (value columns 32 q4 .. +31 = this warp's tensor-memory lanes),
+    // token half hf = warp >> 2 (tokens 32 hf .. +31 in the per-token steps, dk columns 64 hf .. +63 of the masters)
+    const int q4 = warp & 3, hf = (warp - kWarpEpi) >> 2;
+    const int d = q4 * 32 + lane;
+    const int r0 = kTok * hf;
+    const uint32_t tl = tmem + (static_cast<uint32_t>(q4 * 32) << 16);
+
+    for (int c = 0; c <= nch; ++c) {
+      const float* aj = reinterpret_cast<const float*>(smem + kOffAdj + (c & 1) * kAdjBytes);
+      if (c == 0) {
+        // ---------------- the start state into the masters
+#pragma unroll 1
+        for (int i = 0; i < 2; ++i) {
+          const int col0 = hf * 64 + i * 32;
+          uint32_t sr[32], mr[32];
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            const float unit = (col0 + j == d) ? 1.f : 0.f;
+            sr[j] = __float_as_uint(S0p ? __ldg(S0p + (size_t)(col0 + j) * kD + d) : (id_s ? unit : 0.f));
+            mr[j] = __float_as_uint(M0p ? __ldg(M0p + (size_t)(col0 + j) * kD + d) : (id_m ? unit : 0.f));
+          }
+          tmem_st32(tl + kColS + col0, sr);
+          tmem_st32(tl + kColM + col0, mr);
+        }
+        tmem_wait_st();
+        tc_fence_before_sync();
+        mbar_arrive(b_init);
+      }
+      if (c == nch) {
+        // ---------------- final states: [S; M] = G [Sh; Mh]  (the last chunk's MMA-3 was waited for below)
+        MDN_WAIT(b_fin, 0);
+        const float g11 = g_final[0], g12 = g_final[1], g22 = g_final[2];
+        tc_fence_after_sync();
+#pragma unroll 1
+        for (int i = 0; i < 2; ++i) {
+          const int col0 = hf * 64 + i * 32;
+          uint32_t sr[32], mr[32];
+          tmem_ld32(tl + kColS + col0, sr);
+          tmem_ld32(tl + kColM + col0, mr);
+          tmem_wait_ld();
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            const float sv = __uint_as_float(sr[j]), mv = __uint_as_float(mr[j]);
+            if (Sfp) Sfp[(size_t)(col0 + j) * kD + d] = g11 * sv + g12 * mv;
+            if (Mfp) Mfp[(size_t)(col0 + j) * kD + d] = g22 * mv;
+          }
+        }
+        break;
+      }
+      const uint32_t ph = c & 1;
+      uint8_t* stg = smem + kOffStage + (c & 1) * kStageBytes;
+      const __nv_bfloat16* sV = reinterpret_cast<const __nv_bfloat16*>(stg + kStV);
+      MDN_WAIT((c & 1) ? b_full1 : b_full0, (c >> 1) & 1);
+      MDN_WAIT((c & 1) ? b_adj1 : b_adj0, (c >> 1) & 1);
+      // ---------------- EPI-1: R^T = V^T - cX .* X + cY .* Y  -> bf16 hi, lo in X
+      {
+        // V and the coefficients are fetched BEFORE the waits: shared-memory loads issued after a wait would sit on the
+        // chain's critical path, behind whatever the converter warps have queued in the shared-memory pipe
+        float vv[kTok], cf1[kTok];
+#pragma unroll
+        for (int j = 0; j < kTok; ++j) vv[j] = v_zero ? 0.f : __bfloat162float(sV[(r0 + j) * kD + d]);
+#pragma unroll
+        for (int j = 0; j < kTok; j += 4) {
+          const float4 cx = *reinterpret_cast<const float4*>(aj + kCx + r0 + j);
+          cf1[j] = cx.x; cf1[j + 1] = cx.y; cf1[j + 2] = cx.z; cf1[j + 3] = cx.w;
+        }
+        MDN_WAIT(b_mx, ph);          // X is there; Y is still being computed
+        __syncwarp();
+        tc_fence_after_sync();
+        {
+          uint32_t x[kTok];
+          tmem_ld32(tl + kColX + r0, x);
+          tmem_wait_ld();
+#pragma unroll
+          for (int j = 0; j < kTok; ++j) vv[j] -= cf1[j] * __uint_as_float(x[j]);
+        }
+#pragma unroll
+        for (int j = 0; j < kTok; j += 4) {
+          const float4 cy = *reinterpret_cast<const float4*>(aj + kCy + r0 + j);
+          cf1[j] = cy.x; cf1[j + 1] = cy.y; cf1[j + 2] = cy.z; cf1[j + 3] = cy.w;
+        }
+        MDN_WAIT(b_m1, ph);
+        __syncwarp();
+        tc_fence_after_sync();
+        MDN_MARK(c, kEvM1Seen);
+        uint32_t hi[kPk], lo[kPk];
+        {
+          uint32_t y[kTok];
+          tmem_ld32(tl + kColY + r0, y);
+          tmem_wait_ld();
+#pragma unroll
+          for (int j = 0; j < kTok; j += 4) {
+            const float e0 = vv[j + 0] + cf1[j + 0] * __uint_as_float(y[j + 0]);
+            const float e1 = vv[j + 1] + cf1[j + 1] * __uint_as_float(y[j + 1]);
+            const float e2 = vv[j + 2] + cf1[j + 2] * __uint_as_float(y[j + 2]);
+            const float e3 = vv[j + 3] + cf1[j + 3] * __uint_as_float(y[j + 3]);
+            split_pack_bf16(e0, e1, hi[j >> 1], lo[j >> 1]);
+            split_pack_bf16(e2, e3, hi[(j >> 1) + 1], lo[(j >> 1) + 1]);
+          }
+        }
+        // hi and lo both go into the columns this warp has just read (its own kTok columns of X)
+        tmem_st16(tl + kColX + r0, hi);
+        tmem_st16(tl + kColX + r0 + kPk, lo);
+        tmem_wait_st();
+      }
+      tc_fence_before_sync();
+      mbar_arrive(b_r);
+      MDN_MARK(c, kEvRArrive);
+      MDN_MARK2(c, kEvRArrive2);
+      // ---------------- inter-chunk output terms cZ .* Z + cU .* U, left in U for MMA-3' to accumulate onto (under MMA-2)
+      if (write_o) {
+        uint32_t z[kTok], u[kTok];
+        tmem_ld32(tl + kColZ + r0, z);
+        tmem_ld32(tl + kColU + r0, u);
+        float cz[kTok], cu[kTok];   // (their loads run while the tensor-memory loads are in flight)
+#pragma unroll
+        for (int j = 0; j < kTok; j += 4) {
+          const float4 a4 = *reinterpret_cast<const float4*>(aj + kCz + r0 + j);
+          const float4 b4 = *reinterpret_cast<const float4*>(aj + kCu + r0 + j);
+          cz[j] = a4.x; cz[j + 1] = a4.y; cz[j + 2] = a4.z; cz[j + 3] = a4.w;
+          cu[j] = b4.x; cu[j + 1] = b4.y; cu[j + 2] = b4.z; cu[j + 3] = b4.w;
+        }
+        tmem_wait_ld();
+#pragma unroll
+        for (int j = 0; j < kTok; ++j) u[j] = __float_as_uint(cz[j] * __uint_as_float(z[j]) + cu[j] * __uint_as_float(u[j]));
+        tmem_st32(tl + kColU + r0, u);
+        tmem_wait_st();
+        tc_fence_before_sync();
+        mbar_arrive(b_oi);
+        MDN_MARK(c, kEvOiArrive);
+      }
+      // ---------------- EPI-2: wS .* V~ -> X (handed over first), wM .* V~ -> Y, each as bf16 hi, lo.  V~ itself stays
+      // in Y for MMA-3' until that product has read it.  Eager chunks: the masters take G' = D_c G here (MMA-1 of this
+      // chunk, their last reader, is done) and the update is added in true coordinates.
+      const bool eager = aj[kLazy] == 0.f;
+      const float n11 = aj[kN11], n12 = aj[kN12], n22 = aj[kN22];
+      float wsv[kTok], wmv[kTok];   // fetched before the wait, as in EPI-1
+#pragma unroll
+      for (int j = 0; j < kTok; j += 4) {
+        const float4 a4 = *reinterpret_cast<const float4*>(aj + kWs + r0 + j);
+        const float4 b4 = *reinterpret_cast<const float4*>(aj + kWm + r0 + j);
+        wsv[j] = a4.x; wsv[j + 1] = a4.y; wsv[j + 2] = a4.z; wsv[j + 3] = a4.w;
+        wmv[j] = b4.x; wmv[j + 1] = b4.y; wmv[j + 2] = b4.z; wmv[j + 3] = b4.w;
+      }
+      MDN_WAIT(b_m2, ph);
+      __syncwarp();
+      tc_fence_after_sync();
+      MDN_MARK(c, kEvM2Seen);
+      {
+        uint32_t vt[kTok];
+        tmem_ld32(tl + kColY + r0, vt);
+        tmem_wait_ld();
+        {
+          uint32_t sh[kPk], sl[kPk];
+#pragma unroll
+          for (int j = 0; j < kTok; j += 4) {
+            split_pack_bf16(wsv[j] * __uint_as_float(vt[j]), wsv[j + 1] * __uint_as_float(vt[j + 1]), sh[j >> 1], sl[j >> 1]);
+            split_pack_bf16(wsv[j + 2] * __uint_as_float(vt[j + 2]), wsv[j + 3] * __uint_as_float(vt[j + 3]), sh[(j >> 1) + 1],
+                            sl[(j >> 1) + 1]);
+          }
+          tmem_st16(tl + kColX + r0, sh);          // X is free: MMA-2 has consumed R
+          tmem_st16(tl + kColX + r0 + kPk, sl);
+        }
+        if (eager) {   // Sh <- n11 Sh + n12 Mh (Mh still the old one)
+          MDN_MARK(c, kEvEager);
+#pragma unroll 1
+          for (int i = 0; i < 2; ++i) {
+            const int col0 = hf * 64 + i * 32;
+            uint32_t sr[32], mr[32];
+            tmem_ld32(tl + kColS + col0, sr);
+            tmem_ld32(tl + kColM + col0, mr);
+            tmem_wait_ld();
+#pragma unroll
+            for (int j = 0; j < 32; ++j) sr[j] = __float_as_uint(n11 * __uint_as_float(sr[j]) + n12 * __uint_as_float(mr[j]));
+            tmem_st32(tl + kColS + col0, sr);
+          }
+        }
+        tmem_wait_st();
+        tc_fence_before_sync();
+        mbar_arrive(b_v1a);
+        MDN_MARK(c, kEvV1Arrive);
+        MDN_MARK2(c, kEvV1Arrive2);
+        uint32_t mh[kPk], mlo[kPk];
+#pragma unroll
+        for (int j = 0; j < kTok; j += 4) {
+          split_pack_bf16(wmv[j] * __uint_as_float(vt[j]), wmv[j + 1] * __uint_as_float(vt[j + 1]), mh[j >> 1], mlo[j >> 1]);
+          split_pack_bf16(wmv[j + 2] * __uint_as_float(vt[j + 2]), wmv[j + 3] * __uint_as_float(vt[j + 3]), mh[(j >> 1) + 1],
+                          mlo[(j >> 1) + 1]);
+        }
+        if (write_o) {   // MMA-3' reads V~ from Y: it must be done before Y is overwritten
+          MDN_WAIT(b_mo, ph);
+          __syncwarp();
+          tc_fence_after_sync();
+        }
+        tmem_st16(tl + kColY + r0, mh);          // own columns of Y
+        tmem_st16(tl + kColY + r0 + kPk, mlo);
+      }
+      if (eager) {   // Mh <- n22 Mh
+#pragma unroll 1
+        for (int i = 0; i < 2; ++i) {
+          const int col0 = hf * 64 + i * 32;
+          uint32_t mr[32];
+          tmem_ld32(tl + kColM + col0, mr);
+          tmem_wait_ld();
+#pragma unroll
+          for (int j = 0; j < 32; ++j) mr[j] = __float_as_uint(n22 * __uint_as_float(mr[j]));
+          tmem_st32(tl + kColM + col0, mr);
+        }
+      }
+      tmem_wait_st();
+      tc_fence_before_sync();
+      mbar_arrive(b_v1b);
+      MDN_MARK(c, kEvV1bArrive);
+      // ---------------- the chunk's output tile (under MMA-3): U -> [64 x 128] tile in the stage's Q / V area
+      if (write_o) {   // (MMA-3' was waited for above)
+        uint32_t u[kTok];
+        tmem_ld32(tl + kColU + r0, u);
+        tmem_wait_ld();
+        tc_fence_before_sync();
+        mbar_arrive(b_zu);
+        MDN_MARK(c, kEvZuArrive);
+#pragma unroll
+        for (int j = 0; j < kTok; ++j) stage_o<TO>(stg + kStOut, r0 + j, d, __uint_as_float(u[j]));
+        fence_proxy_async_smem();
+        MDN_MARK(c, kEvOutDone);
+      }
+      // the stage may be refilled once MMA-3, the last reader of its K tile, is done
+      MDN_WAIT(b_m3, ph);
+      MDN_MARK(c, kEvM3Seen);
+      mbar_arrive((c & 1) ? b_go1 : b_go0);
+    }
+  }
+#undef MDN_WAIT
+#undef MDN_SPIN
+#undef MDN_MARK
+#undef MDN_MARK2
+
+  if (!ok && lane == 0) atomicCAS(a.status, kDevOk, kDevTimeout);
+  tc_fence_before_sync();
+  __syncthreads();
+#ifdef MDN_DEBUG
+  if (tline != nullptr && tid == 0) {
+    unsigned long long ns;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ns));
+    tline[62] = clock64(); tline[63] = (long long)ns;
+  }
+  if (tline != nullptr && tid < 256) tline[(kTlFirst + (tid >> 5)) * 32 + (tid & 31)] = (tid & 31) < 30 ? tl_sm[tid >> 5][tid & 31] : 0;
+#endif
+  if (warp == kWarpMma) tmem_dealloc(tmem, 512);
+}
+
+}  // namespace
+
+cudaError_t launch_chain_tf32(const Plan& pl, const void* q, const void* k, const void* v, const float* S0,
+                              const float* M0, void* o, float* Sf, float* Mf, int* launches) {
+  const mdn_params& p = pl.p;
+  const uint64_t tokens = (uint64_t)p.B * p.T;
+  const uint64_t mats = (uint64_t)pl.geom.num_slots * p.H;
+  CUtensorMap mq, mk, mv, mt, mw, mo;
+  const uint64_t row = (uint64_t)p.H * kD;
+  if (!encode_tma_2d_bf16(&mq, TmaMap2D{q, row, tokens, row * 2, 64, 64, true}) ||
+      !encode_tma_2d_bf16(&mk, TmaMap2D{k, row, tokens, row * 2, 64, 64, true}) ||
+      !encode_tma_2d_bf16(&mv, TmaMap2D{v, row, tokens, row * 2, 128, 64, false}) ||
+      !encode_tma_2d_bf16(&mt, TmaMap2D{pl.ws + pl.lay.off_T, 64, mats * C, 128, 64, 64, true}) ||
+      !encode_tma_2d(&mw, TmaMap2D{pl.ws + pl.lay.off_W, 64, mats * C, 256, 32, 64, true}, true))
+    return cudaErrorInvalidValue;
+  const bool o_bf16 = p.o_dtype == MDN_BF16;
+  if (!encode_tma_2d(&mo, TmaMap2D{o, row, tokens, row * (o_bf16 ? 2u : 4u), 128, 64, false}, !o_bf16))
+    return cudaErrorInvalidValue;
+  Args a;
+  a.g = pl.geom;
+  a.coef = reinterpret_cast<const float*>(pl.ws + pl.lay.off_coef);
+  a.q = static_cast<const __nv_bfloat16*>(q); a.k = static_cast<const __nv_bfloat16*>(k); a.tokens = (long long)tokens;
+  a.S0 = S0; a.M0 = M0; a.o = o; a.Sf = Sf; a.Mf = Mf;
+  a.status = reinterpret_cast<int32_t*>(pl.ws + pl.lay.off_status);
+  a.scale = p.scale;
+  a.seg_G = 0; a.seg_phase = 0;
+  a.seg_E = a.seg_Psi = a.seg_PhiS = a.seg_PhiM = nullptr;
+  a.timeline = nullptr;
+#ifdef MDN_DEBUG   // debug builds only (-DMDN_DEBUG): the product library reads nothing from the environment
+  const char* tl = getenv("MDN_DEBUG_TIMELINE");   // device address of an int64 buffer, [chunks][32]
+  a.timeline = tl ? reinterpret_cast<long long*>(strtoull(tl, nullptr, 0)) : nullptr;
+#endif
+  const unsigned chains = (unsigned)pl.geom.num_seqs * p.H;
+  auto launch = [&](unsigned grid) -> cudaError_t {
+    auto kern = o_bf16 ? chain_tf32_kernel<__nv_bfloat16> : chain_tf32_kernel<float>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    if (e != cudaSuccess) return e;
+    e = launch_pdl(kern, dim3(grid), dim3(kThreads), kSmemBytes, pl.stream, a, mq, mk, mv, mt, mw, mo);
+    if (e == cudaSuccess) e = cudaGetLastError();
+    if (e == cudaSuccess) ++*launches;
+    return e;
+  };
+  const int G = pl.lay.segments;
+  if (G <= 1) return launch(chains);
+
+  // ---- parallel inter-chunk scan: Psi / Phi of the middle segments, serial combine, then all segments for real
+  constexpr size_t kMat = (size_t)kD * kD;
+  float* seg = reinterpret_cast<float*>(pl.ws + pl.lay.off_seg);
+  a.seg_G = G;
+  a.seg_E = seg;
+  a.seg_Psi = a.seg_E + (size_t)chains * (G - 1) * 2 * kMat;
+  a.seg_PhiS = a.seg_Psi + (size_t)chains * (G - 2) * 2 * kMat;
+  a.seg_PhiM = a.seg_PhiS + (size_t)chains * (G - 2) * 2 * kMat;
+  a.seg_phase = 1;
+  cudaError_t e = launch(chains * (1 + 3 * (G - 2)));
+  if (e != cudaSuccess) return e;
+  e = launch_seg_combine(pl, G, a.seg_E, a.seg_Psi, a.seg_PhiS, a.seg_PhiM, launches);
+  if (e != cudaSuccess) return e;
+  a.seg_phase = 3;
+  return launch(chains * (G - 1));
+}
+
+}  // namespace mdn

@@ -131,7 +131,9 @@ __device__ __forceinline__ void load16x2(uint32_t ta, float (&x)[16], uint32_t t
   for (int j = 0; j < 16; ++j) { x[j] = __uint_as_float(u[j]); y[j] = __uint_as_float(w[j]); }
 }
 
-template <bool kQk>
+// kWf32: W leaves as one fp32 matrix (what the kind::tf32 output product of chain_tf32.cu reads) instead of the bf16
+// hi + lo pair; same bytes, same staging area.
+template <bool kQk, bool kWf32>
 __global__ void __launch_bounds__(kThreads, kQk ? 4 : kCtasPerSm) intra_mma_kernel(ChunkGeom g, const __grid_constant__ CUtensorMap map_q,
                                                             const __grid_constant__ CUtensorMap map_k,
                                                             float* __restrict__ coef, GateArgs gates, GateParam gp,
@@ -385,10 +387,13 @@ __global__ void __launch_bounds__(kThreads, kQk ? 4 : kCtasPerSm) intra_mma_kern
   } else {
     uint8_t* w_hi = smem + kOffWh + r * 128;
     uint8_t* w_lo = smem + kOffWl + r * 128;
+    uint8_t* w_f32 = smem + kOffWh + r * 256;   // fp32 staging: [64] rows of 256 B, 16-byte pieces XOR-swizzled with (row % 8)
 #pragma unroll
     for (int cb = 0; cb < 4; ++cb) {
       uint4 hi4[2] = {make_uint4(0u, 0u, 0u, 0u), make_uint4(0u, 0u, 0u, 0u)};
       uint4 lo4[2] = {make_uint4(0u, 0u, 0u, 0u), make_uint4(0u, 0u, 0u, 0u)};
+      float4 wf[4] = {make_float4(0.f, 0.f, 0.f, 0.f), make_float4(0.f, 0.f, 0.f, 0.f), make_float4(0.f, 0.f, 0.f, 0.f),
+                      make_float4(0.f, 0.f, 0.f, 0.f)};
       if (cb < reach) {
         float x[16];
         if constexpr (kQk) {   // (q_r - d k_r) . k_i / |k_i|; this row of K K^T is in the second product
@@ -406,19 +411,29 @@ __global__ void __launch_bounds__(kThreads, kQk ? 4 : kCtasPerSm) intra_mma_kern
         float w[16];
 #pragma unroll
         for (int j = 0; j < 16; ++j) w[j] = kQk ? rn_r * f[cb * 16 + j] * x[j] : f[cb * 16 + j] * x[j];
+        if constexpr (kWf32) {
 #pragma unroll
-        for (int hf = 0; hf < 2; ++hf) {
-          split_pack_bf16(w[hf * 8 + 0], w[hf * 8 + 1], hi4[hf].x, lo4[hf].x);
-          split_pack_bf16(w[hf * 8 + 2], w[hf * 8 + 3], hi4[hf].y, lo4[hf].y);
-          split_pack_bf16(w[hf * 8 + 4], w[hf * 8 + 5], hi4[hf].z, lo4[hf].z);
-          split_pack_bf16(w[hf * 8 + 6], w[hf * 8 + 7], hi4[hf].w, lo4[hf].w);
+          for (int p4 = 0; p4 < 4; ++p4) wf[p4] = make_float4(w[p4 * 4], w[p4 * 4 + 1], w[p4 * 4 + 2], w[p4 * 4 + 3]);
+        } else {
+#pragma unroll
+          for (int hf = 0; hf < 2; ++hf) {
+            split_pack_bf16(w[hf * 8 + 0], w[hf * 8 + 1], hi4[hf].x, lo4[hf].x);
+            split_pack_bf16(w[hf * 8 + 2], w[hf * 8 + 3], hi4[hf].y, lo4[hf].y);
+            split_pack_bf16(w[hf * 8 + 4], w[hf * 8 + 5], hi4[hf].z, lo4[hf].z);
+            split_pack_bf16(w[hf * 8 + 6], w[hf * 8 + 7], hi4[hf].w, lo4[hf].w);
+          }
         }
       }
+      if constexpr (kWf32) {
 #pragma unroll
-      for (int hf = 0; hf < 2; ++hf) {
-        const int sw = ((cb * 2 + hf) ^ (r & 7)) * 16;
-        *reinterpret_cast<uint4*>(w_hi + sw) = hi4[hf];
-        *reinterpret_cast<uint4*>(w_lo + sw) = lo4[hf];
+        for (int p4 = 0; p4 < 4; ++p4) *reinterpret_cast<float4*>(w_f32 + (((cb * 4 + p4) ^ (r & 7)) * 16)) = wf[p4];
+      } else {
+#pragma unroll
+        for (int hf = 0; hf < 2; ++hf) {
+          const int sw = ((cb * 2 + hf) ^ (r & 7)) * 16;
+          *reinterpret_cast<uint4*>(w_hi + sw) = hi4[hf];
+          *reinterpret_cast<uint4*>(w_lo + sw) = lo4[hf];
+        }
       }
     }
   }
@@ -428,10 +443,19 @@ __global__ void __launch_bounds__(kThreads, kQk ? 4 : kCtasPerSm) intra_mma_kern
     tc_fence_after_sync();
     tmem_dealloc(tmem, kTmemCols);
   }
-  for (int idx = tid; idx < C * 8; idx += kThreads) {   // coalesced 16-byte stores of W_hi, W_lo
-    const int rr = idx >> 3, c = idx & 7, sw = rr * 128 + ((c ^ (rr & 7)) * 16);
-    *reinterpret_cast<uint4*>(Wout + mat + rr * C + c * 8) = *reinterpret_cast<const uint4*>(smem + kOffWh + sw);
-    *reinterpret_cast<uint4*>(Wout + w_lo_offset + mat + rr * C + c * 8) = *reinterpret_cast<const uint4*>(smem + kOffWl + sw);
+  if constexpr (kWf32) {
+    float* Wf = reinterpret_cast<float*>(Wout);   // [slot][H][64][64] fp32
+    for (int idx = tid; idx < C * 16; idx += kThreads) {   // coalesced 16-byte stores
+      const int rr = idx >> 4, c = idx & 15;
+      *reinterpret_cast<uint4*>(Wf + mat + rr * C + c * 4) =
+          *reinterpret_cast<const uint4*>(smem + kOffWh + rr * 256 + ((c ^ (rr & 7)) * 16));
+    }
+  } else {
+    for (int idx = tid; idx < C * 8; idx += kThreads) {   // coalesced 16-byte stores of W_hi, W_lo
+      const int rr = idx >> 3, c = idx & 7, sw = rr * 128 + ((c ^ (rr & 7)) * 16);
+      *reinterpret_cast<uint4*>(Wout + mat + rr * C + c * 8) = *reinterpret_cast<const uint4*>(smem + kOffWh + sw);
+      *reinterpret_cast<uint4*>(Wout + w_lo_offset + mat + rr * C + c * 8) = *reinterpret_cast<const uint4*>(smem + kOffWl + sw);
+    }
   }
   __syncthreads();   // staging read out: T takes its place
 
@@ -522,13 +546,13 @@ __global__ void __launch_bounds__(kThreads, kQk ? 4 : kCtasPerSm) intra_mma_kern
 
 }  // namespace
 
-template <bool kQk>
+template <bool kQk, bool kWf32>
 static cudaError_t launch_intra_variant(const Plan& pl, const CUtensorMap& mq, const CUtensorMap& mk, const GateArgs& gates,
                                         size_t n_mats) {
   constexpr uint32_t smem_bytes = lay_of(kQk).smem;
-  cudaError_t e = cudaFuncSetAttribute(intra_mma_kernel<kQk>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
+  cudaError_t e = cudaFuncSetAttribute(intra_mma_kernel<kQk, kWf32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
   if (e != cudaSuccess) return e;
-  return launch_pdl(intra_mma_kernel<kQk>, dim3((unsigned)n_mats), dim3(kThreads), smem_bytes, pl.stream, pl.geom, mq, mk,
+  return launch_pdl(intra_mma_kernel<kQk, kWf32>, dim3((unsigned)n_mats), dim3(kThreads), smem_bytes, pl.stream, pl.geom, mq, mk,
                     reinterpret_cast<float*>(pl.ws + pl.lay.off_coef), gates, pl.gp, pl.qk, pl.p.scale,
                     reinterpret_cast<__nv_bfloat16*>(pl.ws + pl.lay.off_T),
                     reinterpret_cast<__nv_bfloat16*>(pl.ws + pl.lay.off_W), n_mats * C * C,
@@ -542,8 +566,10 @@ cudaError_t launch_intra_mma(const Plan& pl, const void* q, const void* k, const
   if (!encode_tma_2d_bf16(&mq, TmaMap2D{q, row, tokens, row * 2, 64, 64, true}) ||
       !encode_tma_2d_bf16(&mk, TmaMap2D{k, row, tokens, row * 2, 64, 64, true}))
     return cudaErrorInvalidValue;
-  cudaError_t e = pl.qk.on ? launch_intra_variant<true>(pl, mq, mk, gates, n_mats)
-                           : launch_intra_variant<false>(pl, mq, mk, gates, n_mats);
+  if (pl.qk.on && pl.w_f32) return cudaErrorInvalidValue;   // the fp32 W serves the plain forward only
+  cudaError_t e = pl.qk.on ? launch_intra_variant<true, false>(pl, mq, mk, gates, n_mats)
+                  : pl.w_f32 ? launch_intra_variant<false, true>(pl, mq, mk, gates, n_mats)
+                             : launch_intra_variant<false, false>(pl, mq, mk, gates, n_mats);
   if (e == cudaSuccess) e = cudaGetLastError();
   if (e == cudaSuccess) ++*launches;
   return e;

@@ -155,9 +155,11 @@ mdn_status mdn_intra_chunk(const mdn_params* p, const void* q, const void* k, co
 
 // The forward proper on a finished plan (chunk map, scan, intra-chunk stage, chain); pl.gp / pl.qk / pl.post say
 // which layer operations the kernels absorb.
-static mdn_status run_forward(const Plan& pl, const void* q, const void* k, const void* v, const float* beta,
+static mdn_status run_forward(const Plan& plan, const void* q, const void* k, const void* v, const float* beta,
                               const float* log_alpha, const float* log_mu, const float* eta, const float* initial_S,
                               const float* initial_M, void* o, float* final_S, float* final_M) {
+  Plan pl = plan;
+  pl.w_f32 = chain_uses_tf32_kernel(pl);   // the plain forward's chain kernel reads W as fp32
   if (!q || !k || !v || !o) return MDN_ERR_INVALID_ARG;
   if (!aligned(q, 16) || !aligned(k, 16) || !aligned(v, 16) || !aligned(o, 16)) return MDN_ERR_INVALID_ARG;
   if ((initial_S && !aligned(initial_S, 16)) || (initial_M && !aligned(initial_M, 16)) ||

@@ -147,6 +147,8 @@ struct Plan {
   const ChunkGeom* chain_mirror_geom = nullptr;   // q, k, o belong to this geometry, walked in reverse chunk order
   const char* chain_mirror_T = nullptr;           // ... and T ([slot][H][64][64] bf16 of that problem), used transposed
   int cu_total_may_be_short = 0;   // packed: cu[N] <= T instead of == T (the adjoint chain's padded problem)
+  bool w_f32 = false;              // tensor path: the intra-chunk kernel writes W as fp32 (chain_tf32.cu reads it so)
+                                   // instead of the bf16 hi + lo pair of chain_tensor.cu
 };
 
 // Launchers (one per .cu file).  Each returns the CUDA error of its launches and adds
@@ -184,6 +186,12 @@ cudaError_t launch_intra_mma(const Plan& pl, const void* q, const void* k, const
 cudaError_t launch_chain_tensor(const Plan& pl, const void* q, const void* k, const void* v,
                                 const float* S0, const float* M0, void* o, float* Sf, float* Mf,
                                 int* launches);
+// chain_tf32.cu: the plain forward's chain kernel (no layer operations, no training options); expects an fp32 W
+cudaError_t launch_chain_tf32(const Plan& pl, const void* q, const void* k, const void* v,
+                              const float* S0, const float* M0, void* o, float* Sf, float* Mf,
+                              int* launches);
+// True when a plan's chain runs in chain_tf32.cu (decided before the intra-chunk stage, which then writes W as fp32).
+bool chain_uses_tf32_kernel(const Plan& pl);
 // Segment bookkeeping of the parallel inter-chunk scan: per chain (G-1) states E, (G-2) Psi and 2 (G-2) Phi
 // halves, each a pair of [dk x dv] fp32 matrices.
 size_t seg_scratch_bytes(const mdn_params& p, int segments);

@@ -35,12 +35,23 @@ mdn_status mdn_selftest_umma(int32_t mode, const void* a, const void* b, float* 
  *   mode 1: out[128 x 128] = a[128 x 64]  * b[64 x 128]       (B read MN-major from the same block layout)
  *   mode 2: out[128 x 64]  = (a * b^T) * c[64 x 64]^T, the second product issued right behind the first, whose
  *           accumulator it reads as its A operand;  mode 3: the same with a commit + wait in between
+ *   mode 9: out[128 x 64] = a * b^T while a second product, issued right behind the first, overwrites the columns the
+ *           first one reads its A operand from (write-after-read through the pipe)
+ *   mode 8: stamps of the issuing thread around commits, waits and fences (out[0..19], cycles)
  *   mode 4..7: timings, out[0] = cycles from first issue to completion, out[1] = products issued
  *           (4: tf32 N = 64 A in tensor memory; 5: tf32 N = 128 MN-major B; 6: bf16 N = 64 A in shared memory;
  *            7: as 4 with a commit + wait after every 16 products)
  */
 mdn_status mdn_probe_tf32(int32_t mode, const float* a, const float* b, const float* c, float* out, int32_t* status,
                           void* cuda_stream);
+
+/*
+ * Cost of one tcgen05 product as a function of its shape: a stream of 4 * reps products D[128 x n] += A[128 x K] *
+ * B[n x K]^T (K = 16 bf16 or 8 tf32 elements), A from tensor memory (a_tmem) or from shared memory, issued by one
+ * thread; out[0] = cycles from the first issue to completion, out[1] = products issued.  n in {32, 64, 128, 256}.
+ */
+mdn_status mdn_probe_mma_timing(int32_t tf32, int32_t a_tmem, int32_t n, int32_t reps, float* out, int32_t* status,
+                                void* cuda_stream);
 
 /*
  * One CTA waits on an mbarrier nothing arrives at, with the poll limit given (1 .. 2^20): the wait runs out,

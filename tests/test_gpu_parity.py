@@ -367,12 +367,17 @@ def test_state_handoff_and_determinism_tensor_path(mdn):
     for name in ("q", "k", "v", "beta", "log_alpha", "log_mu", "eta"):
         a[name] = inp[name][:, :256]; b[name] = inp[name][:, 256:]
     a["workload"] = b["workload"] = dataclasses.replace(w, T=256)
-    oa, Sa, Ma = run_gpu(mdn, a, path="tensor")
+    o, S, M = run_gpu(mdn, inp, path="tensor", o_dtype=torch.float32)
+    oa, Sa, Ma = run_gpu(mdn, a, path="tensor", o_dtype=torch.float32)
     b["S0"], b["M0"] = Sa.astype(np.float32), Ma.astype(np.float32)
-    ob, Sb, Mb = run_gpu(mdn, b, path="tensor")
-    # the split falls on a chunk boundary and the state is handed over in fp32: same arithmetic
-    assert np.array_equal(o[:, :256], oa) and np.array_equal(o[:, 256:], ob)
-    assert np.array_equal(S, Sb) and np.array_equal(M, Mb)
+    ob, Sb, Mb = run_gpu(mdn, b, path="tensor", o_dtype=torch.float32)
+    # the split falls on a chunk boundary and the state is handed over in fp32.  The first half is the same
+    # arithmetic; the second half starts from the true state where the single call carries a lazily scaled one
+    # (chain_tf32.cu), so it agrees to fp32 / tf32 rounding, not bit for bit
+    assert np.array_equal(o[:, :256], oa)
+    rms = lambda x: np.sqrt(np.mean(x ** 2))
+    assert np.abs(o[:, 256:] - ob).max() <= 2e-3 * rms(o)
+    assert np.abs(S - Sb).max() <= 2e-3 * rms(S) and np.abs(M - Mb).max() <= 2e-3 * rms(M)
 
 
 def test_packed_varlen_edge_lengths(mdn):
