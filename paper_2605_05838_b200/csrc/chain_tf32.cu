@@ -48,21 +48,23 @@ using namespace tc;
 
 constexpr int kD = 128;
 constexpr int kEpiWarps = 8, kTok = 32, kPk = 16;
-// Warp roles.  The hardware schedulers favour the older (lower-numbered) of their ready warps, and the MMA issuer must
-// never wait for an issue slot behind an epilogue warp that is busy with arithmetic (measured: as the youngest warp of
-// its scheduler it reacted 500-800 cycles late to every hand-over that fell into an epilogue step).  So: warp 0 MMA
-// issuer, warp 1 TMA producer, warps 2..9 epilogue (lane quarter = warp % 4, as tensor memory demands), warps 10 and 11
-// converters (the youngest on the two schedulers that hold neither the MMA nor the TMA warp).  Three warps per
-// scheduler: 168 registers each.
+// Warp roles: warp 0 MMA issuer, warp 1 TMA producer (it also runs the scalar recurrence of G and writes each chunk's
+// coefficient vectors), warps 2..9 epilogue (lane quarter = warp % 4, as tensor memory demands), warps 10, 11 converters
+// (fp32 copies of the next chunk's K and Q tiles; they sit on the two schedulers that hold neither the MMA nor the
+// TMA warp).  Three warps per scheduler: 168 registers each.  Measured alternatives: the conversion inside the
+// epilogue warps (behind the hand-over of the state-update operands) put its 1.5 k cycles of shared-memory traffic
+// on the chain's critical path; four converter warps cost the epilogue its registers.
 constexpr int kWarpMma = 0, kWarpTma = 1, kWarpEpi = 2, kWarpCvt = 10, kCvtWarps = 2;
 constexpr int kThreads = (kEpiWarps + 2 + kCvtWarps) * 32;
 constexpr int kEpiThreads = kEpiWarps * 32, kCvtThreads = kCvtWarps * 32;
 
 // shared memory (offsets from a 1024-byte aligned base)
-// The K tile is read twice: by the converter warps, as rows from global memory a chunk ahead (with the Q rows), for its
-// fp32 copy; and by TMA into the stage, where MMA-3 reads it (MN-major) at the end of the chunk (an L2 hit).
+// The K tile is loaded twice: early into a buffer of its own (with the Q tile), where it is free again as soon as
+// its fp32 copy is made, so that the next chunk's arrives a whole chunk ahead; and into the stage, where MMA-3 reads
+// it (MN-major) at the end of the chunk.  The second load hits the L2.
 constexpr uint32_t kOffKQ32 = 0;        // fp32 [K; Q]: four dk quarters x [128 rows (K tokens, then Q tokens) x 128 B], swizzled
-constexpr uint32_t kOffStage = 65536;
+constexpr uint32_t kOffCvt = 65536;     // bf16 K and Q tiles waiting for their fp32 copies: [K 16 KB | Q 16 KB], single buffer
+constexpr uint32_t kOffStage = 98304;
 constexpr uint32_t kStK = 0, kStV = 16384, kStT = 32768, kStW = 40960, kStCoef = 57344;
 constexpr uint32_t kCoefBytes = kChainCoefs * C * sizeof(float);
 constexpr uint32_t kStageBytes = 59392;
@@ -85,9 +87,11 @@ constexpr uint32_t kColS = 0, kColM = 128, kColX = 256, kColZ = 320, kColY = 384
 struct Bars {
   uint64_t full[2];   // TMA loads of a stage landed                                      (1 + tx bytes)
   uint64_t go[2];     // a stage's output tile is staged and nothing reads the stage any more (256)
+  uint64_t cfull;     // bf16 K, Q of a chunk landed in their buffer                         (1 + tx bytes)
+  uint64_t cfree;     // ... and read: the next chunk's may be loaded                       (64)
   uint64_t kq;        // fp32 [K; Q] of a chunk written                                   (64)
-  uint64_t adj[2];    // a chunk's coefficient block written                              (64)
-  uint64_t fin;       // G after the last chunk written                                   (64)
+  uint64_t adj[2];    // a chunk's coefficient block written                              (32)
+  uint64_t fin;       // G after the last chunk written                                   (32)
   uint64_t init;      // masters of chunk 0 stored                                        (256)
   uint64_t mx;        // first half of MMA-1 done: X, Z                                    (commit)
   uint64_t m1;        // MMA-1 done: X, Z, Y, U                                            (commit)
@@ -105,9 +109,6 @@ struct Bars {
 struct Args {
   ChunkGeom g;
   const float* coef;
-  const __nv_bfloat16* q;   // the converters read the K and Q rows straight from global memory
-  const __nv_bfloat16* k;
-  long long tokens;         // B * T: rows past the end of the tensor read as zeros
   const float* S0;
   const float* M0;
   void* o;
@@ -212,14 +213,14 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tf32_kernel(const Args a, c
   const uint32_t b_m2 = smem_u32(&bars.m2), b_oi = smem_u32(&bars.oi), b_v1a = smem_u32(&bars.v1a);
   const uint32_t b_v1b = smem_u32(&bars.v1b), b_mx = smem_u32(&bars.mx), b_m3s = smem_u32(&bars.m3s);
   const uint32_t b_m3 = smem_u32(&bars.m3), b_mo = smem_u32(&bars.mo), b_zu = smem_u32(&bars.zu);
-  const uint32_t b_fin = smem_u32(&bars.fin);
+  const uint32_t b_fin = smem_u32(&bars.fin), b_cfull = smem_u32(&bars.cfull), b_cfree = smem_u32(&bars.cfree);
 
   if (tid == 0) {
     abort_flag = 0;
     mbar_init(b_full0, 1); mbar_init(b_full1, 1);
     mbar_init(b_go0, kEpiThreads); mbar_init(b_go1, kEpiThreads);
-    mbar_init(b_kq, kCvtThreads); mbar_init(b_adj0, kCvtThreads); mbar_init(b_adj1, kCvtThreads);
-    mbar_init(b_fin, kCvtThreads);
+    mbar_init(b_kq, kCvtThreads); mbar_init(b_adj0, 32); mbar_init(b_adj1, 32);
+    mbar_init(b_fin, 32); mbar_init(b_cfull, 1); mbar_init(b_cfree, kCvtThreads);
     mbar_init(b_init, kEpiThreads); mbar_init(b_r, kEpiThreads); mbar_init(b_oi, kEpiThreads);
     mbar_init(b_v1a, kEpiThreads); mbar_init(b_v1b, kEpiThreads); mbar_init(b_zu, kEpiThreads);
     mbar_init(b_m1, 1); mbar_init(b_m2, 1); mbar_init(b_m3, 1); mbar_init(b_mo, 1); mbar_init(b_mx, 1); mbar_init(b_m3s, 1);
@@ -271,55 +272,99 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tf32_kernel(const Args a, c
   }
 #endif
   if (warp == kWarpTma) {
-    // ================================================================== TMA producer + output stores
+    // ================================================================== TMA producer + output stores + coefficients
     // Stage s = c & 1 serves chunk c, then (as the staged output tile) is written out and refilled for chunk c + 2.
-    if (lane == 0) {
+    // The whole warp walks the loop; lane 0 issues the copies; every lane writes the coefficients of two tokens.
+    {
       int issued = 0;
+      float g11 = 1.f, g12 = 0.f, g22 = 1.f;
       for (int c = 0; c < nch + 2; ++c) {
         const int s = c & 1;
         const uint32_t st = s_base + kOffStage + s * kStageBytes;
         if (c >= 2) {
           const int co = c - 2;
           MDN_WAIT(s ? b_go1 : b_go0, (co >> 1) & 1);
-          const int n = min(C, sq.len - co * C);
-          const int tok0 = sq.tok0 + co * C;
-          const uint32_t src = st + kStOut;
-          if (!write_o) {
-            // Psi / Phi runs of the parallel scan produce states only
-          } else if (n == C) {
-            tma_store_2d(&map_o, h * kD, tok0, src);
-          } else {   // short chunk: rows >= n belong to another sequence; one bulk copy per valid row
-            for (int r = 0; r < n; ++r)
-              bulk_store(static_cast<uint8_t*>(a.o) + (((size_t)(tok0 + r) * H + h) * kD) * sizeof(TO),
-                         src + r * kD * (uint32_t)sizeof(TO), kD * (uint32_t)sizeof(TO));
+          if (lane == 0) {
+            const int n = min(C, sq.len - co * C);
+            const int tok0 = sq.tok0 + co * C;
+            const uint32_t src = st + kStOut;
+            if (!write_o) {
+              // Psi / Phi runs of the parallel scan produce states only
+            } else if (n == C) {
+              tma_store_2d(&map_o, h * kD, tok0, src);
+            } else {   // short chunk: rows >= n belong to another sequence; one bulk copy per valid row
+              for (int r = 0; r < n; ++r)
+                bulk_store(static_cast<uint8_t*>(a.o) + (((size_t)(tok0 + r) * H + h) * kD) * sizeof(TO),
+                           src + r * kD * (uint32_t)sizeof(TO), kD * (uint32_t)sizeof(TO));
+            }
+            tma_store_commit();
+            tma_store_wait_read();
           }
-          tma_store_commit();
-          tma_store_wait_read();
+          __syncwarp();
           MDN_MARK(co, kEvStoresDone);
         }
         if (c < nch) {
+          if (c > 0) MDN_WAIT(b_cfree, (c - 1) & 1);   // the previous chunk's bf16 K, Q have been read
           const uint32_t fb = s ? b_full1 : b_full0;
-          const int tok0 = sq.tok0 + c * C;
-          const int mat = (sq.slot0 + c) * H + h;
-          mbar_arrive_expect_tx(fb, kTxBytes - (write_o ? 0u : kTxW) - (v_zero ? kTxV : 0u));
-          bulk_load(st + kStCoef, a.coef + (size_t)mat * MDN_NUM_COEF * C, kCoefBytes, fb);
-          if (!v_zero) tma_load_2d(st + kStV, &map_v, h * kD, tok0, fb);
-          tma_load_2d(st + kStT, &map_t, 0, mat * C, fb);
-          if (write_o) {
-            tma_load_2d(st + kStW, &map_w, 0, mat * C, fb);
-            tma_load_2d(st + kStW + 8192, &map_w, 32, mat * C, fb);
+          if (lane == 0) {
+            const int tok0 = sq.tok0 + c * C;
+            const int mat = (sq.slot0 + c) * H + h;
+            mbar_arrive_expect_tx(b_cfull, write_o ? 32768u : 16384u);
+            tma_load_2d(s_base + kOffCvt, &map_k, h * kD, tok0, b_cfull);
+            tma_load_2d(s_base + kOffCvt + 8192, &map_k, h * kD + 64, tok0, b_cfull);
+            if (write_o) {
+              tma_load_2d(s_base + kOffCvt + 16384, &map_q, h * kD, tok0, b_cfull);
+              tma_load_2d(s_base + kOffCvt + 24576, &map_q, h * kD + 64, tok0, b_cfull);
+            }
+            mbar_arrive_expect_tx(fb, kTxBytes - (write_o ? 0u : kTxW) - (v_zero ? kTxV : 0u));
+            bulk_load(st + kStCoef, a.coef + (size_t)mat * MDN_NUM_COEF * C, kCoefBytes, fb);
+            if (!v_zero) tma_load_2d(st + kStV, &map_v, h * kD, tok0, fb);
+            tma_load_2d(st + kStT, &map_t, 0, mat * C, fb);
+            if (write_o) {
+              tma_load_2d(st + kStW, &map_w, 0, mat * C, fb);
+              tma_load_2d(st + kStW + 8192, &map_w, 32, mat * C, fb);
+            }
+            tma_load_2d(st + kStK, &map_k, h * kD, tok0, fb);          // for MMA-3 at the end of the chunk (L2 hit)
+            tma_load_2d(st + kStK + 8192, &map_k, h * kD + 64, tok0, fb);
           }
-          tma_load_2d(st + kStK, &map_k, h * kD, tok0, fb);          // for MMA-3 at the end of the chunk (L2 hit)
-          tma_load_2d(st + kStK + 8192, &map_k, h * kD + 64, tok0, fb);
+          __syncwarp();
           MDN_MARK(c, kEvTmaIssued);
           issued = c + 1;
+          // ---- the scalar recurrence of G and the chunk's six coefficient vectors (two tokens per lane), as soon as the
+          // chunk's coefficient vectors have landed: about a chunk before the epilogue needs them
+          MDN_WAIT(fb, (c >> 1) & 1);
+          float* aj = reinterpret_cast<float*>(smem + kOffAdj + s * kAdjBytes);
+          const float* cf = reinterpret_cast<const float*>(smem + kOffStage + s * kStageBytes + kStCoef);
+          const float aC = cf[kAbar * C + C - 1], bC = cf[kB * C + C - 1], mC = cf[kMubar * C + C - 1];
+          const float n11 = __fmul_rn(aC, g11), n12 = __fsub_rn(__fmul_rn(aC, g12), __fmul_rn(bC, g22)), n22 = __fmul_rn(mC, g22);
+          const bool lazy = n11 >= kLazyMin && n22 >= kLazyMin && fabsf(n12) <= kLazyMix * n22;
+#pragma unroll
+          for (int e = 0; e < 2; ++e) {
+            const int t = 2 * lane + e;
+            const float ab = cf[kAbar * C + t], bb = cf[kB * C + t], pp = cf[kAlphaBPrev * C + t];
+            const float gs = cf[kGS * C + t], gm = cf[kGM * C + t];
+            const float cx = ab * g11, cy = pp * g22 - ab * g12;
+            aj[kCx + t] = cx;
+            aj[kCy + t] = cy;
+            aj[kCz + t] = a.scale * cx;
+            aj[kCu + t] = a.scale * (ab * g12 - bb * g22);
+            aj[kWs + t] = lazy ? (gs + (n12 / n22) * gm) / n11 : gs;
+            aj[kWm + t] = lazy ? gm / n22 : gm;
+          }
+          if (lane == 0) { aj[kN11] = n11; aj[kN12] = n12; aj[kN22] = n22; aj[kLazy] = lazy ? 1.f : 0.f; }
+          if (lazy) { g11 = n11; g12 = n12; g22 = n22; } else { g11 = 1.f; g12 = 0.f; g22 = 1.f; }
+          mbar_arrive(s ? b_adj1 : b_adj0);
+        } else if (c == nch) {
+          if (lane == 0) { g_final[0] = g11; g_final[1] = g12; g_final[2] = g22; }
+          mbar_arrive(b_fin);
         }
       }
-      if (!ok) {   // giving up: let the copies already in flight land before the CTA exits
+      if (!ok && lane == 0) {   // giving up: let the copies already in flight land before the CTA exits
         for (int c = max(0, issued - 2); c < issued; ++c)
           for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait((c & 1) ? b_full1 : b_full0, (c >> 1) & 1); ++it) {}
+        for (uint32_t it = 0; it < (1u << 16) && issued > 0 && !mbar_try_wait(b_cfull, (issued - 1) & 1); ++it) {}
       }
-      tma_store_wait_all();
+      if (lane == 0) tma_store_wait_all();
     }
   } else if (warp == kWarpMma) {
     // ================================================================== MMA issuer
@@ -428,93 +473,37 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tf32_kernel(const Args a, c
     }
   } else if (warp >= kWarpCvt) {
     // ================================================================== converter warps
-    // One chunk ahead of the chain: the fp32 copies of the K and Q tiles, then the scalar recurrence of G and the
-    // chunk's six coefficient vectors.
-    const int t = tid - kWarpCvt * 32;   // 0..63: the token whose coefficients this thread writes
-    float g11 = 1.f, g12 = 0.f, g22 = 1.f;
-    // Rows of the K and Q tiles: in step i a warp reads two whole rows (sixteen 16-byte pieces each: coalesced), the two
-    // warps four; row = 4 i + 2 warp + lane / 16, piece = lane % 16.  The fp32 stores of one such step spread evenly
-    // over the banks in the swizzled layout.
-    const int cw = warp - kWarpCvt, piece = lane & 15;
-    const size_t row_stride = (size_t)H * kD;   // elements between consecutive tokens
-    uint4 kq[2][16];
-    auto load_rows = [&](int c) {
-      const long long tok0 = (long long)sq.tok0 + (long long)c * C;
+    // One chunk ahead of the chain: fp32 copies of the K and Q tiles.  bf16 tile: two dk halves of [64 rows x 128 B];
+    // fp32 tile: four dk quarters of [128 rows x 128 B].  A thread takes one token row (rows across the lanes:
+    // minimal wavefronts in both swizzled layouts): the sixteen loads of a tile first, then its thirty-two stores.
+    const uint32_t row = static_cast<uint32_t>(tid - kWarpCvt * 32), sw = row & 7;
+    for (int c = 0; c < nch; ++c) {
+      MDN_WAIT(b_cfull, c & 1);
+      if (c > 0) MDN_WAIT(b_m1, (c - 1) & 1);   // the previous chunk's products have read the fp32 tiles
+      MDN_MARK(c, kEvCvtStart);
+#pragma unroll 1
+      for (int which = 0; which < (write_o ? 2 : 1); ++which) {
+        const uint32_t src = s_base + kOffCvt + which * 16384 + row * 128;
+        const uint32_t dst = s_base + kOffKQ32 + (which * 64 + row) * 128;
+        uint4 u[16];
 #pragma unroll
-      for (int which = 0; which < 2; ++which) {
-        const __nv_bfloat16* base = (which ? a.q : a.k) + (size_t)h * kD + piece * 8;
+        for (int c16 = 0; c16 < 16; ++c16)
+          asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                       : "=r"(u[c16].x), "=r"(u[c16].y), "=r"(u[c16].z), "=r"(u[c16].w)
+                       : "r"(src + (c16 >> 3) * 8192 + ((static_cast<uint32_t>(c16 & 7) ^ sw) << 4)));
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          const long long tok = tok0 + 4 * i + 2 * cw + (lane >> 4);
-          kq[which][i] = make_uint4(0u, 0u, 0u, 0u);
-          if (tok < a.tokens && (which == 0 || write_o)) {
-            // volatile: the loads must be ISSUED here, a chunk ahead of their use, not sunk down to the stores
-            asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
-                         : "=r"(kq[which][i].x), "=r"(kq[which][i].y), "=r"(kq[which][i].z), "=r"(kq[which][i].w)
-                         : "l"(base + (size_t)tok * row_stride));
-          }
+        for (int c16 = 0; c16 < 16; ++c16) {
+          const uint32_t d0 = dst + (c16 >> 2) * 16384, ch = static_cast<uint32_t>((c16 & 3) * 2);
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(d0 + ((ch ^ sw) << 4)), "r"(u[c16].x << 16),
+                       "r"(u[c16].x & 0xffff0000u), "r"(u[c16].y << 16), "r"(u[c16].y & 0xffff0000u) : "memory");
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(d0 + (((ch + 1) ^ sw) << 4)), "r"(u[c16].z << 16),
+                       "r"(u[c16].z & 0xffff0000u), "r"(u[c16].w << 16), "r"(u[c16].w & 0xffff0000u) : "memory");
         }
       }
-    };
-    if (nch > 0) load_rows(0);
-    for (int c = 0; c <= nch; ++c) {
-      if (c < nch) {
-        // ---- fp32 copies of this chunk's K and Q tiles (the chain needs them first); the rows are in registers
-        if (c > 0) MDN_WAIT(b_m1, (c - 1) & 1);   // the previous chunk's products have read the fp32 tiles
-        MDN_MARK(c, kEvCvtStart);
-#pragma unroll
-        for (int which = 0; which < 2; ++which) {
-          if (which == 0 || write_o) {
-#pragma unroll
-            for (int i = 0; i < 16; ++i) {
-              const int row = 4 * i + 2 * cw + (lane >> 4);
-              const uint32_t sw = static_cast<uint32_t>(row & 7);
-              const uint32_t d0 = s_base + kOffKQ32 + (piece >> 2) * 16384 + (which * 64 + row) * 128;
-              const uint32_t ch = static_cast<uint32_t>((piece & 3) * 2);
-              const uint4 u = kq[which][i];
-              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(d0 + ((ch ^ sw) << 4)), "r"(u.x << 16),
-                           "r"(u.x & 0xffff0000u), "r"(u.y << 16), "r"(u.y & 0xffff0000u) : "memory");
-              asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(d0 + (((ch + 1) ^ sw) << 4)), "r"(u.z << 16),
-                           "r"(u.z & 0xffff0000u), "r"(u.w << 16), "r"(u.w & 0xffff0000u) : "memory");
-            }
-          }
-          if (which == 0) MDN_MARK(c, kEvM3sOwn);
-        }
-        MDN_MARK(c, kEvEager);
-        fence_proxy_async_smem();
-        mbar_arrive(b_kq);
-        MDN_MARK(c, kEvCvtDone);
-        // ---- the scalar recurrence of G and the chunk's six coefficient vectors
-        float* aj = reinterpret_cast<float*>(smem + kOffAdj + (c & 1) * kAdjBytes);
-        MDN_WAIT((c & 1) ? b_full1 : b_full0, (c >> 1) & 1);
-        const float* cf = reinterpret_cast<const float*>(smem + kOffStage + (c & 1) * kStageBytes + kStCoef);
-        const float aC = cf[kAbar * C + C - 1], bC = cf[kB * C + C - 1], mC = cf[kMubar * C + C - 1];
-        const float n11 = __fmul_rn(aC, g11), n12 = __fsub_rn(__fmul_rn(aC, g12), __fmul_rn(bC, g22)), n22 = __fmul_rn(mC, g22);
-        const bool lazy = n11 >= kLazyMin && n22 >= kLazyMin && fabsf(n12) <= kLazyMix * n22;
-        const float ab = cf[kAbar * C + t], bb = cf[kB * C + t], pp = cf[kAlphaBPrev * C + t];
-        const float gs = cf[kGS * C + t], gm = cf[kGM * C + t];
-        const float cx = ab * g11, cy = pp * g22 - ab * g12;
-        aj[kCx + t] = cx;
-        aj[kCy + t] = cy;
-        aj[kCz + t] = a.scale * cx;
-        aj[kCu + t] = a.scale * (ab * g12 - bb * g22);
-        if (lazy) {
-          aj[kWs + t] = (gs + (n12 / n22) * gm) / n11;
-          aj[kWm + t] = gm / n22;
-        } else {
-          aj[kWs + t] = gs;
-          aj[kWm + t] = gm;
-        }
-        if (t == 0) { aj[kN11] = n11; aj[kN12] = n12; aj[kN22] = n22; aj[kLazy] = lazy ? 1.f : 0.f; }
-        if (lazy) { g11 = n11; g12 = n12; g22 = n22; } else { g11 = 1.f; g12 = 0.f; g22 = 1.f; }
-        mbar_arrive((c & 1) ? b_adj1 : b_adj0);
-        // the next chunk's rows: in flight while the chain works on this chunk (issued last: nothing this thread
-        // still has to do for the current chunk may queue up behind thirty-two outstanding loads)
-        if (c + 1 < nch) load_rows(c + 1);
-      } else {
-        if (t == 0) { g_final[0] = g11; g_final[1] = g12; g_final[2] = g22; }
-        mbar_arrive(b_fin);
-      }
+      mbar_arrive(b_cfree);          // the bf16 tiles have been read: the next chunk's may land
+      fence_proxy_async_smem();
+      mbar_arrive(b_kq);
+      MDN_MARK(c, kEvCvtDone);
     }
   } else {
     // ================================================================== epilogue warps
@@ -524,7 +513,6 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tf32_kernel(const Args a, c
     const int d = q4 * 32 + lane;
     const int r0 = kTok * hf;
     const uint32_t tl = tmem + (static_cast<uint32_t>(q4 * 32) << 16);
-
     for (int c = 0; c <= nch; ++c) {
       const float* aj = reinterpret_cast<const float*>(smem + kOffAdj + (c & 1) * kAdjBytes);
       if (c == 0) {
@@ -654,14 +642,6 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tf32_kernel(const Args a, c
       // chunk, their last reader, is done) and the update is added in true coordinates.
       const bool eager = aj[kLazy] == 0.f;
       const float n11 = aj[kN11], n12 = aj[kN12], n22 = aj[kN22];
-      float wsv[kTok], wmv[kTok];   // fetched before the wait, as in EPI-1
-#pragma unroll
-      for (int j = 0; j < kTok; j += 4) {
-        const float4 a4 = *reinterpret_cast<const float4*>(aj + kWs + r0 + j);
-        const float4 b4 = *reinterpret_cast<const float4*>(aj + kWm + r0 + j);
-        wsv[j] = a4.x; wsv[j + 1] = a4.y; wsv[j + 2] = a4.z; wsv[j + 3] = a4.w;
-        wmv[j] = b4.x; wmv[j + 1] = b4.y; wmv[j + 2] = b4.z; wmv[j + 3] = b4.w;
-      }
       MDN_WAIT(b_m2, ph);
       __syncwarp();
       tc_fence_after_sync();
@@ -669,6 +649,14 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tf32_kernel(const Args a, c
       {
         uint32_t vt[kTok];
         tmem_ld32(tl + kColY + r0, vt);
+        float wsv[kTok], wmv[kTok];   // (their loads run while the tensor-memory load is in flight)
+#pragma unroll
+        for (int j = 0; j < kTok; j += 4) {
+          const float4 a4 = *reinterpret_cast<const float4*>(aj + kWs + r0 + j);
+          const float4 b4 = *reinterpret_cast<const float4*>(aj + kWm + r0 + j);
+          wsv[j] = a4.x; wsv[j + 1] = a4.y; wsv[j + 2] = a4.z; wsv[j + 3] = a4.w;
+          wmv[j] = b4.x; wmv[j + 1] = b4.y; wmv[j + 2] = b4.z; wmv[j + 3] = b4.w;
+        }
         tmem_wait_ld();
         {
           uint32_t sh[kPk], sl[kPk];
@@ -790,7 +778,6 @@ cudaError_t launch_chain_tf32(const Plan& pl, const void* q, const void* k, cons
   Args a;
   a.g = pl.geom;
   a.coef = reinterpret_cast<const float*>(pl.ws + pl.lay.off_coef);
-  a.q = static_cast<const __nv_bfloat16*>(q); a.k = static_cast<const __nv_bfloat16*>(k); a.tokens = (long long)tokens;
   a.S0 = S0; a.M0 = M0; a.o = o; a.Sf = Sf; a.Mf = Mf;
   a.status = reinterpret_cast<int32_t*>(pl.ws + pl.lay.off_status);
   a.scale = p.scale;

@@ -373,11 +373,11 @@ def test_state_handoff_and_determinism_tensor_path(mdn):
     ob, Sb, Mb = run_gpu(mdn, b, path="tensor", o_dtype=torch.float32)
     # the split falls on a chunk boundary and the state is handed over in fp32.  The first half is the same
     # arithmetic; the second half starts from the true state where the single call carries a lazily scaled one
-    # (chain_tf32.cu), so it agrees to fp32 / tf32 rounding, not bit for bit
+    # (chain_tf32.cu), so it agrees to tf32 operand rounding (half the parity bound is allowed), not bit for bit
     assert np.array_equal(o[:, :256], oa)
     rms = lambda x: np.sqrt(np.mean(x ** 2))
-    assert np.abs(o[:, 256:] - ob).max() <= 2e-3 * rms(o)
-    assert np.abs(S - Sb).max() <= 2e-3 * rms(S) and np.abs(M - Mb).max() <= 2e-3 * rms(M)
+    assert np.abs(o[:, 256:] - ob).max() <= 1e-2 * rms(o)
+    assert np.abs(S - Sb).max() <= 1e-2 * rms(S) and np.abs(M - Mb).max() <= 1e-2 * rms(M)
 
 
 def test_packed_varlen_edge_lengths(mdn):

@@ -55,8 +55,11 @@ def test_keep_chunk_states(mdn, name, kw):
     o1, S1, M1 = mdn.chunk_fwd(t["q"], t["k"], t["v"], t["beta"], t["log_alpha"], t["log_mu"], t["eta"],
                                initial_S=t["initial_S"], initial_M=t["initial_M"], cu_seqlens=t["cu_seqlens"],
                                scale=inp["scale"], path="tensor", o_dtype=torch.float32, segments=1)
-    # the kept states change nothing else
-    assert torch.equal(o, o1) and torch.equal(S, S1) and torch.equal(M, M1)
+    # the kept states change nothing else: the training instantiation (first chain design, bf16 state operands) and the
+    # plain forward (second design, tf32 state operands, lazily scaled masters) compute the same thing, each within
+    # the forward's tolerance of the oracle - so within twice that of each other
+    for x, y in ((o, o1), (S, S1), (M, M1)):
+        assert (x - y).abs().max().item() <= 2 * 2e-2 * y.pow(2).mean().sqrt().item()
     Sc, Mc = mdn.unpack_chunk_states(states, w.H)
     S_ref, M_ref = oracle_chunk_start_states(inp)
     n = S_ref.shape[0]
