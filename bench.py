@@ -35,9 +35,42 @@ METRIC = "MDN chunkwise fwd tokens/s"
 UNIT = "tokens/s"
 BYTES_PER_HEAD_TOKEN_BF16 = 1040      # q,k,v read + o written (bf16, d=128) + four fp32 gates
 L2_BYTES = 126e6
-# dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised in
-# profiles/chain_tensor_cfg2.md and profiles/intra_mma_cfg2.md (same command line as this benchmark)
-NCU_TRAFFIC_BYTES = {("cfg2_1p3b_bf16", "chain"): 745.0e6, ("cfg2_1p3b_bf16", "intra_chunk"): 453.3e6}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch come from the ncu summaries under profiles/ (same command
+# line as this benchmark): each summary carries the lines "kernel = <name>", "workload = <name>" and
+# "traffic_bytes_per_launch = <bytes>", which are read at run time, so the number cannot drift away from its source.
+PROFILE_FILES = {"chain": "chain_tf32_cfg2.md", "intra_chunk": "intra_mma_cfg2.md"}
+STAGE_KERNELS = {"chain": "chain_tf32_kernel", "intra_chunk": "intra_mma_kernel"}
+
+
+def profile_traffic(stage: str, workload: str):
+    """(bytes per launch, source) from the committed ncu summary of this stage's kernel on this workload, or
+    (None, reason) when there is no summary of exactly that kernel and workload."""
+    import re
+    name = PROFILE_FILES.get(stage)
+    path = os.path.join(ROOT, "profiles", name) if name else None
+    if not path or not os.path.exists(path):
+        return None, "no ncu summary for stage %r" % stage
+    text = open(path).read()
+    fields = dict(re.findall(r"^(kernel|workload|traffic_bytes_per_launch)\s*=\s*(\S+)\s*$", text, flags=re.M))
+    if fields.get("kernel") != STAGE_KERNELS[stage] or fields.get("workload") != workload:
+        return None, "profiles/%s covers %s on %s" % (name, fields.get("kernel"), fields.get("workload"))
+    src = {"file": "profiles/" + name, "commit": git_hash(["log", "-1", "--format=%h", "--", "profiles/" + name])}
+    return float(fields["traffic_bytes_per_launch"]), src
+
+
+def git_hash(args=("rev-parse", "--short", "HEAD")):
+    """Short hash from git, else from the stamp the build step leaves beside the library (the GPU machine gets no .git)."""
+    try:
+        out = subprocess.run(["git", "-C", ROOT] + list(args), capture_output=True, text=True, timeout=10)
+        if out.returncode == 0 and out.stdout.strip():
+            return out.stdout.strip()
+    except (OSError, subprocess.SubprocessError):
+        pass
+    try:
+        info = json.load(open(os.path.join(ROOT, "paper_2605_05838_b200", "_build_info.json")))
+        return info.get("git_hash") if list(args) == ["rev-parse", "--short", "HEAD"] else info.get("profiles", {}).get(args[-1])
+    except (OSError, ValueError):
+        return None
 
 
 def load_peaks():
@@ -165,6 +198,74 @@ def oracle_sample_tokens_per_s(w: wl.Workload, inp, target_s: float):
     return ht / w.H / secs, threads, "%d of %d (sequence, head) chains, %d head-tokens" % (len(chains), total, int(ht)), secs
 
 
+def parity_report(mdn, w, inp, t, p, args, ws):
+    """The timed workload's result against the oracle on EVERY (sequence, head) chain, outside any timed region:
+    max |x - ref| / RMS(ref) of o as stored (bf16 on the bf16 workloads), of the oracle's own o rounded to that storage
+    type (what one storage rounding of the exact result costs), of o stored as fp32 by the same kernels, and of
+    the final states."""
+    import oracle
+    import torch
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    from helpers import bf16_floor, rel_err
+    t0 = time.perf_counter()
+    o_ref, S_ref, M_ref = oracle.stepwise(inp["q"], inp["k"], inp["v"], inp["beta"], inp["log_alpha"], inp["log_mu"],
+                                          inp["eta"], scale=inp["scale"], S0=inp["S0"], M0=inp["M0"],
+                                          seq_start=inp["seq_start"], seq_len=inp["seq_len"])
+    secs = time.perf_counter() - t0
+    kw = dict(initial_S=t["initial_S"], initial_M=t["initial_M"], cu_seqlens=t["cu_seqlens"], scale=inp["scale"],
+              path=args.path, workspace=ws)
+    gates = (t["beta"], t["log_alpha"], t["log_mu"], t["eta"])
+    o, S, M = mdn.chunk_fwd(t["q"], t["k"], t["v"], *gates, **kw)
+    o32, _, _ = mdn.chunk_fwd(t["q"], t["k"], t["v"], *gates, o_dtype=torch.float32, **kw)
+    torch.cuda.synchronize()
+    f64 = lambda x: x.float().cpu().numpy().astype(np.float64)
+    out = {"chains": int(len(inp["seq_len"]) * w.H), "oracle_seconds": secs,
+           "o_stored": rel_err(f64(o), o_ref), "o_f32_store": rel_err(f64(o32), o_ref),
+           "S": rel_err(f64(S), S_ref), "M": rel_err(f64(M), M_ref),
+           "metric": "max |x - ref| / RMS(ref) over all elements", "tolerance": 2e-2 if w.dtype == "bf16" else 1e-4}
+    if w.dtype == "bf16":
+        out["o_bf16_floor"] = bf16_floor(o_ref)      # the exact result rounded once to bf16
+    return out
+
+
+def time_config(mdn, w, path, peaks):
+    """ms per step of another named workload (device-resident inputs, CUDA events, 3 warm-up + 10 timed steps)."""
+    import torch
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    from helpers import to_torch
+    inp = wl.make_inputs(w)
+    t = to_torch(inp)
+    N = len(inp["seq_len"])
+    o_dtype = torch.bfloat16 if w.dtype == "bf16" else torch.float32
+    p = mdn.make_params(t["q"], t["v"], num_seqs=(N if w.varlen else 0), scale=inp["scale"], o_dtype=o_dtype, path=path)
+    ws = torch.empty(mdn.workspace_bytes(p), dtype=torch.uint8, device=t["q"].device)
+    io_bytes = algorithmic_bytes(w, N, t["initial_S"] is not None)
+    n_copies = 1 if io_bytes > L2_BYTES else int(2 * L2_BYTES // io_bytes) + 1
+    clone = lambda d: {k_: (v_.clone() if torch.is_tensor(v_) else v_) for k_, v_ in d.items()}
+    sets = [t] + [clone(t) for _ in range(n_copies - 1)]
+    outs = [torch.empty((w.B, w.T, w.H, w.dv), dtype=o_dtype, device=t["q"].device) for _ in range(n_copies)]
+
+    def step(i):
+        ti = sets[i % n_copies]
+        mdn.chunk_fwd(ti["q"], ti["k"], ti["v"], ti["beta"], ti["log_alpha"], ti["log_mu"], ti["eta"],
+                      initial_S=ti["initial_S"], initial_M=ti["initial_M"], cu_seqlens=ti["cu_seqlens"],
+                      scale=inp["scale"], o_dtype=o_dtype, path=path, workspace=ws, out=outs[i % n_copies])
+
+    for i in range(3):
+        step(i)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(10):
+        step(i)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / 10
+    return {"workload": workload_desc(w), "ms_per_step": ms, "tokens_per_s": w.B * w.T / (ms * 1e-3),
+            "frac": io_bytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "launches_per_step": mdn.last_launch_count(),
+            "l2": "single copy" if n_copies == 1 else "%d copies rotated" % n_copies}
+
+
 def run_reference(args, w):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -216,6 +317,9 @@ def run_ours(args, w):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
+    # the clock sampler starts before the inputs are generated (seconds of host work), so that nvidia-smi is already
+    # sampling when the warm-up begins and the warm-up can be exactly what --warmup asks for
+    sampler = ClockSampler(local) if rank == 0 else None
     wr = rank_workload(w, rank)
     inp = wl.make_inputs(wr)
     t = to_torch(inp, device="cuda:%d" % local)
@@ -246,14 +350,9 @@ def run_ours(args, w):
             dist.barrier()
         torch.cuda.synchronize()
 
-    sampler = ClockSampler(local) if rank == 0 else None     # nvidia-smi needs ~0.5 s to start sampling
-    t_warm = time.perf_counter()
-    n_warm = 0
-    while n_warm < max(args.warmup, 3) or (rank == 0 and world == 1 and time.perf_counter() - t_warm < 0.7):
+    n_warm = max(args.warmup, 3)      # the timing rules ask for at least three
+    for _ in range(n_warm):
         step()
-        n_warm += 1
-        if n_warm % 16 == 0:
-            torch.cuda.synchronize()
     launches_per_step = mdn.last_launch_count()
     barrier()
     # timed region 1: exactly K steps, nothing but the calls -> the headline value
@@ -277,7 +376,8 @@ def run_ours(args, w):
     tokens_per_step = w.B * w.T * world
     value = job_tokens_per_s(w, world, args.steps, elapsed_ms)
 
-    # dominant kernel (the chain kernel: inter-chunk propagation + output), timed live
+    # per-kernel durations, timed live; the roofline fraction is that of the WHOLE step (the path is two kernels in
+    # series: algorithmic bytes over the time of one step); the dominant kernel's own figures are given beside it
     names = mdn.STAGE_NAMES
     stage_ms = {names[s]: statistics.mean(stage_ev[i][s].elapsed_time(stage_ev[i][s + 1]) for i in range(args.steps))
                 for s in range(len(names))}
@@ -285,18 +385,24 @@ def run_ours(args, w):
     peaks = load_peaks()
     abytes = algorithmic_bytes(w, N, t["initial_S"] is not None)
     aflops = algorithmic_flops(w)
+    step_s = elapsed_ms / args.steps * 1e-3
     dom_s = stage_ms[dom] * 1e-3
-    achieved = abytes / dom_s / 1e9
-    roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
-                "kernel_ms": stage_ms[dom], "stage_ms": stage_ms,
-                "algorithmic_bytes": abytes, "algorithmic_flops": aflops,
-                "tensor_achieved_tflops": aflops / dom_s / 1e12,
-                "tensor_frac_of_burst_peak": aflops / dom_s / 1e12 / peaks["bf16_tflops"],
+    achieved = abytes / step_s / 1e9
+    tensor_path = mdn.resolved_path(p) == "tensor"
+    traffic, sources = {}, {}
+    for st_name in ("intra_chunk", "chain"):
+        traffic[st_name], sources[st_name] = profile_traffic(st_name, w.name) if tensor_path else (None, "no summary for the SIMT path")
+    whole_traffic = None if None in traffic.values() else sum(traffic.values())
+    roofline = {"bound": "hbm", "kernel": "whole step: intra_chunk + chain (two kernels in series)", "achieved": achieved,
+                "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "traffic": whole_traffic,
+                "traffic_source": sources, "peak_source": peaks["source"],
+                "stage_ms": stage_ms, "algorithmic_bytes": abytes, "algorithmic_flops": aflops,
                 "frac_of_nominal_hbm_8tbs": achieved / 8000.0,
-                "tensor_frac_of_nominal_2250tf": aflops / dom_s / 1e12 / 2250.0,
-                "whole_step_frac_hbm": abytes / (elapsed_ms / args.steps * 1e-3) / 1e9 / peaks["hbm_gbs"]}
-    roofline["traffic"] = NCU_TRAFFIC_BYTES.get((w.name, dom))
+                "tensor_achieved_tflops": aflops / step_s / 1e12,
+                "tensor_frac_of_burst_peak": aflops / step_s / 1e12 / peaks["bf16_tflops"],
+                "dominant_kernel": {"name": dom, "kernel_ms": stage_ms[dom], "traffic": traffic.get(dom),
+                                    "frac_algorithmic_bytes_over_its_time": abytes / dom_s / 1e9 / peaks["hbm_gbs"],
+                                    "tensor_achieved_tflops": aflops / dom_s / 1e12}}
 
     # end to end through the host-buffer entry point (pinned host memory, copies inside the timed region)
     e2e = None
@@ -335,9 +441,15 @@ def run_ours(args, w):
         return
 
     cpu = None
+    parity = None
     if world == 1 and not args.no_cpu_baseline:
         v, threads, desc, secs = oracle_sample_tokens_per_s(w, inp, target_s=args.cpu_seconds)
         cpu = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc, "seconds": secs}
+        parity = parity_report(mdn, w, inp, t, p, args, ws)
+
+    others = None
+    if world == 1 and args.config == 2 and not args.no_other_configs:
+        others = {wl.CONFIGS[i].name: time_config(mdn, wl.CONFIGS[i], args.path, peaks) for i in (1, 3, 4)}
 
     ws_in = abytes
     print(json.dumps({
@@ -352,7 +464,8 @@ def run_ours(args, w):
                          ("inputs+outputs %.0f MB per step fit in the 126 MB L2: %d copies rotated (%.0f MB per round)"
                           % (ws_in / 1e6, n_copies, n_copies * ws_in / 1e6))},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
-        "roofline": roofline, "cpu_baseline": cpu}))
+        "roofline": roofline, "cpu_baseline": cpu, "parity": parity, "other_configs": others,
+        "git": git_hash()}))
     if dist is not None:
         dist.destroy_process_group()
 
@@ -570,6 +683,7 @@ def main():
     ap.add_argument("--path", default="auto", choices=["auto", "simt", "tensor"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg (profiling runs)")
+    ap.add_argument("--no-other-configs", action="store_true", help="skip the short timings of configs 1, 3 and 4")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--decode", action="store_true", help="secondary benchmark: the recurrent decode step")
     ap.add_argument("--decode-batch", type=int, default=128)

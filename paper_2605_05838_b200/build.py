@@ -33,6 +33,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     srcs = sorted(glob.glob(os.path.join(CSRC, "*.cu")))
     hdrs = sorted(glob.glob(os.path.join(CSRC, "*.cuh"))) + sorted(glob.glob(os.path.join(ROOT, "include", "*.h")))
     if not force and _newer(LIB, srcs + hdrs):
+        write_build_info()
         return LIB
     os.makedirs(OBJ_DIR, exist_ok=True)
 
@@ -53,7 +54,30 @@ def build(force: bool = False, verbose: bool = False) -> str:
     subprocess.run(["nvcc", "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", tmp] + objs
                    + ["-lcudart", "-lcuda"], check=True)
     os.replace(tmp, LIB)
+    write_build_info()
     return LIB
+
+
+def write_build_info() -> None:
+    """Leaves the source revision beside the library (a machine that receives the tree without its .git directory
+    can still say which commit it runs): the short hash of HEAD and of the last commit of every profiles/ summary."""
+    import json
+
+    def git(*args):
+        try:
+            r = subprocess.run(["git", "-C", ROOT] + list(args), capture_output=True, text=True, timeout=10)
+            return r.stdout.strip() if r.returncode == 0 and r.stdout.strip() else None
+        except (OSError, subprocess.SubprocessError):
+            return None
+
+    head = git("rev-parse", "--short", "HEAD")
+    if head is None:
+        return
+    dirty = bool(git("status", "--porcelain", "--untracked-files=no"))
+    prof = {"profiles/" + os.path.basename(f): git("log", "-1", "--format=%h", "--", "profiles/" + os.path.basename(f))
+            for f in glob.glob(os.path.join(ROOT, "profiles", "*.md"))}
+    with open(os.path.join(PKG, "_build_info.json"), "w") as fh:
+        json.dump({"git_hash": head + ("+" if dirty else ""), "profiles": prof}, fh)
 
 
 if __name__ == "__main__":
