@@ -319,6 +319,27 @@ def test_degenerate_gates_tensor_path(mdn):
     assert np.allclose(S, abar[:, :, None, None] * inp4["S0"], rtol=1e-4, atol=1e-7)    # purely decayed state, exact path
 
 
+@pytest.mark.parametrize("alpha,mu,beta", [(0.999, 0.8, 0.001), (0.99, 0.9, 0.01), (0.98, 0.97, 0.01), (0.97, 0.98, 0.015),
+                                           (0.9, 0.95, 0.1), (0.995, 0.6, 0.01), (0.999, 0.999, 0.0002), (0.95, 0.999, 0.015),
+                                           (0.3, 0.5, 0.3)])
+def test_gate_regimes_of_the_lazily_scaled_state(mdn, alpha, mu, beta):
+    """The tensor path keeps the state lazily scaled ([S; M] = G [Sh; Mh], rescaled only when G would leave a safe
+    range).  Constant gates from regimes where S decays slower than M, as fast, or much faster exercise every branch of
+    that rule: chunks that all stay lazy, chunks that all rescale, and mixtures; with a loose rule the two hat terms of
+    S cancel catastrophically when alpha > mu (errors of order 100), so this is the test that pins the rule."""
+    import torch
+    w = wl.Workload("regime", B=1, T=1024, H=2, dk=128, dv=128, dtype="bf16", init_state_std=0.05, seed=90)
+    if not tensor_ok(mdn, w):
+        pytest.skip("tensor path not built")
+    inp = wl.make_inputs(w)
+    inp["log_alpha"][:] = np.float32(np.log(alpha))
+    inp["log_mu"][:] = np.float32(np.log(mu))
+    inp["beta"][:] = np.float32(beta)
+    inp["log_alpha"][0, 300:340, 1] = np.float32(np.log(0.2))      # a burst of fast forgetting in one head
+    inp["log_mu"][0, 700:705, 0] = -np.inf                         # and a few mu = 0 tokens in the other
+    compare(mdn, inp, "tensor", label="alpha %.3f mu %.3f beta %.4f" % (alpha, mu, beta))
+
+
 @pytest.mark.parametrize("segments,T", [(3, 64 * 9), (4, 64 * 13 + 17), (8, 64 * 40 + 1), (5, 64 * 3 + 5), (16, 64 * 33)])
 def test_parallel_inter_chunk_scan_forced(mdn, segments, T):
     """The segmented scan (zero-state runs, V = 0 basis runs, serial combine, real runs) against the stepwise
