@@ -46,12 +46,13 @@ mdn_status mdn_probe_tf32(int32_t mode, const float* a, const float* b, const fl
                           void* cuda_stream);
 
 /*
- * Cost of one tcgen05 product as a function of its shape: a stream of 4 * reps products D[128 x n] += A[128 x K] *
+ * Cost of one tcgen05 product as a function of its shape: a stream of 4 * reps products D[m x n] += A[m x K] *
  * B[n x K]^T (K = 16 bf16 or 8 tf32 elements), A from tensor memory (a_tmem) or from shared memory, issued by one
- * thread; out[0] = cycles from the first issue to completion, out[1] = products issued.  n in {32, 64, 128, 256}.
+ * thread; out[0] = cycles from the first issue to completion, out[1] = products issued.  n in {32, 64, 128, 256},
+ * m in {64, 128}.
  */
-mdn_status mdn_probe_mma_timing(int32_t tf32, int32_t a_tmem, int32_t n, int32_t reps, float* out, int32_t* status,
-                                void* cuda_stream);
+mdn_status mdn_probe_mma_timing(int32_t tf32, int32_t a_tmem, int32_t n, int32_t m, int32_t reps, float* out,
+                                int32_t* status, void* cuda_stream);
 
 /*
  * One CTA waits on an mbarrier nothing arrives at, with the poll limit given (1 .. 2^20): the wait runs out,

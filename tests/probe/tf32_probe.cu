@@ -298,7 +298,7 @@ __global__ void __launch_bounds__(128) tf32_probe_kernel(int mode, const float* 
 // Issue-to-completion time of a stream of tcgen05 products of one shape (operand contents irrelevant): how the
 // cost of one product depends on the kind, on where A comes from and on N.  A [128 x K], B [N x K] K-major,
 // K = 64 bf16 or 32 tf32 elements per 128-byte row (one swizzle block): 4 products per pass over the block.
-__global__ void __launch_bounds__(128) mma_timing_kernel(int tf32, int a_tmem, int N, int reps, float* __restrict__ out,
+__global__ void __launch_bounds__(128) mma_timing_kernel(int tf32, int a_tmem, int N, int M, int reps, float* __restrict__ out,
                                                         int32_t* __restrict__ status) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -326,7 +326,7 @@ __global__ void __launch_bounds__(128) mma_timing_kernel(int tf32, int a_tmem, i
   bool ok = true;
   if (tid == 0) {
     tc_fence_after_sync();
-    const uint32_t id = tf32 ? idesc_tf32(128, N, false, false, false) : idesc_bf16(128, N, false, false, false);
+    const uint32_t id = tf32 ? idesc_tf32(M, N, false, false, false) : idesc_bf16(M, N, false, false, false);
     const uint64_t da = smem_desc_sw128(smem_u32(smem), 16, 1024);              // A block: 128 rows x 128 B
     const uint64_t db = smem_desc_sw128(smem_u32(smem) + 16384, 16, 1024);      // B block: up to 256 rows x 128 B
     const uint32_t ta = tmem + 256;
@@ -406,13 +406,14 @@ extern "C" mdn_status mdn_probe_bounded_wait(uint32_t spin_limit, int32_t* statu
   return cudaGetLastError() == cudaSuccess ? MDN_OK : MDN_ERR_CUDA;
 }
 
-extern "C" mdn_status mdn_probe_mma_timing(int32_t tf32, int32_t a_tmem, int32_t n, int32_t reps, float* out,
+extern "C" mdn_status mdn_probe_mma_timing(int32_t tf32, int32_t a_tmem, int32_t n, int32_t m, int32_t reps, float* out,
                                            int32_t* status, void* cuda_stream) {
   using namespace mdn;
-  if (!out || !status || (n != 32 && n != 64 && n != 128 && n != 256) || reps < 1 || reps > 4096) return MDN_ERR_INVALID_ARG;
+  if (!out || !status || (n != 32 && n != 64 && n != 128 && n != 256) || (m != 64 && m != 128) || reps < 1 || reps > 4096)
+    return MDN_ERR_INVALID_ARG;
   const int smem = 16384 + 32768 + 1024;
   if (cudaFuncSetAttribute(mma_timing_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
     return MDN_ERR_CUDA;
-  mma_timing_kernel<<<1, 128, smem, static_cast<cudaStream_t>(cuda_stream)>>>(tf32, a_tmem, n, reps, out, status);
+  mma_timing_kernel<<<1, 128, smem, static_cast<cudaStream_t>(cuda_stream)>>>(tf32, a_tmem, n, m, reps, out, status);
   return cudaGetLastError() == cudaSuccess ? MDN_OK : MDN_ERR_CUDA;
 }

@@ -23,7 +23,7 @@ def probe():
     L.mdn_probe_tf32.restype = ctypes.c_int
     L.mdn_probe_tf32.argtypes = [ctypes.c_int32, vp, vp, vp, vp, vp, vp]
     L.mdn_probe_mma_timing.restype = ctypes.c_int
-    L.mdn_probe_mma_timing.argtypes = [ctypes.c_int32] * 4 + [vp, vp, vp]
+    L.mdn_probe_mma_timing.argtypes = [ctypes.c_int32] * 5 + [vp, vp, vp]
     L.mdn_probe_bounded_wait.restype = ctypes.c_int
     L.mdn_probe_bounded_wait.argtypes = [ctypes.c_uint32, vp, vp]
     return L
@@ -210,20 +210,21 @@ def test_product_cost_by_shape(probe):
     """Cycles per tcgen05 product (M = 128) by kind, A source and N: printed for the design notes; asserts only that
     every shape completes and that a product never gets cheaper when N grows."""
     import torch
-    for tf32 in (0, 1):
-        for a_tmem in (0, 1):
-            row = []
-            for n in (32, 64, 128, 256):
-                out = torch.zeros(2, dtype=torch.float32, device="cuda")
-                status = torch.zeros(4, dtype=torch.int32, device="cuda")
-                assert probe.mdn_probe_mma_timing(tf32, a_tmem, n, 256, _ptr(out), _ptr(status), _stream()) == 0
-                torch.cuda.synchronize()
-                assert int(status[0]) == 0
-                row.append(float(out[0]) / float(out[1]))
-            print("%s, A from %s: cycles per product at N = 32, 64, 128, 256: %s"
-                  % ("tf32 K=8 " if tf32 else "bf16 K=16", "tensor memory" if a_tmem else "shared memory",
-                     ", ".join("%.1f" % x for x in row)))
-            assert row[3] >= row[1] * 0.9
+    for m in (128, 64):
+        for tf32 in (0, 1):
+            for a_tmem in (0, 1):
+                row = []
+                for n in (32, 64, 128, 256):
+                    out = torch.zeros(2, dtype=torch.float32, device="cuda")
+                    status = torch.zeros(4, dtype=torch.int32, device="cuda")
+                    assert probe.mdn_probe_mma_timing(tf32, a_tmem, n, m, 256, _ptr(out), _ptr(status), _stream()) == 0
+                    torch.cuda.synchronize()
+                    assert int(status[0]) == 0
+                    row.append(float(out[0]) / float(out[1]))
+                print("M = %3d, %s, A from %s: cycles per product at N = 32, 64, 128, 256: %s"
+                      % (m, "tf32 K=8 " if tf32 else "bf16 K=16", "tensor memory" if a_tmem else "shared memory",
+                         ", ".join("%.1f" % x for x in row)))
+                assert row[3] >= row[1] * 0.9
 
 
 # ------------------------------------------------------------------------------------------ bounded waits
