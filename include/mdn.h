@@ -62,7 +62,8 @@ typedef enum { MDN_F32 = 0, MDN_BF16 = 1 } mdn_dtype;
 typedef enum {
   MDN_PATH_AUTO = 0,    /* fp32 i/o -> SIMT fp32; bf16 i/o -> tensor-core path          */
   MDN_PATH_SIMT = 1,    /* fp32 FMA everywhere (any i/o dtype)                          */
-  MDN_PATH_TENSOR = 2   /* tcgen05 bf16 MMAs with fp32 TMEM accumulators (bf16 i/o, d=128) */
+  MDN_PATH_TENSOR = 2   /* tcgen05 MMAs with fp32 TMEM accumulators (bf16 i/o, d=128): the state is read as tf32
+                           straight from its fp32 masters, operands made from accumulators are bf16 hi + lo */
 } mdn_path;
 
 typedef struct {
@@ -414,7 +415,9 @@ mdn_status mdn_chunk_bwd(const mdn_params* p,
  * Positions past the end of a short chunk hold exact no-ops (alpha = mu = 1, beta = eta = 0).
  *
  * mdn_intra_chunk (a2, Eq. 15 and the mask of Eq. 12): per (s, h) the 64x64 row-major
- * matrices T and W, as float32 (SIMT path) or bfloat16 (tensor path).
+ * matrices T and W, as float32 (SIMT path) or bfloat16 (tensor path; W as a bf16 hi part and a bf16 lo part of
+ * the residual, W = hi + lo).  Inside mdn_chunk_fwd the plain tensor-path forward has the same kernel write W as
+ * float32 into the same 16 KB per matrix (its chain kernel reads W as a tf32 operand); T is bfloat16 there too.
  */
 #define MDN_NUM_COEF 12
 
@@ -426,7 +429,7 @@ typedef struct {
   uint64_t off_slot_map;    /* int32[num_slots][4]: seq, first token, valid tokens n, local chunk index  */
   uint64_t off_coef;        /* float32[num_slots][H][MDN_NUM_COEF][64]                                   */
   uint64_t off_T;           /* [num_slots][H][64][64]                                                    */
-  uint64_t off_W;           /* [num_slots][H][64][64]  (tensor path: bf16 hi part; lo part follows)      */
+  uint64_t off_W;           /* [num_slots][H][64][64]  (tensor path: bf16 hi part, lo part follows; or fp32) */
   uint64_t total_bytes;
   uint64_t off_seg;         /* segment states, Psi and Phi matrices of the parallel scan (fp32)          */
   int32_t segments;         /* segments per sequence the call will use (1 = plain serial chain)          */

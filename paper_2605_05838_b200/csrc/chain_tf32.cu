@@ -17,8 +17,8 @@
 //        Q S, Q M likewise                                       ->  o_inter = cZ .* Z + cU .* U
 //        dS / g11' + (g12' / (g11' g22')) dM,  dM / g22'         ->  per-token weights wS, wM of V~ in the updates
 //    with cX = abar g11, cY = (alpha b^-) g22 - abar g12, cZ = scale abar g11, cU = scale (abar g12 - b g22),
-//    wS = (gS + (g12'/g22') gM) / g11', wM = gM / g22' (gS = gamma_C eta, gM = (mubar_C/mubar) eta).  The converter
-//    warps run the scalar recurrence of G and write these six vectors per chunk.  When G' would leave a safe range
+//    wS = (gS + (g12'/g22') gM) / g11', wM = gM / g22' (gS = gamma_C eta, gM = (mubar_C/mubar) eta).  The producer
+//    warp runs the scalar recurrence of G and writes these six vectors per chunk.  When G' would leave a safe range
 //    (g11' or g22' below 2^-64, or |g12'| above g22': fast-decaying gates, mu = 0 tokens, S decaying slower than M) the chunk is "eager":
 //    the epilogue warps rescale the masters once by G' (the first design's pre-scaling, with G folded in) and G
 //    returns to the identity.  The result is the same recurrence either way; only rounding differs.
@@ -76,7 +76,7 @@ constexpr uint32_t kAdjBytes = 2048;
 constexpr uint32_t kSmemBytes = kOffAdj + 2 * kAdjBytes + 1024;
 static_assert(kStCoef + kCoefBytes <= kStageBytes && kSmemBytes <= 232448, "shared-memory layout");
 
-// per-chunk block the converter warps publish (float indices)
+// per-chunk block the producer warp publishes (float indices)
 enum Adj : int { kCx = 0, kCy = 64, kCz = 128, kCu = 192, kWs = 256, kWm = 320, kN11 = 384, kN12, kN22, kLazy };
 constexpr float kLazyMin = 5.421010862427522e-20f;   // 2^-64: smallest g11', g22' a lazy chunk may leave
 constexpr float kLazyMix = 1.f;                      // largest |g12'| / g22' (beyond it the two hat terms of S cancel too much)
@@ -419,7 +419,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tf32_kernel(const Args a, c
           umma_commit(b_m1);
         }
         MDN_MARK(c, kEvYuIssued);
-        // (T, W and the bf16 K tile of the stage have landed: the converters waited for them before they published the
+        // (T, W and the bf16 K tile of the stage have landed: the producer warp waited for them before it published the
         // coefficients the epilogue has used by the time it hands R over)
         // ---- MMA-2: Y = (R_hi + R_lo)^T T^T
         MDN_SPIN(b_r, ph);
