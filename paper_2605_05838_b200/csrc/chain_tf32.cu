@@ -344,7 +344,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tf32_kernel(const Args a, c
             const float ab = cf[kAbar * C + t], bb = cf[kB * C + t], pp = cf[kAlphaBPrev * C + t];
             const float gs = cf[kGS * C + t], gm = cf[kGM * C + t];
             const float cx = ab * g11, cy = pp * g22 - ab * g12;
-            aj[kCx + t] = cx;
+            aj[kCx + t] = -cx;     // stored negated: the epilogue's first step is one packed FMA per token pair
             aj[kCy + t] = cy;
             aj[kCz + t] = a.scale * cx;
             aj[kCu + t] = a.scale * (ab * g12 - bb * g22);
@@ -564,13 +564,16 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tf32_kernel(const Args a, c
       {
         // V and the coefficients are fetched BEFORE the waits: shared-memory loads issued after a wait would sit on the
         // chain's critical path, behind whatever the converter warps have queued in the shared-memory pipe
-        float vv[kTok], cf1[kTok];
+        // (token pairs as float2: the per-token arithmetic runs on the packed two-lane fp32 instructions)
+        float2 vv[kTok / 2], cf1[kTok / 2];
 #pragma unroll
-        for (int j = 0; j < kTok; ++j) vv[j] = v_zero ? 0.f : __bfloat162float(sV[(r0 + j) * kD + d]);
+        for (int j = 0; j < kTok; j += 2)
+          vv[j >> 1] = v_zero ? make_float2(0.f, 0.f)
+                              : make_float2(__bfloat162float(sV[(r0 + j) * kD + d]), __bfloat162float(sV[(r0 + j + 1) * kD + d]));
 #pragma unroll
         for (int j = 0; j < kTok; j += 4) {
-          const float4 cx = *reinterpret_cast<const float4*>(aj + kCx + r0 + j);
-          cf1[j] = cx.x; cf1[j + 1] = cx.y; cf1[j + 2] = cx.z; cf1[j + 3] = cx.w;
+          const float4 cx = *reinterpret_cast<const float4*>(aj + kCx + r0 + j);   // -cX
+          cf1[j >> 1] = make_float2(cx.x, cx.y); cf1[(j >> 1) + 1] = make_float2(cx.z, cx.w);
         }
         MDN_WAIT(b_mx, ph);          // X is there; Y is still being computed
         __syncwarp();
@@ -580,12 +583,13 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tf32_kernel(const Args a, c
           tmem_ld32(tl + kColX + r0, x);
           tmem_wait_ld();
 #pragma unroll
-          for (int j = 0; j < kTok; ++j) vv[j] -= cf1[j] * __uint_as_float(x[j]);
+          for (int j = 0; j < kTok; j += 2)
+            vv[j >> 1] = __ffma2_rn(cf1[j >> 1], make_float2(__uint_as_float(x[j]), __uint_as_float(x[j + 1])), vv[j >> 1]);
         }
 #pragma unroll
         for (int j = 0; j < kTok; j += 4) {
           const float4 cy = *reinterpret_cast<const float4*>(aj + kCy + r0 + j);
-          cf1[j] = cy.x; cf1[j + 1] = cy.y; cf1[j + 2] = cy.z; cf1[j + 3] = cy.w;
+          cf1[j >> 1] = make_float2(cy.x, cy.y); cf1[(j >> 1) + 1] = make_float2(cy.z, cy.w);
         }
         MDN_WAIT(b_m1, ph);
         __syncwarp();
@@ -597,14 +601,9 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tf32_kernel(const Args a, c
           tmem_ld32(tl + kColY + r0, y);
           tmem_wait_ld();
 #pragma unroll
-          for (int j = 0; j < kTok; j += 4) {
-            const float e0 = vv[j + 0] + cf1[j + 0] * __uint_as_float(y[j + 0]);
-            const float e1 = vv[j + 1] + cf1[j + 1] * __uint_as_float(y[j + 1]);
-            const float e2 = vv[j + 2] + cf1[j + 2] * __uint_as_float(y[j + 2]);
-            const float e3 = vv[j + 3] + cf1[j + 3] * __uint_as_float(y[j + 3]);
-            split_pack_bf16(e0, e1, hi[j >> 1], lo[j >> 1]);
-            split_pack_bf16(e2, e3, hi[(j >> 1) + 1], lo[(j >> 1) + 1]);
-          }
+          for (int j = 0; j < kTok; j += 2)
+            split_pack_bf16(__ffma2_rn(cf1[j >> 1], make_float2(__uint_as_float(y[j]), __uint_as_float(y[j + 1])), vv[j >> 1]),
+                            hi[j >> 1], lo[j >> 1]);
         }
         // hi and lo both go into the columns this warp has just read (its own kTok columns of X)
         tmem_st16(tl + kColX + r0, hi);
@@ -620,17 +619,21 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tf32_kernel(const Args a, c
         uint32_t z[kTok], u[kTok];
         tmem_ld32(tl + kColZ + r0, z);
         tmem_ld32(tl + kColU + r0, u);
-        float cz[kTok], cu[kTok];   // (their loads run while the tensor-memory loads are in flight)
+        float2 cz[kTok / 2], cu[kTok / 2];   // (their loads run while the tensor-memory loads are in flight)
 #pragma unroll
         for (int j = 0; j < kTok; j += 4) {
           const float4 a4 = *reinterpret_cast<const float4*>(aj + kCz + r0 + j);
           const float4 b4 = *reinterpret_cast<const float4*>(aj + kCu + r0 + j);
-          cz[j] = a4.x; cz[j + 1] = a4.y; cz[j + 2] = a4.z; cz[j + 3] = a4.w;
-          cu[j] = b4.x; cu[j + 1] = b4.y; cu[j + 2] = b4.z; cu[j + 3] = b4.w;
+          cz[j >> 1] = make_float2(a4.x, a4.y); cz[(j >> 1) + 1] = make_float2(a4.z, a4.w);
+          cu[j >> 1] = make_float2(b4.x, b4.y); cu[(j >> 1) + 1] = make_float2(b4.z, b4.w);
         }
         tmem_wait_ld();
 #pragma unroll
-        for (int j = 0; j < kTok; ++j) u[j] = __float_as_uint(cz[j] * __uint_as_float(z[j]) + cu[j] * __uint_as_float(u[j]));
+        for (int j = 0; j < kTok; j += 2) {
+          const float2 t2 = __fmul2_rn(cu[j >> 1], make_float2(__uint_as_float(u[j]), __uint_as_float(u[j + 1])));
+          const float2 o2 = __ffma2_rn(cz[j >> 1], make_float2(__uint_as_float(z[j]), __uint_as_float(z[j + 1])), t2);
+          u[j] = __float_as_uint(o2.x); u[j + 1] = __float_as_uint(o2.y);
+        }
         tmem_st32(tl + kColU + r0, u);
         tmem_wait_st();
         tc_fence_before_sync();
@@ -649,23 +652,21 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tf32_kernel(const Args a, c
       {
         uint32_t vt[kTok];
         tmem_ld32(tl + kColY + r0, vt);
-        float wsv[kTok], wmv[kTok];   // (their loads run while the tensor-memory load is in flight)
+        float2 wsv[kTok / 2], wmv[kTok / 2];   // (their loads run while the tensor-memory load is in flight)
 #pragma unroll
         for (int j = 0; j < kTok; j += 4) {
           const float4 a4 = *reinterpret_cast<const float4*>(aj + kWs + r0 + j);
           const float4 b4 = *reinterpret_cast<const float4*>(aj + kWm + r0 + j);
-          wsv[j] = a4.x; wsv[j + 1] = a4.y; wsv[j + 2] = a4.z; wsv[j + 3] = a4.w;
-          wmv[j] = b4.x; wmv[j + 1] = b4.y; wmv[j + 2] = b4.z; wmv[j + 3] = b4.w;
+          wsv[j >> 1] = make_float2(a4.x, a4.y); wsv[(j >> 1) + 1] = make_float2(a4.z, a4.w);
+          wmv[j >> 1] = make_float2(b4.x, b4.y); wmv[(j >> 1) + 1] = make_float2(b4.z, b4.w);
         }
         tmem_wait_ld();
         {
           uint32_t sh[kPk], sl[kPk];
 #pragma unroll
-          for (int j = 0; j < kTok; j += 4) {
-            split_pack_bf16(wsv[j] * __uint_as_float(vt[j]), wsv[j + 1] * __uint_as_float(vt[j + 1]), sh[j >> 1], sl[j >> 1]);
-            split_pack_bf16(wsv[j + 2] * __uint_as_float(vt[j + 2]), wsv[j + 3] * __uint_as_float(vt[j + 3]), sh[(j >> 1) + 1],
-                            sl[(j >> 1) + 1]);
-          }
+          for (int j = 0; j < kTok; j += 2)
+            split_pack_bf16(__fmul2_rn(wsv[j >> 1], make_float2(__uint_as_float(vt[j]), __uint_as_float(vt[j + 1]))),
+                            sh[j >> 1], sl[j >> 1]);
           tmem_st16(tl + kColX + r0, sh);          // X is free: MMA-2 has consumed R
           tmem_st16(tl + kColX + r0 + kPk, sl);
         }
@@ -690,11 +691,9 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tf32_kernel(const Args a, c
         MDN_MARK2(c, kEvV1Arrive2);
         uint32_t mh[kPk], mlo[kPk];
 #pragma unroll
-        for (int j = 0; j < kTok; j += 4) {
-          split_pack_bf16(wmv[j] * __uint_as_float(vt[j]), wmv[j + 1] * __uint_as_float(vt[j + 1]), mh[j >> 1], mlo[j >> 1]);
-          split_pack_bf16(wmv[j + 2] * __uint_as_float(vt[j + 2]), wmv[j + 3] * __uint_as_float(vt[j + 3]), mh[(j >> 1) + 1],
-                          mlo[(j >> 1) + 1]);
-        }
+        for (int j = 0; j < kTok; j += 2)
+          split_pack_bf16(__fmul2_rn(wmv[j >> 1], make_float2(__uint_as_float(vt[j]), __uint_as_float(vt[j + 1]))),
+                          mh[j >> 1], mlo[j >> 1]);
         if (write_o) {   // MMA-3' reads V~ from Y: it must be done before Y is overwritten
           MDN_WAIT(b_mo, ph);
           __syncwarp();

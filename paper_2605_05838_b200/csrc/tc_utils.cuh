@@ -322,6 +322,15 @@ __device__ __forceinline__ void split_pack_bf16(float x0, float x1, uint32_t& hi
   lo = pack_bf16(x0 - h0, x1 - h1);
 }
 
+// The same for a pair held as float2, with the packed two-lane fp32 instructions of sm_100 (one FFMA2 for the two
+// residuals: x - h = fma(h, -1, x), exact).
+__device__ __forceinline__ void split_pack_bf16(float2 x, uint32_t& hi, uint32_t& lo) {
+  hi = pack_bf16(x.x, x.y);
+  const float2 h = make_float2(__uint_as_float(hi << 16), __uint_as_float(hi & 0xFFFF0000u));
+  const float2 res = __ffma2_rn(h, make_float2(-1.f, -1.f), x);
+  lo = pack_bf16(res.x, res.y);
+}
+
 }  // namespace tc
 
 // ----------------------------------------------------------------------------- host: tensor maps
