@@ -645,6 +645,15 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tf32_kernel(const Args a, c
       // chunk, their last reader, is done) and the update is added in true coordinates.
       const bool eager = aj[kLazy] == 0.f;
       const float n11 = aj[kN11], n12 = aj[kN12], n22 = aj[kN22];
+      // (the first operand's weights are fetched before the wait: shared-memory loads issued after it sit on the
+      // chain's critical path behind whatever the converter warps have queued)
+      float2 wsv[kTok / 2];
+#pragma unroll
+      for (int j = 0; j < kTok; j += 4) {
+        float4 a4;
+        asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(a4.x), "=f"(a4.y), "=f"(a4.z), "=f"(a4.w) : "r"(smem_u32(aj + kWs + r0 + j)));
+        wsv[j >> 1] = make_float2(a4.x, a4.y); wsv[(j >> 1) + 1] = make_float2(a4.z, a4.w);
+      }
       MDN_WAIT(b_m2, ph);
       __syncwarp();
       tc_fence_after_sync();
@@ -652,12 +661,10 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tf32_kernel(const Args a, c
       {
         uint32_t vt[kTok];
         tmem_ld32(tl + kColY + r0, vt);
-        float2 wsv[kTok / 2], wmv[kTok / 2];   // (their loads run while the tensor-memory load is in flight)
+        float2 wmv[kTok / 2];   // (their loads run while the tensor-memory load is in flight)
 #pragma unroll
         for (int j = 0; j < kTok; j += 4) {
-          const float4 a4 = *reinterpret_cast<const float4*>(aj + kWs + r0 + j);
           const float4 b4 = *reinterpret_cast<const float4*>(aj + kWm + r0 + j);
-          wsv[j >> 1] = make_float2(a4.x, a4.y); wsv[(j >> 1) + 1] = make_float2(a4.z, a4.w);
           wmv[j >> 1] = make_float2(b4.x, b4.y); wmv[(j >> 1) + 1] = make_float2(b4.z, b4.w);
         }
         tmem_wait_ld();

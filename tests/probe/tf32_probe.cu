@@ -330,31 +330,28 @@ __global__ void __launch_bounds__(128) mma_timing_kernel(int tf32, int a_tmem, i
     const uint64_t da = smem_desc_sw128(smem_u32(smem), 16, 1024);              // A block: 128 rows x 128 B
     const uint64_t db = smem_desc_sw128(smem_u32(smem) + 16384, 16, 1024);      // B block: up to 256 rows x 128 B
     const uint32_t ta = tmem + 256;
+    const uint32_t id_mn = idesc_bf16(M, N, false, true, false);
+    const uint64_t db_mn = smem_desc_sw128(smem_u32(smem) + 16384, 8192, 1024);
+    // one branch-free, fully unrolled issue loop per variant (a branch inside the loop would time the issuing thread,
+    // not the tensor pipe); sixteen products per iteration, as the kernels issue them
     const long long t0 = clock64();
-    for (int rep = 0; rep < reps; ++rep) {
-      if (tf32) {
-        if (a_tmem) {
-#pragma unroll
-          for (int k = 0; k < 4; ++k) umma_ts_tf32(tmem, ta + 8 * k, db + 2 * k, id, true);
-        } else {
-#pragma unroll
-          for (int k = 0; k < 4; ++k) umma_ss_tf32(tmem, da + 2 * k, db + 2 * k, id, true);
-        }
-      } else {
-        if (a_tmem) {
-#pragma unroll
-          for (int k = 0; k < 4; ++k) umma_ts(tmem, ta + 8 * k, db + 2 * k, id, true);
-        } else {
-#pragma unroll
-          for (int k = 0; k < 4; ++k) umma_ss(tmem, da + 2 * k, db + 2 * k, id, true);
-        }
-      }
+#define MDN_TIMING_LOOP(CALL)                                   \
+    for (int rep = 0; rep < reps; rep += 4) {                   \
+      _Pragma("unroll") for (int k = 0; k < 16; ++k) { CALL; }  \
     }
+    if (tf32 && a_tmem) { MDN_TIMING_LOOP(umma_ts_tf32(tmem, ta + 8 * (k & 3), db + 2 * (k & 3), id, true)) }
+    else if (tf32) { MDN_TIMING_LOOP(umma_ss_tf32(tmem, da + 2 * (k & 3), db + 2 * (k & 3), id, true)) }
+    else if (a_tmem == 2) { MDN_TIMING_LOOP(umma_ts(tmem, ta + 8 * (k & 3), db_mn + 128 * (k & 3), id_mn, true)) }
+    else if (a_tmem) { MDN_TIMING_LOOP(umma_ts(tmem, ta + 8 * (k & 3), db + 2 * (k & 3), id, true)) }
+    else { MDN_TIMING_LOOP(umma_ss(tmem, da + 2 * (k & 3), db + 2 * (k & 3), id, true)) }
+#undef MDN_TIMING_LOOP
+    const long long t_issued = clock64();
     umma_commit(b_done);
     ok = mbar_wait(b_done, 0, &abort_flag);
     const long long t1 = clock64();
+    out[2] = static_cast<float>(t_issued - t0);   // until the last product was issued
     out[0] = static_cast<float>(t1 - t0);
-    out[1] = static_cast<float>(4 * reps);
+    out[1] = static_cast<float>(16 * ((reps + 3) / 4));
   }
   if (!ok && tid == 0) atomicCAS(status, kDevOk, kDevTimeout);
   tc_fence_before_sync();

@@ -213,18 +213,26 @@ def test_product_cost_by_shape(probe):
     for m in (128, 64):
         for tf32 in (0, 1):
             for a_tmem in (0, 1):
-                row = []
+                row, issue = [], []
                 for n in (32, 64, 128, 256):
-                    out = torch.zeros(2, dtype=torch.float32, device="cuda")
+                    out = torch.zeros(4, dtype=torch.float32, device="cuda")
                     status = torch.zeros(4, dtype=torch.int32, device="cuda")
                     assert probe.mdn_probe_mma_timing(tf32, a_tmem, n, m, 256, _ptr(out), _ptr(status), _stream()) == 0
                     torch.cuda.synchronize()
                     assert int(status[0]) == 0
                     row.append(float(out[0]) / float(out[1]))
+                    issue.append(float(out[2]) / float(out[1]))
                 print("M = %3d, %s, A from %s: cycles per product at N = 32, 64, 128, 256: %s"
                       % (m, "tf32 K=8 " if tf32 else "bf16 K=16", "tensor memory" if a_tmem else "shared memory",
-                         ", ".join("%.1f" % x for x in row)))
+                         ", ".join("%.1f" % x for x in row)) + "  (issuing thread alone: %s)" % ", ".join("%.1f" % x for x in issue))
                 assert row[3] >= row[1] * 0.9
+    # the state update's form: bf16, A from tensor memory, B a [64 x 128] tile read MN-major (N = 128 only)
+    out = torch.zeros(4, dtype=torch.float32, device="cuda")
+    status = torch.zeros(4, dtype=torch.int32, device="cuda")
+    assert probe.mdn_probe_mma_timing(0, 2, 128, 128, 256, _ptr(out), _ptr(status), _stream()) == 0
+    torch.cuda.synchronize()
+    assert int(status[0]) == 0
+    print("M = 128, bf16 K=16, A from tensor memory, B MN-major, N = 128: %.1f cycles per product" % (float(out[0]) / float(out[1])))
 
 
 # ------------------------------------------------------------------------------------------ bounded waits
