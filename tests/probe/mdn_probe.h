@@ -47,7 +47,7 @@ mdn_status mdn_probe_tf32(int32_t mode, const float* a, const float* b, const fl
 
 /*
  * Cost of one tcgen05 product as a function of its shape: a stream of 4 * reps products D[m x n] += A[m x K] *
- * B[n x K]^T (K = 16 bf16 or 8 tf32 elements), A from tensor memory (a_tmem = 1; a_tmem = 2: bf16 with B read MN-major, n = 128) or from shared memory, issued by one
+ * B[n x K]^T (K = 16 bf16 or 8 tf32 elements), A from tensor memory (a_tmem = 1; a_tmem = 2: bf16 with B read MN-major, n = 128; a_tmem = 3: tf32, sixteen k-steps over 128 columns of A and 64 KB of B, n = 128) or from shared memory, issued by one
  * thread; out[0] = cycles from the first issue to completion, out[1] = products issued.  n in {32, 64, 128, 256},
  * m in {64, 128}.
  */

@@ -309,7 +309,7 @@ __global__ void __launch_bounds__(128) mma_timing_kernel(int tf32, int a_tmem, i
   const uint32_t b_done = smem_u32(&bar);
   if (tid == 0) { abort_flag = 0; mbar_init(b_done, 1); mbar_fence_init(); }
   if (warp == 0) tmem_alloc(smem_u32(&tmem_slot), 512);
-  for (int i = tid; i < (16384 + 32768) / 4; i += 128) reinterpret_cast<uint32_t*>(smem)[i] = 0x3c003c00u;
+  for (int i = tid; i < (16384 + 65536) / 4; i += 128) reinterpret_cast<uint32_t*>(smem)[i] = 0x3c003c00u;
   fence_proxy_async_smem();
   tc_fence_before_sync();
   __syncthreads();
@@ -318,7 +318,8 @@ __global__ void __launch_bounds__(128) mma_timing_kernel(int tf32, int a_tmem, i
   {
     uint32_t r[32];
     for (int j = 0; j < 32; ++j) r[j] = 0x3c003c00u;
-    tmem_st32(tmem + (static_cast<uint32_t>(warp * 32) << 16) + 256, r);   // A operand columns 256..287
+    for (int c0 = 0; c0 < 128; c0 += 32)
+      tmem_st32(tmem + (static_cast<uint32_t>(warp * 32) << 16) + 256 + c0, r);   // A operand columns 256..383
     tmem_wait_st();
   }
   tc_fence_before_sync();
@@ -339,7 +340,9 @@ __global__ void __launch_bounds__(128) mma_timing_kernel(int tf32, int a_tmem, i
     for (int rep = 0; rep < reps; rep += 4) {                   \
       _Pragma("unroll") for (int k = 0; k < 16; ++k) { CALL; }  \
     }
-    if (tf32 && a_tmem) { MDN_TIMING_LOOP(umma_ts_tf32(tmem, ta + 8 * (k & 3), db + 2 * (k & 3), id, true)) }
+    if (tf32 && a_tmem == 3) {   // the chain kernel's MMA-1: sixteen k-steps over 128 columns of A and four 16 KB panels of B
+      MDN_TIMING_LOOP(umma_ts_tf32(tmem, ta + 8 * k, db + (uint64_t)((k >> 2) * 1024 + (k & 3) * 2), id, true))
+    } else if (tf32 && a_tmem) { MDN_TIMING_LOOP(umma_ts_tf32(tmem, ta + 8 * (k & 3), db + 2 * (k & 3), id, true)) }
     else if (tf32) { MDN_TIMING_LOOP(umma_ss_tf32(tmem, da + 2 * (k & 3), db + 2 * (k & 3), id, true)) }
     else if (a_tmem == 2) { MDN_TIMING_LOOP(umma_ts(tmem, ta + 8 * (k & 3), db_mn + 128 * (k & 3), id_mn, true)) }
     else if (a_tmem) { MDN_TIMING_LOOP(umma_ts(tmem, ta + 8 * (k & 3), db + 2 * (k & 3), id, true)) }
@@ -408,7 +411,7 @@ extern "C" mdn_status mdn_probe_mma_timing(int32_t tf32, int32_t a_tmem, int32_t
   using namespace mdn;
   if (!out || !status || (n != 32 && n != 64 && n != 128 && n != 256) || (m != 64 && m != 128) || reps < 1 || reps > 4096)
     return MDN_ERR_INVALID_ARG;
-  const int smem = 16384 + 32768 + 1024;
+  const int smem = 16384 + 65536 + 1024;
   if (cudaFuncSetAttribute(mma_timing_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
     return MDN_ERR_CUDA;
   mma_timing_kernel<<<1, 128, smem, static_cast<cudaStream_t>(cuda_stream)>>>(tf32, a_tmem, n, m, reps, out, status);

@@ -233,6 +233,11 @@ def test_product_cost_by_shape(probe):
     torch.cuda.synchronize()
     assert int(status[0]) == 0
     print("M = 128, bf16 K=16, A from tensor memory, B MN-major, N = 128: %.1f cycles per product" % (float(out[0]) / float(out[1])))
+    assert probe.mdn_probe_mma_timing(1, 3, 128, 128, 256, _ptr(out), _ptr(status), _stream()) == 0
+    torch.cuda.synchronize()
+    assert int(status[0]) == 0
+    print("M = 128, tf32, A = 128 columns of tensor memory, B = 64 KB in four panels (the chain kernel's first product), "
+          "N = 128: %.1f cycles per product" % (float(out[0]) / float(out[1])))
 
 
 # ------------------------------------------------------------------------------------------ bounded waits
