@@ -968,10 +968,9 @@ cudaError_t launch_intra_tensor(const Plan& pl, const void* q, const void* k, co
 }
 
 bool chain_uses_tf32_kernel(const Plan& pl) {
-  const bool layer = pl.qk.on || pl.post.on;
   const bool train = pl.chain_dump != nullptr || pl.chain_state_only || pl.chain_end_scalars_in_rk ||
                      pl.chain_vt_dump != nullptr || pl.chain_inject || pl.chain_mirror_geom != nullptr;
-  return pl.p.path == MDN_PATH_TENSOR && !layer && !train;
+  return pl.p.path == MDN_PATH_TENSOR && !train;
 }
 
 cudaError_t launch_chain_tensor(const Plan& pl, const void* q, const void* k, const void* v, const float* S0,

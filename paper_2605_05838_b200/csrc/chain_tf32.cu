@@ -1,6 +1,8 @@
 // a3 + a4 of the plain forward on the 5th-generation tensor cores (tcgen05, sm_100a), second design: one CTA walks
 // the chunks of one (sequence, head) in order; bf16 q/k/v, dk = dv = 128, chunk 64.  (The first design,
-// chain_tensor.cu, stays for the forward with layer operations and for the training / backward runs.)
+// chain_tensor.cu, stays for the training / backward runs.)  Template flag kLayer: the layer's element-wise operations
+// of Section 3.3 inside this kernel (q/k norm through the coefficient vectors and the converter warps, RMSNorm and
+// sigmoid gate in the output step); kLayer = false compiles them out.
 //
 // Everything is kept TRANSPOSED: the value dimension (128) is the MMA M dimension and fills the 128 tensor-memory
 // lanes, tokens are N (or K).  What is different here:
@@ -104,6 +106,7 @@ struct Bars {
   uint64_t m3;        // MMA-3 done                                                       (commit)
   uint64_t mo;        // MMA-3' done                                                      (commit)
   uint64_t zu;        // U (the chunk's output) has been read                              (256)
+  uint64_t pn;        // fused output step: the fp32 tile is staged / has been read            (256)
 };
 
 struct Args {
@@ -124,7 +127,20 @@ struct Args {
   float* seg_PhiS;
   float* seg_PhiM;
   long long* timeline;   // debug builds: CTA 0 writes clock64() at [chunk * 32 + event]
+  // layer operations (Section 3.3), kLayer instantiation only
+  int qk_on;             // q <- L2Norm(q - d k), k <- L2Norm(k): 1/|k|, 1/|q - d k| arrive as coefficient vectors 6, 7
+  const float* qk_d;     // [H] or NULL
+  int post_on;           // o <- sigmoid(g) * RMSNorm(o) * w in the output step
+  const float* post_w;   // [dv] or NULL
+  const void* post_g;    // [B,T,H,dv] bf16
+  float post_eps;
 };
+
+__device__ __forceinline__ float sigmoid_fast(float x) {
+  float t;
+  asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(0.5f * x));
+  return fmaf(0.5f, t, 0.5f);
+}
 
 enum Ev : int { kEvMma1 = 0, kEvM1Seen, kEvRArrive, kEvOiArrive, kEvM2Seen, kEvV1Arrive, kEvOutDone, kEvM3Seen, kEvRSeen,
                 kEvV1Seen, kEvCvtStart, kEvCvtDone, kEvTmaIssued, kEvStoresDone, kEvM2Own, kEvEager,
@@ -138,7 +154,7 @@ template <> __device__ __forceinline__ void stage_o<__nv_bfloat16>(uint8_t* tile
   reinterpret_cast<__nv_bfloat16*>(tile)[r * kD + d] = __float2bfloat16_rn(x);
 }
 
-template <typename TO>
+template <typename TO, bool kLayer>
 __global__ void __launch_bounds__(kThreads, 1) chain_tf32_kernel(const Args a, const __grid_constant__ CUtensorMap map_q,
                                                                 const __grid_constant__ CUtensorMap map_k,
                                                                 const __grid_constant__ CUtensorMap map_v,
@@ -151,6 +167,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tf32_kernel(const Args a, c
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
   __shared__ float g_final[4];   // G after the last chunk: what the final states are read through
+  __shared__ __align__(16) float w_sm[kLayer ? kD : 4];   // RMSNorm weight of the fused output step
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int H = a.g.H;
@@ -214,6 +231,10 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tf32_kernel(const Args a, c
   const uint32_t b_v1b = smem_u32(&bars.v1b), b_mx = smem_u32(&bars.mx), b_m3s = smem_u32(&bars.m3s);
   const uint32_t b_m3 = smem_u32(&bars.m3), b_mo = smem_u32(&bars.mo), b_zu = smem_u32(&bars.zu);
   const uint32_t b_fin = smem_u32(&bars.fin), b_cfull = smem_u32(&bars.cfull), b_cfree = smem_u32(&bars.cfree);
+  const uint32_t b_pn = smem_u32(&bars.pn);
+  // kLayer = false compiles the layer operations out
+  const bool qk_on = kLayer && a.qk_on;
+  const float qk_dh = (qk_on && a.qk_d) ? __ldg(a.qk_d + h) : 0.f;
 
   if (tid == 0) {
     abort_flag = 0;
@@ -223,9 +244,11 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tf32_kernel(const Args a, c
     mbar_init(b_fin, 32); mbar_init(b_cfull, 1); mbar_init(b_cfree, kCvtThreads);
     mbar_init(b_init, kEpiThreads); mbar_init(b_r, kEpiThreads); mbar_init(b_oi, kEpiThreads);
     mbar_init(b_v1a, kEpiThreads); mbar_init(b_v1b, kEpiThreads); mbar_init(b_zu, kEpiThreads);
+    if constexpr (kLayer) mbar_init(b_pn, kEpiThreads);
     mbar_init(b_m1, 1); mbar_init(b_m2, 1); mbar_init(b_m3, 1); mbar_init(b_mo, 1); mbar_init(b_mx, 1); mbar_init(b_m3s, 1);
     mbar_fence_init();
   }
+  if (kLayer && tid < kD) w_sm[tid] = (a.post_on && a.post_w) ? __ldg(a.post_w + tid) : 1.f;
   if (warp == kWarpMma) tmem_alloc(smem_u32(&tmem_slot), 512);
   if (warp == kWarpTma && lane == 0) {
     prefetch_tensormap(&map_q); prefetch_tensormap(&map_k); prefetch_tensormap(&map_v);
@@ -276,11 +299,28 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tf32_kernel(const Args a, c
     // Stage s = c & 1 serves chunk c, then (as the staged output tile) is written out and refilled for chunk c + 2.
     // The whole warp walks the loop; lane 0 issues the copies; every lane writes the coefficients of two tokens.
     {
-      int issued = 0;
+      int issued = 0, issued_kq = 0;
       float g11 = 1.f, g12 = 0.f, g22 = 1.f;
       for (int c = 0; c < nch + 2; ++c) {
         const int s = c & 1;
         const uint32_t st = s_base + kOffStage + s * kStageBytes;
+        if (c < nch) {
+          // the chunk's K and Q tiles for the converters first: their buffer is free long before the stage is, and
+          // with the fused q/k norm the converters need the head start
+          if (c > 0) MDN_WAIT(b_cfree, (c - 1) & 1);   // the previous chunk's bf16 K, Q have been read
+          if (lane == 0) {
+            const int tok0 = sq.tok0 + c * C;
+            mbar_arrive_expect_tx(b_cfull, write_o ? 32768u : 16384u);
+            tma_load_2d(s_base + kOffCvt, &map_k, h * kD, tok0, b_cfull);
+            tma_load_2d(s_base + kOffCvt + 8192, &map_k, h * kD + 64, tok0, b_cfull);
+            if (write_o) {
+              tma_load_2d(s_base + kOffCvt + 16384, &map_q, h * kD, tok0, b_cfull);
+              tma_load_2d(s_base + kOffCvt + 24576, &map_q, h * kD + 64, tok0, b_cfull);
+            }
+          }
+          __syncwarp();
+          issued_kq = c + 1;
+        }
         if (c >= 2) {
           const int co = c - 2;
           MDN_WAIT(s ? b_go1 : b_go0, (co >> 1) & 1);
@@ -304,18 +344,10 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tf32_kernel(const Args a, c
           MDN_MARK(co, kEvStoresDone);
         }
         if (c < nch) {
-          if (c > 0) MDN_WAIT(b_cfree, (c - 1) & 1);   // the previous chunk's bf16 K, Q have been read
           const uint32_t fb = s ? b_full1 : b_full0;
           if (lane == 0) {
             const int tok0 = sq.tok0 + c * C;
             const int mat = (sq.slot0 + c) * H + h;
-            mbar_arrive_expect_tx(b_cfull, write_o ? 32768u : 16384u);
-            tma_load_2d(s_base + kOffCvt, &map_k, h * kD, tok0, b_cfull);
-            tma_load_2d(s_base + kOffCvt + 8192, &map_k, h * kD + 64, tok0, b_cfull);
-            if (write_o) {
-              tma_load_2d(s_base + kOffCvt + 16384, &map_q, h * kD, tok0, b_cfull);
-              tma_load_2d(s_base + kOffCvt + 24576, &map_q, h * kD + 64, tok0, b_cfull);
-            }
             mbar_arrive_expect_tx(fb, kTxBytes - (write_o ? 0u : kTxW) - (v_zero ? kTxV : 0u));
             bulk_load(st + kStCoef, a.coef + (size_t)mat * MDN_NUM_COEF * C, kCoefBytes, fb);
             if (!v_zero) tma_load_2d(st + kStV, &map_v, h * kD, tok0, fb);
@@ -343,11 +375,21 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tf32_kernel(const Args a, c
             const int t = 2 * lane + e;
             const float ab = cf[kAbar * C + t], bb = cf[kB * C + t], pp = cf[kAlphaBPrev * C + t];
             const float gs = cf[kGS * C + t], gm = cf[kGM * C + t];
-            const float cx = ab * g11, cy = pp * g22 - ab * g12;
+            // fused q/k norm: k^ = k / |k| scales the rows of K S, K M (vectors 2, 3, 4 carry that factor already),
+            // q^ = (q - d k) / |q - d k| those of the output terms (the converter warps subtract d k from the Q tile)
+            float cx, cy, cz, cu;
+            if constexpr (kLayer) {
+              const float rk = cf[kRk * C + t], sq_ = a.scale * cf[kRq * C + t];
+              cx = ab * rk * g11; cy = pp * g22 - ab * rk * g12;
+              cz = sq_ * (ab * g11); cu = sq_ * (ab * g12 - bb * g22);
+            } else {
+              cx = ab * g11; cy = pp * g22 - ab * g12;
+              cz = a.scale * cx; cu = a.scale * (ab * g12 - bb * g22);
+            }
             aj[kCx + t] = -cx;     // stored negated: the epilogue's first step is one packed FMA per token pair
             aj[kCy + t] = cy;
-            aj[kCz + t] = a.scale * cx;
-            aj[kCu + t] = a.scale * (ab * g12 - bb * g22);
+            aj[kCz + t] = cz;
+            aj[kCu + t] = cu;
             aj[kWs + t] = lazy ? (gs + (n12 / n22) * gm) / n11 : gs;
             aj[kWm + t] = lazy ? gm / n22 : gm;
           }
@@ -362,7 +404,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tf32_kernel(const Args a, c
       if (!ok && lane == 0) {   // giving up: let the copies already in flight land before the CTA exits
         for (int c = max(0, issued - 2); c < issued; ++c)
           for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait((c & 1) ? b_full1 : b_full0, (c >> 1) & 1); ++it) {}
-        for (uint32_t it = 0; it < (1u << 16) && issued > 0 && !mbar_try_wait(b_cfull, (issued - 1) & 1); ++it) {}
+        for (uint32_t it = 0; it < (1u << 16) && issued_kq > 0 && !mbar_try_wait(b_cfull, (issued_kq - 1) & 1); ++it) {}
       }
       if (lane == 0) tma_store_wait_all();
     }
@@ -491,6 +533,27 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tf32_kernel(const Args a, c
           asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
                        : "=r"(u[c16].x), "=r"(u[c16].y), "=r"(u[c16].z), "=r"(u[c16].w)
                        : "r"(src + (c16 >> 3) * 8192 + ((static_cast<uint32_t>(c16 & 7) ^ sw) << 4)));
+        if (kLayer && which == 1 && qk_dh != 0.f) {   // (kLayer = false: compiled out)
+          // fused q/k norm: the Q tile's copy is q - d k (fp32, from the two bf16 rows): the output terms then come out
+          // of the same products as for a plain q (their 1/|q - d k| rides on the coefficients)
+#pragma unroll
+          for (int c16 = 0; c16 < 16; ++c16) {
+            uint4 kk;
+            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                         : "=r"(kk.x), "=r"(kk.y), "=r"(kk.z), "=r"(kk.w)
+                         : "r"(src - 16384 + (c16 >> 3) * 8192 + ((static_cast<uint32_t>(c16 & 7) ^ sw) << 4)));
+            const uint32_t qw[4] = {u[c16].x, u[c16].y, u[c16].z, u[c16].w}, kw[4] = {kk.x, kk.y, kk.z, kk.w};
+            uint32_t f[8];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              f[2 * e] = __float_as_uint(fmaf(-qk_dh, __uint_as_float(kw[e] << 16), __uint_as_float(qw[e] << 16)));
+              f[2 * e + 1] = __float_as_uint(fmaf(-qk_dh, __uint_as_float(kw[e] & 0xffff0000u), __uint_as_float(qw[e] & 0xffff0000u)));
+            }
+            const uint32_t d0 = dst + (c16 >> 2) * 16384, ch = static_cast<uint32_t>((c16 & 3) * 2);
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(d0 + ((ch ^ sw) << 4)), "r"(f[0]), "r"(f[1]), "r"(f[2]), "r"(f[3]) : "memory");
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(d0 + (((ch + 1) ^ sw) << 4)), "r"(f[4]), "r"(f[5]), "r"(f[6]), "r"(f[7]) : "memory");
+          }
+        } else {
 #pragma unroll
         for (int c16 = 0; c16 < 16; ++c16) {
           const uint32_t d0 = dst + (c16 >> 2) * 16384, ch = static_cast<uint32_t>((c16 & 3) * 2);
@@ -498,6 +561,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tf32_kernel(const Args a, c
                        "r"(u[c16].x & 0xffff0000u), "r"(u[c16].y << 16), "r"(u[c16].y & 0xffff0000u) : "memory");
           asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(d0 + (((ch + 1) ^ sw) << 4)), "r"(u[c16].z << 16),
                        "r"(u[c16].z & 0xffff0000u), "r"(u[c16].w << 16), "r"(u[c16].w & 0xffff0000u) : "memory");
+        }
         }
       }
       mbar_arrive(b_cfree);          // the bf16 tiles have been read: the next chunk's may land
@@ -513,8 +577,65 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tf32_kernel(const Args a, c
     const int d = q4 * 32 + lane;
     const int r0 = kTok * hf;
     const uint32_t tl = tmem + (static_cast<uint32_t>(q4 * 32) << 16);
+    const bool post = kLayer && a.post_on && write_o;
+    uint32_t pn_phase = 0;
     for (int c = 0; c <= nch; ++c) {
       const float* aj = reinterpret_cast<const float*>(smem + kOffAdj + (c & 1) * kAdjBytes);
+      if constexpr (kLayer) {
+        if (post && c > 0) {
+          // Fused output step of the previous chunk, second half: y = sigmoid(g) * o / sqrt(mean_d o^2 + eps) * w_d.
+          // The staged fp32 tile is re-read row-wise: four threads per token sum its 128 squares, rescale and gate.
+          // fp32 output: written back in place (a thread rewrites only the pieces it has read); bf16 output: the final
+          // tile goes over the start of the fp32 one, once every row has been read.  Then the stage is handed back.
+          const int cp = c - 1;
+          uint8_t* stp = smem + kOffStage + (cp & 1) * kStageBytes;
+          constexpr int kTpr = 4, kPieces = 8;   // threads per token, 16-byte fp32 pieces (8-byte gate pieces) per thread
+          float* tile = reinterpret_cast<float*>(stp + kStOut);
+          const int t128 = q4 * 32 + lane, prow = r0 + t128 / kTpr, part = t128 % kTpr;
+          const bool g_live = cp * C + prow < sq.len;
+          const uint2* gp = reinterpret_cast<const uint2*>(static_cast<const __nv_bfloat16*>(a.post_g) +
+                                                           ((size_t)(sq.tok0 + cp * C + prow) * H + h) * kD) + part;
+          uint2 graw[kPieces];
+#pragma unroll
+          for (int i = 0; i < kPieces; ++i) graw[i] = g_live ? __ldg(gp + kTpr * i) : make_uint2(0u, 0u);
+          MDN_WAIT(b_pn, pn_phase);
+          pn_phase ^= 1;
+          float4 ov[kPieces];
+          float ss = 0.f;
+#pragma unroll
+          for (int i = 0; i < kPieces; ++i) {   // interleaved 16-byte pieces: a row's threads cover contiguous bytes
+            ov[i] = *reinterpret_cast<const float4*>(tile + prow * kD + (part + kTpr * i) * 4);
+            ss = fmaf(ov[i].x, ov[i].x, fmaf(ov[i].y, ov[i].y, fmaf(ov[i].z, ov[i].z, fmaf(ov[i].w, ov[i].w, ss))));
+          }
+          ss += __shfl_xor_sync(0xffffffffu, ss, 1);
+          ss += __shfl_xor_sync(0xffffffffu, ss, 2);
+          const float rstd = rsqrtf(ss * (1.f / kD) + a.post_eps);
+          if (sizeof(TO) == 2) {   // every row read before any bf16 row lands on top of the fp32 tile
+            mbar_arrive(b_pn);
+            MDN_WAIT(b_pn, pn_phase);
+            pn_phase ^= 1;
+          }
+#pragma unroll
+          for (int i = 0; i < kPieces; ++i) {
+            const int col = (part + kTpr * i) * 4;
+            const float4 wv = *reinterpret_cast<const float4*>(w_sm + col);
+            const uint2 gr = graw[i];
+            const float g0 = __uint_as_float(gr.x << 16), g1 = __uint_as_float(gr.x & 0xffff0000u);
+            const float g2 = __uint_as_float(gr.y << 16), g3 = __uint_as_float(gr.y & 0xffff0000u);
+            const float y0 = ov[i].x * rstd * wv.x * sigmoid_fast(g0), y1 = ov[i].y * rstd * wv.y * sigmoid_fast(g1);
+            const float y2 = ov[i].z * rstd * wv.z * sigmoid_fast(g2), y3 = ov[i].w * rstd * wv.w * sigmoid_fast(g3);
+            if (sizeof(TO) == 4) {
+              *reinterpret_cast<float4*>(tile + prow * kD + col) = make_float4(y0, y1, y2, y3);
+            } else {
+              uint2 pk;
+              pk.x = pack_bf16(y0, y1); pk.y = pack_bf16(y2, y3);
+              *reinterpret_cast<uint2*>(stp + kStOut + (prow * kD + col) * 2) = pk;
+            }
+          }
+          fence_proxy_async_smem();
+          mbar_arrive((cp & 1) ? b_go1 : b_go0);
+        }
+      }
       if (c == 0) {
         // ---------------- the start state into the masters
 #pragma unroll 1
@@ -558,6 +679,12 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tf32_kernel(const Args a, c
       const uint32_t ph = c & 1;
       uint8_t* stg = smem + kOffStage + (c & 1) * kStageBytes;
       const __nv_bfloat16* sV = reinterpret_cast<const __nv_bfloat16*>(stg + kStV);
+      if constexpr (kLayer) if (post) {   // the chunk's output-gate rows towards L2: read at the end of the chunk
+        const int t128 = q4 * 32 + lane, prow = r0 + t128 / 4, part = t128 % 4;
+        if (part < 2 && c * C + prow < sq.len)
+          asm volatile("prefetch.global.L2 [%0];" ::"l"(static_cast<const __nv_bfloat16*>(a.post_g) +
+                                                        ((size_t)(sq.tok0 + c * C + prow) * H + h) * kD + 64 * part));
+      }
       MDN_WAIT((c & 1) ? b_full1 : b_full0, (c >> 1) & 1);
       MDN_WAIT((c & 1) ? b_adj1 : b_adj0, (c >> 1) & 1);
       // ---------------- EPI-1: R^T = V^T - cX .* X + cY .* Y  -> bf16 hi, lo in X
@@ -733,15 +860,26 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tf32_kernel(const Args a, c
         tc_fence_before_sync();
         mbar_arrive(b_zu);
         MDN_MARK(c, kEvZuArrive);
+        bool plain_out = true;
+        if constexpr (kLayer) plain_out = !post;
+        if (plain_out) {
 #pragma unroll
-        for (int j = 0; j < kTok; ++j) stage_o<TO>(stg + kStOut, r0 + j, d, __uint_as_float(u[j]));
+          for (int j = 0; j < kTok; ++j) stage_o<TO>(stg + kStOut, r0 + j, d, __uint_as_float(u[j]));
+        } else if constexpr (kLayer) {
+          // fused output step, first half: the fp32 tile (value columns across the lanes; V, T and half of the W area,
+          // all dead by now).  The rest runs at the top of the next iteration, under the next chunk's MMA-1.
+          float* tile = reinterpret_cast<float*>(stg + kStOut);
+#pragma unroll
+          for (int j = 0; j < kTok; ++j) tile[(r0 + j) * kD + d] = __uint_as_float(u[j]);
+          mbar_arrive(b_pn);
+        }
         fence_proxy_async_smem();
         MDN_MARK(c, kEvOutDone);
       }
       // the stage may be refilled once MMA-3, the last reader of its K tile, is done
       MDN_WAIT(b_m3, ph);
       MDN_MARK(c, kEvM3Seen);
-      mbar_arrive((c & 1) ? b_go1 : b_go0);
+      if (!post) mbar_arrive((c & 1) ? b_go1 : b_go0);   // (fused output step: after its second half)
     }
   }
 #undef MDN_WAIT
@@ -789,6 +927,9 @@ cudaError_t launch_chain_tf32(const Plan& pl, const void* q, const void* k, cons
   a.scale = p.scale;
   a.seg_G = 0; a.seg_phase = 0;
   a.seg_E = a.seg_Psi = a.seg_PhiS = a.seg_PhiM = nullptr;
+  a.qk_on = pl.qk.on; a.qk_d = pl.qk.d;
+  a.post_on = pl.post.on; a.post_w = pl.post.w; a.post_g = pl.post.g; a.post_eps = pl.post.eps;
+  const bool layer = a.qk_on || a.post_on;
   a.timeline = nullptr;
 #ifdef MDN_DEBUG   // debug builds only (-DMDN_DEBUG): the product library reads nothing from the environment
   const char* tl = getenv("MDN_DEBUG_TIMELINE");   // device address of an int64 buffer, [chunks][32]
@@ -796,7 +937,8 @@ cudaError_t launch_chain_tf32(const Plan& pl, const void* q, const void* k, cons
 #endif
   const unsigned chains = (unsigned)pl.geom.num_seqs * p.H;
   auto launch = [&](unsigned grid) -> cudaError_t {
-    auto kern = o_bf16 ? chain_tf32_kernel<__nv_bfloat16> : chain_tf32_kernel<float>;
+    auto kern = layer ? (o_bf16 ? chain_tf32_kernel<__nv_bfloat16, true> : chain_tf32_kernel<float, true>)
+                      : (o_bf16 ? chain_tf32_kernel<__nv_bfloat16, false> : chain_tf32_kernel<float, false>);
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
     if (e != cudaSuccess) return e;
     e = launch_pdl(kern, dim3(grid), dim3(kThreads), kSmemBytes, pl.stream, a, mq, mk, mv, mt, mw, mo);

@@ -566,10 +566,10 @@ cudaError_t launch_intra_mma(const Plan& pl, const void* q, const void* k, const
   if (!encode_tma_2d_bf16(&mq, TmaMap2D{q, row, tokens, row * 2, 64, 64, true}) ||
       !encode_tma_2d_bf16(&mk, TmaMap2D{k, row, tokens, row * 2, 64, 64, true}))
     return cudaErrorInvalidValue;
-  if (pl.qk.on && pl.w_f32) return cudaErrorInvalidValue;   // the fp32 W serves the plain forward only
-  cudaError_t e = pl.qk.on ? launch_intra_variant<true, false>(pl, mq, mk, gates, n_mats)
-                  : pl.w_f32 ? launch_intra_variant<false, true>(pl, mq, mk, gates, n_mats)
-                             : launch_intra_variant<false, false>(pl, mq, mk, gates, n_mats);
+  cudaError_t e = pl.qk.on ? (pl.w_f32 ? launch_intra_variant<true, true>(pl, mq, mk, gates, n_mats)
+                                       : launch_intra_variant<true, false>(pl, mq, mk, gates, n_mats))
+                           : (pl.w_f32 ? launch_intra_variant<false, true>(pl, mq, mk, gates, n_mats)
+                                       : launch_intra_variant<false, false>(pl, mq, mk, gates, n_mats));
   if (e == cudaSuccess) e = cudaGetLastError();
   if (e == cudaSuccess) ++*launches;
   return e;
