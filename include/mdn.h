@@ -229,10 +229,10 @@ mdn_status mdn_chunk_fwd_static_scratch(const mdn_params* p,
  *    1 is what 0 is measured against; the fp32 SIMT path always runs qk_norm and out_norm_gate as passes of
  *    their own, whatever the value.
  *
- * Inside the kernels (tensor path): the gate formulas run inside the coefficient scan; the norms of k and q - d k come
- * from the diagonals of the K K^T and Q K^T tiles the intra-chunk kernel computes anyway and are applied to
- * fp32 accumulators (q and k are never rewritten or re-rounded); the output step runs in the chain kernel's
- * output epilogue.  All pointers are device pointers; the struct itself is host memory, read during the call.
+ * Inside the kernels (tensor path): the gate formulas run inside the coefficient scan; the norms of k and q - d k are
+ * summed from the K and Q tiles the intra-chunk kernel holds anyway and ride on per-token coefficients that scale
+ * fp32 accumulators; q - d k is formed in fp32 where the chain kernel makes its fp32 copy of the Q tile (q and k are
+ * never rewritten or re-rounded in memory); the output step runs in the chain kernel's output epilogue.  All pointers are device pointers; the struct itself is host memory, read during the call.
  */
 typedef struct mdn_layer_ops_s {
   int32_t raw_gates;
