@@ -14,10 +14,12 @@
 //                                      T_21 = -T_22 A_21 T_11 at block sizes 16 and 32 with tf32 tensor-core MMAs
 //                                      (Eq. 15; the paper substitutes row by row over all 64 rows).  T leaves as bf16,
 //                                      so tf32 (10-bit mantissa) block products cost nothing visible.
-// With the fused q/k norm a W thread also needs its row of K K^T: the K tile is loaded a second time behind the Q
-// tile, and a second product with A = Q stacked on that copy puts K K^T into lanes 64..127 of 64 more columns.
+// With the fused q/k norm a W thread also needs its row of K K^T ((q - d k) . k_i = Q K^T - d K K^T), which the product
+// leaves in another warp's lanes: the A thread of that row passes it through the row's slot of the W staging area
+// (one block barrier; a first version loaded the K tile a second time and ran a second product: 52 KB, 128 columns,
+// four CTAs per SM).
 // One 128-thread CTA per (chunk, head); 36 KB of shared memory (the operand tiles, reused for the W staging, A and
-// T; 52 KB with the fused q/k norm) and 64 (128) columns of tensor memory.  Tensor memory is released before the CTA signals its dependents, so the chain kernel
+// T) and 64 columns of tensor memory.  Tensor memory is released before the CTA signals its dependents, so the chain kernel
 // (which takes all 512 columns of an SM) can never be resident beside a CTA of this kernel that still has to allocate.
 #include <cstring>
 #include <type_traits>
@@ -37,8 +39,7 @@ constexpr int kD = 128;
 constexpr int LM = C + 4;     // fp32 elements per row of T (16-byte aligned rows)
 
 // operand tiles, bf16, [64 rows x 128 B] swizzled blocks: K (dk 0..63) | Q (dk 0..63) | K (dk 64..127) | Q (..)
-// so that rows 0..127 of each 16 KB half are K stacked on Q; with the fused q/k norm each half has a third block,
-// K again, so that rows 64..191 are Q stacked on K
+// so that rows 0..127 of each 16 KB half are K stacked on Q
 struct Lay {
   uint32_t k1, cv, tiles, smem;   // offset of the second half, of the vectors; tile bytes; dynamic shared memory
 };
@@ -57,7 +58,7 @@ constexpr uint32_t kOffB32 = kOffB10 + 16 * LB * 4;          // A[48:64, 32:48]
 constexpr uint32_t kOffAd = kOffB32 + 16 * LB * 4;           // the four diagonal blocks; dead after step 1:
 constexpr uint32_t kOffP = kOffAd;                           // product scratch, 2 x [16][LB] in step 2, [32][LA] in step 3
 __host__ __device__ constexpr Lay lay_of(bool qk) {
-  const uint32_t half = qk ? 24576u : 16384u;
+  const uint32_t half = 16384u; (void)qk;
   return Lay{half, 2 * half, 2 * half, 2 * half + kCvVecs * C * 4 + 1024};   // + slack for the 1024-byte alignment
 }
 static_assert(kOffAd + 4 * LD16 * 4 <= 32768 && 32 * LA * 4 <= 4 * LD16 * 4, "reuse of the tile area");
@@ -117,30 +118,17 @@ __device__ __forceinline__ void load16(uint32_t taddr, float (&x)[16], bool ok) 
 #pragma unroll
   for (int j = 0; j < 16; ++j) x[j] = __uint_as_float(u[j]);
 }
-// two such groups with one wait
-__device__ __forceinline__ void load16x2(uint32_t ta, float (&x)[16], uint32_t tb, float (&y)[16], bool ok) {
-  uint32_t u[16], w[16];
-#pragma unroll
-  for (int j = 0; j < 16; ++j) u[j] = w[j] = 0u;
-  if (ok) {
-    tmem_ld16(ta, u);
-    tmem_ld16(tb, w);
-    tmem_wait_ld();
-  }
-#pragma unroll
-  for (int j = 0; j < 16; ++j) { x[j] = __uint_as_float(u[j]); y[j] = __uint_as_float(w[j]); }
-}
-
 // kWf32: W leaves as one fp32 matrix (what the kind::tf32 output product of chain_tf32.cu reads) instead of the bf16
 // hi + lo pair; same bytes, same staging area.
 template <bool kQk, bool kWf32>
-__global__ void __launch_bounds__(kThreads, kQk ? 4 : kCtasPerSm) intra_mma_kernel(ChunkGeom g, const __grid_constant__ CUtensorMap map_q,
+__global__ void __launch_bounds__(kThreads, kCtasPerSm) intra_mma_kernel(ChunkGeom g, const __grid_constant__ CUtensorMap map_q,
                                                             const __grid_constant__ CUtensorMap map_k,
                                                             float* __restrict__ coef, GateArgs gates, GateParam gp,
                                                             QkNorm qkn, float scale,
                                                             __nv_bfloat16* __restrict__ Tout,
                                                             __nv_bfloat16* __restrict__ Wout, size_t w_lo_offset,
                                                             int32_t* __restrict__ status) {
+  static_assert(!kQk || kWf32, "the q/k-norm variant uses the fp32 W staging slots");
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   __shared__ __align__(8) uint64_t bars[2];   // tiles landed; product done
@@ -152,7 +140,7 @@ __global__ void __launch_bounds__(kThreads, kQk ? 4 : kCtasPerSm) intra_mma_kern
   if (si.seq < 0) return;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   constexpr Lay L = lay_of(kQk);
-  constexpr uint32_t kOffK1 = L.k1, kOffQ1 = L.k1 + 8192, kOffCv = L.cv, kTmemCols = kQk ? 128 : 64;
+  constexpr uint32_t kOffK1 = L.k1, kOffQ1 = L.k1 + 8192, kOffCv = L.cv, kTmemCols = 64;
   const int fg = lane >> 2, ft = lane & 3;   // MMA fragment coordinates of the tf32 block products
   float* Tf = reinterpret_cast<float*>(smem + kOffT);
   float* cv = reinterpret_cast<float*>(smem + kOffCv);
@@ -175,10 +163,6 @@ __global__ void __launch_bounds__(kThreads, kQk ? 4 : kCtasPerSm) intra_mma_kern
       tma_load_2d(s_base + kOffK1, &map_k, h * kD + 64, si.tok0, bar_t);
       tma_load_2d(s_base + kOffQ0, &map_q, h * kD, si.tok0, bar_t);
       tma_load_2d(s_base + kOffQ1, &map_q, h * kD + 64, si.tok0, bar_t);
-      if constexpr (kQk) {
-        tma_load_2d(s_base + kOffQ0 + 8192, &map_k, h * kD, si.tok0, bar_t);
-        tma_load_2d(s_base + kOffQ1 + 8192, &map_k, h * kD + 64, si.tok0, bar_t);
-      }
     }
     __syncwarp();
     tmem_alloc(smem_u32(&tmem_slot), kTmemCols);
@@ -244,13 +228,6 @@ __global__ void __launch_bounds__(kThreads, kQk ? 4 : kCtasPerSm) intra_mma_kern
       for (int k = 0; k < 8; ++k) {
         const uint64_t d = ((k >> 2) ? d1 : d0) + 2 * (k & 3);   // A: 128 rows from here (K, then Q); B: the first 64 (K)
         umma_ss(tmem, d, d, idesc, k > 0);
-      }
-      if constexpr (kQk) {   // A: the 128 rows from the Q block on (Q, then K again): K K^T lands in lanes 64..127
-#pragma unroll
-        for (int k = 0; k < 8; ++k) {
-          const uint64_t d = ((k >> 2) ? d1 : d0) + 2 * (k & 3);
-          umma_ss(tmem + 64, d + (8192 >> 4), d, idesc, k > 0);
-        }
       }
       umma_commit(bar_p);
     }
@@ -366,6 +343,15 @@ __global__ void __launch_bounds__(kThreads, kQk ? 4 : kCtasPerSm) intra_mma_kern
       if (cb < reach) {
         float x[16];
         load16(trow + cb * 16, x, ok);
+        if constexpr (kQk) {
+          // fused q/k norm: the W thread of row r needs this row of K K^T as well ((q - d k) . k_i = Q K^T - d K K^T): it
+          // goes through row r's slot of the W staging area (the tiles there are dead), which that thread reads below
+          // and then overwrites with its row of W
+#pragma unroll
+          for (int p4 = 0; p4 < 4; ++p4)
+            *reinterpret_cast<float4*>(smem + kOffWh + r * 256 + (((cb * 4 + p4) ^ (r & 7)) * 16)) =
+                make_float4(x[p4 * 4], x[p4 * 4 + 1], x[p4 * 4 + 2], x[p4 * 4 + 3]);
+        }
         if (cb <= rbk) {
           float* dst = (cb == rbk) ? Ad + rbk * LD16 + rl * LB
                                    : (rbk >= 2 && cb < 2) ? A21 + (r - 32) * LA + cb * 16 : (rbk == 1 ? B10 : B32) + rl * LB;
@@ -384,7 +370,9 @@ __global__ void __launch_bounds__(kThreads, kQk ? 4 : kCtasPerSm) intra_mma_kern
         }
       }
     }
-  } else {
+  }
+  if constexpr (kQk) __syncthreads();   // the rows of K K^T are in their slots
+  if (w_thread) {
     uint8_t* w_hi = smem + kOffWh + r * 128;
     uint8_t* w_lo = smem + kOffWl + r * 128;
     uint8_t* w_f32 = smem + kOffWh + r * 256;   // fp32 staging: [64] rows of 256 B, 16-byte pieces XOR-swizzled with (row % 8)
@@ -396,9 +384,14 @@ __global__ void __launch_bounds__(kThreads, kQk ? 4 : kCtasPerSm) intra_mma_kern
                       make_float4(0.f, 0.f, 0.f, 0.f)};
       if (cb < reach) {
         float x[16];
-        if constexpr (kQk) {   // (q_r - d k_r) . k_i / |k_i|; this row of K K^T is in the second product
+        if constexpr (kQk) {   // (q_r - d k_r) . k_i / |k_i|; this row of K K^T waits in the row's staging slot
           float y[16];
-          load16x2(trow + cb * 16, x, trow + 64 + cb * 16, y, ok);
+          load16(trow + cb * 16, x, ok);
+#pragma unroll
+          for (int p4 = 0; p4 < 4; ++p4) {
+            const float4 y4 = *reinterpret_cast<const float4*>(w_f32 + (((cb * 4 + p4) ^ (r & 7)) * 16));
+            y[p4 * 4] = y4.x; y[p4 * 4 + 1] = y4.y; y[p4 * 4 + 2] = y4.z; y[p4 * 4 + 3] = y4.w;
+          }
 #pragma unroll
           for (int j4 = 0; j4 < 16; j4 += 4) {
             const float4 rki = *reinterpret_cast<const float4*>(cv + 6 * C + cb * 16 + j4);
@@ -566,8 +559,10 @@ cudaError_t launch_intra_mma(const Plan& pl, const void* q, const void* k, const
   if (!encode_tma_2d_bf16(&mq, TmaMap2D{q, row, tokens, row * 2, 64, 64, true}) ||
       !encode_tma_2d_bf16(&mk, TmaMap2D{k, row, tokens, row * 2, 64, 64, true}))
     return cudaErrorInvalidValue;
-  cudaError_t e = pl.qk.on ? (pl.w_f32 ? launch_intra_variant<true, true>(pl, mq, mk, gates, n_mats)
-                                       : launch_intra_variant<true, false>(pl, mq, mk, gates, n_mats))
+  // (the q/k-norm variant passes rows of K K^T through the fp32 W staging slots: it exists with the fp32 W only, which is
+  // what every caller that can switch the q/k norm on uses)
+  if (pl.qk.on && !pl.w_f32) return cudaErrorInvalidValue;
+  cudaError_t e = pl.qk.on ? launch_intra_variant<true, true>(pl, mq, mk, gates, n_mats)
                            : (pl.w_f32 ? launch_intra_variant<false, true>(pl, mq, mk, gates, n_mats)
                                        : launch_intra_variant<false, false>(pl, mq, mk, gates, n_mats));
   if (e == cudaSuccess) e = cudaGetLastError();
