@@ -29,6 +29,7 @@ __global__ void __launch_bounds__(1024) chunk_map_kernel(const int32_t* __restri
   __shared__ int s_bad;
   const int tid = threadIdx.x;
   if (tid == 0) { s_carry = 0; s_bad = 0; }
+  if (tid < 4) status[tid] = 0;   // the call's status word starts clean (this is the call's first kernel)
   __syncthreads();
   // T < 0: the total may fall short of -T (the caller pads its problem to a bound)
   if (tid == 0 && (cu[0] != 0 || (T >= 0 ? cu[num_seqs] != T : cu[num_seqs] > -T))) s_bad = 1;
@@ -77,8 +78,18 @@ __global__ void __launch_bounds__(1024) chunk_map_kernel(const int32_t* __restri
   }
 }
 
+// Fixed-length input has no chunk map to build: the call's first kernel only clears the status word.  A kernel rather
+// than a memset node so that the next kernel's launch overlaps it (programmatic dependent launch).
+__global__ void status_clear_kernel(int32_t* __restrict__ status) {
+  grid_dependency_wait();
+  if (threadIdx.x < 4) status[threadIdx.x] = 0;
+}
+
 cudaError_t launch_chunk_map(const Plan& pl, int* launches) {
-  if (pl.geom.cu == nullptr) return cudaSuccess;
+  if (pl.geom.cu == nullptr) {
+    ++*launches;
+    return launch_pdl(status_clear_kernel, dim3(1), dim3(32), 0, pl.stream, reinterpret_cast<int32_t*>(pl.ws + pl.lay.off_status));
+  }
   chunk_map_kernel<<<1, 1024, 0, pl.stream>>>(pl.geom.cu, pl.geom.num_seqs, pl.cu_total_may_be_short ? -pl.p.T : pl.p.T,
                                               pl.geom.num_slots,
                                               const_cast<int32_t*>(pl.geom.chunk_off),

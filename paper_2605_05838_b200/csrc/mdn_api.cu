@@ -96,9 +96,7 @@ static mdn_status run_prep_and_scan(const Plan& pl, const float* beta, const flo
   if (!beta || !log_alpha || !log_mu) return MDN_ERR_INVALID_ARG;
   if (!aligned(beta, 4) || !aligned(log_alpha, 4) || !aligned(log_mu, 4) || (eta && !aligned(eta, 4)))
     return MDN_ERR_INVALID_ARG;
-  if (cudaMemsetAsync(pl.ws + pl.lay.off_status, 0, 4 * sizeof(int32_t), pl.stream) != cudaSuccess)
-    return MDN_ERR_CUDA;
-  if (launch_chunk_map(pl, launches) != cudaSuccess) return MDN_ERR_CUDA;
+  if (launch_chunk_map(pl, launches) != cudaSuccess) return MDN_ERR_CUDA;   // (also clears the status word)
   if (with_scan && launch_coeff_scan(pl, beta, log_alpha, log_mu, eta, launches) != cudaSuccess) return MDN_ERR_CUDA;
   return MDN_OK;
 }

@@ -182,7 +182,7 @@ def test_tensor_path_fused_with_parallel_scan_and_determinism(mdn):
     inp = wl.make_layer_inputs(w)
     ref = oracle_layer(inp, ALL)
     got = run_fused(mdn, inp, ALL, path="tensor", o_dtype=torch.float32, segments=4)
-    assert mdn.last_launch_count() == 4       # intra-chunk, segment runs, combine, real runs
+    assert mdn.last_launch_count() == 5       # status clear, intra-chunk, segment runs, combine, real runs
     errs = errs3(got, ref)
     print("fused, 4 segments: o %.3e S %.3e M %.3e" % tuple(errs))
     assert max(errs) <= TOL_BF16
