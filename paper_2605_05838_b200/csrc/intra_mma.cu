@@ -364,7 +364,9 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) intra_mma_kernel(ChunkGe
                   make_float4(rn_r * f[i] * rki.x * x[j4], rn_r * f[i + 1] * rki.y * x[j4 + 1], rn_r * f[i + 2] * rki.z * x[j4 + 2],
                               rn_r * f[i + 3] * rki.w * x[j4 + 3]);
             } else {
-              *reinterpret_cast<float4*>(dst + j4) = make_float4(f[i] * x[j4], f[i + 1] * x[j4 + 1], f[i + 2] * x[j4 + 2], f[i + 3] * x[j4 + 3]);
+              const float2 p0 = __fmul2_rn(make_float2(f[i], f[i + 1]), make_float2(x[j4], x[j4 + 1]));
+              const float2 p1 = __fmul2_rn(make_float2(f[i + 2], f[i + 3]), make_float2(x[j4 + 2], x[j4 + 3]));
+              *reinterpret_cast<float4*>(dst + j4) = make_float4(p0.x, p0.y, p1.x, p1.y);
             }
           }
         }
@@ -402,8 +404,16 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) intra_mma_kernel(ChunkGe
           load16(trow + cb * 16, x, ok);
         }
         float w[16];
+        if constexpr (kQk) {
 #pragma unroll
-        for (int j = 0; j < 16; ++j) w[j] = kQk ? rn_r * f[cb * 16 + j] * x[j] : f[cb * 16 + j] * x[j];
+          for (int j = 0; j < 16; ++j) w[j] = rn_r * f[cb * 16 + j] * x[j];
+        } else {
+#pragma unroll
+          for (int j = 0; j < 16; j += 2) {
+            const float2 p = __fmul2_rn(make_float2(f[cb * 16 + j], f[cb * 16 + j + 1]), make_float2(x[j], x[j + 1]));
+            w[j] = p.x; w[j + 1] = p.y;
+          }
+        }
         if constexpr (kWf32) {
 #pragma unroll
           for (int p4 = 0; p4 < 4; ++p4) wf[p4] = make_float4(w[p4 * 4], w[p4 * 4 + 1], w[p4 * 4 + 2], w[p4 * 4 + 3]);
