@@ -68,11 +68,10 @@ __device__ __forceinline__ float4 lds_f4(uint32_t addr) {
   asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
   return v;
 }
-__device__ __forceinline__ uint32_t to_tf32(float x) {
-  uint32_t r;
-  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
-  return r;
-}
+// fp32 bits as a tf32 operand: the tensor core ignores the low 13 mantissa bits (truncation instead of rounding to
+// nearest).  T leaves as bf16 (8 mantissa bits), so the conversion instruction per fragment element bought nothing
+// visible and cost 320 warp-instructions per chunk-head.
+__device__ __forceinline__ uint32_t to_tf32(float x) { return __float_as_uint(x); }
 __device__ __forceinline__ void mma_tf32(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
   asm volatile(
       "mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
