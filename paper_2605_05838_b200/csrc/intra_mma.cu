@@ -89,13 +89,18 @@ __device__ __forceinline__ uint32_t q_tile_chunk(uint32_t half_bytes, uint32_t r
 // a: &A[row0][k0], b: &B[k0][col0].  Fragment coordinates: g = lane / 4, t = lane % 4.
 template <int KS, int NT, int LDA, int LDB>
 __device__ __forceinline__ void block_mma_tf32(float (&acc)[NT][4], const float* a, const float* b, int g, int t) {
+  static_assert((LDA * 4) % 16 == 0, "ldmatrix rows are 16-byte pieces");
+  // The 16 x 8 fp32 A fragment of one k-step in ONE instruction: ldmatrix moves 8 x 8 tiles of 16-bit elements, i.e.
+  // 8 rows of 16 bytes = 8 x 4 fp32, and hands thread (g, t) the 32 bits at row g, piece t - exactly the tf32
+  // fragment layout.  Lane l supplies the row address of tile l / 8: rows 0..7 / 8..15 at columns 0..3, then 4..7.
+  const int lane = g * 4 + t;
+  const uint32_t a_lane = smem_u32(a + ((lane & 7) + 8 * ((lane >> 3) & 1)) * LDA + 4 * (lane >> 4));
 #pragma unroll
   for (int ks = 0; ks < KS; ++ks) {
     uint32_t af[4];
-    af[0] = to_tf32(a[g * LDA + ks * 8 + t]);
-    af[1] = to_tf32(a[(g + 8) * LDA + ks * 8 + t]);
-    af[2] = to_tf32(a[g * LDA + ks * 8 + t + 4]);
-    af[3] = to_tf32(a[(g + 8) * LDA + ks * 8 + t + 4]);
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(af[0]), "=r"(af[1]), "=r"(af[2]), "=r"(af[3])
+                 : "r"(a_lane + ks * 32));
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
       const uint32_t b0 = to_tf32(b[(ks * 8 + t) * LDB + nt * 8 + g]);
