@@ -68,10 +68,20 @@ __device__ __forceinline__ float4 lds_f4(uint32_t addr) {
   asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
   return v;
 }
-// fp32 bits as a tf32 operand: the tensor core ignores the low 13 mantissa bits (truncation instead of rounding to
-// nearest).  T leaves as bf16 (8 mantissa bits), so the conversion instruction per fragment element bought nothing
-// visible and cost 320 warp-instructions per chunk-head.
+// Operands of the tf32 block products.  Their fragments are loaded as plain fp32 bits (a conversion per fragment
+// element cost 320 warp instructions per chunk-head); what the products themselves produce and consume again - the
+// inverted diagonal blocks, the intermediate products, the lower blocks of T - is rounded to tf32 (to nearest) once,
+// where it is written to shared memory; only the blocks of A, written by the row pass, stay unrounded (the tensor
+// core truncates them).  Measured where T is far from I (correlated keys), max error of o / RMS: everything
+// truncated 1.9e-2, this 1.2e-2, a conversion per fragment element 1.2e-2; the A blocks rounded at their write as
+// well was the slowest of all.
 __device__ __forceinline__ uint32_t to_tf32(float x) { return __float_as_uint(x); }
+__device__ __forceinline__ float rnd_tf32(float x) {
+  uint32_t r;
+  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
+  return __uint_as_float(r);
+}
+__device__ __forceinline__ float2 rnd_tf32(float a, float b) { return make_float2(rnd_tf32(a), rnd_tf32(b)); }
 __device__ __forceinline__ void mma_tf32(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
   asm volatile(
       "mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
@@ -362,16 +372,17 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) intra_mma_kernel(ChunkGe
 #pragma unroll
           for (int j4 = 0; j4 < 16; j4 += 4) {
             const int i = cb * 16 + j4;
+            float4 av;
             if constexpr (kQk) {
               const float4 rki = *reinterpret_cast<const float4*>(cv + 6 * C + i);
-              *reinterpret_cast<float4*>(dst + j4) =
-                  make_float4(rn_r * f[i] * rki.x * x[j4], rn_r * f[i + 1] * rki.y * x[j4 + 1], rn_r * f[i + 2] * rki.z * x[j4 + 2],
-                              rn_r * f[i + 3] * rki.w * x[j4 + 3]);
+              av = make_float4(rn_r * f[i] * rki.x * x[j4], rn_r * f[i + 1] * rki.y * x[j4 + 1], rn_r * f[i + 2] * rki.z * x[j4 + 2],
+                               rn_r * f[i + 3] * rki.w * x[j4 + 3]);
             } else {
               const float2 p0 = __fmul2_rn(make_float2(f[i], f[i + 1]), make_float2(x[j4], x[j4 + 1]));
               const float2 p1 = __fmul2_rn(make_float2(f[i + 2], f[i + 3]), make_float2(x[j4 + 2], x[j4 + 3]));
-              *reinterpret_cast<float4*>(dst + j4) = make_float4(p0.x, p0.y, p1.x, p1.y);
+              av = make_float4(p0.x, p0.y, p1.x, p1.y);
             }
+            *reinterpret_cast<float4*>(dst + j4) = av;
           }
         }
       }
@@ -486,7 +497,7 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) intra_mma_kernel(ChunkGe
       x[rr] = acc;
     }
 #pragma unroll
-    for (int rr = 0; rr < 16; ++rr) Tf[(b0 + rr) * LM + b0 + j] = x[rr];
+    for (int rr = 0; rr < 16; ++rr) Tf[(b0 + rr) * LM + b0 + j] = rnd_tf32(x[rr]);   // (an operand of steps 2, 3)
     if (((tid >> 4) & 1) == 0) {   // the zero block right of D_0 (D_2): step 3 reads T_11 and T_22 as full 32x32 blocks
 #pragma unroll
       for (int rr = 0; rr < 16; ++rr) Tf[(b0 + rr) * LM + b0 + 16 + j] = 0.f;
@@ -502,16 +513,16 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) intra_mma_kernel(ChunkGe
     float* P = Pf + warp * 16 * LB;
 #pragma unroll
     for (int nt = 0; nt < 2; ++nt) {
-      *reinterpret_cast<float2*>(P + fg * LB + nt * 8 + 2 * ft) = make_float2(acc[nt][0], acc[nt][1]);
-      *reinterpret_cast<float2*>(P + (fg + 8) * LB + nt * 8 + 2 * ft) = make_float2(acc[nt][2], acc[nt][3]);
+      *reinterpret_cast<float2*>(P + fg * LB + nt * 8 + 2 * ft) = rnd_tf32(acc[nt][0], acc[nt][1]);
+      *reinterpret_cast<float2*>(P + (fg + 8) * LB + nt * 8 + 2 * ft) = rnd_tf32(acc[nt][2], acc[nt][3]);
     }
     __syncwarp();
     float acc2[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
     block_mma_tf32<2, 2, LM, LB>(acc2, Tf + R0 * LM + R0, P, fg, ft);
 #pragma unroll
     for (int nt = 0; nt < 2; ++nt) {
-      *reinterpret_cast<float2*>(Tf + (R0 + fg) * LM + C0 + nt * 8 + 2 * ft) = make_float2(-acc2[nt][0], -acc2[nt][1]);
-      *reinterpret_cast<float2*>(Tf + (R0 + fg + 8) * LM + C0 + nt * 8 + 2 * ft) = make_float2(-acc2[nt][2], -acc2[nt][3]);
+      *reinterpret_cast<float2*>(Tf + (R0 + fg) * LM + C0 + nt * 8 + 2 * ft) = rnd_tf32(-acc2[nt][0], -acc2[nt][1]);
+      *reinterpret_cast<float2*>(Tf + (R0 + fg + 8) * LM + C0 + nt * 8 + 2 * ft) = rnd_tf32(-acc2[nt][2], -acc2[nt][3]);
     }
   }
   __syncthreads();
@@ -522,8 +533,8 @@ __global__ void __launch_bounds__(kThreads, kCtasPerSm) intra_mma_kernel(ChunkGe
     block_mma_tf32<4, 2, LA, LM>(acc, A21 + 16 * mt * LA, Tf + n0, fg, ft);
 #pragma unroll
     for (int nt = 0; nt < 2; ++nt) {
-      *reinterpret_cast<float2*>(Pf + (16 * mt + fg) * LA + n0 + nt * 8 + 2 * ft) = make_float2(acc[nt][0], acc[nt][1]);
-      *reinterpret_cast<float2*>(Pf + (16 * mt + fg + 8) * LA + n0 + nt * 8 + 2 * ft) = make_float2(acc[nt][2], acc[nt][3]);
+      *reinterpret_cast<float2*>(Pf + (16 * mt + fg) * LA + n0 + nt * 8 + 2 * ft) = rnd_tf32(acc[nt][0], acc[nt][1]);
+      *reinterpret_cast<float2*>(Pf + (16 * mt + fg + 8) * LA + n0 + nt * 8 + 2 * ft) = rnd_tf32(acc[nt][2], acc[nt][3]);
     }
     __syncthreads();
     float acc2[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
