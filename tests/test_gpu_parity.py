@@ -264,6 +264,16 @@ def test_fast_forgetting_preset_and_correlated_keys(mdn):
         compare(mdn, inpb, path, label="preset F bf16, correlated keys")
 
 
+def test_slow_forgetting_gates_and_correlated_keys(mdn):
+    """The named configurations' gate preset (long memory) with strongly correlated keys: the triangular system is far
+    from the identity AND its error is carried for hundreds of tokens - where the tensor path's error margin is
+    thinnest (bf16 T; the inversion's tf32 block products)."""
+    wb = wl.Workload("slow_corr", B=1, T=806, H=3, dk=128, dv=128, dtype="bf16", seed=1020)
+    inpb = wl.make_inputs(wb)
+    inpb["k"] = wl.correlated_keys(wb, 0.8)
+    compare(mdn, inpb, "tensor", label="preset S bf16, correlated keys")
+
+
 def test_degenerate_gates(mdn):
     """beta = 0 and mu = 0 tokens (the paper's log-domain kernels NaN at mu = 0), eta = None, scale = 1."""
     w = small(T=140)
